@@ -1,0 +1,162 @@
+/*
+ * deer.h -- C ABI of the DEER-GRU hot path for NVIDIA B200 (sm_100a).
+ *
+ * DEER evaluates a non-linear recurrence y_t = f(y_{t-1}, x_t) for all t at
+ * once by a Newton-type fixed-point iteration (Sec. 3.1, Eq. 3 with Eq. 5);
+ * each iteration evaluates the cell f and its n x n state Jacobian at every
+ * position of the current guess, forms the right-hand side and solves the
+ * linear recurrence y_t = J_t y_{t-1} + b_t with an associative scan
+ * (Sec. 3.3-3.4, Eq. 9-10).  The cell here is a GRU (Sec. 4.1).
+ *
+ * General rules for every entry point
+ *   - All array arguments are DEVICE pointers owned by the caller, fp32,
+ *     dense row-major with the shapes stated, unless marked "host".
+ *   - The library never allocates or frees device memory: scratch comes from
+ *     the caller-supplied workspace `ws` of at least deer_workspace_bytes()
+ *     bytes, 256-byte aligned.  The workspace contents are undefined on entry
+ *     and on return; two calls that overlap in time need distinct workspaces.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Work is enqueued on it; deer_gru_eval synchronises the stream
+ *     before it returns because it writes host outputs, the others do not
+ *     unless stated.
+ *   - Return value: a deer_status.  >= 0 are outcomes of a run that executed,
+ *     < 0 mean nothing (or nothing useful) was computed.  Nothing aborts,
+ *     throws or traps.  Every device-side wait is bounded and reports
+ *     DEER_ERR_DEVICE_TIMEOUT instead of hanging.
+ *   - Batch index b, position t, 0-based.  y[b][-1] = y0[b].
+ *   - Supported hidden sizes: 1 <= n <= 64 (tuned kernels for n in
+ *     {1, 2, 4, 8, 16, 32, 64}, a generic kernel for the rest); 1 <= m <= 1024.
+ */
+#ifndef DEER_H_
+#define DEER_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum deer_status {
+    DEER_OK = 0,
+    DEER_NOT_CONVERGED = 1,        /* max_iter bodies ran, err still > tol; y = last iterate */
+    DEER_NONFINITE = 2,            /* NaN/Inf appeared in the iterate; y = last iterate */
+    DEER_ERR_INVALID_ARG = -1,     /* NULL pointer, non-positive size, NaN tol, max_iter < 1 ... */
+    DEER_ERR_UNSUPPORTED_N = -2,   /* n or m outside the supported range */
+    DEER_ERR_WORKSPACE = -3,       /* ws NULL, misaligned or smaller than deer_workspace_bytes() */
+    DEER_ERR_CUDA = -4,            /* a CUDA runtime call failed; see deer_last_error() */
+    DEER_ERR_DEVICE_TIMEOUT = -5   /* a bounded device-side wait expired; outputs are invalid */
+} deer_status;
+
+/* GRU parameters (Sec. 4.1 uses a standard GRU; the paper prints no
+ * equations, the cell evaluated is
+ *     r = sigmoid(W_ir x + b_ir + W_hr h + b_hr)
+ *     z = sigmoid(W_iz x + b_iz + W_hz h + b_hz)
+ *     c = tanh   (W_in x + b_in + r * (W_hn h + b_hn))
+ *     f(h, x) = (1 - z) * c + z * h ).
+ * Packed along the leading axis in gate order (r, z, n). */
+typedef struct deer_gru_params {
+    int n;              /* hidden size */
+    int m;              /* input size  */
+    const float *W_i;   /* [3n, m] */
+    const float *W_h;   /* [3n, n] */
+    const float *b_i;   /* [3n]    */
+    const float *b_h;   /* [3n]    */
+} deer_gru_params;
+
+/* Parameter gradients, same shapes as the parameters; overwritten. */
+typedef struct deer_gru_grads {
+    float *dW_i, *dW_h, *db_i, *db_h;
+} deer_gru_grads;
+
+/* Operations for deer_workspace_bytes(). */
+enum { DEER_OP_EVAL = 0, DEER_OP_SCAN = 1, DEER_OP_VJP = 2, DEER_OP_CLASSIFIER = 3 };
+
+/* Flags (bit-or). */
+enum {
+    DEER_FLAG_WARM_START = 1,   /* deer_gru_eval: y holds the initial guess on entry (Sec. 3.1:
+                                   the previous training step's solution may seed the next) */
+    DEER_FLAG_GENERIC    = 2,   /* force the generic (any-n) kernels; for testing */
+    DEER_FLAG_MATERIALIZE = 4   /* deer_gru_eval: write J and b to the workspace and run the
+                                   stand-alone scan on them, instead of the fused iteration */
+};
+
+/* Bytes of workspace needed by `op` at the given sizes (0 if the sizes are
+ * invalid).  m is ignored for DEER_OP_SCAN. */
+size_t deer_workspace_bytes(int op, int B, int T, int n, int m, int flags);
+
+/* Solve the linear recurrence (the operator L_G^{-1} of Eq. 10 with J = -G)
+ * with a chunked associative scan whose combine is
+ * (A2, b2) o (A1, b1) = (A2 A1, A2 b1 + b2)  (Eq. 9):
+ *   reverse == 0 :  y[b][t] = J[b][t] y[b][t-1] + b[b][t],   y[b][-1] = y0[b]
+ *   reverse != 0 :  y[b][t] = b[b][t] + J[b][t+1]^T y[b][t+1],
+ *                   y[b][T-1] = b[b][T-1] + y0[b]
+ *     (the adjoint of the forward solve with respect to b -- the "dual
+ *      operator" of Sec. 3.1.1; J[b][0] is not read).
+ *   J  [B,T,n,n]  row = output component        b  [B,T,n]
+ *   y0 [B,n] or NULL (= zeros)                  y  [B,T,n] out (must not alias J or b)
+ * Asynchronous on `stream`.  Returns DEER_OK or a negative status. */
+int deer_linrec_scan(const float *J, const float *b, const float *y0, int B, int T, int n,
+                     int reverse, float *y, void *ws, size_t ws_bytes, int flags, void *stream);
+
+/* Evaluate the GRU over whole sequences with the DEER iteration (Eq. 3 with
+ * G = -df/dy, Eq. 5; loop of App. B.1): starting from y = 0 (or the guess in
+ * y when DEER_FLAG_WARM_START), repeat { J, f at the shifted guess;
+ * rhs = f - J y_prev; y_new = scan(J, rhs, y0); err = max |y_new - y| } while
+ * err > tol and fewer than max_iter bodies have run (err starts at 1e10).
+ * One global err over the whole batch.
+ *   x [B,T,m]   y0 [B,n]   y [B,T,n] out (in: guess if warm start)
+ *   tol        : paper default 1e-4 for fp32; a negative tol runs exactly
+ *                max_iter bodies; NaN is invalid
+ *   iters      : host out, number of executed bodies (may be NULL)
+ *   err        : host out, last max |y_new - y|       (may be NULL)
+ *   err_trace  : host out [max_iter], err after each body, rest untouched (may be NULL)
+ * Synchronises `stream`.  Returns DEER_OK, DEER_NOT_CONVERGED, DEER_NONFINITE
+ * or a negative status. */
+int deer_gru_eval(const deer_gru_params *params, const float *x, const float *y0, int B, int T,
+                  float tol, int max_iter, float *y, int *iters, float *err, float *err_trace,
+                  void *ws, size_t ws_bytes, int flags, void *stream);
+
+/* Gradient through the evaluated sequence (Eq. 7): given gy = dL/dy at a
+ * trajectory y, lambda = gy L_G^{-1} by ONE reverse scan with the Jacobians
+ * recomputed at y (Sec. 3.1.1 allows saving or recomputing them), then the
+ * cell's vector-Jacobian product at every position, summed over positions in
+ * a fixed order (bit-reproducible).
+ *   y  [B,T,n] trajectory (normally deer_gru_eval's output)   gy [B,T,n]
+ *   dparams : device arrays, overwritten       dx  [B,T,m] or NULL
+ *   dy0 [B,n] or NULL
+ * Asynchronous on `stream`.  Returns DEER_OK or a negative status. */
+int deer_gru_vjp(const deer_gru_params *params, const float *x, const float *y0, const float *y,
+                 const float *gy, int B, int T, const deer_gru_grads *dparams, float *dx,
+                 float *dy0, void *ws, size_t ws_bytes, int flags, void *stream);
+
+/* One training step of the long-series classifier (App. B.2 shapes: mean
+ * over the sequence, then a linear decoder and cross-entropy): two stacked
+ * GRU layers of equal hidden size n (layer 1 reads x [B,T,m], layer 2 reads
+ * layer 1's states), zero initial states, p = mean_t y2, logits = W_o p + b_o,
+ * loss = mean over the batch of softmax cross-entropy; forward by
+ * deer_gru_eval per layer, backward by deer_gru_vjp per layer.
+ *   W_o [n_classes, n]  b_o [n_classes]  labels [B] int32 (device)
+ *   loss : host out      iters : host out [2] (may be NULL)
+ *   g1, g2 : parameter gradients per layer;  dW_o [n_classes,n], db_o [n_classes] device out
+ * Synchronises `stream`.  Returns the worst status of the two evaluations. */
+int deer_gru_classifier_step(const deer_gru_params *layer1, const deer_gru_params *layer2,
+                             const float *W_o, const float *b_o, int n_classes, const float *x,
+                             const int *labels, int B, int T, float tol, int max_iter,
+                             float *loss, int *iters, const deer_gru_grads *g1,
+                             const deer_gru_grads *g2, float *dW_o, float *db_o, void *ws,
+                             size_t ws_bytes, int flags, void *stream);
+
+/* Text for a status code (static storage). */
+const char *deer_status_string(int status);
+
+/* Message of the last CUDA error seen by the calling thread ("" if none). */
+const char *deer_last_error(void);
+
+/* Number of kernels this library has launched since it was loaded (all
+ * threads); take differences around a region to count its launches. */
+long long deer_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEER_H_ */

@@ -1,0 +1,249 @@
+"""Thin ctypes binding over the C ABI of ``libdeer_b200.so`` (see include/deer.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  PyTorch supplies device memory and streams.  Loading fails loudly
+if the CUDA library has not been built; there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdeer_b200.so")
+
+DEER_OK, DEER_NOT_CONVERGED, DEER_NONFINITE = 0, 1, 2
+DEER_ERR_INVALID_ARG, DEER_ERR_UNSUPPORTED_N, DEER_ERR_WORKSPACE = -1, -2, -3
+DEER_ERR_CUDA, DEER_ERR_DEVICE_TIMEOUT = -4, -5
+DEER_OP_EVAL, DEER_OP_SCAN, DEER_OP_VJP, DEER_OP_CLASSIFIER = 0, 1, 2, 3
+DEER_FLAG_WARM_START, DEER_FLAG_GENERIC, DEER_FLAG_MATERIALIZE = 1, 2, 4
+
+EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_gru_eval", "deer_gru_vjp",
+           "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count"]
+
+
+class _Params(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int), ("m", ctypes.c_int), ("W_i", ctypes.c_void_p),
+                ("W_h", ctypes.c_void_p), ("b_i", ctypes.c_void_p), ("b_h", ctypes.c_void_p)]
+
+
+class _Grads(ctypes.Structure):
+    _fields_ = [("dW_i", ctypes.c_void_p), ("dW_h", ctypes.c_void_p), ("db_i", ctypes.c_void_p),
+                ("db_h", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """Load the CUDA library; raise if it is missing (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               "`python -m paper_2309_12252_b200.build` (needs nvcc, sm_100a)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.deer_workspace_bytes.restype = ctypes.c_size_t
+        L.deer_workspace_bytes.argtypes = [ctypes.c_int] * 6
+        vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        L.deer_linrec_scan.restype = ci
+        L.deer_linrec_scan.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, ci, vp]
+        L.deer_gru_eval.restype = ci
+        L.deer_gru_eval.argtypes = [ctypes.POINTER(_Params), vp, vp, ci, ci, cf, ci, vp,
+                                    ctypes.POINTER(ci), ctypes.POINTER(cf), vp, vp, sz, ci, vp]
+        L.deer_gru_vjp.restype = ci
+        L.deer_gru_vjp.argtypes = [ctypes.POINTER(_Params), vp, vp, vp, vp, ci, ci,
+                                   ctypes.POINTER(_Grads), vp, vp, vp, sz, ci, vp]
+        L.deer_gru_classifier_step.restype = ci
+        L.deer_gru_classifier_step.argtypes = [ctypes.POINTER(_Params), ctypes.POINTER(_Params), vp, vp,
+                                               ci, vp, vp, ci, ci, cf, ci, ctypes.POINTER(cf),
+                                               ctypes.POINTER(ci), ctypes.POINTER(_Grads),
+                                               ctypes.POINTER(_Grads), vp, vp, vp, sz, ci, vp]
+        L.deer_status_string.restype = ctypes.c_char_p
+        L.deer_status_string.argtypes = [ci]
+        L.deer_last_error.restype = ctypes.c_char_p
+        L.deer_launch_count.restype = ctypes.c_longlong
+        _lib = L
+    return _lib
+
+
+class DeerError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        msg = lib().deer_status_string(status).decode()
+        if status == DEER_ERR_CUDA:
+            msg += ": " + lib().deer_last_error().decode()
+        super().__init__(f"deer status {status}: {msg}")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _f32(t):
+    assert t.dtype == torch.float32
+    return t
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+@dataclass
+class GruParamsDev:
+    """GRU parameters resident on the device (gate order r, z, n)."""
+    n: int
+    m: int
+    W_i: torch.Tensor
+    W_h: torch.Tensor
+    b_i: torch.Tensor
+    b_h: torch.Tensor
+
+    @staticmethod
+    def from_numpy(p, device="cuda"):
+        mk = lambda a: torch.from_numpy(np.ascontiguousarray(a, np.float32)).to(device)
+        return GruParamsDev(p.n, p.m, mk(p.W_i), mk(p.W_h), mk(p.b_i), mk(p.b_h))
+
+    def c_struct(self):
+        for t, shape in ((self.W_i, (3 * self.n, self.m)), (self.W_h, (3 * self.n, self.n)),
+                         (self.b_i, (3 * self.n,)), (self.b_h, (3 * self.n,))):
+            assert tuple(t.shape) == shape and t.dtype == torch.float32 and t.is_cuda and t.is_contiguous()
+        return _Params(self.n, self.m, self.W_i.data_ptr(), self.W_h.data_ptr(), self.b_i.data_ptr(),
+                       self.b_h.data_ptr())
+
+
+def deer_status_string(status: int) -> str:
+    return lib().deer_status_string(int(status)).decode()
+
+
+def deer_launch_count() -> int:
+    return int(lib().deer_launch_count())
+
+
+def deer_workspace_bytes(op: int, B: int, T: int, n: int, m: int = 1, flags: int = 0) -> int:
+    return int(lib().deer_workspace_bytes(op, B, T, n, m, flags))
+
+
+def alloc_workspace(op: int, B: int, T: int, n: int, m: int = 1, flags: int = 0, device="cuda"):
+    nbytes = deer_workspace_bytes(op, B, T, n, m, flags)
+    if nbytes == 0:
+        raise DeerError(DEER_ERR_UNSUPPORTED_N)
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)   # torch allocations are 512-B aligned
+
+
+def deer_linrec_scan(J, b, y0=None, reverse=False, y=None, ws=None, flags=0, stream=None, check=True):
+    """y = scan(J, b, y0); see include/deer.h.  Returns y (asynchronous)."""
+    B, T, n = b.shape
+    assert tuple(J.shape) == (B, T, n, n)
+    if y is None:
+        y = torch.empty_like(b)
+    if ws is None:
+        ws = alloc_workspace(DEER_OP_SCAN, B, T, n, 1, flags, b.device)
+    rc = lib().deer_linrec_scan(_ptr(_f32(J)), _ptr(_f32(b)), _ptr(y0), B, T, n, int(bool(reverse)),
+                                _ptr(y), _ptr(ws), ws.numel(), flags, _stream(stream))
+    if check and rc != DEER_OK:
+        raise DeerError(rc)
+    return y if check else (y, rc)
+
+
+@dataclass
+class EvalResult:
+    y: torch.Tensor
+    iters: int
+    err: float
+    status: int
+    err_trace: np.ndarray
+
+
+def deer_gru_eval(params: GruParamsDev, x, y0, tol=1e-4, max_iter=100, y=None, ws=None, flags=0,
+                  stream=None, check=True) -> EvalResult:
+    """DEER evaluation of the GRU over x [B,T,m]; see include/deer.h."""
+    B, T, m = x.shape
+    n = params.n
+    assert m == params.m and tuple(y0.shape) == (B, n)
+    if y is None:
+        assert not (flags & DEER_FLAG_WARM_START)
+        y = torch.empty((B, T, n), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = alloc_workspace(DEER_OP_EVAL, B, T, n, m, flags, x.device)
+    iters = ctypes.c_int(0)
+    err = ctypes.c_float(0.0)
+    trace = np.full((max(int(max_iter), 1),), np.nan, np.float32)
+    ps = params.c_struct()
+    rc = lib().deer_gru_eval(ctypes.byref(ps), _ptr(_f32(x)), _ptr(_f32(y0)), B, T, float(tol),
+                             int(max_iter), _ptr(y), ctypes.byref(iters), ctypes.byref(err),
+                             trace.ctypes.data_as(ctypes.c_void_p), _ptr(ws), ws.numel(), flags,
+                             _stream(stream))
+    if check and rc < 0:
+        raise DeerError(rc)
+    return EvalResult(y, iters.value, err.value, rc, trace[:iters.value])
+
+
+def deer_gru_eval_host(params: GruParamsDev, x_host, y0_dev, y_host, x_dev, y_dev, ws, tol=1e-4,
+                       max_iter=100, flags=0, stream=None) -> EvalResult:
+    """End-to-end call with HOST buffers: copies x (pinned host) to the device,
+    evaluates, copies y back to pinned host memory."""
+    x_dev.copy_(x_host, non_blocking=True)
+    r = deer_gru_eval(params, x_dev, y0_dev, tol, max_iter, y_dev, ws, flags, stream)
+    y_host.copy_(y_dev, non_blocking=True)
+    torch.cuda.current_stream().synchronize()
+    return r
+
+
+def deer_gru_vjp(params: GruParamsDev, x, y0, y, gy, want_dx=True, want_dy0=True, ws=None, flags=0,
+                 stream=None):
+    """Gradients of L (dL/dy = gy) w.r.t. parameters, x and y0; see include/deer.h."""
+    B, T, m = x.shape
+    n = params.n
+    dev = x.device
+    g = dict(dW_i=torch.empty((3 * n, m), device=dev), dW_h=torch.empty((3 * n, n), device=dev),
+             db_i=torch.empty((3 * n,), device=dev), db_h=torch.empty((3 * n,), device=dev))
+    dx = torch.empty_like(x) if want_dx else None
+    dy0 = torch.empty((B, n), device=dev) if want_dy0 else None
+    if ws is None:
+        ws = alloc_workspace(DEER_OP_VJP, B, T, n, m, flags, dev)
+    ps = params.c_struct()
+    gs = _Grads(g["dW_i"].data_ptr(), g["dW_h"].data_ptr(), g["db_i"].data_ptr(), g["db_h"].data_ptr())
+    rc = lib().deer_gru_vjp(ctypes.byref(ps), _ptr(_f32(x)), _ptr(_f32(y0)), _ptr(_f32(y)), _ptr(_f32(gy)),
+                            B, T, ctypes.byref(gs), _ptr(dx), _ptr(dy0), _ptr(ws), ws.numel(), flags,
+                            _stream(stream))
+    if rc != DEER_OK:
+        raise DeerError(rc)
+    g["dx"], g["dy0"] = dx, dy0
+    return g
+
+
+def deer_gru_classifier_step(layer1: GruParamsDev, layer2: GruParamsDev, W_o, b_o, x, labels, tol=1e-4,
+                             max_iter=100, ws=None, flags=0, stream=None):
+    """Loss and all gradients of the 2-layer GRU classifier; see include/deer.h."""
+    B, T, m = x.shape
+    n = layer1.n
+    ncls = W_o.shape[0]
+    dev = x.device
+    mk = lambda p: dict(dW_i=torch.empty((3 * n, p.m), device=dev), dW_h=torch.empty((3 * n, n), device=dev),
+                        db_i=torch.empty((3 * n,), device=dev), db_h=torch.empty((3 * n,), device=dev))
+    g1, g2 = mk(layer1), mk(layer2)
+    cs = lambda g: _Grads(g["dW_i"].data_ptr(), g["dW_h"].data_ptr(), g["db_i"].data_ptr(), g["db_h"].data_ptr())
+    dW_o = torch.empty_like(W_o); db_o = torch.empty_like(b_o)
+    if ws is None:
+        ws = alloc_workspace(DEER_OP_CLASSIFIER, B, T, n, m, flags, dev)
+    loss = ctypes.c_float(0.0)
+    iters = (ctypes.c_int * 2)()
+    p1, p2 = layer1.c_struct(), layer2.c_struct()
+    s1, s2 = cs(g1), cs(g2)
+    assert labels.dtype == torch.int32
+    rc = lib().deer_gru_classifier_step(ctypes.byref(p1), ctypes.byref(p2), _ptr(_f32(W_o)), _ptr(_f32(b_o)),
+                                        ncls, _ptr(_f32(x)), _ptr(labels), B, T, float(tol), int(max_iter),
+                                        ctypes.byref(loss), iters, ctypes.byref(s1), ctypes.byref(s2),
+                                        _ptr(dW_o), _ptr(db_o), _ptr(ws), ws.numel(), flags, _stream(stream))
+    if rc < 0:
+        raise DeerError(rc)
+    return dict(loss=loss.value, iters=(iters[0], iters[1]), status=rc, g1=g1, g2=g2, dW_o=dW_o, db_o=db_o)

@@ -1,0 +1,82 @@
+// Shared definitions of the DEER-GRU CUDA library (device structs, launch bookkeeping).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <atomic>
+#include "../../include/deer.h"
+
+namespace deer {
+
+extern std::atomic<long long> g_launches;
+void set_error(cudaError_t e, const char *where);
+
+#define DEER_CHECK_LAUNCH(where)                                   \
+    do {                                                           \
+        ::deer::g_launches.fetch_add(1);                           \
+        cudaError_t e_ = cudaGetLastError();                       \
+        if (e_ != cudaSuccess) {                                   \
+            ::deer::set_error(e_, where);                          \
+            return DEER_ERR_CUDA;                                  \
+        }                                                          \
+    } while (0)
+
+#define DEER_CHECK_CUDA(call, where)                               \
+    do {                                                           \
+        cudaError_t e_ = (call);                                   \
+        if (e_ != cudaSuccess) {                                   \
+            ::deer::set_error(e_, where);                          \
+            return DEER_ERR_CUDA;                                  \
+        }                                                          \
+    } while (0)
+
+// Device-resident status of one evaluation (first 256 bytes of the workspace).
+struct StatusBlock {
+    unsigned err_bits;   // max |y_new - y| of the running body, as the bits of a non-negative float
+    unsigned flags;      // FLAG_* bits raised by kernels
+    int iters;           // bodies executed so far (device-side loop control)
+    int done;            // 1 once the loop condition failed
+    unsigned tile_counter;  // dynamic tile id for the single-pass scan
+    unsigned pad[59];
+};
+static_assert(sizeof(StatusBlock) == 256, "status block is one 256-byte line");
+
+constexpr unsigned FLAG_NONFINITE = 1u;
+constexpr unsigned FLAG_TIMEOUT = 2u;
+
+// One linear-recurrence problem in "scan order".  Position s = 0..T-1 of the
+// scan corresponds to t = s (forward) or t = T-1-s (reverse); the matrix of
+// position s is J[t] (forward) or J[t+1]^T (reverse; identity at s = 0).
+struct ScanArgs {
+    const float *J;      // [B,T,n,n]
+    const float *b;      // [B,T,n]
+    const float *y0;     // [B,n] or nullptr
+    float *y;            // [B,T,n] out
+    const float *yold;   // [B,T,n] or nullptr: previous iterate for max|y - yold|
+    int B, T, n, reverse;
+    int L, nch;          // chunk length, chunks per sequence
+    float *carA;         // [B,nch,n,n] chunk aggregates (matrix part)
+    float *carB;         // [B,nch,n]   chunk aggregates (vector part)
+    float *starts;       // [B,nch,n]   state entering each chunk
+    StatusBlock *st;
+};
+
+struct CellArgs {
+    const float *W_h;    // [3n,n]
+    const float *b_h;    // [3n]
+    const float *u;      // [B,T,3n] input projection  x W_i^T + b_i
+    const float *y;      // [B,T,n] current trajectory guess
+    const float *y0;     // [B,n]
+    float *J;            // [B,T,n,n] out
+    float *rhs;          // [B,T,n]   out: f - J y_prev   (nullptr: skip)
+    int B, T, n;
+};
+
+__device__ __forceinline__ float sigmoidf_acc(float a) { return 1.0f / (1.0f + expf(-a)); }
+
+__device__ __forceinline__ unsigned absdiff_bits(float a, float b) {
+    return __float_as_uint(fabsf(a - b));   // NaN keeps bits above +inf: an integer max propagates it
+}
+
+static inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+}  // namespace deer

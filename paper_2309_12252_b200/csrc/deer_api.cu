@@ -1,0 +1,485 @@
+// C-ABI entry points of the DEER-GRU library: validation, workspace carving,
+// kernel sequencing and the Newton loop control.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "kernels_generic.cuh"
+
+namespace deer {
+
+std::atomic<long long> g_launches{0};
+static thread_local char t_err[256] = "";
+
+void set_error(cudaError_t e, const char *where)
+{
+    snprintf(t_err, sizeof(t_err), "%s: %s", where, cudaGetErrorString(e));
+}
+
+// Bump allocator over the caller's workspace; with base == nullptr it only measures.
+struct Carver {
+    char *base;
+    size_t off = 0;
+    explicit Carver(void *b) : base((char *)b) {}
+    template <typename T> T *take(size_t count)
+    {
+        size_t o = off;
+        off = align_up(off + count * sizeof(T));
+        return base ? (T *)(base + o) : nullptr;
+    }
+};
+
+static int gen_chunk_len(int T)
+{
+    int L = (int)ceil(sqrt((double)T));
+    if (L < 16) L = 16;
+    if (L > 256) L = 256;
+    return L;
+}
+
+struct ScanWs {
+    float *carA, *carB, *starts;
+    int L, nch;
+};
+
+static ScanWs carve_scan(Carver &cv, int B, int T, int n)
+{
+    ScanWs w;
+    w.L = gen_chunk_len(T);
+    w.nch = (T + w.L - 1) / w.L;
+    w.carA = cv.take<float>((size_t)B * w.nch * n * n);
+    w.carB = cv.take<float>((size_t)B * w.nch * n);
+    w.starts = cv.take<float>((size_t)B * w.nch * n);
+    return w;
+}
+
+static int opt_in_smem(const void *fn, size_t bytes)
+{
+    if (bytes > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute"); return DEER_ERR_CUDA; }
+    }
+    return DEER_OK;
+}
+
+// Three-level scan with the generic kernels.
+static int scan_generic(ScanArgs a, cudaStream_t st)
+{
+    const int n = a.n, nn = n * n;
+    size_t sm_red = sizeof(float) * (3 * nn + 2 * n);
+    size_t sm_car = sizeof(float) * (nn + n);
+    int rc;
+    if ((rc = opt_in_smem((const void *)gen_reduce_kernel, sm_red)) != DEER_OK) return rc;
+    dim3 grid(a.nch, a.B);
+    if (a.nch > 1) {
+        gen_reduce_kernel<<<grid, GEN_THREADS, sm_red, st>>>(a);
+        DEER_CHECK_LAUNCH("gen_reduce_kernel");
+    }
+    gen_carry_kernel<<<a.B, GEN_THREADS, sm_car, st>>>(a);
+    DEER_CHECK_LAUNCH("gen_carry_kernel");
+    gen_apply_kernel<<<grid, GEN_THREADS, sm_car, st>>>(a);
+    DEER_CHECK_LAUNCH("gen_apply_kernel");
+    return DEER_OK;
+}
+
+static int run_scan(ScanArgs a, int flags, cudaStream_t st)
+{
+    (void)flags;
+    return scan_generic(a, st);
+}
+
+static int run_proj(const deer_gru_params *p, const float *x, float *u, size_t N, cudaStream_t st)
+{
+    size_t total = N * 3 * (size_t)p->n;
+    unsigned blocks = (unsigned)((total + 255) / 256);
+    proj_kernel<<<blocks, 256, 0, st>>>(x, p->W_i, p->b_i, u, N, p->m, 3 * p->n);
+    DEER_CHECK_LAUNCH("proj_kernel");
+    return DEER_OK;
+}
+
+static int run_cell(CellArgs c, cudaStream_t st)
+{
+    const int n = c.n;
+    size_t sm = sizeof(float) * (3 * n * (n + 1) + 3 * n);
+    int rc;
+    if ((rc = opt_in_smem((const void *)cell_kernel, sm)) != DEER_OK) return rc;
+    int threads = 256;
+    int epb = threads / n;
+    size_t N = (size_t)c.B * c.T;
+    unsigned blocks = (unsigned)((N + epb - 1) / epb);
+    cell_kernel<<<blocks, threads, sm, st>>>(c);
+    DEER_CHECK_LAUNCH("cell_kernel");
+    return DEER_OK;
+}
+
+static bool valid_sizes(int B, int T, int n, int m)
+{
+    return B > 0 && T > 0 && n > 0 && m > 0 && (double)B * T * n * n < 9.0e18;
+}
+
+static bool supported(int n, int m) { return n >= 1 && n <= 64 && m >= 1 && m <= 1024; }
+
+// ---------------------------------------------------------------- workspace layouts
+struct EvalWs {
+    StatusBlock *st;
+    float *u, *J, *rhs, *yalt;
+    ScanWs scan;
+    size_t bytes;
+};
+
+static EvalWs carve_eval(void *ws, int B, int T, int n, int m)
+{
+    (void)m;
+    Carver cv(ws);
+    EvalWs w;
+    size_t N = (size_t)B * T;
+    w.st = cv.take<StatusBlock>(1);
+    w.u = cv.take<float>(N * 3 * n);
+    w.J = cv.take<float>(N * n * n);
+    w.rhs = cv.take<float>(N * n);
+    w.yalt = cv.take<float>(N * n);
+    w.scan = carve_scan(cv, B, T, n);
+    w.bytes = cv.off;
+    return w;
+}
+
+struct ScanOnlyWs {
+    StatusBlock *st;
+    ScanWs scan;
+    size_t bytes;
+};
+
+static ScanOnlyWs carve_scan_only(void *ws, int B, int T, int n)
+{
+    Carver cv(ws);
+    ScanOnlyWs w;
+    w.st = cv.take<StatusBlock>(1);
+    w.scan = carve_scan(cv, B, T, n);
+    w.bytes = cv.off;
+    return w;
+}
+
+constexpr int WGRAD_P = 592;   // slices of the position axis in the parameter-gradient reduction
+
+struct VjpWs {
+    StatusBlock *st;
+    float *u, *J, *rhs, *lam, *dGi, *dGh, *partial;
+    ScanWs scan;
+    size_t bytes;
+};
+
+static VjpWs carve_vjp(void *ws, int B, int T, int n, int m)
+{
+    Carver cv(ws);
+    VjpWs w;
+    size_t N = (size_t)B * T;
+    w.st = cv.take<StatusBlock>(1);
+    w.u = cv.take<float>(N * 3 * n);
+    w.J = cv.take<float>(N * n * n);
+    w.lam = cv.take<float>(N * n);
+    w.dGi = cv.take<float>(N * 3 * n);
+    w.dGh = cv.take<float>(N * 3 * n);
+    int kmax = (m > n ? m : n) + 1;
+    w.partial = cv.take<float>((size_t)WGRAD_P * 3 * n * kmax);
+    w.scan = carve_scan(cv, B, T, n);
+    w.rhs = nullptr;
+    w.bytes = cv.off;
+    return w;
+}
+
+struct ClsWs {
+    float *y1, *y2, *gyA, *gyB, *pool_partial, *pooled, *dlog, *gpool, *loss;
+    void *inner;
+    size_t inner_bytes, bytes;
+};
+constexpr int POOL_SEGS = 64;
+
+static ClsWs carve_cls(void *ws, int B, int T, int n, int m, int ncls)
+{
+    Carver cv(ws);
+    ClsWs w;
+    size_t N = (size_t)B * T;
+    w.y1 = cv.take<float>(N * n);
+    w.y2 = cv.take<float>(N * n);
+    w.gyA = cv.take<float>(N * n);
+    w.gyB = cv.take<float>(N * n);
+    w.pool_partial = cv.take<float>((size_t)B * POOL_SEGS * n);
+    w.pooled = cv.take<float>((size_t)B * n);
+    w.dlog = cv.take<float>((size_t)B * ncls);
+    w.gpool = cv.take<float>((size_t)B * n);
+    w.loss = cv.take<float>(64);
+    int mm = m > n ? m : n;
+    size_t e = carve_eval(nullptr, B, T, n, mm).bytes;
+    size_t v = carve_vjp(nullptr, B, T, n, mm).bytes;
+    w.inner_bytes = e > v ? e : v;
+    w.inner = cv.take<char>(w.inner_bytes);
+    w.bytes = cv.off;
+    return w;
+}
+
+static int check_ws(void *ws, size_t have, size_t need)
+{
+    if (!ws || ((uintptr_t)ws & 255) != 0 || have < need) return DEER_ERR_WORKSPACE;
+    return DEER_OK;
+}
+
+// ---------------------------------------------------------------- implementation bodies
+static int linrec_scan_impl(const float *J, const float *b, const float *y0, int B, int T, int n,
+                            int reverse, float *y, void *ws, size_t ws_bytes, int flags,
+                            cudaStream_t st)
+{
+    ScanOnlyWs w = carve_scan_only(ws, B, T, n);
+    int rc = check_ws(ws, ws_bytes, w.bytes);
+    if (rc != DEER_OK) return rc;
+    ScanArgs a{};
+    a.J = J; a.b = b; a.y0 = y0; a.y = y; a.yold = nullptr;
+    a.B = B; a.T = T; a.n = n; a.reverse = reverse ? 1 : 0;
+    a.L = w.scan.L; a.nch = w.scan.nch;
+    a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
+    a.st = w.st;
+    return run_scan(a, flags, st);
+}
+
+static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *y0, int B, int T,
+                         float tol, int max_iter, float *y, int *iters, float *err,
+                         float *err_trace, void *ws, size_t ws_bytes, int flags, cudaStream_t st)
+{
+    const int n = p->n, m = p->m;
+    EvalWs w = carve_eval(ws, B, T, n, m);
+    int rc = check_ws(ws, ws_bytes, w.bytes);
+    if (rc != DEER_OK) return rc;
+    const size_t N = (size_t)B * T;
+    DEER_CHECK_CUDA(cudaMemsetAsync(w.st, 0, sizeof(StatusBlock), st), "memset status");
+    if (!(flags & DEER_FLAG_WARM_START))
+        DEER_CHECK_CUDA(cudaMemsetAsync(y, 0, N * n * sizeof(float), st), "memset y");
+    if ((rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
+
+    float *cur = y, *nxt = w.yalt;
+    float e = 1e10f;
+    int k = 0;
+    int status = DEER_OK;
+    while (e > tol && k < max_iter) {
+        CellArgs c{p->W_h, p->b_h, w.u, cur, y0, w.J, w.rhs, B, T, n};
+        if ((rc = run_cell(c, st)) != DEER_OK) return rc;
+        DEER_CHECK_CUDA(cudaMemsetAsync(&w.st->err_bits, 0, sizeof(unsigned), st), "memset err");
+        ScanArgs a{};
+        a.J = w.J; a.b = w.rhs; a.y0 = y0; a.y = nxt; a.yold = cur;
+        a.B = B; a.T = T; a.n = n; a.reverse = 0;
+        a.L = w.scan.L; a.nch = w.scan.nch;
+        a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
+        a.st = w.st;
+        if ((rc = run_scan(a, flags, st)) != DEER_OK) return rc;
+        unsigned bits = 0;
+        DEER_CHECK_CUDA(cudaMemcpyAsync(&bits, &w.st->err_bits, sizeof(unsigned),
+                                        cudaMemcpyDeviceToHost, st), "read err");
+        DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+        memcpy(&e, &bits, sizeof(float));
+        float *tmp = cur; cur = nxt; nxt = tmp;
+        if (err_trace) err_trace[k] = e;
+        ++k;
+        if (!isfinite(e)) { status = DEER_NONFINITE; break; }
+    }
+    if (cur != y) {
+        DEER_CHECK_CUDA(cudaMemcpyAsync(y, cur, N * n * sizeof(float), cudaMemcpyDeviceToDevice, st),
+                        "copy result");
+        DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+    }
+    if (status == DEER_OK && e > tol && !(tol < 0.0f)) status = DEER_NOT_CONVERGED;
+    if (iters) *iters = k;
+    if (err) *err = e;
+    return status;
+}
+
+static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y0, const float *y,
+                        const float *gy, int B, int T, const deer_gru_grads *g, float *dx,
+                        float *dy0, void *ws, size_t ws_bytes, int flags, cudaStream_t st)
+{
+    const int n = p->n, m = p->m, n3 = 3 * n;
+    VjpWs w = carve_vjp(ws, B, T, n, m);
+    int rc = check_ws(ws, ws_bytes, w.bytes);
+    if (rc != DEER_OK) return rc;
+    const size_t N = (size_t)B * T;
+    if ((rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
+    CellArgs c{p->W_h, p->b_h, w.u, y, y0, w.J, nullptr, B, T, n};
+    if ((rc = run_cell(c, st)) != DEER_OK) return rc;
+    ScanArgs a{};
+    a.J = w.J; a.b = gy; a.y0 = nullptr; a.y = w.lam; a.yold = nullptr;
+    a.B = B; a.T = T; a.n = n; a.reverse = 1;
+    a.L = w.scan.L; a.nch = w.scan.nch;
+    a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
+    a.st = w.st;
+    if ((rc = run_scan(a, flags, st)) != DEER_OK) return rc;
+
+    {
+        VjpArgs v{p->W_h, p->b_h, w.u, y, y0, w.lam, w.dGi, w.dGh, B, T, n};
+        size_t sm = sizeof(float) * (3 * n * (n + 1) + 3 * n);
+        if ((rc = opt_in_smem((const void *)vjp_cell_kernel, sm)) != DEER_OK) return rc;
+        int epb = 256 / n;
+        unsigned blocks = (unsigned)((N + epb - 1) / epb);
+        vjp_cell_kernel<<<blocks, 256, sm, st>>>(v);
+        DEER_CHECK_LAUNCH("vjp_cell_kernel");
+    }
+    const int P = (int)(N < (size_t)WGRAD_P ? N : (size_t)WGRAD_P);
+    for (int side = 0; side < 2; ++side) {
+        WgradArgs wa{};
+        wa.dG = side == 0 ? w.dGi : w.dGh;
+        wa.V = side == 0 ? x : y;
+        wa.y0 = y0;
+        wa.shifted = side;
+        wa.T = T; wa.n3 = n3; wa.K = side == 0 ? m : n;
+        wa.N = N; wa.slice = (N + P - 1) / P;
+        wa.partial = w.partial;
+        int tile = 32;
+        while (tile > 1 && sizeof(float) * tile * (size_t)(n3 + wa.K + 1) > 160 * 1024) tile >>= 1;
+        wa.tile = tile;
+        size_t sm = sizeof(float) * tile * (size_t)(n3 + wa.K + 1);
+        if ((rc = opt_in_smem((const void *)wgrad_partial_kernel, sm)) != DEER_OK) return rc;
+        int outs = n3 * (wa.K + 1);
+        dim3 grid(P, (outs + 255) / 256);
+        wgrad_partial_kernel<<<grid, 256, sm, st>>>(wa);
+        DEER_CHECK_LAUNCH("wgrad_partial_kernel");
+        wgrad_final_kernel<<<(outs + 255) / 256, 256, 0, st>>>(w.partial, P, n3, wa.K,
+                                                                side == 0 ? g->dW_i : g->dW_h,
+                                                                side == 0 ? g->db_i : g->db_h);
+        DEER_CHECK_LAUNCH("wgrad_final_kernel");
+    }
+    if (dx) {
+        size_t total = N * (size_t)m;
+        vjp_dx_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w.dGi, p->W_i, dx, N, m, n3);
+        DEER_CHECK_LAUNCH("vjp_dx_kernel");
+    }
+    if (dy0) {
+        vjp_dy0_kernel<<<(B * n + 127) / 128, 128, 0, st>>>(w.J, w.lam, dy0, B, T, n);
+        DEER_CHECK_LAUNCH("vjp_dy0_kernel");
+    }
+    return DEER_OK;
+}
+
+}  // namespace deer
+
+using namespace deer;
+
+// ---------------------------------------------------------------- exported C ABI
+extern "C" {
+
+size_t deer_workspace_bytes(int op, int B, int T, int n, int m, int flags)
+{
+    (void)flags;
+    if (op == DEER_OP_SCAN) m = 1;
+    if (!valid_sizes(B, T, n, m) || !supported(n, m)) return 0;
+    switch (op) {
+    case DEER_OP_EVAL: return carve_eval(nullptr, B, T, n, m).bytes;
+    case DEER_OP_SCAN: return carve_scan_only(nullptr, B, T, n).bytes;
+    case DEER_OP_VJP: return carve_vjp(nullptr, B, T, n, m).bytes;
+    case DEER_OP_CLASSIFIER: return carve_cls(nullptr, B, T, n, m, 64).bytes;
+    default: return 0;
+    }
+}
+
+int deer_linrec_scan(const float *J, const float *b, const float *y0, int B, int T, int n,
+                     int reverse, float *y, void *ws, size_t ws_bytes, int flags, void *stream)
+{
+    if (!J || !b || !y || B <= 0 || T <= 0 || n <= 0) return DEER_ERR_INVALID_ARG;
+    if (!supported(n, 1)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, n, 1)) return DEER_ERR_INVALID_ARG;
+    return linrec_scan_impl(J, b, y0, B, T, n, reverse, y, ws, ws_bytes, flags, (cudaStream_t)stream);
+}
+
+int deer_gru_eval(const deer_gru_params *p, const float *x, const float *y0, int B, int T, float tol,
+                  int max_iter, float *y, int *iters, float *err, float *err_trace, void *ws,
+                  size_t ws_bytes, int flags, void *stream)
+{
+    if (!p || !x || !y0 || !y || !p->W_i || !p->W_h || !p->b_i || !p->b_h) return DEER_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || p->n <= 0 || p->m <= 0 || max_iter < 1 || tol != tol) return DEER_ERR_INVALID_ARG;
+    if (!supported(p->n, p->m)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
+    return gru_eval_impl(p, x, y0, B, T, tol, max_iter, y, iters, err, err_trace, ws, ws_bytes, flags,
+                         (cudaStream_t)stream);
+}
+
+int deer_gru_vjp(const deer_gru_params *p, const float *x, const float *y0, const float *y,
+                 const float *gy, int B, int T, const deer_gru_grads *g, float *dx, float *dy0,
+                 void *ws, size_t ws_bytes, int flags, void *stream)
+{
+    if (!p || !x || !y0 || !y || !gy || !g || !p->W_i || !p->W_h || !p->b_i || !p->b_h)
+        return DEER_ERR_INVALID_ARG;
+    if (!g->dW_i || !g->dW_h || !g->db_i || !g->db_h) return DEER_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || p->n <= 0 || p->m <= 0) return DEER_ERR_INVALID_ARG;
+    if (!supported(p->n, p->m)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
+    return gru_vjp_impl(p, x, y0, y, gy, B, T, g, dx, dy0, ws, ws_bytes, flags, (cudaStream_t)stream);
+}
+
+int deer_gru_classifier_step(const deer_gru_params *l1, const deer_gru_params *l2, const float *W_o,
+                             const float *b_o, int ncls, const float *x, const int *labels, int B,
+                             int T, float tol, int max_iter, float *loss, int *iters,
+                             const deer_gru_grads *g1, const deer_gru_grads *g2, float *dW_o,
+                             float *db_o, void *ws, size_t ws_bytes, int flags, void *stream)
+{
+    if (!l1 || !l2 || !W_o || !b_o || !x || !labels || !loss || !g1 || !g2 || !dW_o || !db_o)
+        return DEER_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || ncls < 1 || ncls > 64 || max_iter < 1 || tol != tol) return DEER_ERR_INVALID_ARG;
+    if (l1->n != l2->n || l2->m != l1->n) return DEER_ERR_INVALID_ARG;
+    if (!supported(l1->n, l1->m) || !supported(l2->n, l2->m)) return DEER_ERR_UNSUPPORTED_N;
+    if (B * ncls > 4096 || B * l1->n > 65536) return DEER_ERR_INVALID_ARG;
+    const int n = l1->n, m = l1->m;
+    cudaStream_t st = (cudaStream_t)stream;
+    ClsWs w = carve_cls(ws, B, T, n, m, 64);
+    int rc = check_ws(ws, ws_bytes, w.bytes);
+    if (rc != DEER_OK) return rc;
+    const size_t N = (size_t)B * T;
+    // zero initial states live at the head of gyB until the backward pass needs it
+    float *zero0 = w.gyB;
+    DEER_CHECK_CUDA(cudaMemsetAsync(zero0, 0, (size_t)B * n * sizeof(float), st), "memset y0");
+    int it[2] = {0, 0};
+    int s1 = deer_gru_eval(l1, x, zero0, B, T, tol, max_iter, w.y1, &it[0], nullptr, nullptr, w.inner,
+                           w.inner_bytes, flags, stream);
+    if (s1 < 0) return s1;
+    int s2 = deer_gru_eval(l2, w.y1, zero0, B, T, tol, max_iter, w.y2, &it[1], nullptr, nullptr,
+                           w.inner, w.inner_bytes, flags, stream);
+    if (s2 < 0) return s2;
+    if (iters) { iters[0] = it[0]; iters[1] = it[1]; }
+    int seg_len = (T + POOL_SEGS - 1) / POOL_SEGS;
+    pool_partial_kernel<<<dim3(POOL_SEGS, B), n, 0, st>>>(w.y2, T, n, seg_len, w.pool_partial);
+    DEER_CHECK_LAUNCH("pool_partial_kernel");
+    head_kernel<<<1, 256, 0, st>>>(w.pool_partial, POOL_SEGS, B, T, n, ncls, W_o, b_o, labels,
+                                   w.pooled, w.dlog, w.gpool, dW_o, db_o, w.loss);
+    DEER_CHECK_LAUNCH("head_kernel");
+    size_t total = N * n;
+    broadcast_gy_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w.gpool, w.gyA, total, T, n);
+    DEER_CHECK_LAUNCH("broadcast_gy_kernel");
+    // zero states again (gyB is about to be overwritten by dx of layer 2): use pooled' neighbour
+    float *zero1 = w.pool_partial;   // >= B*n floats, no longer needed
+    DEER_CHECK_CUDA(cudaMemsetAsync(zero1, 0, (size_t)B * n * sizeof(float), st), "memset y0");
+    rc = deer_gru_vjp(l2, w.y1, zero1, w.y2, w.gyA, B, T, g2, w.gyB, nullptr, w.inner, w.inner_bytes,
+                      flags, stream);
+    if (rc != DEER_OK) return rc;
+    rc = deer_gru_vjp(l1, x, zero1, w.y1, w.gyB, B, T, g1, nullptr, nullptr, w.inner, w.inner_bytes,
+                      flags, stream);
+    if (rc != DEER_OK) return rc;
+    DEER_CHECK_CUDA(cudaMemcpyAsync(loss, w.loss, sizeof(float), cudaMemcpyDeviceToHost, st), "read loss");
+    DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+    return s1 > s2 ? s1 : s2;
+}
+
+const char *deer_status_string(int s)
+{
+    switch (s) {
+    case DEER_OK: return "ok";
+    case DEER_NOT_CONVERGED: return "not converged within max_iter";
+    case DEER_NONFINITE: return "non-finite values in the iterate";
+    case DEER_ERR_INVALID_ARG: return "invalid argument";
+    case DEER_ERR_UNSUPPORTED_N: return "unsupported hidden or input size";
+    case DEER_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case DEER_ERR_CUDA: return "CUDA runtime error";
+    case DEER_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+    default: return "unknown status";
+    }
+}
+
+const char *deer_last_error(void) { return t_err; }
+
+long long deer_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

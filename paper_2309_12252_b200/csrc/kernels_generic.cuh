@@ -1,0 +1,409 @@
+// Generic (any 1 <= n <= 64) kernels: input projection, cell + Jacobian + rhs,
+// three-level chunked scan, cell VJP and the deterministic parameter-gradient
+// reductions.  Simple shared-memory formulations; the tuned paths for
+// n in {1,2,4,8} and the tensor-core paths replace the scan / cell kernels
+// where they apply.
+#pragma once
+#include "common.cuh"
+
+namespace deer {
+
+constexpr int GEN_THREADS = 128;
+
+// ------------------------------------------------------------------ a0: u = x W_i^T + b_i
+__global__ void proj_kernel(const float *__restrict__ x, const float *__restrict__ W_i,
+                            const float *__restrict__ b_i, float *__restrict__ u, size_t N, int m,
+                            int n3)
+{
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= N * (size_t)n3) return;
+    size_t e = idx / n3;
+    int g = (int)(idx - e * n3);
+    const float *xr = x + e * m;
+    const float *wr = W_i + (size_t)g * m;
+    float acc = b_i[g];
+    for (int k = 0; k < m; ++k) acc = fmaf(wr[k], xr[k], acc);
+    u[idx] = acc;
+}
+
+// ------------------------------------------------------------------ a1-a4: cell, Jacobian, rhs
+// One thread per (position, output row).  Closed-form Jacobian
+//   J = diag(z) + diag(a_z) W_hz + diag(a_n r) W_hn + diag(a_n q r (1-r)) W_hr.
+__global__ void cell_kernel(CellArgs a)
+{
+    extern __shared__ float sW[];          // W_h rows padded to n+1, then b_h
+    const int n = a.n, ld = n + 1;
+    float *sb = sW + 3 * n * ld;
+    for (int i = threadIdx.x; i < 3 * n * n; i += blockDim.x) sW[(i / n) * ld + (i % n)] = a.W_h[i];
+    for (int i = threadIdx.x; i < 3 * n; i += blockDim.x) sb[i] = a.b_h[i];
+    __syncthreads();
+    const int epb = blockDim.x / n;
+    const int le = threadIdx.x / n, i = threadIdx.x % n;
+    const size_t N = (size_t)a.B * a.T;
+    const size_t e = (size_t)blockIdx.x * epb + le;
+    if (le >= epb || e >= N) return;
+    const int t = (int)(e % a.T);
+    const size_t seq = e / a.T;
+    const float *hp = (t == 0) ? a.y0 + seq * n : a.y + (e - 1) * n;
+    float gr = sb[i], gz = sb[n + i], gq = sb[2 * n + i];
+    for (int k = 0; k < n; ++k) {
+        float h = hp[k];
+        gr = fmaf(sW[i * ld + k], h, gr);
+        gz = fmaf(sW[(n + i) * ld + k], h, gz);
+        gq = fmaf(sW[(2 * n + i) * ld + k], h, gq);
+    }
+    const float *ue = a.u + e * 3 * n;
+    float r = sigmoidf_acc(ue[i] + gr);
+    float z = sigmoidf_acc(ue[n + i] + gz);
+    float c = tanhf(ue[2 * n + i] + r * gq);
+    float hi = hp[i];
+    float f = (1.0f - z) * c + z * hi;
+    float az = (hi - c) * z * (1.0f - z);
+    float an = (1.0f - z) * (1.0f - c * c);
+    float kr = an * gq * r * (1.0f - r);
+    float kn = an * r;
+    float acc = 0.0f;
+    float *Jr = a.J + (e * n + i) * n;
+    for (int j = 0; j < n; ++j) {
+        float v = kr * sW[i * ld + j] + az * sW[(n + i) * ld + j] + kn * sW[(2 * n + i) * ld + j];
+        if (j == i) v += z;
+        Jr[j] = v;
+        acc = fmaf(v, hp[j], acc);
+    }
+    if (a.rhs) a.rhs[e * n + i] = f - acc;
+}
+
+// ------------------------------------------------------------------ a5: generic chunked scan
+__device__ __forceinline__ void gen_load_M(float *dst, const ScanArgs &a, size_t seq, int s)
+{
+    const int n = a.n, nn = n * n;
+    if (!a.reverse) {
+        const float *src = a.J + (seq * a.T + s) * nn;
+        for (int i = threadIdx.x; i < nn; i += blockDim.x) dst[i] = src[i];
+    } else if (s == 0) {
+        for (int i = threadIdx.x; i < nn; i += blockDim.x) dst[i] = (i / n == i % n) ? 1.0f : 0.0f;
+    } else {
+        const float *src = a.J + (seq * a.T + (a.T - s)) * nn;     // J[t+1], t = T-1-s
+        for (int i = threadIdx.x; i < nn; i += blockDim.x) dst[(i % n) * n + (i / n)] = src[i];
+    }
+}
+
+__device__ __forceinline__ size_t gen_vec_index(const ScanArgs &a, size_t seq, int s, int i)
+{
+    int t = a.reverse ? a.T - 1 - s : s;
+    return (seq * a.T + t) * a.n + i;
+}
+
+// level 1: one CTA folds one chunk into (A, beta), later positions multiplying on the left.
+__global__ void gen_reduce_kernel(ScanArgs a)
+{
+    extern __shared__ float sm[];
+    const int n = a.n, nn = n * n;
+    float *Jt = sm, *A = sm + nn, *A2 = sm + 2 * nn, *be = sm + 3 * nn, *be2 = be + n;
+    const int c = blockIdx.x;
+    const size_t seq = blockIdx.y;
+    const int s0 = c * a.L, s1 = min(a.T, s0 + a.L);
+    gen_load_M(A, a, seq, s0);
+    if (threadIdx.x < n) be[threadIdx.x] = a.b[gen_vec_index(a, seq, s0, threadIdx.x)];
+    __syncthreads();
+    for (int s = s0 + 1; s < s1; ++s) {
+        gen_load_M(Jt, a, seq, s);
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < nn; idx += blockDim.x) {
+            int i = idx / n, j = idx % n;
+            float acc = 0.0f;
+            for (int k = 0; k < n; ++k) acc = fmaf(Jt[i * n + k], A[k * n + j], acc);
+            A2[idx] = acc;
+        }
+        if (threadIdx.x < n) {
+            float acc = a.b[gen_vec_index(a, seq, s, threadIdx.x)];
+            for (int k = 0; k < n; ++k) acc = fmaf(Jt[threadIdx.x * n + k], be[k], acc);
+            be2[threadIdx.x] = acc;
+        }
+        __syncthreads();
+        float *tmp = A; A = A2; A2 = tmp;
+        tmp = be; be = be2; be2 = tmp;
+    }
+    float *oA = a.carA + (seq * a.nch + c) * nn;
+    for (int i = threadIdx.x; i < nn; i += blockDim.x) oA[i] = A[i];
+    if (threadIdx.x < n) a.carB[(seq * a.nch + c) * n + threadIdx.x] = be[threadIdx.x];
+}
+
+// level 2: one CTA per sequence walks the chunk aggregates in order.
+__global__ void gen_carry_kernel(ScanArgs a)
+{
+    extern __shared__ float sm[];
+    const int n = a.n, nn = n * n;
+    float *Am = sm, *Y = sm + nn;
+    const size_t seq = blockIdx.x;
+    if (threadIdx.x < n) Y[threadIdx.x] = a.y0 ? a.y0[seq * n + threadIdx.x] : 0.0f;
+    __syncthreads();
+    for (int c = 0; c < a.nch; ++c) {
+        if (threadIdx.x < n) a.starts[(seq * a.nch + c) * n + threadIdx.x] = Y[threadIdx.x];
+        if (c == a.nch - 1) break;
+        const float *src = a.carA + (seq * a.nch + c) * nn;
+        for (int i = threadIdx.x; i < nn; i += blockDim.x) Am[i] = src[i];
+        __syncthreads();
+        float v = 0.0f;
+        if (threadIdx.x < n) {
+            v = a.carB[(seq * a.nch + c) * n + threadIdx.x];
+            for (int k = 0; k < n; ++k) v = fmaf(Am[threadIdx.x * n + k], Y[k], v);
+        }
+        __syncthreads();
+        if (threadIdx.x < n) Y[threadIdx.x] = v;
+        __syncthreads();
+    }
+}
+
+// level 3: one CTA replays its chunk from the entering state, writes y and the max deviation.
+__global__ void gen_apply_kernel(ScanArgs a)
+{
+    extern __shared__ float sm[];
+    const int n = a.n, nn = n * n;
+    float *Jt = sm, *Y = sm + nn;
+    const int c = blockIdx.x;
+    const size_t seq = blockIdx.y;
+    const int s0 = c * a.L, s1 = min(a.T, s0 + a.L);
+    if (threadIdx.x < n) Y[threadIdx.x] = a.starts[(seq * a.nch + c) * n + threadIdx.x];
+    unsigned mb = 0;
+    for (int s = s0; s < s1; ++s) {
+        gen_load_M(Jt, a, seq, s);
+        __syncthreads();
+        float v = 0.0f;
+        size_t idx = 0;
+        if (threadIdx.x < n) {
+            idx = gen_vec_index(a, seq, s, threadIdx.x);
+            v = a.b[idx];
+            for (int k = 0; k < n; ++k) v = fmaf(Jt[threadIdx.x * n + k], Y[k], v);
+        }
+        __syncthreads();
+        if (threadIdx.x < n) {
+            Y[threadIdx.x] = v;
+            if (a.yold) mb = max(mb, absdiff_bits(v, a.yold[idx]));
+            a.y[idx] = v;
+        }
+    }
+    if (a.yold) {
+        for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+        if ((threadIdx.x & 31) == 0 && mb) atomicMax(&a.st->err_bits, mb);
+    }
+}
+
+// ------------------------------------------------------------------ a8: cell VJP
+struct VjpArgs {
+    const float *W_h, *b_h, *u, *y, *y0, *lam;   // lam [B,T,n] = dL/df at every position
+    float *dGi, *dGh;                            // [B,T,3n] gradients w.r.t. u and w.r.t. W_h h + b_h
+    int B, T, n;
+};
+
+__global__ void vjp_cell_kernel(VjpArgs a)
+{
+    extern __shared__ float sW[];
+    const int n = a.n, ld = n + 1;
+    float *sb = sW + 3 * n * ld;
+    for (int i = threadIdx.x; i < 3 * n * n; i += blockDim.x) sW[(i / n) * ld + (i % n)] = a.W_h[i];
+    for (int i = threadIdx.x; i < 3 * n; i += blockDim.x) sb[i] = a.b_h[i];
+    __syncthreads();
+    const int epb = blockDim.x / n;
+    const int le = threadIdx.x / n, i = threadIdx.x % n;
+    const size_t N = (size_t)a.B * a.T;
+    const size_t e = (size_t)blockIdx.x * epb + le;
+    if (le >= epb || e >= N) return;
+    const int t = (int)(e % a.T);
+    const size_t seq = e / a.T;
+    const float *hp = (t == 0) ? a.y0 + seq * n : a.y + (e - 1) * n;
+    float gr = sb[i], gz = sb[n + i], gq = sb[2 * n + i];
+    for (int k = 0; k < n; ++k) {
+        float h = hp[k];
+        gr = fmaf(sW[i * ld + k], h, gr);
+        gz = fmaf(sW[(n + i) * ld + k], h, gz);
+        gq = fmaf(sW[(2 * n + i) * ld + k], h, gq);
+    }
+    const float *ue = a.u + e * 3 * n;
+    float r = sigmoidf_acc(ue[i] + gr);
+    float z = sigmoidf_acc(ue[n + i] + gz);
+    float c = tanhf(ue[2 * n + i] + r * gq);
+    float l = a.lam[e * n + i];
+    float dan = l * (1.0f - z) * (1.0f - c * c);
+    float daz = l * (hp[i] - c) * z * (1.0f - z);
+    float dar = dan * gq * r * (1.0f - r);
+    float dq = dan * r;
+    float *gi = a.dGi + e * 3 * n, *gh = a.dGh + e * 3 * n;
+    gi[i] = dar; gi[n + i] = daz; gi[2 * n + i] = dan;
+    gh[i] = dar; gh[n + i] = daz; gh[2 * n + i] = dq;
+}
+
+// dx[e][k] = sum_g W_i[g][k] dGi[e][g]
+__global__ void vjp_dx_kernel(const float *__restrict__ dGi, const float *__restrict__ W_i,
+                              float *__restrict__ dx, size_t N, int m, int n3)
+{
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= N * (size_t)m) return;
+    size_t e = idx / m;
+    int k = (int)(idx - e * m);
+    const float *g = dGi + e * n3;
+    float acc = 0.0f;
+    for (int j = 0; j < n3; ++j) acc = fmaf(W_i[(size_t)j * m + k], g[j], acc);
+    dx[idx] = acc;
+}
+
+// dy0[b][j] = sum_i J[b][0][i][j] lam[b][0][i]
+__global__ void vjp_dy0_kernel(const float *__restrict__ J, const float *__restrict__ lam,
+                               float *__restrict__ dy0, int B, int T, int n)
+{
+    int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= B * n) return;
+    int seq = idx / n, j = idx % n;
+    const float *J0 = J + (size_t)seq * T * n * n;
+    const float *l0 = lam + (size_t)seq * T * n;
+    float acc = 0.0f;
+    for (int i = 0; i < n; ++i) acc = fmaf(J0[i * n + j], l0[i], acc);
+    dy0[idx] = acc;
+}
+
+// Deterministic two-stage reduction  out[g][k] = sum_e dG[e][g] * V[e][k]  (k == K: bias, V = 1).
+// Stage 1: CTA (p, oy) accumulates 256 outputs over slice p of the positions, in position order.
+struct WgradArgs {
+    const float *dG;     // [N, n3]
+    const float *V;      // [N, K]; if shifted: row e is y[e-1] (y0 at t = 0)
+    const float *y0;
+    int shifted, T, n3, K, tile;
+    size_t N, slice;
+    float *partial;      // [P][n3*(K+1)]
+};
+
+__global__ void wgrad_partial_kernel(WgradArgs a)
+{
+    extern __shared__ float sm[];
+    const int K1 = a.K + 1, outs = a.n3 * K1;
+    float *gt = sm, *vt = sm + a.tile * a.n3;
+    const int o = blockIdx.y * blockDim.x + threadIdx.x;
+    const bool valid = o < outs;
+    const int g = valid ? o / K1 : 0, k = valid ? o % K1 : 0;
+    const size_t e0 = (size_t)blockIdx.x * a.slice;
+    const size_t e1 = min(a.N, e0 + a.slice);
+    float acc = 0.0f;
+    for (size_t base = e0; base < e1; base += a.tile) {
+        const int cnt = (int)min((size_t)a.tile, e1 - base);
+        for (int i = threadIdx.x; i < cnt * a.n3; i += blockDim.x) gt[i] = a.dG[base * a.n3 + i];
+        for (int i = threadIdx.x; i < cnt * K1; i += blockDim.x) {
+            int j = i / K1, kk = i % K1;
+            float v = 1.0f;
+            if (kk < a.K) {
+                size_t e = base + j;
+                if (!a.shifted) v = a.V[e * a.K + kk];
+                else {
+                    int t = (int)(e % a.T);
+                    v = (t == 0) ? a.y0[(e / a.T) * a.K + kk] : a.V[(e - 1) * a.K + kk];
+                }
+            }
+            vt[i] = v;
+        }
+        __syncthreads();
+        if (valid)
+            for (int j = 0; j < cnt; ++j) acc = fmaf(gt[j * a.n3 + g], vt[j * K1 + k], acc);
+        __syncthreads();
+    }
+    if (valid) a.partial[(size_t)blockIdx.x * outs + o] = acc;
+}
+
+// Stage 2: one thread per output adds the P slice sums in slice order.
+__global__ void wgrad_final_kernel(const float *__restrict__ partial, int P, int n3, int K,
+                                   float *__restrict__ dW, float *__restrict__ db)
+{
+    const int K1 = K + 1, outs = n3 * K1;
+    int o = blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= outs) return;
+    float acc = 0.0f;
+    for (int p = 0; p < P; ++p) acc += partial[(size_t)p * outs + o];
+    int g = o / K1, k = o % K1;
+    if (k < K) dW[(size_t)g * K + k] = acc;
+    else db[g] = acc;
+}
+
+// ------------------------------------------------------------------ a9: classifier glue
+// partial mean-pool: grid (segments, B), block = n threads
+__global__ void pool_partial_kernel(const float *__restrict__ y, int T, int n, int seg_len,
+                                    float *__restrict__ partial /*[B][S][n]*/)
+{
+    const int sgm = blockIdx.x, S = gridDim.x;
+    const size_t seq = blockIdx.y;
+    const int t0 = sgm * seg_len, t1 = min(T, t0 + seg_len);
+    const int i = threadIdx.x;
+    float acc = 0.0f;
+    for (int t = t0; t < t1; ++t) acc += y[(seq * T + t) * n + i];
+    partial[(seq * S + sgm) * n + i] = acc;
+}
+
+// head: pooled mean, logits, softmax cross-entropy (mean over batch), gradients of the head,
+// gradient w.r.t. the pooled vector scaled by 1/T.  One CTA, thread-serial where order matters.
+__global__ void head_kernel(const float *__restrict__ pool_partial, int S, int B, int T, int n,
+                            int ncls, const float *__restrict__ W_o, const float *__restrict__ b_o,
+                            const int *__restrict__ labels, float *__restrict__ pooled /*[B][n]*/,
+                            float *__restrict__ dlog /*[B][ncls]*/, float *__restrict__ gpool /*[B][n]*/,
+                            float *__restrict__ dW_o, float *__restrict__ db_o,
+                            float *__restrict__ loss_out)
+{
+    for (int idx = threadIdx.x; idx < B * n; idx += blockDim.x) {
+        int seq = idx / n, i = idx % n;
+        float acc = 0.0f;
+        for (int s = 0; s < S; ++s) acc += pool_partial[((size_t)seq * S + s) * n + i];
+        pooled[idx] = acc / (float)T;
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < B * ncls; idx += blockDim.x) {
+        int seq = idx / ncls, c = idx % ncls;
+        float l = b_o[c];
+        for (int i = 0; i < n; ++i) l = fmaf(W_o[c * n + i], pooled[seq * n + i], l);
+        dlog[idx] = l;
+    }
+    __syncthreads();
+    __shared__ float s_loss;
+    if (threadIdx.x == 0) {
+        float loss = 0.0f;
+        for (int seq = 0; seq < B; ++seq) {
+            float *l = dlog + seq * ncls;
+            float mx = l[0];
+            for (int c = 1; c < ncls; ++c) mx = fmaxf(mx, l[c]);
+            float se = 0.0f;
+            for (int c = 0; c < ncls; ++c) se += expf(l[c] - mx);
+            float lse = mx + logf(se);
+            loss += lse - l[labels[seq]];
+            for (int c = 0; c < ncls; ++c)
+                l[c] = (expf(l[c] - lse) - (c == labels[seq] ? 1.0f : 0.0f)) / (float)B;
+        }
+        s_loss = loss / (float)B;
+        *loss_out = s_loss;
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < ncls * n; idx += blockDim.x) {
+        int c = idx / n, i = idx % n;
+        float acc = 0.0f;
+        for (int seq = 0; seq < B; ++seq) acc = fmaf(dlog[seq * ncls + c], pooled[seq * n + i], acc);
+        dW_o[idx] = acc;
+    }
+    for (int c = threadIdx.x; c < ncls; c += blockDim.x) {
+        float acc = 0.0f;
+        for (int seq = 0; seq < B; ++seq) acc += dlog[seq * ncls + c];
+        db_o[c] = acc;
+    }
+    for (int idx = threadIdx.x; idx < B * n; idx += blockDim.x) {
+        int seq = idx / n, i = idx % n;
+        float acc = 0.0f;
+        for (int c = 0; c < ncls; ++c) acc = fmaf(W_o[c * n + i], dlog[seq * ncls + c], acc);
+        gpool[idx] = acc / (float)T;
+    }
+}
+
+// gy[b][t][i] = gpool[b][i] for every t
+__global__ void broadcast_gy_kernel(const float *__restrict__ gpool, float *__restrict__ gy,
+                                    size_t total, int T, int n)
+{
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    size_t seq = idx / ((size_t)T * n);
+    int i = (int)(idx % n);
+    gy[idx] = gpool[seq * n + i];
+}
+
+}  // namespace deer

@@ -1,0 +1,57 @@
+"""Host-side checks that need no GPU: the C-ABI library loads, exports every
+symbol the header declares, sizes workspaces sanely and refuses bad arguments
+before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2309_12252_b200 import build
+    path = build.build()
+    return ctypes.CDLL(path)
+
+
+def declared_functions():
+    src = open(os.path.join(ROOT, "include", "deer.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(deer_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_header_symbols_are_exported(L):
+    names = declared_functions()
+    assert {"deer_gru_eval", "deer_linrec_scan", "deer_gru_vjp", "deer_workspace_bytes"} <= set(names)
+    for name in names:
+        assert hasattr(L, name), name
+    from paper_2309_12252_b200 import binding
+    assert set(binding.EXPORTS) <= set(names)
+
+
+def test_workspace_sizes(L):
+    L.deer_workspace_bytes.restype = ctypes.c_size_t
+    f = lambda *a: int(L.deer_workspace_bytes(*a))
+    ev = f(0, 16, 10000, 8, 4, 0)
+    sc = f(1, 16, 10000, 8, 1, 0)
+    vj = f(2, 16, 10000, 8, 4, 0)
+    assert 0 < sc < ev and 0 < vj
+    assert ev % 256 == 0 and sc % 256 == 0
+    assert ev < 16 * 10000 * 8 * (8 + 3 + 2 + 2) * 4 * 2      # no gross over-allocation
+    assert f(0, 0, 10, 8, 4, 0) == 0 and f(0, 1, 10, 65, 4, 0) == 0 and f(9, 1, 10, 8, 4, 0) == 0
+    assert f(0, 16, 10000, 8, 4, 0) == ev                       # pure function of the sizes
+
+
+def test_status_strings_and_argument_validation(L):
+    L.deer_status_string.restype = ctypes.c_char_p
+    seen = {L.deer_status_string(s) for s in (0, 1, 2, -1, -2, -3, -4, -5)}
+    assert len(seen) == 8 and all(seen)
+    assert L.deer_linrec_scan(None, None, None, 1, 1, 1, 0, None, None, 0, 0, None) == -1
+    assert L.deer_gru_eval(None, None, None, 1, 1, ctypes.c_float(1e-4), 100, None, None, None, None,
+                           None, 0, 0, None) == -1
+    assert L.deer_gru_vjp(None, None, None, None, None, 1, 1, None, None, None, None, 0, 0, None) == -1
+    L.deer_launch_count.restype = ctypes.c_longlong
+    assert L.deer_launch_count() == 0
