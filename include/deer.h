@@ -156,6 +156,15 @@ const char *deer_last_error(void);
  * threads); take differences around a region to count its launches. */
 long long deer_launch_count(void);
 
+/* Benchmark aid (no counterpart in the paper): while enabled, every kernel
+ * launch of the library is bracketed by CUDA events on its stream.
+ * deer_profile_read() waits for the recorded events, writes one line
+ * "kernel_name launches total_ms" per kernel into buf (NUL-terminated, at
+ * most cap bytes), clears the records and returns the full text length.
+ * Adds two event records per launch, so it is kept out of timed regions. */
+void deer_profile_enable(int on);
+size_t deer_profile_read(char *buf, size_t cap);
+
 #ifdef __cplusplus
 }
 #endif

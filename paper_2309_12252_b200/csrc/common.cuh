@@ -20,6 +20,25 @@ void set_error(cudaError_t e, const char *where);
         }                                                          \
     } while (0)
 
+// Optional per-kernel timing (CUDA events on the launching stream) for benchmarks.
+struct KernelScope {
+    const char *name;
+    cudaStream_t st;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    KernelScope(const char *name, cudaStream_t st);
+    ~KernelScope();
+};
+
+// Launch statement wrapped with bookkeeping:  DEER_KERNEL("name", stream, kernel<<<...>>>(args));
+#define DEER_KERNEL(kname, stream, ...)                            \
+    do {                                                           \
+        {                                                          \
+            ::deer::KernelScope ks_(kname, stream);                \
+            __VA_ARGS__;                                           \
+        }                                                          \
+        DEER_CHECK_LAUNCH(kname);                                  \
+    } while (0)
+
 #define DEER_CHECK_CUDA(call, where)                               \
     do {                                                           \
         cudaError_t e_ = (call);                                   \

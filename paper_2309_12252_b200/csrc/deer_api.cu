@@ -4,6 +4,11 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <map>
+#include <mutex>
+#include <string>
+#include <vector>
+
 #include "common.cuh"
 #include "kernels_generic.cuh"
 
@@ -15,6 +20,27 @@ static thread_local char t_err[256] = "";
 void set_error(cudaError_t e, const char *where)
 {
     snprintf(t_err, sizeof(t_err), "%s: %s", where, cudaGetErrorString(e));
+}
+
+// ---- per-kernel profiling (off by default; benchmarks switch it on for a separate pass)
+struct ProfRec { const char *name; cudaEvent_t e0, e1; };
+static std::mutex g_prof_mu;
+static std::atomic<bool> g_prof_on{false};
+static std::vector<ProfRec> g_prof;
+
+KernelScope::KernelScope(const char *name_, cudaStream_t st_) : name(name_), st(st_)
+{
+    if (!g_prof_on.load(std::memory_order_relaxed)) return;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) { e0 = e1 = nullptr; return; }
+    cudaEventRecord(e0, st);
+}
+
+KernelScope::~KernelScope()
+{
+    if (!e0) return;
+    cudaEventRecord(e1, st);
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof.push_back({name, e0, e1});
 }
 
 // Bump allocator over the caller's workspace; with base == nullptr it only measures.
@@ -73,13 +99,10 @@ static int scan_generic(ScanArgs a, cudaStream_t st)
     if ((rc = opt_in_smem((const void *)gen_reduce_kernel, sm_red)) != DEER_OK) return rc;
     dim3 grid(a.nch, a.B);
     if (a.nch > 1) {
-        gen_reduce_kernel<<<grid, GEN_THREADS, sm_red, st>>>(a);
-        DEER_CHECK_LAUNCH("gen_reduce_kernel");
+        DEER_KERNEL("gen_reduce_kernel", st, gen_reduce_kernel<<<grid, GEN_THREADS, sm_red, st>>>(a));
     }
-    gen_carry_kernel<<<a.B, GEN_THREADS, sm_car, st>>>(a);
-    DEER_CHECK_LAUNCH("gen_carry_kernel");
-    gen_apply_kernel<<<grid, GEN_THREADS, sm_car, st>>>(a);
-    DEER_CHECK_LAUNCH("gen_apply_kernel");
+    DEER_KERNEL("gen_carry_kernel", st, gen_carry_kernel<<<a.B, GEN_THREADS, sm_car, st>>>(a));
+    DEER_KERNEL("gen_apply_kernel", st, gen_apply_kernel<<<grid, GEN_THREADS, sm_car, st>>>(a));
     return DEER_OK;
 }
 
@@ -93,8 +116,7 @@ static int run_proj(const deer_gru_params *p, const float *x, float *u, size_t N
 {
     size_t total = N * 3 * (size_t)p->n;
     unsigned blocks = (unsigned)((total + 255) / 256);
-    proj_kernel<<<blocks, 256, 0, st>>>(x, p->W_i, p->b_i, u, N, p->m, 3 * p->n);
-    DEER_CHECK_LAUNCH("proj_kernel");
+    DEER_KERNEL("proj_kernel", st, proj_kernel<<<blocks, 256, 0, st>>>(x, p->W_i, p->b_i, u, N, p->m, 3 * p->n));
     return DEER_OK;
 }
 
@@ -108,8 +130,7 @@ static int run_cell(CellArgs c, cudaStream_t st)
     int epb = threads / n;
     size_t N = (size_t)c.B * c.T;
     unsigned blocks = (unsigned)((N + epb - 1) / epb);
-    cell_kernel<<<blocks, threads, sm, st>>>(c);
-    DEER_CHECK_LAUNCH("cell_kernel");
+    DEER_KERNEL("cell_kernel", st, cell_kernel<<<blocks, threads, sm, st>>>(c));
     return DEER_OK;
 }
 
@@ -317,8 +338,7 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
         if ((rc = opt_in_smem((const void *)vjp_cell_kernel, sm)) != DEER_OK) return rc;
         int epb = 256 / n;
         unsigned blocks = (unsigned)((N + epb - 1) / epb);
-        vjp_cell_kernel<<<blocks, 256, sm, st>>>(v);
-        DEER_CHECK_LAUNCH("vjp_cell_kernel");
+        DEER_KERNEL("vjp_cell_kernel", st, vjp_cell_kernel<<<blocks, 256, sm, st>>>(v));
     }
     const int P = (int)(N < (size_t)WGRAD_P ? N : (size_t)WGRAD_P);
     for (int side = 0; side < 2; ++side) {
@@ -337,21 +357,17 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
         if ((rc = opt_in_smem((const void *)wgrad_partial_kernel, sm)) != DEER_OK) return rc;
         int outs = n3 * (wa.K + 1);
         dim3 grid(P, (outs + 255) / 256);
-        wgrad_partial_kernel<<<grid, 256, sm, st>>>(wa);
-        DEER_CHECK_LAUNCH("wgrad_partial_kernel");
-        wgrad_final_kernel<<<(outs + 255) / 256, 256, 0, st>>>(w.partial, P, n3, wa.K,
+        DEER_KERNEL("wgrad_partial_kernel", st, wgrad_partial_kernel<<<grid, 256, sm, st>>>(wa));
+        DEER_KERNEL("wgrad_final_kernel", st, wgrad_final_kernel<<<(outs + 255) / 256, 256, 0, st>>>(w.partial, P, n3, wa.K,
                                                                 side == 0 ? g->dW_i : g->dW_h,
-                                                                side == 0 ? g->db_i : g->db_h);
-        DEER_CHECK_LAUNCH("wgrad_final_kernel");
+                                                                side == 0 ? g->db_i : g->db_h));
     }
     if (dx) {
         size_t total = N * (size_t)m;
-        vjp_dx_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w.dGi, p->W_i, dx, N, m, n3);
-        DEER_CHECK_LAUNCH("vjp_dx_kernel");
+        DEER_KERNEL("vjp_dx_kernel", st, vjp_dx_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w.dGi, p->W_i, dx, N, m, n3));
     }
     if (dy0) {
-        vjp_dy0_kernel<<<(B * n + 127) / 128, 128, 0, st>>>(w.J, w.lam, dy0, B, T, n);
-        DEER_CHECK_LAUNCH("vjp_dy0_kernel");
+        DEER_KERNEL("vjp_dy0_kernel", st, vjp_dy0_kernel<<<(B * n + 127) / 128, 128, 0, st>>>(w.J, w.lam, dy0, B, T, n));
     }
     return DEER_OK;
 }
@@ -441,14 +457,11 @@ int deer_gru_classifier_step(const deer_gru_params *l1, const deer_gru_params *l
     if (s2 < 0) return s2;
     if (iters) { iters[0] = it[0]; iters[1] = it[1]; }
     int seg_len = (T + POOL_SEGS - 1) / POOL_SEGS;
-    pool_partial_kernel<<<dim3(POOL_SEGS, B), n, 0, st>>>(w.y2, T, n, seg_len, w.pool_partial);
-    DEER_CHECK_LAUNCH("pool_partial_kernel");
-    head_kernel<<<1, 256, 0, st>>>(w.pool_partial, POOL_SEGS, B, T, n, ncls, W_o, b_o, labels,
-                                   w.pooled, w.dlog, w.gpool, dW_o, db_o, w.loss);
-    DEER_CHECK_LAUNCH("head_kernel");
+    DEER_KERNEL("pool_partial_kernel", st, pool_partial_kernel<<<dim3(POOL_SEGS, B), n, 0, st>>>(w.y2, T, n, seg_len, w.pool_partial));
+    DEER_KERNEL("head_kernel", st, head_kernel<<<1, 256, 0, st>>>(w.pool_partial, POOL_SEGS, B, T, n, ncls, W_o, b_o, labels,
+                                   w.pooled, w.dlog, w.gpool, dW_o, db_o, w.loss));
     size_t total = N * n;
-    broadcast_gy_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w.gpool, w.gyA, total, T, n);
-    DEER_CHECK_LAUNCH("broadcast_gy_kernel");
+    DEER_KERNEL("broadcast_gy_kernel", st, broadcast_gy_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w.gpool, w.gyA, total, T, n));
     // zero states again (gyB is about to be overwritten by dx of layer 2): use pooled' neighbour
     float *zero1 = w.pool_partial;   // >= B*n floats, no longer needed
     DEER_CHECK_CUDA(cudaMemsetAsync(zero1, 0, (size_t)B * n * sizeof(float), st), "memset y0");
@@ -481,5 +494,40 @@ const char *deer_status_string(int s)
 const char *deer_last_error(void) { return t_err; }
 
 long long deer_launch_count(void) { return g_launches.load(); }
+
+void deer_profile_enable(int on)
+{
+    g_prof_on.store(on != 0);
+}
+
+size_t deer_profile_read(char *buf, size_t cap)
+{
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    std::map<std::string, std::pair<long, double>> acc;
+    std::vector<std::string> order;
+    for (auto &r : g_prof) {
+        float ms = 0.0f;
+        cudaEventSynchronize(r.e1);
+        cudaEventElapsedTime(&ms, r.e0, r.e1);
+        cudaEventDestroy(r.e0);
+        cudaEventDestroy(r.e1);
+        if (!acc.count(r.name)) order.push_back(r.name);
+        acc[r.name].first += 1;
+        acc[r.name].second += ms;
+    }
+    g_prof.clear();
+    std::string out;
+    char line[160];
+    for (auto &k : order) {
+        snprintf(line, sizeof(line), "%s %ld %.6f\n", k.c_str(), acc[k].first, acc[k].second);
+        out += line;
+    }
+    if (buf && cap) {
+        size_t c = out.size() < cap - 1 ? out.size() : cap - 1;
+        memcpy(buf, out.data(), c);
+        buf[c] = 0;
+    }
+    return out.size();
+}
 
 }  // extern "C"
