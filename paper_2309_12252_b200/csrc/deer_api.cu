@@ -11,6 +11,7 @@
 
 #include "common.cuh"
 #include "kernels_generic.cuh"
+#include "scan_onepass.cuh"
 
 namespace deer {
 
@@ -67,7 +68,19 @@ static int gen_chunk_len(int T)
 struct ScanWs {
     float *carA, *carB, *starts;
     int L, nch;
+    OnePassWs op;        // single-pass path (n in {1,2,4,8}); op.nch == 0 when not applicable
 };
+
+static int onepass_tile_len(int n)
+{
+    switch (n) {
+    case 1: return OnePass<1>::L;
+    case 2: return OnePass<2>::L;
+    case 4: return OnePass<4>::L;
+    case 8: return OnePass<8>::L;
+    default: return 0;
+    }
+}
 
 static ScanWs carve_scan(Carver &cv, int B, int T, int n)
 {
@@ -77,7 +90,73 @@ static ScanWs carve_scan(Carver &cv, int B, int T, int n)
     w.carA = cv.take<float>((size_t)B * w.nch * n * n);
     w.carB = cv.take<float>((size_t)B * w.nch * n);
     w.starts = cv.take<float>((size_t)B * w.nch * n);
+    w.op = OnePassWs{};
+    int L1 = onepass_tile_len(n);
+    if (L1) {
+        w.op.nch = (T + L1 - 1) / L1;
+        size_t tiles = (size_t)B * w.op.nch;
+        w.op.flags = cv.take<unsigned>(tiles);
+        w.op.aggs = cv.take<float>(tiles * (n * n + n));
+        w.op.incl = cv.take<float>(tiles * n);
+    }
     return w;
+}
+
+static int g_num_sms = 0;
+static int num_sms()
+{
+    if (!g_num_sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (g_num_sms <= 0) g_num_sms = 148;
+    }
+    return g_num_sms;
+}
+
+template <int N, bool REV>
+static int launch_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
+{
+    using C = OnePass<N>;
+    static int occ = 0;
+    auto kern = scan_onepass_kernel<N, REV>;
+    if (!occ) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(onepass)"); return DEER_ERR_CUDA; }
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, C::THREADS, C::SMEM);
+        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(onepass)"); return DEER_ERR_CUDA; }
+        occ = o;
+    }
+    size_t tiles = (size_t)a.B * w.nch;
+    size_t resident = (size_t)num_sms() * occ;
+    unsigned grid = (unsigned)(tiles < resident ? tiles : resident);
+    int Wd = (int)(grid / (unsigned)a.B);
+    if (Wd < 1) Wd = 1;
+    if (Wd > 32) Wd = 32;
+    if (Wd > w.nch) Wd = w.nch;
+    w.Wd = Wd;
+    w.nwin = (w.nch + Wd - 1) / Wd;
+    w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
+    DEER_CHECK_CUDA(cudaMemsetAsync(w.flags, 0, tiles * sizeof(unsigned), st), "memset flags");
+    DEER_CHECK_CUDA(cudaMemsetAsync(&a.st->tile_counter, 0, sizeof(unsigned), st), "memset counter");
+    DEER_KERNEL("scan_onepass_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
+    return DEER_OK;
+}
+
+static int scan_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
+{
+    switch (a.n * 2 + (a.reverse ? 1 : 0)) {
+    case 2: return launch_onepass<1, false>(a, w, st);
+    case 3: return launch_onepass<1, true>(a, w, st);
+    case 4: return launch_onepass<2, false>(a, w, st);
+    case 5: return launch_onepass<2, true>(a, w, st);
+    case 8: return launch_onepass<4, false>(a, w, st);
+    case 9: return launch_onepass<4, true>(a, w, st);
+    case 16: return launch_onepass<8, false>(a, w, st);
+    case 17: return launch_onepass<8, true>(a, w, st);
+    default: return DEER_ERR_UNSUPPORTED_N;
+    }
 }
 
 static int opt_in_smem(const void *fn, size_t bytes)
@@ -106,9 +185,9 @@ static int scan_generic(ScanArgs a, cudaStream_t st)
     return DEER_OK;
 }
 
-static int run_scan(ScanArgs a, int flags, cudaStream_t st)
+static int run_scan(ScanArgs a, const ScanWs &w, int flags, cudaStream_t st)
 {
-    (void)flags;
+    if (!(flags & DEER_FLAG_GENERIC) && w.op.nch > 0) return scan_onepass(a, w.op, st);
     return scan_generic(a, st);
 }
 
@@ -259,7 +338,7 @@ static int linrec_scan_impl(const float *J, const float *b, const float *y0, int
     a.L = w.scan.L; a.nch = w.scan.nch;
     a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
     a.st = w.st;
-    return run_scan(a, flags, st);
+    return run_scan(a, w.scan, flags, st);
 }
 
 static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *y0, int B, int T,
@@ -290,7 +369,7 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
         a.L = w.scan.L; a.nch = w.scan.nch;
         a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
         a.st = w.st;
-        if ((rc = run_scan(a, flags, st)) != DEER_OK) return rc;
+        if ((rc = run_scan(a, w.scan, flags, st)) != DEER_OK) return rc;
         unsigned bits = 0;
         DEER_CHECK_CUDA(cudaMemcpyAsync(&bits, &w.st->err_bits, sizeof(unsigned),
                                         cudaMemcpyDeviceToHost, st), "read err");
@@ -330,7 +409,7 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
     a.L = w.scan.L; a.nch = w.scan.nch;
     a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
     a.st = w.st;
-    if ((rc = run_scan(a, flags, st)) != DEER_OK) return rc;
+    if ((rc = run_scan(a, w.scan, flags, st)) != DEER_OK) return rc;
 
     {
         VjpArgs v{p->W_h, p->b_h, w.u, y, y0, w.lam, w.dGi, w.dGh, B, T, n};

@@ -36,7 +36,8 @@ def rel_inf(a, b):
 SCAN_CASES = [  # (n, B, T)
     (1, 3, 1), (1, 2, 2), (1, 4, 4097), (2, 3, 1000), (3, 2, 257), (4, 1, 1000), (4, 5, 2049),
     (5, 2, 130), (8, 2, 1), (8, 3, 2), (8, 16, 1111), (8, 1, 5000), (16, 3, 515), (32, 2, 300),
-    (64, 2, 70), (7, 1, 63),
+    (64, 2, 70), (7, 1, 63), (1, 3, 20001), (1, 1, 40000), (2, 2, 6001), (2, 3, 1001), (4, 1, 10000),
+    (8, 2, 193), (8, 2, 192), (8, 5, 191), (4, 3, 769),
 ]
 
 
