@@ -178,8 +178,45 @@ def read_profile(bd):
     return parse_profile(buf.value.decode())
 
 
+def run_scan_only(args):
+    """Stand-alone linear-recurrence scan at the given size: prints one JSON line."""
+    import torch
+    from paper_2309_12252_b200 import binding as bd
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    n, B, T = args.n, args.B, args.T
+    g = torch.Generator(device=device); g.manual_seed(0)
+    J = (torch.rand((B, T, n, n), device=device, generator=g) * 2 - 1) * (0.9 / n)
+    bb = torch.randn((B, T, n), device=device, generator=g)
+    yy = torch.empty_like(bb)
+    ws = bd.alloc_workspace(bd.DEER_OP_SCAN, B, T, n, 1, args.flags, device)
+    stream = torch.cuda.current_stream()
+    for _ in range(max(args.warmup, 1)):
+        bd.deer_linrec_scan(J, bb, None, bool(args.reverse), yy, ws, args.flags, stream)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    for a, b in ev:
+        a.record(stream)
+        bd.deer_linrec_scan(J, bb, None, bool(args.reverse), yy, ws, args.flags, stream)
+        b.record(stream)
+    torch.cuda.synchronize()
+    ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+    pk = peaks()
+    ach = scan_bytes_per_position(n) * B * T / (ms * 1e-3) / 1e9
+    print(json.dumps(dict(mode="scan", n=n, B=B, T=T, reverse=int(args.reverse), flags=args.flags, ms=ms,
+                          positions_per_s=B * T / (ms * 1e-3), achieved_gbs=ach, peak_gbs=pk["hbm_gbs"],
+                          frac=ach / pk["hbm_gbs"], peak_source=pk["source"],
+                          input_mb=(n * n + n) * 4 * B * T / 1e6)))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--mode", default="step", choices=["step", "scan"])
+    ap.add_argument("--n", type=int, default=8)
+    ap.add_argument("--B", type=int, default=16)
+    ap.add_argument("--T", type=int, default=1_000_000)
+    ap.add_argument("--reverse", type=int, default=0)
+    ap.add_argument("--flags", type=int, default=0)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
@@ -189,6 +226,9 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.mode == "scan":
+        run_scan_only(args)
         return
 
     import torch

@@ -55,7 +55,8 @@ struct StatusBlock {
     int iters;           // bodies executed so far (device-side loop control)
     int done;            // 1 once the loop condition failed
     unsigned tile_counter;  // dynamic tile id for the single-pass scan
-    unsigned pad[59];
+    unsigned role_counter;  // role tickets of the single-pass scan (first ones: resolvers)
+    unsigned pad[58];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is one 256-byte line");
 

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <stdio.h>
 #include <string.h>
+#include <stdlib.h>
 
 #include <map>
 #include <mutex>
@@ -97,7 +98,7 @@ static ScanWs carve_scan(Carver &cv, int B, int T, int n)
         size_t tiles = (size_t)B * w.op.nch;
         w.op.flags = cv.take<unsigned>(tiles);
         w.op.aggs = cv.take<float>(tiles * (n * n + n));
-        w.op.incl = cv.take<float>(tiles * n);
+        w.op.starts = cv.take<float>(tiles * n);
     }
     return w;
 }
@@ -130,16 +131,22 @@ static int launch_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
     }
     size_t tiles = (size_t)a.B * w.nch;
     size_t resident = (size_t)num_sms() * occ;
-    unsigned grid = (unsigned)(tiles < resident ? tiles : resident);
-    int Wd = (int)(grid / (unsigned)a.B);
-    if (Wd < 1) Wd = 1;
-    if (Wd > 32) Wd = 32;
+    // resolver CTAs: one warp per sequence up to 8 CTAs, then several sequences per warp
+    int R = (a.B + C::WARPS - 1) / C::WARPS;
+    if (R > 8) R = 8;
+    const int per_warp_cap = C::WARPS * C::MAX_SEQ_PER_WARP;
+    if ((a.B + per_warp_cap - 1) / per_warp_cap > R) R = (a.B + per_warp_cap - 1) / per_warp_cap;
+    w.resolvers = R;
+    size_t want = tiles + (size_t)R;
+    unsigned grid = (unsigned)(want < resident ? want : resident);
+    if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
+    int Wd = 8;
     if (Wd > w.nch) Wd = w.nch;
     w.Wd = Wd;
     w.nwin = (w.nch + Wd - 1) / Wd;
     w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
     DEER_CHECK_CUDA(cudaMemsetAsync(w.flags, 0, tiles * sizeof(unsigned), st), "memset flags");
-    DEER_CHECK_CUDA(cudaMemsetAsync(&a.st->tile_counter, 0, sizeof(unsigned), st), "memset counter");
+    DEER_CHECK_CUDA(cudaMemsetAsync(&a.st->tile_counter, 0, 2 * sizeof(unsigned), st), "memset counters");
     DEER_KERNEL("scan_onepass_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
     return DEER_OK;
 }
