@@ -98,7 +98,7 @@ static ScanWs carve_scan(Carver &cv, int B, int T, int n)
         size_t tiles = (size_t)B * w.op.nch;
         w.op.flags = cv.take<unsigned>(tiles);
         w.op.aggs = cv.take<float>(tiles * (n * n + n));
-        w.op.starts = cv.take<float>(tiles * n);
+        w.op.starts = cv.take<unsigned long long>(tiles * n);
     }
     return w;
 }
@@ -141,11 +141,13 @@ static int launch_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
     unsigned grid = (unsigned)(want < resident ? want : resident);
     if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
     int Wd = 8;
+    { const char *d = getenv("DEER_DEBUG"); w.debug = d ? atoi(d) : 0; if (w.debug >> 8) Wd = w.debug >> 8; }
     if (Wd > w.nch) Wd = w.nch;
     w.Wd = Wd;
     w.nwin = (w.nch + Wd - 1) / Wd;
     w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
     DEER_CHECK_CUDA(cudaMemsetAsync(w.flags, 0, tiles * sizeof(unsigned), st), "memset flags");
+    DEER_CHECK_CUDA(cudaMemsetAsync(w.starts, 0, tiles * N * sizeof(unsigned long long), st), "memset starts");
     DEER_CHECK_CUDA(cudaMemsetAsync(&a.st->tile_counter, 0, 2 * sizeof(unsigned), st), "memset counters");
     DEER_KERNEL("scan_onepass_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
     return DEER_OK;
@@ -194,7 +196,8 @@ static int scan_generic(ScanArgs a, cudaStream_t st)
 
 static int run_scan(ScanArgs a, const ScanWs &w, int flags, cudaStream_t st)
 {
-    if (!(flags & DEER_FLAG_GENERIC) && w.op.nch > 0) return scan_onepass(a, w.op, st);
+    const bool aligned = (((uintptr_t)a.J | (uintptr_t)a.b | (uintptr_t)a.y) & 15) == 0;
+    if (!(flags & DEER_FLAG_GENERIC) && w.op.nch > 0 && aligned) return scan_onepass(a, w.op, st);
     return scan_generic(a, st);
 }
 

@@ -9,28 +9,28 @@
 //     entering states are produced by resolver warps (a few CTAs that took the
 //     first role tickets) which walk each sequence's published aggregates in
 //     order.  Workers therefore hold no data while a dependency is in flight.
-//   * Tiles are staged in shared memory by bulk asynchronous copies
-//     (cp.async.bulk + mbarrier).  The data of the tile that will be taken one
-//     grid-round later is prefetched into L2 (cp.async.bulk.prefetch.L2), so
-//     HBM stays busy while the SMs compute.
-//   * A chain is LPC lanes that own S consecutive positions.  Each lane keeps
-//     COLS = n / LPC columns of the running product A (and the whole vector
-//     beta, redundantly) in registers and multiplies the next J_t, broadcast
-//     from shared memory, onto them:  (A, beta) <- (J_t A, J_t beta + b_t).
-//   * Bank conflicts: for n >= 4 every chain run is copied on its own and
-//     padded by 16 bytes, which makes the run stride odd in 16-byte units; for
-//     n <= 2 the tile is dense and S is chosen odd (n = 2) or S/4 odd (n = 1,
-//     processed four positions per 128-bit load).
-//   * Chain aggregates are combined per warp and per tile in shared memory
-//     and kept there (a small queue of pending tiles) for the B item.
-//   * Roles and tile ids are handed out by atomic counters to running CTAs
-//     only, and a tile's B item depends only on A items of lower ids, which
-//     their owners execute immediately after claiming: no co-residency
-//     assumption is needed for progress.  Every wait is bounded all the same:
-//     on expiry the kernel raises FLAG_TIMEOUT and all CTAs drain.
-//   * In the B item the tile is replayed from its entering state (matrix-
-//     vector work only), y overwrites b in shared memory and is streamed out
-//     with coalesced stores fused with the max |y - y_old| reduction.
+//   * Chains.  A chain is S consecutive positions.  n <= 4: one thread per
+//     chain keeps the whole running aggregate (A, beta) in registers,
+//     (A, beta) <- (J_t A, J_t beta + b_t), and the chain aggregates of a warp
+//     and of the CTA are combined by warp-shuffle scans.  n = 8: four lanes per
+//     chain, each with two columns of A (beta redundantly); chain aggregates
+//     are combined per warp and per CTA through shared memory.
+//   * Staging and bank conflicts.  n <= 2: the tile is dense in shared memory,
+//     brought in by one bulk copy (cp.async.bulk + mbarrier), and S is chosen
+//     odd (n = 2) or S/4 odd (n = 1, four positions per 128-bit load).  n >= 4:
+//     every chain run is padded by 16 bytes so that the stride between the
+//     chains of a warp is odd in 16-byte units; n = 4 stages with per-thread
+//     16-byte cp.async copies, n = 8 with one bulk copy per chain run.
+//   * Protocol.  Roles and tile ids are handed out by atomic counters to
+//     running CTAs only, and a tile's B item depends only on A items of lower
+//     ids, which their owners execute immediately after claiming: no
+//     co-residency assumption is needed for progress.  Aggregates are
+//     published with a release flag; entering states travel as 64-bit
+//     {value, flag} words, so reading one needs a single round trip and no
+//     fence.  Every wait is bounded: on expiry the kernel raises FLAG_TIMEOUT
+//     and all CTAs drain.
+//   * In the B item y overwrites b in shared memory and is streamed out with
+//     coalesced stores fused with the max |y - y_old| reduction.
 //
 // Reverse scans (the adjoint) use the same kernel with reversed indexing and
 // transposed register access.
@@ -40,36 +40,40 @@
 namespace deer {
 
 template <int N> struct OnePass {
-    static constexpr int LPC = (N >= 4) ? 4 : N;       // lanes per chain
-    static constexpr int COLS = N / LPC;               // columns of A per lane
-    static constexpr int S = (N == 8) ? 5 : (N == 4) ? 24 : (N == 2) ? 39 : 60;   // positions per chain
-    static constexpr int PAD = (N >= 4) ? 4 : 0;       // floats of padding after each chain run
-    static constexpr int THREADS = 128;
+    static constexpr int LPC = (N == 8) ? 4 : 1;       // lanes per chain
+    static constexpr int COLS = N / LPC;               // columns of A per lane (n = 8 path)
+    static constexpr int S = (N == 8) ? 5 : (N == 4) ? 5 : (N == 2) ? 9 : 28;   // positions per chain
+    static constexpr int THREADS = (N >= 4) ? 128 : 256;
     static constexpr int WARPS = THREADS / 32;
     static constexpr int CHAINS = THREADS / LPC;
     static constexpr int CPW = CHAINS / WARPS;         // chains per warp
     static constexpr int L = CHAINS * S;               // positions per tile
-    static constexpr int JRUN = S * N * N + PAD;       // floats per chain run of J
-    static constexpr int BRUN = S * N + PAD;           // floats per chain run of b / y
+    static constexpr bool PADDED = N >= 4;             // run-padded layout
+    static constexpr int JRUN = S * N * N + (PADDED ? 4 : 0);        // floats per chain run of J
+    static constexpr int BRUN = S * N + ((N == 8) ? 4 : 0);          // floats per chain run of b / y
+    static constexpr int JBUF = CHAINS * JRUN, BBUF = CHAINS * BRUN;
     static constexpr int AGG = N * N + N;              // floats of one aggregate (A row-major, then beta)
-    static constexpr int Q = 2;                        // pending tiles (A done, B not yet) per CTA
-    static constexpr int PEND = (CHAINS + WARPS) * AGG; // chain + warp aggregates kept per pending tile
-    static constexpr int SM_FLOATS = CHAINS * JRUN + CHAINS * BRUN + Q * PEND + WARPS * 2 * AGG + AGG +
-                                     CHAINS * N + WARPS * N + N + 4;
+    static constexpr int Q = (N == 8) ? 2 : 3;         // pending tiles (A scheduled, B not yet) per CTA
+    // kept per pending tile: n = 8: chain aggregates + warp aggregates;
+    //                        n <= 4: exclusive chain prefixes (within the warp) + exclusive warp prefixes
+    static constexpr int PEND = (CHAINS + WARPS) * AGG;
+    static constexpr int SM_FLOATS = JBUF + BBUF + Q * PEND + WARPS * 2 * AGG + AGG + CHAINS * N + WARPS * N + N + 4;
+    static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 64 + 128;
     static constexpr int MAX_SEQ_PER_WARP = 8;         // sequences one resolver warp can serve
-    static_assert(32 * AGG <= (CHAINS * JRUN) / WARPS, "resolver staging must fit the tile buffer");
-    static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 64;
-    static_assert(N == 1 ? ((S / 4) % 2 == 1 && S % 4 == 0) : N == 2 ? (S % 2 == 1)
-                  : ((JRUN / 4) % 2 == 1 && (BRUN / 4) % 2 == 1), "chain stride must avoid bank conflicts");
+    static_assert(32 * AGG <= JBUF / WARPS, "resolver staging must fit the tile buffer");
+    // the chains a warp reads together must fall in distinct banks: chain stride odd in 16-byte
+    // units (n = 1 reads four positions per load, so S/4 must be odd)
+    static_assert(N == 1 ? ((S / 4) % 2 == 1 && S % 4 == 0) : ((JRUN / 4) % 2 == 1), "chain stride");
 };
 
 struct OnePassWs {
-    unsigned *flags;     // [B*nch]   0 = nothing, 1 = aggregate published, 2 = entering state published
-    float *aggs;         // [B*nch][n*n+n]
-    float *starts;       // [B*nch][n]  state entering the tile
-    int nch, Wd, nwin;   // tiles per sequence, tiles per sequence per window, windows
+    unsigned *flags;              // [B*nch]  1 once the tile aggregate is published
+    float *aggs;                  // [B*nch][n*n+n]
+    unsigned long long *starts;   // [B*nch][n]  state entering the tile as {flag << 32 | float bits}
+    int nch, Wd, nwin;            // tiles per sequence, tiles per sequence per window, windows
     unsigned total_ids;
-    int resolvers;       // CTAs that take the resolver role
+    int resolvers;                // CTAs that take the resolver role
+    int debug;                    // experiment switches (0 in production)
 };
 
 // ---------------------------------------------------------------- small PTX helpers
@@ -100,10 +104,14 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-__device__ __forceinline__ void bulk_prefetch_l2(const void *src, unsigned bytes)
+// 16-byte asynchronous copy global -> shared (per thread; bypasses L1)
+__device__ __forceinline__ void cp_async16(void *dst, const void *src)
 {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
+
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_0() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void fence_proxy_async()
 {
@@ -162,42 +170,156 @@ __device__ __forceinline__ void matvec_smem(float *out, const float *agg, const 
     __syncwarp();
 }
 
-// Geometry of one tile in the two shared-memory layouts.
-//   padded (n >= 4): run r holds the run's positions in ascending t; scan step q of the
-//                    run sits at local index q (forward) or cnt-1-q (reverse).
-//   dense  (n <= 2): forward: position s0+u at slot u; reverse: ascending t, right-aligned
-//                    in the buffer, so scan offset p = chain*S+q sits at slot L-1-p.
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long *p, unsigned long long v)
+{
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// Geometry of one tile in shared memory.
+//   run-padded (n >= 4): run r (= chain r) holds the run's positions in ascending t; scan step q
+//                        of the run sits at local index q (forward) or cnt-1-q (reverse).
+//   dense (n <= 2):      forward: position s0+u at slot u; reverse: ascending t, right-aligned in
+//                        the buffer, so scan offset p = chain*S+q sits at slot L-1-p (keeps the
+//                        128-bit groups of the n = 1 path aligned).
 template <int N, bool REV> struct TileGeom {
     using C = OnePass<N>;
     int s0, Lt, T;
     __device__ __forceinline__ int run_cnt(int r) const { return min(C::S, max(0, Lt - r * C::S)); }
-    // element slot (in elements) for the dense layout
     __device__ __forceinline__ int dense_slot(int p) const { return REV ? (C::L - 1 - p) : p; }
-    __device__ __forceinline__ int dense_base() const { return REV ? (C::L - Lt) : 0; }   // slot of the lowest t
-    // float offset into sB / sJ(elements * NN) for scan step q of chain `chain`
+    __device__ __forceinline__ int low_slot() const { return (REV && !C::PADDED) ? (C::L - Lt) : 0; }
     __device__ __forceinline__ int b_off(int chain, int q, int cnt) const
     {
-        if constexpr (C::PAD > 0) return chain * C::BRUN + (REV ? cnt - 1 - q : q) * N;
+        if constexpr (C::PADDED) return chain * C::BRUN + (REV ? cnt - 1 - q : q) * N;
         else return dense_slot(chain * C::S + q) * N;
     }
     __device__ __forceinline__ int j_off(int chain, int q, int cnt) const
     {
-        if constexpr (C::PAD > 0) return chain * C::JRUN + (REV ? cnt - 1 - q : q) * N * N;
+        if constexpr (C::PADDED) return chain * C::JRUN + (REV ? cnt - 1 - q : q) * N * N;
         else return dense_slot(chain * C::S + q) * N * N;
     }
-    // float offset into sB of component i at ascending-t index u of the tile
+    // run and local index of ascending-t index u of the tile (run-padded layout)
+    __device__ __forceinline__ void locate(int u, int &r, int &li) const
+    {
+        if (!REV) { r = u / C::S; li = u - r * C::S; }
+        else { const int ps = Lt - 1 - u; r = ps / C::S; li = run_cnt(r) - 1 - (ps - r * C::S); }
+    }
+    // float offset into sB of component i at ascending-t index u
     __device__ __forceinline__ int out_off(int u, int i) const
     {
-        if constexpr (C::PAD > 0) {
-            if (!REV) { const int r = u / C::S; return r * C::BRUN + (u - r * C::S) * N + i; }
-            const int ps = Lt - 1 - u, r = ps / C::S, q = ps % C::S;
-            return r * C::BRUN + (run_cnt(r) - 1 - q) * N + i;
-        } else {
-            return (dense_base() + u) * N + i;
-        }
+        if constexpr (C::PADDED) { int r, li; locate(u, r, li); return r * C::BRUN + li * N + i; }
+        else return (low_slot() + u) * N + i;
+    }
+    // float offset into sJ of the matrix at ascending index u of the tile's J range
+    __device__ __forceinline__ int jmat_off(int u) const
+    {
+        if constexpr (C::PADDED) { int r, li; locate(u, r, li); return r * C::JRUN + li * N * N; }
+        else return (low_slot() + u) * N * N;
     }
     __device__ __forceinline__ size_t t_lo() const { return REV ? (size_t)(T - s0 - Lt) : (size_t)s0; }
 };
+
+// ---- n <= 4: one thread per chain; aggregates live in registers and are combined by warp shuffles
+template <int N> struct RegAgg { float A[N][N]; float be[N]; };
+
+template <int N> __device__ __forceinline__ void ragg_identity(RegAgg<N> &r)
+{
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        r.be[i] = 0.0f;
+#pragma unroll
+        for (int j = 0; j < N; ++j) r.A[i][j] = (i == j) ? 1.0f : 0.0f;
+    }
+}
+
+// r <- later o r
+template <int N> __device__ __forceinline__ void ragg_push(RegAgg<N> &r, const float (&M)[N][N], const float (&b)[N])
+{
+    RegAgg<N> o;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        o.be[i] = b[i];
+#pragma unroll
+        for (int k = 0; k < N; ++k) o.be[i] = fmaf(M[i][k], r.be[k], o.be[i]);
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            float acc = 0.0f;
+#pragma unroll
+            for (int k = 0; k < N; ++k) acc = fmaf(M[i][k], r.A[k][j], acc);
+            o.A[i][j] = acc;
+        }
+    }
+    r = o;
+}
+
+template <int N> __device__ __forceinline__ RegAgg<N> ragg_shfl_up(const RegAgg<N> &r, int d)
+{
+    RegAgg<N> o;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        o.be[i] = __shfl_up_sync(0xffffffffu, r.be[i], d);
+#pragma unroll
+        for (int j = 0; j < N; ++j) o.A[i][j] = __shfl_up_sync(0xffffffffu, r.A[i][j], d);
+    }
+    return o;
+}
+
+// inclusive scan over the lanes of a warp (lane l ends with agg_l o ... o agg_0); returns the
+// exclusive prefix (identity in lane 0) in `excl`
+template <int N> __device__ __forceinline__ void ragg_warp_scan(RegAgg<N> &r, RegAgg<N> &excl, int lane)
+{
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        RegAgg<N> p = ragg_shfl_up<N>(r, d);
+        if (lane >= d) {
+            RegAgg<N> e = p;            // earlier part
+            ragg_push<N>(e, r.A, r.be);  // e <- r o e
+            r = e;
+        }
+    }
+    excl = ragg_shfl_up<N>(r, 1);
+    if (lane == 0) ragg_identity<N>(excl);
+}
+
+template <int N> __device__ __forceinline__ void ragg_store(float *dst, const RegAgg<N> &r)
+{
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        dst[N * N + i] = r.be[i];
+#pragma unroll
+        for (int j = 0; j < N; ++j) dst[i * N + j] = r.A[i][j];
+    }
+}
+
+template <int N> __device__ __forceinline__ void ragg_load(RegAgg<N> &r, const float *src)
+{
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        r.be[i] = src[N * N + i];
+#pragma unroll
+        for (int j = 0; j < N; ++j) r.A[i][j] = src[i * N + j];
+    }
+}
+
+// y <- A y + beta
+template <int N> __device__ __forceinline__ void ragg_apply(const RegAgg<N> &r, float (&y)[N])
+{
+    float o[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        o[i] = r.be[i];
+#pragma unroll
+        for (int k = 0; k < N; ++k) o[i] = fmaf(r.A[i][k], y[k], o[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) y[i] = o[i];
+}
 
 // Flag polling shared by workers and resolvers: true while the run should go on.
 __device__ __forceinline__ bool keep_spinning(StatusBlock *st, unsigned &spins)
@@ -208,56 +330,85 @@ __device__ __forceinline__ bool keep_spinning(StatusBlock *st, unsigned &spins)
     return true;
 }
 
+constexpr unsigned long long LL_FLAG = 1ull << 32;     // "entering state present" marker
+
 // Resolver role: warp `rw` of `nrw` serves sequences rw, rw + nrw, ...  For each it walks the
 // published tile aggregates in order, Y <- A Y + beta, writing the state entering every tile.
+// The flags of the next window are requested before the current batch is processed, so a batch
+// costs one exposed round trip (the aggregate fetch); Y lives in registers (lane i holds Y[i]).
 template <int N>
-__device__ void resolver_loop(const ScanArgs &a, const OnePassWs &w, float *stage_all, float *ybuf_all,
-                              int rw, int nrw, int lane)
+__device__ void resolver_loop(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
 {
     using C = OnePass<N>;
-    constexpr int AGG = C::AGG;
+    constexpr int AGG = C::AGG, NN = N * N;
     float *stage = stage_all + (threadIdx.x >> 5) * 32 * AGG;
-    float *ybuf = ybuf_all + (threadIdx.x >> 5) * C::MAX_SEQ_PER_WARP * N;
     int nseq = 0;
     int pos[C::MAX_SEQ_PER_WARP];
+    float yv[C::MAX_SEQ_PER_WARP];              // lane i < N: component i of the sequence's running state
+    unsigned fnext[C::MAX_SEQ_PER_WARP];        // prefetched flag of tile pos + lane
 #pragma unroll
     for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
-        pos[k] = 0;
+        pos[k] = 0; yv[k] = 0.0f; fnext[k] = 0u;
         const int s = rw + k * nrw;
         if (s < a.B) {
             nseq = k + 1;
-            if (lane < N) ybuf[k * N + lane] = a.y0 ? a.y0[(size_t)s * N + lane] : 0.0f;
+            if (lane < N && a.y0) yv[k] = a.y0[(size_t)s * N + lane];
+            if (lane < w.nch) fnext[k] = ld_acquire_u32(w.flags + (size_t)s * w.nch + lane);
         }
     }
-    __syncwarp();
     int remaining = nseq;
     unsigned spins = 0;
     while (remaining > 0) {
         bool progressed = false;
-#pragma unroll 1
-        for (int k = 0; k < nseq; ++k) {
+#pragma unroll
+        for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
+            if (k >= nseq) break;
             const int c0 = pos[k];
             if (c0 >= w.nch) continue;
             const int s = rw + k * nrw;
-            unsigned *flags = w.flags + (size_t)s * w.nch;
-            const int j = c0 + lane;
-            const unsigned f = (j < w.nch) ? ld_acquire_u32(flags + j) : 0u;
-            const unsigned m = __ballot_sync(0xffffffffu, f >= 1u);
+            const unsigned *flags = w.flags + (size_t)s * w.nch;
+            const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
             const int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);      // contiguous published aggregates
+            // request the flags of the window that follows (used on the next visit)
+            {
+                const int j = c0 + cnt + lane;
+                fnext[k] = (j < w.nch) ? ld_acquire_u32(flags + j) : 0u;
+            }
             if (cnt == 0) continue;
             progressed = true;
             const float *src = w.aggs + ((size_t)s * w.nch + c0) * AGG;
-            for (int i = lane; i < cnt * AGG; i += 32) stage[i] = __ldcg(src + i);
-            __syncwarp();
-            float *y = ybuf + k * N;
-            float *out = w.starts + ((size_t)s * w.nch + c0) * N;
-            for (int q = 0; q < cnt; ++q) {
-                if (lane < N) out[q * N + lane] = y[lane];
-                matvec_smem<N>(y, stage + q * AGG, y, lane);
+            {   // all loads of a group are issued before the first store needs its value
+                const int total = cnt * AGG;
+                for (int i0 = 0; i0 < total; i0 += 32 * 8) {
+                    float v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        v[u] = (i < total) ? __ldcg(src + i) : 0.0f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        if (i < total) stage[i] = v[u];
+                    }
+                }
             }
-            __threadfence();
             __syncwarp();
-            if (lane < cnt) st_release_u32(flags + c0 + lane, 2u);
+            unsigned long long *out = w.starts + ((size_t)s * w.nch + c0) * N;
+            float y = yv[k];
+            for (int q = 0; q < cnt; ++q) {
+                if (lane < N) st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y));
+                const float *ag = stage + q * AGG;
+                float acc = (lane < N) ? ag[NN + lane] : 0.0f;
+#pragma unroll
+                for (int i = 0; i < N; ++i) {
+                    const float yi = __shfl_sync(0xffffffffu, y, i);
+                    if (lane < N) acc = fmaf(ag[lane * N + i], yi, acc);
+                }
+                y = acc;
+            }
+            yv[k] = y;
+            __syncwarp();
             pos[k] = c0 + cnt;
             if (pos[k] >= w.nch) --remaining;
         }
@@ -271,14 +422,15 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
 {
     using C = OnePass<N>;
     constexpr int LPC = C::LPC, COLS = C::COLS, S = C::S, CHAINS = C::CHAINS, CPW = C::CPW;
-    constexpr int JRUN = C::JRUN, BRUN = C::BRUN, AGG = C::AGG, WARPS = C::WARPS, NN = N * N;
+    constexpr int JRUN = C::JRUN, AGG = C::AGG, WARPS = C::WARPS, NN = N * N;
     constexpr int Q = C::Q, PEND = C::PEND;
-    constexpr bool PADDED = C::PAD > 0;
+    constexpr bool CPASYNC = (N == 4);         // J staged by per-thread 16-byte cp.async
+    constexpr bool RUNBULK = (N == 8);         // J staged by one bulk copy per chain run
 
-    extern __shared__ __align__(16) float smem[];
-    float *sJ = smem;
-    float *sB = sJ + CHAINS * JRUN;
-    float *pend = sB + CHAINS * BRUN;          // Q x { chain aggregates, warp aggregates }
+    extern __shared__ __align__(16) float smem_raw[];
+    float *sJ = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    float *sB = sJ + C::JBUF;
+    float *pend = sB + C::BBUF;                // Q x { chain aggregates / prefixes, warp aggregates / prefixes }
     float *tmp = pend + Q * PEND;
     float *tagg = tmp + WARPS * 2 * AGG;
     float *cstart = tagg + AGG;
@@ -301,7 +453,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     fence_proxy_async();
     __syncthreads();
     if (s_role < w.resolvers) {
-        resolver_loop<N>(a, w, sJ, sB, s_role * WARPS + warp, w.resolvers * WARPS, lane);
+        resolver_loop<N>(a, w, sJ, s_role * WARPS + warp, w.resolvers * WARPS, lane);
         return;
     }
     unsigned phase = 0;
@@ -316,33 +468,36 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         c = (int)(win * (unsigned)w.Wd + j);
         if (c >= w.nch) c = -1;
     };
-    // global ranges of one tile: J elements [j_lo, j_lo + jcnt), b elements [p_lo, p_lo + Lt)
-    auto tile_ranges = [&](int c, int &s0, int &Lt, size_t &p_lo, size_t &j_lo, int &jcnt) {
-        s0 = c * C::L;
-        Lt = min(C::L, T - s0);
-        p_lo = REV ? (size_t)(T - s0 - Lt) : (size_t)s0;
-        j_lo = REV ? p_lo + 1 : p_lo;
-        jcnt = (REV && s0 == 0) ? Lt - 1 : Lt;
-    };
 
-    // pending queue (thread 0 only): tiles whose A item is done
+    // pending queue (thread 0 only): tiles whose A item has run
     int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
     bool exhausted = false;
 
+    const bool trace = (w.debug & 2) && tid == 0 && blockIdx.x == gridDim.x / 2;
+    long long tr[2][5] = {{0, 0, 0, 0, 0}, {0, 0, 0, 0, 0}};
+    long long t_prev = 0;
+    int k_prev = -1;
+
     for (;;) {
         __syncthreads();      // previous item done with shared memory and with the s_* words
+        long long t0 = 0, t1 = 0, t2 = 0, t3 = 0;
+        if (trace) {
+            t0 = clock64();
+            if (k_prev >= 0) { tr[k_prev][3] += t0 - t_prev; tr[k_prev][4] += 1; }
+        }
         if (tid == 0) {
+            // next item: the oldest pending tile's B item as soon as its entering state is
+            // there (or when the queue is full / no tiles are left), otherwise a new tile's A item
             int kind = -1, seq = -1, c = -1, slot = 0;
             bool want_b = false;
             if (q_cnt > 0) {
                 want_b = (q_cnt == Q) || exhausted;
                 if (!want_b)
-                    want_b = ld_acquire_u32(w.flags + (size_t)q_seq[q_head] * w.nch + q_c[q_head]) == 2u;
+                    want_b = ld_relaxed_u64(w.starts + ((size_t)q_seq[q_head] * w.nch + q_c[q_head]) * N) != 0ull;
             }
             if (!want_b && !exhausted) {
-                unsigned id = 0;
                 for (;;) {
-                    id = atomicAdd(&a.st->tile_counter, 1u);
+                    const unsigned id = atomicAdd(&a.st->tile_counter, 1u);
                     if (id >= w.total_ids) { c = -1; break; }
                     decode(id, seq, c);
                     if (c >= 0) break;
@@ -351,20 +506,6 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                     kind = 0;
                     slot = (q_head + q_cnt) % Q;
                     q_seq[slot] = seq; q_c[slot] = c; ++q_cnt;
-                    // warm L2 with the tile that some CTA will take one grid-round from now
-                    if (id + gridDim.x < w.total_ids) {
-                        int pseq, pc;
-                        decode(id + gridDim.x, pseq, pc);
-                        if (pc >= 0) {
-                            int ps0, pLt, pj; size_t pp, pjl;
-                            tile_ranges(pc, ps0, pLt, pp, pjl, pj);
-                            const float *jsrc = a.J + ((size_t)pseq * T + pjl) * NN;
-                            const float *bsrc = a.b + ((size_t)pseq * T + pp) * N;
-                            const unsigned jb = (unsigned)pj * NN * 4u, bb = (unsigned)pLt * N * 4u;
-                            if (jb && ((uintptr_t)jsrc & 15) == 0 && (jb & 15) == 0) bulk_prefetch_l2(jsrc, jb);
-                            if (((uintptr_t)bsrc & 15) == 0 && (bb & 15) == 0) bulk_prefetch_l2(bsrc, bb);
-                        }
-                    }
                 } else {
                     exhausted = true;
                     want_b = q_cnt > 0;
@@ -378,22 +519,34 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         }
         __syncthreads();
         if (s_kind < 0 || s_abort) break;
+        if (trace) t1 = clock64();
         const int kind = s_kind, seq = s_seq, c = s_c;
-        float *agg = pend + s_slot * PEND;          // chain aggregates of this tile
-        float *wagg = agg + CHAINS * AGG;           // warp aggregates of this tile
+        float *agg = pend + s_slot * PEND;          // chain aggregates (n = 8) / exclusive chain prefixes
+        float *wagg = agg + CHAINS * AGG;           // warp aggregates (n = 8) / exclusive warp prefixes
         TileGeom<N, REV> tg;
-        size_t p_lo, j_lo;
-        int jcnt_tile;
-        tile_ranges(c, tg.s0, tg.Lt, p_lo, j_lo, jcnt_tile);
+        tg.s0 = c * C::L;
+        tg.Lt = min(C::L, T - tg.s0);
         tg.T = T;
         const int s0 = tg.s0, Lt = tg.Lt;
+        const size_t p_lo = tg.t_lo();                                  // first b element of the tile
+        const size_t j_lo = REV ? p_lo + 1 : p_lo;                      // first J element of the tile
+        const int jcnt_tile = (REV && s0 == 0) ? Lt - 1 : Lt;           // (reverse: J[T] does not exist)
         const size_t tile_index = (size_t)seq * w.nch + c;
         const float *Jt_src = a.J + ((size_t)seq * T + j_lo) * NN;
         const float *bt_src = a.b + ((size_t)seq * T + p_lo) * N;
 
         // ------------------------------------------------ stage the tile
-        if constexpr (PADDED) {
-            if (warp == 0) {          // one bulk copy per chain run of J (always 16-byte aligned for n >= 4)
+        if constexpr (CPASYNC) {
+            constexpr int PPE = NN / 4;                       // 16-byte pieces per J_t
+            for (int g = tid; g < jcnt_tile * PPE; g += C::THREADS) {
+                const int u = g / PPE, v = g - u * PPE;
+                cp_async16(sJ + tg.jmat_off(u) + v * 4, Jt_src + (size_t)u * NN + v * 4);
+            }
+            for (int g = tid; g < Lt * N / 4; g += C::THREADS)
+                cp_async16(sB + tg.out_off(g * 4 / N, (g * 4) % N), bt_src + g * 4);
+            cp_async_commit();
+        } else if constexpr (RUNBULK) {
+            if (warp == 0) {          // one bulk copy per chain run of J (16-byte aligned for n = 8)
                 fence_proxy_async();
                 unsigned bytes = 0;
 #pragma unroll 1
@@ -410,14 +563,12 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                 for (int r = lane; r < CHAINS; r += 32) {
                     const int cnt = tg.run_cnt(r);
                     if (cnt <= 0) continue;
-                    // ascending-t index of the run's first J element inside the tile's J range
-                    int first = REV ? (Lt - (r * S + cnt)) : r * S;
+                    const int first = REV ? (Lt - (r * S + cnt)) : r * S;     // ascending index of the run's first J
                     int jc = cnt;
                     if (REV && s0 + r * S == 0) jc -= 1;
                     if (jc > 0) bulk_g2s(sJ + r * JRUN, Jt_src + (size_t)first * NN, (unsigned)jc * NN * 4u, bar);
                 }
             }
-            // b: coalesced 128-bit loads by everybody into the padded runs
             for (int g4 = tid; g4 < Lt * N / 4; g4 += C::THREADS) {
                 const int g = 4 * g4;
                 const float4 v = __ldg(reinterpret_cast<const float4 *>(bt_src) + g4);
@@ -425,7 +576,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             }
         } else {
             const unsigned jb = (unsigned)jcnt_tile * NN * 4u, bb = (unsigned)Lt * N * 4u;
-            float *jd = sJ + tg.dense_base() * NN, *bd = sB + tg.dense_base() * N;
+            float *jd = sJ + tg.low_slot() * NN, *bd = sB + tg.low_slot() * N;
             const bool jbulk = jb && ((uintptr_t)Jt_src & 15) == 0 && (jb & 15) == 0 && ((uintptr_t)jd & 15) == 0;
             const bool bbulk = ((uintptr_t)bt_src & 15) == 0 && (bb & 15) == 0 && ((uintptr_t)bd & 15) == 0;
             if (tid == 0) {
@@ -437,23 +588,25 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             if (!jbulk) for (int i = tid; i < jcnt_tile * NN; i += C::THREADS) jd[i] = __ldg(Jt_src + i);
             if (!bbulk) for (int i = tid; i < Lt * N; i += C::THREADS) bd[i] = __ldg(bt_src + i);
         }
-        // B item: while the copies fly, one thread waits for the state entering the tile
-        if (kind == 1 && tid == 32) {
-            const unsigned *fl = w.flags + tile_index;
+        if (trace) t2 = clock64();
+        // B item: while the copies fly, warp 1 fetches the state entering the tile ({value, flag} words)
+        if (kind == 1 && warp == 1) {
+            const unsigned long long *src = w.starts + tile_index * N;
             unsigned spins = 0;
             bool ok = true;
-            while (ld_acquire_u32(fl) != 2u) {
+            for (;;) {
+                const unsigned long long v = (lane < N) ? ld_relaxed_u64(src + lane) : LL_FLAG;
+                if (__all_sync(0xffffffffu, v != 0ull)) {
+                    if (lane < N) ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                    break;
+                }
                 if (!keep_spinning(a.st, spins)) { ok = false; break; }
             }
-            if (ok) {
-                __threadfence();
-#pragma unroll
-                for (int k = 0; k < N; ++k) ystart[k] = __ldcg(w.starts + tile_index * N + k);
-            } else {
-                s_abort = 1;
-            }
+            if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
         }
-        {
+        if constexpr (CPASYNC) {
+            cp_async_wait_0();
+        } else {
             unsigned spins = 0;
             while (!mbar_try_wait(bar, phase)) {
                 if (++spins > (SPIN_LIMIT >> 2)) { atomicOr(&a.st->flags, FLAG_TIMEOUT); s_abort = 1; break; }
@@ -462,10 +615,156 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         }
         __syncthreads();      // plain-copied data, ystart and s_abort visible
         if (s_abort) break;
+        if (trace) {
+            t3 = clock64();
+            tr[kind][0] += t1 - t0; tr[kind][1] += t2 - t1; tr[kind][2] += t3 - t2;
+            t_prev = t3; k_prev = kind;
+        }
 
         const int cnt = tg.run_cnt(chain);
+        if constexpr (LPC == 1) {
+            // ============================================ n <= 4: one thread per chain
+            // one step of the chain: M = J (forward) or J^T (reverse; identity at scan position 0)
+            auto load_step = [&](int q, float (&M)[N][N], float (&bq)[N]) {
+                const float *Je = sJ + tg.j_off(chain, q, cnt);
+                const float *bv = sB + tg.b_off(chain, q, cnt);
+                const bool ident = REV && (s0 + chain * S + q == 0);
+                if constexpr (N == 2) {
+                    const float4 f = *reinterpret_cast<const float4 *>(Je);
+                    const float2 g = *reinterpret_cast<const float2 *>(bv);
+                    M[0][0] = f.x; M[0][1] = REV ? f.z : f.y; M[1][0] = REV ? f.y : f.z; M[1][1] = f.w;
+                    bq[0] = g.x; bq[1] = g.y;
+                } else {
+                    float R[4][4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float4 f = reinterpret_cast<const float4 *>(Je)[i];
+                        R[i][0] = f.x; R[i][1] = f.y; R[i][2] = f.z; R[i][3] = f.w;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) M[i][k] = REV ? R[k][i] : R[i][k];
+                    const float4 g = *reinterpret_cast<const float4 *>(bv);
+                    bq[0] = g.x; bq[1] = g.y; bq[2] = g.z; bq[3] = g.w;
+                }
+                if (ident) {
+#pragma unroll
+                    for (int i = 0; i < N; ++i)
+#pragma unroll
+                        for (int k = 0; k < N; ++k) M[i][k] = (i == k) ? 1.0f : 0.0f;
+                }
+            };
+            if (kind == 0) {
+                RegAgg<N> r;
+                ragg_identity<N>(r);
+                if constexpr (N == 1) {
+#pragma unroll
+                    for (int q4 = 0; q4 < S / 4; ++q4) {
+                        const int p = chain * S + 4 * q4;
+                        const int base = REV ? (C::L - 4 - p) : p;
+                        const float4 j4 = *reinterpret_cast<const float4 *>(sJ + base);
+                        const float4 b4 = *reinterpret_cast<const float4 *>(sB + base);
+                        const float jj[4] = {REV ? j4.w : j4.x, REV ? j4.z : j4.y, REV ? j4.y : j4.z, REV ? j4.x : j4.w};
+                        const float bb[4] = {REV ? b4.w : b4.x, REV ? b4.z : b4.y, REV ? b4.y : b4.z, REV ? b4.x : b4.w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            if (4 * q4 + k < cnt) {
+                                const float jv = (REV && s0 + p + k == 0) ? 1.0f : jj[k];
+                                r.A[0][0] = jv * r.A[0][0];
+                                r.be[0] = fmaf(jv, r.be[0], bb[k]);
+                            }
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < S; ++q) {
+                        if (q < cnt) {
+                            float M[N][N], bq[N];
+                            load_step(q, M, bq);
+                            ragg_push<N>(r, M, bq);
+                        }
+                    }
+                }
+                RegAgg<N> ex;
+                ragg_warp_scan<N>(r, ex, lane);
+                ragg_store<N>(agg + chain * AGG, ex);              // exclusive prefix inside the warp
+                if (lane == 31) ragg_store<N>(tmp + warp * AGG, r);   // warp aggregate
+                __syncthreads();
+                if (warp == 0) {
+                    RegAgg<N> wr;
+                    if (lane < WARPS) ragg_load<N>(wr, tmp + lane * AGG);
+                    else ragg_identity<N>(wr);
+                    RegAgg<N> wex;
+                    ragg_warp_scan<N>(wr, wex, lane);
+                    if (lane < WARPS) ragg_store<N>(wagg + lane * AGG, wex);   // exclusive prefix over warps
+                    if (lane == WARPS - 1) {
+                        ragg_store<N>(w.aggs + tile_index * AGG, wr);           // tile aggregate
+                        __threadfence();
+                        st_release_u32(w.flags + tile_index, 1u);
+                    }
+                }
+                continue;
+            }
+            {
+                float y[N];
+#pragma unroll
+                for (int k = 0; k < N; ++k) y[k] = ystart[k];
+                RegAgg<N> e;
+                ragg_load<N>(e, wagg + warp * AGG);
+                ragg_apply<N>(e, y);
+                ragg_load<N>(e, agg + chain * AGG);
+                ragg_apply<N>(e, y);
+                if constexpr (N == 1) {
+                    float yv = y[0];
+#pragma unroll
+                    for (int q4 = 0; q4 < S / 4; ++q4) {
+                        const int p = chain * S + 4 * q4;
+                        const int base = REV ? (C::L - 4 - p) : p;
+                        const float4 j4 = *reinterpret_cast<const float4 *>(sJ + base);
+                        float4 b4 = *reinterpret_cast<const float4 *>(sB + base);
+                        const float jj[4] = {REV ? j4.w : j4.x, REV ? j4.z : j4.y, REV ? j4.y : j4.z, REV ? j4.x : j4.w};
+                        float bb[4] = {REV ? b4.w : b4.x, REV ? b4.z : b4.y, REV ? b4.y : b4.z, REV ? b4.x : b4.w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            if (4 * q4 + k < cnt) {
+                                const float jv = (REV && s0 + p + k == 0) ? 1.0f : jj[k];
+                                yv = fmaf(jv, yv, bb[k]);
+                                bb[k] = yv;
+                            }
+                        }
+                        if (REV) { b4.w = bb[0]; b4.z = bb[1]; b4.y = bb[2]; b4.x = bb[3]; }
+                        else { b4.x = bb[0]; b4.y = bb[1]; b4.z = bb[2]; b4.w = bb[3]; }
+                        if (4 * q4 < cnt) *reinterpret_cast<float4 *>(sB + base) = b4;
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < S; ++q) {
+                        if (q < cnt) {
+                            float M[N][N], bq[N];
+                            load_step(q, M, bq);
+                            float yn[N];
+#pragma unroll
+                            for (int i = 0; i < N; ++i) {
+                                yn[i] = bq[i];
+#pragma unroll
+                                for (int k = 0; k < N; ++k) yn[i] = fmaf(M[i][k], y[k], yn[i]);
+                            }
+#pragma unroll
+                            for (int i = 0; i < N; ++i) y[i] = yn[i];
+                            float *bv = sB + tg.b_off(chain, q, cnt);
+                            if constexpr (N == 2) *reinterpret_cast<float2 *>(bv) = make_float2(yn[0], yn[1]);
+                            else *reinterpret_cast<float4 *>(bv) = make_float4(yn[0], yn[1], yn[2], yn[3]);
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+        } else {
+        // ================================================ n = 8: four lanes per chain
+        const float *cJ = sJ;
+        float *cB = sB;
         if (kind == 0) {
-            // -------------------------------------------- A item: chain aggregate in registers
             float A[N][COLS], be[N];
 #pragma unroll
             for (int i = 0; i < N; ++i) {
@@ -473,85 +772,57 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
 #pragma unroll
                 for (int cc = 0; cc < COLS; ++cc) A[i][cc] = (i == sub * COLS + cc) ? 1.0f : 0.0f;
             }
-            if constexpr (N == 1) {
-                // four positions per 128-bit load; dense layout, groups are 16-byte aligned
-                float am = 1.0f, bm = 0.0f;
-#pragma unroll 1
-                for (int q4 = 0; q4 < S / 4; ++q4) {
-                    if (4 * q4 >= cnt) break;
-                    const int p = chain * S + 4 * q4;
-                    const int base = REV ? (C::L - 4 - p) : p;
-                    const float4 j4 = *reinterpret_cast<const float4 *>(sJ + base);
-                    const float4 b4 = *reinterpret_cast<const float4 *>(sB + base);
-                    const float jj[4] = {REV ? j4.w : j4.x, REV ? j4.z : j4.y, REV ? j4.y : j4.z, REV ? j4.x : j4.w};
-                    const float bb[4] = {REV ? b4.w : b4.x, REV ? b4.z : b4.y, REV ? b4.y : b4.z, REV ? b4.x : b4.w};
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        if (4 * q4 + k < cnt) {
-                            const float jv = (REV && s0 + p + k == 0) ? 1.0f : jj[k];
-                            am = jv * am;
-                            bm = fmaf(jv, bm, bb[k]);
-                        }
+            for (int q = 0; q < S; ++q) {
+                if (q >= cnt) break;
+                const bool ident = REV && (s0 + chain * S + q == 0);
+                const float *Je = cJ + tg.j_off(chain, q, cnt);
+                const float *bv = cB + tg.b_off(chain, q, cnt);
+                float bq[N];
+#pragma unroll
+                for (int v = 0; v < N / 4; ++v) {
+                    const float4 f = reinterpret_cast<const float4 *>(bv)[v];
+                    bq[4 * v] = f.x; bq[4 * v + 1] = f.y; bq[4 * v + 2] = f.z; bq[4 * v + 3] = f.w;
+                }
+                if (q == 0) {
+                    if (!ident) {
+#pragma unroll
+                        for (int i = 0; i < N; ++i)
+#pragma unroll
+                            for (int cc = 0; cc < COLS; ++cc) {
+                                const int j = sub * COLS + cc;
+                                A[i][cc] = REV ? Je[j * N + i] : Je[i * N + j];
+                            }
+                    }
+#pragma unroll
+                    for (int i = 0; i < N; ++i) be[i] = bq[i];
+                    continue;
+                }
+                float Jr[NN];
+#pragma unroll
+                for (int v = 0; v < NN / 4; ++v) {
+                    const float4 f = reinterpret_cast<const float4 *>(Je)[v];
+                    Jr[4 * v] = f.x; Jr[4 * v + 1] = f.y; Jr[4 * v + 2] = f.z; Jr[4 * v + 3] = f.w;
+                }
+                float An[N][COLS], bn[N];
+#pragma unroll
+                for (int i = 0; i < N; ++i) {
+                    bn[i] = bq[i];
+#pragma unroll
+                    for (int cc = 0; cc < COLS; ++cc) An[i][cc] = 0.0f;
+#pragma unroll
+                    for (int k = 0; k < N; ++k) {
+                        const float m = REV ? Jr[k * N + i] : Jr[i * N + k];
+                        bn[i] = fmaf(m, be[k], bn[i]);
+#pragma unroll
+                        for (int cc = 0; cc < COLS; ++cc) An[i][cc] = fmaf(m, A[k][cc], An[i][cc]);
                     }
                 }
-                A[0][0] = am; be[0] = bm;
-            } else {
-#pragma unroll 1
-                for (int q = 0; q < cnt; ++q) {
-                    const bool ident = REV && (s0 + chain * S + q == 0);
-                    const float *Je = sJ + tg.j_off(chain, q, cnt);
-                    const float *bv = sB + tg.b_off(chain, q, cnt);
-                    float bq[N];
-                    if constexpr (N >= 4) {
 #pragma unroll
-                        for (int v = 0; v < N / 4; ++v) {
-                            const float4 f = reinterpret_cast<const float4 *>(bv)[v];
-                            bq[4 * v] = f.x; bq[4 * v + 1] = f.y; bq[4 * v + 2] = f.z; bq[4 * v + 3] = f.w;
-                        }
-                    } else {
-                        const float2 f = *reinterpret_cast<const float2 *>(bv);
-                        bq[0] = f.x; bq[1] = f.y;
-                    }
-                    if (q == 0) {
-                        if (!ident) {
+                for (int i = 0; i < N; ++i) {
+                    be[i] = bn[i];
 #pragma unroll
-                            for (int i = 0; i < N; ++i)
-#pragma unroll
-                                for (int cc = 0; cc < COLS; ++cc) {
-                                    const int j = sub * COLS + cc;
-                                    A[i][cc] = REV ? Je[j * N + i] : Je[i * N + j];
-                                }
-                        }
-#pragma unroll
-                        for (int i = 0; i < N; ++i) be[i] = bq[i];
-                        continue;
-                    }
-                    float Jr[NN];
-#pragma unroll
-                    for (int v = 0; v < NN / 4; ++v) {
-                        const float4 f = reinterpret_cast<const float4 *>(Je)[v];
-                        Jr[4 * v] = f.x; Jr[4 * v + 1] = f.y; Jr[4 * v + 2] = f.z; Jr[4 * v + 3] = f.w;
-                    }
-                    float An[N][COLS], bn[N];
-#pragma unroll
-                    for (int i = 0; i < N; ++i) {
-                        bn[i] = bq[i];
-#pragma unroll
-                        for (int cc = 0; cc < COLS; ++cc) An[i][cc] = 0.0f;
-#pragma unroll
-                        for (int k = 0; k < N; ++k) {
-                            const float m = REV ? Jr[k * N + i] : Jr[i * N + k];
-                            bn[i] = fmaf(m, be[k], bn[i]);
-#pragma unroll
-                            for (int cc = 0; cc < COLS; ++cc) An[i][cc] = fmaf(m, A[k][cc], An[i][cc]);
-                        }
-                    }
-#pragma unroll
-                    for (int i = 0; i < N; ++i) {
-                        be[i] = bn[i];
-#pragma unroll
-                        for (int cc = 0; cc < COLS; ++cc) A[i][cc] = An[i][cc];
-                    }
+                    for (int cc = 0; cc < COLS; ++cc) A[i][cc] = An[i][cc];
                 }
             }
             {
@@ -567,24 +838,20 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             // warp aggregate, then tile aggregate (warp 0), then publish
             {
                 const float *first = agg + (warp * CPW) * AGG;
-                float *t0 = tmp + warp * 2 * AGG, *t1 = t0 + AGG;
+                float *t0s = tmp + warp * 2 * AGG, *t1s = t0s + AGG;
                 const float *cur = first;
                 for (int k = 1; k < CPW; ++k) {
-                    float *dst = (k == CPW - 1) ? (wagg + warp * AGG) : ((k & 1) ? t0 : t1);
+                    float *dst = (k == CPW - 1) ? (wagg + warp * AGG) : ((k & 1) ? t0s : t1s);
                     combine_smem<N>(dst, agg + (warp * CPW + k) * AGG, cur, lane);
                     cur = dst;
-                }
-                if (CPW == 1) {
-                    for (int o = lane; o < AGG; o += 32) wagg[warp * AGG + o] = first[o];
-                    __syncwarp();
                 }
             }
             __syncthreads();
             if (warp == 0) {
-                float *t0 = tmp, *t1 = tmp + AGG;
+                float *t0s = tmp, *t1s = tmp + AGG;
                 const float *cur = wagg;
                 for (int k = 1; k < WARPS; ++k) {
-                    float *dst = (k == WARPS - 1) ? tagg : ((k & 1) ? t0 : t1);
+                    float *dst = (k == WARPS - 1) ? tagg : ((k & 1) ? t0s : t1s);
                     combine_smem<N>(dst, wagg + k * AGG, cur, lane);
                     cur = dst;
                 }
@@ -597,7 +864,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             continue;
         }
 
-        // ------------------------------------------------ B item: states entering each warp, each chain
+        // B item: states entering each warp, each chain
         if (warp == 0) {
             if (lane < N) wstart[lane] = ystart[lane];
             __syncwarp();
@@ -612,40 +879,17 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             for (int k = 0; k + 1 < CPW; ++k)
                 matvec_smem<N>(cs + (k + 1) * N, agg + (warp * CPW + k) * AGG, cs + k * N, lane);
         }
-
-        // ------------------------------------------------ apply: replay the chain, y overwrites b
-        if constexpr (N == 1) {
-            float yv = cstart[chain];
-#pragma unroll 1
-            for (int q4 = 0; q4 < S / 4; ++q4) {
-                if (4 * q4 >= cnt) break;
-                const int p = chain * S + 4 * q4;
-                const int base = REV ? (C::L - 4 - p) : p;
-                const float4 j4 = *reinterpret_cast<const float4 *>(sJ + base);
-                float4 b4 = *reinterpret_cast<const float4 *>(sB + base);
-                const float jj[4] = {REV ? j4.w : j4.x, REV ? j4.z : j4.y, REV ? j4.y : j4.z, REV ? j4.x : j4.w};
-                float bb[4] = {REV ? b4.w : b4.x, REV ? b4.z : b4.y, REV ? b4.y : b4.z, REV ? b4.x : b4.w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    if (4 * q4 + k < cnt) {
-                        const float jv = (REV && s0 + p + k == 0) ? 1.0f : jj[k];
-                        yv = fmaf(jv, yv, bb[k]);
-                        bb[k] = yv;
-                    }
-                }
-                if (REV) { b4.w = bb[0]; b4.z = bb[1]; b4.y = bb[2]; b4.x = bb[3]; }
-                else { b4.x = bb[0]; b4.y = bb[1]; b4.z = bb[2]; b4.w = bb[3]; }
-                *reinterpret_cast<float4 *>(sB + base) = b4;
-            }
-        } else {
+        // apply: replay the chain, y overwrites b
+        {
             float y[N];
 #pragma unroll
             for (int k = 0; k < N; ++k) y[k] = cstart[chain * N + k];
-#pragma unroll 1
-            for (int q = 0; q < cnt; ++q) {
+#pragma unroll
+            for (int q = 0; q < S; ++q) {
+                if (q >= cnt) break;
                 const bool ident = REV && (s0 + chain * S + q == 0);
-                const float *Je = sJ + tg.j_off(chain, q, cnt);
-                float *bv = sB + tg.b_off(chain, q, cnt);
+                const float *Je = cJ + tg.j_off(chain, q, cnt);
+                float *bv = cB + tg.b_off(chain, q, cnt);
                 float v[COLS];
 #pragma unroll
                 for (int cc = 0; cc < COLS; ++cc) {
@@ -655,16 +899,11 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
 #pragma unroll
                         for (int k = 0; k < N; ++k) if (k == i) acc += y[k];
                     } else if (!REV) {
-                        if constexpr (N >= 4) {
 #pragma unroll
-                            for (int v4 = 0; v4 < N / 4; ++v4) {
-                                const float4 f = reinterpret_cast<const float4 *>(Je + i * N)[v4];
-                                acc = fmaf(f.x, y[4 * v4], acc); acc = fmaf(f.y, y[4 * v4 + 1], acc);
-                                acc = fmaf(f.z, y[4 * v4 + 2], acc); acc = fmaf(f.w, y[4 * v4 + 3], acc);
-                            }
-                        } else {
-#pragma unroll
-                            for (int k = 0; k < N; ++k) acc = fmaf(Je[i * N + k], y[k], acc);
+                        for (int v4 = 0; v4 < N / 4; ++v4) {
+                            const float4 f = reinterpret_cast<const float4 *>(Je + i * N)[v4];
+                            acc = fmaf(f.x, y[4 * v4], acc); acc = fmaf(f.y, y[4 * v4 + 1], acc);
+                            acc = fmaf(f.z, y[4 * v4 + 2], acc); acc = fmaf(f.w, y[4 * v4 + 3], acc);
                         }
                     } else {
 #pragma unroll
@@ -679,6 +918,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             }
         }
         __syncthreads();
+        }
 
         // ------------------------------------------------ stream y out (+ max |y - yold|)
         {
@@ -686,7 +926,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             float *yo = a.y + gbase;
             const float *yold = a.yold ? a.yold + gbase : nullptr;
             const int total = Lt * N;
-            const bool vec = (N >= 4 || (tg.dense_base() * N) % 4 == 0) && (((uintptr_t)yo & 15) == 0) &&
+            const bool vec = (N >= 4 || (tg.low_slot() * N) % 4 == 0) && (((uintptr_t)yo & 15) == 0) &&
                              ((total & 3) == 0) && (!yold || ((uintptr_t)yold & 15) == 0);
             if (vec) {
                 for (int g4 = tid; g4 < total / 4; g4 += C::THREADS) {
@@ -707,6 +947,10 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                 }
             }
         }
+    }
+    if (trace) {
+        for (int k = 0; k < 2; ++k)
+            for (int j = 0; j < 5; ++j) a.st->pad[k * 5 + j] = (unsigned)(tr[k][j] > 0xffffffffll ? 0xffffffffu : tr[k][j]);
     }
     if (a.yold) {
 #pragma unroll
