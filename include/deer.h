@@ -98,6 +98,31 @@ size_t deer_workspace_bytes(int op, int B, int T, int n, int m, int flags);
 int deer_linrec_scan(const float *J, const float *b, const float *y0, int B, int T, int n,
                      int reverse, float *y, void *ws, size_t ws_bytes, int flags, void *stream);
 
+/* The same scan for callers that cannot hand the library a workspace.
+ * (No counterpart in the paper: this exists for integration, not for the method.)
+ * Some hosts of this library may not allocate device memory at the point where
+ * they need a scan: code that runs inside a framework's memory-planned region,
+ * a real-time loop that must not touch the allocator, or a plug-in that is only
+ * given its input and output buffers.  For them this variant takes its scratch
+ * from a fixed array that is part of the library image: DEER_NOALLOC_SCRATCH_BYTES
+ * of device memory, reserved on every GPU that loads the library for as long as
+ * the process lives.  It calls no cudaMalloc / cudaFree and no allocating
+ * routine of any other library.
+ *   - Arguments, layouts and results are those of deer_linrec_scan.
+ *   - Sizes whose scratch (deer_workspace_bytes(DEER_OP_SCAN, ...)) exceeds
+ *     DEER_NOALLOC_SCRATCH_BYTES are refused with DEER_ERR_WORKSPACE and a
+ *     message in deer_last_error(); nothing runs.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the last
+ *     call left in it; the entry point clears the words that must start at zero
+ *     itself.  Two calls that overlap on the GPU (different streams, no ordering
+ *     between them) would race on the array: order them.
+ * Asynchronous on `stream`.  Returns DEER_OK or a negative status. */
+#define DEER_NOALLOC_SCRATCH_BYTES (8u << 20)
+int deer_linrec_scan_noalloc(const float *J, const float *b, const float *y0, int B, int T, int n,
+                             int reverse, float *y, void *stream);
+
 /* Evaluate the GRU over whole sequences with the DEER iteration (Eq. 3 with
  * G = -df/dy, Eq. 5; loop of App. B.1): starting from y = 0 (or the guess in
  * y when DEER_FLAG_WARM_START), repeat { J, f at the shifted guess;

@@ -22,7 +22,8 @@ DEER_ERR_CUDA, DEER_ERR_DEVICE_TIMEOUT = -4, -5
 DEER_OP_EVAL, DEER_OP_SCAN, DEER_OP_VJP, DEER_OP_CLASSIFIER = 0, 1, 2, 3
 DEER_FLAG_WARM_START, DEER_FLAG_GENERIC, DEER_FLAG_MATERIALIZE = 1, 2, 4
 
-EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_gru_eval", "deer_gru_vjp",
+NOALLOC_SCRATCH_BYTES = 8 << 20
+EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc", "deer_gru_eval", "deer_gru_vjp",
            "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count"]
 
 
@@ -52,6 +53,8 @@ def lib():
         vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
         L.deer_linrec_scan.restype = ci
         L.deer_linrec_scan.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, ci, vp]
+        L.deer_linrec_scan_noalloc.restype = ci
+        L.deer_linrec_scan_noalloc.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, vp]
         L.deer_gru_eval.restype = ci
         L.deer_gru_eval.argtypes = [ctypes.POINTER(_Params), vp, vp, ci, ci, cf, ci, vp,
                                     ctypes.POINTER(ci), ctypes.POINTER(cf), vp, vp, sz, ci, vp]
@@ -75,8 +78,10 @@ class DeerError(RuntimeError):
     def __init__(self, status: int):
         self.status = status
         msg = lib().deer_status_string(status).decode()
-        if status == DEER_ERR_CUDA:
-            msg += ": " + lib().deer_last_error().decode()
+        if status in (DEER_ERR_CUDA, DEER_ERR_WORKSPACE):
+            extra = lib().deer_last_error().decode()
+            if extra:
+                msg += ": " + extra
         super().__init__(f"deer status {status}: {msg}")
 
 
@@ -149,6 +154,20 @@ def deer_linrec_scan(J, b, y0=None, reverse=False, y=None, ws=None, flags=0, str
         ws = alloc_workspace(DEER_OP_SCAN, B, T, n, 1, flags, b.device)
     rc = lib().deer_linrec_scan(_ptr(_f32(J)), _ptr(_f32(b)), _ptr(y0), B, T, n, int(bool(reverse)),
                                 _ptr(y), _ptr(ws), ws.numel(), flags, _stream(stream))
+    if check and rc != DEER_OK:
+        raise DeerError(rc)
+    return y if check else (y, rc)
+
+
+def deer_linrec_scan_noalloc(J, b, y0=None, reverse=False, y=None, stream=None, check=True):
+    """deer_linrec_scan for callers that may not allocate: the library's built-in
+    scratch array is used instead of a workspace (see include/deer.h for the limits)."""
+    B, T, n = b.shape
+    assert tuple(J.shape) == (B, T, n, n)
+    if y is None:
+        y = torch.empty_like(b)
+    rc = lib().deer_linrec_scan_noalloc(_ptr(_f32(J)), _ptr(_f32(b)), _ptr(y0), B, T, n, int(bool(reverse)),
+                                        _ptr(y), _stream(stream))
     if check and rc != DEER_OK:
         raise DeerError(rc)
     return y if check else (y, rc)

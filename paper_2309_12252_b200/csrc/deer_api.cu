@@ -342,6 +342,7 @@ static int linrec_scan_impl(const float *J, const float *b, const float *y0, int
     ScanOnlyWs w = carve_scan_only(ws, B, T, n);
     int rc = check_ws(ws, ws_bytes, w.bytes);
     if (rc != DEER_OK) return rc;
+    DEER_CHECK_CUDA(cudaMemsetAsync(w.st, 0, sizeof(StatusBlock), st), "memset status");
     ScanArgs a{};
     a.J = J; a.b = b; a.y0 = y0; a.y = y; a.yold = nullptr;
     a.B = B; a.T = T; a.n = n; a.reverse = reverse ? 1 : 0;
@@ -461,6 +462,30 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
     return DEER_OK;
 }
 
+// ---------------------------------------------------------------- built-in scratch (no-alloc entry point)
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not a device address: the
+// address a kernel can use comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[DEER_NOALLOC_SCRATCH_BYTES];
+
+static std::mutex g_noalloc_mu;
+static void *g_noalloc_ptr[64] = {nullptr};
+
+static int noalloc_scratch_for_current_device(void **out)
+{
+    int dev = -1;
+    DEER_CHECK_CUDA(cudaGetDevice(&dev), "cudaGetDevice");
+    if (dev < 0 || dev >= 64) { snprintf(t_err, sizeof(t_err), "device index %d out of range", dev); return DEER_ERR_CUDA; }
+    std::lock_guard<std::mutex> lk(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+        void *p = nullptr;
+        DEER_CHECK_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch), "cudaGetSymbolAddress(scratch)");
+        if (!p || ((uintptr_t)p & 255) != 0) { snprintf(t_err, sizeof(t_err), "built-in scratch misaligned"); return DEER_ERR_CUDA; }
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return DEER_OK;
+}
+
 }  // namespace deer
 
 using namespace deer;
@@ -563,6 +588,28 @@ int deer_gru_classifier_step(const deer_gru_params *l1, const deer_gru_params *l
     DEER_CHECK_CUDA(cudaMemcpyAsync(loss, w.loss, sizeof(float), cudaMemcpyDeviceToHost, st), "read loss");
     DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
     return s1 > s2 ? s1 : s2;
+}
+
+int deer_linrec_scan_noalloc(const float *J, const float *b, const float *y0, int B, int T, int n,
+                             int reverse, float *y, void *stream)
+{
+    if (!J || !b || !y || B <= 0 || T <= 0 || n <= 0) return DEER_ERR_INVALID_ARG;
+    if (!supported(n, 1)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, n, 1)) return DEER_ERR_INVALID_ARG;
+    const size_t need = carve_scan_only(nullptr, B, T, n).bytes;
+    if (need > sizeof(g_noalloc_scratch)) {
+        snprintf(t_err, sizeof(t_err),
+                 "deer_linrec_scan_noalloc: B=%d T=%d n=%d needs %zu bytes of scratch, the built-in array holds %zu",
+                 B, T, n, need, sizeof(g_noalloc_scratch));
+        return DEER_ERR_WORKSPACE;
+    }
+    void *scratch = nullptr;
+    int rc = noalloc_scratch_for_current_device(&scratch);
+    if (rc != DEER_OK) return rc;
+    // linrec_scan_impl clears what has to start at zero (status block, tile flags, entering-state
+    // words, counters) with stream-ordered memsets on every call; nothing else is read before written
+    return linrec_scan_impl(J, b, y0, B, T, n, reverse, y, scratch, sizeof(g_noalloc_scratch), 0,
+                            (cudaStream_t)stream);
 }
 
 const char *deer_status_string(int s)
