@@ -320,7 +320,7 @@ def main():
     kernels = {k: dict(launches_per_step=v["launches"] / prof_steps, us_per_launch=1e3 * v["total_ms"] / v["launches"],
                        share=v["total_ms"] / tot) for k, v in prof.items()}
     pk = peaks()
-    scan_names = [k for k in prof if ("scan" in k or "reduce" in k or "carry" in k or "apply" in k or "newton" in k)]
+    scan_names = [k for k in prof if ("scan" in k or "reduce" in k or "carry" in k or "apply" in k)]
     scan_ms = sum(prof[k]["total_ms"] for k in scan_names)
     scans = prof_steps * iters
     roofline = None

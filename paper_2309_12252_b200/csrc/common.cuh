@@ -56,7 +56,8 @@ struct StatusBlock {
     int done;            // 1 once the loop condition failed
     unsigned tile_counter;  // dynamic tile id for the single-pass scan
     unsigned role_counter;  // role tickets of the single-pass scan (first ones: resolvers)
-    unsigned pad[58];
+    unsigned err_last_bits; // err of the last executed body
+    unsigned pad[57];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is one 256-byte line");
 
@@ -89,7 +90,15 @@ struct CellArgs {
     float *J;            // [B,T,n,n] out
     float *rhs;          // [B,T,n]   out: f - J y_prev   (nullptr: skip)
     int B, T, n;
+    const StatusBlock *st;   // nullptr, or: skip all work once st->done is set (Newton loop ended)
 };
+
+// Device-side loop control lets the host enqueue Newton bodies ahead of knowing whether they
+// are needed: every kernel of a body returns at once when the loop has already ended.
+__device__ __forceinline__ bool loop_ended(const StatusBlock *st)
+{
+    return st != nullptr && *(volatile const int *)&st->done != 0;
+}
 
 __device__ __forceinline__ float sigmoidf_acc(float a) { return 1.0f / (1.0f + expf(-a)); }
 

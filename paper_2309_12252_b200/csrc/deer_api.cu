@@ -146,9 +146,13 @@ static int launch_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
     w.Wd = Wd;
     w.nwin = (w.nch + Wd - 1) / Wd;
     w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
-    DEER_CHECK_CUDA(cudaMemsetAsync(w.flags, 0, tiles * sizeof(unsigned), st), "memset flags");
-    DEER_CHECK_CUDA(cudaMemsetAsync(w.starts, 0, tiles * N * sizeof(unsigned long long), st), "memset starts");
-    DEER_CHECK_CUDA(cudaMemsetAsync(&a.st->tile_counter, 0, 2 * sizeof(unsigned), st), "memset counters");
+    {
+        size_t words = tiles * (size_t)(N + 1);
+        unsigned pb = (unsigned)((words + 255) / 256);
+        if (pb > 592u) pb = 592u;
+        if (pb < 1u) pb = 1u;
+        DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)N));
+    }
     DEER_KERNEL("scan_onepass_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
     return DEER_OK;
 }
@@ -209,8 +213,29 @@ static int run_proj(const deer_gru_params *p, const float *x, float *u, size_t N
     return DEER_OK;
 }
 
+template <int N> static int launch_cell_small(CellArgs c, cudaStream_t st)
+{
+    const size_t total = (size_t)c.B * c.T;
+    const size_t epb = 256 / N;
+    size_t blocks = (total + epb - 1) / epb;
+    const size_t cap = (size_t)num_sms() * 8;
+    if (blocks > cap) blocks = cap;
+    DEER_KERNEL("cell_small_kernel", st, cell_small_kernel<N><<<(unsigned)blocks, 256, 0, st>>>(c));
+    return DEER_OK;
+}
+
 static int run_cell(CellArgs c, cudaStream_t st)
 {
+    const bool aligned = (((uintptr_t)c.y | (uintptr_t)c.y0 | (uintptr_t)c.J) & 15) == 0;
+    if (aligned) {
+        switch (c.n) {
+        case 1: return launch_cell_small<1>(c, st);
+        case 2: return launch_cell_small<2>(c, st);
+        case 4: return launch_cell_small<4>(c, st);
+        case 8: return launch_cell_small<8>(c, st);
+        default: break;
+        }
+    }
     const int n = c.n;
     size_t sm = sizeof(float) * (3 * n * (n + 1) + 3 * n);
     int rc;
@@ -233,6 +258,7 @@ static bool supported(int n, int m) { return n >= 1 && n <= 64 && m >= 1 && m <=
 // ---------------------------------------------------------------- workspace layouts
 struct EvalWs {
     StatusBlock *st;
+    float *trace;        // [ERR_TRACE_CAP] err after each body (device side of err_trace)
     float *u, *J, *rhs, *yalt;
     ScanWs scan;
     size_t bytes;
@@ -245,6 +271,7 @@ static EvalWs carve_eval(void *ws, int B, int T, int n, int m)
     EvalWs w;
     size_t N = (size_t)B * T;
     w.st = cv.take<StatusBlock>(1);
+    w.trace = cv.take<float>(ERR_TRACE_CAP);
     w.u = cv.take<float>(N * 3 * n);
     w.J = cv.take<float>(N * n * n);
     w.rhs = cv.take<float>(N * n);
@@ -366,37 +393,46 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
         DEER_CHECK_CUDA(cudaMemsetAsync(y, 0, N * n * sizeof(float), st), "memset y");
     if ((rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
 
-    float *cur = y, *nxt = w.yalt;
-    float e = 1e10f;
-    int k = 0;
+    // Newton loop (App. B.1): bodies are enqueued ahead of the convergence test -- the control kernel
+    // at the end of each body decides on the device, and the kernels of bodies past the end return
+    // at once -- so the host only synchronises once per group of bodies.
+    float *buf[2] = {y, w.yalt};
+    int enq = 0, group = 4;
+    StatusBlock hs;
+    for (;;) {
+        int todo = max_iter - enq;
+        if (todo > group) todo = group;
+        for (int j = 0; j < todo; ++j, ++enq) {
+            float *cur = buf[enq & 1], *nxt = buf[(enq + 1) & 1];
+            CellArgs c{p->W_h, p->b_h, w.u, cur, y0, w.J, w.rhs, B, T, n, w.st};
+            if ((rc = run_cell(c, st)) != DEER_OK) return rc;
+            ScanArgs a{};
+            a.J = w.J; a.b = w.rhs; a.y0 = y0; a.y = nxt; a.yold = cur;
+            a.B = B; a.T = T; a.n = n; a.reverse = 0;
+            a.L = w.scan.L; a.nch = w.scan.nch;
+            a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
+            a.st = w.st;
+            if ((rc = run_scan(a, w.scan, flags, st)) != DEER_OK) return rc;
+            DEER_KERNEL("newton_control_kernel", st, newton_control_kernel<<<1, 1, 0, st>>>(w.st, tol, max_iter, w.trace));
+        }
+        DEER_CHECK_CUDA(cudaMemcpyAsync(&hs, w.st, 32, cudaMemcpyDeviceToHost, st), "read status");
+        DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+        if (hs.flags & FLAG_TIMEOUT) return DEER_ERR_DEVICE_TIMEOUT;
+        if (hs.done || enq >= max_iter) break;
+        group = 2;
+    }
+    const int k = hs.iters;
+    float e;
+    memcpy(&e, &hs.err_last_bits, sizeof(float));
+    if (k & 1)
+        DEER_CHECK_CUDA(cudaMemcpyAsync(y, w.yalt, N * n * sizeof(float), cudaMemcpyDeviceToDevice, st), "copy result");
+    if (err_trace && k > 0)
+        DEER_CHECK_CUDA(cudaMemcpyAsync(err_trace, w.trace, sizeof(float) * (size_t)(k < ERR_TRACE_CAP ? k : ERR_TRACE_CAP),
+                                        cudaMemcpyDeviceToHost, st), "read trace");
+    DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
     int status = DEER_OK;
-    while (e > tol && k < max_iter) {
-        CellArgs c{p->W_h, p->b_h, w.u, cur, y0, w.J, w.rhs, B, T, n};
-        if ((rc = run_cell(c, st)) != DEER_OK) return rc;
-        DEER_CHECK_CUDA(cudaMemsetAsync(&w.st->err_bits, 0, sizeof(unsigned), st), "memset err");
-        ScanArgs a{};
-        a.J = w.J; a.b = w.rhs; a.y0 = y0; a.y = nxt; a.yold = cur;
-        a.B = B; a.T = T; a.n = n; a.reverse = 0;
-        a.L = w.scan.L; a.nch = w.scan.nch;
-        a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
-        a.st = w.st;
-        if ((rc = run_scan(a, w.scan, flags, st)) != DEER_OK) return rc;
-        unsigned bits = 0;
-        DEER_CHECK_CUDA(cudaMemcpyAsync(&bits, &w.st->err_bits, sizeof(unsigned),
-                                        cudaMemcpyDeviceToHost, st), "read err");
-        DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
-        memcpy(&e, &bits, sizeof(float));
-        float *tmp = cur; cur = nxt; nxt = tmp;
-        if (err_trace) err_trace[k] = e;
-        ++k;
-        if (!isfinite(e)) { status = DEER_NONFINITE; break; }
-    }
-    if (cur != y) {
-        DEER_CHECK_CUDA(cudaMemcpyAsync(y, cur, N * n * sizeof(float), cudaMemcpyDeviceToDevice, st),
-                        "copy result");
-        DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
-    }
-    if (status == DEER_OK && e > tol && !(tol < 0.0f)) status = DEER_NOT_CONVERGED;
+    if (!isfinite(e)) status = DEER_NONFINITE;
+    else if (e > tol && !(tol < 0.0f)) status = DEER_NOT_CONVERGED;
     if (iters) *iters = k;
     if (err) *err = e;
     return status;
@@ -411,8 +447,9 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
     int rc = check_ws(ws, ws_bytes, w.bytes);
     if (rc != DEER_OK) return rc;
     const size_t N = (size_t)B * T;
+    DEER_CHECK_CUDA(cudaMemsetAsync(w.st, 0, sizeof(StatusBlock), st), "memset status");
     if ((rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
-    CellArgs c{p->W_h, p->b_h, w.u, y, y0, w.J, nullptr, B, T, n};
+    CellArgs c{p->W_h, p->b_h, w.u, y, y0, w.J, nullptr, B, T, n, nullptr};
     if ((rc = run_cell(c, st)) != DEER_OK) return rc;
     ScanArgs a{};
     a.J = w.J; a.b = gy; a.y0 = nullptr; a.y = w.lam; a.yold = nullptr;

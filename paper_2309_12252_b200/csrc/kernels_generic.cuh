@@ -31,6 +31,7 @@ __global__ void proj_kernel(const float *__restrict__ x, const float *__restrict
 //   J = diag(z) + diag(a_z) W_hz + diag(a_n r) W_hn + diag(a_n q r (1-r)) W_hr.
 __global__ void cell_kernel(CellArgs a)
 {
+    if (loop_ended(a.st)) return;
     extern __shared__ float sW[];          // W_h rows padded to n+1, then b_h
     const int n = a.n, ld = n + 1;
     float *sb = sW + 3 * n * ld;
@@ -73,6 +74,79 @@ __global__ void cell_kernel(CellArgs a)
     if (a.rhs) a.rhs[e * n + i] = f - acc;
 }
 
+// Same computation for n in {1,2,4,8}: the thread's three weight rows live in registers, positions
+// are visited with a grid stride, h_prev is read and the Jacobian row written with 128-bit accesses.
+template <int N>
+__global__ void __launch_bounds__(256) cell_small_kernel(CellArgs a)
+{
+    if (loop_ended(a.st)) return;
+    constexpr int EPB = 256 / N;                       // positions per block per step
+    const int i = threadIdx.x % N, le = threadIdx.x / N;
+    float wr[N], wz[N], wn[N];
+#pragma unroll
+    for (int k = 0; k < N; ++k) {
+        wr[k] = a.W_h[i * N + k];
+        wz[k] = a.W_h[(N + i) * N + k];
+        wn[k] = a.W_h[(2 * N + i) * N + k];
+    }
+    const float br = a.b_h[i], bz = a.b_h[N + i], bn = a.b_h[2 * N + i];
+    const size_t total = (size_t)a.B * a.T;
+    for (size_t e = (size_t)blockIdx.x * EPB + le; e < total; e += (size_t)gridDim.x * EPB) {
+        const size_t seq = e / a.T;
+        const bool first = (e - seq * a.T) == 0;
+        const float *hp = first ? a.y0 + seq * N : a.y + (e - 1) * N;
+        float h[N];
+        if constexpr (N >= 4) {
+#pragma unroll
+            for (int v = 0; v < N / 4; ++v) {
+                const float4 f = reinterpret_cast<const float4 *>(hp)[v];
+                h[4 * v] = f.x; h[4 * v + 1] = f.y; h[4 * v + 2] = f.z; h[4 * v + 3] = f.w;
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < N; ++k) h[k] = hp[k];
+        }
+        float gr = br, gz = bz, gq = bn;
+#pragma unroll
+        for (int k = 0; k < N; ++k) {
+            gr = fmaf(wr[k], h[k], gr);
+            gz = fmaf(wz[k], h[k], gz);
+            gq = fmaf(wn[k], h[k], gq);
+        }
+        const float *ue = a.u + e * 3 * N;
+        const float r = sigmoidf_acc(ue[i] + gr);
+        const float z = sigmoidf_acc(ue[N + i] + gz);
+        const float c = tanhf(ue[2 * N + i] + r * gq);
+        float hi = 0.0f;
+#pragma unroll
+        for (int k = 0; k < N; ++k) if (k == i) hi = h[k];
+        const float f = (1.0f - z) * c + z * hi;
+        const float az = (hi - c) * z * (1.0f - z);
+        const float an = (1.0f - z) * (1.0f - c * c);
+        const float kr = an * gq * r * (1.0f - r);
+        const float kn = an * r;
+        float v[N];
+        float acc = 0.0f;
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            v[j] = kr * wr[j] + az * wz[j] + kn * wn[j];
+            if (j == i) v[j] += z;
+            acc = fmaf(v[j], h[j], acc);
+        }
+        float *Jr = a.J + (e * N + i) * N;
+        if constexpr (N >= 4) {
+#pragma unroll
+            for (int q = 0; q < N / 4; ++q)
+                reinterpret_cast<float4 *>(Jr)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        } else if constexpr (N == 2) {
+            *reinterpret_cast<float2 *>(Jr) = make_float2(v[0], v[1]);
+        } else {
+            Jr[0] = v[0];
+        }
+        if (a.rhs) a.rhs[e * N + i] = f - acc;
+    }
+}
+
 // ------------------------------------------------------------------ a5: generic chunked scan
 __device__ __forceinline__ void gen_load_M(float *dst, const ScanArgs &a, size_t seq, int s)
 {
@@ -97,6 +171,7 @@ __device__ __forceinline__ size_t gen_vec_index(const ScanArgs &a, size_t seq, i
 // level 1: one CTA folds one chunk into (A, beta), later positions multiplying on the left.
 __global__ void gen_reduce_kernel(ScanArgs a)
 {
+    if (loop_ended(a.st)) return;
     extern __shared__ float sm[];
     const int n = a.n, nn = n * n;
     float *Jt = sm, *A = sm + nn, *A2 = sm + 2 * nn, *be = sm + 3 * nn, *be2 = be + n;
@@ -132,6 +207,7 @@ __global__ void gen_reduce_kernel(ScanArgs a)
 // level 2: one CTA per sequence walks the chunk aggregates in order.
 __global__ void gen_carry_kernel(ScanArgs a)
 {
+    if (loop_ended(a.st)) return;
     extern __shared__ float sm[];
     const int n = a.n, nn = n * n;
     float *Am = sm, *Y = sm + nn;
@@ -158,6 +234,7 @@ __global__ void gen_carry_kernel(ScanArgs a)
 // level 3: one CTA replays its chunk from the entering state, writes y and the max deviation.
 __global__ void gen_apply_kernel(ScanArgs a)
 {
+    if (loop_ended(a.st)) return;
     extern __shared__ float sm[];
     const int n = a.n, nn = n * n;
     float *Jt = sm, *Y = sm + nn;
@@ -187,6 +264,35 @@ __global__ void gen_apply_kernel(ScanArgs a)
         for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
         if ((threadIdx.x & 31) == 0 && mb) atomicMax(&a.st->err_bits, mb);
     }
+}
+
+// ------------------------------------------------------------------ a6: loop control on the device
+// Clears the single-pass scan's per-launch words (tile flags, entering states, counters).
+__global__ void scan_prep_kernel(StatusBlock *st, unsigned *flags, size_t nflags,
+                                 unsigned long long *starts, size_t nstarts)
+{
+    if (loop_ended(st)) return;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (size_t i = i0; i < nflags; i += stride) flags[i] = 0u;
+    for (size_t i = i0; i < nstarts; i += stride) starts[i] = 0ull;
+    if (i0 == 0) { st->tile_counter = 0u; st->role_counter = 0u; }
+}
+
+// End of one Newton body (App. B.1 loop): record err, count the body, decide whether the loop goes on
+// (err > tol and fewer than max_iter bodies).  A NaN err fails "err > tol" and ends the loop, as in
+// the listing; an infinite err ends it too.
+constexpr int ERR_TRACE_CAP = 1024;
+__global__ void newton_control_kernel(StatusBlock *st, float tol, int max_iter, float *trace)
+{
+    if (loop_ended(st)) return;
+    const unsigned bits = st->err_bits;
+    const float e = __uint_as_float(bits);
+    if (st->iters < ERR_TRACE_CAP) trace[st->iters] = e;
+    st->iters += 1;
+    st->err_last_bits = bits;
+    st->err_bits = 0u;
+    if (!(e > tol) || !(e <= 3.402823466e38f) || st->iters >= max_iter) st->done = 1;
 }
 
 // ------------------------------------------------------------------ a8: cell VJP

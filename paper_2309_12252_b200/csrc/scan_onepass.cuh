@@ -53,7 +53,7 @@ template <int N> struct OnePass {
     static constexpr int BRUN = S * N + ((N == 8) ? 4 : 0);          // floats per chain run of b / y
     static constexpr int JBUF = CHAINS * JRUN, BBUF = CHAINS * BRUN;
     static constexpr int AGG = N * N + N;              // floats of one aggregate (A row-major, then beta)
-    static constexpr int Q = (N == 8) ? 2 : 3;         // pending tiles (A scheduled, B not yet) per CTA
+    static constexpr int Q = (N == 1) ? 3 : 2;         // pending tiles (A scheduled, B not yet) per CTA
     // kept per pending tile: n = 8: chain aggregates + warp aggregates;
     //                        n <= 4: exclusive chain prefixes (within the warp) + exclusive warp prefixes
     static constexpr int PEND = (CHAINS + WARPS) * AGG;
@@ -439,6 +439,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     uint64_t *bar = (uint64_t *)(((uintptr_t)(ystart + N) + 15) & ~(uintptr_t)15);
     __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role;
 
+    if (loop_ended(a.st)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chain = tid / LPC, sub = tid % LPC;
     const unsigned chain_mask = (LPC == 32) ? 0xffffffffu : (((1u << LPC) - 1u) << (lane & ~(LPC - 1)));
