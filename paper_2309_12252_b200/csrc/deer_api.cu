@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "kernels_generic.cuh"
 #include "scan_onepass.cuh"
+#include "scan_warp8.cuh"
 
 namespace deer {
 
@@ -72,13 +73,20 @@ struct ScanWs {
     OnePassWs op;        // single-pass path (n in {1,2,4,8}); op.nch == 0 when not applicable
 };
 
+static bool use_warp8()
+{
+    static int v = -1;
+    if (v < 0) { const char *e = getenv("DEER_SCAN8_OLD"); v = (e && atoi(e)) ? 0 : 1; }
+    return v != 0;
+}
+
 static int onepass_tile_len(int n)
 {
     switch (n) {
     case 1: return OnePass<1>::L;
     case 2: return OnePass<2>::L;
     case 4: return OnePass<4>::L;
-    case 8: return OnePass<8>::L;
+    case 8: return use_warp8() ? Warp8::L : OnePass<8>::L;
     default: return 0;
     }
 }
@@ -157,6 +165,51 @@ static int launch_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
     return DEER_OK;
 }
 
+template <bool REV>
+static int launch_warp8(ScanArgs a, OnePassWs w, cudaStream_t st)
+{
+    using C = Warp8;
+    static int occ = 0;
+    auto kern = scan_warp8_kernel<REV>;
+    if (!occ) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(warp8)"); return DEER_ERR_CUDA; }
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, C::THREADS, C::SMEM);
+        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(warp8)"); return DEER_ERR_CUDA; }
+        // more CTAs in flight lengthen the distance between a tile's two visits beyond what L2 holds
+        int cap = 4;
+        if (const char *d = getenv("DEER_W8_CTAS")) cap = atoi(d);
+        occ = o < cap ? o : cap;
+        if (occ < 1) occ = 1;
+    }
+    size_t tiles = (size_t)a.B * w.nch;
+    size_t resident = (size_t)num_sms() * occ;
+    int R = (a.B + C::RES_WARPS - 1) / C::RES_WARPS;
+    if (R > 8) R = 8;
+    const int per_cta_cap = C::RES_WARPS * OnePass<8>::MAX_SEQ_PER_WARP;
+    if ((a.B + per_cta_cap - 1) / per_cta_cap > R) R = (a.B + per_cta_cap - 1) / per_cta_cap;
+    w.resolvers = R;
+    size_t want = tiles + (size_t)R;
+    unsigned grid = (unsigned)(want < resident ? want : resident);
+    if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
+    int Wd = 8;
+    if (Wd > w.nch) Wd = w.nch;
+    w.Wd = Wd;
+    w.nwin = (w.nch + Wd - 1) / Wd;
+    w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
+    w.debug = 0;
+    {
+        size_t words = tiles * (size_t)(C::N + 1);
+        unsigned pb = (unsigned)((words + 255) / 256);
+        if (pb > 592u) pb = 592u;
+        if (pb < 1u) pb = 1u;
+        DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)C::N));
+    }
+    DEER_KERNEL("scan_warp8_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
+    return DEER_OK;
+}
+
 static int scan_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
 {
     switch (a.n * 2 + (a.reverse ? 1 : 0)) {
@@ -166,8 +219,8 @@ static int scan_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
     case 5: return launch_onepass<2, true>(a, w, st);
     case 8: return launch_onepass<4, false>(a, w, st);
     case 9: return launch_onepass<4, true>(a, w, st);
-    case 16: return launch_onepass<8, false>(a, w, st);
-    case 17: return launch_onepass<8, true>(a, w, st);
+    case 16: return use_warp8() ? launch_warp8<false>(a, w, st) : launch_onepass<8, false>(a, w, st);
+    case 17: return use_warp8() ? launch_warp8<true>(a, w, st) : launch_onepass<8, true>(a, w, st);
     default: return DEER_ERR_UNSUPPORTED_N;
     }
 }

@@ -1,0 +1,297 @@
+// Single-pass scan for n = 8 with one WARP per chain and the chain product on tensor cores.
+//
+// Global protocol as in scan_onepass.cuh: a tile (8 chains x SW positions) gets an A item (fold
+// into the tile aggregate, publish) and later a B item (replay from the entering state that a
+// resolver warp published, write y); the tile's second read is served by L2.  Inside a CTA:
+//   * each of the 8 warps owns one chain of SW consecutive positions and streams its J_t straight
+//     from global memory: one coalesced 256-byte load per position (lane l reads floats 2l, 2l+1),
+//     software-prefetched a group of positions ahead in registers.  No shared-memory staging.
+//   * A item: the running product is kept TRANSPOSED, X = P^T with beta^T as a ninth row, in the
+//     accumulator fragment of mma.sync.m16n8k8 (TF32 inputs, fp32 accumulate):
+//         [X; beta^T] <- [X; beta^T] * J_t^T + [0; b_t^T].
+//     The accumulator fragment (row g, columns 2t, 2t+1 in lane 4g+t) is reused as the next A
+//     operand without any shuffle by renaming the contraction index (k-slot t <-> column 2t,
+//     k-slot t+4 <-> column 2t+1); the B operand then is exactly the lane's 8-byte piece of J_t.
+//     Each product is issued as three MMAs on hi/lo TF32 splits (hi*hi + hi*lo + lo*hi), which
+//     keeps fp32-level accuracy.
+//   * B item: y <- J_t y + b_t as a shuffle mat-vec from the same 8-byte pieces.
+//   * The 8 warp aggregates of a tile are combined through shared memory (once per tile).
+// Reverse scans use J[t+1]^T: only the addressing of the lane's piece changes.
+#pragma once
+#include "scan_onepass.cuh"
+
+namespace deer {
+
+struct Warp8 {
+    static constexpr int N = 8, NN = 64, AGG = 72;
+    static constexpr int WARPS = 8, THREADS = 256;
+    static constexpr int SW = 32;                      // positions per warp chain
+    static constexpr int L = WARPS * SW;               // positions per tile
+    static constexpr int GRP = 8;                      // positions loaded ahead per group
+    static constexpr int Q = 2;                        // pending tiles per CTA
+    static constexpr int RES_WARPS = 4;                // warps of a resolver CTA that resolve
+    static constexpr int PEND = WARPS * AGG;           // warp aggregates kept for the B item
+    static constexpr int SM_WORK = Q * PEND + WARPS * N + N + 16;
+    static constexpr int SM_RES = RES_WARPS * 32 * AGG;
+    static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
+    static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
+    static_assert(SW % GRP == 0, "chains are processed in whole groups");
+};
+
+// d = a * b + c   (m16n8k8, A row-major 16x8, B 8x8, TF32 inputs, fp32 accumulate)
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const unsigned (&a)[4], const unsigned (&b)[2], const float (&c)[4])
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]),
+                   "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
+}
+
+// hi / lo TF32 split by truncation: hi keeps the top 10 mantissa bits, lo the next 10 of the exact
+// remainder, so hi*hi + hi*lo + lo*hi carries about 21 mantissa bits of every product
+__device__ __forceinline__ void split_tf32(float x, unsigned &hi, unsigned &lo)
+{
+    hi = __float_as_uint(x) & 0xffffe000u;
+    lo = __float_as_uint(x - __uint_as_float(hi)) & 0xffffe000u;
+}
+
+// one step of the transposed chain on the accumulator fragment:
+//   [X; beta^T] <- [X; beta^T] * M + [0; (bx, by)]   with the lane's piece (j0, j1) of M
+__device__ __forceinline__ void chain_step(float (&acc)[4], float j0, float j1, float bx, float by)
+{
+    unsigned ah[4], al[4], bh[2], bl[2];
+    split_tf32(acc[0], ah[0], al[0]);      // a0 <- c0
+    split_tf32(acc[2], ah[1], al[1]);      // a1 <- c2
+    split_tf32(acc[1], ah[2], al[2]);      // a2 <- c1
+    split_tf32(acc[3], ah[3], al[3]);      // a3 <- c3
+    split_tf32(j0, bh[0], bl[0]);
+    split_tf32(j1, bh[1], bl[1]);
+    float d[4] = {0.0f, 0.0f, bx, by};
+    mma_tf32(d, al, bh, d);
+    mma_tf32(d, ah, bl, d);
+    mma_tf32(d, ah, bh, d);
+    acc[0] = d[0]; acc[1] = d[1]; acc[2] = d[2]; acc[3] = d[3];
+}
+
+template <bool REV>
+__global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs a, OnePassWs w)
+{
+    using C = Warp8;
+    constexpr int N = C::N, NN = C::NN, AGG = C::AGG, WARPS = C::WARPS, SW = C::SW, GRP = C::GRP, Q = C::Q;
+    if (loop_ended(a.st)) return;
+
+    extern __shared__ __align__(16) float smem_raw[];
+    float *sm = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    float *pend = sm;                          // Q x warp aggregates (A row-major, then beta)
+    float *wstart = pend + Q * C::PEND;        // WARPS x N states entering each warp chain
+    float *ystart = wstart + WARPS * N;
+    __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;     // fragment coordinates
+    const int T = a.T;
+
+    if (tid == 0) {
+        s_abort = 0;
+        s_role = (int)atomicAdd(&a.st->role_counter, 1u);
+    }
+    __syncthreads();
+    if (s_role < w.resolvers) {
+        if (warp < C::RES_WARPS)
+            resolver_loop<8>(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        return;
+    }
+    unsigned mb = 0;
+
+    auto decode = [&](unsigned id, int &seq, int &c) {
+        const unsigned j = id % (unsigned)w.Wd;
+        const unsigned ws_ = id / (unsigned)w.Wd;
+        seq = (int)(ws_ % (unsigned)a.B);
+        const unsigned win = ws_ / (unsigned)a.B;
+        c = (int)(win * (unsigned)w.Wd + j);
+        if (c >= w.nch) c = -1;
+    };
+    int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
+    bool exhausted = false;
+
+    for (;;) {
+        __syncthreads();
+        if (tid == 0) {
+            int kind = -1, seq = -1, c = -1, slot = 0;
+            bool want_b = false;
+            if (q_cnt > 0) {
+                want_b = (q_cnt == Q) || exhausted;
+                if (!want_b)
+                    want_b = ld_relaxed_u64(w.starts + ((size_t)q_seq[q_head] * w.nch + q_c[q_head]) * N) != 0ull;
+            }
+            if (!want_b && !exhausted) {
+                for (;;) {
+                    const unsigned id = atomicAdd(&a.st->tile_counter, 1u);
+                    if (id >= w.total_ids) { c = -1; break; }
+                    decode(id, seq, c);
+                    if (c >= 0) break;
+                }
+                if (c >= 0) {
+                    kind = 0;
+                    slot = (q_head + q_cnt) % Q;
+                    q_seq[slot] = seq; q_c[slot] = c; ++q_cnt;
+                } else {
+                    exhausted = true;
+                    want_b = q_cnt > 0;
+                }
+            }
+            if (want_b) {
+                kind = 1; slot = q_head; seq = q_seq[q_head]; c = q_c[q_head];
+                q_head = (q_head + 1) % Q; --q_cnt;
+            }
+            s_kind = kind; s_seq = seq; s_c = c; s_slot = slot;
+        }
+        __syncthreads();
+        if (s_kind < 0 || s_abort) break;
+        const int kind = s_kind, seq = s_seq, c = s_c;
+        float *wagg = pend + s_slot * C::PEND;
+        const int s0 = c * C::L;                               // first scan position of the tile
+        const int Lt = min(C::L, T - s0);
+        const int p0 = warp * SW;                              // first scan offset of this warp's chain
+        const int cnt = min(SW, max(0, Lt - p0));
+        const size_t tile_index = (size_t)seq * w.nch + c;
+        const float *Jseq = a.J + (size_t)seq * T * NN;
+        const float *bseq = a.b + (size_t)seq * T * N;
+
+        const int sbase = s0 + p0;                             // scan position of the chain's first element
+        // per-lane pointers at the chain's first position; the piece advances by a constant per position
+        //   forward: float2 #lane of J[s]            (+32 float2 per position), b[s] pairs (+4 float2)
+        //   reverse: J[T-s] entries (2t,g),(2t+1,g)  (-64 floats per position), b[T-1-s] (-4 float2)
+        const float2 *jp2 = reinterpret_cast<const float2 *>(Jseq + (size_t)sbase * NN) + lane;
+        const float *jpr = Jseq + (size_t)(T - sbase) * NN + (2 * t) * N + g;
+        const size_t tb = REV ? (size_t)(T - 1 - sbase) : (size_t)sbase;
+        auto piece = [&](int q, float &j0, float &j1) {
+            if (!REV) { const float2 f = __ldg(jp2 + q * 32); j0 = f.x; j1 = f.y; }
+            else if (sbase + q == 0) { j0 = (g == 2 * t) ? 1.0f : 0.0f; j1 = (g == 2 * t + 1) ? 1.0f : 0.0f; }
+            else { j0 = __ldg(jpr - q * NN); j1 = __ldg(jpr - q * NN + N); }
+        };
+
+        if (kind == 0) {
+            // ---------------------------------------------- A item: [X; beta^T] in the accumulator fragment
+            float acc[4] = {(g == 2 * t) ? 1.0f : 0.0f, (g == 2 * t + 1) ? 1.0f : 0.0f, 0.0f, 0.0f};
+            const float2 *bp2 = reinterpret_cast<const float2 *>(bseq + tb * N) + t;
+#pragma unroll 1
+            for (int q0 = 0; q0 < cnt; q0 += GRP) {
+                float j0[GRP], j1[GRP], bx[GRP], by[GRP];
+                const bool full = (q0 + GRP <= cnt);
+#pragma unroll
+                for (int u = 0; u < GRP; ++u) {
+                    j0[u] = 0.0f; j1[u] = 0.0f; bx[u] = 0.0f; by[u] = 0.0f;
+                    if (full || q0 + u < cnt) {
+                        piece(q0 + u, j0[u], j1[u]);
+                        if (g == 0) {
+                            const float2 f = __ldg(REV ? bp2 - (q0 + u) * 4 : bp2 + (q0 + u) * 4);
+                            bx[u] = f.x; by[u] = f.y;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < GRP; ++u)
+                    if (full || q0 + u < cnt) chain_step(acc, j0[u], j1[u], bx[u], by[u]);
+            }
+            // X[g][2t] = P[2t][g], X[g][2t+1] = P[2t+1][g]; beta in row 8 (lanes with g == 0)
+            {
+                float *ag = wagg + warp * AGG;
+                ag[(2 * t) * N + g] = acc[0];
+                ag[(2 * t + 1) * N + g] = acc[1];
+                if (g == 0) { ag[NN + 2 * t] = acc[2]; ag[NN + 2 * t + 1] = acc[3]; }
+            }
+            __syncthreads();
+            if (warp == 0) {
+                // tile aggregate: the same step with the warp aggregates as "positions" (forward form:
+                // piece (g,2t),(g,2t+1) of A_k, beta_k as the additive row)
+                float tac[4] = {(g == 2 * t) ? 1.0f : 0.0f, (g == 2 * t + 1) ? 1.0f : 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                for (int k = 0; k < WARPS; ++k) {
+                    const float *ak = wagg + k * AGG;
+                    const float2 f = *reinterpret_cast<const float2 *>(ak + 2 * lane);
+                    float bx = 0.0f, by = 0.0f;
+                    if (g == 0) { bx = ak[NN + 2 * t]; by = ak[NN + 2 * t + 1]; }
+                    chain_step(tac, f.x, f.y, bx, by);
+                }
+                float *gdst = w.aggs + tile_index * AGG;
+                gdst[(2 * t) * N + g] = tac[0];
+                gdst[(2 * t + 1) * N + g] = tac[1];
+                if (g == 0) { gdst[NN + 2 * t] = tac[2]; gdst[NN + 2 * t + 1] = tac[3]; }
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) st_release_u32(w.flags + tile_index, 1u);
+            }
+            continue;
+        }
+
+        // -------------------------------------------------- B item
+        if (warp == 1) {
+            const unsigned long long *src = w.starts + tile_index * N;
+            unsigned spins = 0;
+            bool ok = true;
+            for (;;) {
+                const unsigned long long v = (lane < N) ? ld_relaxed_u64(src + lane) : LL_FLAG;
+                if (__all_sync(0xffffffffu, v != 0ull)) {
+                    if (lane < N) ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                    break;
+                }
+                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+            }
+            if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
+        }
+        __syncthreads();
+        if (s_abort) break;
+        if (warp == 0) {
+            if (lane < N) wstart[lane] = ystart[lane];
+            __syncwarp();
+            for (int k = 0; k + 1 < WARPS; ++k)
+                matvec_smem<8>(wstart + (k + 1) * N, wagg + k * AGG, wstart + k * N, lane);
+        }
+        __syncthreads();
+        {
+            // lane (g,t) carries y[2t], y[2t+1]; every step: partial sums over k = 2t, 2t+1, reduced over t
+            float yk0 = wstart[warp * N + 2 * t], yk1 = wstart[warp * N + 2 * t + 1];
+            const float *bpg = bseq + tb * N + g;
+            const float *yop = a.yold ? a.yold + ((size_t)seq * T + tb) * N + g : nullptr;
+            float *yp = a.y + ((size_t)seq * T + tb) * N + g;
+#pragma unroll 1
+            for (int q0 = 0; q0 < cnt; q0 += GRP) {
+                float j0[GRP], j1[GRP], bg[GRP], yo[GRP];
+                const bool full = (q0 + GRP <= cnt);
+#pragma unroll
+                for (int u = 0; u < GRP; ++u) {
+                    j0[u] = 0.0f; j1[u] = 0.0f; bg[u] = 0.0f; yo[u] = 0.0f;
+                    if (full || q0 + u < cnt) {
+                        const int off = REV ? -(q0 + u) * N : (q0 + u) * N;
+                        piece(q0 + u, j0[u], j1[u]);
+                        bg[u] = __ldg(bpg + off);
+                        if (yop && t == 0) yo[u] = __ldg(yop + off);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < GRP; ++u) {
+                    if (full || q0 + u < cnt) {
+                        float part = fmaf(j0[u], yk0, j1[u] * yk1);
+                        part += __shfl_xor_sync(0xffffffffu, part, 1);
+                        part += __shfl_xor_sync(0xffffffffu, part, 2);
+                        const float yg = part + bg[u];                              // y_new[g], in all 4 lanes of group g
+                        yk0 = __shfl_sync(0xffffffffu, yg, 4 * (2 * t));
+                        yk1 = __shfl_sync(0xffffffffu, yg, 4 * (2 * t + 1));
+                        if (t == 0) {
+                            if (yop) mb = max(mb, absdiff_bits(yg, yo[u]));
+                            yp[REV ? -(q0 + u) * N : (q0 + u) * N] = yg;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    if (a.yold) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+        if (lane == 0 && mb) atomicMax(&a.st->err_bits, mb);
+    }
+}
+
+}  // namespace deer
