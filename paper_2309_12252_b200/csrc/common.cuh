@@ -84,7 +84,11 @@ struct ScanArgs {
 struct CellArgs {
     const float *W_h;    // [3n,n]
     const float *b_h;    // [3n]
-    const float *u;      // [B,T,3n] input projection  x W_i^T + b_i
+    const float *u;      // [B,T,3n] input projection  x W_i^T + b_i  (nullptr: project on the fly from x)
+    const float *x;      // [B,T,m]  only read when u == nullptr
+    const float *W_i;    // [3n,m]
+    const float *b_i;    // [3n]
+    int m;
     const float *y;      // [B,T,n] current trajectory guess
     const float *y0;     // [B,n]
     float *J;            // [B,T,n,n] out

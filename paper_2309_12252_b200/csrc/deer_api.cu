@@ -273,8 +273,22 @@ template <int N> static int launch_cell_small(CellArgs c, cudaStream_t st)
     size_t blocks = (total + epb - 1) / epb;
     const size_t cap = (size_t)num_sms() * 8;
     if (blocks > cap) blocks = cap;
-    DEER_KERNEL("cell_small_kernel", st, cell_small_kernel<N><<<(unsigned)blocks, 256, 0, st>>>(c));
+    const unsigned gb = (unsigned)blocks;
+    if (c.u) { DEER_KERNEL("cell_small_kernel", st, cell_small_kernel<N, 0><<<gb, 256, 0, st>>>(c)); return DEER_OK; }
+    switch (c.m) {
+    case 1: DEER_KERNEL("cell_small_kernel", st, cell_small_kernel<N, 1><<<gb, 256, 0, st>>>(c)); break;
+    case 2: DEER_KERNEL("cell_small_kernel", st, cell_small_kernel<N, 2><<<gb, 256, 0, st>>>(c)); break;
+    case 4: DEER_KERNEL("cell_small_kernel", st, cell_small_kernel<N, 4><<<gb, 256, 0, st>>>(c)); break;
+    case 8: DEER_KERNEL("cell_small_kernel", st, cell_small_kernel<N, 8><<<gb, 256, 0, st>>>(c)); break;
+    default: return DEER_ERR_INVALID_ARG;
+    }
     return DEER_OK;
+}
+
+// the cell kernel can project x itself (no u buffer, no proj pass) for these sizes
+static bool cell_projects(int n, int m)
+{
+    return (n == 1 || n == 2 || n == 4 || n == 8) && (m == 1 || m == 2 || m == 4 || m == 8);
 }
 
 static int run_cell(CellArgs c, cudaStream_t st)
@@ -444,7 +458,8 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     DEER_CHECK_CUDA(cudaMemsetAsync(w.st, 0, sizeof(StatusBlock), st), "memset status");
     if (!(flags & DEER_FLAG_WARM_START))
         DEER_CHECK_CUDA(cudaMemsetAsync(y, 0, N * n * sizeof(float), st), "memset y");
-    if ((rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
+    const bool fused_proj = cell_projects(n, m) && ((((uintptr_t)y | (uintptr_t)y0) & 15) == 0);
+    if (!fused_proj && (rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
 
     // Newton loop (App. B.1): bodies are enqueued ahead of the convergence test -- the control kernel
     // at the end of each body decides on the device, and the kernels of bodies past the end return
@@ -457,7 +472,7 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
         if (todo > group) todo = group;
         for (int j = 0; j < todo; ++j, ++enq) {
             float *cur = buf[enq & 1], *nxt = buf[(enq + 1) & 1];
-            CellArgs c{p->W_h, p->b_h, w.u, cur, y0, w.J, w.rhs, B, T, n, w.st};
+            CellArgs c{p->W_h, p->b_h, fused_proj ? nullptr : w.u, x, p->W_i, p->b_i, m, cur, y0, w.J, w.rhs, B, T, n, w.st};
             if ((rc = run_cell(c, st)) != DEER_OK) return rc;
             ScanArgs a{};
             a.J = w.J; a.b = w.rhs; a.y0 = y0; a.y = nxt; a.yold = cur;
@@ -502,7 +517,7 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
     const size_t N = (size_t)B * T;
     DEER_CHECK_CUDA(cudaMemsetAsync(w.st, 0, sizeof(StatusBlock), st), "memset status");
     if ((rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
-    CellArgs c{p->W_h, p->b_h, w.u, y, y0, w.J, nullptr, B, T, n, nullptr};
+    CellArgs c{p->W_h, p->b_h, w.u, x, p->W_i, p->b_i, m, y, y0, w.J, nullptr, B, T, n, nullptr};
     if ((rc = run_cell(c, st)) != DEER_OK) return rc;
     ScanArgs a{};
     a.J = w.J; a.b = gy; a.y0 = nullptr; a.y = w.lam; a.yold = nullptr;

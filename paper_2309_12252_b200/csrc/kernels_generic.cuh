@@ -76,7 +76,9 @@ __global__ void cell_kernel(CellArgs a)
 
 // Same computation for n in {1,2,4,8}: the thread's three weight rows live in registers, positions
 // are visited with a grid stride, h_prev is read and the Jacobian row written with 128-bit accesses.
-template <int N>
+// M > 0: the input projection (a0) is done on the fly from x with the thread's 3 x M weights in
+// registers (small input sizes: cheaper than a separate pass over u); M == 0: read u.
+template <int N, int M>
 __global__ void __launch_bounds__(256) cell_small_kernel(CellArgs a)
 {
     if (loop_ended(a.st)) return;
@@ -90,6 +92,17 @@ __global__ void __launch_bounds__(256) cell_small_kernel(CellArgs a)
         wn[k] = a.W_h[(2 * N + i) * N + k];
     }
     const float br = a.b_h[i], bz = a.b_h[N + i], bn = a.b_h[2 * N + i];
+    constexpr int MM = M > 0 ? M : 1;
+    float vr[MM], vz[MM], vn[MM], cr = 0.0f, cz = 0.0f, cn = 0.0f;
+    if constexpr (M > 0) {
+#pragma unroll
+        for (int k = 0; k < M; ++k) {
+            vr[k] = a.W_i[i * M + k];
+            vz[k] = a.W_i[(N + i) * M + k];
+            vn[k] = a.W_i[(2 * N + i) * M + k];
+        }
+        cr = a.b_i[i]; cz = a.b_i[N + i]; cn = a.b_i[2 * N + i];
+    }
     const size_t total = (size_t)a.B * a.T;
     for (size_t e = (size_t)blockIdx.x * EPB + le; e < total; e += (size_t)gridDim.x * EPB) {
         const size_t seq = e / a.T;
@@ -113,10 +126,22 @@ __global__ void __launch_bounds__(256) cell_small_kernel(CellArgs a)
             gz = fmaf(wz[k], h[k], gz);
             gq = fmaf(wn[k], h[k], gq);
         }
-        const float *ue = a.u + e * 3 * N;
-        const float r = sigmoidf_acc(ue[i] + gr);
-        const float z = sigmoidf_acc(ue[N + i] + gz);
-        const float c = tanhf(ue[2 * N + i] + r * gq);
+        float ur, uz, un;
+        if constexpr (M > 0) {
+            const float *xe = a.x + e * M;
+            ur = cr; uz = cz; un = cn;
+#pragma unroll
+            for (int k = 0; k < M; ++k) {
+                const float xv = xe[k];
+                ur = fmaf(vr[k], xv, ur); uz = fmaf(vz[k], xv, uz); un = fmaf(vn[k], xv, un);
+            }
+        } else {
+            const float *ue = a.u + e * 3 * N;
+            ur = ue[i]; uz = ue[N + i]; un = ue[2 * N + i];
+        }
+        const float r = sigmoidf_acc(ur + gr);
+        const float z = sigmoidf_acc(uz + gz);
+        const float c = tanhf(un + r * gq);
         float hi = 0.0f;
 #pragma unroll
         for (int k = 0; k < N; ++k) if (k == i) hi = h[k];
