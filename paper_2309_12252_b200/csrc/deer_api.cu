@@ -14,6 +14,7 @@
 #include "kernels_generic.cuh"
 #include "scan_onepass.cuh"
 #include "scan_warp8.cuh"
+#include "scan_warpn.cuh"
 
 namespace deer {
 
@@ -87,6 +88,8 @@ static int onepass_tile_len(int n)
     case 2: return OnePass<2>::L;
     case 4: return OnePass<4>::L;
     case 8: return use_warp8() ? Warp8::L : OnePass<8>::L;
+    case 16: return WarpN<16>::L;
+    case 32: return WarpN<32>::L;
     default: return 0;
     }
 }
@@ -210,6 +213,50 @@ static int launch_warp8(ScanArgs a, OnePassWs w, cudaStream_t st)
     return DEER_OK;
 }
 
+template <int N, bool REV>
+static int launch_warpn(ScanArgs a, OnePassWs w, cudaStream_t st)
+{
+    using C = WarpN<N>;
+    static int occ = 0;
+    auto kern = scan_warpn_kernel<N, REV>;
+    if (!occ) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(warpn)"); return DEER_ERR_CUDA; }
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, C::THREADS, C::SMEM);
+        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(warpn)"); return DEER_ERR_CUDA; }
+        int cap = 8;
+        if (const char *d = getenv("DEER_WN_CTAS")) cap = atoi(d);
+        occ = o < cap ? o : cap;
+        if (occ < 1) occ = 1;
+    }
+    size_t tiles = (size_t)a.B * w.nch;
+    size_t resident = (size_t)num_sms() * occ;
+    int R = (a.B + C::RES_WARPS - 1) / C::RES_WARPS;
+    if (R > 8) R = 8;
+    const int per_cta_cap = C::RES_WARPS * C::MAX_SEQ_PER_WARP;
+    if ((a.B + per_cta_cap - 1) / per_cta_cap > R) R = (a.B + per_cta_cap - 1) / per_cta_cap;
+    w.resolvers = R;
+    size_t want = tiles + (size_t)R;
+    unsigned grid = (unsigned)(want < resident ? want : resident);
+    if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
+    int Wd = 8;
+    if (Wd > w.nch) Wd = w.nch;
+    w.Wd = Wd;
+    w.nwin = (w.nch + Wd - 1) / Wd;
+    w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
+    w.debug = 0;
+    {
+        size_t words = tiles * (size_t)(N + 1);
+        unsigned pb = (unsigned)((words + 255) / 256);
+        if (pb > 592u) pb = 592u;
+        if (pb < 1u) pb = 1u;
+        DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)N));
+    }
+    DEER_KERNEL("scan_warpn_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
+    return DEER_OK;
+}
+
 static int scan_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
 {
     switch (a.n * 2 + (a.reverse ? 1 : 0)) {
@@ -221,6 +268,10 @@ static int scan_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
     case 9: return launch_onepass<4, true>(a, w, st);
     case 16: return use_warp8() ? launch_warp8<false>(a, w, st) : launch_onepass<8, false>(a, w, st);
     case 17: return use_warp8() ? launch_warp8<true>(a, w, st) : launch_onepass<8, true>(a, w, st);
+    case 32: return launch_warpn<16, false>(a, w, st);
+    case 33: return launch_warpn<16, true>(a, w, st);
+    case 64: return launch_warpn<32, false>(a, w, st);
+    case 65: return launch_warpn<32, true>(a, w, st);
     default: return DEER_ERR_UNSUPPORTED_N;
     }
 }

@@ -1,0 +1,475 @@
+// Single-pass scan for n = 16 and n = 32: one warp per chain, chain product on tensor cores.
+//
+// The n = 8 design of scan_warp8.cuh with the n x n running product tiled into m16n8k8 fragments:
+//   * the warp keeps X = P^T (n x n) in (n/16) x (n/8) accumulator fragments and advances it with
+//         X <- X * M,   M = J_t^T (forward)  or  J_{t+1} (reverse),
+//     as (n/16)(n/8)(n/8) MMAs per position, each issued three times on hi/lo TF32 splits; the
+//     accumulator fragment of column block kk is the A operand of contraction block kk (the same
+//     renaming of the contraction index as for n = 8), and the B operand of (kk, nn) is the lane's
+//     8-byte piece J[8nn+g][8kk+2t .. +1] (forward) read straight from global memory;
+//   * beta is carried as a separate mat-vec chain started from zero (the same routine replays the
+//     chain from its true entering state in the B item): lane (g,t) holds y[8kk+2t], y[8kk+2t+1];
+//   * warp aggregates are combined by warp 0 with the same step, reading them from shared memory.
+// Tiles, items, resolvers, flags and bounded waits are those of scan_onepass.cuh.
+#pragma once
+#include "scan_warp8.cuh"
+
+namespace deer {
+
+template <int N> struct WarpN {
+    static constexpr int NN = N * N, AGG = N * N + N;
+    static constexpr int NT = N / 8;                   // 8-wide column / contraction blocks
+    static constexpr int MT = N / 16;                  // 16-high row blocks of X
+    static constexpr int WARPS = (N == 16) ? 8 : 4;    // chains per tile
+    static constexpr int THREADS = WARPS * 32;
+    static constexpr int SW = 16;                      // positions per warp chain
+    static constexpr int L = WARPS * SW;               // positions per tile
+    static constexpr int Q = 2;                        // pending tiles per CTA
+    static constexpr int RES_WARPS = 4;                // warps of a resolver CTA that resolve
+    static constexpr int RES_BATCH = (N == 16) ? 8 : 2;   // aggregates a resolver warp stages at once
+    static constexpr int PEND = WARPS * AGG;           // warp aggregates kept for the B item
+    static constexpr int SM_WORK = Q * PEND + AGG + WARPS * N + N + 16;
+    static constexpr int SM_RES = RES_WARPS * RES_BATCH * AGG;
+    static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
+    static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
+    static constexpr int MAX_SEQ_PER_WARP = 8;
+    static_assert(N == 16 || N == 32, "one row of the state per resolver lane");
+};
+
+// Resolver for n in {16, 32}: as resolver_loop of scan_onepass.cuh (lane i holds component i of the
+// running state, flags of the next window requested ahead), with a smaller staging batch.
+template <int N>
+__device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
+{
+    using C = WarpN<N>;
+    constexpr int AGG = C::AGG, NN = C::NN, BATCH = C::RES_BATCH;
+    float *stage = stage_all + (threadIdx.x >> 5) * BATCH * AGG;
+    int nseq = 0;
+    int pos[C::MAX_SEQ_PER_WARP];
+    float yv[C::MAX_SEQ_PER_WARP];
+    unsigned fnext[C::MAX_SEQ_PER_WARP];
+#pragma unroll
+    for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
+        pos[k] = 0; yv[k] = 0.0f; fnext[k] = 0u;
+        const int s = rw + k * nrw;
+        if (s < a.B) {
+            nseq = k + 1;
+            if (lane < N && a.y0) yv[k] = a.y0[(size_t)s * N + lane];
+            if (lane < w.nch) fnext[k] = ld_acquire_u32(w.flags + (size_t)s * w.nch + lane);
+        }
+    }
+    int remaining = nseq;
+    unsigned spins = 0;
+    while (remaining > 0) {
+        bool progressed = false;
+#pragma unroll
+        for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
+            if (k >= nseq) break;
+            const int c0 = pos[k];
+            if (c0 >= w.nch) continue;
+            const int s = rw + k * nrw;
+            const unsigned *flags = w.flags + (size_t)s * w.nch;
+            const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
+            int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
+            if (cnt > BATCH) cnt = BATCH;
+            {
+                const int j = c0 + cnt + lane;
+                fnext[k] = (j < w.nch) ? ld_acquire_u32(flags + j) : 0u;
+            }
+            if (cnt == 0) continue;
+            progressed = true;
+            const float4 *src = reinterpret_cast<const float4 *>(w.aggs + ((size_t)s * w.nch + c0) * AGG);
+            float4 *dst = reinterpret_cast<float4 *>(stage);
+            const int total4 = cnt * AGG / 4;
+            for (int i0 = 0; i0 < total4; i0 += 32 * 8) {
+                float4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int i = i0 + u * 32 + lane;
+                    if (i < total4) v[u] = __ldcg(src + i);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int i = i0 + u * 32 + lane;
+                    if (i < total4) dst[i] = v[u];
+                }
+            }
+            __syncwarp();
+            unsigned long long *out = w.starts + ((size_t)s * w.nch + c0) * N;
+            float y = yv[k];
+            for (int q = 0; q < cnt; ++q) {
+                if (lane < N) st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y));
+                const float *ag = stage + q * AGG;
+                float acc0 = (lane < N) ? ag[NN + lane] : 0.0f, acc1 = 0.0f;
+                const float *row = ag + (lane < N ? lane : 0) * N;
+#pragma unroll
+                for (int i = 0; i < N; i += 2) {       // skewed column order: conflict-free row reads
+                    const int c0i = (i + lane) & (N - 1), c1i = (i + 1 + lane) & (N - 1);
+                    const float y0 = __shfl_sync(0xffffffffu, y, c0i), y1 = __shfl_sync(0xffffffffu, y, c1i);
+                    acc0 = fmaf(row[c0i], y0, acc0);
+                    acc1 = fmaf(row[c1i], y1, acc1);
+                }
+                y = acc0 + acc1;
+            }
+            yv[k] = y;
+            __syncwarp();
+            pos[k] = c0 + cnt;
+            if (pos[k] >= w.nch) --remaining;
+        }
+        if (progressed) spins = 0;
+        else if (!keep_spinning(a.st, spins)) return;
+    }
+}
+
+// The lane's pieces of one position's matrix, jp[nn][kk] = {M[8kk+2t][8nn+g], M[8kk+2t+1][8nn+g]}:
+// forward M = J^T (a float2 of row 8nn+g of J), reverse M = J (two scalars of column 8nn+g).
+template <int N, bool REV>
+__device__ __forceinline__ void load_pieces(float (&jp)[N / 8][N / 8][2], const float *Jt, int g, int t, bool ident)
+{
+    constexpr int NT = N / 8;
+#pragma unroll
+    for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+        for (int kk = 0; kk < NT; ++kk) {
+            if (ident) {
+                jp[nn][kk][0] = (8 * nn + g == 8 * kk + 2 * t) ? 1.0f : 0.0f;
+                jp[nn][kk][1] = (8 * nn + g == 8 * kk + 2 * t + 1) ? 1.0f : 0.0f;
+            } else if (!REV) {
+                const float2 f = __ldg(reinterpret_cast<const float2 *>(Jt + (8 * nn + g) * N + 8 * kk + 2 * t));
+                jp[nn][kk][0] = f.x; jp[nn][kk][1] = f.y;
+            } else {
+                jp[nn][kk][0] = __ldg(Jt + (8 * kk + 2 * t) * N + 8 * nn + g);
+                jp[nn][kk][1] = __ldg(Jt + (8 * kk + 2 * t + 1) * N + 8 * nn + g);
+            }
+        }
+}
+
+// the same pieces of an aggregate (A row-major in shared memory; always the forward form)
+template <int N>
+__device__ __forceinline__ void load_pieces_smem(float (&jp)[N / 8][N / 8][2], const float *A, int g, int t)
+{
+    constexpr int NT = N / 8;
+#pragma unroll
+    for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+        for (int kk = 0; kk < NT; ++kk) {
+            const float2 f = *reinterpret_cast<const float2 *>(A + (8 * nn + g) * N + 8 * kk + 2 * t);
+            jp[nn][kk][0] = f.x; jp[nn][kk][1] = f.y;
+        }
+}
+
+// X <- X * M on accumulator fragments acc[mm][nn] (row block mm, column block nn), 3 x TF32
+template <int N>
+__device__ __forceinline__ void chain_step_n(float (&acc)[N / 16][N / 8][4], const float (&jp)[N / 8][N / 8][2])
+{
+    constexpr int NT = N / 8, MT = N / 16;
+    float nacc[MT][NT][4];
+#pragma unroll
+    for (int mm = 0; mm < MT; ++mm)
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) nacc[mm][nn][i] = 0.0f;
+#pragma unroll
+    for (int kk = 0; kk < NT; ++kk) {
+        unsigned ah[MT][4], al[MT][4];
+#pragma unroll
+        for (int mm = 0; mm < MT; ++mm) {
+            split_tf32(acc[mm][kk][0], ah[mm][0], al[mm][0]);
+            split_tf32(acc[mm][kk][2], ah[mm][1], al[mm][1]);
+            split_tf32(acc[mm][kk][1], ah[mm][2], al[mm][2]);
+            split_tf32(acc[mm][kk][3], ah[mm][3], al[mm][3]);
+        }
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn) {
+            unsigned bh[2], bl[2];
+            split_tf32(jp[nn][kk][0], bh[0], bl[0]);
+            split_tf32(jp[nn][kk][1], bh[1], bl[1]);
+#pragma unroll
+            for (int mm = 0; mm < MT; ++mm) {
+                mma_tf32(nacc[mm][nn], al[mm], bh, nacc[mm][nn]);
+                mma_tf32(nacc[mm][nn], ah[mm], bl, nacc[mm][nn]);
+                mma_tf32(nacc[mm][nn], ah[mm], bh, nacc[mm][nn]);
+            }
+        }
+    }
+#pragma unroll
+    for (int mm = 0; mm < MT; ++mm)
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[mm][nn][i] = nacc[mm][nn][i];
+}
+
+// y <- M^T-form mat-vec: ynew[nn] = y_new[8nn+g] (in the 4 lanes of group g); yv[kk] = {y[8kk+2t], y[8kk+2t+1]}
+template <int N>
+__device__ __forceinline__ void matvec_step(float (&yv)[N / 8][2], const float (&jp)[N / 8][N / 8][2],
+                                            const float (&bg)[N / 8], float (&ynew)[N / 8], int t)
+{
+    constexpr int NT = N / 8;
+#pragma unroll
+    for (int nn = 0; nn < NT; ++nn) {
+        float p0 = 0.0f, p1 = 0.0f;
+#pragma unroll
+        for (int kk = 0; kk < NT; ++kk) {
+            p0 = fmaf(jp[nn][kk][0], yv[kk][0], p0);
+            p1 = fmaf(jp[nn][kk][1], yv[kk][1], p1);
+        }
+        float part = p0 + p1;
+        part += __shfl_xor_sync(0xffffffffu, part, 1);
+        part += __shfl_xor_sync(0xffffffffu, part, 2);
+        ynew[nn] = part + bg[nn];
+    }
+#pragma unroll
+    for (int kk = 0; kk < NT; ++kk) {
+        yv[kk][0] = __shfl_sync(0xffffffffu, ynew[kk], 4 * (2 * t));
+        yv[kk][1] = __shfl_sync(0xffffffffu, ynew[kk], 4 * (2 * t + 1));
+    }
+}
+
+// X = P^T in fragments  ->  P row-major (+ beta from the distributed vector) at dst (shared or global)
+template <int N>
+__device__ __forceinline__ void store_aggregate(float *dst, const float (&acc)[N / 16][N / 8][4],
+                                                const float (&yv)[N / 8][2], int g, int t)
+{
+    constexpr int NT = N / 8, MT = N / 16, NN = N * N;
+#pragma unroll
+    for (int mm = 0; mm < MT; ++mm)
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn) {
+            const int r = 16 * mm + g, c = 8 * nn + 2 * t;      // X[r][c] = P[c][r]
+            dst[c * N + r] = acc[mm][nn][0];
+            dst[(c + 1) * N + r] = acc[mm][nn][1];
+            dst[c * N + r + 8] = acc[mm][nn][2];
+            dst[(c + 1) * N + r + 8] = acc[mm][nn][3];
+        }
+    if (g == 0) {
+#pragma unroll
+        for (int kk = 0; kk < NT; ++kk) {
+            dst[NN + 8 * kk + 2 * t] = yv[kk][0];
+            dst[NN + 8 * kk + 2 * t + 1] = yv[kk][1];
+        }
+    }
+}
+
+template <int N>
+__device__ __forceinline__ void identity_fragments(float (&acc)[N / 16][N / 8][4], int g, int t)
+{
+#pragma unroll
+    for (int mm = 0; mm < N / 16; ++mm)
+#pragma unroll
+        for (int nn = 0; nn < N / 8; ++nn) {
+            const int r = 16 * mm + g, c = 8 * nn + 2 * t;
+            acc[mm][nn][0] = (r == c) ? 1.0f : 0.0f;
+            acc[mm][nn][1] = (r == c + 1) ? 1.0f : 0.0f;
+            acc[mm][nn][2] = (r + 8 == c) ? 1.0f : 0.0f;
+            acc[mm][nn][3] = (r + 8 == c + 1) ? 1.0f : 0.0f;
+        }
+}
+
+template <int N, bool REV>
+__global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs a, OnePassWs w)
+{
+    using C = WarpN<N>;
+    constexpr int NN = C::NN, AGG = C::AGG, NT = C::NT, MT = C::MT, WARPS = C::WARPS, SW = C::SW, Q = C::Q;
+    if (loop_ended(a.st)) return;
+
+    extern __shared__ __align__(16) float smem_raw[];
+    float *sm = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    float *pend = sm;                          // Q x warp aggregates (A row-major, then beta)
+    float *wstart = pend + Q * C::PEND;        // WARPS x N states entering each warp chain
+    float *ystart = wstart + WARPS * N;
+    __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int T = a.T;
+
+    if (tid == 0) {
+        s_abort = 0;
+        s_role = (int)atomicAdd(&a.st->role_counter, 1u);
+    }
+    __syncthreads();
+    if (s_role < w.resolvers) {
+        if (warp < C::RES_WARPS)
+            resolver_big<N>(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        return;
+    }
+    unsigned mb = 0;
+
+    auto decode = [&](unsigned id, int &seq, int &c) {
+        const unsigned j = id % (unsigned)w.Wd;
+        const unsigned ws_ = id / (unsigned)w.Wd;
+        seq = (int)(ws_ % (unsigned)a.B);
+        const unsigned win = ws_ / (unsigned)a.B;
+        c = (int)(win * (unsigned)w.Wd + j);
+        if (c >= w.nch) c = -1;
+    };
+    int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
+    bool exhausted = false;
+
+    for (;;) {
+        __syncthreads();
+        if (tid == 0) {
+            int kind = -1, seq = -1, c = -1, slot = 0;
+            bool want_b = false;
+            if (q_cnt > 0) {
+                want_b = (q_cnt == Q) || exhausted;
+                if (!want_b)
+                    want_b = ld_relaxed_u64(w.starts + ((size_t)q_seq[q_head] * w.nch + q_c[q_head]) * N) != 0ull;
+            }
+            if (!want_b && !exhausted) {
+                for (;;) {
+                    const unsigned id = atomicAdd(&a.st->tile_counter, 1u);
+                    if (id >= w.total_ids) { c = -1; break; }
+                    decode(id, seq, c);
+                    if (c >= 0) break;
+                }
+                if (c >= 0) {
+                    kind = 0;
+                    slot = (q_head + q_cnt) % Q;
+                    q_seq[slot] = seq; q_c[slot] = c; ++q_cnt;
+                } else {
+                    exhausted = true;
+                    want_b = q_cnt > 0;
+                }
+            }
+            if (want_b) {
+                kind = 1; slot = q_head; seq = q_seq[q_head]; c = q_c[q_head];
+                q_head = (q_head + 1) % Q; --q_cnt;
+            }
+            s_kind = kind; s_seq = seq; s_c = c; s_slot = slot;
+        }
+        __syncthreads();
+        if (s_kind < 0 || s_abort) break;
+        const int kind = s_kind, seq = s_seq, c = s_c;
+        float *wagg = pend + s_slot * C::PEND;
+        const int s0 = c * C::L;
+        const int Lt = min(C::L, T - s0);
+        const int p0 = warp * SW;
+        const int cnt = min(SW, max(0, Lt - p0));
+        const int sbase = s0 + p0;                             // scan position of the chain's first element
+        const size_t tile_index = (size_t)seq * w.nch + c;
+        const float *Jseq = a.J + (size_t)seq * T * NN;
+        const float *bseq = a.b + (size_t)seq * T * N;
+        // matrix of scan position s: forward J[s]; reverse J[T-s] (identity at s = 0); vector at t(s)
+        auto mat_ptr = [&](int s) { return REV ? Jseq + (size_t)(T - s) * NN : Jseq + (size_t)s * NN; };
+        auto pos_t = [&](int s) -> size_t { return REV ? (size_t)(T - 1 - s) : (size_t)s; };
+
+        if (kind == 0) {
+            // ---------------------------------------------- A item
+            float acc[MT][NT][4];
+            identity_fragments<N>(acc, g, t);
+            float yv[NT][2];
+#pragma unroll
+            for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = 0.0f; yv[kk][1] = 0.0f; }
+#pragma unroll 1
+            for (int q = 0; q < cnt; ++q) {
+                const int s = sbase + q;
+                float jp[NT][NT][2], bg[NT], ynew[NT];
+                load_pieces<N, REV>(jp, mat_ptr(s), g, t, REV && s == 0);
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn) bg[nn] = __ldg(bseq + pos_t(s) * N + 8 * nn + g);
+                chain_step_n<N>(acc, jp);
+                matvec_step<N>(yv, jp, bg, ynew, t);
+            }
+            store_aggregate<N>(wagg + warp * AGG, acc, yv, g, t);
+            __syncthreads();
+            if (warp == 0) {
+                // tile aggregate = the same steps with the warp aggregates as positions (forward form)
+                identity_fragments<N>(acc, g, t);
+#pragma unroll
+                for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = 0.0f; yv[kk][1] = 0.0f; }
+#pragma unroll 1
+                for (int k = 0; k < WARPS; ++k) {
+                    const float *ak = wagg + k * AGG;
+                    float jp[NT][NT][2], bg[NT], ynew[NT];
+                    load_pieces_smem<N>(jp, ak, g, t);
+#pragma unroll
+                    for (int nn = 0; nn < NT; ++nn) bg[nn] = ak[NN + 8 * nn + g];
+                    chain_step_n<N>(acc, jp);
+                    matvec_step<N>(yv, jp, bg, ynew, t);
+                }
+                store_aggregate<N>(w.aggs + tile_index * AGG, acc, yv, g, t);
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) st_release_u32(w.flags + tile_index, 1u);
+            }
+            continue;
+        }
+
+        // -------------------------------------------------- B item
+        if (warp == 1) {
+            const unsigned long long *src = w.starts + tile_index * N;
+            unsigned spins = 0;
+            bool ok = true;
+            for (;;) {
+                const unsigned long long v = (lane < N) ? ld_relaxed_u64(src + lane) : LL_FLAG;
+                if (__all_sync(0xffffffffu, v != 0ull)) {
+                    if (lane < N) ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                    break;
+                }
+                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+            }
+            if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
+        }
+        __syncthreads();
+        if (s_abort) break;
+        if (warp == 0) {
+            // states entering each warp chain: walk the warp aggregates from the tile's entering state
+            float yv[NT][2];
+#pragma unroll
+            for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = ystart[8 * kk + 2 * t]; yv[kk][1] = ystart[8 * kk + 2 * t + 1]; }
+#pragma unroll 1
+            for (int k = 0; k < WARPS; ++k) {
+                if (g == 0) {
+#pragma unroll
+                    for (int kk = 0; kk < NT; ++kk) {
+                        wstart[k * N + 8 * kk + 2 * t] = yv[kk][0];
+                        wstart[k * N + 8 * kk + 2 * t + 1] = yv[kk][1];
+                    }
+                }
+                if (k + 1 == WARPS) break;
+                const float *ak = wagg + k * AGG;
+                float jp[NT][NT][2], bg[NT], ynew[NT];
+                load_pieces_smem<N>(jp, ak, g, t);
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn) bg[nn] = ak[NN + 8 * nn + g];
+                matvec_step<N>(yv, jp, bg, ynew, t);
+            }
+        }
+        __syncthreads();
+        {
+            float yv[NT][2];
+#pragma unroll
+            for (int kk = 0; kk < NT; ++kk) {
+                yv[kk][0] = wstart[warp * N + 8 * kk + 2 * t];
+                yv[kk][1] = wstart[warp * N + 8 * kk + 2 * t + 1];
+            }
+#pragma unroll 1
+            for (int q = 0; q < cnt; ++q) {
+                const int s = sbase + q;
+                float jp[NT][NT][2], bg[NT], ynew[NT];
+                load_pieces<N, REV>(jp, mat_ptr(s), g, t, REV && s == 0);
+                const size_t vb = ((size_t)seq * T + pos_t(s)) * N;
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn) bg[nn] = __ldg(a.b + vb + 8 * nn + g);
+                matvec_step<N>(yv, jp, bg, ynew, t);
+                if (t == 0) {
+#pragma unroll
+                    for (int nn = 0; nn < NT; ++nn) {
+                        if (a.yold) mb = max(mb, absdiff_bits(ynew[nn], __ldg(a.yold + vb + 8 * nn + g)));
+                        a.y[vb + 8 * nn + g] = ynew[nn];
+                    }
+                }
+            }
+        }
+    }
+    if (a.yold) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+        if (lane == 0 && mb) atomicMax(&a.st->err_bits, mb);
+    }
+}
+
+}  // namespace deer
