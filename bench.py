@@ -209,9 +209,62 @@ def run_scan_only(args):
                           input_mb=(n * n + n) * 4 * B * T / 1e6)))
 
 
+def run_eval_only(args):
+    """deer_gru_eval (and optionally deer_gru_vjp) at an arbitrary sweep point: one JSON line."""
+    import torch
+    from paper_2309_12252_b200 import binding as bd
+    from paper_2309_12252_b200 import synth
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    n, m, B, T = args.n, (args.m or args.n), args.B, args.T
+    p = bd.GruParamsDev.from_numpy(synth.gru_params(n, m, 0, tag=f"sweep{n}/gru"))
+    g = torch.Generator(device=device); g.manual_seed(0)
+    x = torch.randn((B, T, m), device=device, generator=g)
+    y0 = torch.zeros((B, n), device=device)
+    y = torch.empty((B, T, n), device=device)
+    ws = bd.alloc_workspace(bd.DEER_OP_EVAL, B, T, n, m, args.flags, device)
+    stream = torch.cuda.current_stream()
+    run = lambda: bd.deer_gru_eval(p, x, y0, 1e-4, 100, y, ws, args.flags, stream)
+    for _ in range(max(args.warmup, 1)):
+        r = run()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    for a, b in ev:
+        a.record(stream); r = run(); b.record(stream)
+    torch.cuda.synchronize()
+    ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+    bd.lib().deer_profile_enable(1)
+    run()
+    torch.cuda.synchronize()
+    bd.lib().deer_profile_enable(0)
+    prof = read_profile(bd)
+    out = dict(mode="eval", n=n, m=m, B=B, T=T, flags=args.flags, ms=ms, steps_per_s=B * T / (ms * 1e-3),
+               iters=r.iters, err=r.err, status=r.status,
+               kernels={k: dict(launches=v["launches"], ms=round(v["total_ms"], 4)) for k, v in prof.items()})
+    if args.vjp:
+        gy = torch.randn((B, T, n), device=device, generator=g)
+        del ws
+        wsv = bd.alloc_workspace(bd.DEER_OP_VJP, B, T, n, m, args.flags, device)
+        for _ in range(2):
+            bd.deer_gru_vjp(p, x, y0, y, gy, True, True, wsv, args.flags, stream)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); bd.deer_gru_vjp(p, x, y0, y, gy, True, True, wsv, args.flags, stream); b.record(stream)
+        torch.cuda.synchronize()
+        out["vjp_ms"] = a.elapsed_time(b)
+        bd.lib().deer_profile_enable(1)
+        bd.deer_gru_vjp(p, x, y0, y, gy, True, True, wsv, args.flags, stream)
+        torch.cuda.synchronize()
+        bd.lib().deer_profile_enable(0)
+        out["vjp_kernels"] = {k: round(v["total_ms"], 4) for k, v in read_profile(bd).items()}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--mode", default="step", choices=["step", "scan"])
+    ap.add_argument("--mode", default="step", choices=["step", "scan", "eval"])
+    ap.add_argument("--m", type=int, default=0)
+    ap.add_argument("--vjp", type=int, default=0)
     ap.add_argument("--n", type=int, default=8)
     ap.add_argument("--B", type=int, default=16)
     ap.add_argument("--T", type=int, default=1_000_000)
@@ -229,6 +282,9 @@ def main():
         return
     if args.mode == "scan":
         run_scan_only(args)
+        return
+    if args.mode == "eval":
+        run_eval_only(args)
         return
 
     import torch

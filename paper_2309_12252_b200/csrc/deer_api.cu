@@ -15,6 +15,7 @@
 #include "scan_onepass.cuh"
 #include "scan_warp8.cuh"
 #include "scan_warpn.cuh"
+#include "cell_wide.cuh"
 
 namespace deer {
 
@@ -311,9 +312,37 @@ static int run_scan(ScanArgs a, const ScanWs &w, int flags, cudaStream_t st)
 
 static int run_proj(const deer_gru_params *p, const float *x, float *u, size_t N, cudaStream_t st)
 {
-    size_t total = N * 3 * (size_t)p->n;
+    const int n3 = 3 * p->n, m = p->m;
+    const int G = 256 / n3;
+    const size_t sm = sizeof(float) * ((size_t)m * n3 + (size_t)G * PROJ_PP * (m + 1));
+    if (G >= 1 && sm <= 200 * 1024) {
+        int rc;
+        if ((rc = opt_in_smem((const void *)proj_tiled_kernel, sm)) != DEER_OK) return rc;
+        const size_t tiles = (N + (size_t)G * PROJ_PP - 1) / ((size_t)G * PROJ_PP);
+        const size_t cap = (size_t)num_sms() * 8;
+        const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
+        const int threads = (n3 * G + 31) / 32 * 32;
+        DEER_KERNEL("proj_tiled_kernel", st,
+                    proj_tiled_kernel<<<blocks, threads, sm, st>>>(x, p->W_i, p->b_i, u, N, m, n3, G));
+        return DEER_OK;
+    }
+    size_t total = N * (size_t)n3;
     unsigned blocks = (unsigned)((total + 255) / 256);
-    DEER_KERNEL("proj_kernel", st, proj_kernel<<<blocks, 256, 0, st>>>(x, p->W_i, p->b_i, u, N, p->m, 3 * p->n));
+    DEER_KERNEL("proj_kernel", st, proj_kernel<<<blocks, 256, 0, st>>>(x, p->W_i, p->b_i, u, N, m, n3));
+    return DEER_OK;
+}
+
+template <int N> static int launch_cell_wide(CellArgs c, cudaStream_t st)
+{
+    using C = CellWide<N>;
+    int rc;
+    if ((rc = opt_in_smem((const void *)cell_wide_kernel<N>, C::SMEM)) != DEER_OK) return rc;
+    const size_t total = (size_t)c.B * c.T;
+    const size_t tiles = (total + C::PT - 1) / C::PT;
+    const size_t per_sm = (200 * 1024) / C::SMEM;
+    const size_t cap = (size_t)num_sms() * (per_sm > 4 ? 4 : per_sm);
+    const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
+    DEER_KERNEL("cell_wide_kernel", st, cell_wide_kernel<N><<<blocks, C::THREADS, C::SMEM, st>>>(c));
     return DEER_OK;
 }
 
@@ -352,6 +381,14 @@ static int run_cell(CellArgs c, cudaStream_t st)
         case 4: return launch_cell_small<4>(c, st);
         case 8: return launch_cell_small<8>(c, st);
         default: break;
+        }
+        if (c.u && (((uintptr_t)c.W_h) & 15) == 0) {
+            switch (c.n) {
+            case 16: return launch_cell_wide<16>(c, st);
+            case 32: return launch_cell_wide<32>(c, st);
+            case 64: return launch_cell_wide<64>(c, st);
+            default: break;
+            }
         }
     }
     const int n = c.n;
