@@ -15,6 +15,7 @@
 #include "scan_onepass.cuh"
 #include "scan_warp8.cuh"
 #include "scan_warpn.cuh"
+#include "scan_cta64.cuh"
 #include "cell_wide.cuh"
 
 namespace deer {
@@ -91,6 +92,7 @@ static int onepass_tile_len(int n)
     case 8: return use_warp8() ? Warp8::L : OnePass<8>::L;
     case 16: return WarpN<16>::L;
     case 32: return WarpN<32>::L;
+    case 64: return Cta64::L;
     default: return 0;
     }
 }
@@ -258,6 +260,50 @@ static int launch_warpn(ScanArgs a, OnePassWs w, cudaStream_t st)
     return DEER_OK;
 }
 
+template <bool REV>
+static int launch_cta64(ScanArgs a, OnePassWs w, cudaStream_t st)
+{
+    using C = Cta64;
+    static int occ = 0;
+    auto kern = scan_cta64_kernel<REV>;
+    if (!occ) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(cta64)"); return DEER_ERR_CUDA; }
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, C::THREADS, C::SMEM);
+        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(cta64)"); return DEER_ERR_CUDA; }
+        int cap = 8;
+        if (const char *d = getenv("DEER_WN_CTAS")) cap = atoi(d);
+        occ = o < cap ? o : cap;
+        if (occ < 1) occ = 1;
+    }
+    size_t tiles = (size_t)a.B * w.nch;
+    size_t resident = (size_t)num_sms() * occ;
+    int R = (a.B + C::RES_WARPS - 1) / C::RES_WARPS;
+    if (R > 16) R = 16;
+    const int per_cta_cap = C::RES_WARPS * C::MAX_SEQ_PER_WARP;
+    if ((a.B + per_cta_cap - 1) / per_cta_cap > R) R = (a.B + per_cta_cap - 1) / per_cta_cap;
+    w.resolvers = R;
+    size_t want = tiles + (size_t)R;
+    unsigned grid = (unsigned)(want < resident ? want : resident);
+    if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
+    int Wd = 8;
+    if (Wd > w.nch) Wd = w.nch;
+    w.Wd = Wd;
+    w.nwin = (w.nch + Wd - 1) / Wd;
+    w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
+    w.debug = 0;
+    {
+        size_t words = tiles * (size_t)(C::N + 1);
+        unsigned pb = (unsigned)((words + 255) / 256);
+        if (pb > 592u) pb = 592u;
+        if (pb < 1u) pb = 1u;
+        DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)C::N));
+    }
+    DEER_KERNEL("scan_cta64_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
+    return DEER_OK;
+}
+
 static int scan_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
 {
     switch (a.n * 2 + (a.reverse ? 1 : 0)) {
@@ -273,6 +319,8 @@ static int scan_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
     case 33: return launch_warpn<16, true>(a, w, st);
     case 64: return launch_warpn<32, false>(a, w, st);
     case 65: return launch_warpn<32, true>(a, w, st);
+    case 128: return launch_cta64<false>(a, w, st);
+    case 129: return launch_cta64<true>(a, w, st);
     default: return DEER_ERR_UNSUPPORTED_N;
     }
 }

@@ -1,0 +1,407 @@
+// Single-pass scan for n = 64: one CTA (two warps) per chain, chain product on tensor cores.
+//
+// A 64 x 64 running product does not fit one warp's registers, so a tile is a single chain that
+// the CTA's two warps advance together: warp w keeps rows 32w .. 32w+31 of X = P^T in 2 x 8
+// accumulator fragments and both multiply by the same matrix,
+//       X <- X * M,   M = J_t^T (forward)  or  J_{t+1} (reverse),
+// 2 x 8 x 8 MMAs (m16n8k8) per warp and position, each issued three times on hi/lo TF32 splits.
+// The matrices of the tile stream through a shared-memory ring filled with 16-byte cp.async
+// copies; the 16-byte pieces of a row are XOR-swizzled so that the B-operand reads of both
+// directions (8-byte pieces of a row forward, scalars of a column in reverse) and the row /
+// column reads of the mat-vec are all free of bank conflicts.  beta (the state reached from
+// zero) is carried by an fp32 mat-vec chain, thread r owning component r; the same routine
+// replays the tile from its true entering state in the B item.
+// Tiles, items, resolvers, flags and bounded waits are those of scan_onepass.cuh.
+#pragma once
+#include "scan_warpn.cuh"
+
+namespace deer {
+
+struct Cta64 {
+    static constexpr int N = 64, NN = N * N, AGG = NN + N;
+    static constexpr int NT = 8;                       // 8-wide column / contraction blocks
+    static constexpr int MT = 2;                       // 16-high row blocks of X per warp
+    static constexpr int WARPS = 2, THREADS = 64;
+    static constexpr int L = 64;                       // positions per tile
+    static constexpr int Q = 2;                        // pending tiles per CTA
+    static constexpr int STAGES = 3;                   // ring depth (positions)
+    static constexpr int STAGE_FLOATS = NN + N;        // swizzled matrix, then the vector
+    static constexpr int RES_WARPS = 2;
+    static constexpr int SM_WORK = STAGES * STAGE_FLOATS + 2 * N;
+    static constexpr int SM_RES = RES_WARPS * (AGG + N);
+    static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
+    static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
+    static constexpr int MAX_SEQ_PER_WARP = 8;
+};
+
+// float offset of element (row, col) of a swizzled 64 x 64 matrix: the 16-byte piece index of the
+// row is XORed with 2 * ((row ^ (row >> 2)) & 3)
+__device__ __forceinline__ int sw64(int row, int col)
+{
+    return row * 64 + ((((col >> 2) ^ (((row ^ (row >> 2)) & 3) << 1)) << 2) | (col & 3));
+}
+
+template <int K> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(K) : "memory"); }
+
+// Resolver for n = 64: lane i holds components i and i + 32 of the running state; one aggregate
+// is staged per step (16.6 KB).
+__device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
+{
+    using C = Cta64;
+    constexpr int N = C::N, AGG = C::AGG, NN = C::NN;
+    float *stage = stage_all + (threadIdx.x >> 5) * (AGG + N);
+    float *ysm = stage + AGG;
+    int nseq = 0;
+    int pos[C::MAX_SEQ_PER_WARP];
+    float ya[C::MAX_SEQ_PER_WARP], yb[C::MAX_SEQ_PER_WARP];
+    unsigned fnext[C::MAX_SEQ_PER_WARP];
+#pragma unroll
+    for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
+        pos[k] = 0; ya[k] = 0.0f; yb[k] = 0.0f; fnext[k] = 0u;
+        const int s = rw + k * nrw;
+        if (s < a.B) {
+            nseq = k + 1;
+            if (a.y0) { ya[k] = a.y0[(size_t)s * N + lane]; yb[k] = a.y0[(size_t)s * N + 32 + lane]; }
+            if (lane < w.nch) fnext[k] = ld_acquire_u32(w.flags + (size_t)s * w.nch + lane);
+        }
+    }
+    int remaining = nseq;
+    unsigned spins = 0;
+    while (remaining > 0) {
+        bool progressed = false;
+#pragma unroll
+        for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
+            if (k >= nseq) break;
+            const int c0 = pos[k];
+            if (c0 >= w.nch) continue;
+            const int s = rw + k * nrw;
+            const unsigned *flags = w.flags + (size_t)s * w.nch;
+            const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
+            const int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
+            if (cnt == 0) {
+                fnext[k] = (c0 + lane < w.nch) ? ld_acquire_u32(flags + c0 + lane) : 0u;
+                continue;
+            }
+            progressed = true;
+            unsigned long long *out = w.starts + ((size_t)s * w.nch + c0) * N;
+            float y0v = ya[k], y1v = yb[k];
+            for (int q = 0; q < cnt; ++q) {
+                st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y0v));
+                st_relaxed_u64(out + q * N + 32 + lane, LL_FLAG | (unsigned long long)__float_as_uint(y1v));
+                const float4 *src = reinterpret_cast<const float4 *>(w.aggs + ((size_t)s * w.nch + c0 + q) * AGG);
+                float4 *dst = reinterpret_cast<float4 *>(stage);
+                for (int i0 = 0; i0 < AGG / 4; i0 += 32 * 8) {
+                    float4 v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        if (i < AGG / 4) v[u] = __ldcg(src + i);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        if (i < AGG / 4) dst[i] = v[u];
+                    }
+                }
+                ysm[lane] = y0v; ysm[32 + lane] = y1v;
+                __syncwarp();
+                float a0 = stage[NN + lane], a1 = stage[NN + 32 + lane];
+                const float *r0 = stage + lane * N, *r1 = stage + (32 + lane) * N;
+#pragma unroll 8
+                for (int i = 0; i < N; ++i) {           // skewed column order: conflict-free reads
+                    const int c = (i + lane) & (N - 1);
+                    const float yc = ysm[c];
+                    a0 = fmaf(r0[c], yc, a0);
+                    a1 = fmaf(r1[c], yc, a1);
+                }
+                y0v = a0; y1v = a1;
+                __syncwarp();
+            }
+            ya[k] = y0v; yb[k] = y1v;
+            pos[k] = c0 + cnt;
+            if (pos[k] >= w.nch) --remaining;
+            else fnext[k] = (pos[k] + lane < w.nch) ? ld_acquire_u32(flags + pos[k] + lane) : 0u;
+        }
+        if (progressed) spins = 0;
+        else if (!keep_spinning(a.st, spins)) return;
+    }
+}
+
+// X <- X * M for the warp's 32 rows; B operands read from the swizzled stage
+template <bool REV>
+__device__ __forceinline__ void chain_step64(float (&acc)[2][8][4], const float *Ms, int g, int t)
+{
+    float nacc[2][8][4];
+#pragma unroll
+    for (int mm = 0; mm < 2; ++mm)
+#pragma unroll
+        for (int nn = 0; nn < 8; ++nn)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) nacc[mm][nn][i] = 0.0f;
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+        unsigned ah[2][4], al[2][4];
+#pragma unroll
+        for (int mm = 0; mm < 2; ++mm) {
+            split_tf32(acc[mm][kk][0], ah[mm][0], al[mm][0]);
+            split_tf32(acc[mm][kk][2], ah[mm][1], al[mm][1]);
+            split_tf32(acc[mm][kk][1], ah[mm][2], al[mm][2]);
+            split_tf32(acc[mm][kk][3], ah[mm][3], al[mm][3]);
+        }
+#pragma unroll
+        for (int nn = 0; nn < 8; ++nn) {
+            float j0, j1;       // M[8kk+2t][8nn+g], M[8kk+2t+1][8nn+g]
+            if (!REV) {
+                const float2 f = *reinterpret_cast<const float2 *>(Ms + sw64(8 * nn + g, 8 * kk + 2 * t));
+                j0 = f.x; j1 = f.y;
+            } else {
+                j0 = Ms[sw64(8 * kk + 2 * t, 8 * nn + g)];
+                j1 = Ms[sw64(8 * kk + 2 * t + 1, 8 * nn + g)];
+            }
+            unsigned bh[2], bl[2];
+            split_tf32(j0, bh[0], bl[0]);
+            split_tf32(j1, bh[1], bl[1]);
+#pragma unroll
+            for (int mm = 0; mm < 2; ++mm) {
+                mma_tf32(nacc[mm][nn], al[mm], bh, nacc[mm][nn]);
+                mma_tf32(nacc[mm][nn], ah[mm], bl, nacc[mm][nn]);
+                mma_tf32(nacc[mm][nn], ah[mm], bh, nacc[mm][nn]);
+            }
+        }
+    }
+#pragma unroll
+    for (int mm = 0; mm < 2; ++mm)
+#pragma unroll
+        for (int nn = 0; nn < 8; ++nn)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[mm][nn][i] = nacc[mm][nn][i];
+}
+
+// component `i` of  M^T-form product + vector:  forward  sum_c J[i][c] y[c] + b[i],
+// reverse  sum_k J[k][i] y[k] + b[i]
+template <bool REV>
+__device__ __forceinline__ float matvec64(const float *Ms, const float *ycur, int i)
+{
+    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+    if (!REV) {
+        const int flip = (i >> 2) & 1;             // halves of a quarter-warp start on different pieces
+        const int sw = ((i ^ (i >> 2)) & 3) << 1;
+        const float *row = Ms + i * 64;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const int ch = k ^ flip;
+            const float4 jv = *reinterpret_cast<const float4 *>(row + ((ch ^ sw) << 2));
+            const float4 yv = *reinterpret_cast<const float4 *>(ycur + (ch << 2));
+            s0 = fmaf(jv.x, yv.x, s0); s1 = fmaf(jv.y, yv.y, s1);
+            s2 = fmaf(jv.z, yv.z, s2); s3 = fmaf(jv.w, yv.w, s3);
+        }
+    } else {
+#pragma unroll
+        for (int k4 = 0; k4 < 16; ++k4) {
+            const float4 yv = *reinterpret_cast<const float4 *>(ycur + 4 * k4);
+            s0 = fmaf(Ms[sw64(4 * k4, i)], yv.x, s0);
+            s1 = fmaf(Ms[sw64(4 * k4 + 1, i)], yv.y, s1);
+            s2 = fmaf(Ms[sw64(4 * k4 + 2, i)], yv.z, s2);
+            s3 = fmaf(Ms[sw64(4 * k4 + 3, i)], yv.w, s3);
+        }
+    }
+    return ((s0 + s1) + (s2 + s3)) + Ms[Cta64::NN + i];
+}
+
+template <bool REV>
+__global__ void __launch_bounds__(Cta64::THREADS) scan_cta64_kernel(ScanArgs a, OnePassWs w)
+{
+    using C = Cta64;
+    constexpr int N = C::N, NN = C::NN, AGG = C::AGG, Q = C::Q, S = C::STAGES;
+    if (loop_ended(a.st)) return;
+
+    extern __shared__ __align__(16) float smem_raw[];
+    float *sm = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    float *ring = sm;                              // S x (swizzled matrix, vector)
+    float *ybuf = ring + S * C::STAGE_FLOATS;      // 2 x N: running state of the mat-vec chain
+    __shared__ int s_kind, s_seq, s_c, s_abort, s_role;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int T = a.T;
+
+    if (tid == 0) {
+        s_abort = 0;
+        s_role = (int)atomicAdd(&a.st->role_counter, 1u);
+    }
+    __syncthreads();
+    if (s_role < w.resolvers) {
+        resolver64(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        return;
+    }
+    unsigned mb = 0;
+
+    auto decode = [&](unsigned id, int &seq, int &c) {
+        const unsigned j = id % (unsigned)w.Wd;
+        const unsigned ws_ = id / (unsigned)w.Wd;
+        seq = (int)(ws_ % (unsigned)a.B);
+        const unsigned win = ws_ / (unsigned)a.B;
+        c = (int)(win * (unsigned)w.Wd + j);
+        if (c >= w.nch) c = -1;
+    };
+    int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
+    bool exhausted = false;
+
+    for (;;) {
+        __syncthreads();
+        if (tid == 0) {
+            int kind = -1, seq = -1, c = -1;
+            bool want_b = false;
+            if (q_cnt > 0) {
+                want_b = (q_cnt == Q) || exhausted;
+                if (!want_b)
+                    want_b = ld_relaxed_u64(w.starts + ((size_t)q_seq[q_head] * w.nch + q_c[q_head]) * N) != 0ull;
+            }
+            if (!want_b && !exhausted) {
+                for (;;) {
+                    const unsigned id = atomicAdd(&a.st->tile_counter, 1u);
+                    if (id >= w.total_ids) { c = -1; break; }
+                    decode(id, seq, c);
+                    if (c >= 0) break;
+                }
+                if (c >= 0) {
+                    kind = 0;
+                    const int slot = (q_head + q_cnt) % Q;
+                    q_seq[slot] = seq; q_c[slot] = c; ++q_cnt;
+                } else {
+                    exhausted = true;
+                    want_b = q_cnt > 0;
+                }
+            }
+            if (want_b) {
+                kind = 1; seq = q_seq[q_head]; c = q_c[q_head];
+                q_head = (q_head + 1) % Q; --q_cnt;
+            }
+            s_kind = kind; s_seq = seq; s_c = c;
+        }
+        __syncthreads();
+        if (s_kind < 0 || s_abort) break;
+        const int kind = s_kind, seq = s_seq, c = s_c;
+        const int s0 = c * C::L;
+        const int cnt = min(C::L, T - s0);
+        const size_t tile_index = (size_t)seq * w.nch + c;
+        const float *Jseq = a.J + (size_t)seq * T * NN;
+        const float *bseq = a.b + (size_t)seq * T * N;
+
+        // stage of scan position s: forward J[s]; reverse J[T-s] (identity at s = 0); vector at t(s)
+        auto issue_stage = [&](int q) {
+            if (q < cnt) {
+                const int s = s0 + q;
+                float *dst = ring + (q % S) * C::STAGE_FLOATS;
+                if (REV && s == 0) {
+                    for (int j = tid; j < NN / 4; j += C::THREADS) {
+                        const int row = j >> 4, ch = j & 15;
+                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if ((row >> 2) == ch) {
+                            if ((row & 3) == 0) v.x = 1.0f;
+                            if ((row & 3) == 1) v.y = 1.0f;
+                            if ((row & 3) == 2) v.z = 1.0f;
+                            if ((row & 3) == 3) v.w = 1.0f;
+                        }
+                        *reinterpret_cast<float4 *>(dst + sw64(row, 4 * ch)) = v;
+                    }
+                } else {
+                    const float *src = REV ? Jseq + (size_t)(T - s) * NN : Jseq + (size_t)s * NN;
+#pragma unroll
+                    for (int u = 0; u < NN / 4 / C::THREADS; ++u) {
+                        const int j = tid + u * C::THREADS;
+                        cp_async16(dst + sw64(j >> 4, 4 * (j & 15)), src + 4 * j);
+                    }
+                }
+                const size_t tt = REV ? (size_t)(T - 1 - s) : (size_t)s;
+                if (tid < N / 4) cp_async16(dst + NN + 4 * tid, bseq + tt * N + 4 * tid);
+            }
+            cp_async_commit();
+        };
+
+        if (kind == 0) {
+            // ---------------------------------------------- A item
+            float acc[2][8][4];
+#pragma unroll
+            for (int mm = 0; mm < 2; ++mm)
+#pragma unroll
+                for (int nn = 0; nn < 8; ++nn) {
+                    const int r = 32 * warp + 16 * mm + g, cc = 8 * nn + 2 * t;
+                    acc[mm][nn][0] = (r == cc) ? 1.0f : 0.0f;
+                    acc[mm][nn][1] = (r == cc + 1) ? 1.0f : 0.0f;
+                    acc[mm][nn][2] = (r + 8 == cc) ? 1.0f : 0.0f;
+                    acc[mm][nn][3] = (r + 8 == cc + 1) ? 1.0f : 0.0f;
+                }
+            ybuf[tid] = 0.0f;
+#pragma unroll
+            for (int q = 0; q < S - 1; ++q) issue_stage(q);
+#pragma unroll 1
+            for (int q = 0; q < cnt; ++q) {
+                cp_async_wait<S - 2>();
+                __syncthreads();
+                issue_stage(q + S - 1);
+                const float *Ms = ring + (q % S) * C::STAGE_FLOATS;
+                chain_step64<REV>(acc, Ms, g, t);
+                ybuf[((q + 1) & 1) * N + tid] = matvec64<REV>(Ms, ybuf + (q & 1) * N, tid);
+            }
+            cp_async_wait<0>();
+            __syncthreads();
+            // X = P^T in fragments  ->  P row-major, then beta
+            float *dst = w.aggs + tile_index * AGG;
+#pragma unroll
+            for (int mm = 0; mm < 2; ++mm)
+#pragma unroll
+                for (int nn = 0; nn < 8; ++nn) {
+                    const int r = 32 * warp + 16 * mm + g, cc = 8 * nn + 2 * t;
+                    dst[cc * N + r] = acc[mm][nn][0];
+                    dst[(cc + 1) * N + r] = acc[mm][nn][1];
+                    dst[cc * N + r + 8] = acc[mm][nn][2];
+                    dst[(cc + 1) * N + r + 8] = acc[mm][nn][3];
+                }
+            dst[NN + tid] = ybuf[(cnt & 1) * N + tid];
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) st_release_u32(w.flags + tile_index, 1u);
+            continue;
+        }
+
+        // -------------------------------------------------- B item
+#pragma unroll
+        for (int q = 0; q < S - 1; ++q) issue_stage(q);
+        {
+            const unsigned long long *src = w.starts + tile_index * N;
+            unsigned spins = 0;
+            bool ok = true;
+            for (;;) {
+                const unsigned long long v = ld_relaxed_u64(src + tid);
+                if (v != 0ull) { ybuf[tid] = __uint_as_float((unsigned)(v & 0xffffffffull)); break; }
+                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+            }
+            if (!ok) s_abort = 1;
+        }
+#pragma unroll 1
+        for (int q = 0; q < cnt; ++q) {
+            cp_async_wait<S - 2>();
+            __syncthreads();
+            if (s_abort) break;
+            issue_stage(q + S - 1);
+            const float *Ms = ring + (q % S) * C::STAGE_FLOATS;
+            const float yn = matvec64<REV>(Ms, ybuf + (q & 1) * N, tid);
+            ybuf[((q + 1) & 1) * N + tid] = yn;
+            const int s = s0 + q;
+            const size_t vb = ((size_t)seq * T + (REV ? (size_t)(T - 1 - s) : (size_t)s)) * N + tid;
+            if (a.yold) mb = max(mb, absdiff_bits(yn, __ldg(a.yold + vb)));
+            a.y[vb] = yn;
+        }
+        cp_async_wait<0>();
+        if (s_abort) break;
+    }
+    cp_async_wait<0>();
+    if (a.yold) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+        if (lane == 0 && mb) atomicMax(&a.st->err_bits, mb);
+    }
+}
+
+}  // namespace deer
