@@ -21,6 +21,54 @@ template <int N> struct CellWide {
     static constexpr size_t SMEM = sizeof(float) * (3 * N * N + 3 * N + PT * HS + 4 * PT * N);
 };
 
+// h_prev of the tile's positions -> shared memory rows of stride HS (zero rows past the end)
+template <int N>
+__device__ __forceinline__ void stage_h_prev(float *sH, const float *y, const float *y0, int T, size_t e0, int np, int tid)
+{
+    using C = CellWide<N>;
+    for (int idx = tid; idx < C::PT * (N / 4); idx += C::THREADS) {
+        const int p = idx / (N / 4), k4 = idx % (N / 4);
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (p < np) {
+            const size_t e = e0 + p;
+            const size_t seq = e / T;
+            const float *hp = (e - seq * T == 0) ? y0 + seq * N : y + (e - 1) * N;
+            v = *reinterpret_cast<const float4 *>(hp + 4 * k4);
+        }
+        *reinterpret_cast<float4 *>(sH + p * C::HS + 4 * k4) = v;
+    }
+}
+
+// bias-free hidden projections of P positions for output row gi:  g*[q] = sum_k W_h*[gi][k] h_q[k]
+template <int N>
+__device__ __forceinline__ void gate_accumulate(float (&gr)[CellWide<N>::P], float (&gz)[CellWide<N>::P],
+                                                float (&gq)[CellWide<N>::P], const float *sWT,
+                                                const float *hrow, int gi)
+{
+    using C = CellWide<N>;
+#pragma unroll
+    for (int q = 0; q < C::P; ++q) { gr[q] = 0.0f; gz[q] = 0.0f; gq[q] = 0.0f; }
+#pragma unroll 2
+    for (int k = 0; k < N; k += 4) {
+        float4 h4[C::P];
+#pragma unroll
+        for (int q = 0; q < C::P; ++q) h4[q] = *reinterpret_cast<const float4 *>(hrow + q * C::HS + k);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            const float wr = sWT[(k + kk) * 3 * N + gi];
+            const float wz = sWT[(k + kk) * 3 * N + N + gi];
+            const float wn = sWT[(k + kk) * 3 * N + 2 * N + gi];
+#pragma unroll
+            for (int q = 0; q < C::P; ++q) {
+                const float h = kk == 0 ? h4[q].x : kk == 1 ? h4[q].y : kk == 2 ? h4[q].z : h4[q].w;
+                gr[q] = fmaf(wr, h, gr[q]);
+                gz[q] = fmaf(wz, h, gz[q]);
+                gq[q] = fmaf(wn, h, gq[q]);
+            }
+        }
+    }
+}
+
 // Gate phase: thread (row i, group) accumulates the three hidden projections of its P positions
 // from W_h^T in shared memory (lanes = consecutive rows: conflict-free) and h_prev broadcast
 // from the staged tile; writes rhs = f - J h_prev using
@@ -70,25 +118,12 @@ __global__ void __launch_bounds__(256) cell_wide_kernel(CellArgs a)
     for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const size_t e0 = tile * C::PT;
         const int np = (int)((total - e0) < (size_t)C::PT ? (total - e0) : (size_t)C::PT);
-        // stage h_prev of the tile's positions
-        for (int idx = tid; idx < C::PT * (N / 4); idx += C::THREADS) {
-            const int p = idx / (N / 4), k4 = idx % (N / 4);
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (p < np) {
-                const size_t e = e0 + p;
-                const size_t seq = e / a.T;
-                const float *hp = (e - seq * a.T == 0) ? a.y0 + seq * N : a.y + (e - 1) * N;
-                v = *reinterpret_cast<const float4 *>(hp + 4 * k4);
-            }
-            *reinterpret_cast<float4 *>(sH + p * C::HS + 4 * k4) = v;
-        }
+        stage_h_prev<N>(sH, a.y, a.y0, a.T, e0, np, tid);
         __syncthreads();
 
         // ---- gate phase
         {
             float gr[C::P], gz[C::P], gq[C::P];
-#pragma unroll
-            for (int q = 0; q < C::P; ++q) { gr[q] = 0.0f; gz[q] = 0.0f; gq[q] = 0.0f; }
             const float *hrow = sH + (grp * C::P) * C::HS;
             float ur[C::P], uz[C::P], un[C::P];
 #pragma unroll
@@ -97,25 +132,7 @@ __global__ void __launch_bounds__(256) cell_wide_kernel(CellArgs a)
                 const float *ue = a.u + (e0 + (p < np ? p : 0)) * 3 * N;
                 ur[q] = ue[gi]; uz[q] = ue[N + gi]; un[q] = ue[2 * N + gi];
             }
-#pragma unroll 2
-            for (int k = 0; k < N; k += 4) {
-                float4 h4[C::P];
-#pragma unroll
-                for (int q = 0; q < C::P; ++q) h4[q] = *reinterpret_cast<const float4 *>(hrow + q * C::HS + k);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const float wr = sWT[(k + kk) * 3 * N + gi];
-                    const float wz = sWT[(k + kk) * 3 * N + N + gi];
-                    const float wn = sWT[(k + kk) * 3 * N + 2 * N + gi];
-#pragma unroll
-                    for (int q = 0; q < C::P; ++q) {
-                        const float h = kk == 0 ? h4[q].x : kk == 1 ? h4[q].y : kk == 2 ? h4[q].z : h4[q].w;
-                        gr[q] = fmaf(wr, h, gr[q]);
-                        gz[q] = fmaf(wz, h, gz[q]);
-                        gq[q] = fmaf(wn, h, gq[q]);
-                    }
-                }
-            }
+            gate_accumulate<N>(gr, gz, gq, sWT, hrow, gi);
 #pragma unroll
             for (int q = 0; q < C::P; ++q) {
                 const int p = grp * C::P + q;
@@ -169,14 +186,15 @@ __global__ void __launch_bounds__(256) cell_wide_kernel(CellArgs a)
 }
 
 // ------------------------------------------------------------------ a0: u = x W_i^T + b_i, tiled
-// blockDim.x = n3 * G.  Thread (output g, group) keeps PP positions in registers; W_i^T sits in
+// (also dx = dG_i W_i of the VJP: the same product with the weights already in [input][output]
+// order and no bias).  blockDim.x = n3 * G.  Thread (output g, group) keeps PP positions in registers; W_i^T sits in
 // shared memory (lanes = consecutive outputs: conflict-free), x is staged per tile and read as a
 // broadcast.  Loads of x and stores of u are coalesced.
 constexpr int PROJ_PP = 8;
 
 __global__ void __launch_bounds__(256) proj_tiled_kernel(const float *__restrict__ x, const float *__restrict__ W_i,
                                                          const float *__restrict__ b_i, float *__restrict__ u,
-                                                         size_t N, int m, int n3, int G)
+                                                         size_t N, int m, int n3, int G, int wt_given)
 {
     extern __shared__ __align__(16) float smp[];
     float *sWT = smp;                    // [m][n3]
@@ -185,13 +203,17 @@ __global__ void __launch_bounds__(256) proj_tiled_kernel(const float *__restrict
     const int nthr = n3 * G;
     const int PT = G * PROJ_PP;
     const int xs = m + 1;
-    for (int idx = tid; idx < n3 * m; idx += blockDim.x) {
-        const int g = idx / m, k = idx % m;
-        sWT[k * n3 + g] = W_i[idx];
+    if (wt_given) {                      // weights already stored [m][n3]
+        for (int idx = tid; idx < n3 * m; idx += blockDim.x) sWT[idx] = W_i[idx];
+    } else {
+        for (int idx = tid; idx < n3 * m; idx += blockDim.x) {
+            const int g = idx / m, k = idx % m;
+            sWT[k * n3 + g] = W_i[idx];
+        }
     }
     const bool active = tid < nthr;
     const int g = active ? tid % n3 : 0, grp = active ? tid / n3 : 0;
-    const float bias = b_i[g];
+    const float bias = b_i ? b_i[g] : 0.0f;
     const size_t ntiles = (N + PT - 1) / PT;
     for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const size_t e0 = tile * PT;

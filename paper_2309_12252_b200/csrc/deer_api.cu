@@ -17,6 +17,7 @@
 #include "scan_warpn.cuh"
 #include "scan_cta64.cuh"
 #include "cell_wide.cuh"
+#include "vjp_wide.cuh"
 
 namespace deer {
 
@@ -358,22 +359,30 @@ static int run_scan(ScanArgs a, const ScanWs &w, int flags, cudaStream_t st)
     return scan_generic(a, st);
 }
 
+// out[e][g] = bias[g] + sum_k W[g][k] in[e][k]   (wt_given: W is stored [k][g]; bias may be null)
+static int run_affine(const float *in, const float *W, const float *bias, float *out, size_t N, int m, int n3,
+                      int wt_given, cudaStream_t st)
+{
+    int G = 256 / n3;
+    while (G > 1 && sizeof(float) * (size_t)G * PROJ_PP * (m + 1) > 64 * 1024) --G;
+    const size_t sm = sizeof(float) * ((size_t)m * n3 + (size_t)G * PROJ_PP * (m + 1));
+    if (G < 1 || sm > 200 * 1024) return DEER_ERR_UNSUPPORTED_N;
+    int rc;
+    if ((rc = opt_in_smem((const void *)proj_tiled_kernel, sm)) != DEER_OK) return rc;
+    const size_t tiles = (N + (size_t)G * PROJ_PP - 1) / ((size_t)G * PROJ_PP);
+    const size_t cap = (size_t)num_sms() * 8;
+    const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
+    const int threads = (n3 * G + 31) / 32 * 32;
+    DEER_KERNEL("proj_tiled_kernel", st,
+                proj_tiled_kernel<<<blocks, threads, sm, st>>>(in, W, bias, out, N, m, n3, G, wt_given));
+    return DEER_OK;
+}
+
 static int run_proj(const deer_gru_params *p, const float *x, float *u, size_t N, cudaStream_t st)
 {
     const int n3 = 3 * p->n, m = p->m;
-    const int G = 256 / n3;
-    const size_t sm = sizeof(float) * ((size_t)m * n3 + (size_t)G * PROJ_PP * (m + 1));
-    if (G >= 1 && sm <= 200 * 1024) {
-        int rc;
-        if ((rc = opt_in_smem((const void *)proj_tiled_kernel, sm)) != DEER_OK) return rc;
-        const size_t tiles = (N + (size_t)G * PROJ_PP - 1) / ((size_t)G * PROJ_PP);
-        const size_t cap = (size_t)num_sms() * 8;
-        const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
-        const int threads = (n3 * G + 31) / 32 * 32;
-        DEER_KERNEL("proj_tiled_kernel", st,
-                    proj_tiled_kernel<<<blocks, threads, sm, st>>>(x, p->W_i, p->b_i, u, N, m, n3, G));
-        return DEER_OK;
-    }
+    if (n3 <= 256 && sizeof(float) * ((size_t)m * n3 + (size_t)PROJ_PP * (m + 1)) <= 200 * 1024)
+        return run_affine(x, p->W_i, p->b_i, u, N, m, n3, 0, st);
     size_t total = N * (size_t)n3;
     unsigned blocks = (unsigned)((total + 255) / 256);
     DEER_KERNEL("proj_kernel", st, proj_kernel<<<blocks, 256, 0, st>>>(x, p->W_i, p->b_i, u, N, m, n3));
@@ -449,6 +458,31 @@ static int run_cell(CellArgs c, cudaStream_t st)
     unsigned blocks = (unsigned)((N + epb - 1) / epb);
     DEER_KERNEL("cell_kernel", st, cell_kernel<<<blocks, threads, sm, st>>>(c));
     return DEER_OK;
+}
+
+template <int N> static int launch_vjp_cell_wide_n(VjpArgs v, cudaStream_t st)
+{
+    using C = CellWide<N>;
+    const size_t sm = sizeof(float) * (3 * N * N + 3 * N + C::PT * C::HS);
+    int rc;
+    if ((rc = opt_in_smem((const void *)vjp_cell_wide_kernel<N>, sm)) != DEER_OK) return rc;
+    const size_t total = (size_t)v.B * v.T;
+    const size_t tiles = (total + C::PT - 1) / C::PT;
+    const size_t per_sm = (200 * 1024) / sm;
+    const size_t cap = (size_t)num_sms() * (per_sm > 4 ? 4 : per_sm);
+    const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
+    DEER_KERNEL("vjp_cell_wide_kernel", st, vjp_cell_wide_kernel<N><<<blocks, C::THREADS, sm, st>>>(v));
+    return DEER_OK;
+}
+
+static int launch_vjp_cell_wide(VjpArgs v, cudaStream_t st)
+{
+    switch (v.n) {
+    case 16: return launch_vjp_cell_wide_n<16>(v, st);
+    case 32: return launch_vjp_cell_wide_n<32>(v, st);
+    case 64: return launch_vjp_cell_wide_n<64>(v, st);
+    default: return DEER_ERR_UNSUPPORTED_N;
+    }
 }
 
 static bool valid_sizes(int B, int T, int n, int m)
@@ -665,11 +699,16 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
 
     {
         VjpArgs v{p->W_h, p->b_h, w.u, y, y0, w.lam, w.dGi, w.dGh, B, T, n};
-        size_t sm = sizeof(float) * (3 * n * (n + 1) + 3 * n);
-        if ((rc = opt_in_smem((const void *)vjp_cell_kernel, sm)) != DEER_OK) return rc;
-        int epb = 256 / n;
-        unsigned blocks = (unsigned)((N + epb - 1) / epb);
-        DEER_KERNEL("vjp_cell_kernel", st, vjp_cell_kernel<<<blocks, 256, sm, st>>>(v));
+        const bool aligned = (((uintptr_t)y | (uintptr_t)y0) & 15) == 0;
+        if (aligned && (n == 16 || n == 32 || n == 64)) {
+            if ((rc = launch_vjp_cell_wide(v, st)) != DEER_OK) return rc;
+        } else {
+            size_t sm = sizeof(float) * (3 * n * (n + 1) + 3 * n);
+            if ((rc = opt_in_smem((const void *)vjp_cell_kernel, sm)) != DEER_OK) return rc;
+            int epb = 256 / n;
+            unsigned blocks = (unsigned)((N + epb - 1) / epb);
+            DEER_KERNEL("vjp_cell_kernel", st, vjp_cell_kernel<<<blocks, 256, sm, st>>>(v));
+        }
     }
     const int P = (int)(N < (size_t)WGRAD_P ? N : (size_t)WGRAD_P);
     for (int side = 0; side < 2; ++side) {
@@ -681,21 +720,29 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
         wa.T = T; wa.n3 = n3; wa.K = side == 0 ? m : n;
         wa.N = N; wa.slice = (N + P - 1) / P;
         wa.partial = w.partial;
-        int tile = 32;
-        while (tile > 1 && sizeof(float) * tile * (size_t)(n3 + wa.K + 1) > 160 * 1024) tile >>= 1;
-        wa.tile = tile;
-        size_t sm = sizeof(float) * tile * (size_t)(n3 + wa.K + 1);
-        if ((rc = opt_in_smem((const void *)wgrad_partial_kernel, sm)) != DEER_OK) return rc;
         int outs = n3 * (wa.K + 1);
-        dim3 grid(P, (outs + 255) / 256);
-        DEER_KERNEL("wgrad_partial_kernel", st, wgrad_partial_kernel<<<grid, 256, sm, st>>>(wa));
+        if (n3 % 16 == 0 && n3 <= 192 && wa.K <= 64) {
+            DEER_KERNEL("wgrad_mma_kernel", st, wgrad_mma_kernel<<<P, 32 * (n3 / 16), 0, st>>>(wa));
+        } else {
+            int tile = 32;
+            while (tile > 1 && sizeof(float) * tile * (size_t)(n3 + wa.K + 1) > 160 * 1024) tile >>= 1;
+            wa.tile = tile;
+            size_t sm = sizeof(float) * tile * (size_t)(n3 + wa.K + 1);
+            if ((rc = opt_in_smem((const void *)wgrad_partial_kernel, sm)) != DEER_OK) return rc;
+            dim3 grid(P, (outs + 255) / 256);
+            DEER_KERNEL("wgrad_partial_kernel", st, wgrad_partial_kernel<<<grid, 256, sm, st>>>(wa));
+        }
         DEER_KERNEL("wgrad_final_kernel", st, wgrad_final_kernel<<<(outs + 255) / 256, 256, 0, st>>>(w.partial, P, n3, wa.K,
                                                                 side == 0 ? g->dW_i : g->dW_h,
                                                                 side == 0 ? g->db_i : g->db_h));
     }
     if (dx) {
-        size_t total = N * (size_t)m;
-        DEER_KERNEL("vjp_dx_kernel", st, vjp_dx_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w.dGi, p->W_i, dx, N, m, n3));
+        if (m >= 32 && m <= 256) {
+            if ((rc = run_affine(w.dGi, p->W_i, nullptr, dx, N, n3, m, 1, st)) != DEER_OK) return rc;
+        } else {
+            size_t total = N * (size_t)m;
+            DEER_KERNEL("vjp_dx_kernel", st, vjp_dx_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w.dGi, p->W_i, dx, N, m, n3));
+        }
     }
     if (dy0) {
         DEER_KERNEL("vjp_dy0_kernel", st, vjp_dy0_kernel<<<(B * n + 127) / 128, 128, 0, st>>>(w.J, w.lam, dy0, B, T, n));

@@ -1,0 +1,147 @@
+// Cell VJP (step a8) for n in {16, 32, 64}: gate gradients with the gate phase of cell_wide.cuh,
+// and the parameter-gradient contraction  dW = dG^T V  over all B*T positions on tensor cores.
+#pragma once
+#include "cell_wide.cuh"
+#include "kernels_generic.cuh"
+#include "scan_warp8.cuh"
+
+namespace deer {
+
+// dGi = [da_r, da_z, da_n], dGh = [da_r, da_z, dq] at every position (gates recomputed from u, y_prev).
+template <int N>
+__global__ void __launch_bounds__(256) vjp_cell_wide_kernel(VjpArgs a)
+{
+    using C = CellWide<N>;
+    extern __shared__ __align__(16) float sm[];
+    float *sWT = sm;                           // [N][3N]
+    float *sB = sWT + 3 * N * N;               // [3N]
+    float *sH = sB + 3 * N;                    // [PT][HS]
+    const int tid = threadIdx.x;
+    for (int idx = tid; idx < 3 * N * N; idx += C::THREADS) {
+        const int g = idx / N, k = idx % N;
+        sWT[k * 3 * N + g] = a.W_h[idx];
+    }
+    for (int idx = tid; idx < 3 * N; idx += C::THREADS) sB[idx] = a.b_h[idx];
+    __syncthreads();
+    const int gi = tid % N, grp = tid / N;
+    const float bR = sB[gi], bZ = sB[N + gi], bN = sB[2 * N + gi];
+    const size_t total = (size_t)a.B * a.T;
+    const size_t ntiles = (total + C::PT - 1) / C::PT;
+    for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const size_t e0 = tile * C::PT;
+        const int np = (int)((total - e0) < (size_t)C::PT ? (total - e0) : (size_t)C::PT);
+        __syncthreads();
+        stage_h_prev<N>(sH, a.y, a.y0, a.T, e0, np, tid);
+        __syncthreads();
+        float gr[C::P], gz[C::P], gq[C::P], ur[C::P], uz[C::P], un[C::P], lam[C::P];
+        const float *hrow = sH + (grp * C::P) * C::HS;
+#pragma unroll
+        for (int q = 0; q < C::P; ++q) {
+            const int p = grp * C::P + q;
+            const size_t e = e0 + (p < np ? p : 0);
+            const float *ue = a.u + e * 3 * N;
+            ur[q] = ue[gi]; uz[q] = ue[N + gi]; un[q] = ue[2 * N + gi];
+            lam[q] = a.lam[e * N + gi];
+        }
+        gate_accumulate<N>(gr, gz, gq, sWT, hrow, gi);
+#pragma unroll
+        for (int q = 0; q < C::P; ++q) {
+            const int p = grp * C::P + q;
+            if (p < np) {
+                const size_t e = e0 + p;
+                const float qn = gq[q] + bN;
+                const float r = sigmoidf_acc(ur[q] + (gr[q] + bR));
+                const float z = sigmoidf_acc(uz[q] + (gz[q] + bZ));
+                const float c = tanhf(un[q] + r * qn);
+                const float hi = hrow[q * C::HS + gi];
+                const float dan = lam[q] * (1.0f - z) * (1.0f - c * c);
+                const float daz = lam[q] * (hi - c) * z * (1.0f - z);
+                const float dar = dan * qn * r * (1.0f - r);
+                const float dq = dan * r;
+                float *gI = a.dGi + e * 3 * N, *gH = a.dGh + e * 3 * N;
+                gI[gi] = dar; gI[N + gi] = daz; gI[2 * N + gi] = dan;
+                gH[gi] = dar; gH[N + gi] = daz; gH[2 * N + gi] = dq;
+            }
+        }
+    }
+}
+
+// Stage 1 of the deterministic parameter-gradient reduction on tensor cores.
+//   out[g][k] = sum_e dG[e][g] V[e][k]   (k == K: bias column, V = 1)
+// CTA p covers slice p of the positions; warp w owns output rows 16w .. 16w+15 and all (K+7)/8
+// column blocks.  The contraction index is the position: per step of 8 positions the A fragment
+// is dG^T (rows = gates), the B fragments are V; both are read straight from global memory as
+// 32-byte row segments.  Products use the 3 x TF32 split (fp32-level accuracy); the bias column is
+// the running sum of the A fragment.  blockDim.x = 32 * n3 / 16, K <= 64.
+__global__ void __launch_bounds__(384) wgrad_mma_kernel(WgradArgs a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int n3 = a.n3, K = a.K, K1 = K + 1;
+    const int nb = (K + 7) >> 3;
+    const size_t e0 = (size_t)blockIdx.x * a.slice;
+    const size_t e1 = e0 + a.slice < a.N ? e0 + a.slice : a.N;
+    float acc[8][4];
+#pragma unroll
+    for (int nn = 0; nn < 8; ++nn)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nn][i] = 0.0f;
+    float bs0 = 0.0f, bs1 = 0.0f;
+    const int row = 16 * warp + g;
+    auto vrow = [&](size_t e) -> const float * {
+        if (!a.shifted) return a.V + e * K;
+        const size_t seq = e / a.T;
+        return (e - seq * a.T == 0) ? a.y0 + seq * K : a.V + (e - 1) * K;
+    };
+#pragma unroll 1
+    for (size_t e = e0; e < e1; e += 8) {
+        const size_t p0 = e + t, p1 = e + t + 4;
+        const bool v0 = p0 < e1, v1 = p1 < e1;
+        float av[4];
+        av[0] = v0 ? __ldg(a.dG + p0 * n3 + row) : 0.0f;
+        av[1] = v0 ? __ldg(a.dG + p0 * n3 + row + 8) : 0.0f;
+        av[2] = v1 ? __ldg(a.dG + p1 * n3 + row) : 0.0f;
+        av[3] = v1 ? __ldg(a.dG + p1 * n3 + row + 8) : 0.0f;
+        const float *r0 = v0 ? vrow(p0) : a.V, *r1 = v1 ? vrow(p1) : a.V;
+        float bv[8][2];
+#pragma unroll
+        for (int nn = 0; nn < 8; ++nn) {
+            const int col = 8 * nn + g;
+            const bool cv = nn < nb && col < K;
+            bv[nn][0] = (cv && v0) ? __ldg(r0 + col) : 0.0f;
+            bv[nn][1] = (cv && v1) ? __ldg(r1 + col) : 0.0f;
+        }
+        bs0 += av[0] + av[2];
+        bs1 += av[1] + av[3];
+        unsigned ah[4], al[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) split_tf32(av[i], ah[i], al[i]);
+#pragma unroll
+        for (int nn = 0; nn < 8; ++nn) {
+            if (nn < nb) {
+                unsigned bh[2], bl[2];
+                split_tf32(bv[nn][0], bh[0], bl[0]);
+                split_tf32(bv[nn][1], bh[1], bl[1]);
+                mma_tf32(acc[nn], al, bh, acc[nn]);
+                mma_tf32(acc[nn], ah, bl, acc[nn]);
+                mma_tf32(acc[nn], ah, bh, acc[nn]);
+            }
+        }
+    }
+    float *out = a.partial + (size_t)blockIdx.x * n3 * K1;
+#pragma unroll
+    for (int nn = 0; nn < 8; ++nn) {
+        if (nn < nb) {
+            const int col = 8 * nn + 2 * t;
+            if (col < K) { out[row * K1 + col] = acc[nn][0]; out[(row + 8) * K1 + col] = acc[nn][2]; }
+            if (col + 1 < K) { out[row * K1 + col + 1] = acc[nn][1]; out[(row + 8) * K1 + col + 1] = acc[nn][3]; }
+        }
+    }
+    bs0 += __shfl_xor_sync(0xffffffffu, bs0, 1);
+    bs0 += __shfl_xor_sync(0xffffffffu, bs0, 2);
+    bs1 += __shfl_xor_sync(0xffffffffu, bs1, 1);
+    bs1 += __shfl_xor_sync(0xffffffffu, bs1, 2);
+    if (t == 0) { out[row * K1 + K] = bs0; out[(row + 8) * K1 + K] = bs1; }
+}
+
+}  // namespace deer
