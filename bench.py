@@ -209,60 +209,96 @@ def run_scan_only(args):
                           input_mb=(n * n + n) * 4 * B * T / 1e6)))
 
 
-def run_eval_only(args):
-    """deer_gru_eval (and optionally deer_gru_vjp) at an arbitrary sweep point: one JSON line."""
+def eval_point(bd, synth, device, n, m, B, T, flags, steps, warmup, vjp=False, breakdown=True):
+    """deer_gru_eval (optionally deer_gru_vjp) at one sweep point (x ~ N(0,1), y0 = 0): a dict of timings."""
     import torch
-    from paper_2309_12252_b200 import binding as bd
-    from paper_2309_12252_b200 import synth
-    device = torch.device("cuda", 0)
-    torch.cuda.set_device(0)
-    n, m, B, T = args.n, (args.m or args.n), args.B, args.T
     p = bd.GruParamsDev.from_numpy(synth.gru_params(n, m, 0, tag=f"sweep{n}/gru"))
     g = torch.Generator(device=device); g.manual_seed(0)
     x = torch.randn((B, T, m), device=device, generator=g)
     y0 = torch.zeros((B, n), device=device)
     y = torch.empty((B, T, n), device=device)
-    ws = bd.alloc_workspace(bd.DEER_OP_EVAL, B, T, n, m, args.flags, device)
+    ws = bd.alloc_workspace(bd.DEER_OP_EVAL, B, T, n, m, flags, device)
     stream = torch.cuda.current_stream()
-    run = lambda: bd.deer_gru_eval(p, x, y0, 1e-4, 100, y, ws, args.flags, stream)
-    for _ in range(max(args.warmup, 1)):
+    run = lambda: bd.deer_gru_eval(p, x, y0, 1e-4, 100, y, ws, flags, stream)
+    for _ in range(max(warmup, 1)):
         r = run()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     torch.cuda.synchronize()
     for a, b in ev:
         a.record(stream); r = run(); b.record(stream)
     torch.cuda.synchronize()
     ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
-    bd.lib().deer_profile_enable(1)
-    run()
-    torch.cuda.synchronize()
-    bd.lib().deer_profile_enable(0)
-    prof = read_profile(bd)
-    out = dict(mode="eval", n=n, m=m, B=B, T=T, flags=args.flags, ms=ms, steps_per_s=B * T / (ms * 1e-3),
-               iters=r.iters, err=r.err, status=r.status,
-               kernels={k: dict(launches=v["launches"], ms=round(v["total_ms"], 4)) for k, v in prof.items()})
-    if args.vjp:
+    out = dict(n=n, m=m, B=B, T=T, flags=flags, ms=ms, steps_per_s=B * T / (ms * 1e-3),
+               iters=r.iters, err=r.err, status=r.status)
+    if breakdown:
+        bd.lib().deer_profile_enable(1)
+        run()
+        torch.cuda.synchronize()
+        bd.lib().deer_profile_enable(0)
+        prof = read_profile(bd)
+        out["kernels"] = {k: dict(launches=v["launches"], ms=round(v["total_ms"], 4)) for k, v in prof.items()}
+        scan_ms = sum(v["total_ms"] for k, v in prof.items() if k.startswith("scan_") and "prep" not in k or k.startswith("gen_"))
+        if scan_ms > 0 and r.iters > 0:
+            pk = peaks()
+            per = scan_ms / r.iters
+            out["scan_ms_per_iter"] = per
+            out["scan_frac_hbm"] = scan_bytes_per_position(n) * B * T / (per * 1e-3) / 1e9 / pk["hbm_gbs"]
+    if vjp:
         gy = torch.randn((B, T, n), device=device, generator=g)
         del ws
-        wsv = bd.alloc_workspace(bd.DEER_OP_VJP, B, T, n, m, args.flags, device)
+        wsv = bd.alloc_workspace(bd.DEER_OP_VJP, B, T, n, m, flags, device)
         for _ in range(2):
-            bd.deer_gru_vjp(p, x, y0, y, gy, True, True, wsv, args.flags, stream)
+            bd.deer_gru_vjp(p, x, y0, y, gy, True, True, wsv, flags, stream)
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream); bd.deer_gru_vjp(p, x, y0, y, gy, True, True, wsv, args.flags, stream); b.record(stream)
+        a.record(stream); bd.deer_gru_vjp(p, x, y0, y, gy, True, True, wsv, flags, stream); b.record(stream)
         torch.cuda.synchronize()
         out["vjp_ms"] = a.elapsed_time(b)
         bd.lib().deer_profile_enable(1)
-        bd.deer_gru_vjp(p, x, y0, y, gy, True, True, wsv, args.flags, stream)
+        bd.deer_gru_vjp(p, x, y0, y, gy, True, True, wsv, flags, stream)
         torch.cuda.synchronize()
         bd.lib().deer_profile_enable(0)
         out["vjp_kernels"] = {k: round(v["total_ms"], 4) for k, v in read_profile(bd).items()}
+    return out
+
+
+def run_eval_only(args):
+    """One sweep point chosen on the command line: prints one JSON line."""
+    import torch
+    from paper_2309_12252_b200 import binding as bd
+    from paper_2309_12252_b200 import synth
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    out = eval_point(bd, synth, device, args.n, args.m or args.n, args.B, args.T, args.flags,
+                     args.steps, args.warmup, vjp=bool(args.vjp))
+    out["mode"] = "eval"
     print(json.dumps(out))
+
+
+def run_sweep(args):
+    """The paper's speed grid (Table of forward speed-ups), thinned: n = m in {1..64} x T in {1e3..1e6},
+    B = 16, x ~ N(0,1); one JSON line with one entry per point (n = 64, T = 1e6 is left out)."""
+    import torch
+    from paper_2309_12252_b200 import binding as bd
+    from paper_2309_12252_b200 import synth
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    points = []
+    for n in (1, 2, 4, 8, 16, 32, 64):
+        for T in (1000, 10000, 100000, 1000000):
+            if n == 64 and T == 1000000:
+                continue
+            steps = 5 if n * n * T <= 10 ** 8 else 2
+            pt = eval_point(bd, synth, device, n, n, 16, T, args.flags, steps, 1, breakdown=True)
+            pt.pop("kernels", None)
+            points.append(pt)
+            torch.cuda.empty_cache()
+    print(json.dumps(dict(mode="sweep", B=16, points=points)))
 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--mode", default="step", choices=["step", "scan", "eval"])
+    ap.add_argument("--mode", default="step", choices=["step", "scan", "eval", "sweep"])
     ap.add_argument("--m", type=int, default=0)
     ap.add_argument("--vjp", type=int, default=0)
     ap.add_argument("--n", type=int, default=8)
@@ -285,6 +321,9 @@ def main():
         return
     if args.mode == "eval":
         run_eval_only(args)
+        return
+    if args.mode == "sweep":
+        run_sweep(args)
         return
 
     import torch
