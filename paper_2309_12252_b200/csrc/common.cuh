@@ -57,9 +57,16 @@ struct StatusBlock {
     unsigned tile_counter;  // dynamic tile id for the single-pass scan
     unsigned role_counter;  // role tickets of the single-pass scan (first ones: resolvers)
     unsigned err_last_bits; // err of the last executed body
-    unsigned pad[57];
+    unsigned exit_counter;  // CTAs of the running single-pass scan that have finished
+    int ctl_mode;        // 1: the last CTA of a single-pass scan takes the Newton loop decision
+    int max_iter;
+    float tol;
+    unsigned pad0;
+    float *trace;        // err after each body (first ERR_TRACE_CAP bodies), or nullptr
+    unsigned pad[50];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is one 256-byte line");
+constexpr int ERR_TRACE_CAP = 1024;
 
 constexpr unsigned FLAG_NONFINITE = 1u;
 constexpr unsigned FLAG_TIMEOUT = 2u;
@@ -102,6 +109,37 @@ struct CellArgs {
 __device__ __forceinline__ bool loop_ended(const StatusBlock *st)
 {
     return st != nullptr && *(volatile const int *)&st->done != 0;
+}
+
+// End of one Newton body (App. B.1 loop): record err, count the body, decide whether the loop goes on
+// (err > tol and fewer than max_iter bodies).  A NaN err fails "err > tol" and ends the loop, as in
+// the listing; an infinite err ends it too.  Single thread.
+__device__ __forceinline__ void newton_decide(StatusBlock *st, float tol, int max_iter, float *trace)
+{
+    const unsigned bits = *(volatile unsigned *)&st->err_bits;
+    const float e = __uint_as_float(bits);
+    const int k = st->iters;
+    if (trace && k < ERR_TRACE_CAP) trace[k] = e;
+    st->iters = k + 1;
+    st->err_last_bits = bits;
+    st->err_bits = 0u;
+    if (!(e > tol) || !(e <= 3.402823466e38f) || k + 1 >= max_iter) st->done = 1;
+}
+
+// Called by one thread of every CTA of a single-pass scan after the CTA's last global write.  The
+// last CTA to leave rewinds the per-launch counters (the launch leaves its flag and state words
+// cleared as well: every word is cleared by its only reader) and, in loop-control mode, takes the
+// Newton decision, so a body needs no separate control or clearing launch.
+__device__ __forceinline__ void scan_epilogue(StatusBlock *st)
+{
+    __threadfence();
+    const unsigned prev = atomicAdd(&st->exit_counter, 1u);
+    if (prev + 1u != gridDim.x) return;
+    __threadfence();
+    st->exit_counter = 0u;
+    st->tile_counter = 0u;
+    st->role_counter = 0u;
+    if (st->ctl_mode) newton_decide(st, st->tol, st->max_iter, st->trace);
 }
 
 __device__ __forceinline__ float sigmoidf_acc(float a) { return 1.0f / (1.0f + expf(-a)); }

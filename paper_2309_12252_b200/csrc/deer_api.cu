@@ -77,20 +77,13 @@ struct ScanWs {
     OnePassWs op;        // single-pass path (n in {1,2,4,8}); op.nch == 0 when not applicable
 };
 
-static bool use_warp8()
-{
-    static int v = -1;
-    if (v < 0) { const char *e = getenv("DEER_SCAN8_OLD"); v = (e && atoi(e)) ? 0 : 1; }
-    return v != 0;
-}
-
 static int onepass_tile_len(int n)
 {
     switch (n) {
     case 1: return OnePass<1>::L;
     case 2: return OnePass<2>::L;
     case 4: return OnePass<4>::L;
-    case 8: return use_warp8() ? Warp8::L : OnePass<8>::L;
+    case 8: return Warp8::L;
     case 16: return WarpN<16>::L;
     case 32: return WarpN<32>::L;
     case 64: return Cta64::L;
@@ -130,198 +123,117 @@ static int num_sms()
     return g_num_sms;
 }
 
+// Clears the single-pass scan's flag / state words and counters (needed once per workspace: the
+// scans leave them cleared).
+static int scan_prep(const ScanArgs &a, const OnePassWs &w, cudaStream_t st)
+{
+    const size_t tiles = (size_t)a.B * w.nch;
+    const size_t words = tiles * (size_t)(a.n + 1);
+    unsigned pb = (unsigned)((words + 255) / 256);
+    if (pb > 592u) pb = 592u;
+    if (pb < 1u) pb = 1u;
+    DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)a.n));
+    return DEER_OK;
+}
+
+struct PassCfg {
+    const char *name;
+    int threads;
+    size_t smem;
+    int res_warps;          // resolver warps per resolver CTA
+    int max_seq_per_warp;
+    int cta_cap;            // CTAs per SM at most
+    int res_cap;            // resolver CTAs before warps take several sequences
+};
+
+// One persistent launch: grid = resident CTAs (or fewer when there are few tiles); the first
+// `resolvers` role tickets become resolver CTAs.
+template <typename Kern>
+static int launch_single_pass(Kern kern, int &occ, const PassCfg &c, ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
+{
+    if (!occ) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
+        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(single-pass scan)"); return DEER_ERR_CUDA; }
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, c.threads, c.smem);
+        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(single-pass scan)"); return DEER_ERR_CUDA; }
+        occ = o < c.cta_cap ? o : c.cta_cap;
+    }
+    const size_t tiles = (size_t)a.B * w.nch;
+    const size_t resident = (size_t)num_sms() * occ;
+    // resolver CTAs: one warp per sequence up to res_cap CTAs, then several sequences per warp
+    int R = (a.B + c.res_warps - 1) / c.res_warps;
+    if (R > c.res_cap) R = c.res_cap;
+    const int per_cta_cap = c.res_warps * c.max_seq_per_warp;
+    if ((a.B + per_cta_cap - 1) / per_cta_cap > R) R = (a.B + per_cta_cap - 1) / per_cta_cap;
+    w.resolvers = R;
+    const size_t want = tiles + (size_t)R;
+    unsigned grid = (unsigned)(want < resident ? want : resident);
+    if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
+    int Wd = 8;
+    if (Wd > w.nch) Wd = w.nch;
+    w.Wd = Wd;
+    w.nwin = (w.nch + Wd - 1) / Wd;
+    w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
+    int rc;
+    if (prep && (rc = scan_prep(a, w, st)) != DEER_OK) return rc;
+    DEER_KERNEL(c.name, st, kern<<<grid, c.threads, c.smem, st>>>(a, w));
+    return DEER_OK;
+}
+
 template <int N, bool REV>
-static int launch_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
+static int launch_onepass(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = OnePass<N>;
     static int occ = 0;
-    auto kern = scan_onepass_kernel<N, REV>;
-    if (!occ) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
-        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(onepass)"); return DEER_ERR_CUDA; }
-        int o = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, C::THREADS, C::SMEM);
-        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(onepass)"); return DEER_ERR_CUDA; }
-        occ = o;
-    }
-    size_t tiles = (size_t)a.B * w.nch;
-    size_t resident = (size_t)num_sms() * occ;
-    // resolver CTAs: one warp per sequence up to 8 CTAs, then several sequences per warp
-    int R = (a.B + C::WARPS - 1) / C::WARPS;
-    if (R > 8) R = 8;
-    const int per_warp_cap = C::WARPS * C::MAX_SEQ_PER_WARP;
-    if ((a.B + per_warp_cap - 1) / per_warp_cap > R) R = (a.B + per_warp_cap - 1) / per_warp_cap;
-    w.resolvers = R;
-    size_t want = tiles + (size_t)R;
-    unsigned grid = (unsigned)(want < resident ? want : resident);
-    if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
-    int Wd = 8;
-    { const char *d = getenv("DEER_DEBUG"); w.debug = d ? atoi(d) : 0; if (w.debug >> 8) Wd = w.debug >> 8; }
-    if (Wd > w.nch) Wd = w.nch;
-    w.Wd = Wd;
-    w.nwin = (w.nch + Wd - 1) / Wd;
-    w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
-    {
-        size_t words = tiles * (size_t)(N + 1);
-        unsigned pb = (unsigned)((words + 255) / 256);
-        if (pb > 592u) pb = 592u;
-        if (pb < 1u) pb = 1u;
-        DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)N));
-    }
-    DEER_KERNEL("scan_onepass_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
-    return DEER_OK;
+    const PassCfg c{"scan_onepass_kernel", C::THREADS, C::SMEM, C::WARPS, C::MAX_SEQ_PER_WARP, 32, 8};
+    return launch_single_pass(scan_onepass_kernel<N, REV>, occ, c, a, w, prep, st);
 }
 
 template <bool REV>
-static int launch_warp8(ScanArgs a, OnePassWs w, cudaStream_t st)
+static int launch_warp8(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = Warp8;
     static int occ = 0;
-    auto kern = scan_warp8_kernel<REV>;
-    if (!occ) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
-        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(warp8)"); return DEER_ERR_CUDA; }
-        int o = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, C::THREADS, C::SMEM);
-        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(warp8)"); return DEER_ERR_CUDA; }
-        // more CTAs in flight lengthen the distance between a tile's two visits beyond what L2 holds
-        int cap = 4;
-        if (const char *d = getenv("DEER_W8_CTAS")) cap = atoi(d);
-        occ = o < cap ? o : cap;
-        if (occ < 1) occ = 1;
-    }
-    size_t tiles = (size_t)a.B * w.nch;
-    size_t resident = (size_t)num_sms() * occ;
-    int R = (a.B + C::RES_WARPS - 1) / C::RES_WARPS;
-    if (R > 8) R = 8;
-    const int per_cta_cap = C::RES_WARPS * OnePass<8>::MAX_SEQ_PER_WARP;
-    if ((a.B + per_cta_cap - 1) / per_cta_cap > R) R = (a.B + per_cta_cap - 1) / per_cta_cap;
-    w.resolvers = R;
-    size_t want = tiles + (size_t)R;
-    unsigned grid = (unsigned)(want < resident ? want : resident);
-    if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
-    int Wd = 8;
-    if (Wd > w.nch) Wd = w.nch;
-    w.Wd = Wd;
-    w.nwin = (w.nch + Wd - 1) / Wd;
-    w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
-    w.debug = 0;
-    {
-        size_t words = tiles * (size_t)(C::N + 1);
-        unsigned pb = (unsigned)((words + 255) / 256);
-        if (pb > 592u) pb = 592u;
-        if (pb < 1u) pb = 1u;
-        DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)C::N));
-    }
-    DEER_KERNEL("scan_warp8_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
-    return DEER_OK;
+    const PassCfg c{"scan_warp8_kernel", C::THREADS, C::SMEM, C::RES_WARPS, OnePass<8>::MAX_SEQ_PER_WARP, 4, 8};
+    return launch_single_pass(scan_warp8_kernel<REV>, occ, c, a, w, prep, st);
 }
 
 template <int N, bool REV>
-static int launch_warpn(ScanArgs a, OnePassWs w, cudaStream_t st)
+static int launch_warpn(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = WarpN<N>;
     static int occ = 0;
-    auto kern = scan_warpn_kernel<N, REV>;
-    if (!occ) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
-        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(warpn)"); return DEER_ERR_CUDA; }
-        int o = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, C::THREADS, C::SMEM);
-        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(warpn)"); return DEER_ERR_CUDA; }
-        int cap = 8;
-        if (const char *d = getenv("DEER_WN_CTAS")) cap = atoi(d);
-        occ = o < cap ? o : cap;
-        if (occ < 1) occ = 1;
-    }
-    size_t tiles = (size_t)a.B * w.nch;
-    size_t resident = (size_t)num_sms() * occ;
-    int R = (a.B + C::RES_WARPS - 1) / C::RES_WARPS;
-    if (R > 8) R = 8;
-    const int per_cta_cap = C::RES_WARPS * C::MAX_SEQ_PER_WARP;
-    if ((a.B + per_cta_cap - 1) / per_cta_cap > R) R = (a.B + per_cta_cap - 1) / per_cta_cap;
-    w.resolvers = R;
-    size_t want = tiles + (size_t)R;
-    unsigned grid = (unsigned)(want < resident ? want : resident);
-    if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
-    int Wd = 8;
-    if (Wd > w.nch) Wd = w.nch;
-    w.Wd = Wd;
-    w.nwin = (w.nch + Wd - 1) / Wd;
-    w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
-    w.debug = 0;
-    {
-        size_t words = tiles * (size_t)(N + 1);
-        unsigned pb = (unsigned)((words + 255) / 256);
-        if (pb > 592u) pb = 592u;
-        if (pb < 1u) pb = 1u;
-        DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)N));
-    }
-    DEER_KERNEL("scan_warpn_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
-    return DEER_OK;
+    const PassCfg c{"scan_warpn_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 8};
+    return launch_single_pass(scan_warpn_kernel<N, REV>, occ, c, a, w, prep, st);
 }
 
 template <bool REV>
-static int launch_cta64(ScanArgs a, OnePassWs w, cudaStream_t st)
+static int launch_cta64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = Cta64;
     static int occ = 0;
-    auto kern = scan_cta64_kernel<REV>;
-    if (!occ) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
-        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(cta64)"); return DEER_ERR_CUDA; }
-        int o = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, C::THREADS, C::SMEM);
-        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(cta64)"); return DEER_ERR_CUDA; }
-        int cap = 8;
-        if (const char *d = getenv("DEER_WN_CTAS")) cap = atoi(d);
-        occ = o < cap ? o : cap;
-        if (occ < 1) occ = 1;
-    }
-    size_t tiles = (size_t)a.B * w.nch;
-    size_t resident = (size_t)num_sms() * occ;
-    int R = (a.B + C::RES_WARPS - 1) / C::RES_WARPS;
-    if (R > 16) R = 16;
-    const int per_cta_cap = C::RES_WARPS * C::MAX_SEQ_PER_WARP;
-    if ((a.B + per_cta_cap - 1) / per_cta_cap > R) R = (a.B + per_cta_cap - 1) / per_cta_cap;
-    w.resolvers = R;
-    size_t want = tiles + (size_t)R;
-    unsigned grid = (unsigned)(want < resident ? want : resident);
-    if (grid < (unsigned)R + 1u) grid = (unsigned)R + 1u;
-    int Wd = 8;
-    if (Wd > w.nch) Wd = w.nch;
-    w.Wd = Wd;
-    w.nwin = (w.nch + Wd - 1) / Wd;
-    w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
-    w.debug = 0;
-    {
-        size_t words = tiles * (size_t)(C::N + 1);
-        unsigned pb = (unsigned)((words + 255) / 256);
-        if (pb > 592u) pb = 592u;
-        if (pb < 1u) pb = 1u;
-        DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)C::N));
-    }
-    DEER_KERNEL("scan_cta64_kernel", st, kern<<<grid, C::THREADS, C::SMEM, st>>>(a, w));
-    return DEER_OK;
+    const PassCfg c{"scan_cta64_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 16};
+    return launch_single_pass(scan_cta64_kernel<REV>, occ, c, a, w, prep, st);
 }
 
-static int scan_onepass(ScanArgs a, OnePassWs w, cudaStream_t st)
+static int scan_onepass(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     switch (a.n * 2 + (a.reverse ? 1 : 0)) {
-    case 2: return launch_onepass<1, false>(a, w, st);
-    case 3: return launch_onepass<1, true>(a, w, st);
-    case 4: return launch_onepass<2, false>(a, w, st);
-    case 5: return launch_onepass<2, true>(a, w, st);
-    case 8: return launch_onepass<4, false>(a, w, st);
-    case 9: return launch_onepass<4, true>(a, w, st);
-    case 16: return use_warp8() ? launch_warp8<false>(a, w, st) : launch_onepass<8, false>(a, w, st);
-    case 17: return use_warp8() ? launch_warp8<true>(a, w, st) : launch_onepass<8, true>(a, w, st);
-    case 32: return launch_warpn<16, false>(a, w, st);
-    case 33: return launch_warpn<16, true>(a, w, st);
-    case 64: return launch_warpn<32, false>(a, w, st);
-    case 65: return launch_warpn<32, true>(a, w, st);
-    case 128: return launch_cta64<false>(a, w, st);
-    case 129: return launch_cta64<true>(a, w, st);
+    case 2: return launch_onepass<1, false>(a, w, prep, st);
+    case 3: return launch_onepass<1, true>(a, w, prep, st);
+    case 4: return launch_onepass<2, false>(a, w, prep, st);
+    case 5: return launch_onepass<2, true>(a, w, prep, st);
+    case 8: return launch_onepass<4, false>(a, w, prep, st);
+    case 9: return launch_onepass<4, true>(a, w, prep, st);
+    case 16: return launch_warp8<false>(a, w, prep, st);
+    case 17: return launch_warp8<true>(a, w, prep, st);
+    case 32: return launch_warpn<16, false>(a, w, prep, st);
+    case 33: return launch_warpn<16, true>(a, w, prep, st);
+    case 64: return launch_warpn<32, false>(a, w, prep, st);
+    case 65: return launch_warpn<32, true>(a, w, prep, st);
+    case 128: return launch_cta64<false>(a, w, prep, st);
+    case 129: return launch_cta64<true>(a, w, prep, st);
     default: return DEER_ERR_UNSUPPORTED_N;
     }
 }
@@ -352,10 +264,17 @@ static int scan_generic(ScanArgs a, cudaStream_t st)
     return DEER_OK;
 }
 
-static int run_scan(ScanArgs a, const ScanWs &w, int flags, cudaStream_t st)
+static bool scan_is_single_pass(const ScanArgs &a, const ScanWs &w, int flags)
 {
     const bool aligned = (((uintptr_t)a.J | (uintptr_t)a.b | (uintptr_t)a.y) & 15) == 0;
-    if (!(flags & DEER_FLAG_GENERIC) && w.op.nch > 0 && aligned) return scan_onepass(a, w.op, st);
+    return !(flags & DEER_FLAG_GENERIC) && w.op.nch > 0 && aligned;
+}
+
+// prep: clear the single-pass scan's words first (false when the previous scan on this workspace
+// left them cleared)
+static int run_scan(ScanArgs a, const ScanWs &w, int flags, cudaStream_t st, bool prep = true)
+{
+    if (scan_is_single_pass(a, w, flags)) return scan_onepass(a, w.op, prep, st);
     return scan_generic(a, st);
 }
 
@@ -625,14 +544,33 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     int rc = check_ws(ws, ws_bytes, w.bytes);
     if (rc != DEER_OK) return rc;
     const size_t N = (size_t)B * T;
-    DEER_CHECK_CUDA(cudaMemsetAsync(w.st, 0, sizeof(StatusBlock), st), "memset status");
     if (!(flags & DEER_FLAG_WARM_START))
         DEER_CHECK_CUDA(cudaMemsetAsync(y, 0, N * n * sizeof(float), st), "memset y");
     const bool fused_proj = cell_projects(n, m) && ((((uintptr_t)y | (uintptr_t)y0) & 15) == 0);
-    if (!fused_proj && (rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
 
-    // Newton loop (App. B.1): bodies are enqueued ahead of the convergence test -- the control kernel
-    // at the end of each body decides on the device, and the kernels of bodies past the end return
+    ScanArgs a{};
+    a.J = w.J; a.b = w.rhs; a.y0 = y0; a.y = y;
+    a.B = B; a.T = T; a.n = n; a.reverse = 0;
+    a.L = w.scan.L; a.nch = w.scan.nch;
+    a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
+    a.st = w.st;
+    // With the single-pass scan the last CTA of every scan takes the loop decision and the scan
+    // leaves its flag words cleared: a body is two launches (cell, scan).
+    const bool single = scan_is_single_pass(a, w.scan, flags) && (((uintptr_t)w.yalt) & 15) == 0;
+    {
+        StatusBlock init;
+        memset(&init, 0, sizeof(init));
+        init.ctl_mode = single ? 1 : 0;
+        init.max_iter = max_iter;
+        init.tol = tol;
+        init.trace = w.trace;
+        DEER_CHECK_CUDA(cudaMemcpyAsync(w.st, &init, sizeof(init), cudaMemcpyHostToDevice, st), "init status");
+    }
+    if (!fused_proj && (rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
+    if (single && (rc = scan_prep(a, w.scan.op, st)) != DEER_OK) return rc;
+
+    // Newton loop (App. B.1): bodies are enqueued ahead of the convergence test -- the decision at
+    // the end of each body is taken on the device, and the kernels of bodies past the end return
     // at once -- so the host only synchronises once per group of bodies.
     float *buf[2] = {y, w.yalt};
     int enq = 0, group = 4;
@@ -644,14 +582,13 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
             float *cur = buf[enq & 1], *nxt = buf[(enq + 1) & 1];
             CellArgs c{p->W_h, p->b_h, fused_proj ? nullptr : w.u, x, p->W_i, p->b_i, m, cur, y0, w.J, w.rhs, B, T, n, w.st};
             if ((rc = run_cell(c, st)) != DEER_OK) return rc;
-            ScanArgs a{};
-            a.J = w.J; a.b = w.rhs; a.y0 = y0; a.y = nxt; a.yold = cur;
-            a.B = B; a.T = T; a.n = n; a.reverse = 0;
-            a.L = w.scan.L; a.nch = w.scan.nch;
-            a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
-            a.st = w.st;
-            if ((rc = run_scan(a, w.scan, flags, st)) != DEER_OK) return rc;
-            DEER_KERNEL("newton_control_kernel", st, newton_control_kernel<<<1, 1, 0, st>>>(w.st, tol, max_iter, w.trace));
+            a.y = nxt; a.yold = cur;
+            if (single) {
+                if ((rc = scan_onepass(a, w.scan.op, false, st)) != DEER_OK) return rc;
+            } else {
+                if ((rc = scan_generic(a, st)) != DEER_OK) return rc;
+                DEER_KERNEL("newton_control_kernel", st, newton_control_kernel<<<1, 1, 0, st>>>(w.st, tol, max_iter, w.trace));
+            }
         }
         DEER_CHECK_CUDA(cudaMemcpyAsync(&hs, w.st, 32, cudaMemcpyDeviceToHost, st), "read status");
         DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");

@@ -292,7 +292,8 @@ __global__ void gen_apply_kernel(ScanArgs a)
 }
 
 // ------------------------------------------------------------------ a6: loop control on the device
-// Clears the single-pass scan's per-launch words (tile flags, entering states, counters).
+// Clears the single-pass scan's words (tile flags, entering states, counters) before the first scan
+// on a workspace; the scans leave them cleared.
 __global__ void scan_prep_kernel(StatusBlock *st, unsigned *flags, size_t nflags,
                                  unsigned long long *starts, size_t nstarts)
 {
@@ -301,23 +302,14 @@ __global__ void scan_prep_kernel(StatusBlock *st, unsigned *flags, size_t nflags
     const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (size_t i = i0; i < nflags; i += stride) flags[i] = 0u;
     for (size_t i = i0; i < nstarts; i += stride) starts[i] = 0ull;
-    if (i0 == 0) { st->tile_counter = 0u; st->role_counter = 0u; }
+    if (i0 == 0) { st->tile_counter = 0u; st->role_counter = 0u; st->exit_counter = 0u; }
 }
 
-// End of one Newton body (App. B.1 loop): record err, count the body, decide whether the loop goes on
-// (err > tol and fewer than max_iter bodies).  A NaN err fails "err > tol" and ends the loop, as in
-// the listing; an infinite err ends it too.
-constexpr int ERR_TRACE_CAP = 1024;
+// Loop control as a launch of its own (used when a body's scan ran on the generic kernels).
 __global__ void newton_control_kernel(StatusBlock *st, float tol, int max_iter, float *trace)
 {
     if (loop_ended(st)) return;
-    const unsigned bits = st->err_bits;
-    const float e = __uint_as_float(bits);
-    if (st->iters < ERR_TRACE_CAP) trace[st->iters] = e;
-    st->iters += 1;
-    st->err_last_bits = bits;
-    st->err_bits = 0u;
-    if (!(e > tol) || !(e <= 3.402823466e38f) || st->iters >= max_iter) st->done = 1;
+    newton_decide(st, tol, max_iter, trace);
 }
 
 // ------------------------------------------------------------------ a8: cell VJP

@@ -118,6 +118,7 @@ __device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_a
                 __syncwarp();
             }
             ya[k] = y0v; yb[k] = y1v;
+            if (lane < cnt) w.flags[(size_t)s * w.nch + c0 + lane] = 0u;   // consumed: cleared for the next launch
             pos[k] = c0 + cnt;
             if (pos[k] >= w.nch) --remaining;
             else fnext[k] = (pos[k] + lane < w.nch) ? ld_acquire_u32(flags + pos[k] + lane) : 0u;
@@ -232,6 +233,8 @@ __global__ void __launch_bounds__(Cta64::THREADS) scan_cta64_kernel(ScanArgs a, 
     __syncthreads();
     if (s_role < w.resolvers) {
         resolver64(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        __syncthreads();
+        if (tid == 0) scan_epilogue(a.st);
         return;
     }
     unsigned mb = 0;
@@ -374,7 +377,11 @@ __global__ void __launch_bounds__(Cta64::THREADS) scan_cta64_kernel(ScanArgs a, 
             bool ok = true;
             for (;;) {
                 const unsigned long long v = ld_relaxed_u64(src + tid);
-                if (v != 0ull) { ybuf[tid] = __uint_as_float((unsigned)(v & 0xffffffffull)); break; }
+                if (v != 0ull) {
+                    ybuf[tid] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                    st_relaxed_u64(w.starts + tile_index * N + tid, 0ull);      // consumed: cleared for the next launch
+                    break;
+                }
                 if (!keep_spinning(a.st, spins)) { ok = false; break; }
             }
             if (!ok) s_abort = 1;
@@ -400,8 +407,10 @@ __global__ void __launch_bounds__(Cta64::THREADS) scan_cta64_kernel(ScanArgs a, 
     if (a.yold) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
-        if (lane == 0 && mb) atomicMax(&a.st->err_bits, mb);
+        if (lane == 0 && mb) { atomicMax(&a.st->err_bits, mb); __threadfence(); }
     }
+    __syncthreads();
+    if (tid == 0) scan_epilogue(a.st);
 }
 
 }  // namespace deer

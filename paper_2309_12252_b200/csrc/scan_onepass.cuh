@@ -73,7 +73,6 @@ struct OnePassWs {
     int nch, Wd, nwin;            // tiles per sequence, tiles per sequence per window, windows
     unsigned total_ids;
     int resolvers;                // CTAs that take the resolver role
-    int debug;                    // experiment switches (0 in production)
 };
 
 // ---------------------------------------------------------------- small PTX helpers
@@ -409,6 +408,7 @@ __device__ void resolver_loop(const ScanArgs &a, const OnePassWs &w, float *stag
             }
             yv[k] = y;
             __syncwarp();
+            if (lane < cnt) w.flags[(size_t)s * w.nch + c0 + lane] = 0u;   // consumed: cleared for the next launch
             pos[k] = c0 + cnt;
             if (pos[k] >= w.nch) --remaining;
         }
@@ -455,6 +455,8 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     __syncthreads();
     if (s_role < w.resolvers) {
         resolver_loop<N>(a, w, sJ, s_role * WARPS + warp, w.resolvers * WARPS, lane);
+        __syncthreads();
+        if (tid == 0) scan_epilogue(a.st);
         return;
     }
     unsigned phase = 0;
@@ -474,18 +476,8 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
     bool exhausted = false;
 
-    const bool trace = (w.debug & 2) && tid == 0 && blockIdx.x == gridDim.x / 2;
-    long long tr[2][5] = {{0, 0, 0, 0, 0}, {0, 0, 0, 0, 0}};
-    long long t_prev = 0;
-    int k_prev = -1;
-
     for (;;) {
         __syncthreads();      // previous item done with shared memory and with the s_* words
-        long long t0 = 0, t1 = 0, t2 = 0, t3 = 0;
-        if (trace) {
-            t0 = clock64();
-            if (k_prev >= 0) { tr[k_prev][3] += t0 - t_prev; tr[k_prev][4] += 1; }
-        }
         if (tid == 0) {
             // next item: the oldest pending tile's B item as soon as its entering state is
             // there (or when the queue is full / no tiles are left), otherwise a new tile's A item
@@ -520,7 +512,6 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         }
         __syncthreads();
         if (s_kind < 0 || s_abort) break;
-        if (trace) t1 = clock64();
         const int kind = s_kind, seq = s_seq, c = s_c;
         float *agg = pend + s_slot * PEND;          // chain aggregates (n = 8) / exclusive chain prefixes
         float *wagg = agg + CHAINS * AGG;           // warp aggregates (n = 8) / exclusive warp prefixes
@@ -589,7 +580,6 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             if (!jbulk) for (int i = tid; i < jcnt_tile * NN; i += C::THREADS) jd[i] = __ldg(Jt_src + i);
             if (!bbulk) for (int i = tid; i < Lt * N; i += C::THREADS) bd[i] = __ldg(bt_src + i);
         }
-        if (trace) t2 = clock64();
         // B item: while the copies fly, warp 1 fetches the state entering the tile ({value, flag} words)
         if (kind == 1 && warp == 1) {
             const unsigned long long *src = w.starts + tile_index * N;
@@ -598,7 +588,10 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             for (;;) {
                 const unsigned long long v = (lane < N) ? ld_relaxed_u64(src + lane) : LL_FLAG;
                 if (__all_sync(0xffffffffu, v != 0ull)) {
-                    if (lane < N) ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                    if (lane < N) {
+                        ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                        st_relaxed_u64(w.starts + tile_index * N + lane, 0ull);     // consumed: cleared for the next launch
+                    }
                     break;
                 }
                 if (!keep_spinning(a.st, spins)) { ok = false; break; }
@@ -616,11 +609,6 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         }
         __syncthreads();      // plain-copied data, ystart and s_abort visible
         if (s_abort) break;
-        if (trace) {
-            t3 = clock64();
-            tr[kind][0] += t1 - t0; tr[kind][1] += t2 - t1; tr[kind][2] += t3 - t2;
-            t_prev = t3; k_prev = kind;
-        }
 
         const int cnt = tg.run_cnt(chain);
         if constexpr (LPC == 1) {
@@ -949,15 +937,13 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             }
         }
     }
-    if (trace) {
-        for (int k = 0; k < 2; ++k)
-            for (int j = 0; j < 5; ++j) a.st->pad[k * 5 + j] = (unsigned)(tr[k][j] > 0xffffffffll ? 0xffffffffu : tr[k][j]);
-    }
     if (a.yold) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
-        if (lane == 0 && mb) atomicMax(&a.st->err_bits, mb);
+        if (lane == 0 && mb) { atomicMax(&a.st->err_bits, mb); __threadfence(); }
     }
+    __syncthreads();
+    if (tid == 0) scan_epilogue(a.st);
 }
 
 }  // namespace deer

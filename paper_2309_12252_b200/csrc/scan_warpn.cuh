@@ -113,6 +113,7 @@ __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage
             }
             yv[k] = y;
             __syncwarp();
+            if (lane < cnt) w.flags[(size_t)s * w.nch + c0 + lane] = 0u;   // consumed: cleared for the next launch
             pos[k] = c0 + cnt;
             if (pos[k] >= w.nch) --remaining;
         }
@@ -293,6 +294,8 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
     if (s_role < w.resolvers) {
         if (warp < C::RES_WARPS)
             resolver_big<N>(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        __syncthreads();
+        if (tid == 0) scan_epilogue(a.st);
         return;
     }
     unsigned mb = 0;
@@ -406,7 +409,10 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
             for (;;) {
                 const unsigned long long v = (lane < N) ? ld_relaxed_u64(src + lane) : LL_FLAG;
                 if (__all_sync(0xffffffffu, v != 0ull)) {
-                    if (lane < N) ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                    if (lane < N) {
+                        ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                        st_relaxed_u64(w.starts + tile_index * N + lane, 0ull);     // consumed: cleared for the next launch
+                    }
                     break;
                 }
                 if (!keep_spinning(a.st, spins)) { ok = false; break; }
@@ -468,8 +474,10 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
     if (a.yold) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
-        if (lane == 0 && mb) atomicMax(&a.st->err_bits, mb);
+        if (lane == 0 && mb) { atomicMax(&a.st->err_bits, mb); __threadfence(); }
     }
+    __syncthreads();
+    if (tid == 0) scan_epilogue(a.st);
 }
 
 }  // namespace deer
