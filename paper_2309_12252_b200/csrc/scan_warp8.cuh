@@ -48,11 +48,13 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const unsigned (&a)[4], 
 }
 
 // hi / lo TF32 split by truncation: hi keeps the top 10 mantissa bits, lo the next 10 of the exact
-// remainder, so hi*hi + hi*lo + lo*hi carries about 21 mantissa bits of every product
+// remainder, so hi*hi + hi*lo + lo*hi carries about 21 mantissa bits of every product.  The tensor
+// core reads only the upper 19 bits of a TF32 operand register, so neither half needs masking:
+// hi is x itself, lo is x minus its truncation (bit-identical to the masked form on sm_100a).
 __device__ __forceinline__ void split_tf32(float x, unsigned &hi, unsigned &lo)
 {
-    hi = __float_as_uint(x) & 0xffffe000u;
-    lo = __float_as_uint(x - __uint_as_float(hi)) & 0xffffe000u;
+    hi = __float_as_uint(x);
+    lo = __float_as_uint(x - __uint_as_float(hi & 0xffffe000u));
 }
 
 // one step of the transposed chain on the accumulator fragment:
@@ -177,24 +179,35 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
             // ---------------------------------------------- A item: [X; beta^T] in the accumulator fragment
             float acc[4] = {(g == 2 * t) ? 1.0f : 0.0f, (g == 2 * t + 1) ? 1.0f : 0.0f, 0.0f, 0.0f};
             const float2 *bp2 = reinterpret_cast<const float2 *>(bseq + tb * N) + t;
+            // whole groups: loads with constant offsets from one pointer per group, no per-position tests
+            int q0 = 0;
+            if (REV && sbase == 0 && cnt > 0) {                 // scan position 0 of the reverse scan: identity
+                const float2 f = (g == 0) ? __ldg(bp2) : make_float2(0.0f, 0.0f);
+                chain_step(acc, (g == 2 * t) ? 1.0f : 0.0f, (g == 2 * t + 1) ? 1.0f : 0.0f, f.x, f.y);
+                q0 = 1;
+            }
 #pragma unroll 1
-            for (int q0 = 0; q0 < cnt; q0 += GRP) {
+            for (; q0 + GRP <= cnt; q0 += GRP) {
                 float j0[GRP], j1[GRP], bx[GRP], by[GRP];
-                const bool full = (q0 + GRP <= cnt);
+                const float2 *jq = jp2 + q0 * 32;
+                const float *jr = jpr - q0 * NN;
+                const float2 *bq = REV ? bp2 - q0 * 4 : bp2 + q0 * 4;
 #pragma unroll
                 for (int u = 0; u < GRP; ++u) {
-                    j0[u] = 0.0f; j1[u] = 0.0f; bx[u] = 0.0f; by[u] = 0.0f;
-                    if (full || q0 + u < cnt) {
-                        piece(q0 + u, j0[u], j1[u]);
-                        if (g == 0) {
-                            const float2 f = __ldg(REV ? bp2 - (q0 + u) * 4 : bp2 + (q0 + u) * 4);
-                            bx[u] = f.x; by[u] = f.y;
-                        }
-                    }
+                    if (!REV) { const float2 f = __ldg(jq + u * 32); j0[u] = f.x; j1[u] = f.y; }
+                    else { j0[u] = __ldg(jr - u * NN); j1[u] = __ldg(jr - u * NN + N); }
+                    bx[u] = 0.0f; by[u] = 0.0f;
+                    if (g == 0) { const float2 f = __ldg(REV ? bq - u * 4 : bq + u * 4); bx[u] = f.x; by[u] = f.y; }
                 }
 #pragma unroll
-                for (int u = 0; u < GRP; ++u)
-                    if (full || q0 + u < cnt) chain_step(acc, j0[u], j1[u], bx[u], by[u]);
+                for (int u = 0; u < GRP; ++u) chain_step(acc, j0[u], j1[u], bx[u], by[u]);
+            }
+#pragma unroll 1
+            for (; q0 < cnt; ++q0) {                            // ragged tail
+                float j0, j1, bx = 0.0f, by = 0.0f;
+                piece(q0, j0, j1);
+                if (g == 0) { const float2 f = __ldg(REV ? bp2 - q0 * 4 : bp2 + q0 * 4); bx = f.x; by = f.y; }
+                chain_step(acc, j0, j1, bx, by);
             }
             // X[g][2t] = P[2t][g], X[g][2t+1] = P[2t+1][g]; beta in row 8 (lanes with g == 0)
             {
@@ -260,35 +273,66 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
             const float *bpg = bseq + tb * N + g;
             const float *yop = a.yold ? a.yold + ((size_t)seq * T + tb) * N + g : nullptr;
             float *yp = a.y + ((size_t)seq * T + tb) * N + g;
+            auto step = [&](float j0, float j1, float bgv, float yov, int off) {
+                float part = fmaf(j0, yk0, j1 * yk1);
+                part += __shfl_xor_sync(0xffffffffu, part, 1);
+                part += __shfl_xor_sync(0xffffffffu, part, 2);
+                const float yg = part + bgv;                                    // y_new[g], in all 4 lanes of group g
+                yk0 = __shfl_sync(0xffffffffu, yg, 4 * (2 * t));
+                yk1 = __shfl_sync(0xffffffffu, yg, 4 * (2 * t + 1));
+                if (t == 0) {
+                    if (yop) mb = max(mb, absdiff_bits(yg, yov));
+                    yp[off] = yg;
+                }
+            };
+            int q0 = 0;
+            if (REV && sbase == 0 && cnt > 0) {
+                float yov = 0.0f;
+                if (yop && t == 0) yov = __ldg(yop);
+                step((g == 2 * t) ? 1.0f : 0.0f, (g == 2 * t + 1) ? 1.0f : 0.0f, __ldg(bpg), yov, 0);
+                q0 = 1;
+            }
+            static_assert(GRP % 4 == 0, "lane (g,t) writes positions t, t+4, ... of a group");
 #pragma unroll 1
-            for (int q0 = 0; q0 < cnt; q0 += GRP) {
-                float j0[GRP], j1[GRP], bg[GRP], yo[GRP];
-                const bool full = (q0 + GRP <= cnt);
+            for (; q0 + GRP <= cnt; q0 += GRP) {
+                float j0[GRP], j1[GRP], bg[GRP], yg[GRP];
+                const float2 *jq = jp2 + q0 * 32;
+                const float *jr = jpr - q0 * NN;
+                const int off0 = REV ? -q0 * N : q0 * N;
+                const int offt = off0 + (REV ? -t * N : t * N);               // this lane's first position of the group
+                float yo[GRP / 4];
+#pragma unroll
+                for (int h = 0; h < GRP / 4; ++h) yo[h] = yop ? __ldg(yop + offt + (REV ? -4 * h * N : 4 * h * N)) : 0.0f;
 #pragma unroll
                 for (int u = 0; u < GRP; ++u) {
-                    j0[u] = 0.0f; j1[u] = 0.0f; bg[u] = 0.0f; yo[u] = 0.0f;
-                    if (full || q0 + u < cnt) {
-                        const int off = REV ? -(q0 + u) * N : (q0 + u) * N;
-                        piece(q0 + u, j0[u], j1[u]);
-                        bg[u] = __ldg(bpg + off);
-                        if (yop && t == 0) yo[u] = __ldg(yop + off);
-                    }
+                    if (!REV) { const float2 f = __ldg(jq + u * 32); j0[u] = f.x; j1[u] = f.y; }
+                    else { j0[u] = __ldg(jr - u * NN); j1[u] = __ldg(jr - u * NN + N); }
+                    bg[u] = __ldg(bpg + off0 + (REV ? -u * N : u * N));
                 }
 #pragma unroll
                 for (int u = 0; u < GRP; ++u) {
-                    if (full || q0 + u < cnt) {
-                        float part = fmaf(j0[u], yk0, j1[u] * yk1);
-                        part += __shfl_xor_sync(0xffffffffu, part, 1);
-                        part += __shfl_xor_sync(0xffffffffu, part, 2);
-                        const float yg = part + bg[u];                              // y_new[g], in all 4 lanes of group g
-                        yk0 = __shfl_sync(0xffffffffu, yg, 4 * (2 * t));
-                        yk1 = __shfl_sync(0xffffffffu, yg, 4 * (2 * t + 1));
-                        if (t == 0) {
-                            if (yop) mb = max(mb, absdiff_bits(yg, yo[u]));
-                            yp[REV ? -(q0 + u) * N : (q0 + u) * N] = yg;
-                        }
-                    }
+                    float part = fmaf(j0[u], yk0, j1[u] * yk1);
+                    part += __shfl_xor_sync(0xffffffffu, part, 1);
+                    part += __shfl_xor_sync(0xffffffffu, part, 2);
+                    yg[u] = part + bg[u];                                       // y_new[g], in all 4 lanes of group g
+                    yk0 = __shfl_sync(0xffffffffu, yg[u], 4 * (2 * t));
+                    yk1 = __shfl_sync(0xffffffffu, yg[u], 4 * (2 * t + 1));
                 }
+                // lane (g,t) writes component g of positions t, t+4, ...: stores of 128 contiguous bytes
+#pragma unroll
+                for (int h = 0; h < GRP / 4; ++h) {
+                    const float mine = t == 0 ? yg[4 * h] : t == 1 ? yg[4 * h + 1] : t == 2 ? yg[4 * h + 2] : yg[4 * h + 3];
+                    if (yop) mb = max(mb, absdiff_bits(mine, yo[h]));
+                    yp[offt + (REV ? -4 * h * N : 4 * h * N)] = mine;
+                }
+            }
+#pragma unroll 1
+            for (; q0 < cnt; ++q0) {
+                float j0, j1, yov = 0.0f;
+                const int off = REV ? -q0 * N : q0 * N;
+                piece(q0, j0, j1);
+                if (yop && t == 0) yov = __ldg(yop + off);
+                step(j0, j1, __ldg(bpg + off), yov, off);
             }
         }
     }
