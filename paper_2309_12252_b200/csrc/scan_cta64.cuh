@@ -6,9 +6,9 @@
 //       X <- X * M,   M = J_t^T (forward)  or  J_{t+1} (reverse),
 // 2 x 8 x 8 MMAs (m16n8k8) per warp and position, each issued three times on hi/lo TF32 splits.
 // The matrices of the tile stream through a shared-memory ring filled with 16-byte cp.async
-// copies; the 16-byte pieces of a row are XOR-swizzled so that the B-operand reads of both
-// directions (8-byte pieces of a row forward, scalars of a column in reverse) and the row /
-// column reads of the mat-vec are all free of bank conflicts.  beta (the state reached from
+// copies; rows are padded (by 8 floats forward, 4 in reverse) so that the B-operand reads (8-byte
+// pieces of a row forward, scalars of a column in reverse) and the row / column reads of the
+// mat-vec are all free of bank conflicts.  beta (the state reached from
 // zero) is carried by an fp32 mat-vec chain, thread r owning component r; the same routine
 // replays the tile from its true entering state in the B item.
 // Tiles, items, resolvers, flags and bounded waits are those of scan_onepass.cuh.
@@ -25,7 +25,7 @@ struct Cta64 {
     static constexpr int L = 64;                       // positions per tile
     static constexpr int Q = 2;                        // pending tiles per CTA
     static constexpr int STAGES = 3;                   // ring depth (positions)
-    static constexpr int STAGE_FLOATS = NN + N;        // swizzled matrix, then the vector
+    static constexpr int STAGE_FLOATS = N * (N + 8) + N;   // matrix with padded rows, then the vector
     static constexpr int RES_WARPS = 2;
     static constexpr int SM_WORK = STAGES * STAGE_FLOATS + 2 * N;
     static constexpr int SM_RES = RES_WARPS * (AGG + N);
@@ -33,13 +33,6 @@ struct Cta64 {
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
     static constexpr int MAX_SEQ_PER_WARP = 8;
 };
-
-// float offset of element (row, col) of a swizzled 64 x 64 matrix: the 16-byte piece index of the
-// row is XORed with 2 * ((row ^ (row >> 2)) & 3)
-__device__ __forceinline__ int sw64(int row, int col)
-{
-    return row * 64 + ((((col >> 2) ^ (((row ^ (row >> 2)) & 3) << 1)) << 2) | (col & 3));
-}
 
 template <int K> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(K) : "memory"); }
 
@@ -128,10 +121,12 @@ __device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_a
     }
 }
 
-// X <- X * M for the warp's 32 rows; B operands read from the swizzled stage
+// X <- X * M for the warp's 32 rows; B operands read from the padded stage
 template <bool REV>
 __device__ __forceinline__ void chain_step64(float (&acc)[2][8][4], const float *Ms, int g, int t)
 {
+    constexpr int RS = RingRow<64, REV>::RS;
+    const float *base = REV ? Ms + (2 * t) * RS + g : Ms + g * RS + 2 * t;
     float nacc[2][8][4];
 #pragma unroll
     for (int mm = 0; mm < 2; ++mm)
@@ -153,11 +148,11 @@ __device__ __forceinline__ void chain_step64(float (&acc)[2][8][4], const float 
         for (int nn = 0; nn < 8; ++nn) {
             float j0, j1;       // M[8kk+2t][8nn+g], M[8kk+2t+1][8nn+g]
             if (!REV) {
-                const float2 f = *reinterpret_cast<const float2 *>(Ms + sw64(8 * nn + g, 8 * kk + 2 * t));
+                const float2 f = *reinterpret_cast<const float2 *>(base + 8 * nn * RS + 8 * kk);
                 j0 = f.x; j1 = f.y;
             } else {
-                j0 = Ms[sw64(8 * kk + 2 * t, 8 * nn + g)];
-                j1 = Ms[sw64(8 * kk + 2 * t + 1, 8 * nn + g)];
+                j0 = base[8 * kk * RS + 8 * nn];
+                j1 = base[8 * kk * RS + RS + 8 * nn];
             }
             unsigned bh[2], bl[2];
             split_tf32(j0, bh[0], bl[0]);
@@ -183,42 +178,43 @@ __device__ __forceinline__ void chain_step64(float (&acc)[2][8][4], const float 
 template <bool REV>
 __device__ __forceinline__ float matvec64(const float *Ms, const float *ycur, int i)
 {
+    constexpr int RS = RingRow<64, REV>::RS;
     float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
     if (!REV) {
-        const int flip = (i >> 2) & 1;             // halves of a quarter-warp start on different pieces
-        const int sw = ((i ^ (i >> 2)) & 3) << 1;
-        const float *row = Ms + i * 64;
+        const int flip = (i >> 2) & 1;             // rows 4..7 of a quarter-warp start on the odd pieces
+        const float *row = Ms + i * RS;
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             const int ch = k ^ flip;
-            const float4 jv = *reinterpret_cast<const float4 *>(row + ((ch ^ sw) << 2));
+            const float4 jv = *reinterpret_cast<const float4 *>(row + (ch << 2));
             const float4 yv = *reinterpret_cast<const float4 *>(ycur + (ch << 2));
             s0 = fmaf(jv.x, yv.x, s0); s1 = fmaf(jv.y, yv.y, s1);
             s2 = fmaf(jv.z, yv.z, s2); s3 = fmaf(jv.w, yv.w, s3);
         }
     } else {
+        const float *col = Ms + i;
 #pragma unroll
         for (int k4 = 0; k4 < 16; ++k4) {
             const float4 yv = *reinterpret_cast<const float4 *>(ycur + 4 * k4);
-            s0 = fmaf(Ms[sw64(4 * k4, i)], yv.x, s0);
-            s1 = fmaf(Ms[sw64(4 * k4 + 1, i)], yv.y, s1);
-            s2 = fmaf(Ms[sw64(4 * k4 + 2, i)], yv.z, s2);
-            s3 = fmaf(Ms[sw64(4 * k4 + 3, i)], yv.w, s3);
+            s0 = fmaf(col[(4 * k4) * RS], yv.x, s0);
+            s1 = fmaf(col[(4 * k4 + 1) * RS], yv.y, s1);
+            s2 = fmaf(col[(4 * k4 + 2) * RS], yv.z, s2);
+            s3 = fmaf(col[(4 * k4 + 3) * RS], yv.w, s3);
         }
     }
-    return ((s0 + s1) + (s2 + s3)) + Ms[Cta64::NN + i];
+    return ((s0 + s1) + (s2 + s3)) + Ms[64 * RS + i];
 }
 
 template <bool REV>
 __global__ void __launch_bounds__(Cta64::THREADS) scan_cta64_kernel(ScanArgs a, OnePassWs w)
 {
     using C = Cta64;
-    constexpr int N = C::N, NN = C::NN, AGG = C::AGG, Q = C::Q, S = C::STAGES;
+    constexpr int N = C::N, NN = C::NN, AGG = C::AGG, Q = C::Q, S = C::STAGES, RS = RingRow<64, REV>::RS;
     if (loop_ended(a.st)) return;
 
     extern __shared__ __align__(16) float smem_raw[];
     float *sm = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
-    float *ring = sm;                              // S x (swizzled matrix, vector)
+    float *ring = sm;                              // S x (padded matrix, vector)
     float *ybuf = ring + S * C::STAGE_FLOATS;      // 2 x N: running state of the mat-vec chain
     __shared__ int s_kind, s_seq, s_c, s_abort, s_role;
 
@@ -306,18 +302,18 @@ __global__ void __launch_bounds__(Cta64::THREADS) scan_cta64_kernel(ScanArgs a, 
                             if ((row & 3) == 2) v.z = 1.0f;
                             if ((row & 3) == 3) v.w = 1.0f;
                         }
-                        *reinterpret_cast<float4 *>(dst + sw64(row, 4 * ch)) = v;
+                        *reinterpret_cast<float4 *>(dst + row * RS + 4 * ch) = v;
                     }
                 } else {
                     const float *src = REV ? Jseq + (size_t)(T - s) * NN : Jseq + (size_t)s * NN;
 #pragma unroll
                     for (int u = 0; u < NN / 4 / C::THREADS; ++u) {
                         const int j = tid + u * C::THREADS;
-                        cp_async16(dst + sw64(j >> 4, 4 * (j & 15)), src + 4 * j);
+                        cp_async16(dst + (j >> 4) * RS + 4 * (j & 15), src + 4 * j);
                     }
                 }
                 const size_t tt = REV ? (size_t)(T - 1 - s) : (size_t)s;
-                if (tid < N / 4) cp_async16(dst + NN + 4 * tid, bseq + tt * N + 4 * tid);
+                if (tid < N / 4) cp_async16(dst + N * RS + 4 * tid, bseq + tt * N + 4 * tid);
             }
             cp_async_commit();
         };

@@ -6,7 +6,12 @@
 //     as (n/16)(n/8)(n/8) MMAs per position, each issued three times on hi/lo TF32 splits; the
 //     accumulator fragment of column block kk is the A operand of contraction block kk (the same
 //     renaming of the contraction index as for n = 8), and the B operand of (kk, nn) is the lane's
-//     8-byte piece J[8nn+g][8kk+2t .. +1] (forward) read straight from global memory;
+//     8-byte piece J[8nn+g][8kk+2t .. +1] (forward) or the scalars J[8kk+2t][8nn+g], J[8kk+2t+1][8nn+g]
+//     (reverse);
+//   * the matrices and vectors of a chain stream through a warp-private shared-memory ring filled
+//     with 16-byte cp.async copies (no registers held while loads are in flight, only __syncwarp
+//     between stages); rows are padded so that the operand reads of either direction are free
+//     of bank conflicts;
 //   * beta is carried as a separate mat-vec chain started from zero (the same routine replays the
 //     chain from its true entering state in the B item): lane (g,t) holds y[8kk+2t], y[8kk+2t+1];
 //   * warp aggregates are combined by warp 0 with the same step, reading them from shared memory.
@@ -25,10 +30,12 @@ template <int N> struct WarpN {
     static constexpr int SW = 16;                      // positions per warp chain
     static constexpr int L = WARPS * SW;               // positions per tile
     static constexpr int Q = 2;                        // pending tiles per CTA
+    static constexpr int STAGES = (N == 16) ? 6 : 3;   // ring depth per warp (positions)
+    static constexpr int STAGE_FLOATS = N * (N + 8) + N;   // matrix with padded rows, then the vector
     static constexpr int RES_WARPS = 4;                // warps of a resolver CTA that resolve
     static constexpr int RES_BATCH = (N == 16) ? 8 : 2;   // aggregates a resolver warp stages at once
     static constexpr int PEND = WARPS * AGG;           // warp aggregates kept for the B item
-    static constexpr int SM_WORK = Q * PEND + AGG + WARPS * N + N + 16;
+    static constexpr int SM_WORK = Q * PEND + WARPS * N + N + 16 + WARPS * STAGES * STAGE_FLOATS;
     static constexpr int SM_RES = RES_WARPS * RES_BATCH * AGG;
     static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
@@ -122,25 +129,62 @@ __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage
     }
 }
 
-// The lane's pieces of one position's matrix, jp[nn][kk] = {M[8kk+2t][8nn+g], M[8kk+2t+1][8nn+g]}:
-// forward M = J^T (a float2 of row 8nn+g of J), reverse M = J (two scalars of column 8nn+g).
+// Row stride (floats) of a matrix in a ring stage.  Rows are padded so that the operand reads are
+// free of bank conflicts with plain constant offsets: the forward operand reads 8-byte pieces of
+// 4 rows x 4 columns per half-warp (stride = 8 mod 32 words), the reverse operand scalars of
+// 4 rows (two apart) x 8 columns per warp (stride = 4 mod 16 words).
+template <int N, bool REV> struct RingRow { static constexpr int RS = N + (REV ? 4 : 8); };
+
+template <int K> __device__ __forceinline__ void cp_async_wait_n() { asm volatile("cp.async.wait_group %0;" ::"n"(K) : "memory"); }
+
+// One position into a ring stage: the matrix (identity when `ident`) with padded rows, then the vector.
+// Always commits one group, so the group count follows the position count.
 template <int N, bool REV>
-__device__ __forceinline__ void load_pieces(float (&jp)[N / 8][N / 8][2], const float *Jt, int g, int t, bool ident)
+__device__ __forceinline__ void issue_stage_n(float *dst, const float *Jt, const float *bt, bool valid, bool ident, int lane)
 {
-    constexpr int NT = N / 8;
+    constexpr int NN = N * N, RS = RingRow<N, REV>::RS;
+    if (valid) {
+        if (ident) {
+            for (int j = lane; j < NN / 4; j += 32) {
+                const int row = j / (N / 4), ch = j % (N / 4);
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if ((row >> 2) == ch) {
+                    if ((row & 3) == 0) v.x = 1.0f;
+                    if ((row & 3) == 1) v.y = 1.0f;
+                    if ((row & 3) == 2) v.z = 1.0f;
+                    if ((row & 3) == 3) v.w = 1.0f;
+                }
+                *reinterpret_cast<float4 *>(dst + row * RS + 4 * ch) = v;
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < NN / 4 / 32; ++u) {
+                const int j = lane + 32 * u;
+                cp_async16(dst + (j / (N / 4)) * RS + 4 * (j % (N / 4)), Jt + 4 * j);
+            }
+        }
+        if (lane < N / 4) cp_async16(dst + N * RS + 4 * lane, bt + 4 * lane);
+    }
+    cp_async_commit();
+}
+
+// The lane's pieces of one position's matrix from its ring stage,
+// jp[nn][kk] = {M[8kk+2t][8nn+g], M[8kk+2t+1][8nn+g]}: forward M = J^T, reverse M = J.
+template <int N, bool REV>
+__device__ __forceinline__ void load_pieces(float (&jp)[N / 8][N / 8][2], const float *Ms, int g, int t)
+{
+    constexpr int NT = N / 8, RS = RingRow<N, REV>::RS;
+    const float *base = REV ? Ms + (2 * t) * RS + g : Ms + g * RS + 2 * t;
 #pragma unroll
     for (int nn = 0; nn < NT; ++nn)
 #pragma unroll
         for (int kk = 0; kk < NT; ++kk) {
-            if (ident) {
-                jp[nn][kk][0] = (8 * nn + g == 8 * kk + 2 * t) ? 1.0f : 0.0f;
-                jp[nn][kk][1] = (8 * nn + g == 8 * kk + 2 * t + 1) ? 1.0f : 0.0f;
-            } else if (!REV) {
-                const float2 f = __ldg(reinterpret_cast<const float2 *>(Jt + (8 * nn + g) * N + 8 * kk + 2 * t));
+            if (!REV) {
+                const float2 f = *reinterpret_cast<const float2 *>(base + 8 * nn * RS + 8 * kk);
                 jp[nn][kk][0] = f.x; jp[nn][kk][1] = f.y;
             } else {
-                jp[nn][kk][0] = __ldg(Jt + (8 * kk + 2 * t) * N + 8 * nn + g);
-                jp[nn][kk][1] = __ldg(Jt + (8 * kk + 2 * t + 1) * N + 8 * nn + g);
+                jp[nn][kk][0] = base[8 * kk * RS + 8 * nn];
+                jp[nn][kk][1] = base[8 * kk * RS + RS + 8 * nn];
             }
         }
 }
@@ -280,11 +324,14 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
     float *pend = sm;                          // Q x warp aggregates (A row-major, then beta)
     float *wstart = pend + Q * C::PEND;        // WARPS x N states entering each warp chain
     float *ystart = wstart + WARPS * N;
+    float *ring_all = ystart + N + 16;         // WARPS x STAGES x (padded matrix, vector)
     __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int T = a.T;
+    constexpr int S = C::STAGES;
+    float *ring = ring_all + warp * S * C::STAGE_FLOATS;
 
     if (tid == 0) {
         s_abort = 0;
@@ -358,6 +405,13 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
         // matrix of scan position s: forward J[s]; reverse J[T-s] (identity at s = 0); vector at t(s)
         auto mat_ptr = [&](int s) { return REV ? Jseq + (size_t)(T - s) * NN : Jseq + (size_t)s * NN; };
         auto pos_t = [&](int s) -> size_t { return REV ? (size_t)(T - 1 - s) : (size_t)s; };
+        // chain position q -> ring stage q % S (one commit group per call, also past the end)
+        auto issue = [&](int q) {
+            const int s = sbase + q;
+            const bool valid = q < cnt;
+            issue_stage_n<N, REV>(ring + (q % S) * C::STAGE_FLOATS, valid ? mat_ptr(s) : nullptr,
+                             valid ? bseq + pos_t(s) * N : nullptr, valid, REV && s == 0, lane);
+        };
 
         if (kind == 0) {
             // ---------------------------------------------- A item
@@ -366,16 +420,23 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
             float yv[NT][2];
 #pragma unroll
             for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = 0.0f; yv[kk][1] = 0.0f; }
+#pragma unroll
+            for (int q = 0; q < S - 1; ++q) issue(q);
 #pragma unroll 1
             for (int q = 0; q < cnt; ++q) {
-                const int s = sbase + q;
+                cp_async_wait_n<S - 2>();
+                __syncwarp();                  // stage q landed for every lane; stage q-1 is free again
+                issue(q + S - 1);
+                const float *Ms = ring + (q % S) * C::STAGE_FLOATS;
                 float jp[NT][NT][2], bg[NT], ynew[NT];
-                load_pieces<N, REV>(jp, mat_ptr(s), g, t, REV && s == 0);
+                load_pieces<N, REV>(jp, Ms, g, t);
 #pragma unroll
-                for (int nn = 0; nn < NT; ++nn) bg[nn] = __ldg(bseq + pos_t(s) * N + 8 * nn + g);
+                for (int nn = 0; nn < NT; ++nn) bg[nn] = Ms[N * RingRow<N, REV>::RS + 8 * nn + g];
                 chain_step_n<N>(acc, jp);
                 matvec_step<N>(yv, jp, bg, ynew, t);
             }
+            cp_async_wait_n<0>();
+            __syncwarp();
             store_aggregate<N>(wagg + warp * AGG, acc, yv, g, t);
             __syncthreads();
             if (warp == 0) {
@@ -402,6 +463,8 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
         }
 
         // -------------------------------------------------- B item
+#pragma unroll
+        for (int q = 0; q < S - 1; ++q) issue(q);      // the chain's first positions fly while the state arrives
         if (warp == 1) {
             const unsigned long long *src = w.starts + tile_index * N;
             unsigned spins = 0;
@@ -420,7 +483,7 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
             if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
         }
         __syncthreads();
-        if (s_abort) break;
+        if (s_abort) { cp_async_wait_n<0>(); break; }
         if (warp == 0) {
             // states entering each warp chain: walk the warp aggregates from the tile's entering state
             float yv[NT][2];
@@ -455,11 +518,15 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
 #pragma unroll 1
             for (int q = 0; q < cnt; ++q) {
                 const int s = sbase + q;
+                cp_async_wait_n<S - 2>();
+                __syncwarp();
+                issue(q + S - 1);
+                const float *Ms = ring + (q % S) * C::STAGE_FLOATS;
                 float jp[NT][NT][2], bg[NT], ynew[NT];
-                load_pieces<N, REV>(jp, mat_ptr(s), g, t, REV && s == 0);
+                load_pieces<N, REV>(jp, Ms, g, t);
                 const size_t vb = ((size_t)seq * T + pos_t(s)) * N;
 #pragma unroll
-                for (int nn = 0; nn < NT; ++nn) bg[nn] = __ldg(a.b + vb + 8 * nn + g);
+                for (int nn = 0; nn < NT; ++nn) bg[nn] = Ms[N * RingRow<N, REV>::RS + 8 * nn + g];
                 matvec_step<N>(yv, jp, bg, ynew, t);
                 if (t == 0) {
 #pragma unroll
@@ -469,6 +536,7 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
                     }
                 }
             }
+            cp_async_wait_n<0>();
         }
     }
     if (a.yold) {
