@@ -30,11 +30,12 @@ template <int N> struct WarpN {
     static constexpr int SW = 16;                      // positions per warp chain
     static constexpr int L = WARPS * SW;               // positions per tile
     static constexpr int Q = 2;                        // pending tiles per CTA
-    static constexpr int STAGES = (N == 16) ? 6 : 3;   // ring depth per warp (positions)
+    static constexpr int STAGES = (N == 16) ? 4 : 2;   // ring depth per warp (positions)
     static constexpr int STAGE_FLOATS = N * (N + 8) + N;   // matrix with padded rows, then the vector
     static constexpr int RES_WARPS = 4;                // warps of a resolver CTA that resolve
     static constexpr int RES_BATCH = (N == 16) ? 8 : 2;   // aggregates a resolver warp stages at once
-    static constexpr int PEND = WARPS * AGG;           // warp aggregates kept for the B item
+    static constexpr int PEND = (WARPS - 1) * AGG;     // warp aggregates kept for the B item (the last warp's
+                                                       // is only needed by the tile combine: it sits in that warp's ring)
     static constexpr int SM_WORK = Q * PEND + WARPS * N + N + 16 + WARPS * STAGES * STAGE_FLOATS;
     static constexpr int SM_RES = RES_WARPS * RES_BATCH * AGG;
     static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
@@ -313,7 +314,7 @@ __device__ __forceinline__ void identity_fragments(float (&acc)[N / 16][N / 8][4
 }
 
 template <int N, bool REV>
-__global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs a, OnePassWs w)
+__global__ void __launch_bounds__(WarpN<N>::THREADS, (N == 16) ? 2 : 3) scan_warpn_kernel(ScanArgs a, OnePassWs w)
 {
     using C = WarpN<N>;
     constexpr int NN = C::NN, AGG = C::AGG, NT = C::NT, MT = C::MT, WARPS = C::WARPS, SW = C::SW, Q = C::Q;
@@ -437,7 +438,7 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
             }
             cp_async_wait_n<0>();
             __syncwarp();
-            store_aggregate<N>(wagg + warp * AGG, acc, yv, g, t);
+            store_aggregate<N>(warp + 1 < WARPS ? wagg + warp * AGG : ring, acc, yv, g, t);
             __syncthreads();
             if (warp == 0) {
                 // tile aggregate = the same steps with the warp aggregates as positions (forward form)
@@ -446,7 +447,7 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS) scan_warpn_kernel(ScanArgs 
                 for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = 0.0f; yv[kk][1] = 0.0f; }
 #pragma unroll 1
                 for (int k = 0; k < WARPS; ++k) {
-                    const float *ak = wagg + k * AGG;
+                    const float *ak = k + 1 < WARPS ? wagg + k * AGG : ring_all + (WARPS - 1) * S * C::STAGE_FLOATS;
                     float jp[NT][NT][2], bg[NT], ynew[NT];
                     load_pieces_smem<N>(jp, ak, g, t);
 #pragma unroll
