@@ -77,13 +77,16 @@ struct ScanWs {
     OnePassWs op;        // single-pass path (n in {1,2,4,8}); op.nch == 0 when not applicable
 };
 
-static int onepass_tile_len(int n)
+static int num_sms();
+
+static int onepass_tile_len(int n, int B, int T, int *sw)
 {
+    *sw = 0;
     switch (n) {
     case 1: return OnePass<1>::L;
     case 2: return OnePass<2>::L;
     case 4: return OnePass<4>::L;
-    case 8: return Warp8::L;
+    case 8: *sw = Warp8::chain_len(B, T, 4 * num_sms()); return Warp8::WARPS * *sw;
     case 16: return WarpN<16>::L;
     case 32: return WarpN<32>::L;
     case 64: return Cta64::L;
@@ -100,7 +103,7 @@ static ScanWs carve_scan(Carver &cv, int B, int T, int n)
     w.carB = cv.take<float>((size_t)B * w.nch * n);
     w.starts = cv.take<float>((size_t)B * w.nch * n);
     w.op = OnePassWs{};
-    int L1 = onepass_tile_len(n);
+    int L1 = onepass_tile_len(n, B, T, &w.op.sw);
     if (L1) {
         w.op.nch = (T + L1 - 1) / L1;
         size_t tiles = (size_t)B * w.op.nch;

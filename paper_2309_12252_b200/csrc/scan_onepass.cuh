@@ -73,6 +73,7 @@ struct OnePassWs {
     int nch, Wd, nwin;            // tiles per sequence, tiles per sequence per window, windows
     unsigned total_ids;
     int resolvers;                // CTAs that take the resolver role
+    int sw;                       // positions per warp chain where the kernel takes it at run time (n = 8)
 };
 
 // ---------------------------------------------------------------- small PTX helpers

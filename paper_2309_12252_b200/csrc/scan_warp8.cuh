@@ -25,8 +25,7 @@ namespace deer {
 struct Warp8 {
     static constexpr int N = 8, NN = 64, AGG = 72;
     static constexpr int WARPS = 8, THREADS = 256;
-    static constexpr int SW = 32;                      // positions per warp chain
-    static constexpr int L = WARPS * SW;               // positions per tile
+    static constexpr int SW_MIN = 32, SW_MAX = 256;    // positions per warp chain (chosen per problem size)
     static constexpr int GRP = 8;                      // positions loaded ahead per group
     static constexpr int Q = 2;                        // pending tiles per CTA
     static constexpr int RES_WARPS = 4;                // warps of a resolver CTA that resolve
@@ -35,7 +34,17 @@ struct Warp8 {
     static constexpr int SM_RES = RES_WARPS * 32 * AGG;
     static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
-    static_assert(SW % GRP == 0, "chains are processed in whole groups");
+    static_assert(SW_MIN % GRP == 0, "chains are processed in whole groups");
+    // Longer chains mean fewer tiles for the resolvers to walk (their per-tile cost is what bounds
+    // the scan at large T), shorter ones more tiles to spread over the SMs: take the longest
+    // chain that still leaves about 1.5 tiles per resident CTA (measured optimum for B = 16,
+    // T = 3e3 ... 1e6).
+    static int chain_len(int B, int T, int resident_ctas)
+    {
+        int sw = SW_MAX;
+        while (sw > SW_MIN && (long long)B * ((T + WARPS * sw - 1) / (WARPS * sw)) < 3LL * resident_ctas / 2) sw >>= 1;
+        return sw;
+    }
 };
 
 // d = a * b + c   (m16n8k8, A row-major 16x8, B 8x8, TF32 inputs, fp32 accumulate)
@@ -79,8 +88,9 @@ template <bool REV>
 __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs a, OnePassWs w)
 {
     using C = Warp8;
-    constexpr int N = C::N, NN = C::NN, AGG = C::AGG, WARPS = C::WARPS, SW = C::SW, GRP = C::GRP, Q = C::Q;
+    constexpr int N = C::N, NN = C::NN, AGG = C::AGG, WARPS = C::WARPS, GRP = C::GRP, Q = C::Q;
     if (loop_ended(a.st)) return;
+    const int SW = w.sw, L = WARPS * SW;
 
     extern __shared__ __align__(16) float smem_raw[];
     float *sm = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
@@ -154,8 +164,8 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
         if (s_kind < 0 || s_abort) break;
         const int kind = s_kind, seq = s_seq, c = s_c;
         float *wagg = pend + s_slot * C::PEND;
-        const int s0 = c * C::L;                               // first scan position of the tile
-        const int Lt = min(C::L, T - s0);
+        const int s0 = c * L;                                  // first scan position of the tile
+        const int Lt = min(L, T - s0);
         const int p0 = warp * SW;                              // first scan offset of this warp's chain
         const int cnt = min(SW, max(0, Lt - p0));
         const size_t tile_index = (size_t)seq * w.nch + c;
