@@ -87,8 +87,8 @@ static int onepass_tile_len(int n, int B, int T, int *sw)
     case 2: return OnePass<2>::L;
     case 4: return OnePass<4>::L;
     case 8: *sw = Warp8::chain_len(B, T, 4 * num_sms()); return Warp8::WARPS * *sw;
-    case 16: return WarpN<16>::L;
-    case 32: return WarpN<32>::L;
+    case 16: *sw = WarpN<16>::chain_len(B, T, WarpN<16>::CTAS_PER_SM * num_sms()); return WarpN<16>::WARPS * *sw;
+    case 32: *sw = WarpN<32>::chain_len(B, T, WarpN<32>::CTAS_PER_SM * num_sms()); return WarpN<32>::WARPS * *sw;
     case 64: return Cta64::L;
     default: return 0;
     }

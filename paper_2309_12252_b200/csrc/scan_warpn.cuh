@@ -27,8 +27,15 @@ template <int N> struct WarpN {
     static constexpr int MT = N / 16;                  // 16-high row blocks of X
     static constexpr int WARPS = (N == 16) ? 8 : 4;    // chains per tile
     static constexpr int THREADS = WARPS * 32;
-    static constexpr int SW = 16;                      // positions per warp chain
-    static constexpr int L = WARPS * SW;               // positions per tile
+    static constexpr int SW_MIN = 16, SW_MAX = 64;     // positions per warp chain (chosen per problem size)
+    static constexpr int CTAS_PER_SM = (N == 16) ? 2 : 3;
+    // longest chain that still leaves about 1.5 tiles per resident CTA (see Warp8::chain_len)
+    static int chain_len(int B, int T, int resident_ctas)
+    {
+        int sw = SW_MAX;
+        while (sw > SW_MIN && (long long)B * ((T + WARPS * sw - 1) / (WARPS * sw)) < 3LL * resident_ctas / 2) sw >>= 1;
+        return sw;
+    }
     static constexpr int Q = 2;                        // pending tiles per CTA
     static constexpr int STAGES = (N == 16) ? 4 : 2;   // ring depth per warp (positions)
     static constexpr int STAGE_FLOATS = N * (N + 8) + N;   // matrix with padded rows, then the vector
@@ -314,10 +321,10 @@ __device__ __forceinline__ void identity_fragments(float (&acc)[N / 16][N / 8][4
 }
 
 template <int N, bool REV>
-__global__ void __launch_bounds__(WarpN<N>::THREADS, (N == 16) ? 2 : 3) scan_warpn_kernel(ScanArgs a, OnePassWs w)
+__global__ void __launch_bounds__(WarpN<N>::THREADS, WarpN<N>::CTAS_PER_SM) scan_warpn_kernel(ScanArgs a, OnePassWs w)
 {
     using C = WarpN<N>;
-    constexpr int NN = C::NN, AGG = C::AGG, NT = C::NT, MT = C::MT, WARPS = C::WARPS, SW = C::SW, Q = C::Q;
+    constexpr int NN = C::NN, AGG = C::AGG, NT = C::NT, MT = C::MT, WARPS = C::WARPS, Q = C::Q;
     if (loop_ended(a.st)) return;
 
     extern __shared__ __align__(16) float smem_raw[];
@@ -333,6 +340,7 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS, (N == 16) ? 2 : 3) scan_war
     const int T = a.T;
     constexpr int S = C::STAGES;
     float *ring = ring_all + warp * S * C::STAGE_FLOATS;
+    const int SW = w.sw, L = WARPS * SW;
 
     if (tid == 0) {
         s_abort = 0;
@@ -395,8 +403,8 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS, (N == 16) ? 2 : 3) scan_war
         if (s_kind < 0 || s_abort) break;
         const int kind = s_kind, seq = s_seq, c = s_c;
         float *wagg = pend + s_slot * C::PEND;
-        const int s0 = c * C::L;
-        const int Lt = min(C::L, T - s0);
+        const int s0 = c * L;
+        const int Lt = min(L, T - s0);
         const int p0 = warp * SW;
         const int cnt = min(SW, max(0, Lt - p0));
         const int sbase = s0 + p0;                             // scan position of the chain's first element
