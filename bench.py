@@ -46,6 +46,11 @@ def peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
 
 
+# DRAM bytes (read + write) per position of the stand-alone scan, from the ncu captures summarised in
+# profiles/scan_kernels_standalone_B16.md (inputs larger than L2; traffic grows in proportion to positions).
+NCU_SCAN_TRAFFIC_PER_POSITION = {1: 13.9, 2: 35.8, 4: 95.6, 8: 606.6, 16: 2213.0, 32: 8622.0, 64: 34116.0}
+
+
 def scan_bytes_per_position(n: int) -> int:
     """Algorithmic bytes of one scan per position: read J and b once, write y."""
     return 4 * (n * n + n) + 4 * n
@@ -275,6 +280,39 @@ def run_eval_only(args):
     print(json.dumps(out))
 
 
+def run_classifier(args):
+    """Config 4: one full training step (loss + all gradients) of the 2-layer GRU classifier: one JSON line."""
+    import torch
+    from paper_2309_12252_b200 import binding as bd
+    from paper_2309_12252_b200 import synth
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    w = synth.config4(seed=0, B=args.B, T=args.T)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
+    l1 = bd.GruParamsDev.from_numpy(w.layers[0]); l2 = bd.GruParamsDev.from_numpy(w.layers[1])
+    W_o, b_o, x, labels = dev(w.W_o), dev(w.b_o), dev(w.x), dev(w.labels)
+    n, m = w.layers[0].n, w.layers[0].m
+    ws = bd.alloc_workspace(bd.DEER_OP_CLASSIFIER, args.B, args.T, n, m, args.flags, device)
+    stream = torch.cuda.current_stream()
+    run = lambda: bd.deer_gru_classifier_step(l1, l2, W_o, b_o, x, labels, ws=ws, flags=args.flags, stream=stream)
+    for _ in range(max(args.warmup, 1)):
+        r = run()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    for a, b in ev:
+        a.record(stream); r = run(); b.record(stream)
+    torch.cuda.synchronize()
+    ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+    bd.lib().deer_profile_enable(1)
+    run()
+    torch.cuda.synchronize()
+    bd.lib().deer_profile_enable(0)
+    prof = read_profile(bd)
+    print(json.dumps(dict(mode="classifier", B=args.B, T=args.T, n=n, m=m, ms=ms, steps_per_s=args.B * args.T / (ms * 1e-3),
+                          loss=r["loss"], iters=list(r["iters"]), status=r["status"],
+                          kernels={k: dict(launches=v["launches"], ms=round(v["total_ms"], 4)) for k, v in prof.items()})))
+
+
 def run_sweep(args):
     """The paper's speed grid (Table of forward speed-ups), thinned: n = m in {1..64} x T in {1e3..1e6},
     B = 16, x ~ N(0,1); one JSON line with one entry per point (n = 64, T = 1e6 is left out)."""
@@ -298,7 +336,7 @@ def run_sweep(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--mode", default="step", choices=["step", "scan", "eval", "sweep"])
+    ap.add_argument("--mode", default="step", choices=["step", "scan", "eval", "sweep", "classifier"])
     ap.add_argument("--m", type=int, default=0)
     ap.add_argument("--vjp", type=int, default=0)
     ap.add_argument("--n", type=int, default=8)
@@ -324,6 +362,9 @@ def main():
         return
     if args.mode == "sweep":
         run_sweep(args)
+        return
+    if args.mode == "classifier":
+        run_classifier(args)
         return
 
     import torch
@@ -449,7 +490,12 @@ def main():
         ach = scan_bytes_per_position(sn) * sB * sT / (ms * 1e-3) / 1e9
         roofline_hbm = dict(bound="hbm", kernel="deer_linrec_scan", workload=f"n={sn} B={sB} T={sT} (J 4.1 GB, inputs > L2)",
                             achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
-                            peak_source=pk["source"], ms=ms, traffic=None)
+                            peak_source=pk["source"], ms=ms,
+                            traffic=NCU_SCAN_TRAFFIC_PER_POSITION[sn] * sB * sT,
+                            traffic_note="bytes per launch: ncu capture at T=200000 scaled by positions "
+                                         "(profiles/scan_kernels_standalone_B16.md)",
+                            frac_two_reads=(scan_bytes_per_position(sn) + 4 * (sn * sn + sn)) * sB * sT
+                                           / (ms * 1e-3) / 1e9 / pk["hbm_gbs"])
         del J, bb, yy, sws
 
     cpu = None
