@@ -247,8 +247,26 @@ def test_config3_gradient_reduced_T(bd):
         assert rel_inf(got[k].cpu().numpy().astype(np.float64), want[k]) <= TOL_GRAD, k
 
 
+def test_config3_gradient_full_size(bd):
+    """Config 3 at its full size (B=16, T=1e5, n=m=32), in the launch configuration the benchmark
+    uses: both losses of the benchmark definition (terminal L = sum(y_T . w), and a dense gy)."""
+    w = synth.config(3)
+    r = run_eval(bd, w)
+    assert r.status == 0
+    y32 = oracle.gru_seq(w.params, w.x, w.y0, np.float32)
+    p = bd.GruParamsDev.from_numpy(w.params)
+    wv = synth.normal(0, "c3/w", (16, 32))
+    gy_last = np.zeros((16, 100000, 32), np.float32); gy_last[:, -1] = wv
+    gy_dense = synth.normal(0, "c3/gy", (16, 100000, 32)).astype(np.float32)
+    for gy in (gy_last, gy_dense):
+        want = oracle.gru_bptt(w.params, w.x, w.y0, y32.astype(np.float64), gy, np.float64)
+        got = bd.deer_gru_vjp(p, dev(w.x), dev(w.y0), r.y, dev(gy))
+        for k in ("dW_i", "dW_h", "db_i", "db_h", "dx", "dy0"):
+            assert rel_inf(got[k].cpu().numpy().astype(np.float64), want[k]) <= TOL_GRAD, k
+
+
 # ----------------------------------------------------------------------------- classifier
-@pytest.mark.parametrize("B,T,n,m", [(3, 200, 8, 3), (4, 1500, 64, 6)])
+@pytest.mark.parametrize("B,T,n,m", [(3, 200, 8, 3), (4, 1500, 64, 6), (32, 17984, 64, 6)])
 def test_classifier_step_matches_oracle(bd, B, T, n, m):
     w = synth.config4(seed=2, B=B, T=T, n=n, m=m)
     want = oracle.classifier(w.layers, w.W_o, w.b_o, w.x, w.labels, np.float64)
