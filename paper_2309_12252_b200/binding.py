@@ -20,7 +20,7 @@ DEER_OK, DEER_NOT_CONVERGED, DEER_NONFINITE = 0, 1, 2
 DEER_ERR_INVALID_ARG, DEER_ERR_UNSUPPORTED_N, DEER_ERR_WORKSPACE = -1, -2, -3
 DEER_ERR_CUDA, DEER_ERR_DEVICE_TIMEOUT = -4, -5
 DEER_OP_EVAL, DEER_OP_SCAN, DEER_OP_VJP, DEER_OP_CLASSIFIER = 0, 1, 2, 3
-DEER_FLAG_WARM_START, DEER_FLAG_GENERIC, DEER_FLAG_MATERIALIZE = 1, 2, 4
+DEER_FLAG_WARM_START, DEER_FLAG_GENERIC, DEER_FLAG_MATERIALIZE, DEER_FLAG_TCGEN05 = 1, 2, 4, 8
 
 NOALLOC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc", "deer_gru_eval", "deer_gru_vjp",

@@ -16,6 +16,7 @@
 #include "scan_warp8.cuh"
 #include "scan_warpn.cuh"
 #include "scan_cta64.cuh"
+#include "scan_umma64.cuh"
 #include "cell_wide.cuh"
 #include "vjp_wide.cuh"
 
@@ -220,8 +221,18 @@ static int launch_cta64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
     return launch_single_pass(scan_cta64_kernel<REV>, occ, c, a, w, prep, st);
 }
 
-static int scan_onepass(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
+template <bool REV>
+static int launch_umma64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
+    using C = Umma64;
+    static int occ = 0;
+    const PassCfg c{"scan_umma64_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 2, 8};
+    return launch_single_pass(scan_umma64_kernel<REV>, occ, c, a, w, prep, st);
+}
+
+static int scan_onepass(ScanArgs a, OnePassWs w, bool prep, int flags, cudaStream_t st)
+{
+    const bool umma = (flags & DEER_FLAG_TCGEN05) != 0;
     switch (a.n * 2 + (a.reverse ? 1 : 0)) {
     case 2: return launch_onepass<1, false>(a, w, prep, st);
     case 3: return launch_onepass<1, true>(a, w, prep, st);
@@ -235,8 +246,8 @@ static int scan_onepass(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
     case 33: return launch_warpn<16, true>(a, w, prep, st);
     case 64: return launch_warpn<32, false>(a, w, prep, st);
     case 65: return launch_warpn<32, true>(a, w, prep, st);
-    case 128: return launch_cta64<false>(a, w, prep, st);
-    case 129: return launch_cta64<true>(a, w, prep, st);
+    case 128: return umma ? launch_umma64<false>(a, w, prep, st) : launch_cta64<false>(a, w, prep, st);
+    case 129: return umma ? launch_umma64<true>(a, w, prep, st) : launch_cta64<true>(a, w, prep, st);
     default: return DEER_ERR_UNSUPPORTED_N;
     }
 }
@@ -277,7 +288,7 @@ static bool scan_is_single_pass(const ScanArgs &a, const ScanWs &w, int flags)
 // left them cleared)
 static int run_scan(ScanArgs a, const ScanWs &w, int flags, cudaStream_t st, bool prep = true)
 {
-    if (scan_is_single_pass(a, w, flags)) return scan_onepass(a, w.op, prep, st);
+    if (scan_is_single_pass(a, w, flags)) return scan_onepass(a, w.op, prep, flags, st);
     return scan_generic(a, st);
 }
 
@@ -587,7 +598,7 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
             if ((rc = run_cell(c, st)) != DEER_OK) return rc;
             a.y = nxt; a.yold = cur;
             if (single) {
-                if ((rc = scan_onepass(a, w.scan.op, false, st)) != DEER_OK) return rc;
+                if ((rc = scan_onepass(a, w.scan.op, false, flags, st)) != DEER_OK) return rc;
             } else {
                 if ((rc = scan_generic(a, st)) != DEER_OK) return rc;
                 DEER_KERNEL("newton_control_kernel", st, newton_control_kernel<<<1, 1, 0, st>>>(w.st, tol, max_iter, w.trace));

@@ -56,6 +56,19 @@ def test_linrec_scan_vs_oracle(bd, n, B, T, reverse, flags):
         assert np.max(np.abs(got - want)) <= TOL_SCAN * scale
 
 
+@pytest.mark.parametrize("B,T", [(2, 70), (3, 64), (2, 1), (4, 1000), (16, 333)])
+@pytest.mark.parametrize("reverse", [False, True])
+def test_linrec_scan_n64_tcgen05_path(bd, B, T, reverse):
+    """The n = 64 chain product on tcgen05 (tensor-memory accumulator) gives the same scan."""
+    n = 64
+    J = synth.contractive_J(B, T, n, seed=7 + T, tag="g/J64", scale=1.0)
+    b = synth.normal(7 + T, "g/b64", (B, T, n))
+    y0 = synth.normal(7 + T, "g/y064", (B, n))
+    want = oracle.linrec(J, b, y0, reverse=reverse, dtype=np.float64)
+    got = bd.deer_linrec_scan(dev(J), dev(b), dev(y0), reverse=reverse, flags=bd.DEER_FLAG_TCGEN05).cpu().numpy()
+    assert np.max(np.abs(got - want)) <= TOL_SCAN * max(1.0, float(np.max(np.abs(want))))
+
+
 def test_linrec_scan_growing_products(bd):
     """Non-contractive J (norm > 1 over short stretches): error relative to max|y|."""
     n, B, T = 4, 2, 60
