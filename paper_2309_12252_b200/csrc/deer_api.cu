@@ -115,16 +115,19 @@ static ScanWs carve_scan(Carver &cv, int B, int T, int n)
     return w;
 }
 
-static int g_num_sms = 0;
+constexpr int MAX_DEVICES = 64;
+static int g_num_sms[MAX_DEVICES] = {0};
 static int num_sms()
 {
-    if (!g_num_sms) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (g_num_sms <= 0) g_num_sms = 148;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= MAX_DEVICES) dev = 0;
+    if (!g_num_sms[dev]) {
+        int v = 0;
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+        g_num_sms[dev] = v > 0 ? v : 148;
     }
-    return g_num_sms;
+    return g_num_sms[dev];
 }
 
 // Clears the single-pass scan's flag / state words and counters (needed once per workspace: the
@@ -153,8 +156,14 @@ struct PassCfg {
 // One persistent launch: grid = resident CTAs (or fewer when there are few tiles); the first
 // `resolvers` role tickets become resolver CTAs.
 template <typename Kern>
-static int launch_single_pass(Kern kern, int &occ, const PassCfg &c, ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
+static int launch_single_pass(Kern kern, int (&occ_dev)[MAX_DEVICES], const PassCfg &c, ScanArgs a, OnePassWs w, bool prep,
+                              cudaStream_t st)
 {
+    // the shared-memory opt-in and the occupancy are per device: looked up on each device's first launch
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= MAX_DEVICES) dev = 0;
+    int &occ = occ_dev[dev];
     if (!occ) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
         if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(single-pass scan)"); return DEER_ERR_CUDA; }
@@ -189,7 +198,7 @@ template <int N, bool REV>
 static int launch_onepass(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = OnePass<N>;
-    static int occ = 0;
+    static int occ[MAX_DEVICES] = {0};
     const PassCfg c{"scan_onepass_kernel", C::THREADS, C::SMEM, C::WARPS, C::MAX_SEQ_PER_WARP, 32, 8};
     return launch_single_pass(scan_onepass_kernel<N, REV>, occ, c, a, w, prep, st);
 }
@@ -198,7 +207,7 @@ template <bool REV>
 static int launch_warp8(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = Warp8;
-    static int occ = 0;
+    static int occ[MAX_DEVICES] = {0};
     const PassCfg c{"scan_warp8_kernel", C::THREADS, C::SMEM, C::RES_WARPS, OnePass<8>::MAX_SEQ_PER_WARP, 4, 8};
     return launch_single_pass(scan_warp8_kernel<REV>, occ, c, a, w, prep, st);
 }
@@ -207,7 +216,7 @@ template <int N, bool REV>
 static int launch_warpn(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = WarpN<N>;
-    static int occ = 0;
+    static int occ[MAX_DEVICES] = {0};
     const PassCfg c{"scan_warpn_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 8};
     return launch_single_pass(scan_warpn_kernel<N, REV>, occ, c, a, w, prep, st);
 }
@@ -216,7 +225,7 @@ template <bool REV>
 static int launch_cta64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = Cta64;
-    static int occ = 0;
+    static int occ[MAX_DEVICES] = {0};
     const PassCfg c{"scan_cta64_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 16};
     return launch_single_pass(scan_cta64_kernel<REV>, occ, c, a, w, prep, st);
 }
@@ -225,7 +234,7 @@ template <bool REV>
 static int launch_umma64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = Umma64;
-    static int occ = 0;
+    static int occ[MAX_DEVICES] = {0};
     const PassCfg c{"scan_umma64_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 2, 8};
     return launch_single_pass(scan_umma64_kernel<REV>, occ, c, a, w, prep, st);
 }

@@ -119,13 +119,14 @@ __global__ void __launch_bounds__(256) cell_small_kernel(CellArgs a)
 #pragma unroll
             for (int k = 0; k < N; ++k) h[k] = hp[k];
         }
-        float gr = br, gz = bz, gq = bn;
+        float sr = 0.0f, sz = 0.0f, sq = 0.0f;          // bias-free products W_h* h
 #pragma unroll
         for (int k = 0; k < N; ++k) {
-            gr = fmaf(wr[k], h[k], gr);
-            gz = fmaf(wz[k], h[k], gz);
-            gq = fmaf(wn[k], h[k], gq);
+            sr = fmaf(wr[k], h[k], sr);
+            sz = fmaf(wz[k], h[k], sz);
+            sq = fmaf(wn[k], h[k], sq);
         }
+        const float gr = sr + br, gz = sz + bz, gq = sq + bn;
         float ur, uz, un;
         if constexpr (M > 0) {
             const float *xe = a.x + e * M;
@@ -142,22 +143,20 @@ __global__ void __launch_bounds__(256) cell_small_kernel(CellArgs a)
         const float r = sigmoidf_acc(ur + gr);
         const float z = sigmoidf_acc(uz + gz);
         const float c = tanhf(un + r * gq);
-        float hi = 0.0f;
-#pragma unroll
-        for (int k = 0; k < N; ++k) if (k == i) hi = h[k];
+        const float hi = hp[i];
         const float f = (1.0f - z) * c + z * hi;
         const float az = (hi - c) * z * (1.0f - z);
         const float an = (1.0f - z) * (1.0f - c * c);
         const float kr = an * gq * r * (1.0f - r);
         const float kn = an * r;
         float v[N];
-        float acc = 0.0f;
 #pragma unroll
         for (int j = 0; j < N; ++j) {
             v[j] = kr * wr[j] + az * wz[j] + kn * wn[j];
             if (j == i) v[j] += z;
-            acc = fmaf(v[j], h[j], acc);
         }
+        // J h = z h_i + a_z (W_hz h)_i + k_n (W_hn h)_i + k_r (W_hr h)_i, from the gate accumulators
+        const float acc = fmaf(kr, sr, fmaf(kn, sq, fmaf(az, sz, z * hi)));
         float *Jr = a.J + (e * N + i) * N;
         if constexpr (N >= 4) {
 #pragma unroll
