@@ -301,10 +301,37 @@ static int run_scan(ScanArgs a, const ScanWs &w, int flags, cudaStream_t st, boo
     return scan_generic(a, st);
 }
 
+// tensor-core affine map (K = inputs, nout = outputs; see affine_mma_kernel)
+template <int NB_MAX, bool WT>
+static int launch_affine_mma(const float *in, const float *W, const float *bias, float *out, size_t N, int K, int nout,
+                             cudaStream_t st)
+{
+    const size_t sm = sizeof(float) * 2 * (size_t)K * (nout + 4);
+    int rc;
+    if ((rc = opt_in_smem((const void *)affine_mma_kernel<NB_MAX, WT>, sm)) != DEER_OK) return rc;
+    const size_t tiles = (N + 127) / 128;
+    const size_t per_sm = sm > 110 * 1024 ? 1 : 2;
+    const size_t cap = (size_t)num_sms() * per_sm;
+    const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
+    DEER_KERNEL("affine_mma_kernel", st, (affine_mma_kernel<NB_MAX, WT><<<blocks, 256, sm, st>>>(in, W, bias, out, N, K, nout)));
+    return DEER_OK;
+}
+
 // out[e][g] = bias[g] + sum_k W[g][k] in[e][k]   (wt_given: W is stored [k][g]; bias may be null)
 static int run_affine(const float *in, const float *W, const float *bias, float *out, size_t N, int m, int n3,
                       int wt_given, cudaStream_t st)
 {
+    // tensor-core path: K and the output count multiples of 8, 8-byte aligned rows, weights fit shared memory
+    const bool aligned8 = (((uintptr_t)in | (uintptr_t)out) & 7) == 0;
+    if (aligned8 && m % 8 == 0 && m >= 16 && n3 % 8 == 0 && n3 <= 192 &&
+        sizeof(float) * 2 * (size_t)m * (n3 + 4) <= 200 * 1024) {
+        if (n3 <= 64) return wt_given ? launch_affine_mma<8, true>(in, W, bias, out, N, m, n3, st)
+                                      : launch_affine_mma<8, false>(in, W, bias, out, N, m, n3, st);
+        if (n3 <= 96) return wt_given ? launch_affine_mma<12, true>(in, W, bias, out, N, m, n3, st)
+                                      : launch_affine_mma<12, false>(in, W, bias, out, N, m, n3, st);
+        return wt_given ? launch_affine_mma<24, true>(in, W, bias, out, N, m, n3, st)
+                        : launch_affine_mma<24, false>(in, W, bias, out, N, m, n3, st);
+    }
     int G = 256 / n3;
     while (G > 1 && sizeof(float) * (size_t)G * PROJ_PP * (m + 1) > 64 * 1024) --G;
     const size_t sm = sizeof(float) * ((size_t)m * n3 + (size_t)G * PROJ_PP * (m + 1));

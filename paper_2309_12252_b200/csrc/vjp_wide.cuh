@@ -144,4 +144,76 @@ __global__ void __launch_bounds__(384) wgrad_mma_kernel(WgradArgs a)
     if (t == 0) { out[row * K1 + K] = bs0; out[(row + 8) * K1 + K] = bs1; }
 }
 
+// ------------------------------------------------------------------ a0 / a8: dense affine map on tensor cores
+//   out[e][c] = bias[c] + sum_k W(c,k) in[e][k],   W(c,k) = W[c*K + k]  (weights [out][in], the input
+//   projection u = x W_i^T + b_i)  or  W[k*NOUT + c]  (WT_GIVEN: weights [in][out], dx = dG_i W_i).
+// The batched [B*T, K] x [K, NOUT] contraction of the path: CTA = 8 warps, warp = 16 positions x all
+// NOUT outputs, m16n8k8 TF32 MMAs issued three times on hi/lo splits (fp32-level accuracy).  The
+// weights are split once per CTA into shared memory, rows padded so that the B-fragment reads are
+// conflict-free; the contraction index is renamed so that a lane's two A values of a K step are
+// adjacent in memory (one 8-byte load per row).  K % 8 == 0, NOUT % 8 == 0, NOUT <= 192.
+template <int NB_MAX, bool WT_GIVEN>
+__global__ void __launch_bounds__(256) affine_mma_kernel(const float *__restrict__ in, const float *__restrict__ W,
+                                                         const float *__restrict__ bias, float *__restrict__ out,
+                                                         size_t N, int K, int NOUT)
+{
+    extern __shared__ __align__(16) float smw[];
+    const int NS = NOUT + 4;                  // row stride: 2 * NS = 8 (mod 32) words
+    float *sBh = smw, *sBl = smw + (size_t)K * NS;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    for (int idx = tid; idx < K * NOUT; idx += 256) {
+        const int k = idx / NOUT, c = idx % NOUT;
+        const float v = WT_GIVEN ? W[idx] : W[(size_t)c * K + k];
+        sBh[k * NS + c] = v;
+        sBl[k * NS + c] = v - __uint_as_float(__float_as_uint(v) & 0xffffe000u);
+    }
+    __syncthreads();
+    const int nb = NOUT >> 3;
+    const size_t ntiles = (N + 127) / 128;
+    for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const size_t p0 = tile * 128 + warp * 16;
+        if (p0 >= N) continue;
+        const size_t r0 = p0 + g, r1 = p0 + g + 8;
+        const bool v0 = r0 < N, v1 = r1 < N;
+        float acc[NB_MAX][4];
+#pragma unroll
+        for (int nn = 0; nn < NB_MAX; ++nn) {
+            const float b0 = (bias && nn < nb) ? bias[8 * nn + 2 * t] : 0.0f, b1 = (bias && nn < nb) ? bias[8 * nn + 2 * t + 1] : 0.0f;
+            acc[nn][0] = b0; acc[nn][1] = b1; acc[nn][2] = b0; acc[nn][3] = b1;
+        }
+        const float *a0p = in + (v0 ? r0 : 0) * K + 2 * t, *a1p = in + (v1 ? r1 : 0) * K + 2 * t;
+#pragma unroll 1
+        for (int k0 = 0; k0 < K; k0 += 8) {
+            // slots t and t+4 of the K step hold k0+2t and k0+2t+1
+            const float2 x0 = v0 ? __ldg(reinterpret_cast<const float2 *>(a0p + k0)) : make_float2(0.f, 0.f);
+            const float2 x1 = v1 ? __ldg(reinterpret_cast<const float2 *>(a1p + k0)) : make_float2(0.f, 0.f);
+            unsigned ah[4], al[4];
+            split_tf32(x0.x, ah[0], al[0]);      // a0: (row g,   slot t)
+            split_tf32(x1.x, ah[1], al[1]);      // a1: (row g+8, slot t)
+            split_tf32(x0.y, ah[2], al[2]);      // a2: (row g,   slot t+4)
+            split_tf32(x1.y, ah[3], al[3]);      // a3: (row g+8, slot t+4)
+            const float *bh0 = sBh + (k0 + 2 * t) * NS + g, *bl0 = sBl + (k0 + 2 * t) * NS + g;
+#pragma unroll
+            for (int nn = 0; nn < NB_MAX; ++nn) {
+                if (nn < nb) {
+                    unsigned bh[2], bl[2];
+                    bh[0] = __float_as_uint(bh0[8 * nn]); bh[1] = __float_as_uint(bh0[8 * nn + NS]);
+                    bl[0] = __float_as_uint(bl0[8 * nn]); bl[1] = __float_as_uint(bl0[8 * nn + NS]);
+                    mma_tf32(acc[nn], al, bh, acc[nn]);
+                    mma_tf32(acc[nn], ah, bl, acc[nn]);
+                    mma_tf32(acc[nn], ah, bh, acc[nn]);
+                }
+            }
+        }
+#pragma unroll
+        for (int nn = 0; nn < NB_MAX; ++nn) {
+            if (nn < nb) {
+                if (v0) *reinterpret_cast<float2 *>(out + r0 * NOUT + 8 * nn + 2 * t) = make_float2(acc[nn][0], acc[nn][1]);
+                if (v1) *reinterpret_cast<float2 *>(out + r1 * NOUT + 8 * nn + 2 * t) = make_float2(acc[nn][2], acc[nn][3]);
+            }
+        }
+    }
+}
+
 }  // namespace deer
