@@ -34,7 +34,8 @@ struct Umma64 {
     static constexpr int OPERAND_BYTES = 16384;        // one 64 x 64 fp32 operand in canonical layout
     static constexpr int RES_WARPS = 4;
     static constexpr int MAX_SEQ_PER_WARP = 8;
-    static constexpr size_t SM_WORK = 4 * OPERAND_BYTES + sizeof(float) * (STAGES * RAW_FLOATS + 2 * N);
+    static constexpr size_t SM_WORK = 4 * OPERAND_BYTES + sizeof(float) * (STAGES * RAW_FLOATS + 2 * N);   // reverse; forward:
+    static_assert(6 * OPERAND_BYTES + sizeof(float) * 4 * N <= SM_WORK, "the forward layout fits the same allocation");
     static constexpr size_t SM_RES = sizeof(float) * RES_WARPS * (AGG + N);
     static constexpr size_t SMEM = (SM_WORK > SM_RES ? SM_WORK : SM_RES) + 1024;
     static constexpr unsigned TMEM_COLS = 64;
@@ -115,6 +116,23 @@ __device__ __forceinline__ float matvec_raw64(const float *Ms, const float *ycur
         }
     }
     return ((s0 + s1) + (s2 + s3)) + Ms[64 * RS + i];
+}
+
+// forward mat-vec straight from a staged B operand (hi part = the raw matrix in the swizzled layout):
+// component i of  sum_c J[i][c] y[c] + b[i]; eight consecutive rows read eight different 16-byte pieces
+__device__ __forceinline__ float matvec_swz64(const unsigned char *Bh, const float *bvec, const float *ycur, int i)
+{
+    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+    const unsigned char *row = Bh + i * 128;
+    const int x = i & 7;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        const float4 jv = *reinterpret_cast<const float4 *>(row + (k >> 3) * 8192 + (((k & 7) ^ x) << 4));
+        const float4 yv = *reinterpret_cast<const float4 *>(ycur + 4 * k);
+        s0 = fmaf(jv.x, yv.x, s0); s1 = fmaf(jv.y, yv.y, s1);
+        s2 = fmaf(jv.z, yv.z, s2); s3 = fmaf(jv.w, yv.w, s3);
+    }
+    return ((s0 + s1) + (s2 + s3)) + bvec[i];
 }
 
 template <bool REV>
@@ -246,8 +264,133 @@ __global__ void __launch_bounds__(Umma64::THREADS) scan_umma64_kernel(ScanArgs a
             cp_async_commit();
         };
 
+        if (kind == 0 && !REV) {
+            // ---------------------------------------------- A item, forward: software-pipelined.
+            // Shared memory: A hi/lo, two B buffers (hi, lo each), two vectors.  J[s] goes by cp.async
+            // straight into the hi part of a B buffer (row-major rows are already K-major); while the
+            // MMAs of position q run, the threads make the lo part of position q+1 and advance beta.
+            unsigned char *sB[2] = {sm + 2 * C::OPERAND_BYTES, sm + 4 * C::OPERAND_BYTES};      // hi at +0, lo at +16 KB
+            float *bvec = reinterpret_cast<float *>(sm + 6 * C::OPERAND_BYTES);                 // 2 x N
+            float *yb = bvec + 2 * N;                                                           // 2 x N
+            auto stage_fwd = [&](int q) {
+                if (q < cnt) {
+                    const float *src = Jseq + (size_t)(s0 + q) * NN;
+                    unsigned char *dst = sB[q & 1];
+#pragma unroll
+                    for (int u = 0; u < NN / 4 / C::THREADS; ++u) {
+                        const int j = tid + u * C::THREADS;
+                        cp_async16(dst + umma_off(j >> 4, 4 * (j & 15)), src + 4 * j);
+                    }
+                    if (tid < N / 4) cp_async16(bvec + (q & 1) * N + 4 * tid, bseq + (size_t)(s0 + q) * N + 4 * tid);
+                }
+                cp_async_commit();
+            };
+            // lo part of the staged matrix and one step of the beta chain (position q)
+            auto prepare = [&](int q) {
+                unsigned char *B = sB[q & 1];
+#pragma unroll
+                for (int u = 0; u < NN / 4 / C::THREADS; ++u) {
+                    const int off = (tid + u * C::THREADS) * 16;
+                    const float4 v = *reinterpret_cast<const float4 *>(B + off);
+                    *reinterpret_cast<float4 *>(B + C::OPERAND_BYTES + off) = make_float4(tf32_lo(v.x), tf32_lo(v.y), tf32_lo(v.z), tf32_lo(v.w));
+                }
+                if (tid < N) yb[((q + 1) & 1) * N + tid] = matvec_swz64(B, bvec + (q & 1) * N, yb + (q & 1) * N, tid);
+            };
+            for (int j = tid; j < NN / 4; j += C::THREADS) {
+                const int row = j >> 4, ch = j & 15;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if ((row >> 2) == ch) {
+                    if ((row & 3) == 0) v.x = 1.0f;
+                    if ((row & 3) == 1) v.y = 1.0f;
+                    if ((row & 3) == 2) v.z = 1.0f;
+                    if ((row & 3) == 3) v.w = 1.0f;
+                }
+                *reinterpret_cast<float4 *>(sAh + umma_off(row, 4 * ch)) = v;
+                *reinterpret_cast<float4 *>(sAl + umma_off(row, 4 * ch)) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (tid < N) yb[tid] = 0.0f;
+            stage_fwd(0);
+            stage_fwd(1);
+            cp_async_wait<1>();
+            __syncthreads();
+            prepare(0);
+            fence_proxy_async();
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
+            unsigned xv[64];
+#pragma unroll
+            for (int i = 0; i < 64; ++i) xv[i] = 0u;
+            bool ok = true;
+#pragma unroll 1
+            for (int q = 0; q < cnt; ++q) {
+                if (tid == 0) {
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const unsigned ah = smem_u32(sAh), al = smem_u32(sAl), bh = smem_u32(sB[q & 1]), bl = bh + C::OPERAND_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const unsigned off = (ks >> 2) * 8192 + (ks & 3) * 32;
+                        umma_tf32(tmem, umma_desc(al + off), umma_desc(bh + off), IDESC, ks ? 1u : 0u);
+                        umma_tf32(tmem, umma_desc(ah + off), umma_desc(bl + off), IDESC, 1u);
+                        umma_tf32(tmem, umma_desc(ah + off), umma_desc(bh + off), IDESC, 1u);
+                    }
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_mbar)) : "memory");
+                }
+                // meanwhile: the next position's operand (its matrix was requested one step ago)
+                cp_async_wait<0>();
+                __syncthreads();
+                if (q + 1 < cnt) prepare(q + 1);
+                {
+                    unsigned spins = 0;
+                    while (!mbar_try_wait(&s_mbar, mphase)) {
+                        if (++spins > SPIN_LIMIT) { atomicOr(&a.st->flags, FLAG_TIMEOUT); ok = false; break; }
+                    }
+                    mphase ^= 1u;
+                }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (__syncthreads_or(!ok)) { s_abort = 1; break; }
+                stage_fwd(q + 2);                  // buffer q & 1 is free: the MMAs of position q are done
+                {
+                    const unsigned taddr = tmem + ((unsigned)(32 * warp) << 16);
+                    unsigned lo32[32], hi32[32];
+                    tmem_ld32(taddr, lo32);
+                    tmem_ld32(taddr + 32, hi32);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) { xv[i] = lo32[i]; xv[32 + i] = hi32[i]; }
+                }
+                if (lane < 16 && q + 1 < cnt) {
+                    const int row = 16 * warp + lane;
+#pragma unroll
+                    for (int c4 = 0; c4 < 16; ++c4) {
+                        const float4 h = make_float4(__uint_as_float(xv[4 * c4]), __uint_as_float(xv[4 * c4 + 1]),
+                                                     __uint_as_float(xv[4 * c4 + 2]), __uint_as_float(xv[4 * c4 + 3]));
+                        const int off = umma_off(row, 4 * c4);
+                        *reinterpret_cast<float4 *>(sAh + off) = h;
+                        *reinterpret_cast<float4 *>(sAl + off) = make_float4(tf32_lo(h.x), tf32_lo(h.y), tf32_lo(h.z), tf32_lo(h.w));
+                    }
+                }
+                fence_proxy_async();
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncthreads();
+            }
+            cp_async_wait<0>();
+            __syncthreads();
+            if (s_abort) break;
+            float *dst = w.aggs + tile_index * AGG;
+            if (lane < 16) {
+                const int row = 16 * warp + lane;
+#pragma unroll
+                for (int cc = 0; cc < 64; ++cc) dst[cc * N + row] = __uint_as_float(xv[cc]);
+            }
+            if (tid < N) dst[NN + tid] = yb[(cnt & 1) * N + tid];
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) st_release_u32(w.flags + tile_index, 1u);
+            continue;
+        }
         if (kind == 0) {
-            // ---------------------------------------------- A item
+            // ---------------------------------------------- A item (reverse: the matrix is transposed while
+            // it is rewritten as the B operand, so it goes through a raw stage first)
             // X = I as the first A operand (hi = I, lo = 0); beta chain starts from zero
             for (int j = tid; j < NN / 4; j += C::THREADS) {
                 const int row = j >> 4, ch = j & 15;
