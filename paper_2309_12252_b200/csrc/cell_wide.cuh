@@ -79,7 +79,7 @@ __device__ __forceinline__ void gate_accumulate(float (&gr)[CellWide<N>::P], flo
 // weight blocks in registers and streams  k_r W_hr + a_z W_hz + k_n W_hn + z I  for the tile's
 // positions; a warp writes 512 contiguous bytes per store instruction.
 template <int N>
-__global__ void __launch_bounds__(256) cell_wide_kernel(CellArgs a)
+__global__ void __launch_bounds__(256, (N <= 32) ? 4 : 0) cell_wide_kernel(CellArgs a)
 {
     if (loop_ended(a.st)) return;
     using C = CellWide<N>;
