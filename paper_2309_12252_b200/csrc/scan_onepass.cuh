@@ -12,15 +12,15 @@
 //   * Chains.  A chain is S consecutive positions.  n <= 4: one thread per
 //     chain keeps the whole running aggregate (A, beta) in registers,
 //     (A, beta) <- (J_t A, J_t beta + b_t), and the chain aggregates of a warp
-//     and of the CTA are combined by warp-shuffle scans.  n = 8: four lanes per
-//     chain, each with two columns of A (beta redundantly); chain aggregates
-//     are combined per warp and per CTA through shared memory.
+//     and of the CTA are combined by warp-shuffle scans.  (n >= 8 share this
+//     file's protocol, resolvers and helpers; their workers are in
+//     scan_warp8.cuh, scan_warpn.cuh, scan_cta64.cuh.)
 //   * Staging and bank conflicts.  n <= 2: the tile is dense in shared memory,
 //     brought in by one bulk copy (cp.async.bulk + mbarrier), and S is chosen
-//     odd (n = 2) or S/4 odd (n = 1, four positions per 128-bit load).  n >= 4:
+//     odd (n = 2) or S/4 odd (n = 1, four positions per 128-bit load).  n = 4:
 //     every chain run is padded by 16 bytes so that the stride between the
-//     chains of a warp is odd in 16-byte units; n = 4 stages with per-thread
-//     16-byte cp.async copies, n = 8 with one bulk copy per chain run.
+//     chains of a warp is odd in 16-byte units, staged with per-thread
+//     16-byte cp.async copies.
 //   * Protocol.  Roles and tile ids are handed out by atomic counters to
 //     running CTAs only, and a tile's B item depends only on A items of lower
 //     ids, which their owners execute immediately after claiming: no
@@ -422,11 +422,11 @@ template <int N, bool REV>
 __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanArgs a, OnePassWs w)
 {
     using C = OnePass<N>;
-    constexpr int LPC = C::LPC, COLS = C::COLS, S = C::S, CHAINS = C::CHAINS, CPW = C::CPW;
-    constexpr int JRUN = C::JRUN, AGG = C::AGG, WARPS = C::WARPS, NN = N * N;
+    constexpr int S = C::S, CHAINS = C::CHAINS;
+    constexpr int AGG = C::AGG, WARPS = C::WARPS, NN = N * N;
     constexpr int Q = C::Q, PEND = C::PEND;
     constexpr bool CPASYNC = (N == 4);         // J staged by per-thread 16-byte cp.async
-    constexpr bool RUNBULK = (N == 8);         // J staged by one bulk copy per chain run
+    static_assert(N <= 4, "thread-per-chain kernel: n = 8 and above have their own kernels");
 
     extern __shared__ __align__(16) float smem_raw[];
     float *sJ = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
@@ -442,9 +442,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
 
     if (loop_ended(a.st)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int chain = tid / LPC, sub = tid % LPC;
-    const unsigned chain_mask = (LPC == 32) ? 0xffffffffu : (((1u << LPC) - 1u) << (lane & ~(LPC - 1)));
-    const int chain_lane0 = lane & ~(LPC - 1);
+    const int chain = tid;
     const int T = a.T;
 
     if (tid == 0) {
@@ -538,35 +536,6 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             for (int g = tid; g < Lt * N / 4; g += C::THREADS)
                 cp_async16(sB + tg.out_off(g * 4 / N, (g * 4) % N), bt_src + g * 4);
             cp_async_commit();
-        } else if constexpr (RUNBULK) {
-            if (warp == 0) {          // one bulk copy per chain run of J (16-byte aligned for n = 8)
-                fence_proxy_async();
-                unsigned bytes = 0;
-#pragma unroll 1
-                for (int r = lane; r < CHAINS; r += 32) {
-                    int cnt = tg.run_cnt(r);
-                    if (REV && s0 + r * S == 0) cnt -= 1;
-                    if (cnt > 0) bytes += (unsigned)cnt * NN * 4u;
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) bytes += __shfl_xor_sync(0xffffffffu, bytes, o);
-                if (lane == 0) mbar_arrive_expect_tx(bar, bytes);
-                __syncwarp();
-#pragma unroll 1
-                for (int r = lane; r < CHAINS; r += 32) {
-                    const int cnt = tg.run_cnt(r);
-                    if (cnt <= 0) continue;
-                    const int first = REV ? (Lt - (r * S + cnt)) : r * S;     // ascending index of the run's first J
-                    int jc = cnt;
-                    if (REV && s0 + r * S == 0) jc -= 1;
-                    if (jc > 0) bulk_g2s(sJ + r * JRUN, Jt_src + (size_t)first * NN, (unsigned)jc * NN * 4u, bar);
-                }
-            }
-            for (int g4 = tid; g4 < Lt * N / 4; g4 += C::THREADS) {
-                const int g = 4 * g4;
-                const float4 v = __ldg(reinterpret_cast<const float4 *>(bt_src) + g4);
-                *reinterpret_cast<float4 *>(sB + tg.out_off(g / N, g % N)) = v;
-            }
         } else {
             const unsigned jb = (unsigned)jcnt_tile * NN * 4u, bb = (unsigned)Lt * N * 4u;
             float *jd = sJ + tg.low_slot() * NN, *bd = sB + tg.low_slot() * N;
@@ -612,7 +581,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         if (s_abort) break;
 
         const int cnt = tg.run_cnt(chain);
-        if constexpr (LPC == 1) {
+        {
             // ============================================ n <= 4: one thread per chain
             // one step of the chain: M = J (forward) or J^T (reverse; identity at scan position 0)
             auto load_step = [&](int q, float (&M)[N][N], float (&bq)[N]) {
@@ -750,164 +719,6 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                 }
             }
             __syncthreads();
-        } else {
-        // ================================================ n = 8: four lanes per chain
-        const float *cJ = sJ;
-        float *cB = sB;
-        if (kind == 0) {
-            float A[N][COLS], be[N];
-#pragma unroll
-            for (int i = 0; i < N; ++i) {
-                be[i] = 0.0f;
-#pragma unroll
-                for (int cc = 0; cc < COLS; ++cc) A[i][cc] = (i == sub * COLS + cc) ? 1.0f : 0.0f;
-            }
-#pragma unroll
-            for (int q = 0; q < S; ++q) {
-                if (q >= cnt) break;
-                const bool ident = REV && (s0 + chain * S + q == 0);
-                const float *Je = cJ + tg.j_off(chain, q, cnt);
-                const float *bv = cB + tg.b_off(chain, q, cnt);
-                float bq[N];
-#pragma unroll
-                for (int v = 0; v < N / 4; ++v) {
-                    const float4 f = reinterpret_cast<const float4 *>(bv)[v];
-                    bq[4 * v] = f.x; bq[4 * v + 1] = f.y; bq[4 * v + 2] = f.z; bq[4 * v + 3] = f.w;
-                }
-                if (q == 0) {
-                    if (!ident) {
-#pragma unroll
-                        for (int i = 0; i < N; ++i)
-#pragma unroll
-                            for (int cc = 0; cc < COLS; ++cc) {
-                                const int j = sub * COLS + cc;
-                                A[i][cc] = REV ? Je[j * N + i] : Je[i * N + j];
-                            }
-                    }
-#pragma unroll
-                    for (int i = 0; i < N; ++i) be[i] = bq[i];
-                    continue;
-                }
-                float Jr[NN];
-#pragma unroll
-                for (int v = 0; v < NN / 4; ++v) {
-                    const float4 f = reinterpret_cast<const float4 *>(Je)[v];
-                    Jr[4 * v] = f.x; Jr[4 * v + 1] = f.y; Jr[4 * v + 2] = f.z; Jr[4 * v + 3] = f.w;
-                }
-                float An[N][COLS], bn[N];
-#pragma unroll
-                for (int i = 0; i < N; ++i) {
-                    bn[i] = bq[i];
-#pragma unroll
-                    for (int cc = 0; cc < COLS; ++cc) An[i][cc] = 0.0f;
-#pragma unroll
-                    for (int k = 0; k < N; ++k) {
-                        const float m = REV ? Jr[k * N + i] : Jr[i * N + k];
-                        bn[i] = fmaf(m, be[k], bn[i]);
-#pragma unroll
-                        for (int cc = 0; cc < COLS; ++cc) An[i][cc] = fmaf(m, A[k][cc], An[i][cc]);
-                    }
-                }
-#pragma unroll
-                for (int i = 0; i < N; ++i) {
-                    be[i] = bn[i];
-#pragma unroll
-                    for (int cc = 0; cc < COLS; ++cc) A[i][cc] = An[i][cc];
-                }
-            }
-            {
-                float *ag = agg + chain * AGG;
-#pragma unroll
-                for (int i = 0; i < N; ++i) {
-#pragma unroll
-                    for (int cc = 0; cc < COLS; ++cc) ag[i * N + sub * COLS + cc] = A[i][cc];
-                    if (sub == 0) ag[NN + i] = be[i];
-                }
-            }
-            __syncwarp();
-            // warp aggregate, then tile aggregate (warp 0), then publish
-            {
-                const float *first = agg + (warp * CPW) * AGG;
-                float *t0s = tmp + warp * 2 * AGG, *t1s = t0s + AGG;
-                const float *cur = first;
-                for (int k = 1; k < CPW; ++k) {
-                    float *dst = (k == CPW - 1) ? (wagg + warp * AGG) : ((k & 1) ? t0s : t1s);
-                    combine_smem<N>(dst, agg + (warp * CPW + k) * AGG, cur, lane);
-                    cur = dst;
-                }
-            }
-            __syncthreads();
-            if (warp == 0) {
-                float *t0s = tmp, *t1s = tmp + AGG;
-                const float *cur = wagg;
-                for (int k = 1; k < WARPS; ++k) {
-                    float *dst = (k == WARPS - 1) ? tagg : ((k & 1) ? t0s : t1s);
-                    combine_smem<N>(dst, wagg + k * AGG, cur, lane);
-                    cur = dst;
-                }
-                float *g = w.aggs + tile_index * AGG;
-                for (int o = lane; o < AGG; o += 32) g[o] = tagg[o];
-                __threadfence();
-                __syncwarp();
-                if (lane == 0) st_release_u32(w.flags + tile_index, 1u);
-            }
-            continue;
-        }
-
-        // B item: states entering each warp, each chain
-        if (warp == 0) {
-            if (lane < N) wstart[lane] = ystart[lane];
-            __syncwarp();
-            for (int k = 0; k + 1 < WARPS; ++k)
-                matvec_smem<N>(wstart + (k + 1) * N, wagg + k * AGG, wstart + k * N, lane);
-        }
-        __syncthreads();
-        {
-            float *cs = cstart + (warp * CPW) * N;
-            if (lane < N) cs[lane] = wstart[warp * N + lane];
-            __syncwarp();
-            for (int k = 0; k + 1 < CPW; ++k)
-                matvec_smem<N>(cs + (k + 1) * N, agg + (warp * CPW + k) * AGG, cs + k * N, lane);
-        }
-        // apply: replay the chain, y overwrites b
-        {
-            float y[N];
-#pragma unroll
-            for (int k = 0; k < N; ++k) y[k] = cstart[chain * N + k];
-#pragma unroll
-            for (int q = 0; q < S; ++q) {
-                if (q >= cnt) break;
-                const bool ident = REV && (s0 + chain * S + q == 0);
-                const float *Je = cJ + tg.j_off(chain, q, cnt);
-                float *bv = cB + tg.b_off(chain, q, cnt);
-                float v[COLS];
-#pragma unroll
-                for (int cc = 0; cc < COLS; ++cc) {
-                    const int i = sub * COLS + cc;
-                    float acc = bv[i];
-                    if (ident) {
-#pragma unroll
-                        for (int k = 0; k < N; ++k) if (k == i) acc += y[k];
-                    } else if (!REV) {
-#pragma unroll
-                        for (int v4 = 0; v4 < N / 4; ++v4) {
-                            const float4 f = reinterpret_cast<const float4 *>(Je + i * N)[v4];
-                            acc = fmaf(f.x, y[4 * v4], acc); acc = fmaf(f.y, y[4 * v4 + 1], acc);
-                            acc = fmaf(f.z, y[4 * v4 + 2], acc); acc = fmaf(f.w, y[4 * v4 + 3], acc);
-                        }
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < N; ++k) acc = fmaf(Je[k * N + i], y[k], acc);
-                    }
-                    v[cc] = acc;
-                }
-#pragma unroll
-                for (int cc = 0; cc < COLS; ++cc) bv[sub * COLS + cc] = v[cc];
-#pragma unroll
-                for (int k = 0; k < N; ++k) y[k] = __shfl_sync(chain_mask, v[k % COLS], chain_lane0 + k / COLS);
-            }
-        }
-        __syncthreads();
         }
 
         // ------------------------------------------------ stream y out (+ max |y - yold|)
