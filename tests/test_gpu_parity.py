@@ -95,7 +95,10 @@ def run_eval(bd, w, **kw):
 
 @pytest.mark.parametrize("n,m,B,T", [(1, 1, 2, 50), (2, 3, 3, 333), (3, 2, 2, 100), (4, 2, 1, 1000),
                                      (8, 4, 4, 2500), (16, 16, 2, 700), (32, 32, 2, 400),
-                                     (64, 6, 2, 150), (5, 7, 3, 129)])
+                                     (64, 6, 2, 150), (5, 7, 3, 129),
+                                     # input-projection shapes: tensor-core path with ragged position tiles
+                                     # (m % 8 == 0, m >= 16), tiled path otherwise
+                                     (8, 16, 3, 77), (16, 24, 1, 131), (32, 8, 2, 200), (64, 64, 1, 300)])
 @pytest.mark.parametrize("flags", [0, 2, 4])
 def test_eval_matches_sequential(bd, n, m, B, T, flags):
     p = synth.gru_params(n, m, seed=7, tag="e/gru")
@@ -232,7 +235,8 @@ def grad_case(bd, n, m, B, T, dense, seed=5):
 
 
 @pytest.mark.parametrize("n,m,B,T", [(1, 1, 2, 40), (2, 2, 3, 300), (4, 2, 2, 1000), (8, 4, 3, 1500),
-                                     (16, 8, 2, 600), (32, 32, 2, 500), (64, 6, 2, 200), (3, 5, 2, 77)])
+                                     (16, 8, 2, 600), (32, 32, 2, 500), (64, 6, 2, 200), (3, 5, 2, 77),
+                                     (16, 40, 1, 131), (64, 64, 1, 260)])
 @pytest.mark.parametrize("dense", [True, False])
 def test_vjp_matches_bptt(bd, n, m, B, T, dense):
     grad_case(bd, n, m, B, T, dense)
