@@ -41,8 +41,15 @@ struct Warp8 {
     // T = 3e3 ... 1e6).
     static int chain_len(int B, int T, int resident_ctas)
     {
+        auto tiles = [&](int sw) { return (long long)B * ((T + WARPS * sw - 1) / (WARPS * sw)); };
         int sw = SW_MAX;
-        while (sw > SW_MIN && (long long)B * ((T + WARPS * sw - 1) / (WARPS * sw)) < 3LL * resident_ctas / 2) sw >>= 1;
+        while (sw > SW_MIN && tiles(sw) < 3LL * resident_ctas / 2) sw >>= 1;
+        // a nearly empty second wave costs a whole extra item per CTA: if chains at most twice as
+        // long bring every tile into the first wave (a few CTAs are resolvers), take them
+        const long long workers = resident_ctas - 8;
+        if (tiles(sw) > workers)
+            for (int s2 = sw + GRP; s2 <= 2 * sw && s2 <= SW_MAX; s2 += GRP)
+                if (tiles(s2) <= workers) { sw = s2; break; }
         return sw;
     }
 };
