@@ -31,8 +31,8 @@ __device__ __forceinline__ void stage_h_prev(float *sH, const float *y, const fl
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (p < np) {
             const size_t e = e0 + p;
-            const size_t seq = e / T;
-            const float *hp = (e - seq * T == 0) ? y0 + seq * N : y + (e - 1) * N;
+            size_t seq;
+            const float *hp = seq_start(e, T, seq) ? y0 + seq * N : y + (e - 1) * N;
             v = *reinterpret_cast<const float4 *>(hp + 4 * k4);
         }
         *reinterpret_cast<float4 *>(sH + p * C::HS + 4 * k4) = v;

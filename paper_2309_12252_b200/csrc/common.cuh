@@ -142,6 +142,18 @@ __device__ __forceinline__ void scan_epilogue(StatusBlock *st)
     if (st->ctl_mode) newton_decide(st, st->tol, st->max_iter, st->trace);
 }
 
+// Is flat position e = seq * T + t the first of its sequence?  (32-bit division whenever e fits.)
+__device__ __forceinline__ bool seq_start(size_t e, int T, size_t &seq)
+{
+    if (e <= 0xffffffffull) {
+        const unsigned q = (unsigned)e / (unsigned)T;
+        seq = q;
+        return (unsigned)e - q * (unsigned)T == 0u;
+    }
+    seq = e / (size_t)T;
+    return e - seq * (size_t)T == 0;
+}
+
 __device__ __forceinline__ float sigmoidf_acc(float a) { return 1.0f / (1.0f + expf(-a)); }
 
 __device__ __forceinline__ unsigned absdiff_bits(float a, float b) {

@@ -104,9 +104,16 @@ __global__ void __launch_bounds__(256) cell_small_kernel(CellArgs a)
         cr = a.b_i[i]; cz = a.b_i[N + i]; cn = a.b_i[2 * N + i];
     }
     const size_t total = (size_t)a.B * a.T;
-    for (size_t e = (size_t)blockIdx.x * EPB + le; e < total; e += (size_t)gridDim.x * EPB) {
-        const size_t seq = e / a.T;
-        const bool first = (e - seq * a.T) == 0;
+    // (seq, t) of the thread's position is carried along the grid-stride loop instead of divided out
+    const size_t stride = (size_t)gridDim.x * EPB;
+    const size_t stride_seq = stride / a.T;
+    const unsigned stride_t = (unsigned)(stride - stride_seq * a.T);
+    size_t e = (size_t)blockIdx.x * EPB + le;
+    size_t seq = e / a.T;
+    unsigned t = (unsigned)(e - seq * a.T);
+    for (; e < total; e += stride, seq += stride_seq, t += stride_t) {
+        if (t >= (unsigned)a.T) { t -= (unsigned)a.T; ++seq; }
+        const bool first = t == 0u;
         const float *hp = first ? a.y0 + seq * N : a.y + (e - 1) * N;
         float h[N];
         if constexpr (N >= 4) {

@@ -90,8 +90,8 @@ __global__ void __launch_bounds__(384) wgrad_mma_kernel(WgradArgs a)
     const int row = 16 * warp + g;
     auto vrow = [&](size_t e) -> const float * {
         if (!a.shifted) return a.V + e * K;
-        const size_t seq = e / a.T;
-        return (e - seq * a.T == 0) ? a.y0 + seq * K : a.V + (e - 1) * K;
+        size_t seq;
+        return seq_start(e, a.T, seq) ? a.y0 + seq * K : a.V + (e - 1) * K;
     };
 #pragma unroll 1
     for (size_t e = e0; e < e1; e += 8) {
