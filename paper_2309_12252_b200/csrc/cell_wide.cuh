@@ -81,6 +81,7 @@ __device__ __forceinline__ void gate_accumulate(float (&gr)[CellWide<N>::P], flo
 template <int N>
 __global__ void __launch_bounds__(256, (N <= 32) ? 4 : 0) cell_wide_kernel(CellArgs a)
 {
+    pdl_prologue();
     if (loop_ended(a.st)) return;
     using C = CellWide<N>;
     extern __shared__ __align__(16) float sm[];

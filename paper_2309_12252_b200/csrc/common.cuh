@@ -39,6 +39,29 @@ struct KernelScope {
         DEER_CHECK_LAUNCH(kname);                                  \
     } while (0)
 
+// Launch with the programmatic-stream-serialization attribute (see pdl_prologue):
+//   DEER_KERNEL_PDL("name", stream, kernel, grid, block, smem, args...)
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
+#define DEER_KERNEL_PDL(kname, stream, kern, grid, block, smem, ...)                        \
+    do {                                                                                    \
+        {                                                                                   \
+            ::deer::KernelScope ks_(kname, stream);                                         \
+            ::deer::launch_pdl(kern, grid, block, smem, stream, __VA_ARGS__);               \
+        }                                                                                   \
+        DEER_CHECK_LAUNCH(kname);                                                           \
+    } while (0)
+
 #define DEER_CHECK_CUDA(call, where)                               \
     do {                                                           \
         cudaError_t e_ = (call);                                   \
@@ -103,6 +126,16 @@ struct CellArgs {
     int B, T, n;
     const StatusBlock *st;   // nullptr, or: skip all work once st->done is set (Newton loop ended)
 };
+
+// Programmatic dependent launch: a kernel of the Newton loop lets the next launch in the stream be set
+// up and its CTAs become resident as soon as all of this kernel's CTAs are running, then waits for the
+// previous kernel to have completed (with its memory visible) before it reads anything that kernel
+// produced.  Without the launch attribute both instructions do nothing.
+__device__ __forceinline__ void pdl_prologue()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 
 // Device-side loop control lets the host enqueue Newton bodies ahead of knowing whether they
 // are needed: every kernel of a body returns at once when the loop has already ended.

@@ -81,6 +81,7 @@ __global__ void cell_kernel(CellArgs a)
 template <int N, int M>
 __global__ void __launch_bounds__(256) cell_small_kernel(CellArgs a)
 {
+    pdl_prologue();
     if (loop_ended(a.st)) return;
     constexpr int EPB = 256 / N;                       // positions per block per step
     const int i = threadIdx.x % N, le = threadIdx.x / N;

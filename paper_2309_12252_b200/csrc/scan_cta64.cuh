@@ -210,6 +210,7 @@ __global__ void __launch_bounds__(Cta64::THREADS) scan_cta64_kernel(ScanArgs a, 
 {
     using C = Cta64;
     constexpr int N = C::N, NN = C::NN, AGG = C::AGG, Q = C::Q, S = C::STAGES, RS = RingRow<64, REV>::RS;
+    pdl_prologue();
     if (loop_ended(a.st)) return;
 
     extern __shared__ __align__(16) float smem_raw[];

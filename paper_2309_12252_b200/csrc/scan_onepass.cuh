@@ -440,6 +440,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     uint64_t *bar = (uint64_t *)(((uintptr_t)(ystart + N) + 15) & ~(uintptr_t)15);
     __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role;
 
+    pdl_prologue();
     if (loop_ended(a.st)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chain = tid;

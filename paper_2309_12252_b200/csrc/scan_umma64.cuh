@@ -140,6 +140,7 @@ __global__ void __launch_bounds__(Umma64::THREADS) scan_umma64_kernel(ScanArgs a
 {
     using C = Umma64;
     constexpr int N = C::N, NN = C::NN, AGG = C::AGG, Q = C::Q, S = C::STAGES, RS = C::RS;
+    pdl_prologue();
     if (loop_ended(a.st)) return;
 
     extern __shared__ __align__(16) unsigned char smem_bytes[];

@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
 {
     using C = Warp8;
     constexpr int N = C::N, NN = C::NN, AGG = C::AGG, WARPS = C::WARPS, GRP = C::GRP, Q = C::Q;
+    pdl_prologue();
     if (loop_ended(a.st)) return;
     const int SW = w.sw, L = WARPS * SW;
 

@@ -325,6 +325,7 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS, WarpN<N>::CTAS_PER_SM) scan
 {
     using C = WarpN<N>;
     constexpr int NN = C::NN, AGG = C::AGG, NT = C::NT, MT = C::MT, WARPS = C::WARPS, Q = C::Q;
+    pdl_prologue();
     if (loop_ended(a.st)) return;
 
     extern __shared__ __align__(16) float smem_raw[];
