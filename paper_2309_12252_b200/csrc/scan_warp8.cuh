@@ -91,6 +91,94 @@ __device__ __forceinline__ void chain_step(float (&acc)[4], float j0, float j1, 
     acc[0] = d[0]; acc[1] = d[1]; acc[2] = d[2]; acc[3] = d[3];
 }
 
+// Resolver for n = 8 (see resolver_loop of scan_onepass.cuh).  The walk Y <- A Y + beta is the critical
+// path of a latency-bound scan, so a step is kept short: lane (r, p) = (lane / 4, lane % 4) holds
+// Y[2p], Y[2p+1]; one step is two FMAs on the lane's 8-byte piece of row r, two xor-shuffles, the add
+// of beta[r] and two shuffles that hand the new pair to every lane (about a dozen instructions).
+__device__ void resolver_loop8(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
+{
+    constexpr int N = 8, NN = 64, AGG = 72, MAXS = OnePass<8>::MAX_SEQ_PER_WARP;
+    float *stage = stage_all + (threadIdx.x >> 5) * 32 * AGG;
+    const int r = lane >> 2, p = lane & 3;
+    int nseq = 0;
+    int pos[MAXS];
+    float ya[MAXS], yb[MAXS];
+    unsigned fnext[MAXS];
+#pragma unroll
+    for (int k = 0; k < MAXS; ++k) {
+        pos[k] = 0; ya[k] = 0.0f; yb[k] = 0.0f; fnext[k] = 0u;
+        const int s = rw + k * nrw;
+        if (s < a.B) {
+            nseq = k + 1;
+            if (a.y0) { ya[k] = a.y0[(size_t)s * N + 2 * p]; yb[k] = a.y0[(size_t)s * N + 2 * p + 1]; }
+            if (lane < w.nch) fnext[k] = ld_acquire_u32(w.flags + (size_t)s * w.nch + lane);
+        }
+    }
+    int remaining = nseq;
+    unsigned spins = 0;
+    while (remaining > 0) {
+        bool progressed = false;
+#pragma unroll
+        for (int k = 0; k < MAXS; ++k) {
+            if (k >= nseq) break;
+            const int c0 = pos[k];
+            if (c0 >= w.nch) continue;
+            const int s = rw + k * nrw;
+            const unsigned *flags = w.flags + (size_t)s * w.nch;
+            const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
+            const int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
+            {
+                const int j = c0 + cnt + lane;
+                fnext[k] = (j < w.nch) ? ld_acquire_u32(flags + j) : 0u;
+            }
+            if (cnt == 0) continue;
+            progressed = true;
+            const float *src = w.aggs + ((size_t)s * w.nch + c0) * AGG;
+            {
+                const int total = cnt * AGG;
+                for (int i0 = 0; i0 < total; i0 += 32 * 8) {
+                    float v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        v[u] = (i < total) ? __ldcg(src + i) : 0.0f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        if (i < total) stage[i] = v[u];
+                    }
+                }
+            }
+            __syncwarp();
+            unsigned long long *out = w.starts + ((size_t)s * w.nch + c0) * N;
+            float y0v = ya[k], y1v = yb[k];
+#pragma unroll 2
+            for (int q = 0; q < cnt; ++q) {
+                if (r == 0) {
+                    st_relaxed_u64(out + q * N + 2 * p, LL_FLAG | (unsigned long long)__float_as_uint(y0v));
+                    st_relaxed_u64(out + q * N + 2 * p + 1, LL_FLAG | (unsigned long long)__float_as_uint(y1v));
+                }
+                const float *ag = stage + q * AGG;
+                const float2 a2 = *reinterpret_cast<const float2 *>(ag + r * N + 2 * p);
+                float part = fmaf(a2.x, y0v, a2.y * y1v);
+                part += __shfl_xor_sync(0xffffffffu, part, 1);
+                part += __shfl_xor_sync(0xffffffffu, part, 2);
+                const float yn = part + ag[NN + r];
+                y0v = __shfl_sync(0xffffffffu, yn, 8 * p);
+                y1v = __shfl_sync(0xffffffffu, yn, 8 * p + 4);
+            }
+            ya[k] = y0v; yb[k] = y1v;
+            __syncwarp();
+            if (lane < cnt) w.flags[(size_t)s * w.nch + c0 + lane] = 0u;   // consumed: cleared for the next launch
+            pos[k] = c0 + cnt;
+            if (pos[k] >= w.nch) --remaining;
+        }
+        if (progressed) spins = 0;
+        else if (!keep_spinning(a.st, spins)) return;
+    }
+}
+
 template <bool REV>
 __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs a, OnePassWs w)
 {
@@ -118,7 +206,7 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
     __syncthreads();
     if (s_role < w.resolvers) {
         if (warp < C::RES_WARPS)
-            resolver_loop<8>(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+            resolver_loop8(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
         __syncthreads();
         if (tid == 0) scan_epilogue(a.st);
         return;
