@@ -84,11 +84,14 @@ __device__ __forceinline__ void chain_step(float (&acc)[4], float j0, float j1, 
     split_tf32(acc[3], ah[3], al[3]);      // a3 <- c3
     split_tf32(j0, bh[0], bl[0]);
     split_tf32(j1, bh[1], bl[1]);
-    float d[4] = {0.0f, 0.0f, bx, by};
-    mma_tf32(d, al, bh, d);
-    mma_tf32(d, ah, bl, d);
-    mma_tf32(d, ah, bh, d);
-    acc[0] = d[0]; acc[1] = d[1]; acc[2] = d[2]; acc[3] = d[3];
+    // three independent MMAs (the next step waits for one MMA latency, not three), summed afterwards
+    const float z[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    float d0[4] = {0.0f, 0.0f, bx, by}, d1[4], d2[4];
+    mma_tf32(d1, al, bh, z);
+    mma_tf32(d2, ah, bl, z);
+    mma_tf32(d0, ah, bh, d0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] = d0[i] + (d1[i] + d2[i]);
 }
 
 // Resolver for n = 8 (see resolver_loop of scan_onepass.cuh).  The walk Y <- A Y + beta is the critical
