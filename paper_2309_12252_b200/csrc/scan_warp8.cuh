@@ -54,6 +54,8 @@ struct Warp8 {
     }
 };
 
+__device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+
 // d = a * b + c   (m16n8k8, A row-major 16x8, B 8x8, TF32 inputs, fp32 accumulate)
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const unsigned (&a)[4], const unsigned (&b)[2], const float (&c)[4])
 {
@@ -301,6 +303,14 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
                 const float2 *jq = jp2 + q0 * 32;
                 const float *jr = jpr - q0 * NN;
                 const float2 *bq = REV ? bp2 - q0 * 4 : bp2 + q0 * 4;
+                if (q0 + 2 * GRP <= cnt) {              // next group towards L1 while this one is used
+#pragma unroll
+                    for (int u = 0; u < GRP; ++u) {
+                        if (!REV) prefetch_l1(jq + (GRP + u) * 32);
+                        else { prefetch_l1(jr - (GRP + u) * NN); prefetch_l1(jr - (GRP + u) * NN + N); }
+                    }
+                    if (g == 0) prefetch_l1(REV ? bq - (2 * GRP - 1) * 4 : bq + GRP * 4);
+                }
 #pragma unroll
                 for (int u = 0; u < GRP; ++u) {
                     if (!REV) { const float2 f = __ldg(jq + u * 32); j0[u] = f.x; j1[u] = f.y; }
@@ -408,6 +418,14 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
                 const float2 *jq = jp2 + q0 * 32;
                 const float *jr = jpr - q0 * NN;
                 const int off0 = REV ? -q0 * N : q0 * N;
+                if (q0 + 2 * GRP <= cnt) {
+#pragma unroll
+                    for (int u = 0; u < GRP; ++u) {
+                        if (!REV) prefetch_l1(jq + (GRP + u) * 32);
+                        else { prefetch_l1(jr - (GRP + u) * NN); prefetch_l1(jr - (GRP + u) * NN + N); }
+                    }
+                    if (t == 0) prefetch_l1(bpg + (REV ? off0 - (2 * GRP - 1) * N : off0 + GRP * N));
+                }
                 const int offt = off0 + (REV ? -t * N : t * N);               // this lane's first position of the group
                 float yo[GRP / 4];
 #pragma unroll
