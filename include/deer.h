@@ -84,7 +84,9 @@ enum {
 };
 
 /* Bytes of workspace needed by `op` at the given sizes (0 if the sizes are
- * invalid).  m is ignored for DEER_OP_SCAN. */
+ * invalid).  m is ignored for DEER_OP_SCAN.  The tile length of the scan, and
+ * with it the size, depends on the SM count of the current device: query with
+ * the device current on which the call will run. */
 size_t deer_workspace_bytes(int op, int B, int T, int n, int m, int flags);
 
 /* Solve the linear recurrence (the operator L_G^{-1} of Eq. 10 with J = -G)
