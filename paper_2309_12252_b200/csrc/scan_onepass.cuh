@@ -53,7 +53,7 @@ template <int N> struct OnePass {
     static constexpr int BRUN = S * N + ((N == 8) ? 4 : 0);          // floats per chain run of b / y
     static constexpr int JBUF = CHAINS * JRUN, BBUF = CHAINS * BRUN;
     static constexpr int AGG = N * N + N;              // floats of one aggregate (A row-major, then beta)
-    static constexpr int Q = (N == 1) ? 3 : 2;         // pending tiles (A scheduled, B not yet) per CTA
+    static constexpr int Q = (N == 1) ? 3 : (N == 4) ? 1 : 2;   // pending tiles (A scheduled, B not yet) per CTA
     // kept per pending tile: n = 8: chain aggregates + warp aggregates;
     //                        n <= 4: exclusive chain prefixes (within the warp) + exclusive warp prefixes
     static constexpr int PEND = (CHAINS + WARPS) * AGG;
