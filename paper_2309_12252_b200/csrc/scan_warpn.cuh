@@ -28,7 +28,7 @@ template <int N> struct WarpN {
     static constexpr int WARPS = (N == 16) ? 8 : 4;    // chains per tile
     static constexpr int THREADS = WARPS * 32;
     static constexpr int SW_MIN = 16, SW_MAX = 64;     // positions per warp chain (chosen per problem size)
-    static constexpr int CTAS_PER_SM = (N == 16) ? 2 : 3;
+    static constexpr int CTAS_PER_SM = 3;
     // longest chain that still leaves about 1.5 tiles per resident CTA (see Warp8::chain_len)
     static int chain_len(int B, int T, int resident_ctas)
     {
