@@ -528,12 +528,17 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         const float *bt_src = a.b + ((size_t)seq * T + p_lo) * N;
 
         // ------------------------------------------------ stage the tile
+        // (with one pending tile per CTA the B item follows its own A item directly: the tile is
+        // still in shared memory, untouched, and is not staged again)
+        constexpr bool HOLD = (Q == 1);
         if constexpr (CPASYNC) {
             constexpr int PPE = NN / 4;                       // 16-byte pieces per J_t
+            if (!(HOLD && kind == 1))
             for (int g = tid; g < jcnt_tile * PPE; g += C::THREADS) {
                 const int u = g / PPE, v = g - u * PPE;
                 cp_async16(sJ + tg.jmat_off(u) + v * 4, Jt_src + (size_t)u * NN + v * 4);
             }
+            if (!(HOLD && kind == 1))
             for (int g = tid; g < Lt * N / 4; g += C::THREADS)
                 cp_async16(sB + tg.out_off(g * 4 / N, (g * 4) % N), bt_src + g * 4);
             cp_async_commit();
