@@ -542,7 +542,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             for (int g = tid; g < Lt * N / 4; g += C::THREADS)
                 cp_async16(sB + tg.out_off(g * 4 / N, (g * 4) % N), bt_src + g * 4);
             cp_async_commit();
-        } else {
+        } else if (!(HOLD && kind == 1)) {
             const unsigned jb = (unsigned)jcnt_tile * NN * 4u, bb = (unsigned)Lt * N * 4u;
             float *jd = sJ + tg.low_slot() * NN, *bd = sB + tg.low_slot() * N;
             const bool jbulk = jb && ((uintptr_t)Jt_src & 15) == 0 && (jb & 15) == 0 && ((uintptr_t)jd & 15) == 0;
@@ -576,7 +576,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         }
         if constexpr (CPASYNC) {
             cp_async_wait_0();
-        } else {
+        } else if (!(HOLD && kind == 1)) {
             unsigned spins = 0;
             while (!mbar_try_wait(bar, phase)) {
                 if (++spins > (SPIN_LIMIT >> 2)) { atomicOr(&a.st->flags, FLAG_TIMEOUT); s_abort = 1; break; }
