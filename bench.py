@@ -48,6 +48,7 @@ def peaks():
 
 # DRAM bytes (read + write) per position of the stand-alone scan, from the ncu captures summarised in
 # profiles/scan_kernels_standalone_B16.md (inputs larger than L2; traffic grows in proportion to positions).
+NCU_STEP_SCAN_TRAFFIC = 51.43e6      # config-2 step, scan_warp8_kernel: dram read + write per launch
 NCU_SCAN_TRAFFIC_PER_POSITION = {1: 13.9, 2: 35.8, 4: 95.6, 8: 606.6, 16: 2213.0, 32: 8622.0, 64: 34116.0}
 
 
@@ -463,7 +464,10 @@ def main():
     if scan_ms > 0:
         ach = scan_bytes_per_position(n) * B * T / (scan_ms / scans * 1e-3) / 1e9
         roofline = dict(bound="hbm", kernel="+".join(scan_names), achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
-                        frac=ach / pk["hbm_gbs"], peak_source=pk["source"], traffic=None,
+                        frac=ach / pk["hbm_gbs"], peak_source=pk["source"], traffic=NCU_STEP_SCAN_TRAFFIC,
+                        traffic_note="DRAM bytes per scan launch of this workload under ncu (caches flushed before each "
+                                     "kernel): one read of J, b, y_old; the second visit of every tile is served by L2 "
+                                     "(profiles/bench_step_config2_launch_list.md)",
                         note="scan inside the step; this workload (46 MB of J,b per body) is L2-resident, "
                              "so this is an effective rate; see roofline_scan_hbm for the HBM-sized scan")
 
