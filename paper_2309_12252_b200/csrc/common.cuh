@@ -39,25 +39,29 @@ struct KernelScope {
         DEER_CHECK_LAUNCH(kname);                                  \
     } while (0)
 
-// Launch with the programmatic-stream-serialization attribute (see pdl_prologue):
-//   DEER_KERNEL_PDL("name", stream, kernel, grid, block, smem, args...)
+// Launch with the programmatic-stream-serialization attribute (see pdl_prologue) when `overlap`:
+//   DEER_KERNEL_PDL("name", overlap, stream, kernel, grid, block, smem, args...)
+// Measured: the overlap pays for the small-n kernels (config 2: -4 %, config 1: -12 %) and costs for
+// n >= 16 at small T (CTAs of two kernels with different shared-memory footprints resident together:
+// n = 64, T = 1000: 2.1 ms with, 1.5 ms without), so only the n <= 8 kernels ask for it.
 template <typename... KArgs, typename... Args>
-static inline cudaError_t launch_pdl(void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args... args)
+static inline cudaError_t launch_pdl(bool overlap, void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st,
+                                     Args... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = overlap ? 1 : 0;
     cfg.attrs = attr; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
-#define DEER_KERNEL_PDL(kname, stream, kern, grid, block, smem, ...)                        \
+#define DEER_KERNEL_PDL(kname, overlap, stream, kern, grid, block, smem, ...)               \
     do {                                                                                    \
         {                                                                                   \
             ::deer::KernelScope ks_(kname, stream);                                         \
-            ::deer::launch_pdl(kern, grid, block, smem, stream, __VA_ARGS__);               \
+            ::deer::launch_pdl(overlap, kern, grid, block, smem, stream, __VA_ARGS__);      \
         }                                                                                   \
         DEER_CHECK_LAUNCH(kname);                                                           \
     } while (0)

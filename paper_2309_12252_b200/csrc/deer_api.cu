@@ -190,7 +190,7 @@ static int launch_single_pass(Kern kern, int (&occ_dev)[MAX_DEVICES], const Pass
     w.total_ids = (unsigned)((size_t)w.nwin * a.B * Wd);
     int rc;
     if (prep && (rc = scan_prep(a, w, st)) != DEER_OK) return rc;
-    DEER_KERNEL_PDL(c.name, st, kern, grid, (unsigned)c.threads, c.smem, a, w);
+    DEER_KERNEL_PDL(c.name, a.n <= 8, st, kern, grid, (unsigned)c.threads, c.smem, a, w);
     return DEER_OK;
 }
 
@@ -368,7 +368,7 @@ template <int N> static int launch_cell_wide(CellArgs c, cudaStream_t st)
     const size_t per_sm = (200 * 1024) / C::SMEM;
     const size_t cap = (size_t)num_sms() * (per_sm > 4 ? 4 : per_sm);
     const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
-    DEER_KERNEL_PDL("cell_wide_kernel", st, cell_wide_kernel<N>, blocks, (unsigned)C::THREADS, C::SMEM, c);
+    DEER_KERNEL_PDL("cell_wide_kernel", false, st, cell_wide_kernel<N>, blocks, (unsigned)C::THREADS, C::SMEM, c);
     return DEER_OK;
 }
 
@@ -383,12 +383,12 @@ template <int N> static int launch_cell_small(CellArgs c, cudaStream_t st)
     const size_t cap = blocks < 16 * resident ? resident : (size_t)num_sms() * 8;
     if (blocks > cap) blocks = cap;
     const unsigned gb = (unsigned)blocks;
-    if (c.u) { DEER_KERNEL_PDL("cell_small_kernel", st, (cell_small_kernel<N, 0>), gb, 256u, 0, c); return DEER_OK; }
+    if (c.u) { DEER_KERNEL_PDL("cell_small_kernel", true, st, (cell_small_kernel<N, 0>), gb, 256u, 0, c); return DEER_OK; }
     switch (c.m) {
-    case 1: DEER_KERNEL_PDL("cell_small_kernel", st, (cell_small_kernel<N, 1>), gb, 256u, 0, c); break;
-    case 2: DEER_KERNEL_PDL("cell_small_kernel", st, (cell_small_kernel<N, 2>), gb, 256u, 0, c); break;
-    case 4: DEER_KERNEL_PDL("cell_small_kernel", st, (cell_small_kernel<N, 4>), gb, 256u, 0, c); break;
-    case 8: DEER_KERNEL_PDL("cell_small_kernel", st, (cell_small_kernel<N, 8>), gb, 256u, 0, c); break;
+    case 1: DEER_KERNEL_PDL("cell_small_kernel", true, st, (cell_small_kernel<N, 1>), gb, 256u, 0, c); break;
+    case 2: DEER_KERNEL_PDL("cell_small_kernel", true, st, (cell_small_kernel<N, 2>), gb, 256u, 0, c); break;
+    case 4: DEER_KERNEL_PDL("cell_small_kernel", true, st, (cell_small_kernel<N, 4>), gb, 256u, 0, c); break;
+    case 8: DEER_KERNEL_PDL("cell_small_kernel", true, st, (cell_small_kernel<N, 8>), gb, 256u, 0, c); break;
     default: return DEER_ERR_INVALID_ARG;
     }
     return DEER_OK;
