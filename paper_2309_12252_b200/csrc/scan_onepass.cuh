@@ -54,10 +54,13 @@ template <int N> struct OnePass {
     static constexpr int JBUF = CHAINS * JRUN, BBUF = CHAINS * BRUN;
     static constexpr int AGG = N * N + N;              // floats of one aggregate (A row-major, then beta)
     static constexpr int Q = (N == 1) ? 3 : (N == 4) ? 1 : 2;   // pending tiles (A scheduled, B not yet) per CTA
-    // kept per pending tile: n = 8: chain aggregates + warp aggregates;
-    //                        n <= 4: exclusive chain prefixes (within the warp) + exclusive warp prefixes
-    static constexpr int PEND = (CHAINS + WARPS) * AGG;
-    static constexpr int SM_FLOATS = JBUF + BBUF + Q * PEND + WARPS * 2 * AGG + AGG + CHAINS * N + WARPS * N + N + 4;
+    // with one pending tile the B item follows its own A item directly: the tile stays staged and
+    // each thread keeps its chain's exclusive prefix in registers
+    static constexpr bool HOLD = (Q == 1);
+    // kept per pending tile: exclusive chain prefixes within the warp (not when held in registers)
+    // + exclusive warp prefixes
+    static constexpr int PEND = ((HOLD ? 0 : CHAINS) + WARPS) * AGG;
+    static constexpr int SM_FLOATS = JBUF + BBUF + Q * PEND + WARPS * 2 * AGG + N + 4;
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 64 + 128;
     static constexpr int MAX_SEQ_PER_WARP = 8;         // sequences one resolver warp can serve
     static_assert(32 * AGG <= JBUF / WARPS, "resolver staging must fit the tile buffer");
@@ -270,12 +273,13 @@ template <int N> __device__ __forceinline__ RegAgg<N> ragg_shfl_up(const RegAgg<
     return o;
 }
 
-// inclusive scan over the lanes of a warp (lane l ends with agg_l o ... o agg_0); returns the
-// exclusive prefix (identity in lane 0) in `excl`
-template <int N> __device__ __forceinline__ void ragg_warp_scan(RegAgg<N> &r, RegAgg<N> &excl, int lane)
+// inclusive scan over the first W lanes of a warp (lane l ends with agg_l o ... o agg_0; the other
+// lanes hold identities); returns the exclusive prefix (identity in lane 0) in `excl`
+template <int N, int W = 32>
+__device__ __forceinline__ void ragg_warp_scan(RegAgg<N> &r, RegAgg<N> &excl, int lane)
 {
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
+    for (int d = 1; d < W; d <<= 1) {
         RegAgg<N> p = ragg_shfl_up<N>(r, d);
         if (lane >= d) {
             RegAgg<N> e = p;            // earlier part
@@ -431,12 +435,9 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     extern __shared__ __align__(16) float smem_raw[];
     float *sJ = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     float *sB = sJ + C::JBUF;
-    float *pend = sB + C::BBUF;                // Q x { chain aggregates / prefixes, warp aggregates / prefixes }
+    float *pend = sB + C::BBUF;                // Q x { chain prefixes (unless held), warp prefixes }
     float *tmp = pend + Q * PEND;
-    float *tagg = tmp + WARPS * 2 * AGG;
-    float *cstart = tagg + AGG;
-    float *wstart = cstart + CHAINS * N;
-    float *ystart = wstart + WARPS * N;
+    float *ystart = tmp + WARPS * 2 * AGG;
     uint64_t *bar = (uint64_t *)(((uintptr_t)(ystart + N) + 15) & ~(uintptr_t)15);
     __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role;
 
@@ -475,6 +476,8 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     // pending queue (thread 0 only): tiles whose A item has run
     int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
     bool exhausted = false;
+    RegAgg<N> held;           // this thread's exclusive chain prefix, A item -> B item (one pending tile)
+    ragg_identity<N>(held);
 
     for (;;) {
         __syncthreads();      // previous item done with shared memory and with the s_* words
@@ -513,8 +516,9 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         __syncthreads();
         if (s_kind < 0 || s_abort) break;
         const int kind = s_kind, seq = s_seq, c = s_c;
-        float *agg = pend + s_slot * PEND;          // chain aggregates (n = 8) / exclusive chain prefixes
-        float *wagg = agg + CHAINS * AGG;           // warp aggregates (n = 8) / exclusive warp prefixes
+        constexpr bool HOLD = C::HOLD;
+        float *agg = pend + s_slot * PEND;                      // exclusive chain prefixes (unless held)
+        float *wagg = agg + (HOLD ? 0 : CHAINS * AGG);          // exclusive warp prefixes
         TileGeom<N, REV> tg;
         tg.s0 = c * C::L;
         tg.Lt = min(C::L, T - tg.s0);
@@ -526,21 +530,43 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         const size_t tile_index = (size_t)seq * w.nch + c;
         const float *Jt_src = a.J + ((size_t)seq * T + j_lo) * NN;
         const float *bt_src = a.b + ((size_t)seq * T + p_lo) * N;
+        // n = 4 fast paths: a full tile (all runs complete, every J_t present)
+        const bool full_tile = (N == 4) && Lt == C::L && jcnt_tile == C::L;
+        auto full_off = [&](int u) {        // float offset into sB of ascending-t position u of a full tile
+            const int blk = u / S, within = u - blk * S;
+            return (REV ? CHAINS - 1 - blk : blk) * C::BRUN + within * N;
+        };
 
         // ------------------------------------------------ stage the tile
         // (with one pending tile per CTA the B item follows its own A item directly: the tile is
         // still in shared memory, untouched, and is not staged again)
-        constexpr bool HOLD = (Q == 1);
         if constexpr (CPASYNC) {
             constexpr int PPE = NN / 4;                       // 16-byte pieces per J_t
-            if (!(HOLD && kind == 1))
-            for (int g = tid; g < jcnt_tile * PPE; g += C::THREADS) {
-                const int u = g / PPE, v = g - u * PPE;
-                cp_async16(sJ + tg.jmat_off(u) + v * 4, Jt_src + (size_t)u * NN + v * 4);
+            if (!(HOLD && kind == 1)) {
+                if (full_tile) {
+                    // a full tile: every chain's run is one contiguous block of S positions in global
+                    // memory, so the destination follows from the piece index by constants
+                    constexpr int RUN_PIECES = S * PPE;
+#pragma unroll
+                    for (int k = 0; k < C::L * PPE / C::THREADS; ++k) {
+                        const int p = tid + k * C::THREADS;
+                        const int blk = p / RUN_PIECES, within = p - blk * RUN_PIECES;
+                        cp_async16(sJ + (REV ? CHAINS - 1 - blk : blk) * C::JRUN + within * 4, Jt_src + (size_t)p * 4);
+                    }
+#pragma unroll
+                    for (int k = 0; k < C::L / C::THREADS; ++k) {
+                        const int u = tid + k * C::THREADS;
+                        cp_async16(sB + full_off(u), bt_src + (size_t)u * 4);
+                    }
+                } else {
+                    for (int g = tid; g < jcnt_tile * PPE; g += C::THREADS) {
+                        const int u = g / PPE, v = g - u * PPE;
+                        cp_async16(sJ + tg.jmat_off(u) + v * 4, Jt_src + (size_t)u * NN + v * 4);
+                    }
+                    for (int g = tid; g < Lt * N / 4; g += C::THREADS)
+                        cp_async16(sB + tg.out_off(g * 4 / N, (g * 4) % N), bt_src + g * 4);
+                }
             }
-            if (!(HOLD && kind == 1))
-            for (int g = tid; g < Lt * N / 4; g += C::THREADS)
-                cp_async16(sB + tg.out_off(g * 4 / N, (g * 4) % N), bt_src + g * 4);
             cp_async_commit();
         } else if (!(HOLD && kind == 1)) {
             const unsigned jb = (unsigned)jcnt_tile * NN * 4u, bb = (unsigned)Lt * N * 4u;
@@ -653,7 +679,8 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                 }
                 RegAgg<N> ex;
                 ragg_warp_scan<N>(r, ex, lane);
-                ragg_store<N>(agg + chain * AGG, ex);              // exclusive prefix inside the warp
+                if constexpr (HOLD) held = ex;                     // exclusive prefix inside the warp
+                else ragg_store<N>(agg + chain * AGG, ex);
                 if (lane == 31) ragg_store<N>(tmp + warp * AGG, r);   // warp aggregate
                 __syncthreads();
                 if (warp == 0) {
@@ -661,7 +688,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                     if (lane < WARPS) ragg_load<N>(wr, tmp + lane * AGG);
                     else ragg_identity<N>(wr);
                     RegAgg<N> wex;
-                    ragg_warp_scan<N>(wr, wex, lane);
+                    ragg_warp_scan<N, WARPS>(wr, wex, lane);
                     if (lane < WARPS) ragg_store<N>(wagg + lane * AGG, wex);   // exclusive prefix over warps
                     if (lane == WARPS - 1) {
                         ragg_store<N>(w.aggs + tile_index * AGG, wr);           // tile aggregate
@@ -678,8 +705,12 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                 RegAgg<N> e;
                 ragg_load<N>(e, wagg + warp * AGG);
                 ragg_apply<N>(e, y);
-                ragg_load<N>(e, agg + chain * AGG);
-                ragg_apply<N>(e, y);
+                if constexpr (HOLD) {
+                    ragg_apply<N>(held, y);
+                } else {
+                    ragg_load<N>(e, agg + chain * AGG);
+                    ragg_apply<N>(e, y);
+                }
                 if constexpr (N == 1) {
                     float yv = y[0];
 #pragma unroll
@@ -735,7 +766,19 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             const int total = Lt * N;
             const bool vec = (N >= 4 || (tg.low_slot() * N) % 4 == 0) && (((uintptr_t)yo & 15) == 0) &&
                              ((total & 3) == 0) && (!yold || ((uintptr_t)yold & 15) == 0);
-            if (vec) {
+            if (vec && full_tile) {
+#pragma unroll
+                for (int k = 0; k < C::L / C::THREADS; ++k) {
+                    const int u = tid + k * C::THREADS;
+                    const float4 val = *reinterpret_cast<const float4 *>(sB + full_off(u));
+                    if (yold) {
+                        const float4 o = __ldg(reinterpret_cast<const float4 *>(yold) + u);
+                        mb = max(mb, absdiff_bits(val.x, o.x)); mb = max(mb, absdiff_bits(val.y, o.y));
+                        mb = max(mb, absdiff_bits(val.z, o.z)); mb = max(mb, absdiff_bits(val.w, o.w));
+                    }
+                    reinterpret_cast<float4 *>(yo)[u] = val;
+                }
+            } else if (vec) {
                 for (int g4 = tid; g4 < total / 4; g4 += C::THREADS) {
                     const int g = 4 * g4;
                     const float4 val = *reinterpret_cast<const float4 *>(sB + tg.out_off(g / N, g % N));
