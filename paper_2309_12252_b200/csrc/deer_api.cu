@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "kernels_generic.cuh"
 #include "scan_onepass.cuh"
+#include "scan_hold4.cuh"
 #include "scan_warp8.cuh"
 #include "scan_warpn.cuh"
 #include "scan_cta64.cuh"
@@ -204,6 +205,15 @@ static int launch_onepass(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 }
 
 template <bool REV>
+static int launch_hold4(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
+{
+    using C = OnePass<4>;
+    static int occ[MAX_DEVICES] = {0};
+    const PassCfg c{"scan_hold4_kernel", C::THREADS, C::SMEM, C::WARPS, C::MAX_SEQ_PER_WARP, 32, 8};
+    return launch_single_pass(scan_hold4_kernel<REV>, occ, c, a, w, prep, st);
+}
+
+template <bool REV>
 static int launch_warp8(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = Warp8;
@@ -247,8 +257,8 @@ static int scan_onepass(ScanArgs a, OnePassWs w, bool prep, int flags, cudaStrea
     case 3: return launch_onepass<1, true>(a, w, prep, st);
     case 4: return launch_onepass<2, false>(a, w, prep, st);
     case 5: return launch_onepass<2, true>(a, w, prep, st);
-    case 8: return launch_onepass<4, false>(a, w, prep, st);
-    case 9: return launch_onepass<4, true>(a, w, prep, st);
+    case 8: return launch_hold4<false>(a, w, prep, st);
+    case 9: return launch_hold4<true>(a, w, prep, st);
     case 16: return launch_warp8<false>(a, w, prep, st);
     case 17: return launch_warp8<true>(a, w, prep, st);
     case 32: return launch_warpn<16, false>(a, w, prep, st);

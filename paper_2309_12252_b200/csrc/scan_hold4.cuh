@@ -1,0 +1,254 @@
+// Single-pass scan of the linear recurrence for n = 4 (Sec. 2.2 / Eq. 5 solve; App. B.1 adjoint).
+//
+// Same protocol as the n <= 2 kernel (tile aggregates published with a release flag, resolver
+// warps that walk a sequence's aggregates in order, entering states as {value, flag} words, every
+// wait bounded), but a worker CTA holds ONE tile at a time and visits it twice back to back:
+//
+//   stage the tile (per-thread 16-byte cp.async into run-padded shared memory)
+//   A: every thread folds its chain of S positions into (A, beta) in registers; a warp-shuffle
+//      scan gives each thread its chain's exclusive prefix inside the warp, which STAYS IN
+//      REGISTERS; warp 0 combines the warp aggregates and publishes the tile aggregate
+//   while warp 1 polls for the state entering the tile, the last thread claims the CTA's next
+//   tile (the atomic's latency hides behind the replay)
+//   B: every thread replays its chain from (warp prefix, chain prefix)(entering state); y
+//      overwrites b in shared memory and is streamed out with the max |y - y_old| reduction
+//
+// The tile is read from HBM once and never staged twice; five CTA barriers per tile.  Shared
+// memory per CTA is the tile plus a few hundred bytes, so four CTAs share an SM.
+#pragma once
+#include "scan_onepass.cuh"
+
+namespace deer {
+
+template <bool REV>
+__global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArgs a, OnePassWs w)
+{
+    constexpr int N = 4, NN = 16;
+    using C = OnePass<N>;
+    static_assert(C::HOLD && C::PADDED, "one tile per CTA, run-padded layout");
+    constexpr int S = C::S, CHAINS = C::CHAINS, AGG = C::AGG, WARPS = C::WARPS, THREADS = C::THREADS;
+    constexpr int PPE = NN / 4;                     // 16-byte pieces per J_t
+    constexpr int CLAIMER = THREADS - 1;
+    static_assert((C::L * PPE) % THREADS == 0 && C::L % THREADS == 0, "full-tile loops have constant trip counts");
+
+    extern __shared__ __align__(16) float smem_raw[];
+    float *sJ = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    float *sB = sJ + C::JBUF;
+    float *wagg = sB + C::BBUF;                     // exclusive warp prefixes
+    float *tmp = wagg + C::PEND;                    // warp aggregates
+    float *ystart = tmp + WARPS * 2 * AGG;
+    __shared__ int s_seq, s_c, s_abort, s_role;
+
+    pdl_prologue();
+    if (loop_ended(a.st)) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int chain = tid;
+    const int T = a.T;
+
+    if (tid == 0) {
+        s_abort = 0;
+        s_role = (int)atomicAdd(&a.st->role_counter, 1u);
+    }
+    __syncthreads();
+    if (s_role < w.resolvers) {
+        resolver_loop<N>(a, w, sJ, s_role * WARPS + warp, w.resolvers * WARPS, lane);
+        __syncthreads();
+        if (tid == 0) scan_epilogue(a.st);
+        return;
+    }
+    unsigned mb = 0;          // running max |y - yold| bits of this thread
+
+    // claim: ids come from the launch-wide counter; id -> (seq, tile), padding ids of the last
+    // window are skipped; c < 0 when no tile is left
+    auto claim_from = [&](unsigned id, int &seq, int &c) {
+        for (;;) {
+            if (id >= w.total_ids) { c = -1; return; }
+            const unsigned j = id % (unsigned)w.Wd;
+            const unsigned ws_ = id / (unsigned)w.Wd;
+            seq = (int)(ws_ % (unsigned)a.B);
+            const unsigned win = ws_ / (unsigned)a.B;
+            c = (int)(win * (unsigned)w.Wd + j);
+            if (c < w.nch) return;
+            id = atomicAdd(&a.st->tile_counter, 1u);
+        }
+    };
+    if (tid == CLAIMER) {
+        int seq = -1, c = -1;
+        claim_from(atomicAdd(&a.st->tile_counter, 1u), seq, c);
+        s_seq = seq; s_c = c;
+    }
+    __syncthreads();
+
+    for (;;) {
+        const int seq = s_seq, c = s_c;
+        if (c < 0) break;
+        TileGeom<N, REV> tg;
+        tg.s0 = c * C::L;
+        tg.Lt = min(C::L, T - tg.s0);
+        tg.T = T;
+        const int Lt = tg.Lt;
+        const size_t p_lo = tg.t_lo();                                  // first b element of the tile
+        const size_t j_lo = REV ? p_lo + 1 : p_lo;                      // first J element of the tile
+        const int jcnt_tile = (REV && tg.s0 == 0) ? Lt - 1 : Lt;        // (reverse: J[T] does not exist)
+        const size_t tile_index = (size_t)seq * w.nch + c;
+        const float *Jt_src = a.J + ((size_t)seq * T + j_lo) * NN;
+        const float *bt_src = a.b + ((size_t)seq * T + p_lo) * N;
+        // a full tile (all runs complete, every J_t present): every chain's run is one contiguous
+        // block of S positions in global memory and offsets follow from the index by constants
+        const bool full_tile = Lt == C::L && jcnt_tile == C::L;
+        auto full_off = [&](int u) {        // float offset into sB of ascending-t position u of a full tile
+            const int blk = u / S, within = u - blk * S;
+            return (REV ? CHAINS - 1 - blk : blk) * C::BRUN + within * N;
+        };
+
+        // ------------------------------------------------ stage the tile
+        if (full_tile) {
+            constexpr int RUN_PIECES = S * PPE;
+#pragma unroll
+            for (int k = 0; k < C::L * PPE / THREADS; ++k) {
+                const int p = tid + k * THREADS;
+                const int blk = p / RUN_PIECES, within = p - blk * RUN_PIECES;
+                cp_async16(sJ + (REV ? CHAINS - 1 - blk : blk) * C::JRUN + within * 4, Jt_src + (size_t)p * 4);
+            }
+#pragma unroll
+            for (int k = 0; k < C::L / THREADS; ++k) {
+                const int u = tid + k * THREADS;
+                cp_async16(sB + full_off(u), bt_src + (size_t)u * 4);
+            }
+        } else {
+            for (int g = tid; g < jcnt_tile * PPE; g += THREADS) {
+                const int u = g / PPE, v = g - u * PPE;
+                cp_async16(sJ + tg.jmat_off(u) + v * 4, Jt_src + (size_t)u * NN + v * 4);
+            }
+            for (int u = tid; u < Lt; u += THREADS) cp_async16(sB + tg.out_off(u, 0), bt_src + (size_t)u * 4);
+        }
+        cp_async_commit();
+        cp_async_wait_0();
+        __syncthreads();      // tile staged; every thread has read s_seq / s_c
+
+        // ------------------------------------------------ A: chain aggregates, prefixes, publish
+        const int cnt = tg.run_cnt(chain);
+        RegAgg<N> held;       // this chain's exclusive prefix inside the warp
+        {
+            RegAgg<N> r;
+            ragg_identity<N>(r);
+#pragma unroll
+            for (int q = 0; q < S; ++q) {
+                if (q < cnt) {
+                    float M[N][N], bq[N];
+                    load_chain_step<N, REV>(sJ, sB, tg, chain, q, cnt, M, bq);
+                    ragg_push<N>(r, M, bq);
+                }
+            }
+            ragg_warp_scan<N>(r, held, lane);
+            if (lane == 31) ragg_store<N>(tmp + warp * AGG, r);   // warp aggregate
+        }
+        __syncthreads();
+        if (warp == 0) {
+            RegAgg<N> wr, wex;
+            if (lane < WARPS) ragg_load<N>(wr, tmp + lane * AGG);
+            else ragg_identity<N>(wr);
+            ragg_warp_scan<N, WARPS>(wr, wex, lane);
+            if (lane == WARPS - 1) {
+                ragg_store<N>(w.aggs + tile_index * AGG, wr);           // tile aggregate
+                __threadfence();
+                st_release_u32(w.flags + tile_index, 1u);
+            }
+            if (lane < WARPS) ragg_store<N>(wagg + lane * AGG, wex);   // exclusive prefix over warps
+        } else if (warp == 1) {
+            // the state entering the tile ({value, flag} words written by the sequence's resolver)
+            const unsigned long long *src = w.starts + tile_index * N;
+            unsigned spins = 0;
+            bool ok = true;
+            for (;;) {
+                const unsigned long long v = (lane < N) ? ld_relaxed_u64(src + lane) : LL_FLAG;
+                if (__all_sync(0xffffffffu, v != 0ull)) {
+                    if (lane < N) {
+                        ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                        st_relaxed_u64(w.starts + tile_index * N + lane, 0ull);     // consumed: cleared for the next launch
+                    }
+                    break;
+                }
+                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+            }
+            if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
+        }
+        __syncthreads();      // ystart, warp prefixes and s_abort visible
+        if (s_abort) break;
+        unsigned next_id = 0;
+        if (tid == CLAIMER) next_id = atomicAdd(&a.st->tile_counter, 1u);
+
+        // ------------------------------------------------ B: replay from the entering state
+        {
+            float y[N];
+#pragma unroll
+            for (int k = 0; k < N; ++k) y[k] = ystart[k];
+            RegAgg<N> e;
+            ragg_load<N>(e, wagg + warp * AGG);
+            ragg_apply<N>(e, y);
+            ragg_apply<N>(held, y);
+#pragma unroll
+            for (int q = 0; q < S; ++q) {
+                if (q < cnt) {
+                    float M[N][N], bq[N];
+                    load_chain_step<N, REV>(sJ, sB, tg, chain, q, cnt, M, bq);
+                    float yn[N];
+#pragma unroll
+                    for (int i = 0; i < N; ++i) {
+                        yn[i] = bq[i];
+#pragma unroll
+                        for (int k = 0; k < N; ++k) yn[i] = fmaf(M[i][k], y[k], yn[i]);
+                    }
+#pragma unroll
+                    for (int i = 0; i < N; ++i) y[i] = yn[i];
+                    *reinterpret_cast<float4 *>(sB + tg.b_off(chain, q, cnt)) = make_float4(yn[0], yn[1], yn[2], yn[3]);
+                }
+            }
+        }
+        __syncthreads();      // y complete in shared memory
+        if (tid == CLAIMER) {
+            int nseq = -1, nc = -1;
+            claim_from(next_id, nseq, nc);
+            s_seq = nseq; s_c = nc;
+        }
+
+        // ------------------------------------------------ stream y out (+ max |y - yold|)
+        {
+            const size_t gbase = ((size_t)seq * T + p_lo) * N;
+            float *yo = a.y + gbase;
+            const float *yold = a.yold ? a.yold + gbase : nullptr;
+            const bool vec = (((uintptr_t)yo & 15) == 0) && (!yold || ((uintptr_t)yold & 15) == 0);
+            auto put = [&](int u, int off) {
+                const float4 val = *reinterpret_cast<const float4 *>(sB + off);
+                if (yold) {
+                    const float4 o = __ldg(reinterpret_cast<const float4 *>(yold) + u);
+                    mb = max(mb, absdiff_bits(val.x, o.x)); mb = max(mb, absdiff_bits(val.y, o.y));
+                    mb = max(mb, absdiff_bits(val.z, o.z)); mb = max(mb, absdiff_bits(val.w, o.w));
+                }
+                reinterpret_cast<float4 *>(yo)[u] = val;
+            };
+            if (vec && full_tile) {
+#pragma unroll
+                for (int k = 0; k < C::L / THREADS; ++k) put(tid + k * THREADS, full_off(tid + k * THREADS));
+            } else if (vec) {
+                for (int u = tid; u < Lt; u += THREADS) put(u, tg.out_off(u, 0));
+            } else {
+                for (int g = tid; g < Lt * N; g += THREADS) {
+                    const float val = sB[tg.out_off(g / N, g % N)];
+                    if (yold) mb = max(mb, absdiff_bits(val, yold[g]));
+                    yo[g] = val;
+                }
+            }
+        }
+        __syncthreads();      // shared memory free; the next tile's id visible
+    }
+    if (a.yold) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+        if (lane == 0 && mb) { atomicMax(&a.st->err_bits, mb); __threadfence(); }
+    }
+    __syncthreads();
+    if (tid == 0) scan_epilogue(a.st);
+}
+
+}  // namespace deer

@@ -228,6 +228,42 @@ template <int N, bool REV> struct TileGeom {
     __device__ __forceinline__ size_t t_lo() const { return REV ? (size_t)(T - s0 - Lt) : (size_t)s0; }
 };
 
+// one step of a chain from the staged tile: M = J (forward) or J^T (reverse; identity at scan position 0)
+template <int N, bool REV>
+__device__ __forceinline__ void load_chain_step(const float *sJ, const float *sB, const TileGeom<N, REV> &tg, int chain,
+                                                int q, int cnt, float (&M)[N][N], float (&bq)[N])
+{
+    const float *Je = sJ + tg.j_off(chain, q, cnt);
+    const float *bv = sB + tg.b_off(chain, q, cnt);
+    const bool ident = REV && (tg.s0 + chain * OnePass<N>::S + q == 0);
+    if constexpr (N == 2) {
+        const float4 f = *reinterpret_cast<const float4 *>(Je);
+        const float2 g = *reinterpret_cast<const float2 *>(bv);
+        M[0][0] = f.x; M[0][1] = REV ? f.z : f.y; M[1][0] = REV ? f.y : f.z; M[1][1] = f.w;
+        bq[0] = g.x; bq[1] = g.y;
+    } else {
+        static_assert(N == 2 || N == 4, "chain steps are read as 128-bit words");
+        float R[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 f = reinterpret_cast<const float4 *>(Je)[i];
+            R[i][0] = f.x; R[i][1] = f.y; R[i][2] = f.z; R[i][3] = f.w;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) M[i][k] = REV ? R[k][i] : R[i][k];
+        const float4 g = *reinterpret_cast<const float4 *>(bv);
+        bq[0] = g.x; bq[1] = g.y; bq[2] = g.z; bq[3] = g.w;
+    }
+    if (ident) {
+#pragma unroll
+        for (int i = 0; i < N; ++i)
+#pragma unroll
+            for (int k = 0; k < N; ++k) M[i][k] = (i == k) ? 1.0f : 0.0f;
+    }
+}
+
 // ---- n <= 4: one thread per chain; aggregates live in registers and are combined by warp shuffles
 template <int N> struct RegAgg { float A[N][N]; float be[N]; };
 
@@ -429,13 +465,12 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     constexpr int S = C::S, CHAINS = C::CHAINS;
     constexpr int AGG = C::AGG, WARPS = C::WARPS, NN = N * N;
     constexpr int Q = C::Q, PEND = C::PEND;
-    constexpr bool CPASYNC = (N == 4);         // J staged by per-thread 16-byte cp.async
-    static_assert(N <= 4, "thread-per-chain kernel: n = 8 and above have their own kernels");
+    static_assert(N <= 2, "thread-per-chain kernel with a queue of pending tiles: n = 4 and above have their own kernels");
 
     extern __shared__ __align__(16) float smem_raw[];
     float *sJ = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     float *sB = sJ + C::JBUF;
-    float *pend = sB + C::BBUF;                // Q x { chain prefixes (unless held), warp prefixes }
+    float *pend = sB + C::BBUF;                // Q x { chain prefixes, warp prefixes }
     float *tmp = pend + Q * PEND;
     float *ystart = tmp + WARPS * 2 * AGG;
     uint64_t *bar = (uint64_t *)(((uintptr_t)(ystart + N) + 15) & ~(uintptr_t)15);
@@ -476,8 +511,6 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     // pending queue (thread 0 only): tiles whose A item has run
     int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
     bool exhausted = false;
-    RegAgg<N> held;           // this thread's exclusive chain prefix, A item -> B item (one pending tile)
-    ragg_identity<N>(held);
 
     for (;;) {
         __syncthreads();      // previous item done with shared memory and with the s_* words
@@ -516,9 +549,8 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         __syncthreads();
         if (s_kind < 0 || s_abort) break;
         const int kind = s_kind, seq = s_seq, c = s_c;
-        constexpr bool HOLD = C::HOLD;
-        float *agg = pend + s_slot * PEND;                      // exclusive chain prefixes (unless held)
-        float *wagg = agg + (HOLD ? 0 : CHAINS * AGG);          // exclusive warp prefixes
+        float *agg = pend + s_slot * PEND;          // exclusive chain prefixes within the warp
+        float *wagg = agg + CHAINS * AGG;           // exclusive warp prefixes
         TileGeom<N, REV> tg;
         tg.s0 = c * C::L;
         tg.Lt = min(C::L, T - tg.s0);
@@ -530,45 +562,8 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
         const size_t tile_index = (size_t)seq * w.nch + c;
         const float *Jt_src = a.J + ((size_t)seq * T + j_lo) * NN;
         const float *bt_src = a.b + ((size_t)seq * T + p_lo) * N;
-        // n = 4 fast paths: a full tile (all runs complete, every J_t present)
-        const bool full_tile = (N == 4) && Lt == C::L && jcnt_tile == C::L;
-        auto full_off = [&](int u) {        // float offset into sB of ascending-t position u of a full tile
-            const int blk = u / S, within = u - blk * S;
-            return (REV ? CHAINS - 1 - blk : blk) * C::BRUN + within * N;
-        };
-
-        // ------------------------------------------------ stage the tile
-        // (with one pending tile per CTA the B item follows its own A item directly: the tile is
-        // still in shared memory, untouched, and is not staged again)
-        if constexpr (CPASYNC) {
-            constexpr int PPE = NN / 4;                       // 16-byte pieces per J_t
-            if (!(HOLD && kind == 1)) {
-                if (full_tile) {
-                    // a full tile: every chain's run is one contiguous block of S positions in global
-                    // memory, so the destination follows from the piece index by constants
-                    constexpr int RUN_PIECES = S * PPE;
-#pragma unroll
-                    for (int k = 0; k < C::L * PPE / C::THREADS; ++k) {
-                        const int p = tid + k * C::THREADS;
-                        const int blk = p / RUN_PIECES, within = p - blk * RUN_PIECES;
-                        cp_async16(sJ + (REV ? CHAINS - 1 - blk : blk) * C::JRUN + within * 4, Jt_src + (size_t)p * 4);
-                    }
-#pragma unroll
-                    for (int k = 0; k < C::L / C::THREADS; ++k) {
-                        const int u = tid + k * C::THREADS;
-                        cp_async16(sB + full_off(u), bt_src + (size_t)u * 4);
-                    }
-                } else {
-                    for (int g = tid; g < jcnt_tile * PPE; g += C::THREADS) {
-                        const int u = g / PPE, v = g - u * PPE;
-                        cp_async16(sJ + tg.jmat_off(u) + v * 4, Jt_src + (size_t)u * NN + v * 4);
-                    }
-                    for (int g = tid; g < Lt * N / 4; g += C::THREADS)
-                        cp_async16(sB + tg.out_off(g * 4 / N, (g * 4) % N), bt_src + g * 4);
-                }
-            }
-            cp_async_commit();
-        } else if (!(HOLD && kind == 1)) {
+        // ------------------------------------------------ stage the tile (bulk copies where aligned)
+        {
             const unsigned jb = (unsigned)jcnt_tile * NN * 4u, bb = (unsigned)Lt * N * 4u;
             float *jd = sJ + tg.low_slot() * NN, *bd = sB + tg.low_slot() * N;
             const bool jbulk = jb && ((uintptr_t)Jt_src & 15) == 0 && (jb & 15) == 0 && ((uintptr_t)jd & 15) == 0;
@@ -600,9 +595,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             }
             if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
         }
-        if constexpr (CPASYNC) {
-            cp_async_wait_0();
-        } else if (!(HOLD && kind == 1)) {
+        {
             unsigned spins = 0;
             while (!mbar_try_wait(bar, phase)) {
                 if (++spins > (SPIN_LIMIT >> 2)) { atomicOr(&a.st->flags, FLAG_TIMEOUT); s_abort = 1; break; }
@@ -614,38 +607,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
 
         const int cnt = tg.run_cnt(chain);
         {
-            // ============================================ n <= 4: one thread per chain
-            // one step of the chain: M = J (forward) or J^T (reverse; identity at scan position 0)
-            auto load_step = [&](int q, float (&M)[N][N], float (&bq)[N]) {
-                const float *Je = sJ + tg.j_off(chain, q, cnt);
-                const float *bv = sB + tg.b_off(chain, q, cnt);
-                const bool ident = REV && (s0 + chain * S + q == 0);
-                if constexpr (N == 2) {
-                    const float4 f = *reinterpret_cast<const float4 *>(Je);
-                    const float2 g = *reinterpret_cast<const float2 *>(bv);
-                    M[0][0] = f.x; M[0][1] = REV ? f.z : f.y; M[1][0] = REV ? f.y : f.z; M[1][1] = f.w;
-                    bq[0] = g.x; bq[1] = g.y;
-                } else {
-                    float R[4][4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float4 f = reinterpret_cast<const float4 *>(Je)[i];
-                        R[i][0] = f.x; R[i][1] = f.y; R[i][2] = f.z; R[i][3] = f.w;
-                    }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i)
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) M[i][k] = REV ? R[k][i] : R[i][k];
-                    const float4 g = *reinterpret_cast<const float4 *>(bv);
-                    bq[0] = g.x; bq[1] = g.y; bq[2] = g.z; bq[3] = g.w;
-                }
-                if (ident) {
-#pragma unroll
-                    for (int i = 0; i < N; ++i)
-#pragma unroll
-                        for (int k = 0; k < N; ++k) M[i][k] = (i == k) ? 1.0f : 0.0f;
-                }
-            };
+            // ============================================ one thread per chain
             if (kind == 0) {
                 RegAgg<N> r;
                 ragg_identity<N>(r);
@@ -672,15 +634,14 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                     for (int q = 0; q < S; ++q) {
                         if (q < cnt) {
                             float M[N][N], bq[N];
-                            load_step(q, M, bq);
+                            load_chain_step<N, REV>(sJ, sB, tg, chain, q, cnt, M, bq);
                             ragg_push<N>(r, M, bq);
                         }
                     }
                 }
                 RegAgg<N> ex;
                 ragg_warp_scan<N>(r, ex, lane);
-                if constexpr (HOLD) held = ex;                     // exclusive prefix inside the warp
-                else ragg_store<N>(agg + chain * AGG, ex);
+                ragg_store<N>(agg + chain * AGG, ex);              // exclusive prefix inside the warp
                 if (lane == 31) ragg_store<N>(tmp + warp * AGG, r);   // warp aggregate
                 __syncthreads();
                 if (warp == 0) {
@@ -705,12 +666,8 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                 RegAgg<N> e;
                 ragg_load<N>(e, wagg + warp * AGG);
                 ragg_apply<N>(e, y);
-                if constexpr (HOLD) {
-                    ragg_apply<N>(held, y);
-                } else {
-                    ragg_load<N>(e, agg + chain * AGG);
-                    ragg_apply<N>(e, y);
-                }
+                ragg_load<N>(e, agg + chain * AGG);
+                ragg_apply<N>(e, y);
                 if constexpr (N == 1) {
                     float yv = y[0];
 #pragma unroll
@@ -738,7 +695,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                     for (int q = 0; q < S; ++q) {
                         if (q < cnt) {
                             float M[N][N], bq[N];
-                            load_step(q, M, bq);
+                            load_chain_step<N, REV>(sJ, sB, tg, chain, q, cnt, M, bq);
                             float yn[N];
 #pragma unroll
                             for (int i = 0; i < N; ++i) {
@@ -766,19 +723,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             const int total = Lt * N;
             const bool vec = (N >= 4 || (tg.low_slot() * N) % 4 == 0) && (((uintptr_t)yo & 15) == 0) &&
                              ((total & 3) == 0) && (!yold || ((uintptr_t)yold & 15) == 0);
-            if (vec && full_tile) {
-#pragma unroll
-                for (int k = 0; k < C::L / C::THREADS; ++k) {
-                    const int u = tid + k * C::THREADS;
-                    const float4 val = *reinterpret_cast<const float4 *>(sB + full_off(u));
-                    if (yold) {
-                        const float4 o = __ldg(reinterpret_cast<const float4 *>(yold) + u);
-                        mb = max(mb, absdiff_bits(val.x, o.x)); mb = max(mb, absdiff_bits(val.y, o.y));
-                        mb = max(mb, absdiff_bits(val.z, o.z)); mb = max(mb, absdiff_bits(val.w, o.w));
-                    }
-                    reinterpret_cast<float4 *>(yo)[u] = val;
-                }
-            } else if (vec) {
+            if (vec) {
                 for (int g4 = tid; g4 < total / 4; g4 += C::THREADS) {
                     const int g = 4 * g4;
                     const float4 val = *reinterpret_cast<const float4 *>(sB + tg.out_off(g / N, g % N));
