@@ -81,6 +81,8 @@ struct ScanWs {
 
 static int num_sms();
 
+static bool onepass_ll_aggs(int n) { return n == 4; }
+
 static int onepass_tile_len(int n, int B, int T, int *sw)
 {
     *sw = 0;
@@ -110,7 +112,8 @@ static ScanWs carve_scan(Carver &cv, int B, int T, int n)
         w.op.nch = (T + L1 - 1) / L1;
         size_t tiles = (size_t)B * w.op.nch;
         w.op.flags = cv.take<unsigned>(tiles);
-        w.op.aggs = cv.take<float>(tiles * (n * n + n));
+        // (n = 4 publishes its aggregates as 64-bit {value, flag} words)
+        w.op.aggs = cv.take<float>(tiles * (n * n + n) * (onepass_ll_aggs(n) ? 2 : 1));
         w.op.starts = cv.take<unsigned long long>(tiles * n);
     }
     return w;
@@ -136,11 +139,13 @@ static int num_sms()
 static int scan_prep(const ScanArgs &a, const OnePassWs &w, cudaStream_t st)
 {
     const size_t tiles = (size_t)a.B * w.nch;
-    const size_t words = tiles * (size_t)(a.n + 1);
+    const size_t agg_words = onepass_ll_aggs(a.n) ? tiles * (size_t)(a.n * a.n + a.n) : 0;
+    const size_t words = tiles * (size_t)(a.n + 1) + agg_words;
     unsigned pb = (unsigned)((words + 255) / 256);
     if (pb > 592u) pb = 592u;
     if (pb < 1u) pb = 1u;
-    DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)a.n));
+    DEER_KERNEL("scan_prep_kernel", st, scan_prep_kernel<<<pb, 256, 0, st>>>(a.st, w.flags, tiles, w.starts, tiles * (size_t)a.n,
+                                                      (unsigned long long *)w.aggs, agg_words));
     return DEER_OK;
 }
 

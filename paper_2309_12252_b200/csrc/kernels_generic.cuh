@@ -302,13 +302,15 @@ __global__ void gen_apply_kernel(ScanArgs a)
 // Clears the single-pass scan's words (tile flags, entering states, counters) before the first scan
 // on a workspace; the scans leave them cleared.
 __global__ void scan_prep_kernel(StatusBlock *st, unsigned *flags, size_t nflags,
-                                 unsigned long long *starts, size_t nstarts)
+                                 unsigned long long *starts, size_t nstarts,
+                                 unsigned long long *agg_words, size_t nagg_words)
 {
     if (loop_ended(st)) return;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (size_t i = i0; i < nflags; i += stride) flags[i] = 0u;
     for (size_t i = i0; i < nstarts; i += stride) starts[i] = 0ull;
+    for (size_t i = i0; i < nagg_words; i += stride) agg_words[i] = 0ull;
     if (i0 == 0) { st->tile_counter = 0u; st->role_counter = 0u; st->exit_counter = 0u; }
 }
 

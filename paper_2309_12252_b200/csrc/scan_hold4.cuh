@@ -1,17 +1,19 @@
 // Single-pass scan of the linear recurrence for n = 4 (Sec. 2.2 / Eq. 5 solve; App. B.1 adjoint).
 //
-// Same protocol as the n <= 2 kernel (tile aggregates published with a release flag, resolver
-// warps that walk a sequence's aggregates in order, entering states as {value, flag} words, every
-// wait bounded), but a worker CTA holds ONE tile at a time and visits it twice back to back:
+// Same roles as the n <= 2 kernel (workers publish tile aggregates, resolver warps walk a
+// sequence's aggregates in order and publish the state entering every tile, every wait bounded),
+// with both directions of the exchange as 64-bit {value, flag} words (one round trip, no fence),
+// and a worker CTA holds ONE tile at a time and visits it twice back to back:
 //
 //   stage the tile (per-thread 16-byte cp.async into run-padded shared memory)
 //   A: every thread folds its chain of S positions into (A, beta) in registers; a warp-shuffle
 //      scan gives each thread its chain's exclusive prefix inside the warp, which STAYS IN
 //      REGISTERS; warp 0 combines the warp aggregates and publishes the tile aggregate
-//   while warp 1 polls for the state entering the tile, the last thread claims the CTA's next
-//   tile (the atomic's latency hides behind the replay)
+//   warp 1 polls for the state entering the tile; once it is there the last thread claims the
+//   CTA's next tile (the atomic's latency hides behind the replay)
 //   B: every thread replays its chain from (warp prefix, chain prefix)(entering state); y
-//      overwrites b in shared memory and is streamed out with the max |y - y_old| reduction
+//      overwrites b in shared memory and is streamed out with the max |y - y_old| reduction,
+//      while the next tile's J is already being copied into the freed J buffer
 //
 // The tile is read from HBM once and never staged twice; five CTA barriers per tile.  Shared
 // memory per CTA is the tile plus a few hundred bytes, so four CTAs share an SM.
@@ -19,6 +21,92 @@
 #include "scan_onepass.cuh"
 
 namespace deer {
+
+// Resolver role with aggregates published as 64-bit {value, flag} words: warp `rw` of `nrw` serves
+// sequences rw, rw + nrw, ...  A visit loads the words of the next WIN tiles of a sequence in one
+// round trip, takes the leading tiles whose words are all present, clears those words for the next
+// launch, and walks them, Y <- A Y + beta, writing the state entering every tile (lane i holds Y[i]).
+template <int N>
+__device__ void resolver_ll_loop(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
+{
+    using C = OnePass<N>;
+    constexpr int AGG = C::AGG, NN = N * N;
+    constexpr int WIN = 16;                         // tiles looked at per visit
+    constexpr int PER = WIN * AGG / 32;             // words per lane
+    static_assert((WIN * AGG) % 32 == 0 && WIN < 32, "window of whole words per lane");
+    float *stage = stage_all + (threadIdx.x >> 5) * 32 * AGG;
+    int nseq = 0;
+    int pos[C::MAX_SEQ_PER_WARP];
+    float yv[C::MAX_SEQ_PER_WARP];              // lane i < N: component i of the sequence's running state
+#pragma unroll
+    for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
+        pos[k] = 0; yv[k] = 0.0f;
+        const int s = rw + k * nrw;
+        if (s < a.B) {
+            nseq = k + 1;
+            if (lane < N && a.y0) yv[k] = a.y0[(size_t)s * N + lane];
+        }
+    }
+    int remaining = nseq;
+    unsigned spins = 0;
+    while (remaining > 0) {
+        bool progressed = false;
+#pragma unroll
+        for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
+            if (k >= nseq) break;
+            const int c0 = pos[k];
+            if (c0 >= w.nch) continue;
+            const int s = rw + k * nrw;
+            unsigned long long *words = reinterpret_cast<unsigned long long *>(w.aggs) + ((size_t)s * w.nch + c0) * AGG;
+            const int nt = min(WIN, w.nch - c0);
+            const int total = nt * AGG;
+            unsigned long long v[PER];
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int i = lane + 32 * u;
+                v[u] = (i < total) ? ld_relaxed_u64(words + i) : 0ull;
+            }
+            unsigned missing = ~0u << nt;           // tiles beyond the window or the sequence
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int i = lane + 32 * u;
+                if (i < total && (v[u] >> 32) == 0ull) missing |= 1u << (i / AGG);
+            }
+            missing = __reduce_or_sync(0xffffffffu, missing);
+            const int cnt = __ffs(missing) - 1;     // leading tiles with every word present
+            if (cnt == 0) continue;
+            progressed = true;
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int i = lane + 32 * u;
+                if (i < cnt * AGG) {
+                    stage[i] = __uint_as_float((unsigned)(v[u] & 0xffffffffull));
+                    st_relaxed_u64(words + i, 0ull);                 // consumed: cleared for the next launch
+                }
+            }
+            __syncwarp();
+            unsigned long long *out = w.starts + ((size_t)s * w.nch + c0) * N;
+            float y = yv[k];
+            for (int q = 0; q < cnt; ++q) {
+                if (lane < N) st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y));
+                const float *ag = stage + q * AGG;
+                float acc = (lane < N) ? ag[NN + lane] : 0.0f;
+#pragma unroll
+                for (int i = 0; i < N; ++i) {
+                    const float yi = __shfl_sync(0xffffffffu, y, i);
+                    if (lane < N) acc = fmaf(ag[lane * N + i], yi, acc);
+                }
+                y = acc;
+            }
+            yv[k] = y;
+            __syncwarp();
+            pos[k] = c0 + cnt;
+            if (pos[k] >= w.nch) --remaining;
+        }
+        if (progressed) spins = 0;
+        else if (!keep_spinning(a.st, spins)) return;
+    }
+}
 
 template <bool REV>
 __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArgs a, OnePassWs w)
@@ -51,7 +139,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
     }
     __syncthreads();
     if (s_role < w.resolvers) {
-        resolver_loop<N>(a, w, sJ, s_role * WARPS + warp, w.resolvers * WARPS, lane);
+        resolver_ll_loop<N>(a, w, sJ, s_role * WARPS + warp, w.resolvers * WARPS, lane);
         __syncthreads();
         if (tid == 0) scan_epilogue(a.st);
         return;
@@ -72,56 +160,78 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
             id = atomicAdd(&a.st->tile_counter, 1u);
         }
     };
+    // geometry and sources of one tile
+    struct Tile {
+        TileGeom<N, REV> tg;
+        const float *Jsrc, *bsrc;
+        size_t index, gbase;
+        int jcnt;
+        bool full;      // all runs complete and every J_t present: each chain's run is one contiguous
+                        // block of S positions in global memory and offsets follow by constants
+    };
+    auto make_tile = [&](int seq, int c) {
+        Tile t;
+        t.tg.s0 = c * C::L;
+        t.tg.Lt = min(C::L, T - t.tg.s0);
+        t.tg.T = T;
+        const size_t p_lo = t.tg.t_lo();                                   // first b element of the tile
+        const size_t j_lo = REV ? p_lo + 1 : p_lo;                         // first J element of the tile
+        t.jcnt = (REV && t.tg.s0 == 0) ? t.tg.Lt - 1 : t.tg.Lt;            // (reverse: J[T] does not exist)
+        t.index = (size_t)seq * w.nch + c;
+        t.Jsrc = a.J + ((size_t)seq * T + j_lo) * NN;
+        t.gbase = ((size_t)seq * T + p_lo) * N;
+        t.bsrc = a.b + t.gbase;
+        t.full = t.tg.Lt == C::L && t.jcnt == C::L;
+        return t;
+    };
+    auto full_off = [&](int u) {        // float offset into sB of ascending-t position u of a full tile
+        const int blk = u / S, within = u - blk * S;
+        return (REV ? CHAINS - 1 - blk : blk) * C::BRUN + within * N;
+    };
+    auto stage_J = [&](const Tile &t) {
+        if (t.full) {
+            constexpr int RUN_PIECES = S * PPE;
+#pragma unroll
+            for (int k = 0; k < C::L * PPE / THREADS; ++k) {
+                const int p = tid + k * THREADS;
+                const int blk = p / RUN_PIECES, within = p - blk * RUN_PIECES;
+                cp_async16(sJ + (REV ? CHAINS - 1 - blk : blk) * C::JRUN + within * 4, t.Jsrc + (size_t)p * 4);
+            }
+        } else {
+            for (int g = tid; g < t.jcnt * PPE; g += THREADS) {
+                const int u = g / PPE, v = g - u * PPE;
+                cp_async16(sJ + t.tg.jmat_off(u) + v * 4, t.Jsrc + (size_t)u * NN + v * 4);
+            }
+        }
+    };
+    auto stage_b = [&](const Tile &t) {
+        if (t.full) {
+#pragma unroll
+            for (int k = 0; k < C::L / THREADS; ++k) {
+                const int u = tid + k * THREADS;
+                cp_async16(sB + full_off(u), t.bsrc + (size_t)u * 4);
+            }
+        } else {
+            for (int u = tid; u < t.tg.Lt; u += THREADS) cp_async16(sB + t.tg.out_off(u, 0), t.bsrc + (size_t)u * 4);
+        }
+    };
+
     if (tid == CLAIMER) {
         int seq = -1, c = -1;
         claim_from(atomicAdd(&a.st->tile_counter, 1u), seq, c);
         s_seq = seq; s_c = c;
     }
     __syncthreads();
+    int seq = s_seq, c = s_c;
+    if (c >= 0) {
+        const Tile t = make_tile(seq, c);
+        stage_J(t);
+        stage_b(t);
+    }
 
-    for (;;) {
-        const int seq = s_seq, c = s_c;
-        if (c < 0) break;
-        TileGeom<N, REV> tg;
-        tg.s0 = c * C::L;
-        tg.Lt = min(C::L, T - tg.s0);
-        tg.T = T;
-        const int Lt = tg.Lt;
-        const size_t p_lo = tg.t_lo();                                  // first b element of the tile
-        const size_t j_lo = REV ? p_lo + 1 : p_lo;                      // first J element of the tile
-        const int jcnt_tile = (REV && tg.s0 == 0) ? Lt - 1 : Lt;        // (reverse: J[T] does not exist)
-        const size_t tile_index = (size_t)seq * w.nch + c;
-        const float *Jt_src = a.J + ((size_t)seq * T + j_lo) * NN;
-        const float *bt_src = a.b + ((size_t)seq * T + p_lo) * N;
-        // a full tile (all runs complete, every J_t present): every chain's run is one contiguous
-        // block of S positions in global memory and offsets follow from the index by constants
-        const bool full_tile = Lt == C::L && jcnt_tile == C::L;
-        auto full_off = [&](int u) {        // float offset into sB of ascending-t position u of a full tile
-            const int blk = u / S, within = u - blk * S;
-            return (REV ? CHAINS - 1 - blk : blk) * C::BRUN + within * N;
-        };
-
-        // ------------------------------------------------ stage the tile
-        if (full_tile) {
-            constexpr int RUN_PIECES = S * PPE;
-#pragma unroll
-            for (int k = 0; k < C::L * PPE / THREADS; ++k) {
-                const int p = tid + k * THREADS;
-                const int blk = p / RUN_PIECES, within = p - blk * RUN_PIECES;
-                cp_async16(sJ + (REV ? CHAINS - 1 - blk : blk) * C::JRUN + within * 4, Jt_src + (size_t)p * 4);
-            }
-#pragma unroll
-            for (int k = 0; k < C::L / THREADS; ++k) {
-                const int u = tid + k * THREADS;
-                cp_async16(sB + full_off(u), bt_src + (size_t)u * 4);
-            }
-        } else {
-            for (int g = tid; g < jcnt_tile * PPE; g += THREADS) {
-                const int u = g / PPE, v = g - u * PPE;
-                cp_async16(sJ + tg.jmat_off(u) + v * 4, Jt_src + (size_t)u * NN + v * 4);
-            }
-            for (int u = tid; u < Lt; u += THREADS) cp_async16(sB + tg.out_off(u, 0), bt_src + (size_t)u * 4);
-        }
+    while (c >= 0) {
+        const Tile t = make_tile(seq, c);
+        const TileGeom<N, REV> &tg = t.tg;
         cp_async_commit();
         cp_async_wait_0();
         __syncthreads();      // tile staged; every thread has read s_seq / s_c
@@ -150,14 +260,20 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
             else ragg_identity<N>(wr);
             ragg_warp_scan<N, WARPS>(wr, wex, lane);
             if (lane == WARPS - 1) {
-                ragg_store<N>(w.aggs + tile_index * AGG, wr);           // tile aggregate
-                __threadfence();
-                st_release_u32(w.flags + tile_index, 1u);
+                // tile aggregate as {value, flag} words: no fence, and one round trip for the reader
+                unsigned long long *dst = reinterpret_cast<unsigned long long *>(w.aggs) + t.index * AGG;
+#pragma unroll
+                for (int i = 0; i < N; ++i) {
+#pragma unroll
+                    for (int j = 0; j < N; ++j)
+                        st_relaxed_u64(dst + i * N + j, LL_FLAG | (unsigned long long)__float_as_uint(wr.A[i][j]));
+                    st_relaxed_u64(dst + N * N + i, LL_FLAG | (unsigned long long)__float_as_uint(wr.be[i]));
+                }
             }
             if (lane < WARPS) ragg_store<N>(wagg + lane * AGG, wex);   // exclusive prefix over warps
         } else if (warp == 1) {
             // the state entering the tile ({value, flag} words written by the sequence's resolver)
-            const unsigned long long *src = w.starts + tile_index * N;
+            const unsigned long long *src = w.starts + t.index * N;
             unsigned spins = 0;
             bool ok = true;
             for (;;) {
@@ -165,7 +281,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
                 if (__all_sync(0xffffffffu, v != 0ull)) {
                     if (lane < N) {
                         ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
-                        st_relaxed_u64(w.starts + tile_index * N + lane, 0ull);     // consumed: cleared for the next launch
+                        st_relaxed_u64(w.starts + t.index * N + lane, 0ull);     // consumed: cleared for the next launch
                     }
                     break;
                 }
@@ -175,6 +291,9 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
         }
         __syncthreads();      // ystart, warp prefixes and s_abort visible
         if (s_abort) break;
+        // the CTA's next tile is claimed only now, when nothing this CTA still has to do depends on
+        // another CTA (a tile claimed earlier would sit unstarted while the sequence's chain waits
+        // for its aggregate); the atomic's latency hides behind the replay
         unsigned next_id = 0;
         if (tid == CLAIMER) next_id = atomicAdd(&a.st->tile_counter, 1u);
 
@@ -205,18 +324,19 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
                 }
             }
         }
-        __syncthreads();      // y complete in shared memory
         if (tid == CLAIMER) {
-            int nseq = -1, nc = -1;
-            claim_from(next_id, nseq, nc);
-            s_seq = nseq; s_c = nc;
+            int ns = -1, nc_ = -1;
+            claim_from(next_id, ns, nc_);
+            s_seq = ns; s_c = nc_;
         }
+        __syncthreads();      // y complete in shared memory; the J buffer is free; next tile known
+        const int nseq = s_seq, nc = s_c;
+        if (nc >= 0) stage_J(make_tile(nseq, nc));      // the next tile's J flies during the output
 
         // ------------------------------------------------ stream y out (+ max |y - yold|)
         {
-            const size_t gbase = ((size_t)seq * T + p_lo) * N;
-            float *yo = a.y + gbase;
-            const float *yold = a.yold ? a.yold + gbase : nullptr;
+            float *yo = a.y + t.gbase;
+            const float *yold = a.yold ? a.yold + t.gbase : nullptr;
             const bool vec = (((uintptr_t)yo & 15) == 0) && (!yold || ((uintptr_t)yold & 15) == 0);
             auto put = [&](int u, int off) {
                 const float4 val = *reinterpret_cast<const float4 *>(sB + off);
@@ -227,21 +347,25 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
                 }
                 reinterpret_cast<float4 *>(yo)[u] = val;
             };
-            if (vec && full_tile) {
+            if (vec && t.full) {
 #pragma unroll
                 for (int k = 0; k < C::L / THREADS; ++k) put(tid + k * THREADS, full_off(tid + k * THREADS));
             } else if (vec) {
-                for (int u = tid; u < Lt; u += THREADS) put(u, tg.out_off(u, 0));
+                for (int u = tid; u < tg.Lt; u += THREADS) put(u, tg.out_off(u, 0));
             } else {
-                for (int g = tid; g < Lt * N; g += THREADS) {
+                for (int g = tid; g < tg.Lt * N; g += THREADS) {
                     const float val = sB[tg.out_off(g / N, g % N)];
                     if (yold) mb = max(mb, absdiff_bits(val, yold[g]));
                     yo[g] = val;
                 }
             }
         }
-        __syncthreads();      // shared memory free; the next tile's id visible
+        __syncthreads();      // the b / y buffer is free
+        if (nc >= 0) stage_b(make_tile(nseq, nc));
+        seq = nseq; c = nc;
     }
+    cp_async_commit();
+    cp_async_wait_0();        // (a drained CTA leaves no copy in flight)
     if (a.yold) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
