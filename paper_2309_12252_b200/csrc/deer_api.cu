@@ -81,7 +81,7 @@ struct ScanWs {
 
 static int num_sms();
 
-static bool onepass_ll_aggs(int n) { return n == 4; }
+static bool onepass_ll_aggs(int n) { return n <= 4; }
 
 static int onepass_tile_len(int n, int B, int T, int *sw)
 {
@@ -112,7 +112,7 @@ static ScanWs carve_scan(Carver &cv, int B, int T, int n)
         w.op.nch = (T + L1 - 1) / L1;
         size_t tiles = (size_t)B * w.op.nch;
         w.op.flags = cv.take<unsigned>(tiles);
-        // (n = 4 publishes its aggregates as 64-bit {value, flag} words)
+        // (n <= 4 publish their aggregates as 64-bit {value, flag} words)
         w.op.aggs = cv.take<float>(tiles * (n * n + n) * (onepass_ll_aggs(n) ? 2 : 1));
         w.op.starts = cv.take<unsigned long long>(tiles * n);
     }

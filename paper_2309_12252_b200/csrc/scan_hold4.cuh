@@ -22,92 +22,6 @@
 
 namespace deer {
 
-// Resolver role with aggregates published as 64-bit {value, flag} words: warp `rw` of `nrw` serves
-// sequences rw, rw + nrw, ...  A visit loads the words of the next WIN tiles of a sequence in one
-// round trip, takes the leading tiles whose words are all present, clears those words for the next
-// launch, and walks them, Y <- A Y + beta, writing the state entering every tile (lane i holds Y[i]).
-template <int N>
-__device__ void resolver_ll_loop(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
-{
-    using C = OnePass<N>;
-    constexpr int AGG = C::AGG, NN = N * N;
-    constexpr int WIN = 16;                         // tiles looked at per visit
-    constexpr int PER = WIN * AGG / 32;             // words per lane
-    static_assert((WIN * AGG) % 32 == 0 && WIN < 32, "window of whole words per lane");
-    float *stage = stage_all + (threadIdx.x >> 5) * 32 * AGG;
-    int nseq = 0;
-    int pos[C::MAX_SEQ_PER_WARP];
-    float yv[C::MAX_SEQ_PER_WARP];              // lane i < N: component i of the sequence's running state
-#pragma unroll
-    for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
-        pos[k] = 0; yv[k] = 0.0f;
-        const int s = rw + k * nrw;
-        if (s < a.B) {
-            nseq = k + 1;
-            if (lane < N && a.y0) yv[k] = a.y0[(size_t)s * N + lane];
-        }
-    }
-    int remaining = nseq;
-    unsigned spins = 0;
-    while (remaining > 0) {
-        bool progressed = false;
-#pragma unroll
-        for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
-            if (k >= nseq) break;
-            const int c0 = pos[k];
-            if (c0 >= w.nch) continue;
-            const int s = rw + k * nrw;
-            unsigned long long *words = reinterpret_cast<unsigned long long *>(w.aggs) + ((size_t)s * w.nch + c0) * AGG;
-            const int nt = min(WIN, w.nch - c0);
-            const int total = nt * AGG;
-            unsigned long long v[PER];
-#pragma unroll
-            for (int u = 0; u < PER; ++u) {
-                const int i = lane + 32 * u;
-                v[u] = (i < total) ? ld_relaxed_u64(words + i) : 0ull;
-            }
-            unsigned missing = ~0u << nt;           // tiles beyond the window or the sequence
-#pragma unroll
-            for (int u = 0; u < PER; ++u) {
-                const int i = lane + 32 * u;
-                if (i < total && (v[u] >> 32) == 0ull) missing |= 1u << (i / AGG);
-            }
-            missing = __reduce_or_sync(0xffffffffu, missing);
-            const int cnt = __ffs(missing) - 1;     // leading tiles with every word present
-            if (cnt == 0) continue;
-            progressed = true;
-#pragma unroll
-            for (int u = 0; u < PER; ++u) {
-                const int i = lane + 32 * u;
-                if (i < cnt * AGG) {
-                    stage[i] = __uint_as_float((unsigned)(v[u] & 0xffffffffull));
-                    st_relaxed_u64(words + i, 0ull);                 // consumed: cleared for the next launch
-                }
-            }
-            __syncwarp();
-            unsigned long long *out = w.starts + ((size_t)s * w.nch + c0) * N;
-            float y = yv[k];
-            for (int q = 0; q < cnt; ++q) {
-                if (lane < N) st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y));
-                const float *ag = stage + q * AGG;
-                float acc = (lane < N) ? ag[NN + lane] : 0.0f;
-#pragma unroll
-                for (int i = 0; i < N; ++i) {
-                    const float yi = __shfl_sync(0xffffffffu, y, i);
-                    if (lane < N) acc = fmaf(ag[lane * N + i], yi, acc);
-                }
-                y = acc;
-            }
-            yv[k] = y;
-            __syncwarp();
-            pos[k] = c0 + cnt;
-            if (pos[k] >= w.nch) --remaining;
-        }
-        if (progressed) spins = 0;
-        else if (!keep_spinning(a.st, spins)) return;
-    }
-}
-
 template <bool REV>
 __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArgs a, OnePassWs w)
 {

@@ -1,5 +1,5 @@
-// Single-pass chunked scan of the linear recurrence for n in {1, 2, 4, 8}:
-// J and b are read from HBM once, y written once.
+// Single-pass chunked scan of the linear recurrence for n in {1, 2} (and the protocol, resolver
+// and helpers shared by the kernels for larger n): J and b are read from HBM once, y written once.
 //
 //   * One persistent kernel.  Every tile of L consecutive positions of one
 //     sequence is visited twice by a worker CTA: an A item (stage the tile,
@@ -24,11 +24,11 @@
 //   * Protocol.  Roles and tile ids are handed out by atomic counters to
 //     running CTAs only, and a tile's B item depends only on A items of lower
 //     ids, which their owners execute immediately after claiming: no
-//     co-residency assumption is needed for progress.  Aggregates are
-//     published with a release flag; entering states travel as 64-bit
-//     {value, flag} words, so reading one needs a single round trip and no
-//     fence.  Every wait is bounded: on expiry the kernel raises FLAG_TIMEOUT
-//     and all CTAs drain.
+//     co-residency assumption is needed for progress.  Aggregates (n <= 4)
+//     and entering states travel as 64-bit {value, flag} words, so reading
+//     one needs a single round trip and no fence (n >= 8 publish their larger
+//     aggregates with a release flag).  Every wait is bounded: on expiry the
+//     kernel raises FLAG_TIMEOUT and all CTAs drain.
 //   * In the B item y overwrites b in shared memory and is streamed out with
 //     coalesced stores fused with the max |y - y_old| reduction.
 //
@@ -70,8 +70,8 @@ template <int N> struct OnePass {
 };
 
 struct OnePassWs {
-    unsigned *flags;              // [B*nch]  1 once the tile aggregate is published
-    float *aggs;                  // [B*nch][n*n+n]
+    unsigned *flags;              // [B*nch]  1 once the tile aggregate is published (n >= 8)
+    float *aggs;                  // [B*nch][n*n+n] floats (n >= 8) or {flag << 32 | float bits} words (n <= 4)
     unsigned long long *starts;   // [B*nch][n]  state entering the tile as {flag << 32 | float bits}
     int nch, Wd, nwin;            // tiles per sequence, tiles per sequence per window, windows
     unsigned total_ids;
@@ -372,28 +372,29 @@ __device__ __forceinline__ bool keep_spinning(StatusBlock *st, unsigned &spins)
 
 constexpr unsigned long long LL_FLAG = 1ull << 32;     // "entering state present" marker
 
-// Resolver role: warp `rw` of `nrw` serves sequences rw, rw + nrw, ...  For each it walks the
-// published tile aggregates in order, Y <- A Y + beta, writing the state entering every tile.
-// The flags of the next window are requested before the current batch is processed, so a batch
-// costs one exposed round trip (the aggregate fetch); Y lives in registers (lane i holds Y[i]).
+// Resolver role with aggregates published as 64-bit {value, flag} words: warp `rw` of `nrw` serves
+// sequences rw, rw + nrw, ...  A visit loads the words of the next WIN tiles of a sequence in one
+// round trip, takes the leading tiles whose words are all present, clears those words for the next
+// launch, and walks them, Y <- A Y + beta, writing the state entering every tile (lane i holds Y[i]).
 template <int N>
-__device__ void resolver_loop(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
+__device__ void resolver_ll_loop(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
 {
     using C = OnePass<N>;
     constexpr int AGG = C::AGG, NN = N * N;
+    constexpr int WIN = 16;                         // tiles looked at per visit
+    constexpr int PER = WIN * AGG / 32;             // words per lane
+    static_assert((WIN * AGG) % 32 == 0 && WIN < 32, "window of whole words per lane");
     float *stage = stage_all + (threadIdx.x >> 5) * 32 * AGG;
     int nseq = 0;
     int pos[C::MAX_SEQ_PER_WARP];
     float yv[C::MAX_SEQ_PER_WARP];              // lane i < N: component i of the sequence's running state
-    unsigned fnext[C::MAX_SEQ_PER_WARP];        // prefetched flag of tile pos + lane
 #pragma unroll
     for (int k = 0; k < C::MAX_SEQ_PER_WARP; ++k) {
-        pos[k] = 0; yv[k] = 0.0f; fnext[k] = 0u;
+        pos[k] = 0; yv[k] = 0.0f;
         const int s = rw + k * nrw;
         if (s < a.B) {
             nseq = k + 1;
             if (lane < N && a.y0) yv[k] = a.y0[(size_t)s * N + lane];
-            if (lane < w.nch) fnext[k] = ld_acquire_u32(w.flags + (size_t)s * w.nch + lane);
         }
     }
     int remaining = nseq;
@@ -406,31 +407,31 @@ __device__ void resolver_loop(const ScanArgs &a, const OnePassWs &w, float *stag
             const int c0 = pos[k];
             if (c0 >= w.nch) continue;
             const int s = rw + k * nrw;
-            const unsigned *flags = w.flags + (size_t)s * w.nch;
-            const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
-            const int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);      // contiguous published aggregates
-            // request the flags of the window that follows (used on the next visit)
-            {
-                const int j = c0 + cnt + lane;
-                fnext[k] = (j < w.nch) ? ld_acquire_u32(flags + j) : 0u;
+            unsigned long long *words = reinterpret_cast<unsigned long long *>(w.aggs) + ((size_t)s * w.nch + c0) * AGG;
+            const int nt = min(WIN, w.nch - c0);
+            const int total = nt * AGG;
+            unsigned long long v[PER];
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int i = lane + 32 * u;
+                v[u] = (i < total) ? ld_relaxed_u64(words + i) : 0ull;
             }
+            unsigned missing = ~0u << nt;           // tiles beyond the window or the sequence
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int i = lane + 32 * u;
+                if (i < total && (v[u] >> 32) == 0ull) missing |= 1u << (i / AGG);
+            }
+            missing = __reduce_or_sync(0xffffffffu, missing);
+            const int cnt = __ffs(missing) - 1;     // leading tiles with every word present
             if (cnt == 0) continue;
             progressed = true;
-            const float *src = w.aggs + ((size_t)s * w.nch + c0) * AGG;
-            {   // all loads of a group are issued before the first store needs its value
-                const int total = cnt * AGG;
-                for (int i0 = 0; i0 < total; i0 += 32 * 8) {
-                    float v[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        v[u] = (i < total) ? __ldcg(src + i) : 0.0f;
-                    }
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        if (i < total) stage[i] = v[u];
-                    }
+            for (int u = 0; u < PER; ++u) {
+                const int i = lane + 32 * u;
+                if (i < cnt * AGG) {
+                    stage[i] = __uint_as_float((unsigned)(v[u] & 0xffffffffull));
+                    st_relaxed_u64(words + i, 0ull);                 // consumed: cleared for the next launch
                 }
             }
             __syncwarp();
@@ -449,7 +450,6 @@ __device__ void resolver_loop(const ScanArgs &a, const OnePassWs &w, float *stag
             }
             yv[k] = y;
             __syncwarp();
-            if (lane < cnt) w.flags[(size_t)s * w.nch + c0 + lane] = 0u;   // consumed: cleared for the next launch
             pos[k] = c0 + cnt;
             if (pos[k] >= w.nch) --remaining;
         }
@@ -490,7 +490,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     fence_proxy_async();
     __syncthreads();
     if (s_role < w.resolvers) {
-        resolver_loop<N>(a, w, sJ, s_role * WARPS + warp, w.resolvers * WARPS, lane);
+        resolver_ll_loop<N>(a, w, sJ, s_role * WARPS + warp, w.resolvers * WARPS, lane);
         __syncthreads();
         if (tid == 0) scan_epilogue(a.st);
         return;
@@ -652,9 +652,15 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
                     ragg_warp_scan<N, WARPS>(wr, wex, lane);
                     if (lane < WARPS) ragg_store<N>(wagg + lane * AGG, wex);   // exclusive prefix over warps
                     if (lane == WARPS - 1) {
-                        ragg_store<N>(w.aggs + tile_index * AGG, wr);           // tile aggregate
-                        __threadfence();
-                        st_release_u32(w.flags + tile_index, 1u);
+                        // tile aggregate as {value, flag} words: no fence, one round trip for the reader
+                        unsigned long long *dst = reinterpret_cast<unsigned long long *>(w.aggs) + tile_index * AGG;
+#pragma unroll
+                        for (int i = 0; i < N; ++i) {
+#pragma unroll
+                            for (int j = 0; j < N; ++j)
+                                st_relaxed_u64(dst + i * N + j, LL_FLAG | (unsigned long long)__float_as_uint(wr.A[i][j]));
+                            st_relaxed_u64(dst + N * N + i, LL_FLAG | (unsigned long long)__float_as_uint(wr.be[i]));
+                        }
                     }
                 }
                 continue;

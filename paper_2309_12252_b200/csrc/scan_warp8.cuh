@@ -139,21 +139,11 @@ __device__ void resolver_loop8(const ScanArgs &a, const OnePassWs &w, float *sta
             if (cnt == 0) continue;
             progressed = true;
             const float *src = w.aggs + ((size_t)s * w.nch + c0) * AGG;
-            {
-                const int total = cnt * AGG;
-                for (int i0 = 0; i0 < total; i0 += 32 * 8) {
-                    float v[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        v[u] = (i < total) ? __ldcg(src + i) : 0.0f;
-                    }
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        if (i < total) stage[i] = v[u];
-                    }
-                }
+            {   // the whole batch in flight at once: asynchronous 16-byte copies straight into the stage
+                const int total4 = cnt * AGG / 4;
+                for (int i = lane; i < total4; i += 32) cp_async16(stage + 4 * i, src + 4 * i);
+                cp_async_commit();
+                cp_async_wait_0();
             }
             __syncwarp();
             unsigned long long *out = w.starts + ((size_t)s * w.nch + c0) * N;
