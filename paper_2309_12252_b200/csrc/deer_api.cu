@@ -612,8 +612,6 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     int rc = check_ws(ws, ws_bytes, w.bytes);
     if (rc != DEER_OK) return rc;
     const size_t N = (size_t)B * T;
-    if (!(flags & DEER_FLAG_WARM_START))
-        DEER_CHECK_CUDA(cudaMemsetAsync(y, 0, N * n * sizeof(float), st), "memset y");
     const bool fused_proj = cell_projects(n, m) && ((((uintptr_t)y | (uintptr_t)y0) & 15) == 0);
 
     ScanArgs a{};
@@ -632,10 +630,24 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
         init.max_iter = max_iter;
         init.tol = tol;
         init.trace = w.trace;
-        DEER_CHECK_CUDA(cudaMemcpyAsync(w.st, &init, sizeof(init), cudaMemcpyHostToDevice, st), "init status");
+        // one launch: status block, zero initial guess, cleared words of the single-pass scan
+        EvalBeginArgs e{};
+        if (!(flags & DEER_FLAG_WARM_START)) { e.y = y; e.ny = N * n; }
+        if (single) {
+            const OnePassWs &op = w.scan.op;
+            const size_t tiles = (size_t)B * op.nch;
+            e.flags = op.flags; e.nflags = tiles;
+            e.starts = op.starts; e.nstarts = tiles * (size_t)n;
+            if (onepass_ll_aggs(n)) { e.agg_words = (unsigned long long *)op.aggs; e.nagg_words = tiles * (size_t)(n * n + n); }
+        }
+        const size_t words = e.ny / 4 + e.nflags + e.nstarts + e.nagg_words;
+        unsigned blocks = (unsigned)((words + 1023) / 1024);
+        const unsigned cap = 4u * (unsigned)num_sms();
+        if (blocks > cap) blocks = cap;
+        if (blocks < 1u) blocks = 1u;
+        DEER_KERNEL("eval_begin_kernel", st, eval_begin_kernel<<<blocks, 256, 0, st>>>(w.st, init, e));
     }
     if (!fused_proj && (rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
-    if (single && (rc = scan_prep(a, w.scan.op, st)) != DEER_OK) return rc;
 
     // Newton loop (App. B.1): bodies are enqueued ahead of the convergence test -- the decision at
     // the end of each body is taken on the device, and the kernels of bodies past the end return

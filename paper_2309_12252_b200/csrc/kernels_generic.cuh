@@ -314,6 +314,35 @@ __global__ void scan_prep_kernel(StatusBlock *st, unsigned *flags, size_t nflags
     if (i0 == 0) { st->tile_counter = 0u; st->role_counter = 0u; st->exit_counter = 0u; }
 }
 
+// Everything an evaluation needs before its first body, in one launch: the status block (loop
+// control state, passed by value), the zero initial guess, and the cleared exchange words and
+// counters of the single-pass scan.
+struct EvalBeginArgs {
+    float *y; size_t ny;                         // initial guess to zero (nullptr: warm start)
+    unsigned *flags; size_t nflags;              // single-pass scan words (nullptr / 0 when not used)
+    unsigned long long *starts; size_t nstarts;
+    unsigned long long *agg_words; size_t nagg_words;
+};
+__global__ void eval_begin_kernel(StatusBlock *st, StatusBlock init, EvalBeginArgs e)
+{
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i0 == 0) *st = init;
+    if (e.y) {
+        if (((uintptr_t)e.y & 15) == 0) {
+            float4 *y4 = reinterpret_cast<float4 *>(e.y);
+            const size_t n4 = e.ny / 4;
+            for (size_t i = i0; i < n4; i += stride) y4[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            for (size_t i = 4 * n4 + i0; i < e.ny; i += stride) e.y[i] = 0.0f;
+        } else {
+            for (size_t i = i0; i < e.ny; i += stride) e.y[i] = 0.0f;
+        }
+    }
+    for (size_t i = i0; i < e.nflags; i += stride) e.flags[i] = 0u;
+    for (size_t i = i0; i < e.nstarts; i += stride) e.starts[i] = 0ull;
+    for (size_t i = i0; i < e.nagg_words; i += stride) e.agg_words[i] = 0ull;
+}
+
 // Loop control as a launch of its own (used when a body's scan ran on the generic kernels).
 __global__ void newton_control_kernel(StatusBlock *st, float tol, int max_iter, float *trace)
 {
