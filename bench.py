@@ -341,8 +341,8 @@ def main():
     ap.add_argument("--m", type=int, default=0)
     ap.add_argument("--vjp", type=int, default=0)
     ap.add_argument("--n", type=int, default=8)
-    ap.add_argument("--B", type=int, default=16)
-    ap.add_argument("--T", type=int, default=1_000_000)
+    ap.add_argument("--B", type=int, default=None, help="default 16 (classifier mode: 32, config 4)")
+    ap.add_argument("--T", type=int, default=None, help="default 1,000,000 (classifier mode: 17,984, config 4)")
     ap.add_argument("--reverse", type=int, default=0)
     ap.add_argument("--flags", type=int, default=0)
     ap.add_argument("--gpus", type=int, default=1)
@@ -352,6 +352,10 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-scan-hbm", action="store_true", help="skip the HBM-sized stand-alone scan measurement")
     args = ap.parse_args()
+    if args.B is None:
+        args.B = 32 if args.mode == "classifier" else 16
+    if args.T is None:
+        args.T = 17_984 if args.mode == "classifier" else 1_000_000
     if args.impl == "reference":
         run_reference(args)
         return
