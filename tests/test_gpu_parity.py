@@ -38,6 +38,9 @@ SCAN_CASES = [  # (n, B, T)
     (5, 2, 130), (8, 2, 1), (8, 3, 2), (8, 16, 1111), (8, 1, 5000), (16, 3, 515), (32, 2, 300),
     (64, 2, 70), (7, 1, 63), (1, 3, 20001), (1, 1, 40000), (2, 2, 6001), (2, 3, 1001), (4, 1, 10000),
     (8, 2, 193), (8, 2, 192), (8, 5, 191), (4, 3, 769),
+    # more sequences than resolver warps (several sequences per warp), and sequences with more tiles than
+    # one resolver visit looks at
+    (4, 40, 1500), (2, 70, 5000), (1, 70, 15000), (8, 40, 700), (4, 2, 30001), (2, 1, 50000), (1, 1, 150000),
 ]
 
 
