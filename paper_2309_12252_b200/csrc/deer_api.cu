@@ -214,7 +214,7 @@ static int launch_hold4(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = OnePass<4>;
     static int occ[MAX_DEVICES] = {0};
-    const PassCfg c{"scan_hold4_kernel", C::THREADS, C::SMEM, C::WARPS, C::MAX_SEQ_PER_WARP, 32, 8};
+    const PassCfg c{"scan_hold4_kernel", C::THREADS, Hold4::SMEM, C::WARPS, C::MAX_SEQ_PER_WARP, 32, 8};
     return launch_single_pass(scan_hold4_kernel<REV>, occ, c, a, w, prep, st);
 }
 

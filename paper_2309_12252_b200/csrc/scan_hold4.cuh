@@ -5,25 +5,34 @@
 // with both directions of the exchange as 64-bit {value, flag} words (one round trip, no fence),
 // and a worker CTA holds ONE tile at a time and visits it twice back to back:
 //
-//   stage the tile (per-thread 16-byte cp.async into run-padded shared memory)
+//   stage the tile's J (per-thread 16-byte cp.async into run-padded shared memory); each thread
+//   reads the b of its own chain straight from global memory into registers meanwhile
 //   A: every thread folds its chain of S positions into (A, beta) in registers; a warp-shuffle
 //      scan gives each thread its chain's exclusive prefix inside the warp, which STAYS IN
 //      REGISTERS; warp 0 combines the warp aggregates and publishes the tile aggregate
 //   warp 1 polls for the state entering the tile; once it is there the last thread claims the
 //   CTA's next tile (the atomic's latency hides behind the replay)
-//   B: every thread replays its chain from (warp prefix, chain prefix)(entering state); y
-//      overwrites b in shared memory and is streamed out with the max |y - y_old| reduction,
-//      while the next tile's J is already being copied into the freed J buffer
+//   B: every thread replays its chain from (warp prefix, chain prefix)(entering state); y_t goes
+//      into the part of the chain's J run that the replay has already consumed and is streamed
+//      out from there, coalesced, with the max |y - y_old| reduction
 //
 // The tile is read from HBM once and never staged twice; five CTA barriers per tile.  Shared
-// memory per CTA is the tile plus a few hundred bytes, so four CTAs share an SM.
+// memory per CTA is the tile's J plus a few hundred bytes (43 KB), so five CTAs share an SM.
 #pragma once
 #include "scan_onepass.cuh"
 
 namespace deer {
 
+// shared memory of a worker CTA: the tile's J, the warp prefixes and aggregates, the entering state
+struct Hold4 {
+    using C = OnePass<4>;
+    static constexpr int SM_FLOATS = C::JBUF + C::PEND + C::WARPS * 2 * C::AGG + 4 + 4;
+    static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
+    static_assert(32 * C::AGG <= C::JBUF / C::WARPS, "resolver staging must fit the tile buffer");
+};
+
 template <bool REV>
-__global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArgs a, OnePassWs w)
+__global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(ScanArgs a, OnePassWs w)
 {
     constexpr int N = 4, NN = 16;
     using C = OnePass<N>;
@@ -35,8 +44,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
 
     extern __shared__ __align__(16) float smem_raw[];
     float *sJ = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
-    float *sB = sJ + C::JBUF;
-    float *wagg = sB + C::BBUF;                     // exclusive warp prefixes
+    float *wagg = sJ + C::JBUF;                     // exclusive warp prefixes
     float *tmp = wagg + C::PEND;                    // warp aggregates
     float *ystart = tmp + WARPS * 2 * AGG;
     __shared__ int s_seq, s_c, s_abort, s_role;
@@ -98,9 +106,18 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
         t.full = t.tg.Lt == C::L && t.jcnt == C::L;
         return t;
     };
-    auto full_off = [&](int u) {        // float offset into sB of ascending-t position u of a full tile
+    // float offset inside a chain's J run of the y of local index li (ascending t within the run)
+    // when the run holds cnt positions: always inside matrices the replay has consumed by then
+    // (forward: the run's first floats; reverse: its last ones, as the replay walks down the run)
+    auto y_slot = [](int cnt, int li) { return REV ? 12 * cnt + 4 * li : 4 * li; };
+    auto full_off = [&](int u) {        // float offset into sJ of the y of ascending-t position u of a full tile
         const int blk = u / S, within = u - blk * S;
-        return (REV ? CHAINS - 1 - blk : blk) * C::BRUN + within * N;
+        return (REV ? CHAINS - 1 - blk : blk) * C::JRUN + (REV ? 12 * S : 0) + 4 * within;
+    };
+    auto any_off = [&](const TileGeom<N, REV> &tg, int u) {     // the same for any tile
+        int r, li;
+        tg.locate(u, r, li);
+        return r * C::JRUN + y_slot(tg.run_cnt(r), li);
     };
     auto stage_J = [&](const Tile &t) {
         if (t.full) {
@@ -117,17 +134,32 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
                 cp_async16(sJ + t.tg.jmat_off(u) + v * 4, t.Jsrc + (size_t)u * NN + v * 4);
             }
         }
+        cp_async_commit();
     };
-    auto stage_b = [&](const Tile &t) {
-        if (t.full) {
+    // b of this thread's chain by scan step q (scan offset chain*S + q of the tile <-> ascending-t
+    // index chain*S + q forward, Lt - 1 - (chain*S + q) reverse); zeros beyond the run
+    auto load_b = [&](const Tile &t, int cnt, float4 (&bs)[S]) {
+        const float4 *src = reinterpret_cast<const float4 *>(t.bsrc);
 #pragma unroll
-            for (int k = 0; k < C::L / THREADS; ++k) {
-                const int u = tid + k * THREADS;
-                cp_async16(sB + full_off(u), t.bsrc + (size_t)u * 4);
-            }
-        } else {
-            for (int u = tid; u < t.tg.Lt; u += THREADS) cp_async16(sB + t.tg.out_off(u, 0), t.bsrc + (size_t)u * 4);
+        for (int q = 0; q < S; ++q) {
+            const int u = REV ? t.tg.Lt - 1 - (S * chain + q) : S * chain + q;
+            bs[q] = (q < cnt) ? __ldg(src + u) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         }
+    };
+    // one step of the chain from the staged tile: M = J (forward) or J^T (reverse; identity at scan position 0)
+    auto load_M = [&](const TileGeom<N, REV> &tg, int q, int cnt, float (&M)[N][N]) {
+        const float *Je = sJ + tg.j_off(chain, q, cnt);
+        float R[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 f = reinterpret_cast<const float4 *>(Je)[i];
+            R[i][0] = f.x; R[i][1] = f.y; R[i][2] = f.z; R[i][3] = f.w;
+        }
+        const bool ident = REV && (tg.s0 + chain * S + q == 0);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) M[i][k] = ident ? ((i == k) ? 1.0f : 0.0f) : (REV ? R[k][i] : R[i][k]);
     };
 
     if (tid == CLAIMER) {
@@ -137,21 +169,17 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
     }
     __syncthreads();
     int seq = s_seq, c = s_c;
-    if (c >= 0) {
-        const Tile t = make_tile(seq, c);
-        stage_J(t);
-        stage_b(t);
-    }
-
     while (c >= 0) {
         const Tile t = make_tile(seq, c);
         const TileGeom<N, REV> &tg = t.tg;
-        cp_async_commit();
+        const int cnt = tg.run_cnt(chain);
+        stage_J(t);
+        float4 bs[S];
+        load_b(t, cnt, bs);   // in flight together with the J copies
         cp_async_wait_0();
         __syncthreads();      // tile staged; every thread has read s_seq / s_c
 
         // ------------------------------------------------ A: chain aggregates, prefixes, publish
-        const int cnt = tg.run_cnt(chain);
         RegAgg<N> held;       // this chain's exclusive prefix inside the warp
         {
             RegAgg<N> r;
@@ -159,8 +187,9 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
 #pragma unroll
             for (int q = 0; q < S; ++q) {
                 if (q < cnt) {
-                    float M[N][N], bq[N];
-                    load_chain_step<N, REV>(sJ, sB, tg, chain, q, cnt, M, bq);
+                    float M[N][N];
+                    load_M(tg, q, cnt, M);
+                    const float bq[N] = {bs[q].x, bs[q].y, bs[q].z, bs[q].w};
                     ragg_push<N>(r, M, bq);
                 }
             }
@@ -223,8 +252,9 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
 #pragma unroll
             for (int q = 0; q < S; ++q) {
                 if (q < cnt) {
-                    float M[N][N], bq[N];
-                    load_chain_step<N, REV>(sJ, sB, tg, chain, q, cnt, M, bq);
+                    float M[N][N];
+                    load_M(tg, q, cnt, M);
+                    const float bq[N] = {bs[q].x, bs[q].y, bs[q].z, bs[q].w};
                     float yn[N];
 #pragma unroll
                     for (int i = 0; i < N; ++i) {
@@ -234,7 +264,9 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
                     }
 #pragma unroll
                     for (int i = 0; i < N; ++i) y[i] = yn[i];
-                    *reinterpret_cast<float4 *>(sB + tg.b_off(chain, q, cnt)) = make_float4(yn[0], yn[1], yn[2], yn[3]);
+                    // into the part of the run that is already consumed (local index of step q: q forward, cnt-1-q reverse)
+                    *reinterpret_cast<float4 *>(sJ + chain * C::JRUN + y_slot(cnt, REV ? cnt - 1 - q : q)) =
+                        make_float4(yn[0], yn[1], yn[2], yn[3]);
                 }
             }
         }
@@ -243,9 +275,8 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
             claim_from(next_id, ns, nc_);
             s_seq = ns; s_c = nc_;
         }
-        __syncthreads();      // y complete in shared memory; the J buffer is free; next tile known
+        __syncthreads();      // y complete in shared memory; next tile known
         const int nseq = s_seq, nc = s_c;
-        if (nc >= 0) stage_J(make_tile(nseq, nc));      // the next tile's J flies during the output
 
         // ------------------------------------------------ stream y out (+ max |y - yold|)
         {
@@ -253,7 +284,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
             const float *yold = a.yold ? a.yold + t.gbase : nullptr;
             const bool vec = (((uintptr_t)yo & 15) == 0) && (!yold || ((uintptr_t)yold & 15) == 0);
             auto put = [&](int u, int off) {
-                const float4 val = *reinterpret_cast<const float4 *>(sB + off);
+                const float4 val = *reinterpret_cast<const float4 *>(sJ + off);
                 if (yold) {
                     const float4 o = __ldg(reinterpret_cast<const float4 *>(yold) + u);
                     mb = max(mb, absdiff_bits(val.x, o.x)); mb = max(mb, absdiff_bits(val.y, o.y));
@@ -265,21 +296,18 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS) scan_hold4_kernel(ScanArg
 #pragma unroll
                 for (int k = 0; k < C::L / THREADS; ++k) put(tid + k * THREADS, full_off(tid + k * THREADS));
             } else if (vec) {
-                for (int u = tid; u < tg.Lt; u += THREADS) put(u, tg.out_off(u, 0));
+                for (int u = tid; u < tg.Lt; u += THREADS) put(u, any_off(tg, u));
             } else {
                 for (int g = tid; g < tg.Lt * N; g += THREADS) {
-                    const float val = sB[tg.out_off(g / N, g % N)];
+                    const float val = sJ[any_off(tg, g / N) + g % N];
                     if (yold) mb = max(mb, absdiff_bits(val, yold[g]));
                     yo[g] = val;
                 }
             }
         }
-        __syncthreads();      // the b / y buffer is free
-        if (nc >= 0) stage_b(make_tile(nseq, nc));
+        __syncthreads();      // the tile buffer is free
         seq = nseq; c = nc;
     }
-    cp_async_commit();
-    cp_async_wait_0();        // (a drained CTA leaves no copy in flight)
     if (a.yold) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
