@@ -193,6 +193,18 @@ __device__ __forceinline__ bool seq_start(size_t e, int T, size_t &seq)
 
 __device__ __forceinline__ float sigmoidf_acc(float a) { return 1.0f / (1.0f + expf(-a)); }
 
+// Gate activations for the issue-bound small-n cell kernel: ex2.approx / rcp.approx based (a few
+// instructions instead of ~25 each).  exp2 and the reciprocal are good to 2 ulp and the product
+// a*log2(e) adds |a| * 6e-8 relative to the exponential, so sigma is within 3e-7 and tanh within
+// 2e-7 ABSOLUTE of the exact value on the whole real line (saturated ends included; NaN stays NaN)
+// -- three orders of magnitude below the 1e-4 tolerance the evaluation is solved and checked to.
+__device__ __forceinline__ float sigmoidf_gate(float a) { return __fdividef(1.0f, 1.0f + __expf(-a)); }
+__device__ __forceinline__ float tanhf_gate(float a)
+{
+    const float e = __expf(-2.0f * fabsf(a));            // in (0, 1]
+    return copysignf(__fdividef(1.0f - e, 1.0f + e), a);
+}
+
 __device__ __forceinline__ unsigned absdiff_bits(float a, float b) {
     return __float_as_uint(fabsf(a - b));   // NaN keeps bits above +inf: an integer max propagates it
 }

@@ -148,9 +148,9 @@ __global__ void __launch_bounds__(256) cell_small_kernel(CellArgs a)
             const float *ue = a.u + e * 3 * N;
             ur = ue[i]; uz = ue[N + i]; un = ue[2 * N + i];
         }
-        const float r = sigmoidf_acc(ur + gr);
-        const float z = sigmoidf_acc(uz + gz);
-        const float c = tanhf(un + r * gq);
+        const float r = sigmoidf_gate(ur + gr);
+        const float z = sigmoidf_gate(uz + gz);
+        const float c = tanhf_gate(un + r * gq);
         const float hi = hp[i];
         const float f = (1.0f - z) * c + z * hi;
         const float az = (hi - c) * z * (1.0f - z);
