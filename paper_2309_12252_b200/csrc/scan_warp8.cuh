@@ -180,7 +180,6 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
     using C = Warp8;
     constexpr int N = C::N, NN = C::NN, AGG = C::AGG, WARPS = C::WARPS, GRP = C::GRP, Q = C::Q;
     pdl_prologue();
-    if (loop_ended(a.st)) return;
     const int SW = w.sw, L = WARPS * SW;
 
     extern __shared__ __align__(16) float smem_raw[];
@@ -188,17 +187,22 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
     float *pend = sm;                          // Q x warp aggregates (A row-major, then beta)
     float *wstart = pend + Q * C::PEND;        // WARPS x N states entering each warp chain
     float *ystart = wstart + WARPS * N;
-    __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role;
+    __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role, s_done;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;     // fragment coordinates
     const int T = a.T;
 
+    // the role ticket and the loop-ended word travel together (one round trip; a ticket taken by a
+    // launch that then returns is harmless: the counters are rewound before the next evaluation)
     if (tid == 0) {
+        const unsigned ticket = atomicAdd(&a.st->role_counter, 1u);
+        s_done = loop_ended(a.st) ? 1 : 0;
         s_abort = 0;
-        s_role = (int)atomicAdd(&a.st->role_counter, 1u);
+        s_role = (int)ticket;
     }
     __syncthreads();
+    if (s_done) return;
     if (s_role < w.resolvers) {
         if (warp < C::RES_WARPS)
             resolver_loop8(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
@@ -218,6 +222,10 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
     };
     int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
     bool exhausted = false;
+    // tile ids: a worker's first id is its own index (no second atomic before the first tile), later
+    // ones come from the counter, offset by the number of workers
+    const unsigned workers = gridDim.x - (unsigned)w.resolvers;
+    bool first_claim = true;
 
     for (;;) {
         __syncthreads();
@@ -231,7 +239,10 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
             }
             if (!want_b && !exhausted) {
                 for (;;) {
-                    const unsigned id = atomicAdd(&a.st->tile_counter, 1u);
+                    unsigned id;
+                    if (first_claim) { id = (unsigned)(s_role - w.resolvers); first_claim = false; }
+                    else if (workers >= w.total_ids) { c = -1; break; }       // every id was a first id
+                    else id = workers + atomicAdd(&a.st->tile_counter, 1u);
                     if (id >= w.total_ids) { c = -1; break; }
                     decode(id, seq, c);
                     if (c >= 0) break;
