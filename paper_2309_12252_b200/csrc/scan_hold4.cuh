@@ -47,19 +47,23 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
     float *wagg = sJ + C::JBUF;                     // exclusive warp prefixes
     float *tmp = wagg + C::PEND;                    // warp aggregates
     float *ystart = tmp + WARPS * 2 * AGG;
-    __shared__ int s_seq, s_c, s_abort, s_role;
+    __shared__ int s_seq, s_c, s_abort, s_role, s_done;
 
     pdl_prologue();
-    if (loop_ended(a.st)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chain = tid;
     const int T = a.T;
 
+    // the role ticket and the loop-ended word travel together (one round trip; a ticket taken by a
+    // launch that then returns is harmless: the counters are rewound before the next evaluation)
     if (tid == 0) {
+        const unsigned ticket = atomicAdd(&a.st->role_counter, 1u);
+        s_done = loop_ended(a.st) ? 1 : 0;
         s_abort = 0;
-        s_role = (int)atomicAdd(&a.st->role_counter, 1u);
+        s_role = (int)ticket;
     }
     __syncthreads();
+    if (s_done) return;
     if (s_role < w.resolvers) {
         resolver_ll_loop<N>(a, w, sJ, s_role * WARPS + warp, w.resolvers * WARPS, lane);
         __syncthreads();
@@ -68,8 +72,10 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
     }
     unsigned mb = 0;          // running max |y - yold| bits of this thread
 
-    // claim: ids come from the launch-wide counter; id -> (seq, tile), padding ids of the last
-    // window are skipped; c < 0 when no tile is left
+    // claim: a worker's first id is its own index (no second atomic before the first tile), later
+    // ones come from the launch-wide counter offset by the number of workers; id -> (seq, tile),
+    // padding ids of the last window are skipped; c < 0 when no tile is left
+    const unsigned workers = gridDim.x - (unsigned)w.resolvers;
     auto claim_from = [&](unsigned id, int &seq, int &c) {
         for (;;) {
             if (id >= w.total_ids) { c = -1; return; }
@@ -79,7 +85,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
             const unsigned win = ws_ / (unsigned)a.B;
             c = (int)(win * (unsigned)w.Wd + j);
             if (c < w.nch) return;
-            id = atomicAdd(&a.st->tile_counter, 1u);
+            id = workers + atomicAdd(&a.st->tile_counter, 1u);
         }
     };
     // geometry and sources of one tile
@@ -164,7 +170,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
 
     if (tid == CLAIMER) {
         int seq = -1, c = -1;
-        claim_from(atomicAdd(&a.st->tile_counter, 1u), seq, c);
+        claim_from((unsigned)(s_role - w.resolvers), seq, c);
         s_seq = seq; s_c = c;
     }
     __syncthreads();
@@ -238,7 +244,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
         // another CTA (a tile claimed earlier would sit unstarted while the sequence's chain waits
         // for its aggregate); the atomic's latency hides behind the replay
         unsigned next_id = 0;
-        if (tid == CLAIMER) next_id = atomicAdd(&a.st->tile_counter, 1u);
+        if (tid == CLAIMER) next_id = workers >= w.total_ids ? w.total_ids : workers + atomicAdd(&a.st->tile_counter, 1u);
 
         // ------------------------------------------------ B: replay from the entering state
         {

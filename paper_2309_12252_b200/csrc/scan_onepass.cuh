@@ -474,21 +474,25 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     float *tmp = pend + Q * PEND;
     float *ystart = tmp + WARPS * 2 * AGG;
     uint64_t *bar = (uint64_t *)(((uintptr_t)(ystart + N) + 15) & ~(uintptr_t)15);
-    __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role;
+    __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role, s_done;
 
     pdl_prologue();
-    if (loop_ended(a.st)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chain = tid;
     const int T = a.T;
 
+    // the role ticket and the loop-ended word travel together (one round trip; a ticket taken by a
+    // launch that then returns is harmless: the counters are rewound before the next evaluation)
     if (tid == 0) {
+        const unsigned ticket = atomicAdd(&a.st->role_counter, 1u);
+        s_done = loop_ended(a.st) ? 1 : 0;
         mbar_init(bar, 1);
         s_abort = 0;
-        s_role = (int)atomicAdd(&a.st->role_counter, 1u);
+        s_role = (int)ticket;
     }
     fence_proxy_async();
     __syncthreads();
+    if (s_done) return;
     if (s_role < w.resolvers) {
         resolver_ll_loop<N>(a, w, sJ, s_role * WARPS + warp, w.resolvers * WARPS, lane);
         __syncthreads();
@@ -511,6 +515,10 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
     // pending queue (thread 0 only): tiles whose A item has run
     int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
     bool exhausted = false;
+    // tile ids: a worker's first id is its own index (no second atomic before the first tile), later
+    // ones come from the counter, offset by the number of workers
+    const unsigned workers = gridDim.x - (unsigned)w.resolvers;
+    bool first_claim = true;
 
     for (;;) {
         __syncthreads();      // previous item done with shared memory and with the s_* words
@@ -526,7 +534,10 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanA
             }
             if (!want_b && !exhausted) {
                 for (;;) {
-                    const unsigned id = atomicAdd(&a.st->tile_counter, 1u);
+                    unsigned id;
+                    if (first_claim) { id = (unsigned)(s_role - w.resolvers); first_claim = false; }
+                    else if (workers >= w.total_ids) { c = -1; break; }       // every id was a first id
+                    else id = workers + atomicAdd(&a.st->tile_counter, 1u);
                     if (id >= w.total_ids) { c = -1; break; }
                     decode(id, seq, c);
                     if (c >= 0) break;
