@@ -291,6 +291,7 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
             // ---------------------------------------------- A item: [X; beta^T] in the accumulator fragment
             float acc[4] = {(g == 2 * t) ? 1.0f : 0.0f, (g == 2 * t + 1) ? 1.0f : 0.0f, 0.0f, 0.0f};
             const float2 *bp2 = reinterpret_cast<const float2 *>(bseq + tb * N) + t;
+            const float *bch = bseq + tb * N;
             // whole groups: loads with constant offsets from one pointer per group, no per-position tests
             int q0 = 0;
             if (REV && sbase == 0 && cnt > 0) {                 // scan position 0 of the reverse scan: identity
@@ -310,7 +311,8 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
                         if (!REV) prefetch_l1(jq + (GRP + u) * 32);
                         else { prefetch_l1(jr - (GRP + u) * NN); prefetch_l1(jr - (GRP + u) * NN + N); }
                     }
-                    if (g == 0) prefetch_l1(REV ? bq - (2 * GRP - 1) * 4 : bq + GRP * 4);
+                    // the next group's b: 256 contiguous bytes, up to three lines
+                    if (lane < 3) prefetch_l1(bch + (REV ? -(q0 + 2 * GRP - 1) * N : (q0 + GRP) * N) + min(lane * 32, GRP * N - 1));
                 }
 #pragma unroll
                 for (int u = 0; u < GRP; ++u) {
@@ -425,7 +427,10 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
                         if (!REV) prefetch_l1(jq + (GRP + u) * 32);
                         else { prefetch_l1(jr - (GRP + u) * NN); prefetch_l1(jr - (GRP + u) * NN + N); }
                     }
-                    if (t == 0) prefetch_l1(bpg + (REV ? off0 - (2 * GRP - 1) * N : off0 + GRP * N));
+                    // the next group's b and y_old: 256 contiguous bytes each, up to three lines
+                    const int nx = (REV ? -(q0 + 2 * GRP - 1) * N : (q0 + GRP) * N) + min((lane & 3) * 32, GRP * N - 1);
+                    if (lane < 3) prefetch_l1(bpg - g + nx);
+                    else if (yop && lane >= 4 && lane < 7) prefetch_l1(yop - g + nx);
                 }
                 const int offt = off0 + (REV ? -t * N : t * N);               // this lane's first position of the group
                 float yo[GRP / 4];
