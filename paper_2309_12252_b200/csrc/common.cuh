@@ -81,8 +81,9 @@ struct StatusBlock {
     unsigned flags;      // FLAG_* bits raised by kernels
     int iters;           // bodies executed so far (device-side loop control)
     int done;            // 1 once the loop condition failed
-    unsigned tile_counter;  // dynamic tile id for the single-pass scan
-    unsigned role_counter;  // role tickets of the single-pass scan (first ones: resolvers)
+    unsigned tile_counter;  // dynamic tile id for the single-pass scan (n >= 16 kernels)
+    unsigned role_counter;  // role tickets of the single-pass scan (first ones: resolvers); the n <= 8
+                            // kernels take their tile ids from it too (ticket - resolvers)
     unsigned err_last_bits; // err of the last executed body
     unsigned exit_counter;  // CTAs of the running single-pass scan that have finished
     int ctl_mode;        // 1: the last CTA of a single-pass scan takes the Newton loop decision

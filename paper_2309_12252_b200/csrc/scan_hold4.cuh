@@ -72,10 +72,11 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
     }
     unsigned mb = 0;          // running max |y - yold| bits of this thread
 
-    // claim: a worker's first id is its own index (no second atomic before the first tile), later
-    // ones come from the launch-wide counter offset by the number of workers; id -> (seq, tile),
-    // padding ids of the last window are skipped; c < 0 when no tile is left
-    const unsigned workers = gridDim.x - (unsigned)w.resolvers;
+    // claim: tile ids come from the same counter as the role tickets (ticket - resolvers), so a
+    // worker's ticket is its first tile id (no second atomic before the first tile) and ids are still
+    // handed out in order to running CTAs only; id -> (seq, tile), padding ids of the last window are
+    // skipped; c < 0 when no tile is left
+    auto next_ticket = [&]() { return atomicAdd(&a.st->role_counter, 1u) - (unsigned)w.resolvers; };
     auto claim_from = [&](unsigned id, int &seq, int &c) {
         for (;;) {
             if (id >= w.total_ids) { c = -1; return; }
@@ -85,7 +86,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
             const unsigned win = ws_ / (unsigned)a.B;
             c = (int)(win * (unsigned)w.Wd + j);
             if (c < w.nch) return;
-            id = workers + atomicAdd(&a.st->tile_counter, 1u);
+            id = next_ticket();
         }
     };
     // geometry and sources of one tile
@@ -244,7 +245,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
         // another CTA (a tile claimed earlier would sit unstarted while the sequence's chain waits
         // for its aggregate); the atomic's latency hides behind the replay
         unsigned next_id = 0;
-        if (tid == CLAIMER) next_id = workers >= w.total_ids ? w.total_ids : workers + atomicAdd(&a.st->tile_counter, 1u);
+        if (tid == CLAIMER) next_id = next_ticket();
 
         // ------------------------------------------------ B: replay from the entering state
         {

@@ -222,9 +222,9 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
     };
     int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
     bool exhausted = false;
-    // tile ids: a worker's first id is its own index (no second atomic before the first tile), later
-    // ones come from the counter, offset by the number of workers
-    const unsigned workers = gridDim.x - (unsigned)w.resolvers;
+    // tile ids come from the same counter as the role tickets (ticket - resolvers): a worker's ticket
+    // is its first tile id (no second atomic before the first tile), and ids are still handed out in
+    // order to running CTAs only
     bool first_claim = true;
 
     for (;;) {
@@ -241,8 +241,7 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
                 for (;;) {
                     unsigned id;
                     if (first_claim) { id = (unsigned)(s_role - w.resolvers); first_claim = false; }
-                    else if (workers >= w.total_ids) { c = -1; break; }       // every id was a first id
-                    else id = workers + atomicAdd(&a.st->tile_counter, 1u);
+                    else id = atomicAdd(&a.st->role_counter, 1u) - (unsigned)w.resolvers;
                     if (id >= w.total_ids) { c = -1; break; }
                     decode(id, seq, c);
                     if (c >= 0) break;
