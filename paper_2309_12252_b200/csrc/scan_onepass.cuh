@@ -459,7 +459,7 @@ __device__ void resolver_ll_loop(const ScanArgs &a, const OnePassWs &w, float *s
 }
 
 template <int N, bool REV>
-__global__ void __launch_bounds__(OnePass<N>::THREADS) scan_onepass_kernel(ScanArgs a, OnePassWs w)
+__global__ void __launch_bounds__(OnePass<N>::THREADS, 3) scan_onepass_kernel(ScanArgs a, OnePassWs w)
 {
     using C = OnePass<N>;
     constexpr int S = C::S, CHAINS = C::CHAINS;
