@@ -740,6 +740,8 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
         int outs = n3 * (wa.K + 1);
         if (n3 % 16 == 0 && n3 <= 192 && wa.K <= 64) {
             DEER_KERNEL("wgrad_mma_kernel", st, wgrad_mma_kernel<<<P, 32 * (n3 / 16), 0, st>>>(wa));
+        } else if (n3 <= 32 && wa.K <= 8) {
+            DEER_KERNEL("wgrad_small_kernel", st, wgrad_small_kernel<<<P, 256, 0, st>>>(wa));
         } else {
             int tile = 32;
             while (tile > 1 && sizeof(float) * tile * (size_t)(n3 + wa.K + 1) > 160 * 1024) tile >>= 1;
@@ -749,7 +751,7 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
             dim3 grid(P, (outs + 255) / 256);
             DEER_KERNEL("wgrad_partial_kernel", st, wgrad_partial_kernel<<<grid, 256, sm, st>>>(wa));
         }
-        DEER_KERNEL("wgrad_final_kernel", st, wgrad_final_kernel<<<(outs + 255) / 256, 256, 0, st>>>(w.partial, P, n3, wa.K,
+        DEER_KERNEL("wgrad_final_kernel", st, wgrad_final_kernel<<<(outs + 7) / 8, 256, 0, st>>>(w.partial, P, n3, wa.K,
                                                                 side == 0 ? g->dW_i : g->dW_h,
                                                                 side == 0 ? g->db_i : g->db_h));
     }

@@ -468,18 +468,91 @@ __global__ void wgrad_partial_kernel(WgradArgs a)
     if (valid) a.partial[(size_t)blockIdx.x * outs + o] = acc;
 }
 
-// Stage 2: one thread per output adds the P slice sums in slice order.
+// Stage 1 for small gates (n3 <= 32, K <= 8): lane g keeps out[g][0..K] in registers; the warps of
+// CTA p take blocks of four consecutive positions of slice p in turn (warp w: blocks w, w + 8, ...),
+// a lane reading its dG[e][g] (one coalesced row per position) and the row V[e][:] (broadcast).
+// The eight warp sums are added in warp order, so the result is bit-reproducible.
+__global__ void __launch_bounds__(256) wgrad_small_kernel(WgradArgs a)
+{
+    constexpr int KMAX = 8, WARPS = 8, BLK = 4;
+    __shared__ float part[WARPS][32 * (KMAX + 1)];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int K = a.K, K1 = K + 1, n3 = a.n3;
+    const size_t e0 = (size_t)blockIdx.x * a.slice;
+    const size_t e1 = min(a.N, e0 + a.slice);
+    const bool vec = (K % 4 == 0) && ((((uintptr_t)a.V | (uintptr_t)a.y0) & 15) == 0);
+    float acc[KMAX + 1];
+#pragma unroll
+    for (int k = 0; k <= KMAX; ++k) acc[k] = 0.0f;
+    for (size_t base = e0 + (size_t)warp * BLK; base < e1; base += (size_t)WARPS * BLK) {
+        float dg[BLK], v[BLK][KMAX];
+        size_t seq = 0;
+        int t = 0;                                        // (seq, t) of position base + u, carried along
+        if (a.shifted) { seq = base / (size_t)a.T; t = (int)(base - seq * (size_t)a.T); }
+#pragma unroll
+        for (int u = 0; u < BLK; ++u) {
+            const size_t e = base + u;
+            const bool in = e < e1;
+            dg[u] = (in && lane < n3) ? a.dG[e * n3 + lane] : 0.0f;
+            const float *row = a.V;                       // row of V paired with position e
+            if (in) {
+                if (!a.shifted) row = a.V + e * K;
+                else row = (t == 0) ? a.y0 + seq * K : a.V + (e - 1) * K;
+            }
+            if (++t >= a.T) { t = 0; ++seq; }
+            if (vec) {
+#pragma unroll
+                for (int q = 0; q < KMAX / 4; ++q) {
+                    float4 f = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    if (in && 4 * q < K) f = __ldg(reinterpret_cast<const float4 *>(row) + q);
+                    v[u][4 * q] = f.x; v[u][4 * q + 1] = f.y; v[u][4 * q + 2] = f.z; v[u][4 * q + 3] = f.w;
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < KMAX; ++k) v[u][k] = (in && k < K) ? __ldg(row + k) : 0.0f;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < BLK; ++u) {
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k) acc[k] = fmaf(dg[u], v[u][k], acc[k]);
+            acc[KMAX] += dg[u];                           // bias column (V = 1)
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < KMAX; ++k) part[warp][lane * (KMAX + 1) + k] = acc[k];
+    part[warp][lane * (KMAX + 1) + KMAX] = acc[KMAX];
+    __syncthreads();
+    const int outs = n3 * K1;
+    for (int o = threadIdx.x; o < outs; o += blockDim.x) {
+        const int g = o / K1, k = o - g * K1;
+        const int src = g * (KMAX + 1) + (k < K ? k : KMAX);
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) s += part[w][src];
+        a.partial[(size_t)blockIdx.x * outs + o] = s;
+    }
+}
+
+// Stage 2: one warp per output.  Lane l adds slices l, l + 32, ... in that order (all loads in
+// flight together), then the 32 lane sums are combined by a fixed shuffle tree: the order of the
+// additions depends on P only, so the result is bit-reproducible.
 __global__ void wgrad_final_kernel(const float *__restrict__ partial, int P, int n3, int K,
                                    float *__restrict__ dW, float *__restrict__ db)
 {
     const int K1 = K + 1, outs = n3 * K1;
-    int o = blockIdx.x * blockDim.x + threadIdx.x;
+    const int o = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (o >= outs) return;
     float acc = 0.0f;
-    for (int p = 0; p < P; ++p) acc += partial[(size_t)p * outs + o];
-    int g = o / K1, k = o % K1;
-    if (k < K) dW[(size_t)g * K + k] = acc;
-    else db[g] = acc;
+#pragma unroll 4
+    for (int p = lane; p < P; p += 32) acc += partial[(size_t)p * outs + o];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
+    if (lane == 0) {
+        const int g = o / K1, k = o % K1;
+        if (k < K) dW[(size_t)g * K + k] = acc;
+        else db[g] = acc;
+    }
 }
 
 // ------------------------------------------------------------------ a9: classifier glue
