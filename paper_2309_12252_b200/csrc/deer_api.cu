@@ -525,7 +525,7 @@ constexpr int WGRAD_P = 592;   // slices of the position axis in the parameter-g
 
 struct VjpWs {
     StatusBlock *st;
-    float *u, *J, *rhs, *lam, *dGi, *dGh, *partial;
+    float *u, *J, *rhs, *lam, *dGi, *dGh, *partial, *partial2;
     ScanWs scan;
     size_t bytes;
 };
@@ -543,6 +543,7 @@ static VjpWs carve_vjp(void *ws, int B, int T, int n, int m)
     w.dGh = cv.take<float>(N * 3 * n);
     int kmax = (m > n ? m : n) + 1;
     w.partial = cv.take<float>((size_t)WGRAD_P * 3 * n * kmax);
+    w.partial2 = cv.take<float>((size_t)WGRAD_P * 3 * n * kmax);
     w.scan = carve_scan(cv, B, T, n);
     w.rhs = nullptr;
     w.bytes = cv.off;
@@ -693,6 +694,45 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     return status;
 }
 
+// cell VJP, parameter-gradient slices and dx in one pass (n, m in {1,2,4,8}); P = slices written
+template <int N, int M>
+static int launch_vjp_small_nm(const VjpSmallArgs &v, int *P, cudaStream_t st)
+{
+    constexpr int EPB = 256 / N;
+    constexpr size_t SM = sizeof(float) * 256 * (3 * (M + 1) + 3 * (N + 1) + 1);
+    int rc = opt_in_smem((const void *)vjp_small_kernel<N, M>, SM);
+    if (rc != DEER_OK) return rc;
+    const size_t total = (size_t)v.B * v.T;
+    size_t blocks = (total + EPB - 1) / EPB;
+    if (blocks > (size_t)WGRAD_P) blocks = WGRAD_P;
+    *P = (int)blocks;
+    DEER_KERNEL("vjp_small_kernel", st, (vjp_small_kernel<N, M><<<(unsigned)blocks, 256, SM, st>>>(v)));
+    return DEER_OK;
+}
+
+template <int N>
+static int launch_vjp_small_n(const VjpSmallArgs &v, int m, int *P, cudaStream_t st)
+{
+    switch (m) {
+    case 1: return launch_vjp_small_nm<N, 1>(v, P, st);
+    case 2: return launch_vjp_small_nm<N, 2>(v, P, st);
+    case 4: return launch_vjp_small_nm<N, 4>(v, P, st);
+    case 8: return launch_vjp_small_nm<N, 8>(v, P, st);
+    default: return DEER_ERR_UNSUPPORTED_N;
+    }
+}
+
+static int launch_vjp_small(const VjpSmallArgs &v, int n, int m, int *P, cudaStream_t st)
+{
+    switch (n) {
+    case 1: return launch_vjp_small_n<1>(v, m, P, st);
+    case 2: return launch_vjp_small_n<2>(v, m, P, st);
+    case 4: return launch_vjp_small_n<4>(v, m, P, st);
+    case 8: return launch_vjp_small_n<8>(v, m, P, st);
+    default: return DEER_ERR_UNSUPPORTED_N;
+    }
+}
+
 static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y0, const float *y,
                         const float *gy, int B, int T, const deer_gru_grads *g, float *dx,
                         float *dy0, void *ws, size_t ws_bytes, int flags, cudaStream_t st)
@@ -703,8 +743,12 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
     if (rc != DEER_OK) return rc;
     const size_t N = (size_t)B * T;
     DEER_CHECK_CUDA(cudaMemsetAsync(w.st, 0, sizeof(StatusBlock), st), "memset status");
-    if ((rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
-    CellArgs c{p->W_h, p->b_h, w.u, x, p->W_i, p->b_i, m, y, y0, w.J, nullptr, B, T, n, nullptr};
+    // small n and m: the cell projects x itself and one kernel does the cell VJP, the slices of the
+    // parameter-gradient reduction and dx (no u, dG_i, dG_h arrays)
+    const bool small = cell_projects(n, m) && !(flags & DEER_FLAG_GENERIC) && y0 != nullptr &&
+                       ((((uintptr_t)y | (uintptr_t)y0) & 15) == 0);
+    if (!small && (rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
+    CellArgs c{p->W_h, p->b_h, small ? nullptr : w.u, x, p->W_i, p->b_i, m, y, y0, w.J, nullptr, B, T, n, nullptr};
     if ((rc = run_cell(c, st)) != DEER_OK) return rc;
     ScanArgs a{};
     a.J = w.J; a.b = gy; a.y0 = nullptr; a.y = w.lam; a.yold = nullptr;
@@ -714,6 +758,17 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
     a.st = w.st;
     if ((rc = run_scan(a, w.scan, flags, st)) != DEER_OK) return rc;
 
+    if (small) {
+        VjpSmallArgs v{p->W_h, p->b_h, p->W_i, p->b_i, x, y, y0, w.lam, dx, w.partial, w.partial2, B, T};
+        int P = 0;
+        if ((rc = launch_vjp_small(v, n, m, &P, st)) != DEER_OK) return rc;
+        DEER_KERNEL("wgrad_final_kernel", st, wgrad_final_kernel<<<(n3 * (m + 1) + 7) / 8, 256, 0, st>>>(w.partial, P, n3, m, g->dW_i, g->db_i));
+        DEER_KERNEL("wgrad_final_kernel", st, wgrad_final_kernel<<<(n3 * (n + 1) + 7) / 8, 256, 0, st>>>(w.partial2, P, n3, n, g->dW_h, g->db_h));
+        if (dy0) {
+            DEER_KERNEL("vjp_dy0_kernel", st, vjp_dy0_kernel<<<(B * n + 127) / 128, 128, 0, st>>>(w.J, w.lam, dy0, B, T, n));
+        }
+        return DEER_OK;
+    }
     {
         VjpArgs v{p->W_h, p->b_h, w.u, y, y0, w.lam, w.dGi, w.dGh, B, T, n};
         const bool aligned = (((uintptr_t)y | (uintptr_t)y0) & 15) == 0;

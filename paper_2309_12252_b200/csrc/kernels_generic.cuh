@@ -394,6 +394,146 @@ __global__ void vjp_cell_kernel(VjpArgs a)
     gh[i] = dar; gh[n + i] = daz; gh[2 * n + i] = dq;
 }
 
+// ------------------------------------------------------------------ a8 for small n: cell VJP and reductions in one pass
+// n in {1,2,4,8}, m in {1,2,4,8} (Eq. 7 applied to the GRU; App. B.1).  One thread per (position, row i), as
+// in cell_small_kernel: gates from h_prev and x (projection on the fly), then with lam = dL/df at the position
+//   d_an = lam (1-z)(1-c^2),  d_az = lam (h_i - c) z (1-z),  d_ar = d_an q r (1-r),  d_q = d_an r
+// (the gradients w.r.t. the three input-side and hidden-side pre-activations of row i), accumulated
+// in registers straight into this thread's share of dW_i, dW_h, db_i, db_h -- no per-position gradient
+// arrays exist -- and dx = W_i^T dG_i reduced over the rows of the position by shuffles.
+// CTA p then adds its threads' sums in thread order and writes slice p of the two-stage reduction
+// (stage 2: wgrad_final_kernel), so the result is bit-reproducible.
+struct VjpSmallArgs {
+    const float *W_h, *b_h, *W_i, *b_i, *x, *y, *y0, *lam;
+    float *dx;                 // [B,T,m] or nullptr
+    float *partial_i;          // [P][3n*(m+1)]
+    float *partial_h;          // [P][3n*(n+1)]
+    int B, T;
+};
+
+template <int N, int M>
+__global__ void __launch_bounds__(256, 2) vjp_small_kernel(VjpSmallArgs a)
+{
+    constexpr int EPB = 256 / N;                       // positions per block per step
+    constexpr int VI = 3 * (M + 1), VH = 3 * (N + 1), VALS = VI + VH;
+    extern __shared__ float red[];                     // [256][VALS + 1]
+    const int i = threadIdx.x % N, le = threadIdx.x / N;
+    float wr[N], wz[N], wn[N], vr[M], vz[M], vn[M];
+#pragma unroll
+    for (int k = 0; k < N; ++k) {
+        wr[k] = a.W_h[i * N + k];
+        wz[k] = a.W_h[(N + i) * N + k];
+        wn[k] = a.W_h[(2 * N + i) * N + k];
+    }
+#pragma unroll
+    for (int k = 0; k < M; ++k) {
+        vr[k] = a.W_i[i * M + k];
+        vz[k] = a.W_i[(N + i) * M + k];
+        vn[k] = a.W_i[(2 * N + i) * M + k];
+    }
+    const float br = a.b_h[i], bz = a.b_h[N + i], bn = a.b_h[2 * N + i];
+    const float cr = a.b_i[i], cz = a.b_i[N + i], cn = a.b_i[2 * N + i];
+    float ai[3][M + 1], ah[3][N + 1];
+#pragma unroll
+    for (int g = 0; g < 3; ++g) {
+#pragma unroll
+        for (int k = 0; k <= M; ++k) ai[g][k] = 0.0f;
+#pragma unroll
+        for (int k = 0; k <= N; ++k) ah[g][k] = 0.0f;
+    }
+    const size_t total = (size_t)a.B * a.T;
+    const size_t stride = (size_t)gridDim.x * EPB;
+    const size_t stride_seq = stride / a.T;
+    const unsigned stride_t = (unsigned)(stride - stride_seq * a.T);
+    size_t e = (size_t)blockIdx.x * EPB + le;
+    size_t seq = e / a.T;
+    unsigned t = (unsigned)(e - seq * a.T);
+    // (every thread of a warp runs the same number of iterations when it shuffles: the loop bound is
+    // taken on the position of the warp's first row group, and late positions are masked)
+    for (; ; e += stride, seq += stride_seq, t += stride_t) {
+        if (t >= (unsigned)a.T) { t -= (unsigned)a.T; ++seq; }
+        const bool in = e < total;
+        if (!__any_sync(0xffffffffu, in)) break;
+        float h[N], xv[M], l = 0.0f, hi = 0.0f;
+#pragma unroll
+        for (int k = 0; k < N; ++k) h[k] = 0.0f;
+#pragma unroll
+        for (int k = 0; k < M; ++k) xv[k] = 0.0f;
+        if (in) {
+            const float *hp = (t == 0u) ? a.y0 + seq * N : a.y + (e - 1) * N;
+#pragma unroll
+            for (int k = 0; k < N; ++k) h[k] = hp[k];
+#pragma unroll
+            for (int k = 0; k < M; ++k) xv[k] = a.x[e * M + k];
+            l = a.lam[e * N + i];
+            hi = hp[i];
+        }
+        float gr = br, gz = bz, gq = bn, ur = cr, uz = cz, un = cn;
+#pragma unroll
+        for (int k = 0; k < N; ++k) {
+            gr = fmaf(wr[k], h[k], gr);
+            gz = fmaf(wz[k], h[k], gz);
+            gq = fmaf(wn[k], h[k], gq);
+        }
+#pragma unroll
+        for (int k = 0; k < M; ++k) {
+            ur = fmaf(vr[k], xv[k], ur); uz = fmaf(vz[k], xv[k], uz); un = fmaf(vn[k], xv[k], un);
+        }
+        const float r = sigmoidf_gate(ur + gr);          // the activations of the forward small-n cell
+        const float z = sigmoidf_gate(uz + gz);
+        const float c = tanhf_gate(un + r * gq);
+        const float dan = l * (1.0f - z) * (1.0f - c * c);
+        const float daz = l * (hi - c) * z * (1.0f - z);
+        const float dar = dan * gq * r * (1.0f - r);
+        const float dq = dan * r;
+#pragma unroll
+        for (int k = 0; k < M; ++k) {
+            ai[0][k] = fmaf(dar, xv[k], ai[0][k]); ai[1][k] = fmaf(daz, xv[k], ai[1][k]); ai[2][k] = fmaf(dan, xv[k], ai[2][k]);
+        }
+        ai[0][M] += dar; ai[1][M] += daz; ai[2][M] += dan;
+#pragma unroll
+        for (int k = 0; k < N; ++k) {
+            ah[0][k] = fmaf(dar, h[k], ah[0][k]); ah[1][k] = fmaf(daz, h[k], ah[1][k]); ah[2][k] = fmaf(dq, h[k], ah[2][k]);
+        }
+        ah[0][N] += dar; ah[1][N] += daz; ah[2][N] += dq;
+        if (a.dx) {
+            float pk[M];
+#pragma unroll
+            for (int k = 0; k < M; ++k) {
+                pk[k] = fmaf(vr[k], dar, fmaf(vz[k], daz, vn[k] * dan));
+#pragma unroll
+                for (int d = 1; d < N; d <<= 1) pk[k] += __shfl_xor_sync(0xffffffffu, pk[k], d);
+            }
+            if (in && i == 0) {
+#pragma unroll
+                for (int k = 0; k < M; ++k) a.dx[e * M + k] = pk[k];
+            }
+        }
+    }
+    // CTA reduction in thread order: thread (le, i) -> red[tid][...]; output (row i, value v) adds le = 0 .. EPB-1
+    float *mine = red + threadIdx.x * (VALS + 1);
+#pragma unroll
+    for (int g = 0; g < 3; ++g) {
+#pragma unroll
+        for (int k = 0; k <= M; ++k) mine[g * (M + 1) + k] = ai[g][k];
+#pragma unroll
+        for (int k = 0; k <= N; ++k) mine[VI + g * (N + 1) + k] = ah[g][k];
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < N * VALS; o += blockDim.x) {
+        const int row = o / VALS, v = o - row * VALS;
+        float s = 0.0f;
+        for (int q = 0; q < EPB; ++q) s += red[(q * N + row) * (VALS + 1) + v];
+        if (v < VI) {
+            const int g = v / (M + 1), k = v - g * (M + 1);
+            a.partial_i[(size_t)blockIdx.x * (3 * N * (M + 1)) + (g * N + row) * (M + 1) + k] = s;
+        } else {
+            const int vv = v - VI, g = vv / (N + 1), k = vv - g * (N + 1);
+            a.partial_h[(size_t)blockIdx.x * (3 * N * (N + 1)) + (g * N + row) * (N + 1) + k] = s;
+        }
+    }
+}
+
 // dx[e][k] = sum_g W_i[g][k] dGi[e][g]
 __global__ void vjp_dx_kernel(const float *__restrict__ dGi, const float *__restrict__ W_i,
                               float *__restrict__ dx, size_t N, int m, int n3)
