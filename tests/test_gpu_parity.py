@@ -221,7 +221,7 @@ def test_batch_with_sequences_converging_at_different_bodies(bd):
 
 
 # ----------------------------------------------------------------------------- gradients
-def grad_case(bd, n, m, B, T, dense, seed=5):
+def grad_case(bd, n, m, B, T, dense, seed=5, flags=0, want_dx=True):
     p = synth.gru_params(n, m, seed, tag="v/gru")
     x = synth.x_gaussian(B, T, m, seed, tag="v/x")
     y0 = synth.normal(seed, "v/y0", (B, n)) * 0.3
@@ -231,8 +231,10 @@ def grad_case(bd, n, m, B, T, dense, seed=5):
         last = gy[:, -1].copy(); gy = np.zeros_like(gy); gy[:, -1] = last
     want = oracle.gru_bptt(p, x, y0, y32.astype(np.float64), gy, np.float64)
     pd = bd.GruParamsDev.from_numpy(p)
-    got = bd.deer_gru_vjp(pd, dev(x), dev(y0), dev(y32), dev(gy))
+    got = bd.deer_gru_vjp(pd, dev(x), dev(y0), dev(y32), dev(gy), want_dx=want_dx, flags=flags)
     for k in ("dW_i", "dW_h", "db_i", "db_h", "dx", "dy0"):
+        if k == "dx" and not want_dx:
+            continue
         assert rel_inf(got[k].cpu().numpy().astype(np.float64), want[k]) <= TOL_GRAD, k
     return got
 
@@ -243,6 +245,19 @@ def grad_case(bd, n, m, B, T, dense, seed=5):
 @pytest.mark.parametrize("dense", [True, False])
 def test_vjp_matches_bptt(bd, n, m, B, T, dense):
     grad_case(bd, n, m, B, T, dense)
+
+
+@pytest.mark.parametrize("n,m,B,T", [(8, 8, 2, 900), (4, 8, 3, 333), (2, 1, 2, 50), (1, 4, 3, 211), (8, 4, 16, 5000),
+                                     (8, 1, 5, 77), (4, 4, 1, 1)])
+def test_vjp_small_fused_path(bd, n, m, B, T):
+    """The one-pass gradient kernel for n, m in {1,2,4,8}: more shapes (positions beyond one pass of the
+    grid, ragged warps, T = 1), without dx, and against the separate kernels it replaces."""
+    a = grad_case(bd, n, m, B, T, True)
+    grad_case(bd, n, m, B, T, False, want_dx=False)
+    b = grad_case(bd, n, m, B, T, True, flags=bd.DEER_FLAG_GENERIC)
+    for k in ("dW_i", "dW_h", "db_i", "db_h", "dx", "dy0"):
+        ref = b[k].cpu().numpy()
+        assert np.max(np.abs(a[k].cpu().numpy() - ref)) <= 1e-4 * max(1.0, float(np.max(np.abs(ref)))), k
 
 
 def test_vjp_is_bit_reproducible(bd):
