@@ -49,7 +49,7 @@ def peaks():
 # DRAM bytes (read + write) per position of the stand-alone scan, from the ncu captures summarised in
 # profiles/scan_kernels_standalone_B16.md (inputs larger than L2; traffic grows in proportion to positions).
 NCU_STEP_SCAN_TRAFFIC = 51.43e6      # config-2 step, scan_warp8_kernel: dram read + write per launch
-NCU_SCAN_TRAFFIC_PER_POSITION = {1: 13.0, 2: 33.6, 4: 95.4, 8: 606.6, 16: 2213.0, 32: 8622.0, 64: 34116.0}
+NCU_SCAN_TRAFFIC_PER_POSITION = {1: 12.8, 2: 32.7, 4: 95.3, 8: 606.6, 16: 2213.0, 32: 8622.0, 64: 34116.0}
 
 
 def scan_bytes_per_position(n: int) -> int:
