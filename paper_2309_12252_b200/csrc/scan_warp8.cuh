@@ -86,14 +86,15 @@ __device__ __forceinline__ void chain_step(float (&acc)[4], float j0, float j1, 
     split_tf32(acc[3], ah[3], al[3]);      // a3 <- c3
     split_tf32(j0, bh[0], bl[0]);
     split_tf32(j1, bh[1], bl[1]);
-    // three independent MMAs (the next step waits for one MMA latency, not three), summed afterwards
+    // the two small products chain through one accumulator, the large one runs beside them (the next
+    // step waits for two MMA latencies and four adds; measured best of: all three independent, this, all chained)
     const float z[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-    float d0[4] = {0.0f, 0.0f, bx, by}, d1[4], d2[4];
+    float d0[4] = {0.0f, 0.0f, bx, by}, d1[4];
     mma_tf32(d1, al, bh, z);
-    mma_tf32(d2, ah, bl, z);
     mma_tf32(d0, ah, bh, d0);
+    mma_tf32(d1, ah, bl, d1);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) acc[i] = d0[i] + (d1[i] + d2[i]);
+    for (int i = 0; i < 4; ++i) acc[i] = d0[i] + d1[i];
 }
 
 // Resolver for n = 8 (see resolver_loop of scan_onepass.cuh).  The walk Y <- A Y + beta is the critical
