@@ -146,6 +146,22 @@ int deer_gru_eval(const deer_gru_params *params, const float *x, const float *y0
                   float tol, int max_iter, float *y, int *iters, float *err, float *err_trace,
                   void *ws, size_t ws_bytes, int flags, void *stream);
 
+/* deer_gru_eval with the sequence data in HOST memory (the end-to-end call):
+ * copies x_host to x_dev, evaluates into y_dev as deer_gru_eval does, copies
+ * the result to y_host; the copies run on `stream` (asynchronously when the
+ * host buffers are page-locked) and the result copy is enqueued behind the
+ * Newton bodies, so an evaluation that converges within the first group of
+ * bodies synchronises the host once.
+ *   x_host [B,T,m] host in     y_host [B,T,n] host out
+ *   x_dev  [B,T,m], y_dev [B,T,n] : device staging buffers owned by the caller
+ *            (y_dev holds the guess on entry if DEER_FLAG_WARM_START, and the
+ *            result on return)
+ *   params, y0, ws : device, as for deer_gru_eval
+ * Synchronises `stream`.  Returns what deer_gru_eval returns. */
+int deer_gru_eval_host(const deer_gru_params *params, const float *x_host, const float *y0, int B, int T,
+                       float tol, int max_iter, float *y_host, int *iters, float *err, float *x_dev,
+                       float *y_dev, void *ws, size_t ws_bytes, int flags, void *stream);
+
 /* Gradient through the evaluated sequence (Eq. 7): given gy = dL/dy at a
  * trajectory y, lambda = gy L_G^{-1} by ONE reverse scan with the Jacobians
  * recomputed at y (Sec. 3.1.1 allows saving or recomputing them), then the

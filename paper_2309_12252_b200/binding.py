@@ -23,7 +23,8 @@ DEER_OP_EVAL, DEER_OP_SCAN, DEER_OP_VJP, DEER_OP_CLASSIFIER = 0, 1, 2, 3
 DEER_FLAG_WARM_START, DEER_FLAG_GENERIC, DEER_FLAG_MATERIALIZE, DEER_FLAG_TCGEN05 = 1, 2, 4, 8
 
 NOALLOC_SCRATCH_BYTES = 8 << 20
-EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc", "deer_gru_eval", "deer_gru_vjp",
+EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc", "deer_gru_eval",
+           "deer_gru_eval_host", "deer_gru_vjp",
            "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count"]
 
 
@@ -58,6 +59,9 @@ def lib():
         L.deer_gru_eval.restype = ci
         L.deer_gru_eval.argtypes = [ctypes.POINTER(_Params), vp, vp, ci, ci, cf, ci, vp,
                                     ctypes.POINTER(ci), ctypes.POINTER(cf), vp, vp, sz, ci, vp]
+        L.deer_gru_eval_host.restype = ci
+        L.deer_gru_eval_host.argtypes = [ctypes.POINTER(_Params), vp, vp, ci, ci, cf, ci, vp,
+                                         ctypes.POINTER(ci), ctypes.POINTER(cf), vp, vp, vp, sz, ci, vp]
         L.deer_gru_vjp.restype = ci
         L.deer_gru_vjp.argtypes = [ctypes.POINTER(_Params), vp, vp, vp, vp, ci, ci,
                                    ctypes.POINTER(_Grads), vp, vp, vp, sz, ci, vp]
@@ -89,6 +93,12 @@ def _ptr(t):
     if t is None:
         return None
     assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _hptr(t):
+    """Pointer to a contiguous HOST tensor (pinned for asynchronous copies)."""
+    assert not t.is_cuda and t.is_contiguous() and t.dtype == torch.float32
     return ctypes.c_void_p(t.data_ptr())
 
 
@@ -208,13 +218,21 @@ def deer_gru_eval(params: GruParamsDev, x, y0, tol=1e-4, max_iter=100, y=None, w
 
 def deer_gru_eval_host(params: GruParamsDev, x_host, y0_dev, y_host, x_dev, y_dev, ws, tol=1e-4,
                        max_iter=100, flags=0, stream=None) -> EvalResult:
-    """End-to-end call with HOST buffers: copies x (pinned host) to the device,
-    evaluates, copies y back to pinned host memory."""
-    x_dev.copy_(x_host, non_blocking=True)
-    r = deer_gru_eval(params, x_dev, y0_dev, tol, max_iter, y_dev, ws, flags, stream)
-    y_host.copy_(y_dev, non_blocking=True)
-    torch.cuda.current_stream().synchronize()
-    return r
+    """End-to-end call with HOST buffers (x_host, y_host: pinned host tensors; x_dev, y_dev: device
+    staging buffers): the library copies x to the device, evaluates, copies y back; see include/deer.h."""
+    B, T, m = x_host.shape
+    n = params.n
+    assert m == params.m and not x_host.is_cuda and not y_host.is_cuda and x_dev.is_cuda and y_dev.is_cuda
+    assert tuple(y_host.shape) == (B, T, n) == tuple(y_dev.shape) and tuple(x_dev.shape) == (B, T, m)
+    iters = ctypes.c_int(0)
+    err = ctypes.c_float(0.0)
+    ps = params.c_struct()
+    rc = lib().deer_gru_eval_host(ctypes.byref(ps), _hptr(x_host), _ptr(_f32(y0_dev)), B, T, float(tol),
+                                  int(max_iter), _hptr(y_host), ctypes.byref(iters), ctypes.byref(err),
+                                  _ptr(x_dev), _ptr(y_dev), _ptr(ws), ws.numel(), flags, _stream(stream))
+    if rc < 0:
+        raise DeerError(rc)
+    return EvalResult(y_dev, iters.value, err.value, rc, np.zeros((0,), np.float32))
 
 
 def deer_gru_vjp(params: GruParamsDev, x, y0, y, gy, want_dx=True, want_dy0=True, ws=None, flags=0,

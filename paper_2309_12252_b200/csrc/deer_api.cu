@@ -604,9 +604,13 @@ static int linrec_scan_impl(const float *J, const float *b, const float *y0, int
     return run_scan(a, w.scan, flags, st);
 }
 
+// y_host (optional, host memory): the result is also copied there.  The copy is enqueued behind every
+// group of bodies, after a device-side selection of the buffer that holds the current iterate, so that
+// an evaluation that converges within its first group costs one host synchronisation in all.
 static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *y0, int B, int T,
                          float tol, int max_iter, float *y, int *iters, float *err,
-                         float *err_trace, void *ws, size_t ws_bytes, int flags, cudaStream_t st)
+                         float *err_trace, void *ws, size_t ws_bytes, int flags, cudaStream_t st,
+                         float *y_host = nullptr)
 {
     const int n = p->n, m = p->m;
     EvalWs w = carve_eval(ws, B, T, n, m);
@@ -671,6 +675,15 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
                 DEER_KERNEL("newton_control_kernel", st, newton_control_kernel<<<1, 1, 0, st>>>(w.st, tol, max_iter, w.trace));
             }
         }
+        if (y_host) {
+            size_t words = N * n / 4;
+            unsigned blocks = (unsigned)((words + 1023) / 1024);
+            const unsigned cap = 4u * (unsigned)num_sms();
+            if (blocks > cap) blocks = cap;
+            if (blocks < 1u) blocks = 1u;
+            DEER_KERNEL("result_select_kernel", st, result_select_kernel<<<blocks, 256, 0, st>>>(w.st, y, w.yalt, N * n));
+            DEER_CHECK_CUDA(cudaMemcpyAsync(y_host, y, N * n * sizeof(float), cudaMemcpyDeviceToHost, st), "copy result to host");
+        }
         DEER_CHECK_CUDA(cudaMemcpyAsync(&hs, w.st, 32, cudaMemcpyDeviceToHost, st), "read status");
         DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
         if (hs.flags & FLAG_TIMEOUT) return DEER_ERR_DEVICE_TIMEOUT;
@@ -680,7 +693,7 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     const int k = hs.iters;
     float e;
     memcpy(&e, &hs.err_last_bits, sizeof(float));
-    if (k & 1)
+    if ((k & 1) && !y_host)
         DEER_CHECK_CUDA(cudaMemcpyAsync(y, w.yalt, N * n * sizeof(float), cudaMemcpyDeviceToDevice, st), "copy result");
     if (err_trace && k > 0)
         DEER_CHECK_CUDA(cudaMemcpyAsync(err_trace, w.trace, sizeof(float) * (size_t)(k < ERR_TRACE_CAP ? k : ERR_TRACE_CAP),
@@ -888,6 +901,21 @@ int deer_gru_eval(const deer_gru_params *p, const float *x, const float *y0, int
     if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
     return gru_eval_impl(p, x, y0, B, T, tol, max_iter, y, iters, err, err_trace, ws, ws_bytes, flags,
                          (cudaStream_t)stream);
+}
+
+int deer_gru_eval_host(const deer_gru_params *p, const float *x_host, const float *y0, int B, int T, float tol,
+                       int max_iter, float *y_host, int *iters, float *err, float *x_dev, float *y_dev,
+                       void *ws, size_t ws_bytes, int flags, void *stream)
+{
+    if (!p || !x_host || !y0 || !y_host || !x_dev || !y_dev || !p->W_i || !p->W_h || !p->b_i || !p->b_h)
+        return DEER_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || p->n <= 0 || p->m <= 0 || max_iter < 1 || tol != tol) return DEER_ERR_INVALID_ARG;
+    if (!supported(p->n, p->m)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    DEER_CHECK_CUDA(cudaMemcpyAsync(x_dev, x_host, sizeof(float) * (size_t)B * T * p->m, cudaMemcpyHostToDevice, st),
+                    "copy x to the device");
+    return gru_eval_impl(p, x_dev, y0, B, T, tol, max_iter, y_dev, iters, err, nullptr, ws, ws_bytes, flags, st, y_host);
 }
 
 int deer_gru_vjp(const deer_gru_params *p, const float *x, const float *y0, const float *y,

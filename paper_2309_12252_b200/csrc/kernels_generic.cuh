@@ -343,6 +343,23 @@ __global__ void eval_begin_kernel(StatusBlock *st, StatusBlock init, EvalBeginAr
     for (size_t i = i0; i < e.nagg_words; i += stride) e.agg_words[i] = 0ull;
 }
 
+// After an odd number of bodies the current iterate sits in the workspace copy: bring it into the
+// caller's buffer on the device, without the host having to know the count (the buffer it overwrites
+// is the one the next body, if any, overwrites anyway).  Runs whether or not the loop has ended.
+__global__ void result_select_kernel(const StatusBlock *st, float *y, const float *yalt, size_t ny)
+{
+    if ((st->iters & 1) == 0) return;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if ((((uintptr_t)y | (uintptr_t)yalt) & 15) == 0) {
+        const size_t n4 = ny / 4;
+        for (size_t i = i0; i < n4; i += stride) reinterpret_cast<float4 *>(y)[i] = reinterpret_cast<const float4 *>(yalt)[i];
+        for (size_t i = 4 * n4 + i0; i < ny; i += stride) y[i] = yalt[i];
+    } else {
+        for (size_t i = i0; i < ny; i += stride) y[i] = yalt[i];
+    }
+}
+
 // Loop control as a launch of its own (used when a body's scan ran on the generic kernels).
 __global__ void newton_control_kernel(StatusBlock *st, float tol, int max_iter, float *trace)
 {

@@ -209,6 +209,22 @@ def test_eval_is_bit_reproducible_and_warm_start(bd):
     assert torch.max(torch.abs(r.y - a.y)).item() <= 1e-5
 
 
+@pytest.mark.parametrize("max_iter,tol", [(100, 1e-4), (3, 1e-4), (5, -1.0), (7, -1.0)])
+def test_eval_with_host_buffers_matches_device_call(bd, max_iter, tol):
+    """deer_gru_eval_host (copies inside the library, result selected on the device) returns exactly what
+    deer_gru_eval returns, for even and odd body counts and for more bodies than the first group."""
+    w = synth.config(2, B=3, T=1200)
+    p = bd.GruParamsDev.from_numpy(w.params)
+    ref = bd.deer_gru_eval(p, dev(w.x), dev(w.y0), tol=tol, max_iter=max_iter, check=False)
+    x_host = torch.from_numpy(np.ascontiguousarray(w.x)).pin_memory()
+    y_host = torch.empty((3, 1200, 8), dtype=torch.float32).pin_memory()
+    x_dev = torch.empty((3, 1200, 4), device="cuda"); y_dev = torch.empty((3, 1200, 8), device="cuda")
+    ws = bd.alloc_workspace(bd.DEER_OP_EVAL, 3, 1200, 8, 4, 0, x_dev.device)
+    r = bd.deer_gru_eval_host(p, x_host, dev(w.y0), y_host, x_dev, y_dev, ws, tol=tol, max_iter=max_iter)
+    assert (r.iters, r.status) == (ref.iters, ref.status) and r.err == ref.err
+    assert torch.equal(y_host, ref.y.cpu()) and torch.equal(y_dev, ref.y)
+
+
 def test_batch_with_sequences_converging_at_different_bodies(bd):
     """One global err: a sequence that is easy (zero input, tiny weights effect)
     next to a hard one still ends at the sequential values for both."""
