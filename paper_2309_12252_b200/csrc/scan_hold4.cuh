@@ -249,6 +249,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
 
         // ------------------------------------------------ B: replay from the entering state
         {
+            if constexpr (REV) load_b(t, cnt, bs);      // (reverse: read again rather than kept in registers)
             float y[N];
 #pragma unroll
             for (int k = 0; k < N; ++k) y[k] = ystart[k];
