@@ -146,6 +146,20 @@ int deer_gru_eval(const deer_gru_params *params, const float *x, const float *y0
                   float tol, int max_iter, float *y, int *iters, float *err, float *err_trace,
                   void *ws, size_t ws_bytes, int flags, void *stream);
 
+/* deer_gru_eval with diagnostics of the last executed body (App. B.1: the
+ * quantity the loop tests is max |y_new - y|):
+ *   err_b      : host out [B], max |y_new - y| per sequence (may be NULL)
+ *   err_argmax : host out, flat index (b*T + t)*n + i of the element where the
+ *                global maximum is attained; ties go to the smallest index
+ *                (may be NULL)
+ * Both are pure functions of the last two iterates and, like iters, err and
+ * every bit of y, identical across runs.  T*n must fit 32 bits.  Everything
+ * else as deer_gru_eval. */
+int deer_gru_eval_diag(const deer_gru_params *params, const float *x, const float *y0, int B, int T,
+                       float tol, int max_iter, float *y, int *iters, float *err, float *err_trace,
+                       float *err_b, unsigned long long *err_argmax, void *ws, size_t ws_bytes, int flags,
+                       void *stream);
+
 /* deer_gru_eval with the sequence data in HOST memory (the end-to-end call):
  * copies x_host to x_dev, evaluates into y_dev as deer_gru_eval does, copies
  * the result to y_host; the copies run on `stream` (asynchronously when the

@@ -24,7 +24,7 @@ DEER_FLAG_WARM_START, DEER_FLAG_GENERIC, DEER_FLAG_MATERIALIZE, DEER_FLAG_TCGEN0
 
 NOALLOC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc", "deer_gru_eval",
-           "deer_gru_eval_host", "deer_gru_vjp",
+           "deer_gru_eval_diag", "deer_gru_eval_host", "deer_gru_vjp",
            "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count"]
 
 
@@ -59,6 +59,10 @@ def lib():
         L.deer_gru_eval.restype = ci
         L.deer_gru_eval.argtypes = [ctypes.POINTER(_Params), vp, vp, ci, ci, cf, ci, vp,
                                     ctypes.POINTER(ci), ctypes.POINTER(cf), vp, vp, sz, ci, vp]
+        L.deer_gru_eval_diag.restype = ci
+        L.deer_gru_eval_diag.argtypes = [ctypes.POINTER(_Params), vp, vp, ci, ci, cf, ci, vp,
+                                         ctypes.POINTER(ci), ctypes.POINTER(cf), vp, vp,
+                                         ctypes.POINTER(ctypes.c_ulonglong), vp, sz, ci, vp]
         L.deer_gru_eval_host.restype = ci
         L.deer_gru_eval_host.argtypes = [ctypes.POINTER(_Params), vp, vp, ci, ci, cf, ci, vp,
                                          ctypes.POINTER(ci), ctypes.POINTER(cf), vp, vp, vp, sz, ci, vp]
@@ -214,6 +218,29 @@ def deer_gru_eval(params: GruParamsDev, x, y0, tol=1e-4, max_iter=100, y=None, w
     if check and rc < 0:
         raise DeerError(rc)
     return EvalResult(y, iters.value, err.value, rc, trace[:iters.value])
+
+
+def deer_gru_eval_diag(params: GruParamsDev, x, y0, tol=1e-4, max_iter=100, y=None, ws=None, flags=0, stream=None):
+    """deer_gru_eval plus the diagnostics of the last body: returns (EvalResult, err_b [B] numpy, err_argmax int)."""
+    B, T, m = x.shape
+    n = params.n
+    if y is None:
+        y = torch.empty((B, T, n), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = alloc_workspace(DEER_OP_EVAL, B, T, n, m, flags, x.device)
+    iters = ctypes.c_int(0)
+    err = ctypes.c_float(0.0)
+    trace = np.full((max(int(max_iter), 1),), np.nan, np.float32)
+    err_b = np.full((B,), np.nan, np.float32)
+    argmax = ctypes.c_ulonglong(0)
+    ps = params.c_struct()
+    rc = lib().deer_gru_eval_diag(ctypes.byref(ps), _ptr(_f32(x)), _ptr(_f32(y0)), B, T, float(tol), int(max_iter),
+                                  _ptr(y), ctypes.byref(iters), ctypes.byref(err),
+                                  trace.ctypes.data_as(ctypes.c_void_p), err_b.ctypes.data_as(ctypes.c_void_p),
+                                  ctypes.byref(argmax), _ptr(ws), ws.numel(), flags, _stream(stream))
+    if rc < 0:
+        raise DeerError(rc)
+    return EvalResult(y, iters.value, err.value, rc, trace[:iters.value]), err_b, int(argmax.value)
 
 
 def deer_gru_eval_host(params: GruParamsDev, x_host, y0_dev, y_host, x_dev, y_dev, ws, tol=1e-4,

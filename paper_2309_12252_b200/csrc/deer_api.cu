@@ -483,6 +483,7 @@ static bool supported(int n, int m) { return n >= 1 && n <= 64 && m >= 1 && m <=
 struct EvalWs {
     StatusBlock *st;
     float *trace;        // [ERR_TRACE_CAP] err after each body (device side of err_trace)
+    unsigned long long *diag;   // [B] per-sequence {err bits, inverted index} of the last body
     float *u, *J, *rhs, *yalt;
     ScanWs scan;
     size_t bytes;
@@ -496,6 +497,7 @@ static EvalWs carve_eval(void *ws, int B, int T, int n, int m)
     size_t N = (size_t)B * T;
     w.st = cv.take<StatusBlock>(1);
     w.trace = cv.take<float>(ERR_TRACE_CAP);
+    w.diag = cv.take<unsigned long long>((size_t)B);
     w.u = cv.take<float>(N * 3 * n);
     w.J = cv.take<float>(N * n * n);
     w.rhs = cv.take<float>(N * n);
@@ -610,7 +612,7 @@ static int linrec_scan_impl(const float *J, const float *b, const float *y0, int
 static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *y0, int B, int T,
                          float tol, int max_iter, float *y, int *iters, float *err,
                          float *err_trace, void *ws, size_t ws_bytes, int flags, cudaStream_t st,
-                         float *y_host = nullptr)
+                         float *y_host = nullptr, float *err_b = nullptr, unsigned long long *err_argmax = nullptr)
 {
     const int n = p->n, m = p->m;
     EvalWs w = carve_eval(ws, B, T, n, m);
@@ -693,6 +695,23 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     const int k = hs.iters;
     float e;
     memcpy(&e, &hs.err_last_bits, sizeof(float));
+    if ((err_b || err_argmax) && k > 0) {
+        // the last two iterates are still in the two buffers (before the result copy below)
+        std::vector<unsigned long long> keys((size_t)B);
+        DEER_KERNEL("err_diag_kernel", st, err_diag_kernel<<<(unsigned)B, 256, 0, st>>>(buf[k & 1], buf[(k + 1) & 1], (size_t)T * n, w.diag));
+        DEER_CHECK_CUDA(cudaMemcpyAsync(keys.data(), w.diag, sizeof(unsigned long long) * (size_t)B, cudaMemcpyDeviceToHost, st), "read diagnostics");
+        DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+        unsigned long long best = 0ull;
+        int best_b = 0;
+        for (int b = 0; b < B; ++b) {
+            const unsigned bits = (unsigned)(keys[b] >> 32);
+            if (err_b) memcpy(&err_b[b], &bits, sizeof(float));
+            if ((keys[b] >> 32) > (best >> 32) || b == 0) { best = keys[b]; best_b = b; }
+        }
+        if (err_argmax)
+            *err_argmax = (unsigned long long)best_b * (unsigned long long)T * (unsigned long long)n +
+                          (unsigned long long)(0xffffffffu - (unsigned)(best & 0xffffffffull));
+    }
     if ((k & 1) && !y_host)
         DEER_CHECK_CUDA(cudaMemcpyAsync(y, w.yalt, N * n * sizeof(float), cudaMemcpyDeviceToDevice, st), "copy result");
     if (err_trace && k > 0)
@@ -901,6 +920,19 @@ int deer_gru_eval(const deer_gru_params *p, const float *x, const float *y0, int
     if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
     return gru_eval_impl(p, x, y0, B, T, tol, max_iter, y, iters, err, err_trace, ws, ws_bytes, flags,
                          (cudaStream_t)stream);
+}
+
+int deer_gru_eval_diag(const deer_gru_params *p, const float *x, const float *y0, int B, int T, float tol,
+                       int max_iter, float *y, int *iters, float *err, float *err_trace, float *err_b,
+                       unsigned long long *err_argmax, void *ws, size_t ws_bytes, int flags, void *stream)
+{
+    if (!p || !x || !y0 || !y || !p->W_i || !p->W_h || !p->b_i || !p->b_h) return DEER_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || p->n <= 0 || p->m <= 0 || max_iter < 1 || tol != tol) return DEER_ERR_INVALID_ARG;
+    if (!supported(p->n, p->m)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
+    if ((unsigned long long)T * (unsigned long long)p->n > 0xffffffffull) return DEER_ERR_INVALID_ARG;
+    return gru_eval_impl(p, x, y0, B, T, tol, max_iter, y, iters, err, err_trace, ws, ws_bytes, flags,
+                         (cudaStream_t)stream, nullptr, err_b, err_argmax);
 }
 
 int deer_gru_eval_host(const deer_gru_params *p, const float *x_host, const float *y0, int B, int T, float tol,

@@ -360,6 +360,34 @@ __global__ void result_select_kernel(const StatusBlock *st, float *y, const floa
     }
 }
 
+// Diagnostics of the last body (one CTA per sequence): key[b] = max |y_new - y_old| over the sequence
+// as float bits in the upper word, and 0xffffffff - (index within the sequence of its first occurrence)
+// in the lower word, so that an integer max gives the largest deviation and, among equals, the
+// smallest index.  Pure function of the two iterates: identical across runs.
+__global__ void __launch_bounds__(256) err_diag_kernel(const float *__restrict__ ynew, const float *__restrict__ yold,
+                                                        size_t per_seq, unsigned long long *__restrict__ key)
+{
+    __shared__ unsigned long long red[8];
+    const size_t base = (size_t)blockIdx.x * per_seq;
+    unsigned long long best = 0ull;
+    for (size_t i = threadIdx.x; i < per_seq; i += blockDim.x) {
+        const unsigned long long k = ((unsigned long long)absdiff_bits(ynew[base + i], yold[base + i]) << 32) |
+                                     (unsigned long long)(0xffffffffu - (unsigned)i);
+        best = k > best ? k : best;
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, d);
+        best = o > best ? o : best;
+    }
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) best = red[w] > best ? red[w] : best;
+        key[blockIdx.x] = best;
+    }
+}
+
 // Loop control as a launch of its own (used when a body's scan ran on the generic kernels).
 __global__ void newton_control_kernel(StatusBlock *st, float tol, int max_iter, float *trace)
 {

@@ -225,6 +225,27 @@ def test_eval_with_host_buffers_matches_device_call(bd, max_iter, tol):
     assert torch.equal(y_host, ref.y.cpu()) and torch.equal(y_dev, ref.y)
 
 
+@pytest.mark.parametrize("n,m,B,T,k", [(8, 4, 5, 700, 3), (8, 4, 5, 700, 4), (4, 2, 3, 1000, 2), (32, 32, 2, 300, 3),
+                                       (2, 2, 4, 50, 1)])
+def test_eval_diagnostics_of_the_last_body(bd, n, m, B, T, k):
+    """err_b and err_argmax describe max |y_k - y_{k-1}|: checked against the two iterates themselves
+    (exactly k and k - 1 bodies from the same start are bit-reproducible), ties to the smallest index,
+    identical across runs."""
+    p_np = synth.gru_params(n, m, 3, tag="d/gru")
+    x = dev(synth.x_gaussian(B, T, m, 3, tag="d/x"))
+    y0 = dev(synth.normal(3, "d/y0", (B, n)) * 0.3)
+    p = bd.GruParamsDev.from_numpy(p_np)
+    r, err_b, amax = bd.deer_gru_eval_diag(p, x, y0, tol=-1.0, max_iter=k)
+    r2, err_b2, amax2 = bd.deer_gru_eval_diag(p, x, y0, tol=-1.0, max_iter=k)
+    assert r.iters == k and amax == amax2 and np.array_equal(err_b, err_b2) and torch.equal(r.y, r2.y)
+    prev = (bd.deer_gru_eval(p, x, y0, tol=-1.0, max_iter=k - 1, check=False).y if k > 1
+            else torch.zeros_like(r.y))
+    d = (r.y - prev).abs().cpu().numpy()
+    assert np.array_equal(err_b, d.reshape(B, -1).max(axis=1))
+    assert float(err_b.max()) == r.err
+    assert amax == int(np.argmax(d.reshape(-1)))          # numpy: first occurrence of the maximum
+
+
 def test_batch_with_sequences_converging_at_different_bodies(bd):
     """One global err: a sequence that is easy (zero input, tiny weights effect)
     next to a hard one still ends at the sequential values for both."""
