@@ -345,11 +345,17 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
                 float tac[4] = {(g == 2 * t) ? 1.0f : 0.0f, (g == 2 * t + 1) ? 1.0f : 0.0f, 0.0f, 0.0f};
 #pragma unroll
                 for (int k = 0; k < WARPS; ++k) {
-                    const float *ak = wagg + k * AGG;
+                    float *ak = wagg + k * AGG;
                     const float2 f = *reinterpret_cast<const float2 *>(ak + 2 * lane);
                     float bx = 0.0f, by = 0.0f;
                     if (g == 0) { bx = ak[NN + 2 * t]; by = ak[NN + 2 * t + 1]; }
                     chain_step(tac, f.x, f.y, bx, by);
+                    // warp k's aggregate is replaced by the aggregate of warps 0..k: in the B item every
+                    // warp then gets the state entering its chain by one mat-vec of its own
+                    __syncwarp();
+                    ak[(2 * t) * N + g] = tac[0];
+                    ak[(2 * t + 1) * N + g] = tac[1];
+                    if (g == 0) { ak[NN + 2 * t] = tac[2]; ak[NN + 2 * t + 1] = tac[3]; }
                 }
                 float *gdst = w.aggs + tile_index * AGG;
                 gdst[(2 * t) * N + g] = tac[0];
@@ -385,10 +391,9 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
         if (warp == 0) {
             if (lane < N) wstart[lane] = ystart[lane];
             __syncwarp();
-            for (int k = 0; k + 1 < WARPS; ++k)
-                matvec_smem<8>(wstart + (k + 1) * N, wagg + k * AGG, wstart + k * N, lane);
+        } else {
+            matvec_smem<8>(wstart + warp * N, wagg + (warp - 1) * AGG, ystart, lane);
         }
-        __syncthreads();
         {
             // lane (g,t) carries y[2t], y[2t+1]; every step: partial sums over k = 2t, 2t+1, reduced over t
             float yk0 = wstart[warp * N + 2 * t], yk1 = wstart[warp * N + 2 * t + 1];
