@@ -41,6 +41,8 @@ SCAN_CASES = [  # (n, B, T)
     # more sequences than resolver warps (several sequences per warp), and sequences with more tiles than
     # one resolver visit looks at
     (4, 40, 1500), (2, 70, 5000), (1, 70, 15000), (8, 40, 700), (4, 2, 30001), (2, 1, 50000), (1, 1, 150000),
+    # tiny T and tile boundaries of the n = 4 and n = 2 kernels (640 and 2304 positions per tile)
+    (4, 2, 1), (4, 3, 2), (4, 2, 5), (4, 1, 640), (4, 2, 641), (4, 1, 1279), (2, 2, 1), (2, 1, 2304), (2, 2, 2305),
 ]
 
 
