@@ -76,8 +76,10 @@ enum {
     DEER_FLAG_WARM_START = 1,   /* deer_gru_eval: y holds the initial guess on entry (Sec. 3.1:
                                    the previous training step's solution may seed the next) */
     DEER_FLAG_GENERIC    = 2,   /* force the generic (any-n) kernels; for testing */
-    DEER_FLAG_MATERIALIZE = 4,  /* deer_gru_eval: write J and b to the workspace and run the
-                                   stand-alone scan on them, instead of the fused iteration */
+    DEER_FLAG_MATERIALIZE = 4,  /* deer_gru_eval, n = 16 and 32: have the cell write the Jacobians
+                                   J [B,T,n,n] to the workspace and scan them, instead of writing
+                                   four coefficient vectors per position from which the scan builds
+                                   J_t itself (the default there; the results are bit-identical) */
     DEER_FLAG_TCGEN05    = 8    /* n = 64 scans: run the chain product (Eq. 10's matrix half) as
                                    tcgen05.mma in tensor memory instead of register-resident
                                    mma.sync fragments; same results to rounding, currently slower */

@@ -149,7 +149,8 @@ __global__ void __launch_bounds__(256, (N <= 32) ? 4 : 0) cell_wide_kernel(CellA
                     const float an = (1.0f - z) * (1.0f - c * c);
                     const float kr = an * qn * r * (1.0f - r);
                     const float kn = an * r;
-                    sC[p * N + gi] = make_float4(kr, az, kn, z);
+                    if (a.coef_only) reinterpret_cast<float4 *>(a.J)[e * N + gi] = make_float4(kr, az, kn, z);
+                    else sC[p * N + gi] = make_float4(kr, az, kn, z);
                     if (a.rhs) {
                         float jh = z * hi;
                         jh = fmaf(az, gz[q], jh);
@@ -162,8 +163,8 @@ __global__ void __launch_bounds__(256, (N <= 32) ? 4 : 0) cell_wide_kernel(CellA
         }
         __syncthreads();
 
-        // ---- Jacobian phase
-        for (int p = tid / C::CHUNKS; p < np; p += C::PPAR) {       // tid / CHUNKS == 0 when CPT >= 1 piece
+        // ---- Jacobian phase (not when only the coefficient rows are wanted)
+        for (int p = tid / C::CHUNKS; p < (a.coef_only ? 0 : np); p += C::PPAR) {       // tid / CHUNKS == 0 when CPT >= 1 piece
             float *Je = a.J + (e0 + p) * (size_t)(N * N);
 #pragma unroll
             for (int r = 0; r < C::CPT; ++r) {

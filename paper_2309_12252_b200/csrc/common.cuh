@@ -114,6 +114,8 @@ struct ScanArgs {
     float *carB;         // [B,nch,n]   chunk aggregates (vector part)
     float *starts;       // [B,nch,n]   state entering each chunk
     StatusBlock *st;
+    const float *Wh;     // [3n,n] hidden weights when J holds coefficient rows [B,T,n,4] instead of
+                         // matrices (the scan generates J_t itself); nullptr otherwise
 };
 
 struct CellArgs {
@@ -130,6 +132,8 @@ struct CellArgs {
     float *rhs;          // [B,T,n]   out: f - J y_prev   (nullptr: skip)
     int B, T, n;
     const StatusBlock *st;   // nullptr, or: skip all work once st->done is set (Newton loop ended)
+    int coef_only;           // wide kernels: write the coefficient rows {k_r, a_z, k_n, z} [B,T,n,4] to J
+                             // instead of the matrices (the scan generates J_t from them)
 };
 
 // Programmatic dependent launch: a kernel of the Newton loop lets the next launch in the stream be set

@@ -16,6 +16,7 @@
 #include "scan_hold4.cuh"
 #include "scan_warp8.cuh"
 #include "scan_warpn.cuh"
+#include "scan_warpn_fused.cuh"
 #include "scan_cta64.cuh"
 #include "scan_umma64.cuh"
 #include "cell_wide.cuh"
@@ -236,6 +237,16 @@ static int launch_warpn(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
     return launch_single_pass(scan_warpn_kernel<N, REV>, occ, c, a, w, prep, st);
 }
 
+// forward scan that generates J_t from coefficient rows (a.J) and a.Wh
+template <int N>
+static int launch_warpnf(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
+{
+    using C = WarpNF<N>;
+    static int occ[MAX_DEVICES] = {0};
+    const PassCfg c{"scan_warpnf_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 8};
+    return launch_single_pass(scan_warpnf_kernel<N>, occ, c, a, w, prep, st);
+}
+
 template <bool REV>
 static int launch_cta64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
@@ -266,9 +277,9 @@ static int scan_onepass(ScanArgs a, OnePassWs w, bool prep, int flags, cudaStrea
     case 9: return launch_hold4<true>(a, w, prep, st);
     case 16: return launch_warp8<false>(a, w, prep, st);
     case 17: return launch_warp8<true>(a, w, prep, st);
-    case 32: return launch_warpn<16, false>(a, w, prep, st);
+    case 32: return a.Wh ? launch_warpnf<16>(a, w, prep, st) : launch_warpn<16, false>(a, w, prep, st);
     case 33: return launch_warpn<16, true>(a, w, prep, st);
-    case 64: return launch_warpn<32, false>(a, w, prep, st);
+    case 64: return a.Wh ? launch_warpnf<32>(a, w, prep, st) : launch_warpn<32, false>(a, w, prep, st);
     case 65: return launch_warpn<32, true>(a, w, prep, st);
     case 128: return umma ? launch_umma64<false>(a, w, prep, st) : launch_cta64<false>(a, w, prep, st);
     case 129: return umma ? launch_umma64<true>(a, w, prep, st) : launch_cta64<true>(a, w, prep, st);
@@ -630,6 +641,11 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     // With the single-pass scan the last CTA of every scan takes the loop decision and the scan
     // leaves its flag words cleared: a body is two launches (cell, scan).
     const bool single = scan_is_single_pass(a, w.scan, flags) && (((uintptr_t)w.yalt) & 15) == 0;
+    // n = 16, 32: the cell writes coefficient rows and the scan generates J_t itself, unless the caller
+    // asks for materialised Jacobians
+    const bool gen_J = single && (n == 16 || n == 32) && !(flags & DEER_FLAG_MATERIALIZE) &&
+                       ((((uintptr_t)y | (uintptr_t)y0) & 15) == 0);
+    if (gen_J) a.Wh = p->W_h;
     {
         StatusBlock init;
         memset(&init, 0, sizeof(init));
@@ -667,7 +683,8 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
         if (todo > group) todo = group;
         for (int j = 0; j < todo; ++j, ++enq) {
             float *cur = buf[enq & 1], *nxt = buf[(enq + 1) & 1];
-            CellArgs c{p->W_h, p->b_h, fused_proj ? nullptr : w.u, x, p->W_i, p->b_i, m, cur, y0, w.J, w.rhs, B, T, n, w.st};
+            CellArgs c{p->W_h, p->b_h, fused_proj ? nullptr : w.u, x, p->W_i, p->b_i, m, cur, y0, w.J, w.rhs, B, T, n, w.st,
+                       gen_J ? 1 : 0};
             if ((rc = run_cell(c, st)) != DEER_OK) return rc;
             a.y = nxt; a.yold = cur;
             if (single) {

@@ -1,0 +1,305 @@
+// Single-pass scan for n = 16 and n = 32 INSIDE deer_gru_eval, with J_t generated on the fly.
+//
+// The GRU Jacobian at a position is a function of four n-vectors and the shared hidden weights,
+//     J = diag(k_r) W_hr + diag(a_z) W_hz + diag(k_n) W_hn + diag(z)
+// (k_r = a_n q r (1-r), k_n = a_n r, a_z = (h - c) z (1-z), a_n = (1-z)(1-c^2); Sec. 3.1 / Eq. 5 with the
+// closed-form GRU derivative), so the cell writes 16 n bytes per position instead of 4 n^2 and this
+// kernel, identical to scan_warpn_kernel in everything else (forward direction), builds the lane's
+// operand pieces of J_t from the staged coefficient rows and W_h kept in shared memory: 3 n^2 FMAs per
+// position and visit on the fp32 pipes in exchange for n/5 times less memory traffic.
+#pragma once
+#include "scan_warpn.cuh"
+
+namespace deer {
+
+template <int N> struct WarpNF {
+    using B_ = WarpN<N>;
+    static constexpr int NN = N * N, AGG = N * N + N, NT = N / 8, MT = N / 16;
+    static constexpr int WARPS = B_::WARPS, THREADS = B_::THREADS;
+    static constexpr int CTAS_PER_SM = B_::CTAS_PER_SM;
+    static constexpr int Q = B_::Q;
+    static constexpr int STAGES = 8;                   // ring depth per warp (positions): a stage is 5 n floats
+    static constexpr int STAGE_FLOATS = 5 * N;         // coefficient rows [N][4], then the vector [N]
+    static constexpr int WS = N + 8;                   // row stride of the weights (conflict-free 8-byte operand reads)
+    static constexpr int RES_WARPS = B_::RES_WARPS, RES_BATCH = B_::RES_BATCH;
+    static constexpr int PEND = B_::PEND;
+    static constexpr int SM_WORK = Q * PEND + WARPS * N + N + 16 + 3 * N * WS + WARPS * STAGES * STAGE_FLOATS;
+    static constexpr int SM_RES = RES_WARPS * RES_BATCH * AGG;
+    static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
+    static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
+    static constexpr int MAX_SEQ_PER_WARP = B_::MAX_SEQ_PER_WARP;
+    static_assert(STAGES * STAGE_FLOATS >= AGG, "the last warp's aggregate is parked in its ring");
+};
+
+// The lane's pieces of J_t, jp[nn][kk] = {J[8nn+g][8kk+2t], J[8nn+g][8kk+2t+1]}, from the staged
+// coefficient rows cf[i] = {k_r, a_z, k_n, z}_i and the weights in shared memory.
+template <int N>
+__device__ __forceinline__ void gen_pieces(float (&jp)[N / 8][N / 8][2], const float *stage, const float *sW,
+                                           int g, int t, bool d0, bool d1)
+{
+    constexpr int NT = N / 8, WS = WarpNF<N>::WS;
+#pragma unroll
+    for (int nn = 0; nn < NT; ++nn) {
+        const float4 cf = *reinterpret_cast<const float4 *>(stage + 4 * (8 * nn + g));
+        const float *wr = sW + (8 * nn + g) * WS + 2 * t;
+#pragma unroll
+        for (int kk = 0; kk < NT; ++kk) {
+            const float2 r2 = *reinterpret_cast<const float2 *>(wr + 8 * kk);
+            const float2 z2 = *reinterpret_cast<const float2 *>(wr + N * WS + 8 * kk);
+            const float2 n2 = *reinterpret_cast<const float2 *>(wr + 2 * N * WS + 8 * kk);
+            float v0 = fmaf(cf.x, r2.x, fmaf(cf.y, z2.x, cf.z * n2.x));
+            float v1 = fmaf(cf.x, r2.y, fmaf(cf.y, z2.y, cf.z * n2.y));
+            if (nn == kk) { v0 += d0 ? cf.w : 0.0f; v1 += d1 ? cf.w : 0.0f; }
+            jp[nn][kk][0] = v0; jp[nn][kk][1] = v1;
+        }
+    }
+}
+
+template <int N>
+__global__ void __launch_bounds__(WarpNF<N>::THREADS, WarpNF<N>::CTAS_PER_SM) scan_warpnf_kernel(ScanArgs a, OnePassWs w)
+{
+    using C = WarpNF<N>;
+    constexpr int NN = C::NN, AGG = C::AGG, NT = C::NT, MT = C::MT, WARPS = C::WARPS, Q = C::Q;
+    pdl_prologue();
+    if (loop_ended(a.st)) return;
+
+    extern __shared__ __align__(16) float smem_raw[];
+    float *sm = (float *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    float *pend = sm;                          // Q x warp aggregates (A row-major, then beta)
+    float *wstart = pend + Q * C::PEND;        // WARPS x N states entering each warp chain
+    float *ystart = wstart + WARPS * N;
+    float *sW = ystart + N + 16;               // W_hr, W_hz, W_hn with rows padded to WS floats
+    float *ring_all = sW + 3 * N * C::WS;      // WARPS x STAGES x (coefficients [N][4], vector [N])
+    __shared__ int s_kind, s_seq, s_c, s_slot, s_abort, s_role;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int T = a.T;
+    constexpr int S = C::STAGES;
+    float *ring = ring_all + warp * S * C::STAGE_FLOATS;
+    const int SW = w.sw, L = WARPS * SW;
+    for (int i = tid; i < 3 * NN; i += C::THREADS) sW[(i / N) * C::WS + (i % N)] = a.Wh[i];
+    const bool d0 = g == 2 * t, d1 = g == 2 * t + 1;      // this lane's pieces touch the diagonal where nn == kk
+
+    if (tid == 0) {
+        s_abort = 0;
+        s_role = (int)atomicAdd(&a.st->role_counter, 1u);
+    }
+    __syncthreads();
+    if (s_role < w.resolvers) {
+        if (warp < C::RES_WARPS)
+            resolver_big<N>(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        __syncthreads();
+        if (tid == 0) scan_epilogue(a.st);
+        return;
+    }
+    unsigned mb = 0;
+
+    auto decode = [&](unsigned id, int &seq, int &c) {
+        const unsigned j = id % (unsigned)w.Wd;
+        const unsigned ws_ = id / (unsigned)w.Wd;
+        seq = (int)(ws_ % (unsigned)a.B);
+        const unsigned win = ws_ / (unsigned)a.B;
+        c = (int)(win * (unsigned)w.Wd + j);
+        if (c >= w.nch) c = -1;
+    };
+    int q_seq[Q], q_c[Q], q_head = 0, q_cnt = 0;
+    bool exhausted = false;
+
+    for (;;) {
+        __syncthreads();
+        if (tid == 0) {
+            int kind = -1, seq = -1, c = -1, slot = 0;
+            bool want_b = false;
+            if (q_cnt > 0) {
+                want_b = (q_cnt == Q) || exhausted;
+                if (!want_b)
+                    want_b = ld_relaxed_u64(w.starts + ((size_t)q_seq[q_head] * w.nch + q_c[q_head]) * N) != 0ull;
+            }
+            if (!want_b && !exhausted) {
+                for (;;) {
+                    const unsigned id = atomicAdd(&a.st->tile_counter, 1u);
+                    if (id >= w.total_ids) { c = -1; break; }
+                    decode(id, seq, c);
+                    if (c >= 0) break;
+                }
+                if (c >= 0) {
+                    kind = 0;
+                    slot = (q_head + q_cnt) % Q;
+                    q_seq[slot] = seq; q_c[slot] = c; ++q_cnt;
+                } else {
+                    exhausted = true;
+                    want_b = q_cnt > 0;
+                }
+            }
+            if (want_b) {
+                kind = 1; slot = q_head; seq = q_seq[q_head]; c = q_c[q_head];
+                q_head = (q_head + 1) % Q; --q_cnt;
+            }
+            s_kind = kind; s_seq = seq; s_c = c; s_slot = slot;
+        }
+        __syncthreads();
+        if (s_kind < 0 || s_abort) break;
+        const int kind = s_kind, seq = s_seq, c = s_c;
+        float *wagg = pend + s_slot * C::PEND;
+        const int s0 = c * L;
+        const int Lt = min(L, T - s0);
+        const int p0 = warp * SW;
+        const int cnt = min(SW, max(0, Lt - p0));
+        const int sbase = s0 + p0;                             // scan position of the chain's first element
+        const size_t tile_index = (size_t)seq * w.nch + c;
+        const float *Cseq = a.J + (size_t)seq * T * 4 * N;      // coefficient rows {k_r, a_z, k_n, z}[N] per position
+        const float *bseq = a.b + (size_t)seq * T * N;
+        auto pos_t = [&](int s) -> size_t { return (size_t)s; };
+        // chain position q -> ring stage q % S (one commit group per call, also past the end)
+        auto issue = [&](int q) {
+            const int s = sbase + q;
+            if (q < cnt) {
+                float *dst = ring + (q % S) * C::STAGE_FLOATS;
+                const float *cs = Cseq + (size_t)s * 4 * N, *bs = bseq + (size_t)s * N;
+#pragma unroll
+                for (int u = 0; u < (5 * N / 4 + 31) / 32; ++u) {
+                    const int j = lane + 32 * u;
+                    if (j < N) cp_async16(dst + 4 * j, cs + 4 * j);
+                    else if (j < N + N / 4) cp_async16(dst + 4 * j, bs + 4 * (j - N));
+                }
+            }
+            cp_async_commit();
+        };
+
+        if (kind == 0) {
+            // ---------------------------------------------- A item
+            float acc[MT][NT][4];
+            identity_fragments<N>(acc, g, t);
+            float yv[NT][2];
+#pragma unroll
+            for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = 0.0f; yv[kk][1] = 0.0f; }
+#pragma unroll
+            for (int q = 0; q < S - 1; ++q) issue(q);
+#pragma unroll 1
+            for (int q = 0; q < cnt; ++q) {
+                cp_async_wait_n<S - 2>();
+                __syncwarp();                  // stage q landed for every lane; stage q-1 is free again
+                issue(q + S - 1);
+                const float *Ms = ring + (q % S) * C::STAGE_FLOATS;
+                float jp[NT][NT][2], bg[NT], ynew[NT];
+                gen_pieces<N>(jp, Ms, sW, g, t, d0, d1);
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn) bg[nn] = Ms[4 * N + 8 * nn + g];
+                chain_step_n<N>(acc, jp);
+                matvec_step<N>(yv, jp, bg, ynew, t);
+            }
+            cp_async_wait_n<0>();
+            __syncwarp();
+            store_aggregate<N>(warp + 1 < WARPS ? wagg + warp * AGG : ring, acc, yv, g, t);
+            __syncthreads();
+            if (warp == 0) {
+                // tile aggregate = the same steps with the warp aggregates as positions (forward form)
+                identity_fragments<N>(acc, g, t);
+#pragma unroll
+                for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = 0.0f; yv[kk][1] = 0.0f; }
+#pragma unroll 1
+                for (int k = 0; k < WARPS; ++k) {
+                    const float *ak = k + 1 < WARPS ? wagg + k * AGG : ring_all + (WARPS - 1) * S * C::STAGE_FLOATS;
+                    float jp[NT][NT][2], bg[NT], ynew[NT];
+                    load_pieces_smem<N>(jp, ak, g, t);
+#pragma unroll
+                    for (int nn = 0; nn < NT; ++nn) bg[nn] = ak[NN + 8 * nn + g];
+                    chain_step_n<N>(acc, jp);
+                    matvec_step<N>(yv, jp, bg, ynew, t);
+                }
+                store_aggregate<N>(w.aggs + tile_index * AGG, acc, yv, g, t);
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) st_release_u32(w.flags + tile_index, 1u);
+            }
+            continue;
+        }
+
+        // -------------------------------------------------- B item
+#pragma unroll
+        for (int q = 0; q < S - 1; ++q) issue(q);      // the chain's first positions fly while the state arrives
+        if (warp == 1) {
+            const unsigned long long *src = w.starts + tile_index * N;
+            unsigned spins = 0;
+            bool ok = true;
+            for (;;) {
+                const unsigned long long v = (lane < N) ? ld_relaxed_u64(src + lane) : LL_FLAG;
+                if (__all_sync(0xffffffffu, v != 0ull)) {
+                    if (lane < N) {
+                        ystart[lane] = __uint_as_float((unsigned)(v & 0xffffffffull));
+                        st_relaxed_u64(w.starts + tile_index * N + lane, 0ull);     // consumed: cleared for the next launch
+                    }
+                    break;
+                }
+                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+            }
+            if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
+        }
+        __syncthreads();
+        if (s_abort) { cp_async_wait_n<0>(); break; }
+        if (warp == 0) {
+            // states entering each warp chain: walk the warp aggregates from the tile's entering state
+            float yv[NT][2];
+#pragma unroll
+            for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = ystart[8 * kk + 2 * t]; yv[kk][1] = ystart[8 * kk + 2 * t + 1]; }
+#pragma unroll 1
+            for (int k = 0; k < WARPS; ++k) {
+                if (g == 0) {
+#pragma unroll
+                    for (int kk = 0; kk < NT; ++kk) {
+                        wstart[k * N + 8 * kk + 2 * t] = yv[kk][0];
+                        wstart[k * N + 8 * kk + 2 * t + 1] = yv[kk][1];
+                    }
+                }
+                if (k + 1 == WARPS) break;
+                const float *ak = wagg + k * AGG;
+                float jp[NT][NT][2], bg[NT], ynew[NT];
+                load_pieces_smem<N>(jp, ak, g, t);
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn) bg[nn] = ak[NN + 8 * nn + g];
+                matvec_step<N>(yv, jp, bg, ynew, t);
+            }
+        }
+        __syncthreads();
+        {
+            float yv[NT][2];
+#pragma unroll
+            for (int kk = 0; kk < NT; ++kk) {
+                yv[kk][0] = wstart[warp * N + 8 * kk + 2 * t];
+                yv[kk][1] = wstart[warp * N + 8 * kk + 2 * t + 1];
+            }
+#pragma unroll 1
+            for (int q = 0; q < cnt; ++q) {
+                const int s = sbase + q;
+                cp_async_wait_n<S - 2>();
+                __syncwarp();
+                issue(q + S - 1);
+                const float *Ms = ring + (q % S) * C::STAGE_FLOATS;
+                float jp[NT][NT][2], bg[NT], ynew[NT];
+                gen_pieces<N>(jp, Ms, sW, g, t, d0, d1);
+                const size_t vb = ((size_t)seq * T + pos_t(s)) * N;
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn) bg[nn] = Ms[4 * N + 8 * nn + g];
+                matvec_step<N>(yv, jp, bg, ynew, t);
+                if (t == 0) {
+#pragma unroll
+                    for (int nn = 0; nn < NT; ++nn) {
+                        if (a.yold) mb = max(mb, absdiff_bits(ynew[nn], __ldg(a.yold + vb + 8 * nn + g)));
+                        a.y[vb + 8 * nn + g] = ynew[nn];
+                    }
+                }
+            }
+            cp_async_wait_n<0>();
+        }
+    }
+    if (a.yold) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+        if (lane == 0 && mb) { atomicMax(&a.st->err_bits, mb); __threadfence(); }
+    }
+    __syncthreads();
+    if (tid == 0) scan_epilogue(a.st);
+}
+
+}  // namespace deer

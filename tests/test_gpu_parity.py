@@ -248,6 +248,18 @@ def test_eval_diagnostics_of_the_last_body(bd, n, m, B, T, k):
     assert amax == int(np.argmax(d.reshape(-1)))          # numpy: first occurrence of the maximum
 
 
+@pytest.mark.parametrize("n,m,B,T", [(16, 16, 3, 900), (32, 32, 2, 700), (16, 5, 2, 333), (32, 8, 1, 65)])
+def test_generated_and_materialised_jacobians_agree_bitwise(bd, n, m, B, T):
+    """n = 16, 32: by default the scan builds J_t from the coefficient rows the cell writes; with
+    DEER_FLAG_MATERIALIZE the cell writes J itself.  Same formula, same order of operations: same bits."""
+    p = bd.GruParamsDev.from_numpy(synth.gru_params(n, m, 11, tag="f/gru"))
+    x = dev(synth.x_gaussian(B, T, m, 11, tag="f/x"))
+    y0 = dev(synth.normal(11, "f/y0", (B, n)) * 0.3)
+    a = bd.deer_gru_eval(p, x, y0)
+    b = bd.deer_gru_eval(p, x, y0, flags=bd.DEER_FLAG_MATERIALIZE)
+    assert a.status == 0 and (a.iters, a.err) == (b.iters, b.err) and torch.equal(a.y, b.y)
+
+
 def test_batch_with_sequences_converging_at_different_bodies(bd):
     """One global err: a sequence that is easy (zero input, tiny weights effect)
     next to a hard one still ends at the sequential values for both."""
