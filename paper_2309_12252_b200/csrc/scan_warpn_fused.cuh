@@ -20,7 +20,10 @@ template <int N> struct WarpNF {
     static constexpr int Q = B_::Q;
     static constexpr int STAGES = 8;                   // ring depth per warp (positions): a stage is 5 n floats
     static constexpr int STAGE_FLOATS = 5 * N;         // coefficient rows [N][4], then the vector [N]
-    static constexpr int WS = N + 8;                   // row stride of the weights (conflict-free 8-byte operand reads)
+    // weights in shared memory: row i of a matrix holds, for t = 0..3, the 2*NT values a lane (g,t) needs
+    // from that row, {W[i][8kk+2t], W[i][8kk+2t+1]} for kk = 0..NT-1, contiguously (128-bit reads); the row
+    // stride makes the reads of a quarter-warp (two rows, four t) fall in distinct banks
+    static constexpr int WS = N + (N == 32 ? 4 : 0);
     static constexpr int RES_WARPS = B_::RES_WARPS, RES_BATCH = B_::RES_BATCH;
     static constexpr int PEND = B_::PEND;
     static constexpr int SM_WORK = Q * PEND + WARPS * N + N + 16 + 3 * N * WS + WARPS * STAGES * STAGE_FLOATS;
@@ -41,14 +44,21 @@ __device__ __forceinline__ void gen_pieces(float (&jp)[N / 8][N / 8][2], const f
 #pragma unroll
     for (int nn = 0; nn < NT; ++nn) {
         const float4 cf = *reinterpret_cast<const float4 *>(stage + 4 * (8 * nn + g));
-        const float *wr = sW + (8 * nn + g) * WS + 2 * t;
+        const float *wrow = sW + (8 * nn + g) * WS + t * 2 * NT;
+        float wr[2 * NT], wz[2 * NT], wn[2 * NT];
+#pragma unroll
+        for (int v = 0; v < 2 * NT / 4; ++v) {
+            const float4 r4 = reinterpret_cast<const float4 *>(wrow)[v];
+            const float4 z4 = reinterpret_cast<const float4 *>(wrow + N * WS)[v];
+            const float4 n4 = reinterpret_cast<const float4 *>(wrow + 2 * N * WS)[v];
+            wr[4 * v] = r4.x; wr[4 * v + 1] = r4.y; wr[4 * v + 2] = r4.z; wr[4 * v + 3] = r4.w;
+            wz[4 * v] = z4.x; wz[4 * v + 1] = z4.y; wz[4 * v + 2] = z4.z; wz[4 * v + 3] = z4.w;
+            wn[4 * v] = n4.x; wn[4 * v + 1] = n4.y; wn[4 * v + 2] = n4.z; wn[4 * v + 3] = n4.w;
+        }
 #pragma unroll
         for (int kk = 0; kk < NT; ++kk) {
-            const float2 r2 = *reinterpret_cast<const float2 *>(wr + 8 * kk);
-            const float2 z2 = *reinterpret_cast<const float2 *>(wr + N * WS + 8 * kk);
-            const float2 n2 = *reinterpret_cast<const float2 *>(wr + 2 * N * WS + 8 * kk);
-            float v0 = fmaf(cf.x, r2.x, fmaf(cf.y, z2.x, cf.z * n2.x));
-            float v1 = fmaf(cf.x, r2.y, fmaf(cf.y, z2.y, cf.z * n2.y));
+            float v0 = fmaf(cf.x, wr[2 * kk], fmaf(cf.y, wz[2 * kk], cf.z * wn[2 * kk]));
+            float v1 = fmaf(cf.x, wr[2 * kk + 1], fmaf(cf.y, wz[2 * kk + 1], cf.z * wn[2 * kk + 1]));
             if (nn == kk) { v0 += d0 ? cf.w : 0.0f; v1 += d1 ? cf.w : 0.0f; }
             jp[nn][kk][0] = v0; jp[nn][kk][1] = v1;
         }
@@ -78,7 +88,10 @@ __global__ void __launch_bounds__(WarpNF<N>::THREADS, WarpNF<N>::CTAS_PER_SM) sc
     constexpr int S = C::STAGES;
     float *ring = ring_all + warp * S * C::STAGE_FLOATS;
     const int SW = w.sw, L = WARPS * SW;
-    for (int i = tid; i < 3 * NN; i += C::THREADS) sW[(i / N) * C::WS + (i % N)] = a.Wh[i];
+    for (int i = tid; i < 3 * NN; i += C::THREADS) {
+        const int col = i % N, kk = col >> 3, tt = (col & 7) >> 1, e = col & 1;
+        sW[(i / N) * C::WS + tt * 2 * NT + 2 * kk + e] = a.Wh[i];
+    }
     const bool d0 = g == 2 * t, d1 = g == 2 * t + 1;      // this lane's pieces touch the diagonal where nn == kk
 
     if (tid == 0) {
