@@ -237,14 +237,14 @@ static int launch_warpn(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
     return launch_single_pass(scan_warpn_kernel<N, REV>, occ, c, a, w, prep, st);
 }
 
-// forward scan that generates J_t from coefficient rows (a.J) and a.Wh
-template <int N>
+// scans that generate J_t from coefficient rows (a.J) and a.Wh
+template <int N, bool REV>
 static int launch_warpnf(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
-    using C = WarpNF<N>;
+    using C = WarpNF<N, REV>;
     static int occ[MAX_DEVICES] = {0};
     const PassCfg c{"scan_warpnf_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 8};
-    return launch_single_pass(scan_warpnf_kernel<N>, occ, c, a, w, prep, st);
+    return launch_single_pass(scan_warpnf_kernel<N, REV>, occ, c, a, w, prep, st);
 }
 
 template <bool REV>
@@ -277,10 +277,10 @@ static int scan_onepass(ScanArgs a, OnePassWs w, bool prep, int flags, cudaStrea
     case 9: return launch_hold4<true>(a, w, prep, st);
     case 16: return launch_warp8<false>(a, w, prep, st);
     case 17: return launch_warp8<true>(a, w, prep, st);
-    case 32: return a.Wh ? launch_warpnf<16>(a, w, prep, st) : launch_warpn<16, false>(a, w, prep, st);
-    case 33: return launch_warpn<16, true>(a, w, prep, st);
-    case 64: return a.Wh ? launch_warpnf<32>(a, w, prep, st) : launch_warpn<32, false>(a, w, prep, st);
-    case 65: return launch_warpn<32, true>(a, w, prep, st);
+    case 32: return a.Wh ? launch_warpnf<16, false>(a, w, prep, st) : launch_warpn<16, false>(a, w, prep, st);
+    case 33: return a.Wh ? launch_warpnf<16, true>(a, w, prep, st) : launch_warpn<16, true>(a, w, prep, st);
+    case 64: return a.Wh ? launch_warpnf<32, false>(a, w, prep, st) : launch_warpn<32, false>(a, w, prep, st);
+    case 65: return a.Wh ? launch_warpnf<32, true>(a, w, prep, st) : launch_warpn<32, true>(a, w, prep, st);
     case 128: return umma ? launch_umma64<false>(a, w, prep, st) : launch_cta64<false>(a, w, prep, st);
     case 129: return umma ? launch_umma64<true>(a, w, prep, st) : launch_cta64<true>(a, w, prep, st);
     default: return DEER_ERR_UNSUPPORTED_N;
@@ -797,14 +797,19 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
     const bool small = cell_projects(n, m) && !(flags & DEER_FLAG_GENERIC) && y0 != nullptr &&
                        ((((uintptr_t)y | (uintptr_t)y0) & 15) == 0);
     if (!small && (rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
-    CellArgs c{p->W_h, p->b_h, small ? nullptr : w.u, x, p->W_i, p->b_i, m, y, y0, w.J, nullptr, B, T, n, nullptr};
-    if ((rc = run_cell(c, st)) != DEER_OK) return rc;
     ScanArgs a{};
     a.J = w.J; a.b = gy; a.y0 = nullptr; a.y = w.lam; a.yold = nullptr;
     a.B = B; a.T = T; a.n = n; a.reverse = 1;
     a.L = w.scan.L; a.nch = w.scan.nch;
     a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
     a.st = w.st;
+    // n = 16, 32: coefficient rows instead of Jacobians, J_{t+1}^T built in the reverse scan (as in the evaluation)
+    const bool gen_J = (n == 16 || n == 32) && !(flags & DEER_FLAG_MATERIALIZE) && scan_is_single_pass(a, w.scan, flags) &&
+                       ((((uintptr_t)y | (uintptr_t)y0) & 15) == 0);
+    if (gen_J) a.Wh = p->W_h;
+    CellArgs c{p->W_h, p->b_h, small ? nullptr : w.u, x, p->W_i, p->b_i, m, y, y0, w.J, nullptr, B, T, n, nullptr,
+               gen_J ? 1 : 0};
+    if ((rc = run_cell(c, st)) != DEER_OK) return rc;
     if ((rc = run_scan(a, w.scan, flags, st)) != DEER_OK) return rc;
 
     if (small) {
@@ -868,7 +873,11 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
         }
     }
     if (dy0) {
-        DEER_KERNEL("vjp_dy0_kernel", st, vjp_dy0_kernel<<<(B * n + 127) / 128, 128, 0, st>>>(w.J, w.lam, dy0, B, T, n));
+        if (gen_J) {
+            DEER_KERNEL("vjp_dy0_coef_kernel", st, vjp_dy0_coef_kernel<<<(B * n + 127) / 128, 128, 0, st>>>(w.J, p->W_h, w.lam, dy0, B, T, n));
+        } else {
+            DEER_KERNEL("vjp_dy0_kernel", st, vjp_dy0_kernel<<<(B * n + 127) / 128, 128, 0, st>>>(w.J, w.lam, dy0, B, T, n));
+        }
     }
     return DEER_OK;
 }

@@ -607,6 +607,26 @@ __global__ void vjp_dy0_kernel(const float *__restrict__ J, const float *__restr
     dy0[idx] = acc;
 }
 
+// the same from the coefficient rows {k_r, a_z, k_n, z}[n] of position 0 (J = diag(k_r) W_hr + diag(a_z) W_hz +
+// diag(k_n) W_hn + diag(z), evaluated in the order of the cell's Jacobian phase)
+__global__ void vjp_dy0_coef_kernel(const float *__restrict__ coef, const float *__restrict__ W_h,
+                                    const float *__restrict__ lam, float *__restrict__ dy0, int B, int T, int n)
+{
+    int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= B * n) return;
+    int seq = idx / n, j = idx % n;
+    const float4 *c0 = reinterpret_cast<const float4 *>(coef) + (size_t)seq * T * n;
+    const float *l0 = lam + (size_t)seq * T * n;
+    float acc = 0.0f;
+    for (int i = 0; i < n; ++i) {
+        const float4 k = c0[i];
+        float v = fmaf(k.x, W_h[(size_t)i * n + j], fmaf(k.y, W_h[(size_t)(n + i) * n + j], k.z * W_h[(size_t)(2 * n + i) * n + j]));
+        if (i == j) v += k.w;
+        acc = fmaf(v, l0[i], acc);
+    }
+    dy0[idx] = acc;
+}
+
 // Deterministic two-stage reduction  out[g][k] = sum_e dG[e][g] * V[e][k]  (k == K: bias, V = 1).
 // Stage 1: CTA (p, oy) accumulates 256 outputs over slice p of the positions, in position order.
 struct WgradArgs {

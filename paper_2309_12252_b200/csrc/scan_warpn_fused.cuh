@@ -1,18 +1,19 @@
-// Single-pass scan for n = 16 and n = 32 INSIDE deer_gru_eval, with J_t generated on the fly.
+// Single-pass scans for n = 16 and n = 32 inside deer_gru_eval and deer_gru_vjp, with J_t generated on the fly.
 //
 // The GRU Jacobian at a position is a function of four n-vectors and the shared hidden weights,
 //     J = diag(k_r) W_hr + diag(a_z) W_hz + diag(k_n) W_hn + diag(z)
 // (k_r = a_n q r (1-r), k_n = a_n r, a_z = (h - c) z (1-z), a_n = (1-z)(1-c^2); Sec. 3.1 / Eq. 5 with the
 // closed-form GRU derivative), so the cell writes 16 n bytes per position instead of 4 n^2 and this
-// kernel, identical to scan_warpn_kernel in everything else (forward direction), builds the lane's
-// operand pieces of J_t from the staged coefficient rows and W_h kept in shared memory: 3 n^2 FMAs per
+// kernel, identical to scan_warpn_kernel in everything else (both directions), builds the lane's
+// operand pieces of J_t (forward) or J_{t+1}^T (reverse; identity at the first scan position: coefficient
+// rows {0,0,0,1}) from the staged coefficient rows and W_h kept in shared memory: 3 n^2 FMAs per
 // position and visit on the fp32 pipes in exchange for n/5 times less memory traffic.
 #pragma once
 #include "scan_warpn.cuh"
 
 namespace deer {
 
-template <int N> struct WarpNF {
+template <int N, bool REV = false> struct WarpNF {
     using B_ = WarpN<N>;
     static constexpr int NN = N * N, AGG = N * N + N, NT = N / 8, MT = N / 16;
     static constexpr int WARPS = B_::WARPS, THREADS = B_::THREADS;
@@ -20,10 +21,11 @@ template <int N> struct WarpNF {
     static constexpr int Q = B_::Q;
     static constexpr int STAGES = 8;                   // ring depth per warp (positions): a stage is 5 n floats
     static constexpr int STAGE_FLOATS = 5 * N;         // coefficient rows [N][4], then the vector [N]
-    // weights in shared memory: row i of a matrix holds, for t = 0..3, the 2*NT values a lane (g,t) needs
-    // from that row, {W[i][8kk+2t], W[i][8kk+2t+1]} for kk = 0..NT-1, contiguously (128-bit reads); the row
-    // stride makes the reads of a quarter-warp (two rows, four t) fall in distinct banks
-    static constexpr int WS = N + (N == 32 ? 4 : 0);
+    // weights in shared memory, laid out so that what a lane (g,t) needs from one row is contiguous:
+    //   forward: row i holds, for t = 0..3, {W[i][8kk+2t], W[i][8kk+2t+1]} for kk = 0..NT-1
+    //   reverse: row i holds, for g = 0..7, W[i][8nn+g] for nn = 0..NT-1
+    // (128-bit reads at n = 32); the row stride makes the reads of a quarter- or half-warp fall in distinct banks
+    static constexpr int WS = N + (N == 32 ? 4 : (REV ? 4 : 0));
     static constexpr int RES_WARPS = B_::RES_WARPS, RES_BATCH = B_::RES_BATCH;
     static constexpr int PEND = B_::PEND;
     static constexpr int SM_WORK = Q * PEND + WARPS * N + N + 16 + 3 * N * WS + WARPS * STAGES * STAGE_FLOATS;
@@ -36,6 +38,43 @@ template <int N> struct WarpNF {
 
 // The lane's pieces of J_t, jp[nn][kk] = {J[8nn+g][8kk+2t], J[8nn+g][8kk+2t+1]}, from the staged
 // coefficient rows cf[i] = {k_r, a_z, k_n, z}_i and the weights in shared memory.
+// reverse form: jp[nn][kk] = {J[8kk+2t][8nn+g], J[8kk+2t+1][8nn+g]} (the operand is J, not its transpose)
+template <int N>
+__device__ __forceinline__ void gen_pieces_rev(float (&jp)[N / 8][N / 8][2], const float *stage, const float *sW,
+                                               int g, int t, bool d0, bool d1)
+{
+    constexpr int NT = N / 8, WS = WarpNF<N, true>::WS;
+#pragma unroll
+    for (int kk = 0; kk < NT; ++kk) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int row = 8 * kk + 2 * t + e;
+            const float4 cf = *reinterpret_cast<const float4 *>(stage + 4 * row);
+            const float *wrow = sW + row * WS + g * NT;
+            float wr[NT], wz[NT], wn[NT];
+            if constexpr (NT == 4) {
+                const float4 r4 = *reinterpret_cast<const float4 *>(wrow);
+                const float4 z4 = *reinterpret_cast<const float4 *>(wrow + N * WS);
+                const float4 n4 = *reinterpret_cast<const float4 *>(wrow + 2 * N * WS);
+                wr[0] = r4.x; wr[1] = r4.y; wr[2] = r4.z; wr[3] = r4.w;
+                wz[0] = z4.x; wz[1] = z4.y; wz[2] = z4.z; wz[3] = z4.w;
+                wn[0] = n4.x; wn[1] = n4.y; wn[2] = n4.z; wn[3] = n4.w;
+            } else {
+                const float2 r2 = *reinterpret_cast<const float2 *>(wrow);
+                const float2 z2 = *reinterpret_cast<const float2 *>(wrow + N * WS);
+                const float2 n2 = *reinterpret_cast<const float2 *>(wrow + 2 * N * WS);
+                wr[0] = r2.x; wr[1] = r2.y; wz[0] = z2.x; wz[1] = z2.y; wn[0] = n2.x; wn[1] = n2.y;
+            }
+#pragma unroll
+            for (int nn = 0; nn < NT; ++nn) {
+                float v = fmaf(cf.x, wr[nn], fmaf(cf.y, wz[nn], cf.z * wn[nn]));
+                if (nn == kk) v += (e == 0 ? d0 : d1) ? cf.w : 0.0f;
+                jp[nn][kk][e] = v;
+            }
+        }
+    }
+}
+
 template <int N>
 __device__ __forceinline__ void gen_pieces(float (&jp)[N / 8][N / 8][2], const float *stage, const float *sW,
                                            int g, int t, bool d0, bool d1)
@@ -65,10 +104,10 @@ __device__ __forceinline__ void gen_pieces(float (&jp)[N / 8][N / 8][2], const f
     }
 }
 
-template <int N>
-__global__ void __launch_bounds__(WarpNF<N>::THREADS, WarpNF<N>::CTAS_PER_SM) scan_warpnf_kernel(ScanArgs a, OnePassWs w)
+template <int N, bool REV>
+__global__ void __launch_bounds__(WarpNF<N, REV>::THREADS, WarpNF<N, REV>::CTAS_PER_SM) scan_warpnf_kernel(ScanArgs a, OnePassWs w)
 {
-    using C = WarpNF<N>;
+    using C = WarpNF<N, REV>;
     constexpr int NN = C::NN, AGG = C::AGG, NT = C::NT, MT = C::MT, WARPS = C::WARPS, Q = C::Q;
     pdl_prologue();
     if (loop_ended(a.st)) return;
@@ -90,7 +129,8 @@ __global__ void __launch_bounds__(WarpNF<N>::THREADS, WarpNF<N>::CTAS_PER_SM) sc
     const int SW = w.sw, L = WARPS * SW;
     for (int i = tid; i < 3 * NN; i += C::THREADS) {
         const int col = i % N, kk = col >> 3, tt = (col & 7) >> 1, e = col & 1;
-        sW[(i / N) * C::WS + tt * 2 * NT + 2 * kk + e] = a.Wh[i];
+        if (!REV) sW[(i / N) * C::WS + tt * 2 * NT + 2 * kk + e] = a.Wh[i];
+        else sW[(i / N) * C::WS + (col & 7) * NT + kk] = a.Wh[i];
     }
     const bool d0 = g == 2 * t, d1 = g == 2 * t + 1;      // this lane's pieces touch the diagonal where nn == kk
 
@@ -163,18 +203,23 @@ __global__ void __launch_bounds__(WarpNF<N>::THREADS, WarpNF<N>::CTAS_PER_SM) sc
         const size_t tile_index = (size_t)seq * w.nch + c;
         const float *Cseq = a.J + (size_t)seq * T * 4 * N;      // coefficient rows {k_r, a_z, k_n, z}[N] per position
         const float *bseq = a.b + (size_t)seq * T * N;
-        auto pos_t = [&](int s) -> size_t { return (size_t)s; };
+        // scan position s: forward matrix J[s], vector at s; reverse matrix J[T-s] (identity at s = 0:
+        // coefficient rows {0,0,0,1}), vector at T-1-s
+        auto pos_t = [&](int s) -> size_t { return REV ? (size_t)(T - 1 - s) : (size_t)s; };
         // chain position q -> ring stage q % S (one commit group per call, also past the end)
         auto issue = [&](int q) {
             const int s = sbase + q;
             if (q < cnt) {
                 float *dst = ring + (q % S) * C::STAGE_FLOATS;
-                const float *cs = Cseq + (size_t)s * 4 * N, *bs = bseq + (size_t)s * N;
+                const float *cs = Cseq + (REV ? (size_t)(T - s) : (size_t)s) * 4 * N, *bs = bseq + pos_t(s) * N;
+                const bool ident = REV && s == 0;
 #pragma unroll
                 for (int u = 0; u < (5 * N / 4 + 31) / 32; ++u) {
                     const int j = lane + 32 * u;
-                    if (j < N) cp_async16(dst + 4 * j, cs + 4 * j);
-                    else if (j < N + N / 4) cp_async16(dst + 4 * j, bs + 4 * (j - N));
+                    if (j < N) {
+                        if (ident) *reinterpret_cast<float4 *>(dst + 4 * j) = make_float4(0.0f, 0.0f, 0.0f, 1.0f);
+                        else cp_async16(dst + 4 * j, cs + 4 * j);
+                    } else if (j < N + N / 4) cp_async16(dst + 4 * j, bs + 4 * (j - N));
                 }
             }
             cp_async_commit();
@@ -196,7 +241,7 @@ __global__ void __launch_bounds__(WarpNF<N>::THREADS, WarpNF<N>::CTAS_PER_SM) sc
                 issue(q + S - 1);
                 const float *Ms = ring + (q % S) * C::STAGE_FLOATS;
                 float jp[NT][NT][2], bg[NT], ynew[NT];
-                gen_pieces<N>(jp, Ms, sW, g, t, d0, d1);
+                if constexpr (REV) gen_pieces_rev<N>(jp, Ms, sW, g, t, d0, d1); else gen_pieces<N>(jp, Ms, sW, g, t, d0, d1);
 #pragma unroll
                 for (int nn = 0; nn < NT; ++nn) bg[nn] = Ms[4 * N + 8 * nn + g];
                 chain_step_n<N>(acc, jp);
@@ -290,7 +335,7 @@ __global__ void __launch_bounds__(WarpNF<N>::THREADS, WarpNF<N>::CTAS_PER_SM) sc
                 issue(q + S - 1);
                 const float *Ms = ring + (q % S) * C::STAGE_FLOATS;
                 float jp[NT][NT][2], bg[NT], ynew[NT];
-                gen_pieces<N>(jp, Ms, sW, g, t, d0, d1);
+                if constexpr (REV) gen_pieces_rev<N>(jp, Ms, sW, g, t, d0, d1); else gen_pieces<N>(jp, Ms, sW, g, t, d0, d1);
                 const size_t vb = ((size_t)seq * T + pos_t(s)) * N;
 #pragma unroll
                 for (int nn = 0; nn < NT; ++nn) bg[nn] = Ms[4 * N + 8 * nn + g];

@@ -258,6 +258,12 @@ def test_generated_and_materialised_jacobians_agree_bitwise(bd, n, m, B, T):
     a = bd.deer_gru_eval(p, x, y0)
     b = bd.deer_gru_eval(p, x, y0, flags=bd.DEER_FLAG_MATERIALIZE)
     assert a.status == 0 and (a.iters, a.err) == (b.iters, b.err) and torch.equal(a.y, b.y)
+    # the gradient: reverse scan on J_{t+1}^T built from the same rows (incl. the identity at the last position and dy0)
+    gy = dev(synth.normal(11, "f/gy", (B, T, n)))
+    ga = bd.deer_gru_vjp(p, x, y0, a.y, gy)
+    gb = bd.deer_gru_vjp(p, x, y0, a.y, gy, flags=bd.DEER_FLAG_MATERIALIZE)
+    for k in ga:
+        assert torch.equal(ga[k], gb[k]), k
 
 
 def test_batch_with_sequences_converging_at_different_bodies(bd):
