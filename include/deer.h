@@ -79,7 +79,7 @@ enum {
     DEER_FLAG_MATERIALIZE = 4,  /* deer_gru_eval, n = 16 and 32: have the cell write the Jacobians
                                    J [B,T,n,n] to the workspace and scan them, instead of writing
                                    four coefficient vectors per position from which the scan builds
-                                   J_t itself (the default there; the results are bit-identical) */
+                                   J_t itself (the default there; the two agree to rounding) */
     DEER_FLAG_TCGEN05    = 8    /* n = 64 scans: run the chain product (Eq. 10's matrix half) as
                                    tcgen05.mma in tensor memory instead of register-resident
                                    mma.sync fragments; same results to rounding, currently slower */

@@ -398,6 +398,20 @@ template <int N> static int launch_cell_wide(CellArgs c, cudaStream_t st)
     return DEER_OK;
 }
 
+// coefficient rows + rhs only (the scan builds J_t): the hidden contraction on tensor cores
+template <int N> static int launch_cell_coef_mma(CellArgs c, cudaStream_t st)
+{
+    constexpr size_t SM = sizeof(float) * (2 * (size_t)N * (3 * N + 4) + 3 * N);
+    int rc;
+    if ((rc = opt_in_smem((const void *)cell_coef_mma_kernel<N>, SM)) != DEER_OK) return rc;
+    const size_t total = (size_t)c.B * c.T;
+    const size_t tiles = (total + 127) / 128;
+    const size_t cap = (size_t)num_sms() * 4;
+    const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
+    DEER_KERNEL_PDL("cell_coef_mma_kernel", false, st, cell_coef_mma_kernel<N>, blocks, 256u, SM, c);
+    return DEER_OK;
+}
+
 template <int N> static int launch_cell_small(CellArgs c, cudaStream_t st)
 {
     const size_t total = (size_t)c.B * c.T;
@@ -439,8 +453,8 @@ static int run_cell(CellArgs c, cudaStream_t st)
         }
         if (c.u && (((uintptr_t)c.W_h) & 15) == 0) {
             switch (c.n) {
-            case 16: return launch_cell_wide<16>(c, st);
-            case 32: return launch_cell_wide<32>(c, st);
+            case 16: return launch_cell_wide<16>(c, st);      // (coefficient rows too: measured equal to the tensor-core kernel)
+            case 32: return c.coef_only ? launch_cell_coef_mma<32>(c, st) : launch_cell_wide<32>(c, st);
             case 64: return launch_cell_wide<64>(c, st);
             default: break;
             }
@@ -644,7 +658,7 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     // n = 16, 32: the cell writes coefficient rows and the scan generates J_t itself, unless the caller
     // asks for materialised Jacobians
     const bool gen_J = single && (n == 16 || n == 32) && !(flags & DEER_FLAG_MATERIALIZE) &&
-                       ((((uintptr_t)y | (uintptr_t)y0) & 15) == 0);
+                       ((((uintptr_t)y | (uintptr_t)y0 | (uintptr_t)p->W_h) & 15) == 0);
     if (gen_J) a.Wh = p->W_h;
     {
         StatusBlock init;
@@ -805,7 +819,7 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
     a.st = w.st;
     // n = 16, 32: coefficient rows instead of Jacobians, J_{t+1}^T built in the reverse scan (as in the evaluation)
     const bool gen_J = (n == 16 || n == 32) && !(flags & DEER_FLAG_MATERIALIZE) && scan_is_single_pass(a, w.scan, flags) &&
-                       ((((uintptr_t)y | (uintptr_t)y0) & 15) == 0);
+                       ((((uintptr_t)y | (uintptr_t)y0 | (uintptr_t)p->W_h) & 15) == 0);
     if (gen_J) a.Wh = p->W_h;
     CellArgs c{p->W_h, p->b_h, small ? nullptr : w.u, x, p->W_i, p->b_i, m, y, y0, w.J, nullptr, B, T, n, nullptr,
                gen_J ? 1 : 0};

@@ -216,4 +216,112 @@ __global__ void __launch_bounds__(256) affine_mma_kernel(const float *__restrict
     }
 }
 
+// ------------------------------------------------------------------ a1-a4 for n in {16, 32} when the scan builds J_t itself
+// The cell as one tensor-core contraction with the gate math as its epilogue: [B*T, n] x [n, 3n]
+// (h_prev times W_h^T; the input half u = x W_i^T + b_i comes from affine_mma_kernel) as m16n8k8 TF32 MMAs
+// issued three times on hi/lo splits, warp = 16 positions x all 3n outputs, weights split once per CTA
+// into padded shared memory.  A lane's accumulator fragments hold, for its two positions and each of
+// its columns i, the three bias-free products (W_hr h)_i, (W_hz h)_i, (W_hn h)_i -- the column blocks of
+// the gates are n/8 apart -- so r, z, c, f, the coefficient row {k_r, a_z, k_n, z}_i and
+// rhs_i = f_i - (J h)_i  (J h = z h + a_z W_hz h + k_n W_hn h + k_r W_hr h) follow in registers.
+// Writes 16 n + 4 n bytes per position; no Jacobian.
+template <int N>
+__global__ void __launch_bounds__(256) cell_coef_mma_kernel(CellArgs a)
+{
+    pdl_prologue();
+    if (loop_ended(a.st)) return;
+    constexpr int NOUT = 3 * N, NB = NOUT / 8, NBG = N / 8, NS = NOUT + 4;      // 2 * NS = 8 (mod 32) words
+    extern __shared__ __align__(16) float smw[];
+    float *sBh = smw, *sBl = smw + N * NS, *sb = sBl + N * NS;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    for (int idx = tid; idx < N * NOUT; idx += 256) {
+        const int k = idx / NOUT, c = idx % NOUT;
+        const float v = a.W_h[(size_t)c * N + k];
+        sBh[k * NS + c] = v;
+        sBl[k * NS + c] = v - __uint_as_float(__float_as_uint(v) & 0xffffe000u);
+    }
+    for (int idx = tid; idx < NOUT; idx += 256) sb[idx] = a.b_h[idx];
+    __syncthreads();
+    const size_t total = (size_t)a.B * a.T;
+    const size_t ntiles = (total + 127) / 128;
+    float4 *coef = reinterpret_cast<float4 *>(a.J);
+    for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const size_t p0 = tile * 128 + warp * 16;
+        if (p0 >= total) continue;
+        const size_t rr[2] = {p0 + g, p0 + g + 8};
+        const bool vv[2] = {rr[0] < total, rr[1] < total};
+        const float *hp[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            size_t seq = 0;
+            hp[h] = a.y;
+            if (vv[h]) hp[h] = seq_start(rr[h], a.T, seq) ? a.y0 + seq * N : a.y + (rr[h] - 1) * N;
+        }
+        float acc[NB][4];
+#pragma unroll
+        for (int nn = 0; nn < NB; ++nn) { acc[nn][0] = 0.0f; acc[nn][1] = 0.0f; acc[nn][2] = 0.0f; acc[nn][3] = 0.0f; }
+#pragma unroll
+        for (int k0 = 0; k0 < N; k0 += 8) {
+            // slots t and t+4 of the K step hold k0+2t and k0+2t+1
+            const float2 x0 = vv[0] ? __ldg(reinterpret_cast<const float2 *>(hp[0] + k0 + 2 * t)) : make_float2(0.f, 0.f);
+            const float2 x1 = vv[1] ? __ldg(reinterpret_cast<const float2 *>(hp[1] + k0 + 2 * t)) : make_float2(0.f, 0.f);
+            unsigned ah[4], al[4];
+            split_tf32(x0.x, ah[0], al[0]);
+            split_tf32(x1.x, ah[1], al[1]);
+            split_tf32(x0.y, ah[2], al[2]);
+            split_tf32(x1.y, ah[3], al[3]);
+            const float *bh0 = sBh + (k0 + 2 * t) * NS + g, *bl0 = sBl + (k0 + 2 * t) * NS + g;
+#pragma unroll
+            for (int nn = 0; nn < NB; ++nn) {
+                unsigned bh[2], bl[2];
+                bh[0] = __float_as_uint(bh0[8 * nn]); bh[1] = __float_as_uint(bh0[8 * nn + NS]);
+                bl[0] = __float_as_uint(bl0[8 * nn]); bl[1] = __float_as_uint(bl0[8 * nn + NS]);
+                mma_tf32(acc[nn], al, bh, acc[nn]);
+                mma_tf32(acc[nn], ah, bl, acc[nn]);
+                mma_tf32(acc[nn], ah, bh, acc[nn]);
+            }
+        }
+        // ---- epilogue: gates, coefficient rows, rhs for (position rr[h], columns 8nn+2t, 8nn+2t+1)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if (!vv[h]) continue;
+            const size_t e = rr[h];
+            const float *ue = a.u + e * NOUT;
+#pragma unroll
+            for (int nn = 0; nn < NBG; ++nn) {
+                const int i0 = 8 * nn + 2 * t;
+                const float2 ur2 = __ldg(reinterpret_cast<const float2 *>(ue + i0));
+                const float2 uz2 = __ldg(reinterpret_cast<const float2 *>(ue + N + i0));
+                const float2 un2 = __ldg(reinterpret_cast<const float2 *>(ue + 2 * N + i0));
+                const float2 h2 = __ldg(reinterpret_cast<const float2 *>(hp[h] + i0));
+                float out_rhs[2];
+#pragma unroll
+                for (int el = 0; el < 2; ++el) {
+                    const int i = i0 + el;
+                    const float sr = acc[nn][2 * h + el], sz = acc[nn + NBG][2 * h + el], sq = acc[nn + 2 * NBG][2 * h + el];
+                    const float ur = el ? ur2.y : ur2.x, uz = el ? uz2.y : uz2.x, un = el ? un2.y : un2.x;
+                    const float hi = el ? h2.y : h2.x;
+                    const float qn = sq + sb[2 * N + i];                 // q = W_hn h + b_hn
+                    const float r = sigmoidf_acc(ur + (sr + sb[i]));
+                    const float z = sigmoidf_acc(uz + (sz + sb[N + i]));
+                    const float c = tanhf(un + r * qn);
+                    const float f = (1.0f - z) * c + z * hi;
+                    const float az = (hi - c) * z * (1.0f - z);
+                    const float an = (1.0f - z) * (1.0f - c * c);
+                    const float kr = an * qn * r * (1.0f - r);
+                    const float kn = an * r;
+                    coef[e * N + i] = make_float4(kr, az, kn, z);
+                    float jh = z * hi;
+                    jh = fmaf(az, sz, jh);
+                    jh = fmaf(kn, sq, jh);
+                    jh = fmaf(kr, sr, jh);
+                    out_rhs[el] = f - jh;
+                }
+                if (a.rhs) *reinterpret_cast<float2 *>(a.rhs + e * N + i0) = make_float2(out_rhs[0], out_rhs[1]);
+            }
+        }
+    }
+}
+
 }  // namespace deer

@@ -249,21 +249,27 @@ def test_eval_diagnostics_of_the_last_body(bd, n, m, B, T, k):
 
 
 @pytest.mark.parametrize("n,m,B,T", [(16, 16, 3, 900), (32, 32, 2, 700), (16, 5, 2, 333), (32, 8, 1, 65)])
-def test_generated_and_materialised_jacobians_agree_bitwise(bd, n, m, B, T):
-    """n = 16, 32: by default the scan builds J_t from the coefficient rows the cell writes; with
-    DEER_FLAG_MATERIALIZE the cell writes J itself.  Same formula, same order of operations: same bits."""
-    p = bd.GruParamsDev.from_numpy(synth.gru_params(n, m, 11, tag="f/gru"))
-    x = dev(synth.x_gaussian(B, T, m, 11, tag="f/x"))
-    y0 = dev(synth.normal(11, "f/y0", (B, n)) * 0.3)
+def test_generated_and_materialised_jacobians_agree(bd, n, m, B, T):
+    """n = 16, 32: by default the cell (hidden contraction on tensor cores, 3 x TF32) writes coefficient rows
+    and the scans build J_t / J_{t+1}^T from them; with DEER_FLAG_MATERIALIZE the fp32-pipe cell writes J itself.
+    Two implementations of the same path: they agree to rounding, and both match the oracle."""
+    p_np = synth.gru_params(n, m, 11, tag="f/gru")
+    x_np = synth.x_gaussian(B, T, m, 11, tag="f/x")
+    y0_np = synth.normal(11, "f/y0", (B, n)) * 0.3
+    p = bd.GruParamsDev.from_numpy(p_np)
+    x, y0 = dev(x_np), dev(y0_np)
     a = bd.deer_gru_eval(p, x, y0)
     b = bd.deer_gru_eval(p, x, y0, flags=bd.DEER_FLAG_MATERIALIZE)
-    assert a.status == 0 and (a.iters, a.err) == (b.iters, b.err) and torch.equal(a.y, b.y)
-    # the gradient: reverse scan on J_{t+1}^T built from the same rows (incl. the identity at the last position and dy0)
+    seq = oracle.gru_seq(p_np, x_np, y0_np, np.float32)
+    assert a.status == 0 and b.status == 0 and a.iters == b.iters
+    assert np.max(np.abs(a.y.cpu().numpy() - seq)) <= TOL_Y and np.max(np.abs(b.y.cpu().numpy() - seq)) <= TOL_Y
+    assert float((a.y - b.y).abs().max()) <= 2e-6
     gy = dev(synth.normal(11, "f/gy", (B, T, n)))
     ga = bd.deer_gru_vjp(p, x, y0, a.y, gy)
     gb = bd.deer_gru_vjp(p, x, y0, a.y, gy, flags=bd.DEER_FLAG_MATERIALIZE)
     for k in ga:
-        assert torch.equal(ga[k], gb[k]), k
+        ref = gb[k].cpu().numpy()
+        assert np.max(np.abs(ga[k].cpu().numpy() - ref)) <= 1e-4 * max(1e-30, float(np.max(np.abs(ref)))), k
 
 
 def test_batch_with_sequences_converging_at_different_bodies(bd):
