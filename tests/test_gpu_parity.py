@@ -364,7 +364,7 @@ def test_config3_gradient_full_size(bd):
 
 
 # ----------------------------------------------------------------------------- classifier
-@pytest.mark.parametrize("B,T,n,m", [(3, 200, 8, 3), (4, 1500, 64, 6), (32, 17984, 64, 6)])
+@pytest.mark.parametrize("B,T,n,m", [(3, 200, 8, 3), (4, 1500, 64, 6), (32, 17984, 64, 6), (2, 300, 16, 5), (2, 150, 32, 4)])
 def test_classifier_step_matches_oracle(bd, B, T, n, m):
     w = synth.config4(seed=2, B=B, T=T, n=n, m=m)
     want = oracle.classifier(w.layers, w.W_o, w.b_o, w.x, w.labels, np.float64)
