@@ -113,6 +113,12 @@ __device__ __forceinline__ void cp_async16(void *dst, const void *src)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
 
+// 4-byte asynchronous copy global -> shared (for sources without 16-byte alignment)
+__device__ __forceinline__ void cp_async4(void *dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_0() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
@@ -584,8 +590,11 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS, 3) scan_onepass_kernel(Sc
                 if (jbulk) bulk_g2s(jd, Jt_src, jb, bar);
                 if (bbulk) bulk_g2s(bd, bt_src, bb, bar);
             }
-            if (!jbulk) for (int i = tid; i < jcnt_tile * NN; i += C::THREADS) jd[i] = __ldg(Jt_src + i);
-            if (!bbulk) for (int i = tid; i < Lt * N; i += C::THREADS) bd[i] = __ldg(bt_src + i);
+            // sources that are not 16-byte aligned (the reverse scan of n = 1 reads J one element on): 4-byte
+            // asynchronous copies, one instruction per element and no registers in between
+            if (!jbulk) for (int i = tid; i < jcnt_tile * NN; i += C::THREADS) cp_async4(jd + i, Jt_src + i);
+            if (!bbulk) for (int i = tid; i < Lt * N; i += C::THREADS) cp_async4(bd + i, bt_src + i);
+            cp_async_commit();
         }
         // B item: while the copies fly, warp 1 fetches the state entering the tile ({value, flag} words)
         if (kind == 1 && warp == 1) {
@@ -605,6 +614,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS, 3) scan_onepass_kernel(Sc
             }
             if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
         }
+        cp_async_wait_0();      // this thread's 4-byte copies, if any
         {
             unsigned spins = 0;
             while (!mbar_try_wait(bar, phase)) {
