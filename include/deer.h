@@ -21,8 +21,12 @@
  *     unless stated.
  *   - Return value: a deer_status.  >= 0 are outcomes of a run that executed,
  *     < 0 mean nothing (or nothing useful) was computed.  Nothing aborts,
- *     throws or traps.  Every device-side wait is bounded and reports
- *     DEER_ERR_DEVICE_TIMEOUT instead of hanging.
+ *     throws or traps.  Every device-side wait is bounded: when one expires
+ *     the kernels drain and raise a flag in the workspace's status block.
+ *     The entry points that synchronise (deer_gru_eval*, deer_gru_classifier_step)
+ *     return DEER_ERR_DEVICE_TIMEOUT themselves; the asynchronous ones
+ *     (deer_linrec_scan*, deer_gru_vjp) return before the kernels have run, so
+ *     their caller asks with deer_workspace_status / deer_noalloc_status.
  *   - Batch index b, position t, 0-based.  y[b][-1] = y0[b].
  *   - Supported hidden sizes: 1 <= n <= 64 (tuned kernels for n in
  *     {1, 2, 4, 8, 16, 32, 64}, a generic kernel for the rest); 1 <= m <= 1024.
@@ -80,9 +84,16 @@ enum {
                                    J [B,T,n,n] to the workspace and scan them, instead of writing
                                    four coefficient vectors per position from which the scan builds
                                    J_t itself (the default there; the two agree to rounding) */
-    DEER_FLAG_TCGEN05    = 8    /* n = 64 scans: run the chain product (Eq. 10's matrix half) as
+    DEER_FLAG_TCGEN05    = 8,   /* n = 64 scans: run the chain product (Eq. 10's matrix half) as
                                    tcgen05.mma in tensor memory instead of register-resident
                                    mma.sync fragments; same results to rounding, currently slower */
+    DEER_FLAG_EXPIRE_WAITS = 16, /* test aid for the bounded waits of the single-pass scans: the
+                                   CTAs that publish the states entering each tile return at once
+                                   and every wait gives up after a few polls, so the scan drains
+                                   and the call reports DEER_ERR_DEVICE_TIMEOUT (outputs invalid).
+                                   Nothing traps or hangs; the workspace can be used again */
+    DEER_FLAG_COEF_ROWS  = 32   /* deer_gru_cell_jac, n = 16 and 32: write the four coefficient
+                                   vectors per position instead of the matrices (see there) */
 };
 
 /* Bytes of workspace needed by `op` at the given sizes (0 if the sizes are
@@ -101,7 +112,9 @@ size_t deer_workspace_bytes(int op, int B, int T, int n, int m, int flags);
  *      operator" of Sec. 3.1.1; J[b][0] is not read).
  *   J  [B,T,n,n]  row = output component        b  [B,T,n]
  *   y0 [B,n] or NULL (= zeros)                  y  [B,T,n] out (must not alias J or b)
- * Asynchronous on `stream`.  Returns DEER_OK or a negative status. */
+ * Asynchronous on `stream`: the return value covers argument checks and launches
+ * only; deer_workspace_status(ws, stream) tells whether the kernels ran to the end.
+ * Returns DEER_OK or a negative status. */
 int deer_linrec_scan(const float *J, const float *b, const float *y0, int B, int T, int n,
                      int reverse, float *y, void *ws, size_t ws_bytes, int flags, void *stream);
 
@@ -125,10 +138,48 @@ int deer_linrec_scan(const float *J, const float *b, const float *y0, int B, int
  *     call left in it; the entry point clears the words that must start at zero
  *     itself.  Two calls that overlap on the GPU (different streams, no ordering
  *     between them) would race on the array: order them.
- * Asynchronous on `stream`.  Returns DEER_OK or a negative status. */
+ * Asynchronous on `stream` (deer_noalloc_status tells whether the kernels ran to
+ * the end).  Returns DEER_OK or a negative status. */
 #define DEER_NOALLOC_SCRATCH_BYTES (8u << 20)
 int deer_linrec_scan_noalloc(const float *J, const float *b, const float *y0, int B, int T, int n,
                              int reverse, float *y, void *stream);
+
+/* Outcome of the last asynchronous call (deer_linrec_scan, deer_gru_vjp) that used
+ * workspace `ws`: synchronises `stream`, reads the status block at the head of the
+ * workspace and returns DEER_OK, or DEER_ERR_DEVICE_TIMEOUT when a bounded wait of
+ * that call's kernels expired (its outputs are then invalid).  No counterpart in the
+ * paper: failure reporting of this implementation's scan (Eq. 9-10). */
+int deer_workspace_status(const void *ws, void *stream);
+
+/* The same for the last deer_linrec_scan_noalloc call on the current device. */
+int deer_noalloc_status(void *stream);
+
+/* Launch geometry the scan (Eq. 9-10: chunked, chunk aggregates combined, applied back
+ * down) would use for these sizes on the current device, for tests and tuning:
+ *   out[0] 1: single-pass kernels, 0: three-kernel (reduce / carry / apply) path
+ *          (taken for other n, DEER_FLAG_GENERIC, unaligned buffers -- not visible
+ *          here -- and batches too large for the single-pass resolvers)
+ *   out[1] positions per tile (chunk)      out[2] positions per warp chain where the
+ *          kernel chooses it at launch (n = 8, 16, 32), else 0
+ *   out[3] tiles per sequence              out[4] resolver CTAs (single-pass)
+ *   out[5] SM count the choice was made for
+ * `out` is a host array of 6 ints.  Returns DEER_OK or a negative status. */
+int deer_scan_geometry(int B, int T, int n, int flags, int *out);
+
+/* The steps of one Newton body before the solve, on their own (Eq. 3 with Eq. 5;
+ * App. B.1: function evaluation, Jacobian, rhs): at every position of the guess y,
+ * with y_prev[b][t] = t ? y[b][t-1] : y0[b],
+ *     J[b][t]   = df/dy_prev (y_prev, x[b][t])            [B,T,n,n] out, row = output
+ *     rhs[b][t] = f(y_prev, x[b][t]) - J[b][t] y_prev     [B,T,n]   out
+ * by the kernel deer_gru_eval uses for these sizes (DEER_FLAG_GENERIC: the any-n kernel).
+ * With DEER_FLAG_COEF_ROWS (n = 16, 32, 16-byte aligned buffers) J receives instead the
+ * coefficient rows [B,T,n,4] = {k_r, a_z, k_n, z} from which the scans of deer_gru_eval
+ * build J = diag(k_r) W_hr + diag(a_z) W_hz + diag(k_n) W_hn + diag(z) themselves.
+ *   ws : workspace of deer_workspace_bytes(DEER_OP_EVAL, ...) bytes (holds x W_i^T + b_i)
+ * Asynchronous on `stream`.  Returns DEER_OK or a negative status. */
+int deer_gru_cell_jac(const deer_gru_params *params, const float *x, const float *y0, const float *y,
+                      int B, int T, float *J, float *rhs, void *ws, size_t ws_bytes, int flags,
+                      void *stream);
 
 /* Evaluate the GRU over whole sequences with the DEER iteration (Eq. 3 with
  * G = -df/dy, Eq. 5; loop of App. B.1): starting from y = 0 (or the guess in
@@ -186,12 +237,13 @@ int deer_gru_eval_host(const deer_gru_params *params, const float *x_host, const
  *   y  [B,T,n] trajectory (normally deer_gru_eval's output)   gy [B,T,n]
  *   dparams : device arrays, overwritten       dx  [B,T,m] or NULL
  *   dy0 [B,n] or NULL
- * Asynchronous on `stream`.  Returns DEER_OK or a negative status. */
+ * Asynchronous on `stream` (see deer_workspace_status).  Returns DEER_OK or a
+ * negative status. */
 int deer_gru_vjp(const deer_gru_params *params, const float *x, const float *y0, const float *y,
                  const float *gy, int B, int T, const deer_gru_grads *dparams, float *dx,
                  float *dy0, void *ws, size_t ws_bytes, int flags, void *stream);
 
-/* One training step of the long-series classifier (App. B.2 shapes: mean
+/* One training step of the long-series classifier (App. B.3 shapes: mean
  * over the sequence, then a linear decoder and cross-entropy): two stacked
  * GRU layers of equal hidden size n (layer 1 reads x [B,T,m], layer 2 reads
  * layer 1's states), zero initial states, p = mean_t y2, logits = W_o p + b_o,
@@ -200,7 +252,8 @@ int deer_gru_vjp(const deer_gru_params *params, const float *x, const float *y0,
  *   W_o [n_classes, n]  b_o [n_classes]  labels [B] int32 (device)
  *   loss : host out      iters : host out [2] (may be NULL)
  *   g1, g2 : parameter gradients per layer;  dW_o [n_classes,n], db_o [n_classes] device out
- * Synchronises `stream`.  Returns the worst status of the two evaluations. */
+ * Synchronises `stream`.  Returns the worst status of the two evaluations, or
+ * DEER_ERR_DEVICE_TIMEOUT when a bounded wait expired in either backward pass. */
 int deer_gru_classifier_step(const deer_gru_params *layer1, const deer_gru_params *layer2,
                              const float *W_o, const float *b_o, int n_classes, const float *x,
                              const int *labels, int B, int T, float tol, int max_iter,

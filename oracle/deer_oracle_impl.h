@@ -350,7 +350,7 @@ void FN(oracle_deer_grad_)(int n, int m, const REAL *W_i, const REAL *W_h, const
  * O-5  Long-series classifier: two stacked GRU layers (layer 2 reads layer
  * 1's output), mean over t of the layer-2 states, linear head, softmax
  * cross-entropy averaged over the batch; sequential forward and BPTT.
- * (App. B.2: mean over the sequence, then a decoder to 5 classes.)
+ * (App. B.3: mean over the sequence, then a decoder to 5 classes.)
  * Gradient arrays are overwritten.  Pinned by finite differences.
  * ------------------------------------------------------------------------ */
 REAL FN(oracle_classifier_)(int n, int m, int ncls, const REAL *W_i1, const REAL *W_h1,

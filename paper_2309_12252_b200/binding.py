@@ -21,11 +21,13 @@ DEER_ERR_INVALID_ARG, DEER_ERR_UNSUPPORTED_N, DEER_ERR_WORKSPACE = -1, -2, -3
 DEER_ERR_CUDA, DEER_ERR_DEVICE_TIMEOUT = -4, -5
 DEER_OP_EVAL, DEER_OP_SCAN, DEER_OP_VJP, DEER_OP_CLASSIFIER = 0, 1, 2, 3
 DEER_FLAG_WARM_START, DEER_FLAG_GENERIC, DEER_FLAG_MATERIALIZE, DEER_FLAG_TCGEN05 = 1, 2, 4, 8
+DEER_FLAG_EXPIRE_WAITS, DEER_FLAG_COEF_ROWS = 16, 32
 
 NOALLOC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc", "deer_gru_eval",
            "deer_gru_eval_diag", "deer_gru_eval_host", "deer_gru_vjp",
-           "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count"]
+           "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count",
+           "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_cell_jac"]
 
 
 class _Params(ctypes.Structure):
@@ -74,6 +76,14 @@ def lib():
                                                ci, vp, vp, ci, ci, cf, ci, ctypes.POINTER(cf),
                                                ctypes.POINTER(ci), ctypes.POINTER(_Grads),
                                                ctypes.POINTER(_Grads), vp, vp, vp, sz, ci, vp]
+        L.deer_workspace_status.restype = ci
+        L.deer_workspace_status.argtypes = [vp, vp]
+        L.deer_noalloc_status.restype = ci
+        L.deer_noalloc_status.argtypes = [vp]
+        L.deer_scan_geometry.restype = ci
+        L.deer_scan_geometry.argtypes = [ci, ci, ci, ci, ctypes.POINTER(ci)]
+        L.deer_gru_cell_jac.restype = ci
+        L.deer_gru_cell_jac.argtypes = [ctypes.POINTER(_Params), vp, vp, vp, ci, ci, vp, vp, vp, sz, ci, vp]
         L.deer_status_string.restype = ctypes.c_char_p
         L.deer_status_string.argtypes = [ci]
         L.deer_last_error.restype = ctypes.c_char_p
@@ -171,6 +181,41 @@ def deer_linrec_scan(J, b, y0=None, reverse=False, y=None, ws=None, flags=0, str
     if check and rc != DEER_OK:
         raise DeerError(rc)
     return y if check else (y, rc)
+
+
+def deer_workspace_status(ws, stream=None) -> int:
+    """Outcome of the last asynchronous call on workspace ``ws`` (synchronises the stream)."""
+    return int(lib().deer_workspace_status(_ptr(ws), _stream(stream)))
+
+
+def deer_noalloc_status(stream=None) -> int:
+    return int(lib().deer_noalloc_status(_stream(stream)))
+
+
+def deer_scan_geometry(B: int, T: int, n: int, flags: int = 0) -> dict:
+    """Launch geometry of the scan for these sizes on the current device; see include/deer.h."""
+    out = (ctypes.c_int * 6)()
+    rc = lib().deer_scan_geometry(B, T, n, flags, out)
+    if rc != DEER_OK:
+        raise DeerError(rc)
+    return dict(single_pass=bool(out[0]), tile_len=out[1], chain_len=out[2], tiles_per_seq=out[3],
+                resolver_ctas=out[4], sms=out[5])
+
+
+def deer_gru_cell_jac(params: "GruParamsDev", x, y0, y, flags=0, ws=None, stream=None):
+    """Cell Jacobians (or coefficient rows with DEER_FLAG_COEF_ROWS) and rhs at the guess y; see include/deer.h."""
+    B, T, m = x.shape
+    n = params.n
+    J = torch.empty((B, T, n, 4 if flags & DEER_FLAG_COEF_ROWS else n), dtype=torch.float32, device=x.device)
+    rhs = torch.empty((B, T, n), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = alloc_workspace(DEER_OP_EVAL, B, T, n, m, 0, x.device)
+    ps = params.c_struct()
+    rc = lib().deer_gru_cell_jac(ctypes.byref(ps), _ptr(_f32(x)), _ptr(_f32(y0)), _ptr(_f32(y)), B, T, _ptr(J),
+                                 _ptr(rhs), _ptr(ws), ws.numel(), flags, _stream(stream))
+    if rc != DEER_OK:
+        raise DeerError(rc)
+    return J, rhs
 
 
 def deer_linrec_scan_noalloc(J, b, y0=None, reverse=False, y=None, stream=None, check=True):

@@ -116,6 +116,9 @@ struct ScanArgs {
     StatusBlock *st;
     const float *Wh;     // [3n,n] hidden weights when J holds coefficient rows [B,T,n,4] instead of
                          // matrices (the scan generates J_t itself); nullptr otherwise
+    unsigned spin_limit; // polls a bounded wait makes before it gives up (0: the default, SPIN_LIMIT)
+    int no_resolve;      // 1: resolver CTAs return at once, so every wait for an entering state runs
+                         // out (DEER_FLAG_EXPIRE_WAITS; exercises the timeout path, nothing else)
 };
 
 struct CellArgs {

@@ -150,6 +150,40 @@ static int scan_prep(const ScanArgs &a, const OnePassWs &w, cudaStream_t st)
     return DEER_OK;
 }
 
+// Resolver warps per resolver CTA x sequences one warp can serve, for the kernel that scans size n.
+static int resolver_cta_capacity(int n, bool umma)
+{
+    switch (n) {
+    case 1: return OnePass<1>::WARPS * OnePass<1>::MAX_SEQ_PER_WARP;
+    case 2: return OnePass<2>::WARPS * OnePass<2>::MAX_SEQ_PER_WARP;
+    case 4: return OnePass<4>::WARPS * OnePass<4>::MAX_SEQ_PER_WARP;
+    case 8: return Warp8::RES_WARPS * OnePass<8>::MAX_SEQ_PER_WARP;
+    case 16: return WarpN<16>::RES_WARPS * WarpN<16>::MAX_SEQ_PER_WARP;
+    case 32: return WarpN<32>::RES_WARPS * WarpN<32>::MAX_SEQ_PER_WARP;
+    case 64: return umma ? Umma64::RES_WARPS * Umma64::MAX_SEQ_PER_WARP : Cta64::RES_WARPS * Cta64::MAX_SEQ_PER_WARP;
+    default: return 0;
+    }
+}
+
+// Resolver CTAs of a single-pass launch: one warp per sequence up to res_cap CTAs, then several
+// sequences per warp, and as many CTAs as the batch needs at max_seq_per_warp sequences per warp.
+static int resolver_ctas(int B, int res_warps, int max_seq_per_warp, int res_cap)
+{
+    int R = (B + res_warps - 1) / res_warps;
+    if (R > res_cap) R = res_cap;
+    const int per_cta_cap = res_warps * max_seq_per_warp;
+    const int need = (B + per_cta_cap - 1) / per_cta_cap;
+    return need > R ? need : R;
+}
+
+// Resolver CTAs only spin; the workers that feed them must be resident beside them.  At least one CTA
+// per SM is resident whatever the kernel, so the single-pass path is taken only while the resolvers a
+// batch needs fit a quarter of the SMs; larger batches use the three-level scan.
+static long long single_pass_max_batch(int n, bool umma)
+{
+    return (long long)(num_sms() / 4) * resolver_cta_capacity(n, umma);
+}
+
 struct PassCfg {
     const char *name;
     int threads;
@@ -181,11 +215,11 @@ static int launch_single_pass(Kern kern, int (&occ_dev)[MAX_DEVICES], const Pass
     }
     const size_t tiles = (size_t)a.B * w.nch;
     const size_t resident = (size_t)num_sms() * occ;
-    // resolver CTAs: one warp per sequence up to res_cap CTAs, then several sequences per warp
-    int R = (a.B + c.res_warps - 1) / c.res_warps;
-    if (R > c.res_cap) R = c.res_cap;
-    const int per_cta_cap = c.res_warps * c.max_seq_per_warp;
-    if ((a.B + per_cta_cap - 1) / per_cta_cap > R) R = (a.B + per_cta_cap - 1) / per_cta_cap;
+    const int R = resolver_ctas(a.B, c.res_warps, c.max_seq_per_warp, c.res_cap);
+    if ((size_t)R * 4 > resident) {      // (scan_is_single_pass keeps such batches off this path)
+        snprintf(t_err, sizeof(t_err), "single-pass scan: %d resolver CTAs for %zu resident", R, resident);
+        return DEER_ERR_INVALID_ARG;
+    }
     w.resolvers = R;
     const size_t want = tiles + (size_t)R;
     unsigned grid = (unsigned)(want < resident ? want : resident);
@@ -316,13 +350,20 @@ static int scan_generic(ScanArgs a, cudaStream_t st)
 static bool scan_is_single_pass(const ScanArgs &a, const ScanWs &w, int flags)
 {
     const bool aligned = (((uintptr_t)a.J | (uintptr_t)a.b | (uintptr_t)a.y) & 15) == 0;
-    return !(flags & DEER_FLAG_GENERIC) && w.op.nch > 0 && aligned;
+    return !(flags & DEER_FLAG_GENERIC) && w.op.nch > 0 && aligned &&
+           a.B <= single_pass_max_batch(a.n, (flags & DEER_FLAG_TCGEN05) != 0);
 }
 
 // prep: clear the single-pass scan's words first (false when the previous scan on this workspace
 // left them cleared)
+static void apply_test_flags(ScanArgs &a, int flags)
+{
+    if (flags & DEER_FLAG_EXPIRE_WAITS) { a.spin_limit = 4u; a.no_resolve = 1; }
+}
+
 static int run_scan(ScanArgs a, const ScanWs &w, int flags, cudaStream_t st, bool prep = true)
 {
+    apply_test_flags(a, flags);
     if (scan_is_single_pass(a, w, flags)) return scan_onepass(a, w.op, prep, flags, st);
     return scan_generic(a, st);
 }
@@ -440,10 +481,10 @@ static bool cell_projects(int n, int m)
     return (n == 1 || n == 2 || n == 4 || n == 8) && (m == 1 || m == 2 || m == 4 || m == 8);
 }
 
-static int run_cell(CellArgs c, cudaStream_t st)
+static int run_cell(CellArgs c, cudaStream_t st, bool generic = false)
 {
     const bool aligned = (((uintptr_t)c.y | (uintptr_t)c.y0 | (uintptr_t)c.J) & 15) == 0;
-    if (aligned) {
+    if (aligned && !generic) {
         switch (c.n) {
         case 1: return launch_cell_small<1>(c, st);
         case 2: return launch_cell_small<2>(c, st);
@@ -660,6 +701,7 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     const bool gen_J = single && (n == 16 || n == 32) && !(flags & DEER_FLAG_MATERIALIZE) &&
                        ((((uintptr_t)y | (uintptr_t)y0 | (uintptr_t)p->W_h) & 15) == 0);
     if (gen_J) a.Wh = p->W_h;
+    apply_test_flags(a, flags);
     {
         StatusBlock init;
         memset(&init, 0, sizeof(init));
@@ -1041,14 +1083,24 @@ int deer_gru_classifier_step(const deer_gru_params *l1, const deer_gru_params *l
     // zero states again (gyB is about to be overwritten by dx of layer 2): use pooled' neighbour
     float *zero1 = w.pool_partial;   // >= B*n floats, no longer needed
     DEER_CHECK_CUDA(cudaMemsetAsync(zero1, 0, (size_t)B * n * sizeof(float), st), "memset y0");
+    // the backward passes are asynchronous and share one status block: the flags word of each is
+    // saved beside the loss before the next call clears it, and both are read after the final sync
+    const unsigned *vflags = &reinterpret_cast<const StatusBlock *>(w.inner)->flags;
     rc = deer_gru_vjp(l2, w.y1, zero1, w.y2, w.gyA, B, T, g2, w.gyB, nullptr, w.inner, w.inner_bytes,
                       flags, stream);
     if (rc != DEER_OK) return rc;
+    DEER_CHECK_CUDA(cudaMemcpyAsync(w.loss + 1, vflags, sizeof(unsigned), cudaMemcpyDeviceToDevice, st), "save status");
     rc = deer_gru_vjp(l1, x, zero1, w.y1, w.gyB, B, T, g1, nullptr, nullptr, w.inner, w.inner_bytes,
                       flags, stream);
     if (rc != DEER_OK) return rc;
-    DEER_CHECK_CUDA(cudaMemcpyAsync(loss, w.loss, sizeof(float), cudaMemcpyDeviceToHost, st), "read loss");
+    DEER_CHECK_CUDA(cudaMemcpyAsync(w.loss + 2, vflags, sizeof(unsigned), cudaMemcpyDeviceToDevice, st), "save status");
+    float tail[3];
+    DEER_CHECK_CUDA(cudaMemcpyAsync(tail, w.loss, sizeof(tail), cudaMemcpyDeviceToHost, st), "read loss");
     DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+    unsigned f1, f2;
+    memcpy(&f1, &tail[1], sizeof(unsigned)); memcpy(&f2, &tail[2], sizeof(unsigned));
+    if ((f1 | f2) & FLAG_TIMEOUT) return DEER_ERR_DEVICE_TIMEOUT;
+    *loss = tail[0];
     return s1 > s2 ? s1 : s2;
 }
 
@@ -1072,6 +1124,78 @@ int deer_linrec_scan_noalloc(const float *J, const float *b, const float *y0, in
     // words, counters) with stream-ordered memsets on every call; nothing else is read before written
     return linrec_scan_impl(J, b, y0, B, T, n, reverse, y, scratch, sizeof(g_noalloc_scratch), 0,
                             (cudaStream_t)stream);
+}
+
+static int status_from_block(const void *block, cudaStream_t st)
+{
+    StatusBlock hs;
+    DEER_CHECK_CUDA(cudaMemcpyAsync(&hs, block, 32, cudaMemcpyDeviceToHost, st), "read status");
+    DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+    return (hs.flags & FLAG_TIMEOUT) ? DEER_ERR_DEVICE_TIMEOUT : DEER_OK;
+}
+
+int deer_workspace_status(const void *ws, void *stream)
+{
+    if (!ws || ((uintptr_t)ws & 255) != 0) return DEER_ERR_WORKSPACE;
+    return status_from_block(ws, (cudaStream_t)stream);
+}
+
+int deer_noalloc_status(void *stream)
+{
+    void *scratch = nullptr;
+    int rc = noalloc_scratch_for_current_device(&scratch);
+    if (rc != DEER_OK) return rc;
+    return status_from_block(scratch, (cudaStream_t)stream);
+}
+
+int deer_scan_geometry(int B, int T, int n, int flags, int *out)
+{
+    if (!out || B <= 0 || T <= 0 || n <= 0) return DEER_ERR_INVALID_ARG;
+    if (!supported(n, 1)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, n, 1)) return DEER_ERR_INVALID_ARG;
+    const bool umma = (flags & DEER_FLAG_TCGEN05) != 0;
+    int sw = 0;
+    const int L1 = onepass_tile_len(n, B, T, &sw);
+    const bool single = L1 > 0 && !(flags & DEER_FLAG_GENERIC) && B <= single_pass_max_batch(n, umma);
+    if (single) {
+        int res_warps = 0, max_seq = 0, res_cap = 8;
+        switch (n) {
+        case 1: case 2: case 4: res_warps = n == 4 ? OnePass<4>::WARPS : OnePass<1>::WARPS; max_seq = OnePass<1>::MAX_SEQ_PER_WARP; break;
+        case 8: res_warps = Warp8::RES_WARPS; max_seq = OnePass<8>::MAX_SEQ_PER_WARP; break;
+        case 16: case 32: res_warps = WarpN<16>::RES_WARPS; max_seq = WarpN<16>::MAX_SEQ_PER_WARP; break;
+        default: res_warps = umma ? Umma64::RES_WARPS : Cta64::RES_WARPS; max_seq = Cta64::MAX_SEQ_PER_WARP; res_cap = umma ? 8 : 16; break;
+        }
+        out[0] = 1; out[1] = L1; out[2] = sw; out[3] = (T + L1 - 1) / L1;
+        out[4] = resolver_ctas(B, res_warps, max_seq, res_cap);
+    } else {
+        const int L = gen_chunk_len(T);
+        out[0] = 0; out[1] = L; out[2] = 0; out[3] = (T + L - 1) / L; out[4] = 0;
+    }
+    out[5] = num_sms();
+    return DEER_OK;
+}
+
+int deer_gru_cell_jac(const deer_gru_params *p, const float *x, const float *y0, const float *y, int B, int T,
+                      float *J, float *rhs, void *ws, size_t ws_bytes, int flags, void *stream)
+{
+    if (!p || !x || !y0 || !y || !J || !rhs || !p->W_i || !p->W_h || !p->b_i || !p->b_h) return DEER_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || p->n <= 0 || p->m <= 0) return DEER_ERR_INVALID_ARG;
+    if (!supported(p->n, p->m)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
+    const int n = p->n, m = p->m;
+    const bool coef = (flags & DEER_FLAG_COEF_ROWS) != 0;
+    if (coef && !(n == 16 || n == 32)) return DEER_ERR_UNSUPPORTED_N;
+    if (coef && (flags & DEER_FLAG_GENERIC)) return DEER_ERR_INVALID_ARG;
+    if (coef && ((((uintptr_t)y | (uintptr_t)y0 | (uintptr_t)J | (uintptr_t)p->W_h) & 15) != 0)) return DEER_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    EvalWs w = carve_eval(ws, B, T, n, m);
+    int rc = check_ws(ws, ws_bytes, w.bytes);
+    if (rc != DEER_OK) return rc;
+    const bool generic = (flags & DEER_FLAG_GENERIC) != 0;
+    const bool fused_proj = !generic && cell_projects(n, m) && ((((uintptr_t)y | (uintptr_t)y0 | (uintptr_t)J) & 15) == 0);
+    if (!fused_proj && (rc = run_proj(p, x, w.u, (size_t)B * T, st)) != DEER_OK) return rc;
+    CellArgs c{p->W_h, p->b_h, fused_proj ? nullptr : w.u, x, p->W_i, p->b_i, m, y, y0, J, rhs, B, T, n, nullptr, coef ? 1 : 0};
+    return run_cell(c, st, generic);
 }
 
 const char *deer_status_string(int s)

@@ -40,6 +40,7 @@ template <int K> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 // is staged per step (16.6 KB).
 __device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
 {
+    if (a.no_resolve) return;     // (wait-expiry test: nobody publishes entering states)
     using C = Cta64;
     constexpr int N = C::N, AGG = C::AGG, NN = C::NN;
     float *stage = stage_all + (threadIdx.x >> 5) * (AGG + N);
@@ -70,6 +71,7 @@ __device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_a
             const int s = rw + k * nrw;
             const unsigned *flags = w.flags + (size_t)s * w.nch;
             const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
+            __syncwarp();      // orders every lane's aggregate loads below after the acquiring lanes' flag loads
             const int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
             if (cnt == 0) {
                 fnext[k] = (c0 + lane < w.nch) ? ld_acquire_u32(flags + c0 + lane) : 0u;
@@ -117,7 +119,7 @@ __device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_a
             else fnext[k] = (pos[k] + lane < w.nch) ? ld_acquire_u32(flags + pos[k] + lane) : 0u;
         }
         if (progressed) spins = 0;
-        else if (!keep_spinning(a.st, spins)) return;
+        else if (!keep_spinning(a, spins)) return;
     }
 }
 
@@ -379,7 +381,7 @@ __global__ void __launch_bounds__(Cta64::THREADS) scan_cta64_kernel(ScanArgs a, 
                     st_relaxed_u64(w.starts + tile_index * N + tid, 0ull);      // consumed: cleared for the next launch
                     break;
                 }
-                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+                if (!keep_spinning(a, spins)) { ok = false; break; }
             }
             if (!ok) s_abort = 1;
         }

@@ -235,7 +235,7 @@ __global__ void __launch_bounds__(OnePass<4>::THREADS, 5) scan_hold4_kernel(Scan
                     }
                     break;
                 }
-                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+                if (!keep_spinning(a, spins)) { ok = false; break; }
             }
             if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
         }

@@ -368,11 +368,14 @@ template <int N> __device__ __forceinline__ void ragg_apply(const RegAgg<N> &r, 
 }
 
 // Flag polling shared by workers and resolvers: true while the run should go on.
-__device__ __forceinline__ bool keep_spinning(StatusBlock *st, unsigned &spins)
+// The limit is SPIN_LIMIT unless the launch carries its own (a.spin_limit: used by the test that makes
+// a wait run out).
+__device__ __forceinline__ bool keep_spinning(const ScanArgs &a, unsigned &spins)
 {
     __nanosleep(64);
-    if (++spins > SPIN_LIMIT) { atomicOr(&st->flags, FLAG_TIMEOUT); return false; }
-    if ((spins & 255u) == 0 && (*(volatile unsigned *)&st->flags & FLAG_TIMEOUT)) return false;
+    const unsigned limit = a.spin_limit ? a.spin_limit : SPIN_LIMIT;
+    if (++spins > limit) { atomicOr(&a.st->flags, FLAG_TIMEOUT); return false; }
+    if ((spins & 255u) == 0 && (*(volatile unsigned *)&a.st->flags & FLAG_TIMEOUT)) return false;
     return true;
 }
 
@@ -385,6 +388,7 @@ constexpr unsigned long long LL_FLAG = 1ull << 32;     // "entering state presen
 template <int N>
 __device__ void resolver_ll_loop(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
 {
+    if (a.no_resolve) return;     // (wait-expiry test: nobody publishes entering states)
     using C = OnePass<N>;
     constexpr int AGG = C::AGG, NN = N * N;
     constexpr int WIN = 16;                         // tiles looked at per visit
@@ -460,7 +464,7 @@ __device__ void resolver_ll_loop(const ScanArgs &a, const OnePassWs &w, float *s
             if (pos[k] >= w.nch) --remaining;
         }
         if (progressed) spins = 0;
-        else if (!keep_spinning(a.st, spins)) return;
+        else if (!keep_spinning(a, spins)) return;
     }
 }
 
@@ -610,7 +614,7 @@ __global__ void __launch_bounds__(OnePass<N>::THREADS, 3) scan_onepass_kernel(Sc
                     }
                     break;
                 }
-                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+                if (!keep_spinning(a, spins)) { ok = false; break; }
             }
             if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
         }

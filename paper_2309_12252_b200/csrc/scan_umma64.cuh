@@ -517,7 +517,7 @@ __global__ void __launch_bounds__(Umma64::THREADS) scan_umma64_kernel(ScanArgs a
                     st_relaxed_u64(w.starts + tile_index * N + tid, 0ull);      // consumed: cleared for the next launch
                     break;
                 }
-                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+                if (!keep_spinning(a, spins)) { ok = false; break; }
             }
             if (!ok) s_abort = 1;
         }

@@ -103,6 +103,7 @@ __device__ __forceinline__ void chain_step(float (&acc)[4], float j0, float j1, 
 // of beta[r] and two shuffles that hand the new pair to every lane (about a dozen instructions).
 __device__ void resolver_loop8(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
 {
+    if (a.no_resolve) return;     // (wait-expiry test: nobody publishes entering states)
     constexpr int N = 8, NN = 64, AGG = 72, MAXS = OnePass<8>::MAX_SEQ_PER_WARP;
     float *stage = stage_all + (threadIdx.x >> 5) * 32 * AGG;
     const int r = lane >> 2, p = lane & 3;
@@ -132,6 +133,7 @@ __device__ void resolver_loop8(const ScanArgs &a, const OnePassWs &w, float *sta
             const int s = rw + k * nrw;
             const unsigned *flags = w.flags + (size_t)s * w.nch;
             const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
+            __syncwarp();      // orders every lane's aggregate loads below after the acquiring lanes' flag loads
             const int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
             {
                 const int j = c0 + cnt + lane;
@@ -171,7 +173,7 @@ __device__ void resolver_loop8(const ScanArgs &a, const OnePassWs &w, float *sta
             if (pos[k] >= w.nch) --remaining;
         }
         if (progressed) spins = 0;
-        else if (!keep_spinning(a.st, spins)) return;
+        else if (!keep_spinning(a, spins)) return;
     }
 }
 
@@ -382,7 +384,7 @@ __global__ void __launch_bounds__(Warp8::THREADS, 4) scan_warp8_kernel(ScanArgs 
                     }
                     break;
                 }
-                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+                if (!keep_spinning(a, spins)) { ok = false; break; }
             }
             if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
         }

@@ -56,6 +56,7 @@ template <int N> struct WarpN {
 template <int N>
 __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
 {
+    if (a.no_resolve) return;     // (wait-expiry test: nobody publishes entering states)
     using C = WarpN<N>;
     constexpr int AGG = C::AGG, NN = C::NN, BATCH = C::RES_BATCH;
     float *stage = stage_all + (threadIdx.x >> 5) * BATCH * AGG;
@@ -85,6 +86,7 @@ __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage
             const int s = rw + k * nrw;
             const unsigned *flags = w.flags + (size_t)s * w.nch;
             const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
+            __syncwarp();      // orders every lane's aggregate loads below after the acquiring lanes' flag loads
             int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
             if (cnt > BATCH) cnt = BATCH;
             {
@@ -133,7 +135,7 @@ __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage
             if (pos[k] >= w.nch) --remaining;
         }
         if (progressed) spins = 0;
-        else if (!keep_spinning(a.st, spins)) return;
+        else if (!keep_spinning(a, spins)) return;
     }
 }
 
@@ -488,7 +490,7 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS, WarpN<N>::CTAS_PER_SM) scan
                     }
                     break;
                 }
-                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+                if (!keep_spinning(a, spins)) { ok = false; break; }
             }
             if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
         }

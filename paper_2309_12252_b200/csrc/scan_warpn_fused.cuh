@@ -290,7 +290,7 @@ __global__ void __launch_bounds__(WarpNF<N, REV>::THREADS, WarpNF<N, REV>::CTAS_
                     }
                     break;
                 }
-                if (!keep_spinning(a.st, spins)) { ok = false; break; }
+                if (!keep_spinning(a, spins)) { ok = false; break; }
             }
             if (!__all_sync(0xffffffffu, ok)) s_abort = 1;
         }

@@ -19,7 +19,7 @@ Generator (documented so that any other implementation can reproduce it):
 The workloads mirror the shapes and value distributions of the paper's GRU
 speed benchmark (Sec. 4.1: untrained GRU, random fp32 inputs, batch 16, zero
 initial state) and of its long-series classification task (Sec. 4.3 /
-App. B.2: 17,984 samples, 6 channels, 5 classes), for which seeded random
+App. B.3: 17,984 samples, 6 channels, 5 classes), for which seeded random
 walks stand in for the dataset.
 """
 from __future__ import annotations

@@ -55,3 +55,30 @@ def test_status_strings_and_argument_validation(L):
     assert L.deer_gru_vjp(None, None, None, None, None, 1, 1, None, None, None, None, 0, 0, None) == -1
     L.deer_launch_count.restype = ctypes.c_longlong
     assert L.deer_launch_count() == 0
+
+
+def test_scan_geometry_bounds_the_resolver_ctas(L):
+    """The single-pass scans give the first role tickets to resolver CTAs, which only spin: a batch
+    that would need more of them than a quarter of the SMs must take the three-kernel path instead
+    (host logic only; with no device the SM count falls back to 148)."""
+    geo = (ctypes.c_int * 6)()
+    for n in (1, 2, 4, 8, 16, 32, 64):
+        last_single = 0
+        for B in (1, 16, 100, 500, 1000, 1184, 1185, 2368, 2369, 5000, 20000, 100000):
+            assert L.deer_scan_geometry(B, 3, n, 0, geo) == 0
+            single, tile, chain, tiles, res, sms = list(geo)
+            assert sms > 0 and tile > 0 and tiles == (3 + tile - 1) // tile
+            if single:
+                assert 1 <= res and 4 * res <= sms, (n, B, res)
+                last_single = B
+            else:
+                assert res == 0
+        assert last_single >= 500                       # ordinary batches stay on the single-pass kernels
+        assert L.deer_scan_geometry(100000, 3, n, 0, geo) == 0 and geo[0] == 0
+    assert L.deer_scan_geometry(16, 1000, 5, 0, geo) == 0 and geo[0] == 0      # other n: three-kernel path
+    assert L.deer_scan_geometry(16, 1000, 8, 2, geo) == 0 and geo[0] == 0      # DEER_FLAG_GENERIC
+    assert L.deer_scan_geometry(0, 1000, 8, 0, geo) == -1 and L.deer_scan_geometry(1, 1, 65, 0, geo) == -2
+    # chain lengths the n = 8 kernel takes at benchmark sizes (148 SMs)
+    if geo[5] == 148:
+        for T, want in ((10000, 40), (40000, 64), (80000, 128), (120000, 256), (1000000, 256)):
+            assert L.deer_scan_geometry(16, T, 8, 0, geo) == 0 and geo[2] == want, (T, list(geo))

@@ -171,7 +171,7 @@ def test_P8_reverse_scan_is_adjoint_of_forward():
 
 def test_P10_n1_matches_cumprod_form():
     """n = 1: y_t = P_t (y0 + sum_k b_k / P_k), P_t = prod_{k<=t} a_k
-    (integrating-factor form, App. A.4) on well-conditioned coefficients."""
+    (integrating-factor form, App. A.5) on well-conditioned coefficients."""
     T = 60
     a = synth.uniform(8, "t/a", (1, T, 1, 1), 0.7, 1.1, dtype=np.float64)
     b = synth.normal(8, "t/b1", (1, T, 1)).astype(np.float64)
