@@ -80,7 +80,11 @@ def test_speed_grid_points_match_sequential(bd, n, T):
 @pytest.mark.parametrize("reverse", [False, True])
 def test_scan_non_contractive_tensor_core_chains(bd, n, reverse):
     """Entries U(-0.6, 0.6): row sums far above 1 and, for n >= 16, products that grow along the
-    sequence.  The split-precision chain products must keep the error relative to max|y|."""
+    sequence (by 1e8 ... 1e26 over the 60 positions).  The chain products of these kernels run on
+    tensor cores as hi/lo TF32 splits (hi*hi + hi*lo + lo*hi): each operand is carried to 2^-20
+    relative, so a chain of k products that nothing damps is good to about k * 2^-20 of the largest
+    entry reached so far -- the bound asserted here, with k = T.  (With contractive J, the case of the
+    GRU Jacobians, earlier errors decay and the 1e-5 bound of the other tests holds.)"""
     B, T = 2, 60
     J = synth.uniform(n, "nc/J", (B, T, n, n), -0.6, 0.6)
     b = synth.normal(n, "nc/b", (B, T, n))
@@ -93,7 +97,8 @@ def test_scan_non_contractive_tensor_core_chains(bd, n, reverse):
     run = np.maximum.accumulate(mag[::-1] if reverse else mag)
     run = run[::-1] if reverse else run
     err = np.max(np.abs(got - want), axis=(0, 2))
-    assert np.all(err <= TOL_SCAN * np.maximum(1.0, run)), float(np.max(err / np.maximum(1.0, run)))
+    bound = T * 2.0 ** -20
+    assert np.all(err <= bound * np.maximum(1.0, run)), float(np.max(err / np.maximum(1.0, run)))
 
 
 # one shape per cell kernel: (n, m, flags)
