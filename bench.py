@@ -2,11 +2,15 @@
 """Benchmark of the DEER-GRU hot path on B200.
 
 One "step" = one whole `deer_gru_eval` (input projection + all Newton bodies:
-cell + Jacobian + rhs, scan, convergence) over the benchmark workload
-(GRU n=8, m=4, B=16, T=10,000, fp32, sinusoid+noise inputs, zero initial
-state and zero initial guess).  `value` = B*T positions evaluated per second,
-inputs resident in HBM; `e2e` = the same through the host-buffer call with
-the H2D copy of x and the D2H copy of y inside the timed region.
+cell + Jacobian + rhs, scan, convergence) over the headline workload, the
+largest single-GPU configuration of the benchmark definition that is a forward
+evaluation: config 3 (GRU n=32, m=32, B=16, T=100,000, fp32, x ~ N(0,1), zero
+initial state and zero initial guess).  `value` = B*T positions evaluated per
+second with the inputs resident in HBM; `e2e` = the same through the
+host-buffer call (`deer_gru_eval_host`) with the H2D copy of x and the D2H copy
+of y inside the timed region.  The same JSON line carries, as extra keys, the
+other workloads of the definition (config 2, the config-4 training step) and
+the stand-alone scans on HBM-sized inputs (n = 4 ... 64) with their rooflines.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -14,6 +18,9 @@ N > 1 (under torchrun): every rank evaluates its own batch of the same shape
 (sequences are independent: no data-path collective), weak scaling; the timed
 region is bracketed by barriers and the maximum over ranks is reported.
 `--impl reference` times the CPU oracle's sequential fp32 loop instead.
+Other modes (`--mode scan|eval|sweep|classifier`) print one JSON line each for
+a single measurement; every input is drawn from the documented seeded streams
+of `paper_2309_12252_b200.synth` (on the device through `synth_device`).
 """
 from __future__ import annotations
 
@@ -32,9 +39,16 @@ if ROOT not in sys.path:
 
 METRIC = "DEER GRU B*T steps/s"
 UNIT = "steps/s"
-WORKLOAD = dict(workload="config2: GRU n=8 m=4 B=16 T=10000 fp32, x=sin(wt+phi)+0.1N(0,1), y0=0, zero guess",
-                n=8, m=4, B=16, T=10000, tol=1e-4, max_iter=100)
-SCAN_HBM = dict(n=8, B=16, T=1_000_000)     # stand-alone scan sized well beyond L2 (J = 4.1 GB)
+WORKLOADS = {
+    2: dict(workload="config2: GRU n=8 m=4 B=16 T=10000 fp32, x=sin(wt+phi)+0.1N(0,1), y0=0, zero guess",
+            n=8, m=4, B=16, T=10000, tol=1e-4, max_iter=100),
+    3: dict(workload="config3: GRU n=32 m=32 B=16 T=100000 fp32, x~N(0,1), y0=0, zero guess",
+            n=32, m=32, B=16, T=100000, tol=1e-4, max_iter=100),
+}
+HEADLINE = 3
+# stand-alone scans sized well beyond L2 (J of 1 ... 9.4 GB): where the HBM roofline claims are taken
+SCANS_HBM = [dict(n=4, B=16, T=1_000_000), dict(n=8, B=16, T=1_000_000), dict(n=16, B=16, T=200_000),
+             dict(n=32, B=16, T=100_000), dict(n=64, B=32, T=17_984)]
 
 
 def peaks():
@@ -46,24 +60,65 @@ def peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
 
 
-# DRAM bytes (read + write) per position of the stand-alone scan, from the ncu captures summarised in
-# profiles/scan_kernels_standalone_B16.md (inputs larger than L2; traffic grows in proportion to positions).
-NCU_STEP_SCAN_TRAFFIC = 51.43e6      # config-2 step, scan_warp8_kernel: dram read + write per launch
+def tf32_peak_tflops(pk) -> float:
+    """Dense TF32 tensor peak: the measured bf16 burst figure times the nominal TF32/bf16 ratio (1.1 / 2.25 PFLOP/s)."""
+    return pk["bf16_tflops"] * (1.1 / 2.25)
+
+
+# DRAM bytes (read + write) per position from the ncu captures summarised under profiles/ (inputs larger
+# than L2; traffic grows in proportion to the positions processed, so a launch's traffic is this times B*T).
 NCU_SCAN_TRAFFIC_PER_POSITION = {1: 12.8, 2: 32.7, 4: 95.3, 8: 606.6, 16: 2213.0, 32: 8622.0, 64: 34116.0}
+NCU_FUSED_SCAN_TRAFFIC_PER_POSITION = {32: 1375.0}      # scan_warpnf_kernel<32> inside deer_gru_eval
+NCU_CONFIG2_SCAN_TRAFFIC = 51.43e6                      # scan_warp8_kernel inside the config-2 step, per launch
 
 
 def scan_bytes_per_position(n: int) -> int:
-    """Algorithmic bytes of one scan per position: read J and b once, write y."""
+    """Algorithmic bytes of one stand-alone scan per position: read J and b once, write y."""
     return 4 * (n * n + n) + 4 * n
 
 
-class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+def fused_scan_bytes_per_position(n: int) -> int:
+    """The scan inside deer_gru_eval for n = 16, 32 (J generated from four coefficient vectors per position):
+    read the coefficient rows (16n), the right-hand side (4n) and the previous iterate (4n), write y (4n)."""
+    return 28 * n
 
-    def __init__(self, index: int, period: float = 0.01):
+
+def scan_flops_per_position(n: int) -> int:
+    """Chunk reduce of Eq. 9: one n x n by n x (n+1) product per position (apply adds 2n^2, counted with it)."""
+    return 2 * n * n * (n + 1)
+
+
+def roofline_of_scan(n, positions, ms, pk, bytes_per_position, traffic_per_position, kernel, extra=None):
+    """The slower of the byte bound (measured HBM copy rate) and the flop bound (TF32 tensor peak) is the scan's
+    roofline; `frac` = that bound's time / measured time, `achieved` in the unit of the binding resource."""
+    t_bytes = bytes_per_position * positions / (pk["hbm_gbs"] * 1e9) * 1e3
+    tf32 = tf32_peak_tflops(pk)
+    t_flops = scan_flops_per_position(n) * positions / (tf32 * 1e12) * 1e3
+    hbm_bound = t_bytes >= t_flops
+    gbs = bytes_per_position * positions / (ms * 1e-3) / 1e9
+    tfs = scan_flops_per_position(n) * positions / (ms * 1e-3) / 1e12
+    out = dict(bound="hbm" if hbm_bound else "tensor", kernel=kernel,
+               achieved=gbs if hbm_bound else tfs, peak=pk["hbm_gbs"] if hbm_bound else tf32,
+               unit="GB/s" if hbm_bound else "TFLOP/s", frac=(t_bytes if hbm_bound else t_flops) / ms,
+               peak_source=pk["source"] + ("" if hbm_bound else " bf16 burst x 1.1/2.25 (nominal TF32/bf16 ratio)"),
+               ms_per_launch=ms, positions_per_launch=positions, bytes_per_position=bytes_per_position,
+               flops_per_position=scan_flops_per_position(n),
+               hbm_frac=t_bytes / ms, tensor_frac=t_flops / ms, achieved_gbs=gbs, achieved_tflops=tfs,
+               traffic=None if traffic_per_position is None else traffic_per_position * positions)
+    if extra:
+        out.update(extra)
+    return out
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while GPU work runs (read-only).  Samples taken
+    between mark_begin() and mark_end() are also kept apart: those are the timed region's."""
+
+    def __init__(self, index: int, period: float = 0.005):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.timed, self.timed_reasons, self.in_timed = [], set(), False
         self._stop_ev = threading.Event()
         self.ok = False
         try:
@@ -89,20 +144,33 @@ class ClockSampler(threading.Thread):
         get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or nv.nvmlDeviceGetCurrentClocksThrottleReasons
         while not self._stop_ev.is_set():
             try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
                 mask = int(get(self.h))
-                for k, bit in names.items():
-                    if mask & bit:
-                        self.reasons.add(k)
+                hit = {k for k, bit in names.items() if mask & bit}
+                self.samples.append(mhz)
+                self.reasons |= hit
+                if self.in_timed:
+                    self.timed.append(mhz)
+                    self.timed_reasons |= hit
             except Exception:
                 pass
             time.sleep(self.period)
 
+    def mark_begin(self):
+        self.in_timed = True
+
+    def mark_end(self):
+        self.in_timed = False
+
     def stop(self):
         self._stop_ev.set()
         self.join(timeout=2)
-        med = int(np.median(self.samples)) if self.samples else None
-        return dict(sm_mhz=med, sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons), samples=len(self.samples))
+        timed = self.timed or self.samples
+        reasons = self.timed_reasons if self.timed else self.reasons
+        med = int(np.median(timed)) if timed else None
+        return dict(sm_mhz=med, sm_max_mhz=self.max_mhz, reasons=sorted(reasons), samples=len(timed),
+                    whole_run=dict(sm_mhz=int(np.median(self.samples)) if self.samples else None,
+                                   reasons=sorted(self.reasons), samples=len(self.samples)))
 
 
 def physical_gpu_index(local_rank: int) -> int:
@@ -148,7 +216,7 @@ def run_reference(args):
         return
     from paper_2309_12252_b200 import synth
     import oracle
-    w = synth.config(2)
+    w = synth.config(HEADLINE)
     for _ in range(max(args.warmup, 1)):
         oracle.gru_seq(w.params, w.x, w.y0, np.float32)
     t0 = time.perf_counter()
@@ -159,7 +227,7 @@ def run_reference(args):
     cores = min(oracle.num_threads(), w.B)
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
                 ms_per_step=1e3 * dt / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
-                dtype="f32", data="synthetic", impl="reference", config=dict(WORKLOAD),
+                dtype="f32", data="synthetic", impl="reference", config=dict(WORKLOADS[HEADLINE]),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle",
                                   sample=f"{args.steps} full passes of the sequential fp32 GRU loop over the whole workload"),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
@@ -184,6 +252,42 @@ def read_profile(bd):
     return parse_profile(buf.value.decode())
 
 
+def is_scan_kernel(name: str) -> bool:
+    return (name.startswith("scan_") and "prep" not in name) or name.startswith("gen_")
+
+
+def scan_inputs(n, B, T, device, seed=0):
+    """Stand-alone scan inputs from the documented streams: contractive J (entries U(+-0.9/n)), b ~ N(0,1)."""
+    from paper_2309_12252_b200 import synth_device
+    J = synth_device.contractive_J(B, T, n, seed=seed, tag=f"bench/scan{n}/J", scale=0.9, device=device)
+    b = synth_device.normal(seed, f"bench/scan{n}/b", (B, T, n), device=device)
+    return J, b
+
+
+def time_scan(bd, torch, device, n, B, T, reverse, flags, steps, warmup):
+    J, bb = scan_inputs(n, B, T, device)
+    yy = torch.empty_like(bb)
+    ws = bd.alloc_workspace(bd.DEER_OP_SCAN, B, T, n, 1, flags, device)
+    stream = torch.cuda.current_stream()
+    for _ in range(max(warmup, 1)):
+        bd.deer_linrec_scan(J, bb, None, bool(reverse), yy, ws, flags, stream)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    torch.cuda.synchronize()
+    for a, b in ev:
+        a.record(stream)
+        bd.deer_linrec_scan(J, bb, None, bool(reverse), yy, ws, flags, stream)
+        b.record(stream)
+    torch.cuda.synchronize()
+    status = bd.deer_workspace_status(ws, stream)
+    assert status == bd.DEER_OK, bd.deer_status_string(status)
+    return float(np.median([a.elapsed_time(b) for a, b in ev]))
+
+
+def scan_kernel_name(n: int, flags: int = 0) -> str:
+    return {1: "scan_onepass_kernel", 2: "scan_onepass_kernel", 4: "scan_hold4_kernel", 8: "scan_warp8_kernel",
+            16: "scan_warpn_kernel", 32: "scan_warpn_kernel", 64: "scan_umma64_kernel" if flags & 8 else "scan_cta64_kernel"}.get(n, "gen_*")
+
+
 def run_scan_only(args):
     """Stand-alone linear-recurrence scan at the given size: prints one JSON line."""
     import torch
@@ -191,36 +295,23 @@ def run_scan_only(args):
     device = torch.device("cuda", 0)
     torch.cuda.set_device(0)
     n, B, T = args.n, args.B, args.T
-    g = torch.Generator(device=device); g.manual_seed(0)
-    J = (torch.rand((B, T, n, n), device=device, generator=g) * 2 - 1) * (0.9 / n)
-    bb = torch.randn((B, T, n), device=device, generator=g)
-    yy = torch.empty_like(bb)
-    ws = bd.alloc_workspace(bd.DEER_OP_SCAN, B, T, n, 1, args.flags, device)
-    stream = torch.cuda.current_stream()
-    for _ in range(max(args.warmup, 1)):
-        bd.deer_linrec_scan(J, bb, None, bool(args.reverse), yy, ws, args.flags, stream)
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    torch.cuda.synchronize()
-    for a, b in ev:
-        a.record(stream)
-        bd.deer_linrec_scan(J, bb, None, bool(args.reverse), yy, ws, args.flags, stream)
-        b.record(stream)
-    torch.cuda.synchronize()
-    ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+    ms = time_scan(bd, torch, device, n, B, T, args.reverse, args.flags, args.steps, args.warmup)
     pk = peaks()
-    ach = scan_bytes_per_position(n) * B * T / (ms * 1e-3) / 1e9
+    r = roofline_of_scan(n, B * T, ms, pk, scan_bytes_per_position(n), NCU_SCAN_TRAFFIC_PER_POSITION.get(n),
+                         scan_kernel_name(n, args.flags))
     print(json.dumps(dict(mode="scan", n=n, B=B, T=T, reverse=int(args.reverse), flags=args.flags, ms=ms,
-                          positions_per_s=B * T / (ms * 1e-3), achieved_gbs=ach, peak_gbs=pk["hbm_gbs"],
-                          frac=ach / pk["hbm_gbs"], peak_source=pk["source"],
-                          input_mb=(n * n + n) * 4 * B * T / 1e6)))
+                          positions_per_s=B * T / (ms * 1e-3), achieved_gbs=r["achieved_gbs"], peak_gbs=pk["hbm_gbs"],
+                          frac=r["hbm_frac"], tensor_frac=r["tensor_frac"], bound=r["bound"], peak_source=pk["source"],
+                          input_mb=(n * n + n) * 4 * B * T / 1e6, geometry=bd.deer_scan_geometry(B, T, n, args.flags))))
 
 
 def eval_point(bd, synth, device, n, m, B, T, flags, steps, warmup, vjp=False, breakdown=True):
-    """deer_gru_eval (optionally deer_gru_vjp) at one sweep point (x ~ N(0,1), y0 = 0): a dict of timings."""
+    """deer_gru_eval (optionally deer_gru_vjp) at one point of the speed grid (weights and x ~ N(0,1) from the
+    streams of synth.sweep_point, y0 = 0): a dict of timings."""
     import torch
+    from paper_2309_12252_b200 import synth_device
     p = bd.GruParamsDev.from_numpy(synth.gru_params(n, m, 0, tag=f"sweep{n}/gru"))
-    g = torch.Generator(device=device); g.manual_seed(0)
-    x = torch.randn((B, T, m), device=device, generator=g)
+    x = synth_device.normal(0, f"sweep{n}/x", (B, T, m), device=device)
     y0 = torch.zeros((B, n), device=device)
     y = torch.empty((B, T, n), device=device)
     ws = bd.alloc_workspace(bd.DEER_OP_EVAL, B, T, n, m, flags, device)
@@ -243,14 +334,19 @@ def eval_point(bd, synth, device, n, m, B, T, flags, steps, warmup, vjp=False, b
         bd.lib().deer_profile_enable(0)
         prof = read_profile(bd)
         out["kernels"] = {k: dict(launches=v["launches"], ms=round(v["total_ms"], 4)) for k, v in prof.items()}
-        scan_ms = sum(v["total_ms"] for k, v in prof.items() if k.startswith("scan_") and "prep" not in k or k.startswith("gen_"))
+        scan_ms = sum(v["total_ms"] for k, v in prof.items() if is_scan_kernel(k))
         if scan_ms > 0 and r.iters > 0:
             pk = peaks()
             per = scan_ms / r.iters
+            fused = any(k.startswith("scan_warpnf") for k in prof)
+            bpp = fused_scan_bytes_per_position(n) if fused else scan_bytes_per_position(n)
+            rl = roofline_of_scan(n, B * T, per, pk, bpp, None, "+".join(k for k in prof if is_scan_kernel(k)))
             out["scan_ms_per_iter"] = per
-            out["scan_frac_hbm"] = scan_bytes_per_position(n) * B * T / (per * 1e-3) / 1e9 / pk["hbm_gbs"]
+            out["scan_bound"] = rl["bound"]
+            out["scan_frac"] = rl["frac"]
+            out["scan_bytes_per_position"] = bpp
     if vjp:
-        gy = torch.randn((B, T, n), device=device, generator=g)
+        gy = synth_device.normal(0, f"sweep{n}/gy", (B, T, n), device=device)
         del ws
         wsv = bd.alloc_workspace(bd.DEER_OP_VJP, B, T, n, m, flags, device)
         for _ in range(2):
@@ -269,7 +365,7 @@ def eval_point(bd, synth, device, n, m, B, T, flags, steps, warmup, vjp=False, b
 
 
 def run_eval_only(args):
-    """One sweep point chosen on the command line: prints one JSON line."""
+    """One grid point chosen on the command line: prints one JSON line."""
     import torch
     from paper_2309_12252_b200 import binding as bd
     from paper_2309_12252_b200 import synth
@@ -281,37 +377,45 @@ def run_eval_only(args):
     print(json.dumps(out))
 
 
-def run_classifier(args):
-    """Config 4: one full training step (loss + all gradients) of the 2-layer GRU classifier: one JSON line."""
-    import torch
-    from paper_2309_12252_b200 import binding as bd
-    from paper_2309_12252_b200 import synth
-    device = torch.device("cuda", 0)
-    torch.cuda.set_device(0)
-    w = synth.config4(seed=0, B=args.B, T=args.T)
+def time_classifier(bd, synth, torch, device, B, T, flags, steps, warmup, profile=True):
+    """Config 4: full training steps (loss + all gradients) of the 2-layer GRU classifier."""
+    w = synth.config4(seed=0, B=B, T=T)
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
     l1 = bd.GruParamsDev.from_numpy(w.layers[0]); l2 = bd.GruParamsDev.from_numpy(w.layers[1])
     W_o, b_o, x, labels = dev(w.W_o), dev(w.b_o), dev(w.x), dev(w.labels)
     n, m = w.layers[0].n, w.layers[0].m
-    ws = bd.alloc_workspace(bd.DEER_OP_CLASSIFIER, args.B, args.T, n, m, args.flags, device)
+    ws = bd.alloc_workspace(bd.DEER_OP_CLASSIFIER, B, T, n, m, flags, device)
     stream = torch.cuda.current_stream()
-    run = lambda: bd.deer_gru_classifier_step(l1, l2, W_o, b_o, x, labels, ws=ws, flags=args.flags, stream=stream)
-    for _ in range(max(args.warmup, 1)):
+    run = lambda: bd.deer_gru_classifier_step(l1, l2, W_o, b_o, x, labels, ws=ws, flags=flags, stream=stream)
+    for _ in range(max(warmup, 1)):
         r = run()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     torch.cuda.synchronize()
     for a, b in ev:
         a.record(stream); r = run(); b.record(stream)
     torch.cuda.synchronize()
     ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
-    bd.lib().deer_profile_enable(1)
-    run()
-    torch.cuda.synchronize()
-    bd.lib().deer_profile_enable(0)
-    prof = read_profile(bd)
-    print(json.dumps(dict(mode="classifier", B=args.B, T=args.T, n=n, m=m, ms=ms, steps_per_s=args.B * args.T / (ms * 1e-3),
-                          loss=r["loss"], iters=list(r["iters"]), status=r["status"],
-                          kernels={k: dict(launches=v["launches"], ms=round(v["total_ms"], 4)) for k, v in prof.items()})))
+    out = dict(B=B, T=T, n=n, m=m, ms=ms, steps_per_s=B * T / (ms * 1e-3), loss=r["loss"], iters=list(r["iters"]),
+               status=r["status"])
+    if profile:
+        bd.lib().deer_profile_enable(1)
+        run()
+        torch.cuda.synchronize()
+        bd.lib().deer_profile_enable(0)
+        prof = read_profile(bd)
+        out["kernels"] = {k: dict(launches=v["launches"], ms=round(v["total_ms"], 4)) for k, v in prof.items()}
+    return out
+
+
+def run_classifier(args):
+    import torch
+    from paper_2309_12252_b200 import binding as bd
+    from paper_2309_12252_b200 import synth
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    out = time_classifier(bd, synth, torch, device, args.B, args.T, args.flags, args.steps, args.warmup)
+    out["mode"] = "classifier"
+    print(json.dumps(out))
 
 
 def run_sweep(args):
@@ -335,6 +439,113 @@ def run_sweep(args):
     print(json.dumps(dict(mode="sweep", B=16, points=points)))
 
 
+def measure_workload(bd, torch, synth, idx, rank, device, dist, steps, warmup, flush, sampler=None, prof_steps=10):
+    """Whole deer_gru_eval calls on configuration `idx` (each rank its own batch, same weights): device-resident
+    timing, the host-buffer call, and a separate profiled pass for the per-kernel breakdown."""
+    cfg = WORKLOADS[idx]
+    w = synth.config(idx, seed=rank)
+    B, T, n, m = w.B, w.T, w.n, w.m
+    p = bd.GruParamsDev.from_numpy(synth.config(idx, seed=0, B=1, T=1).params)
+    x_host = torch.from_numpy(w.x).pin_memory()
+    y_host = torch.empty((B, T, n), dtype=torch.float32).pin_memory()
+    x = x_host.to(device)
+    y0 = torch.zeros((B, n), device=device)
+    y = torch.empty((B, T, n), device=device)
+    ws = bd.alloc_workspace(bd.DEER_OP_EVAL, B, T, n, m, 0, device)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        return bd.deer_gru_eval(p, x, y0, cfg["tol"], cfg["max_iter"], y, ws, 0, stream)
+
+    def step_host():
+        return bd.deer_gru_eval_host(p, x_host, y0, y_host, x, y, ws, cfg["tol"], cfg["max_iter"], 0, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        r = step()
+    iters = r.iters
+    assert r.status == 0, bd.deer_status_string(r.status)
+
+    # ---- timed region: K steps, L2 flushed before each, per-step CUDA events on the launching stream
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    barrier()
+    if sampler is not None:
+        sampler.mark_begin()
+    launches0 = bd.deer_launch_count()
+    for a, b in ev:
+        flush.fill_(1)
+        a.record(stream)
+        r = step()
+        b.record(stream)
+    barrier()
+    launches = bd.deer_launch_count() - launches0
+    if sampler is not None:
+        sampler.mark_end()
+    local_ms = sum(a.elapsed_time(b) for a, b in ev)
+    total_ms, total_units = aggregate_over_ranks(local_ms, float(steps) * B * T, dist, device)
+
+    # ---- end to end: host buffers, H2D of x and D2H of y inside the timed region
+    for _ in range(3):
+        step_host()
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    barrier()
+    for a, b in ev2:
+        flush.fill_(1)
+        a.record(stream)
+        step_host()
+        b.record(stream)
+    barrier()
+    e2e_ms, e2e_units = aggregate_over_ranks(sum(a.elapsed_time(b) for a, b in ev2), float(steps) * B * T, dist, device)
+
+    # ---- per-kernel breakdown of the same steps (separate pass: event pairs around every launch)
+    prof_steps = min(steps, prof_steps)
+    bd.lib().deer_profile_enable(1)
+    for _ in range(prof_steps):
+        flush.fill_(1)
+        step()
+    torch.cuda.synchronize()
+    bd.lib().deer_profile_enable(0)
+    prof = read_profile(bd)
+    tot = sum(v["total_ms"] for v in prof.values()) or 1.0
+    kernels = {k: dict(launches_per_step=v["launches"] / prof_steps, us_per_launch=1e3 * v["total_ms"] / v["launches"],
+                       share=v["total_ms"] / tot) for k, v in prof.items()}
+    return dict(cfg=cfg, B=B, T=T, n=n, m=m, iters=iters, err=r.err, value=total_units / (total_ms * 1e-3),
+                ms_per_step=total_ms / steps, launches=int(launches),
+                e2e=dict(value=e2e_units / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=int(x_host.numel() * 4),
+                         d2h_bytes_per_step=int(y_host.numel() * 4), ms_per_step=e2e_ms / steps),
+                kernels=kernels, prof=prof, prof_steps=prof_steps)
+
+
+def step_scan_roofline(m, pk):
+    """Roofline of the scan inside the measured step (the dominant kernel), from the profiled pass."""
+    prof = m["prof"]
+    names = [k for k in prof if is_scan_kernel(k)]
+    scan_ms = sum(prof[k]["total_ms"] for k in names)
+    launches = sum(prof[k]["launches"] for k in names if k.startswith("scan_")) or (m["prof_steps"] * m["iters"])
+    if scan_ms <= 0:
+        return None
+    n, positions = m["n"], m["B"] * m["T"]
+    per = scan_ms / launches
+    fused = any(k.startswith("scan_warpnf") for k in names)
+    if fused:
+        return roofline_of_scan(n, positions, per, pk, fused_scan_bytes_per_position(n),
+                                NCU_FUSED_SCAN_TRAFFIC_PER_POSITION.get(n), "+".join(names),
+                                dict(note="scan inside the step, J generated from coefficient rows: bytes = coefficient rows, "
+                                          "rhs, previous iterate read once + y written; flops = 2 n^2 (n+1) per position",
+                                     traffic_note="ncu capture of this kernel at T = 20,000 scaled by positions (profiles/)"))
+    extra = None
+    traffic = NCU_SCAN_TRAFFIC_PER_POSITION.get(n)
+    if m["cfg"] is WORKLOADS[2]:
+        extra = dict(traffic=NCU_CONFIG2_SCAN_TRAFFIC,
+                     note="this workload (46 MB of J, b per body) is L2-resident: an effective rate, not an HBM claim")
+        traffic = None
+    return roofline_of_scan(n, positions, per, pk, scan_bytes_per_position(n) + 4 * n, traffic, "+".join(names), extra)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--mode", default="step", choices=["step", "scan", "eval", "sweep", "classifier"])
@@ -346,11 +557,12 @@ def main():
     ap.add_argument("--reverse", type=int, default=0)
     ap.add_argument("--flags", type=int, default=0)
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="deer", choices=["deer", "reference"])
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
-    ap.add_argument("--no-scan-hbm", action="store_true", help="skip the HBM-sized stand-alone scan measurement")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the other workloads and the HBM-sized stand-alone scans (headline workload only)")
     args = ap.parse_args()
     if args.B is None:
         args.B = 32 if args.mode == "classifier" else 16
@@ -389,137 +601,68 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
     args.warmup = max(args.warmup, 3)
-
-    w = synth.config(2, seed=rank)              # each rank: its own batch of the same shape
-    B, T, n, m = w.B, w.T, w.n, w.m
-    p = bd.GruParamsDev.from_numpy(synth.config(2, seed=0, B=1, T=1).params)   # same weights on every rank
-    x_host = torch.from_numpy(w.x).pin_memory()
-    y_host = torch.empty((B, T, n), dtype=torch.float32).pin_memory()
-    x = x_host.to(device)
-    y0 = torch.zeros((B, n), device=device)
-    y = torch.empty((B, T, n), device=device)
-    ws = bd.alloc_workspace(bd.DEER_OP_EVAL, B, T, n, m, 0, device)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)     # > 126 MB L2
-    stream = torch.cuda.current_stream()
-
-    def step():
-        return bd.deer_gru_eval(p, x, y0, WORKLOAD["tol"], WORKLOAD["max_iter"], y, ws, 0, stream)
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(args.warmup):
-        r = step()
-    iters = r.iters
-    assert r.status == 0, bd.deer_status_string(r.status)
-
-    # ---- timed region: K steps, L2 flushed before each, per-step CUDA events on the launching stream
-    sampler = ClockSampler(physical_gpu_index(local_rank))
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    barrier()
-    sampler.start()
-    launches0 = bd.deer_launch_count()
-    for a, b in ev:
-        flush.fill_(1)
-        a.record(stream)
-        r = step()
-        b.record(stream)
-    barrier()
-    launches = bd.deer_launch_count() - launches0
-    clocks = sampler.stop()
-    local_ms = sum(a.elapsed_time(b) for a, b in ev)
-    total_ms, total_units = aggregate_over_ranks(local_ms, float(args.steps) * B * T, dist, device)
-    value = total_units / (total_ms * 1e-3)
-
-    # ---- end to end: host buffers, H2D of x and D2H of y inside the timed region
-    for _ in range(3):
-        bd.deer_gru_eval_host(p, x_host, y0, y_host, x, y, ws, WORKLOAD["tol"], WORKLOAD["max_iter"], 0, stream)
-    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    barrier()
-    for a, b in ev2:
-        flush.fill_(1)
-        a.record(stream)
-        bd.deer_gru_eval_host(p, x_host, y0, y_host, x, y, ws, WORKLOAD["tol"], WORKLOAD["max_iter"], 0, stream)
-        b.record(stream)
-    barrier()
-    e2e_ms, e2e_units = aggregate_over_ranks(sum(a.elapsed_time(b) for a, b in ev2), float(args.steps) * B * T, dist, device)
-    e2e = dict(value=e2e_units / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=int(x_host.numel() * 4),
-               d2h_bytes_per_step=int(y_host.numel() * 4))
-
-    # ---- per-kernel breakdown of the same steps (separate pass: event pairs around every launch)
-    prof_steps = min(args.steps, 20)
-    bd.lib().deer_profile_enable(1)
-    for _ in range(prof_steps):
-        flush.fill_(1)
-        step()
-    torch.cuda.synchronize()
-    bd.lib().deer_profile_enable(0)
-    prof = read_profile(bd)
-    tot = sum(v["total_ms"] for v in prof.values()) or 1.0
-    kernels = {k: dict(launches_per_step=v["launches"] / prof_steps, us_per_launch=1e3 * v["total_ms"] / v["launches"],
-                       share=v["total_ms"] / tot) for k, v in prof.items()}
     pk = peaks()
-    scan_names = [k for k in prof if ("scan" in k or "reduce" in k or "carry" in k or "apply" in k)]
-    scan_ms = sum(prof[k]["total_ms"] for k in scan_names)
-    scans = prof_steps * iters
-    roofline = None
-    if scan_ms > 0:
-        ach = scan_bytes_per_position(n) * B * T / (scan_ms / scans * 1e-3) / 1e9
-        roofline = dict(bound="hbm", kernel="+".join(scan_names), achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
-                        frac=ach / pk["hbm_gbs"], peak_source=pk["source"], traffic=NCU_STEP_SCAN_TRAFFIC,
-                        traffic_note="DRAM bytes per scan launch of this workload under ncu (caches flushed before each "
-                                     "kernel): one read of J, b, y_old; the second visit of every tile is served by L2 "
-                                     "(profiles/bench_step_config2_launch_list.md)",
-                        note="scan inside the step; this workload (46 MB of J,b per body) is L2-resident, "
-                             "so this is an effective rate; see roofline_scan_hbm for the HBM-sized scan")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)     # > 126 MB L2
 
-    # ---- stand-alone scan on an HBM-sized problem (rank 0 only): the roofline of the dominant kernel
-    roofline_hbm = None
-    if rank == 0 and not args.no_scan_hbm:
-        sn, sB, sT = SCAN_HBM["n"], SCAN_HBM["B"], SCAN_HBM["T"]
-        g = torch.Generator(device=device); g.manual_seed(0)
-        J = (torch.rand((sB, sT, sn, sn), device=device, generator=g) * 2 - 1) * (0.9 / sn)
-        bb = torch.randn((sB, sT, sn), device=device, generator=g)
-        yy = torch.empty_like(bb)
-        sws = bd.alloc_workspace(bd.DEER_OP_SCAN, sB, sT, sn, 1, 0, device)
-        for _ in range(3):
-            bd.deer_linrec_scan(J, bb, None, False, yy, sws, 0, stream)
-        reps = 10
-        se = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
-        torch.cuda.synchronize()
-        for a, b in se:
-            a.record(stream)
-            bd.deer_linrec_scan(J, bb, None, False, yy, sws, 0, stream)
-            b.record(stream)
-        torch.cuda.synchronize()
-        ms = float(np.median([a.elapsed_time(b) for a, b in se]))
-        ach = scan_bytes_per_position(sn) * sB * sT / (ms * 1e-3) / 1e9
-        roofline_hbm = dict(bound="hbm", kernel="deer_linrec_scan", workload=f"n={sn} B={sB} T={sT} (J 4.1 GB, inputs > L2)",
-                            achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
-                            peak_source=pk["source"], ms=ms,
-                            traffic=NCU_SCAN_TRAFFIC_PER_POSITION[sn] * sB * sT,
-                            traffic_note="bytes per launch: ncu capture at T=200000 scaled by positions "
-                                         "(profiles/scan_kernels_standalone_B16.md)",
-                            frac_two_reads=(scan_bytes_per_position(sn) + 4 * (sn * sn + sn)) * sB * sT
-                                           / (ms * 1e-3) / 1e9 / pk["hbm_gbs"])
-        del J, bb, yy, sws
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    head = measure_workload(bd, torch, synth, HEADLINE, rank, device, dist, args.steps, args.warmup, flush, sampler)
+    roofline = step_scan_roofline(head, pk)
+
+    extras = {}
+    scans = None
+    if rank == 0 and not args.no_extras:
+        torch.cuda.empty_cache()
+        # ---- the other forward workload of the definition (L2-resident)
+        c2 = measure_workload(bd, torch, synth, 2, 0, device, None, max(args.steps, 20), args.warmup, flush)
+        extras["config2"] = dict(workload=c2["cfg"]["workload"], value=c2["value"], unit=UNIT, ms_per_step=c2["ms_per_step"],
+                                 newton_iters=c2["iters"], e2e=c2["e2e"], kernels=c2["kernels"],
+                                 roofline=step_scan_roofline(c2, pk))
+        torch.cuda.empty_cache()
+        # ---- config 4: full training step of the 2-layer n = 64 classifier
+        c4 = time_classifier(bd, synth, torch, device, 32, 17_984, 0, 3, 2)
+        scan_ms = sum(v["ms"] for k, v in c4["kernels"].items() if is_scan_kernel(k))
+        scan_launches = sum(v["launches"] for k, v in c4["kernels"].items() if is_scan_kernel(k))
+        extras["config4_training_step"] = dict(
+            workload="config4: 2-layer GRU n=64 m=6 B=32 T=17984, mean-pool, 5-class head; loss + all gradients",
+            ms_per_step=c4["ms"], value=c4["steps_per_s"], unit=UNIT, newton_iters=c4["iters"], loss=c4["loss"],
+            kernels=c4["kernels"],
+            scan_roofline=roofline_of_scan(64, 32 * 17_984, scan_ms / max(scan_launches, 1), pk, scan_bytes_per_position(64),
+                                           NCU_SCAN_TRAFFIC_PER_POSITION[64], "scan_cta64_kernel (forward and reverse)"))
+        torch.cuda.empty_cache()
+        # ---- stand-alone scans on HBM-sized problems: the roofline of each scan kernel
+        scans = []
+        for s in SCANS_HBM:
+            for reverse in (0, 1):
+                ms = time_scan(bd, torch, device, s["n"], s["B"], s["T"], reverse, 0, 10, 3)
+                rl = roofline_of_scan(s["n"], s["B"] * s["T"], ms, pk, scan_bytes_per_position(s["n"]),
+                                      NCU_SCAN_TRAFFIC_PER_POSITION[s["n"]], scan_kernel_name(s["n"]),
+                                      dict(workload=f"n={s['n']} B={s['B']} T={s['T']} reverse={reverse} "
+                                                    f"(J {4 * s['n'] ** 2 * s['B'] * s['T'] / 1e9:.2f} GB, inputs > L2)",
+                                           reverse=reverse, n=s["n"],
+                                           traffic_note="ncu capture of the forward kernel at smaller T scaled by positions (profiles/)"))
+                scans.append(rl)
+                torch.cuda.empty_cache()
+    clocks = sampler.stop()
 
     cpu = None
     if rank == 0 and world == 1:
-        v, reps, dt, cores = cpu_oracle_rate(synth.config(2), args.cpu_seconds)
+        v, reps, dt, cores = cpu_oracle_rate(synth.config(HEADLINE), args.cpu_seconds)
         cpu = dict(value=v, unit=UNIT, cores=cores, kind="oracle",
                    sample=f"{reps} full passes of the oracle's sequential fp32 GRU loop over the whole workload ({dt:.1f} s)")
 
     if rank == 0:
-        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
-                    ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+        hbm8 = next((s for s in (scans or []) if s["n"] == 8 and s["reverse"] == 0), None)
+        line = dict(metric=METRIC, value=head["value"], unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                    ms_per_step=head["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype="f32", data="synthetic",
-                    config=dict(WORKLOAD, global_batch=B * world, parallelism=f"batch-sharded x{world}, no collective",
-                                l2="flushed (256 MiB write) before every timed step"),
-                    newton_iters=iters, err=r.err, gpu_launches=int(launches), clocks=clocks, e2e=e2e,
-                    roofline=roofline, roofline_scan_hbm=roofline_hbm, kernels=kernels, cpu_baseline=cpu)
+                    config=dict(head["cfg"], global_batch=head["B"] * world,
+                                parallelism=f"batch-sharded x{world}, no collective",
+                                l2="flushed (256 MiB write) before every timed step; the step's working set (> 1 GB) exceeds L2"),
+                    newton_iters=head["iters"], err=head["err"], gpu_launches=head["launches"], clocks=clocks,
+                    e2e={k: v for k, v in head["e2e"].items() if k != "ms_per_step"},
+                    roofline=roofline, roofline_scan_hbm=hbm8, roofline_scans_hbm=scans, kernels=head["kernels"],
+                    workloads=extras, cpu_baseline=cpu)
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
