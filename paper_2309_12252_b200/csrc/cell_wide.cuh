@@ -152,11 +152,15 @@ __global__ void __launch_bounds__(256, (N <= 32) ? 4 : 0) cell_wide_kernel(CellA
                     if (a.coef_only) reinterpret_cast<float4 *>(a.J)[e * N + gi] = make_float4(kr, az, kn, z);
                     else sC[p * N + gi] = make_float4(kr, az, kn, z);
                     if (a.rhs) {
-                        float jh = z * hi;
-                        jh = fmaf(az, gz[q], jh);
-                        jh = fmaf(kn, gq[q], jh);
-                        jh = fmaf(kr, gr[q], jh);
-                        a.rhs[e * N + gi] = f - jh;
+                        if (a.residual) {
+                            a.rhs[e * N + gi] = f - a.y[e * N + gi];
+                        } else {
+                            float jh = z * hi;
+                            jh = fmaf(az, gz[q], jh);
+                            jh = fmaf(kn, gq[q], jh);
+                            jh = fmaf(kr, gr[q], jh);
+                            a.rhs[e * N + gi] = f - jh;
+                        }
                     }
                 }
             }

@@ -116,6 +116,8 @@ struct ScanArgs {
     StatusBlock *st;
     const float *Wh;     // [3n,n] hidden weights when J holds coefficient rows [B,T,n,4] instead of
                          // matrices (the scan generates J_t itself); nullptr otherwise
+    int residual;        // 1: Newton-update form (App. A.1): b holds f - y_old, the scan solves for the
+                         // update d_t = J_t d_{t-1} + b_t from d_{-1} = 0 and writes y = y_old + d, err = max|d|
     unsigned spin_limit; // polls a bounded wait makes before it gives up (0: the default, SPIN_LIMIT)
     int no_resolve;      // 1: resolver CTAs return at once, so every wait for an entering state runs
                          // out (DEER_FLAG_EXPIRE_WAITS; exercises the timeout path, nothing else)
@@ -137,6 +139,8 @@ struct CellArgs {
     const StatusBlock *st;   // nullptr, or: skip all work once st->done is set (Newton loop ended)
     int coef_only;           // wide kernels: write the coefficient rows {k_r, a_z, k_n, z} [B,T,n,4] to J
                              // instead of the matrices (the scan generates J_t from them)
+    int residual;            // coefficient-row kernels: rhs receives the residual f - y[t] of the Newton-update
+                             // form (App. A.1) instead of f - J y_prev
 };
 
 // Programmatic dependent launch: a kernel of the Newton loop lets the next launch in the stream be set
@@ -175,7 +179,8 @@ __device__ __forceinline__ void newton_decide(StatusBlock *st, float tol, int ma
 // last CTA to leave rewinds the per-launch counters (the launch leaves its flag and state words
 // cleared as well: every word is cleared by its only reader) and, in loop-control mode, takes the
 // Newton decision, so a body needs no separate control or clearing launch.
-__device__ __forceinline__ void scan_epilogue(StatusBlock *st)
+// decide = false: a launch that is not the last one of its scan (counters are rewound, no decision).
+__device__ __forceinline__ void scan_epilogue(StatusBlock *st, bool decide = true)
 {
     __threadfence();
     const unsigned prev = atomicAdd(&st->exit_counter, 1u);
@@ -184,7 +189,7 @@ __device__ __forceinline__ void scan_epilogue(StatusBlock *st)
     st->exit_counter = 0u;
     st->tile_counter = 0u;
     st->role_counter = 0u;
-    if (st->ctl_mode) newton_decide(st, st->tol, st->max_iter, st->trace);
+    if (decide && st->ctl_mode) newton_decide(st, st->tol, st->max_iter, st->trace);
 }
 
 // Is flat position e = seq * T + t the first of its sequence?  (32-bit division whenever e fits.)
@@ -211,6 +216,29 @@ __device__ __forceinline__ float tanhf_gate(float a)
 {
     const float e = __expf(-2.0f * fabsf(a));            // in (0, 1]
     return copysignf(__fdividef(1.0f - e, 1.0f + e), a);
+}
+
+// Packed pairs of fp32 operations (sm_100: one instruction for two lanes of a 64-bit register pair).
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c)
+{
+    unsigned long long ra, rb, rc, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rc) : "f"(c.x), "f"(c.y));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+__device__ __forceinline__ float2 fmul2(float2 a, float2 b)
+{
+    unsigned long long ra, rb, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
 }
 
 __device__ __forceinline__ unsigned absdiff_bits(float a, float b) {

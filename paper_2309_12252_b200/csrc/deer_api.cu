@@ -17,6 +17,7 @@
 #include "scan_warp8.cuh"
 #include "scan_warpn.cuh"
 #include "scan_warpn_fused.cuh"
+#include "scan_fused_fwd.cuh"
 #include "scan_cta64.cuh"
 #include "scan_umma64.cuh"
 #include "cell_wide.cuh"
@@ -116,6 +117,9 @@ static ScanWs carve_scan(Carver &cv, int B, int T, int n)
         // (n <= 4 publish their aggregates as 64-bit {value, flag} words)
         w.op.aggs = cv.take<float>(tiles * (n * n + n) * (onepass_ll_aggs(n) ? 2 : 1));
         w.op.starts = cv.take<unsigned long long>(tiles * n);
+        w.op.pfx = nullptr;
+        if (n == 16) w.op.pfx = cv.take<float>(tiles * (FusedFwd<16>::WARPS - 1) * FusedFwd<16>::AGG);
+        if (n == 32) w.op.pfx = cv.take<float>(tiles * (FusedFwd<32>::WARPS - 1) * FusedFwd<32>::AGG);
     }
     return w;
 }
@@ -281,6 +285,37 @@ static int launch_warpnf(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
     return launch_single_pass(scan_warpnf_kernel<N, REV>, occ, c, a, w, prep, st);
 }
 
+// forward scan of deer_gru_eval in the Newton-update form, two launches: chunk reduce + carries, then the
+// replay of all chains (16 per warp in lockstep)
+template <int N>
+static int launch_fused_fwd(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
+{
+    using C = FusedFwd<N>;
+    static int occ[MAX_DEVICES] = {0};
+    static int occ_apply[MAX_DEVICES] = {0};
+    const PassCfg c{"scan_fused_reduce_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 8};
+    int rc = launch_single_pass(scan_fused_reduce_kernel<N>, occ, c, a, w, prep, st);
+    if (rc != DEER_OK) return rc;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= MAX_DEVICES) dev = 0;
+    if (!occ_apply[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(scan_fused_apply_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::A_SMEM);
+        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(scan apply)"); return DEER_ERR_CUDA; }
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, scan_fused_apply_kernel<N>, C::A_THREADS, C::A_SMEM);
+        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(scan apply)"); return DEER_ERR_CUDA; }
+        occ_apply[dev] = o;
+    }
+    const long long nchain = (a.T + w.sw - 1) / w.sw;
+    const long long groups = ((long long)a.B * nchain + C::ROWS - 1) / C::ROWS;
+    const long long want = (groups + C::A_WARPS - 1) / C::A_WARPS;
+    const long long resident = (long long)num_sms() * occ_apply[dev];
+    const unsigned grid = (unsigned)(want < resident ? want : resident);
+    DEER_KERNEL_PDL("scan_fused_apply_kernel", false, st, scan_fused_apply_kernel<N>, grid, (unsigned)C::A_THREADS, C::A_SMEM, a, w);
+    return DEER_OK;
+}
+
 template <bool REV>
 static int launch_cta64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
@@ -311,9 +346,11 @@ static int scan_onepass(ScanArgs a, OnePassWs w, bool prep, int flags, cudaStrea
     case 9: return launch_hold4<true>(a, w, prep, st);
     case 16: return launch_warp8<false>(a, w, prep, st);
     case 17: return launch_warp8<true>(a, w, prep, st);
-    case 32: return a.Wh ? launch_warpnf<16, false>(a, w, prep, st) : launch_warpn<16, false>(a, w, prep, st);
+    case 32: return a.Wh ? (a.residual ? launch_fused_fwd<16>(a, w, prep, st) : launch_warpnf<16, false>(a, w, prep, st))
+                         : launch_warpn<16, false>(a, w, prep, st);
     case 33: return a.Wh ? launch_warpnf<16, true>(a, w, prep, st) : launch_warpn<16, true>(a, w, prep, st);
-    case 64: return a.Wh ? launch_warpnf<32, false>(a, w, prep, st) : launch_warpn<32, false>(a, w, prep, st);
+    case 64: return a.Wh ? (a.residual ? launch_fused_fwd<32>(a, w, prep, st) : launch_warpnf<32, false>(a, w, prep, st))
+                         : launch_warpn<32, false>(a, w, prep, st);
     case 65: return a.Wh ? launch_warpnf<32, true>(a, w, prep, st) : launch_warpn<32, true>(a, w, prep, st);
     case 128: return umma ? launch_umma64<false>(a, w, prep, st) : launch_cta64<false>(a, w, prep, st);
     case 129: return umma ? launch_umma64<true>(a, w, prep, st) : launch_cta64<true>(a, w, prep, st);
@@ -700,7 +737,9 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     // asks for materialised Jacobians
     const bool gen_J = single && (n == 16 || n == 32) && !(flags & DEER_FLAG_MATERIALIZE) &&
                        ((((uintptr_t)y | (uintptr_t)y0 | (uintptr_t)p->W_h) & 15) == 0);
-    if (gen_J) a.Wh = p->W_h;
+    // ... and the iteration runs in its Newton-update form: the scan solves for the update from a zero
+    // entering update (its linear solve may then be approximate: single TF32 chain products)
+    if (gen_J) { a.Wh = p->W_h; a.residual = 1; a.y0 = nullptr; }
     apply_test_flags(a, flags);
     {
         StatusBlock init;
@@ -740,7 +779,7 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
         for (int j = 0; j < todo; ++j, ++enq) {
             float *cur = buf[enq & 1], *nxt = buf[(enq + 1) & 1];
             CellArgs c{p->W_h, p->b_h, fused_proj ? nullptr : w.u, x, p->W_i, p->b_i, m, cur, y0, w.J, w.rhs, B, T, n, w.st,
-                       gen_J ? 1 : 0};
+                       gen_J ? 1 : 0, gen_J ? 1 : 0};
             if ((rc = run_cell(c, st)) != DEER_OK) return rc;
             a.y = nxt; a.yold = cur;
             if (single) {

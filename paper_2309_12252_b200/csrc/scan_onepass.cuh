@@ -77,6 +77,8 @@ struct OnePassWs {
     unsigned total_ids;
     int resolvers;                // CTAs that take the resolver role
     int sw;                       // positions per warp chain where the kernel takes it at run time (n = 8)
+    float *pfx;                   // [B*nch][chains per tile - 1][n*n+n] prefix aggregates inside each tile (n = 16, 32:
+                                  // written by the reduce launch of the two-launch scan of deer_gru_eval)
 };
 
 // ---------------------------------------------------------------- small PTX helpers

@@ -256,6 +256,45 @@ __device__ __forceinline__ void chain_step_n(float (&acc)[N / 16][N / 8][4], con
             for (int i = 0; i < 4; ++i) acc[mm][nn][i] = nacc[mm][nn][i];
 }
 
+// X <- X * M with ONE TF32 product per tile (operands truncated to 10 mantissa bits by the tensor core, fp32
+// accumulate: relative error about 1e-3).  Only for the Newton-update form of the iteration, whose fixed
+// point does not depend on the accuracy of the linear solve.
+template <int N>
+__device__ __forceinline__ void chain_step_n1(float (&acc)[N / 16][N / 8][4], const float (&jp)[N / 8][N / 8][2])
+{
+    constexpr int NT = N / 8, MT = N / 16;
+    float nacc[MT][NT][4];
+#pragma unroll
+    for (int mm = 0; mm < MT; ++mm)
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) nacc[mm][nn][i] = 0.0f;
+#pragma unroll
+    for (int kk = 0; kk < NT; ++kk) {
+        unsigned af[MT][4];
+#pragma unroll
+        for (int mm = 0; mm < MT; ++mm) {
+            af[mm][0] = __float_as_uint(acc[mm][kk][0]);
+            af[mm][1] = __float_as_uint(acc[mm][kk][2]);
+            af[mm][2] = __float_as_uint(acc[mm][kk][1]);
+            af[mm][3] = __float_as_uint(acc[mm][kk][3]);
+        }
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn) {
+            const unsigned bf[2] = {__float_as_uint(jp[nn][kk][0]), __float_as_uint(jp[nn][kk][1])};
+#pragma unroll
+            for (int mm = 0; mm < MT; ++mm) mma_tf32(nacc[mm][nn], af[mm], bf, nacc[mm][nn]);
+        }
+    }
+#pragma unroll
+    for (int mm = 0; mm < MT; ++mm)
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[mm][nn][i] = nacc[mm][nn][i];
+}
+
 // y <- M^T-form mat-vec: ynew[nn] = y_new[8nn+g] (in the 4 lanes of group g); yv[kk] = {y[8kk+2t], y[8kk+2t+1]}
 template <int N>
 __device__ __forceinline__ void matvec_step(float (&yv)[N / 8][2], const float (&jp)[N / 8][N / 8][2],
@@ -264,13 +303,11 @@ __device__ __forceinline__ void matvec_step(float (&yv)[N / 8][2], const float (
     constexpr int NT = N / 8;
 #pragma unroll
     for (int nn = 0; nn < NT; ++nn) {
-        float p0 = 0.0f, p1 = 0.0f;
+        float2 p2 = make_float2(0.0f, 0.0f);
 #pragma unroll
-        for (int kk = 0; kk < NT; ++kk) {
-            p0 = fmaf(jp[nn][kk][0], yv[kk][0], p0);
-            p1 = fmaf(jp[nn][kk][1], yv[kk][1], p1);
-        }
-        float part = p0 + p1;
+        for (int kk = 0; kk < NT; ++kk)
+            p2 = ffma2(make_float2(jp[nn][kk][0], jp[nn][kk][1]), make_float2(yv[kk][0], yv[kk][1]), p2);
+        float part = p2.x + p2.y;
         part += __shfl_xor_sync(0xffffffffu, part, 1);
         part += __shfl_xor_sync(0xffffffffu, part, 2);
         ynew[nn] = part + bg[nn];

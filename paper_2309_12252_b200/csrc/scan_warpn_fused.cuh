@@ -8,6 +8,13 @@
 // operand pieces of J_t (forward) or J_{t+1}^T (reverse; identity at the first scan position: coefficient
 // rows {0,0,0,1}) from the staged coefficient rows and W_h kept in shared memory: 3 n^2 FMAs per
 // position and visit on the fp32 pipes in exchange for n/5 times less memory traffic.
+//
+// The forward kernel (inside deer_gru_eval) runs the iteration in its Newton-update form (App. A.1, shown there
+// to be the same iteration as Eq. 3): the cell hands over the residual f - y_old, the scan solves
+// d_t = J_t d_{t-1} + (f - y_old)_t from d_{-1} = 0 and writes y = y_old + d, err = max|d|.  In this form the
+// fixed point is f(y) = y whatever the accuracy of the linear solve, so the chain products of the A item are
+// single TF32 MMAs (no hi/lo split: a third of the tensor work and none of the split instructions); the
+// replay of the B item stays fp32.  The reverse kernel (the gradient's one-shot solve) keeps 3 x TF32.
 #pragma once
 #include "scan_warpn.cuh"
 
@@ -94,12 +101,13 @@ __device__ __forceinline__ void gen_pieces(float (&jp)[N / 8][N / 8][2], const f
             wz[4 * v] = z4.x; wz[4 * v + 1] = z4.y; wz[4 * v + 2] = z4.z; wz[4 * v + 3] = z4.w;
             wn[4 * v] = n4.x; wn[4 * v + 1] = n4.y; wn[4 * v + 2] = n4.z; wn[4 * v + 3] = n4.w;
         }
+        const float2 cx = make_float2(cf.x, cf.x), cy = make_float2(cf.y, cf.y), cz = make_float2(cf.z, cf.z);
 #pragma unroll
         for (int kk = 0; kk < NT; ++kk) {
-            float v0 = fmaf(cf.x, wr[2 * kk], fmaf(cf.y, wz[2 * kk], cf.z * wn[2 * kk]));
-            float v1 = fmaf(cf.x, wr[2 * kk + 1], fmaf(cf.y, wz[2 * kk + 1], cf.z * wn[2 * kk + 1]));
-            if (nn == kk) { v0 += d0 ? cf.w : 0.0f; v1 += d1 ? cf.w : 0.0f; }
-            jp[nn][kk][0] = v0; jp[nn][kk][1] = v1;
+            float2 v = ffma2(cx, make_float2(wr[2 * kk], wr[2 * kk + 1]),
+                             ffma2(cy, make_float2(wz[2 * kk], wz[2 * kk + 1]), fmul2(cz, make_float2(wn[2 * kk], wn[2 * kk + 1]))));
+            if (nn == kk) { v.x += d0 ? cf.w : 0.0f; v.y += d1 ? cf.w : 0.0f; }
+            jp[nn][kk][0] = v.x; jp[nn][kk][1] = v.y;
         }
     }
 }
@@ -244,7 +252,7 @@ __global__ void __launch_bounds__(WarpNF<N, REV>::THREADS, WarpNF<N, REV>::CTAS_
                 if constexpr (REV) gen_pieces_rev<N>(jp, Ms, sW, g, t, d0, d1); else gen_pieces<N>(jp, Ms, sW, g, t, d0, d1);
 #pragma unroll
                 for (int nn = 0; nn < NT; ++nn) bg[nn] = Ms[4 * N + 8 * nn + g];
-                chain_step_n<N>(acc, jp);
+                if constexpr (REV) chain_step_n<N>(acc, jp); else chain_step_n1<N>(acc, jp);
                 matvec_step<N>(yv, jp, bg, ynew, t);
             }
             cp_async_wait_n<0>();
@@ -263,7 +271,7 @@ __global__ void __launch_bounds__(WarpNF<N, REV>::THREADS, WarpNF<N, REV>::CTAS_
                     load_pieces_smem<N>(jp, ak, g, t);
 #pragma unroll
                     for (int nn = 0; nn < NT; ++nn) bg[nn] = ak[NN + 8 * nn + g];
-                    chain_step_n<N>(acc, jp);
+                    if constexpr (REV) chain_step_n<N>(acc, jp); else chain_step_n1<N>(acc, jp);
                     matvec_step<N>(yv, jp, bg, ynew, t);
                 }
                 store_aggregate<N>(w.aggs + tile_index * AGG, acc, yv, g, t);
@@ -343,8 +351,16 @@ __global__ void __launch_bounds__(WarpNF<N, REV>::THREADS, WarpNF<N, REV>::CTAS_
                 if (t == 0) {
 #pragma unroll
                     for (int nn = 0; nn < NT; ++nn) {
-                        if (a.yold) mb = max(mb, absdiff_bits(ynew[nn], __ldg(a.yold + vb + 8 * nn + g)));
-                        a.y[vb + 8 * nn + g] = ynew[nn];
+                        if constexpr (!REV) {
+                            // Newton-update form: the scanned quantity is the update; y = y_old + update
+                            // (err is taken from the two stored iterates, as the diagnostics kernel does)
+                            const float yo = __ldg(a.yold + vb + 8 * nn + g), yn = yo + ynew[nn];
+                            mb = max(mb, absdiff_bits(yn, yo));
+                            a.y[vb + 8 * nn + g] = yn;
+                        } else {
+                            if (a.yold) mb = max(mb, absdiff_bits(ynew[nn], __ldg(a.yold + vb + 8 * nn + g)));
+                            a.y[vb + 8 * nn + g] = ynew[nn];
+                        }
                     }
                 }
             }

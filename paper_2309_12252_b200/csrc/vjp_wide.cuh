@@ -317,6 +317,11 @@ __global__ void __launch_bounds__(256) cell_coef_mma_kernel(CellArgs a)
                     jh = fmaf(kn, sq, jh);
                     jh = fmaf(kr, sr, jh);
                     out_rhs[el] = f - jh;
+                    if (a.residual) out_rhs[el] = f;
+                }
+                if (a.rhs && a.residual) {
+                    const float2 yc = __ldg(reinterpret_cast<const float2 *>(a.y + e * N + i0));
+                    out_rhs[0] -= yc.x; out_rhs[1] -= yc.y;
                 }
                 if (a.rhs) *reinterpret_cast<float2 *>(a.rhs + e * N + i0) = make_float2(out_rhs[0], out_rhs[1]);
             }

@@ -161,7 +161,9 @@ FIRST_ITERATE_CASES = [(1, 1, 0), (2, 2, 0), (4, 2, 0), (8, 4, 0), (16, 16, 0), 
 def test_first_iterates_match_the_oracle_iteration(bd, n, m, flags, bodies):
     """After one and two bodies from the zero guess (before convergence hides a wrong Jacobian or rhs)
     the iterate equals the oracle's Newton iterate (App. B.1 loop in fp64), for every cell kernel and
-    both ways of handing J to the scan (flags = 4: materialised)."""
+    both ways of handing J to the scan (flags = 4: materialised).  The default path for n = 16, 32 solves the
+    update with single-TF32 products (Newton-update form, App. A.1: same fixed point, the solve good to about
+    1e-3 of the update), so there the iterate is compared at 2e-3 of the largest update instead of 2e-5."""
     B, T = 3, 700
     p_np = synth.gru_params(n, m, 23, tag="fi/gru")
     x = synth.x_gaussian(B, T, m, 23, tag="fi/x")
@@ -171,8 +173,9 @@ def test_first_iterates_match_the_oracle_iteration(bd, n, m, flags, bodies):
     o = oracle.deer(p_np, x, y0, tol=-1.0, max_iter=bodies, dtype=np.float64)
     assert r.iters == bodies and r.status == 0
     scale = max(1.0, float(np.max(np.abs(o["y"]))))
-    assert float(np.max(np.abs(r.y.cpu().numpy() - o["y"]))) <= 2e-5 * scale
-    assert abs(r.err - o["err"]) <= 2e-5 * max(1.0, o["err"])
+    tol = 2e-3 * max(1.0, float(o["trace"][0])) if (n in (16, 32) and flags == 0) else 2e-5 * scale
+    assert float(np.max(np.abs(r.y.cpu().numpy() - o["y"]))) <= tol
+    assert abs(r.err - o["err"]) <= tol * max(1.0, o["err"])
 
 
 WARM_CASES = [(1, 1, 4, 3000), (2, 2, 4, 3000), (4, 2, 3, 2500), (8, 4, 4, 3000), (16, 16, 2, 900),
