@@ -188,3 +188,42 @@ def classifier(layers, W_o, b_o, x, labels, dtype=np.float64, want_grad=True, wa
     if want_states:
         g["y1"], g["y2"] = y1, y2
     return g
+
+
+def _stack_heads(heads, dtype):
+    return (_c(np.stack([h.W_i for h in heads]), dtype), _c(np.stack([h.W_h for h in heads]), dtype),
+            _c(np.stack([h.b_i for h in heads]), dtype), _c(np.stack([h.b_h for h in heads]), dtype))
+
+
+def multihead_seq(heads, strides, x, y0, dtype=np.float64):
+    """O-6: sequential multi-head GRU.  heads: list of H parameter sets (same n, m); strides [H];
+    x [B,T,m]; y0 [B,H,n].  Returns y [B,T,H,n]."""
+    sfx, _ = _sfx(dtype)
+    H, n, m = len(heads), heads[0].n, heads[0].m
+    W_i, W_h, b_i, b_h = _stack_heads(heads, dtype)
+    st = np.ascontiguousarray(strides, np.int32)
+    x = _c(x, dtype); y0 = _c(y0, dtype)
+    B, T, _m = x.shape
+    assert _m == m and y0.shape == (B, H, n) and st.shape == (H,) and np.all(st >= 1)
+    y = np.empty((B, T, H, n), dtype)
+    getattr(lib(), f"oracle_multihead_seq_{sfx}")(H, n, m, _p(W_i), _p(W_h), _p(b_i), _p(b_h), _p(st), _p(x),
+                                                  _p(y0), B, T, _p(y))
+    return y
+
+
+def multihead_bptt(heads, strides, x, y0, y, gy, dtype=np.float64):
+    """BPTT through the multi-head unit at trajectory y for dL/dy = gy [B,T,H,n]: dict of
+    dW_i [H,3n,m], dW_h [H,3n,n], db_i, db_h [H,3n], dx [B,T,m], dy0 [B,H,n]."""
+    sfx, _ = _sfx(dtype)
+    H, n, m = len(heads), heads[0].n, heads[0].m
+    W_i, W_h, b_i, b_h = _stack_heads(heads, dtype)
+    st = np.ascontiguousarray(strides, np.int32)
+    x = _c(x, dtype); y0 = _c(y0, dtype); y = _c(y, dtype); gy = _c(gy, dtype)
+    B, T, _m = x.shape
+    g = dict(dW_i=np.empty((H, 3 * n, m), dtype), dW_h=np.empty((H, 3 * n, n), dtype),
+             db_i=np.empty((H, 3 * n), dtype), db_h=np.empty((H, 3 * n), dtype),
+             dx=np.empty((B, T, m), dtype), dy0=np.empty((B, H, n), dtype))
+    getattr(lib(), f"oracle_multihead_bptt_{sfx}")(H, n, m, _p(W_i), _p(W_h), _p(b_i), _p(b_h), _p(st), _p(x),
+                                                   _p(y0), _p(y), _p(gy), B, T, _p(g["dW_i"]), _p(g["dW_h"]),
+                                                   _p(g["db_i"]), _p(g["db_h"]), _p(g["dx"]), _p(g["dy0"]))
+    return g

@@ -419,6 +419,74 @@ REAL FN(oracle_classifier_)(int n, int m, int ncls, const REAL *W_i1, const REAL
     return loss;
 }
 
+/* ------------------------------------------------------------------------
+ * O-6  Multi-head GRU (Sec. 4.4; App. B.4): H independent GRU heads of hidden
+ * size n read the same input x[b][t] (m channels); head h has its own
+ * parameters and a stride s_h and advances
+ *     y[b][t][h] = f_h(y[b][t - s_h][h], x[b][t]),   y[b][t'][h] = y0[b][h] for t' < 0
+ * (a head of stride s is s interleaved sequences).  The unit's output is the
+ * heads' states side by side: y [B,T,H,n].  Parameters are stacked per head:
+ * W_i [H,3n,m], W_h [H,3n,n], b_i, b_h [H,3n].
+ * Pinned by: H = 1, stride 1 equals oracle_gru_seq; a stride-s head equals s
+ * interleaved runs of oracle_gru_seq; finite differences for the gradient.
+ * ------------------------------------------------------------------------ */
+void FN(oracle_multihead_seq_)(int H, int n, int m, const REAL *W_i, const REAL *W_h,
+                               const REAL *b_i, const REAL *b_h, const int *stride, const REAL *x,
+                               const REAL *y0, int B, int T, REAL *y)
+{
+#pragma omp parallel for schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int t = 0; t < T; ++t)
+            for (int h = 0; h < H; ++h) {
+                const int tp = t - stride[h];
+                const REAL *hp = tp >= 0 ? y + (((size_t)b * T + tp) * H + h) * n
+                                         : y0 + ((size_t)b * H + h) * n;
+                FN(gru_cell_)(n, m, W_i + (size_t)h * 3 * n * m, W_h + (size_t)h * 3 * n * n,
+                              b_i + (size_t)h * 3 * n, b_h + (size_t)h * 3 * n, hp,
+                              x + ((size_t)b * T + t) * m, y + (((size_t)b * T + t) * H + h) * n, NULL);
+            }
+}
+
+/* Back-propagation through the multi-head unit for dL/dy = gy [B,T,H,n] at the
+ * trajectory y: the adjoint of head h flows from t to t - s_h.  Outputs are
+ * overwritten; dx [B,T,m] sums the heads' contributions; dy0 [B,H,n]. */
+void FN(oracle_multihead_bptt_)(int H, int n, int m, const REAL *W_i, const REAL *W_h,
+                                const REAL *b_i, const REAL *b_h, const int *stride, const REAL *x,
+                                const REAL *y0, const REAL *y, const REAL *gy, int B, int T,
+                                REAL *dW_i, REAL *dW_h, REAL *db_i, REAL *db_h, REAL *dx, REAL *dy0)
+{
+    size_t N = (size_t)B * T;
+    memset(dW_i, 0, sizeof(REAL) * (size_t)H * 3 * n * m);
+    memset(dW_h, 0, sizeof(REAL) * (size_t)H * 3 * n * n);
+    memset(db_i, 0, sizeof(REAL) * (size_t)H * 3 * n);
+    memset(db_h, 0, sizeof(REAL) * (size_t)H * 3 * n);
+    memset(dx, 0, sizeof(REAL) * N * m);
+    memset(dy0, 0, sizeof(REAL) * (size_t)B * H * n);
+    REAL *lam = (REAL *)malloc(sizeof(REAL) * N * H * n);
+    memcpy(lam, gy, sizeof(REAL) * N * H * n);
+    REAL *dh = (REAL *)malloc(sizeof(REAL) * (size_t)n);
+    REAL *dxe = (REAL *)malloc(sizeof(REAL) * (size_t)m);
+    REAL *scratch = (REAL *)malloc(sizeof(REAL) * 11 * (size_t)n);
+    for (int b = 0; b < B; ++b)
+        for (int t = T - 1; t >= 0; --t)
+            for (int h = 0; h < H; ++h) {
+                const size_t e = (size_t)b * T + t;
+                const int tp = t - stride[h];
+                const REAL *hp = tp >= 0 ? y + (((size_t)b * T + tp) * H + h) * n
+                                         : y0 + ((size_t)b * H + h) * n;
+                FN(gru_cell_vjp_)(n, m, W_i + (size_t)h * 3 * n * m, W_h + (size_t)h * 3 * n * n,
+                                  b_i + (size_t)h * 3 * n, b_h + (size_t)h * 3 * n, hp, x + e * m,
+                                  lam + (e * H + h) * n, dW_i + (size_t)h * 3 * n * m,
+                                  dW_h + (size_t)h * 3 * n * n, db_i + (size_t)h * 3 * n,
+                                  db_h + (size_t)h * 3 * n, dxe, dh, scratch);
+                for (int k = 0; k < m; ++k) dx[e * m + k] += dxe[k];
+                REAL *dst = tp >= 0 ? lam + (((size_t)b * T + tp) * H + h) * n
+                                    : dy0 + ((size_t)b * H + h) * n;
+                for (int i = 0; i < n; ++i) dst[i] += dh[i];
+            }
+    free(lam); free(dh); free(dxe); free(scratch);
+}
+
 #undef FN
 #undef CAT
 #undef CAT2

@@ -222,6 +222,16 @@ def config4(seed: int = 0, B: int = 32, T: int = 17984, n: int = 64, m: int = 6,
     return ClassifierWorkload("config4", B, T, [l1, l2], W_o, b_o, x, labels)
 
 
+def multihead_params(H: int, n: int, m: int, seed: int = 0, tag: str = "mh") -> list:
+    """H independent parameter sets (one GRU head each), streams ``{tag}/head{h}/...``."""
+    return [gru_params(n, m, seed, tag=f"{tag}/head{h}") for h in range(H)]
+
+
+def multihead_strides(H: int, kinds: int = 8) -> np.ndarray:
+    """Strides 2^0 .. 2^(kinds-1) assigned uniformly to the heads (App. B.4): head h gets 2^(h mod kinds)."""
+    return (2 ** (np.arange(H) % kinds)).astype(np.int32)
+
+
 def contractive_J(B: int, T: int, n: int, seed: int = 0, tag: str = "scanJ",
                   scale: float = 0.9) -> np.ndarray:
     """Random matrices with entries U(-s, s), s = scale / n, so that every

@@ -380,3 +380,92 @@ def test_synth_is_deterministic_and_distributed_as_documented():
     rw = synth.x_random_walk(2, 500, 3, 0)
     np.testing.assert_allclose(rw.mean(axis=1), 0, atol=1e-5)
     np.testing.assert_allclose(rw.std(axis=1), 1, atol=1e-4)
+
+
+# ----------------------------------------------------------------------------- multi-head GRU (Sec. 4.4, App. B.4)
+def mh_case(H, n, m, B, T, strides, seed=5):
+    heads = synth.multihead_params(H, n, m, seed, tag="t/mh")
+    x = synth.x_gaussian(B, T, m, seed, tag="t/mhx")
+    y0 = synth.normal(seed, "t/mhy0", (B, H, n)) * 0.5
+    return heads, np.asarray(strides, np.int32), x, y0
+
+
+def test_multihead_reading_reproduces_the_papers_parameter_count():
+    """The paper prints the model's parameter count (App. B.4) but not how a head is wired.  The reading
+    taken here -- every head is a GRU of 8 channels that reads ALL 256 input channels, with the
+    parameters of the cited GRU cell (input kernels with biases for r, z, n; hidden kernels without bias
+    for r, z and with bias for n) -- gives exactly that count; heads reading only a 1/32 slice of the
+    input would not."""
+    H, n, m, layers = 32, 8, 256, 4
+    head = 3 * (m * n + n) + 3 * n * n + n
+    composite = H * head + (256 * 512 + 512) + 2 * 256          # multi-head GRU, linear 256 -> 512 (GLU has none), layer norm
+    total = (3 * 256 + 256) + layers * composite + (256 * 10 + 10)
+    assert total == int(GOLD["multihead_model_trainable_parameters"])
+    sliced = 3 * ((m // H) * n + n) + 3 * n * n + n
+    assert (3 * 256 + 256) + layers * (H * sliced + 256 * 512 + 512 + 512) + 2570 != total
+
+
+def test_multihead_one_head_stride_one_is_the_plain_gru():
+    heads, st, x, y0 = mh_case(1, 4, 3, 2, 50, [1])
+    y = oracle.multihead_seq(heads, st, x, y0)
+    assert np.array_equal(y[:, :, 0], oracle.gru_seq(heads[0], x, y0[:, 0]))
+
+
+def test_multihead_strided_head_is_interleaved_sequences_and_heads_are_independent():
+    """Head h with stride s is s independent GRU runs over x[:, p::s], each from y0 (Sec. 4.4)."""
+    strides = [1, 2, 4, 3]
+    heads, st, x, y0 = mh_case(4, 3, 5, 2, 41, strides)
+    y = oracle.multihead_seq(heads, st, x, y0)
+    for h, s in enumerate(strides):
+        for p in range(s):
+            want = oracle.gru_seq(heads[h], x[:, p::s], y0[:, h])
+            assert np.array_equal(y[:, p::s, h], want), (h, p)
+    for dtype in (np.float32,):
+        y32 = oracle.multihead_seq(heads, st, x, y0, dtype)
+        assert np.max(np.abs(y32 - y)) <= 2e-6
+
+
+def test_multihead_bptt_matches_finite_differences():
+    strides = [2, 1, 3]
+    heads, st, x, y0 = mh_case(3, 2, 2, 2, 9, strides)
+    gy = synth.normal(9, "t/mhgy", (2, 9, 3, 2)).astype(np.float64)
+    loss = lambda hd, xx, yy0: float(np.sum(gy * oracle.multihead_seq(hd, st, xx, yy0)))
+    y = oracle.multihead_seq(heads, st, x, y0)
+    g = oracle.multihead_bptt(heads, st, x, y0, y, gy)
+    eps = 1e-6
+    x64, y064 = x.astype(np.float64), y0.astype(np.float64)
+    h64 = [h.astype(np.float64) for h in heads]
+    for hh in range(3):
+        for name in ("W_i", "W_h", "b_i", "b_h"):
+            arr = getattr(h64[hh], name)
+            for idx in list(np.ndindex(arr.shape))[::3]:
+                old = arr[idx]
+                arr[idx] = old + eps; lp = loss(h64, x64, y064)
+                arr[idx] = old - eps; lm = loss(h64, x64, y064)
+                arr[idx] = old
+                assert abs((lp - lm) / (2 * eps) - g["d" + name][(hh,) + idx]) <= 1e-7, (hh, name, idx)
+    for arr, key in ((x64, "dx"), (y064, "dy0")):
+        for idx in list(np.ndindex(arr.shape))[::2]:
+            old = arr[idx]
+            arr[idx] = old + eps; lp = loss(h64, x64, y064)
+            arr[idx] = old - eps; lm = loss(h64, x64, y064)
+            arr[idx] = old
+            assert abs((lp - lm) / (2 * eps) - g[key][idx]) <= 1e-7, (key, idx)
+
+
+def test_multihead_bptt_reduces_to_plain_bptt_per_phase():
+    """One head of stride s: its gradient is the sum of plain BPTT over the s interleaved sequences."""
+    s = 3
+    heads, st, x, y0 = mh_case(1, 3, 2, 2, 20, [s])
+    y = oracle.multihead_seq(heads, st, x, y0)
+    gy = synth.normal(4, "t/mhgy2", y.shape).astype(np.float64)
+    g = oracle.multihead_bptt(heads, st, x, y0, y, gy)
+    acc = None
+    for p in range(s):
+        gp = oracle.gru_bptt(heads[0], x[:, p::s], y0[:, 0], y[:, p::s, 0], gy[:, p::s, 0])
+        assert np.allclose(g["dx"][:, p::s], gp["dx"], atol=1e-13)
+        gp = {k: gp[k] for k in ("dW_i", "dW_h", "db_i", "db_h", "dy0")}
+        acc = gp if acc is None else {k: acc[k] + gp[k] for k in gp}
+    for k in ("dW_i", "dW_h", "db_i", "db_h"):
+        assert np.allclose(g[k][0], acc[k], atol=1e-12), k
+    assert np.allclose(g["dy0"][:, 0], acc["dy0"], atol=1e-13)
