@@ -407,6 +407,61 @@ def time_classifier(bd, synth, torch, device, B, T, flags, steps, warmup, profil
     return out
 
 
+def time_multihead(bd, synth, torch, device, B, T, H, n, m, steps, warmup, cpu_seconds=0.0):
+    """The multi-head GRU unit of the paper's sequential-image model (Sec. 4.4, App. B.4: 32 heads of 8 channels
+    on 256 input channels, strides 2^0 .. 2^7, T = 1024): forward evaluation and gradient."""
+    heads = synth.multihead_params(H, n, m, 0, tag="bench/mh")
+    strides = synth.multihead_strides(H)
+    x_np = synth.x_gaussian(B, T, m, 0, tag="bench/mhx")
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
+    hd = [bd.GruParamsDev.from_numpy(h) for h in heads]
+    x = dev(x_np); y0 = torch.zeros((B, H, n), device=device)
+    ws = bd.alloc_multihead_workspace(hd, strides, B, T, device)
+    y = torch.empty((B, T, H, n), device=device)
+    stream = torch.cuda.current_stream()
+    run = lambda: bd.deer_gru_multihead_eval(hd, strides, x, y0, y=y, ws=ws, stream=stream)
+    for _ in range(max(warmup, 1)):
+        _, iters, status = run()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    torch.cuda.synchronize()
+    for a, b in ev:
+        a.record(stream); run(); b.record(stream)
+    torch.cuda.synchronize()
+    ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+    gy = torch.ones_like(y)
+    bd.deer_gru_multihead_vjp(hd, strides, x, y0, y, gy, ws=ws, stream=stream)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream); bd.deer_gru_multihead_vjp(hd, strides, x, y0, y, gy, ws=ws, stream=stream); b.record(stream)
+    torch.cuda.synchronize()
+    out = dict(workload=f"multi-head GRU unit: H={H} heads x n={n}, m={m}, strides 2^(h mod 8), B={B} T={T}, x~N(0,1), y0=0",
+               ms_per_step=ms, value=B * T / (ms * 1e-3), unit=UNIT, newton_iters=iters, status=status,
+               vjp_ms=a.elapsed_time(b))
+    if cpu_seconds > 0:
+        import oracle
+        y0_np = np.zeros((B, H, n), np.float32)
+        oracle.multihead_seq(heads, strides, x_np, y0_np, np.float32)
+        reps, t0 = 0, time.perf_counter()
+        while time.perf_counter() - t0 < cpu_seconds:
+            oracle.multihead_seq(heads, strides, x_np, y0_np, np.float32)
+            reps += 1
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = dict(value=reps * B * T / dt, unit=UNIT, cores=min(oracle.num_threads(), B), kind="oracle",
+                                   sample=f"{reps} passes of the oracle's sequential multi-head loop ({dt:.1f} s)")
+    return out
+
+
+def run_multihead(args):
+    import torch
+    from paper_2309_12252_b200 import binding as bd
+    from paper_2309_12252_b200 import synth
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    out = time_multihead(bd, synth, torch, device, args.B, args.T, 32, 8, 256, args.steps, args.warmup, args.cpu_seconds)
+    out["mode"] = "multihead"
+    print(json.dumps(out))
+
+
 def run_classifier(args):
     import torch
     from paper_2309_12252_b200 import binding as bd
@@ -548,7 +603,7 @@ def step_scan_roofline(m, pk):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--mode", default="step", choices=["step", "scan", "eval", "sweep", "classifier"])
+    ap.add_argument("--mode", default="step", choices=["step", "scan", "eval", "sweep", "classifier", "multihead"])
     ap.add_argument("--m", type=int, default=0)
     ap.add_argument("--vjp", type=int, default=0)
     ap.add_argument("--n", type=int, default=8)
@@ -565,9 +620,9 @@ def main():
                     help="skip the other workloads and the HBM-sized stand-alone scans (headline workload only)")
     args = ap.parse_args()
     if args.B is None:
-        args.B = 32 if args.mode == "classifier" else 16
+        args.B = 32 if args.mode in ("classifier", "multihead") else 16
     if args.T is None:
-        args.T = 17_984 if args.mode == "classifier" else 1_000_000
+        args.T = 17_984 if args.mode == "classifier" else 1024 if args.mode == "multihead" else 1_000_000
     if args.impl == "reference":
         run_reference(args)
         return
@@ -582,6 +637,9 @@ def main():
         return
     if args.mode == "classifier":
         run_classifier(args)
+        return
+    if args.mode == "multihead":
+        run_multihead(args)
         return
 
     import torch
@@ -629,6 +687,9 @@ def main():
             kernels=c4["kernels"],
             scan_roofline=roofline_of_scan(64, 32 * 17_984, scan_ms / max(scan_launches, 1), pk, scan_bytes_per_position(64),
                                            NCU_SCAN_TRAFFIC_PER_POSITION[64], "scan_cta64_kernel (forward and reverse)"))
+        torch.cuda.empty_cache()
+        # ---- the multi-head GRU unit of the paper's sequential-image model
+        extras["multihead_unit"] = time_multihead(bd, synth, torch, device, 32, 1024, 32, 8, 256, 5, 2, cpu_seconds=2.0)
         torch.cuda.empty_cache()
         # ---- stand-alone scans on HBM-sized problems: the roofline of each scan kernel
         scans = []

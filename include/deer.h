@@ -261,6 +261,36 @@ int deer_gru_classifier_step(const deer_gru_params *layer1, const deer_gru_param
                              const deer_gru_grads *g2, float *dW_o, float *db_o, void *ws,
                              size_t ws_bytes, int flags, void *stream);
 
+/* Multi-head GRU unit (Sec. 4.4 "Sequence classification with multiple heads RNN"; App. B.4): H independent
+ * GRU heads of hidden size n, every one reading the whole input x[b][t] (m channels) with its own
+ * parameters, head h advancing with stride s_h,
+ *     y[b][t][h] = f_h(y[b][t - s_h][h], x[b][t]),      y[b][t'][h] = y0[b][h] for t' < 0,
+ * so that a head of stride s is s interleaved sequences.  The Jacobian of the whole unit is block-diagonal
+ * over the heads (the paper's way around the n^3 cost of the scan): every head is evaluated by the DEER
+ * iteration of deer_gru_eval on its own, its interleaved sequences laid out as a dense batch of B * s_h
+ * sequences of ceil(T / s_h) positions by a gather kernel (heads of equal stride share the gathered input).
+ *   heads   : HOST array of H parameter sets (device pointers inside), equal n and m
+ *   strides : HOST array of H strides >= 1 (the paper uses 2^0 ... 2^7, assigned uniformly to 32 heads)
+ *   x [B,T,m]   y0 [B,H,n]   y [B,T,H,n] out (the heads' states side by side; the guess on entry if
+ *   DEER_FLAG_WARM_START)      iters : host out [H], bodies executed per head (may be NULL)
+ *   ws : deer_multihead_workspace_bytes(...) bytes
+ * Synchronises `stream`.  Returns the worst status of the heads' evaluations or a negative status. */
+size_t deer_multihead_workspace_bytes(const int *strides, int H, int B, int T, int n, int m, int flags);
+int deer_gru_multihead_eval(const deer_gru_params *heads, const int *strides, int H, const float *x,
+                            const float *y0, int B, int T, float tol, int max_iter, float *y, int *iters,
+                            void *ws, size_t ws_bytes, int flags, void *stream);
+
+/* Gradient through the multi-head unit (Eq. 7 per head: one reverse scan and the cell's vector-Jacobian
+ * product), for dL/dy = gy [B,T,H,n] at the trajectory y:
+ *   dheads : HOST array of H gradient sets (device arrays, overwritten)
+ *   dx [B,T,m] or NULL : the heads' contributions added head by head in a fixed order
+ *   dy0 [B,H,n] or NULL
+ * Synchronises `stream`.  Returns DEER_OK, DEER_ERR_DEVICE_TIMEOUT or another negative status. */
+int deer_gru_multihead_vjp(const deer_gru_params *heads, const int *strides, int H, const float *x,
+                           const float *y0, const float *y, const float *gy, int B, int T,
+                           const deer_gru_grads *dheads, float *dx, float *dy0, void *ws, size_t ws_bytes,
+                           int flags, void *stream);
+
 /* Text for a status code (static storage). */
 const char *deer_status_string(int status);
 

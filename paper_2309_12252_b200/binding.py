@@ -27,7 +27,8 @@ NOALLOC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc", "deer_gru_eval",
            "deer_gru_eval_diag", "deer_gru_eval_host", "deer_gru_vjp",
            "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count",
-           "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_cell_jac"]
+           "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_cell_jac",
+           "deer_multihead_workspace_bytes", "deer_gru_multihead_eval", "deer_gru_multihead_vjp"]
 
 
 class _Params(ctypes.Structure):
@@ -84,6 +85,14 @@ def lib():
         L.deer_scan_geometry.argtypes = [ci, ci, ci, ci, ctypes.POINTER(ci)]
         L.deer_gru_cell_jac.restype = ci
         L.deer_gru_cell_jac.argtypes = [ctypes.POINTER(_Params), vp, vp, vp, ci, ci, vp, vp, vp, sz, ci, vp]
+        L.deer_multihead_workspace_bytes.restype = sz
+        L.deer_multihead_workspace_bytes.argtypes = [ctypes.POINTER(ci), ci, ci, ci, ci, ci, ci]
+        L.deer_gru_multihead_eval.restype = ci
+        L.deer_gru_multihead_eval.argtypes = [ctypes.POINTER(_Params), ctypes.POINTER(ci), ci, vp, vp, ci, ci, cf, ci, vp,
+                                              ctypes.POINTER(ci), vp, sz, ci, vp]
+        L.deer_gru_multihead_vjp.restype = ci
+        L.deer_gru_multihead_vjp.argtypes = [ctypes.POINTER(_Params), ctypes.POINTER(ci), ci, vp, vp, vp, vp, ci, ci,
+                                             ctypes.POINTER(_Grads), vp, vp, vp, sz, ci, vp]
         L.deer_status_string.restype = ctypes.c_char_p
         L.deer_status_string.argtypes = [ci]
         L.deer_last_error.restype = ctypes.c_char_p
@@ -356,3 +365,59 @@ def deer_gru_classifier_step(layer1: GruParamsDev, layer2: GruParamsDev, W_o, b_
     if rc < 0:
         raise DeerError(rc)
     return dict(loss=loss.value, iters=(iters[0], iters[1]), status=rc, g1=g1, g2=g2, dW_o=dW_o, db_o=db_o)
+
+
+def _mh_args(heads, strides):
+    H = len(heads)
+    ps = (_Params * H)(*[h.c_struct() for h in heads])
+    st = (ctypes.c_int * H)(*[int(v) for v in strides])
+    return H, ps, st
+
+
+def alloc_multihead_workspace(heads, strides, B, T, device="cuda"):
+    H, _, st = _mh_args(heads, strides)
+    nbytes = int(lib().deer_multihead_workspace_bytes(st, H, B, T, heads[0].n, heads[0].m, 0))
+    if nbytes == 0:
+        raise DeerError(DEER_ERR_INVALID_ARG)
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
+def deer_gru_multihead_eval(heads, strides, x, y0, tol=1e-4, max_iter=100, y=None, ws=None, flags=0, stream=None):
+    """Multi-head GRU unit: heads = list of GruParamsDev, strides = list of ints, x [B,T,m], y0 [B,H,n].
+    Returns (y [B,T,H,n], iters per head, status); see include/deer.h."""
+    B, T, m = x.shape
+    H, ps, st = _mh_args(heads, strides)
+    n = heads[0].n
+    assert tuple(y0.shape) == (B, H, n)
+    if y is None:
+        y = torch.empty((B, T, H, n), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = alloc_multihead_workspace(heads, strides, B, T, x.device)
+    iters = (ctypes.c_int * H)()
+    rc = lib().deer_gru_multihead_eval(ps, st, H, _ptr(_f32(x)), _ptr(_f32(y0)), B, T, float(tol), int(max_iter), _ptr(y),
+                                       iters, _ptr(ws), ws.numel(), flags, _stream(stream))
+    if rc < 0:
+        raise DeerError(rc)
+    return y, list(iters), rc
+
+
+def deer_gru_multihead_vjp(heads, strides, x, y0, y, gy, ws=None, flags=0, stream=None):
+    """Gradients of the multi-head unit: dict with per-head lists dW_i, dW_h, db_i, db_h and dx, dy0."""
+    B, T, m = x.shape
+    H, ps, st = _mh_args(heads, strides)
+    n = heads[0].n
+    dev = x.device
+    g = dict(dW_i=[torch.empty((3 * n, m), device=dev) for _ in range(H)], dW_h=[torch.empty((3 * n, n), device=dev) for _ in range(H)],
+             db_i=[torch.empty((3 * n,), device=dev) for _ in range(H)], db_h=[torch.empty((3 * n,), device=dev) for _ in range(H)])
+    gs = (_Grads * H)(*[_Grads(g["dW_i"][h].data_ptr(), g["dW_h"][h].data_ptr(), g["db_i"][h].data_ptr(),
+                               g["db_h"][h].data_ptr()) for h in range(H)])
+    dx = torch.empty_like(x)
+    dy0 = torch.empty_like(y0)
+    if ws is None:
+        ws = alloc_multihead_workspace(heads, strides, B, T, dev)
+    rc = lib().deer_gru_multihead_vjp(ps, st, H, _ptr(_f32(x)), _ptr(_f32(y0)), _ptr(_f32(y)), _ptr(_f32(gy)), B, T, gs,
+                                      _ptr(dx), _ptr(dy0), _ptr(ws), ws.numel(), flags, _stream(stream))
+    if rc != DEER_OK:
+        raise DeerError(rc)
+    g["dx"], g["dy0"] = dx, dy0
+    return g

@@ -685,6 +685,61 @@ static ClsWs carve_cls(void *ws, int B, int T, int n, int m, int ncls)
     return w;
 }
 
+// multi-head unit: dense batches of one stride group at a time + the inner evaluation / gradient workspace
+struct MhWs {
+    float *xs, *y0s, *ys, *gys, *dxs, *dy0s;
+    void *inner;
+    size_t inner_bytes, bytes;
+};
+
+static MhWs carve_mh(void *ws, int H, const int *strides, int B, int T, int n, int m)
+{
+    Carver cv(ws);
+    MhWs w;
+    size_t maxN = 0, maxB = 0, inner = 0;
+    for (int h = 0; h < H; ++h) {
+        const int s = strides[h];
+        const int Tp = (T + s - 1) / s;
+        const size_t Bs = (size_t)B * s;
+        maxN = Bs * Tp > maxN ? Bs * Tp : maxN;
+        maxB = Bs > maxB ? Bs : maxB;
+        const size_t e = carve_eval(nullptr, (int)Bs, Tp, n, m).bytes, v = carve_vjp(nullptr, (int)Bs, Tp, n, m).bytes;
+        inner = e > inner ? e : inner;
+        inner = v > inner ? v : inner;
+    }
+    w.xs = cv.take<float>(maxN * m);
+    w.y0s = cv.take<float>(maxB * n);
+    w.ys = cv.take<float>(maxN * n);
+    w.gys = cv.take<float>(maxN * n);
+    w.dxs = cv.take<float>(maxN * m);
+    w.dy0s = cv.take<float>(maxB * n);
+    w.inner_bytes = inner;
+    w.inner = cv.take<char>(inner);
+    w.bytes = cv.off;
+    return w;
+}
+
+static int check_mh_args(const deer_gru_params *heads, const int *strides, int H, int B, int T)
+{
+    if (!heads || !strides || H < 1 || B <= 0 || T <= 0) return DEER_ERR_INVALID_ARG;
+    for (int h = 0; h < H; ++h) {
+        if (!heads[h].W_i || !heads[h].W_h || !heads[h].b_i || !heads[h].b_h) return DEER_ERR_INVALID_ARG;
+        if (heads[h].n != heads[0].n || heads[h].m != heads[0].m || heads[h].n <= 0 || heads[h].m <= 0) return DEER_ERR_INVALID_ARG;
+        if (strides[h] < 1 || (long long)B * strides[h] > 0x7fffffffLL) return DEER_ERR_INVALID_ARG;
+    }
+    if (!supported(heads[0].n, heads[0].m)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, heads[0].n, heads[0].m)) return DEER_ERR_INVALID_ARG;
+    return DEER_OK;
+}
+
+static unsigned mh_blocks(size_t total)
+{
+    size_t b = (total + 255) / 256;
+    const size_t cap = (size_t)num_sms() * 8;
+    if (b > cap) b = cap;
+    return (unsigned)(b < 1 ? 1 : b);
+}
+
 static int check_ws(void *ws, size_t have, size_t need)
 {
     if (!ws || ((uintptr_t)ws & 255) != 0 || have < need) return DEER_ERR_WORKSPACE;
@@ -1141,6 +1196,90 @@ int deer_gru_classifier_step(const deer_gru_params *l1, const deer_gru_params *l
     if ((f1 | f2) & FLAG_TIMEOUT) return DEER_ERR_DEVICE_TIMEOUT;
     *loss = tail[0];
     return s1 > s2 ? s1 : s2;
+}
+
+size_t deer_multihead_workspace_bytes(const int *strides, int H, int B, int T, int n, int m, int flags)
+{
+    (void)flags;
+    if (!strides || H < 1 || !valid_sizes(B, T, n, m) || !supported(n, m)) return 0;
+    for (int h = 0; h < H; ++h)
+        if (strides[h] < 1 || (long long)B * strides[h] > 0x7fffffffLL) return 0;
+    return carve_mh(nullptr, H, strides, B, T, n, m).bytes;
+}
+
+int deer_gru_multihead_eval(const deer_gru_params *heads, const int *strides, int H, const float *x, const float *y0,
+                            int B, int T, float tol, int max_iter, float *y, int *iters, void *ws, size_t ws_bytes,
+                            int flags, void *stream)
+{
+    int rc = check_mh_args(heads, strides, H, B, T);
+    if (rc != DEER_OK) return rc;
+    if (!x || !y0 || !y || max_iter < 1 || tol != tol) return DEER_ERR_INVALID_ARG;
+    const int n = heads[0].n, m = heads[0].m;
+    cudaStream_t st = (cudaStream_t)stream;
+    MhWs w = carve_mh(ws, H, strides, B, T, n, m);
+    if ((rc = check_ws(ws, ws_bytes, w.bytes)) != DEER_OK) return rc;
+    int worst = DEER_OK;
+    int packed_stride = 0;                     // stride whose dense batch of x is in w.xs
+    for (int h = 0; h < H; ++h) {
+        const int s = strides[h], Tp = (T + s - 1) / s, Bs = B * s;
+        if (s != packed_stride) {              // heads of equal stride read the same dense batch of x
+            DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(x, w.xs, B, T, s, Tp, m, m, 0));
+            packed_stride = s;
+        }
+        DEER_KERNEL("mh_y0_pack_kernel", st, mh_y0_pack_kernel<<<mh_blocks((size_t)Bs * n), 256, 0, st>>>(y0, w.y0s, B, s, n, H, h));
+        if (flags & DEER_FLAG_WARM_START)
+            DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(y, w.ys, B, T, s, Tp, n, H * n, h * n));
+        int it = 0;
+        rc = gru_eval_impl(&heads[h], w.xs, w.y0s, Bs, Tp, tol, max_iter, w.ys, &it, nullptr, nullptr, w.inner, w.inner_bytes,
+                           flags, st);
+        if (rc < 0) return rc;
+        if (iters) iters[h] = it;
+        if (rc > worst) worst = rc;
+        DEER_KERNEL("mh_unpack_kernel", st, mh_unpack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(w.ys, y, B, T, s, Tp, n, H * n, h * n, 0));
+    }
+    DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+    return worst;
+}
+
+int deer_gru_multihead_vjp(const deer_gru_params *heads, const int *strides, int H, const float *x, const float *y0,
+                           const float *y, const float *gy, int B, int T, const deer_gru_grads *dheads, float *dx,
+                           float *dy0, void *ws, size_t ws_bytes, int flags, void *stream)
+{
+    int rc = check_mh_args(heads, strides, H, B, T);
+    if (rc != DEER_OK) return rc;
+    if (!x || !y0 || !y || !gy || !dheads) return DEER_ERR_INVALID_ARG;
+    for (int h = 0; h < H; ++h)
+        if (!dheads[h].dW_i || !dheads[h].dW_h || !dheads[h].db_i || !dheads[h].db_h) return DEER_ERR_INVALID_ARG;
+    const int n = heads[0].n, m = heads[0].m;
+    cudaStream_t st = (cudaStream_t)stream;
+    MhWs w = carve_mh(ws, H, strides, B, T, n, m);
+    if ((rc = check_ws(ws, ws_bytes, w.bytes)) != DEER_OK) return rc;
+    unsigned timeout_flags = 0;
+    int packed_stride = 0;
+    for (int h = 0; h < H; ++h) {
+        const int s = strides[h], Tp = (T + s - 1) / s, Bs = B * s;
+        if (s != packed_stride) {
+            DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(x, w.xs, B, T, s, Tp, m, m, 0));
+            packed_stride = s;
+        }
+        DEER_KERNEL("mh_y0_pack_kernel", st, mh_y0_pack_kernel<<<mh_blocks((size_t)Bs * n), 256, 0, st>>>(y0, w.y0s, B, s, n, H, h));
+        DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(y, w.ys, B, T, s, Tp, n, H * n, h * n));
+        DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(gy, w.gys, B, T, s, Tp, n, H * n, h * n));
+        rc = gru_vjp_impl(&heads[h], w.xs, w.y0s, w.ys, w.gys, Bs, Tp, &dheads[h], dx ? w.dxs : nullptr, dy0 ? w.dy0s : nullptr,
+                          w.inner, w.inner_bytes, flags, st);
+        if (rc != DEER_OK) return rc;
+        if (dx)     // the heads' input gradients add up, head by head in a fixed order
+            DEER_KERNEL("mh_unpack_kernel", st, mh_unpack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(w.dxs, dx, B, T, s, Tp, m, m, 0, h > 0));
+        if (dy0)
+            DEER_KERNEL("mh_dy0_reduce_kernel", st, mh_dy0_reduce_kernel<<<mh_blocks((size_t)B * n), 256, 0, st>>>(w.dy0s, dy0, B, s, n, H, h));
+        // the inner gradient calls share one status block: keep every head's flags
+        unsigned f = 0;
+        DEER_CHECK_CUDA(cudaMemcpyAsync(&f, &reinterpret_cast<const StatusBlock *>(w.inner)->flags, sizeof(unsigned),
+                                        cudaMemcpyDeviceToHost, st), "read status");
+        DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+        timeout_flags |= f;
+    }
+    return (timeout_flags & FLAG_TIMEOUT) ? DEER_ERR_DEVICE_TIMEOUT : DEER_OK;
 }
 
 int deer_linrec_scan_noalloc(const float *J, const float *b, const float *y0, int B, int T, int n,

@@ -845,4 +845,70 @@ __global__ void broadcast_gy_kernel(const float *__restrict__ gpool, float *__re
     gy[idx] = gpool[seq * n + i];
 }
 
+
+// ---------------------------------------------------------------- multi-head GRU: strided views <-> dense batches
+// A head of stride s over [B,T] is s interleaved sequences per batch entry (Sec. 4.4): sequence (b, p) holds the
+// positions t = p + s t', t' = 0 .. T'-1 with T' = ceil(T / s); shorter phases are padded at the END with zeros
+// (a GRU is causal: padding behind the last position changes nothing before it).
+//   pack  : dst[(b s + p), t', c] = src[b, p + s t', off + c]     (src rows of C_src channels; 0 past T)
+//   unpack: dst[b, p + s t', off + c] (+)= src[(b s + p), t', c]  (valid positions only)
+__global__ void mh_pack_kernel(const float *__restrict__ src, float *__restrict__ dst, int B, int T, int s, int Tp, int C,
+                               int C_src, int off)
+{
+    const size_t total = (size_t)B * s * Tp * C;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % C);
+        const size_t r = i / C;
+        const int tp = (int)(r % Tp);
+        const size_t q = r / Tp;
+        const int p = (int)(q % s);
+        const size_t b = q / s;
+        const long long t = (long long)p + (long long)s * tp;
+        dst[i] = t < T ? src[(b * T + (size_t)t) * C_src + off + c] : 0.0f;
+    }
+}
+
+__global__ void mh_unpack_kernel(const float *__restrict__ src, float *__restrict__ dst, int B, int T, int s, int Tp, int C,
+                                 int C_dst, int off, int accumulate)
+{
+    const size_t total = (size_t)B * s * Tp * C;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % C);
+        const size_t r = i / C;
+        const int tp = (int)(r % Tp);
+        const size_t q = r / Tp;
+        const int p = (int)(q % s);
+        const size_t b = q / s;
+        const long long t = (long long)p + (long long)s * tp;
+        if (t < T) {
+            float *d = dst + (b * T + (size_t)t) * C_dst + off + c;
+            *d = accumulate ? *d + src[i] : src[i];
+        }
+    }
+}
+
+// y0s[(b s + p), i] = y0[b, h, i]
+__global__ void mh_y0_pack_kernel(const float *__restrict__ y0, float *__restrict__ y0s, int B, int s, int n, int H, int h)
+{
+    const size_t total = (size_t)B * s * n;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % n);
+        const size_t b = i / n / s;
+        y0s[i] = y0[(b * H + h) * n + c];
+    }
+}
+
+// dy0[b, h, i] = sum over the phases p, in order, of dy0s[(b s + p), i]
+__global__ void mh_dy0_reduce_kernel(const float *__restrict__ dy0s, float *__restrict__ dy0, int B, int s, int n, int H, int h)
+{
+    const size_t total = (size_t)B * n;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % n);
+        const size_t b = i / n;
+        float acc = 0.0f;
+        for (int p = 0; p < s; ++p) acc += dy0s[(b * s + p) * n + c];
+        dy0[(b * H + h) * n + c] = acc;
+    }
+}
+
 }  // namespace deer
