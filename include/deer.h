@@ -80,7 +80,7 @@ enum {
     DEER_FLAG_WARM_START = 1,   /* deer_gru_eval: y holds the initial guess on entry (Sec. 3.1:
                                    the previous training step's solution may seed the next) */
     DEER_FLAG_GENERIC    = 2,   /* force the generic (any-n) kernels; for testing */
-    DEER_FLAG_MATERIALIZE = 4,  /* deer_gru_eval, n = 16 and 32: have the cell write the Jacobians
+    DEER_FLAG_MATERIALIZE = 4,  /* deer_gru_eval, n = 16, 32 and 64: have the cell write the Jacobians
                                    J [B,T,n,n] to the workspace and scan them, instead of writing
                                    four coefficient vectors per position from which the scan builds
                                    J_t itself (the default there; the two agree to rounding) */
@@ -92,7 +92,7 @@ enum {
                                    and every wait gives up after a few polls, so the scan drains
                                    and the call reports DEER_ERR_DEVICE_TIMEOUT (outputs invalid).
                                    Nothing traps or hangs; the workspace can be used again */
-    DEER_FLAG_COEF_ROWS  = 32   /* deer_gru_cell_jac, n = 16 and 32: write the four coefficient
+    DEER_FLAG_COEF_ROWS  = 32   /* deer_gru_cell_jac, n = 16, 32 and 64: write the four coefficient
                                    vectors per position instead of the matrices (see there) */
 };
 
@@ -172,7 +172,7 @@ int deer_scan_geometry(int B, int T, int n, int flags, int *out);
  *     J[b][t]   = df/dy_prev (y_prev, x[b][t])            [B,T,n,n] out, row = output
  *     rhs[b][t] = f(y_prev, x[b][t]) - J[b][t] y_prev     [B,T,n]   out
  * by the kernel deer_gru_eval uses for these sizes (DEER_FLAG_GENERIC: the any-n kernel).
- * With DEER_FLAG_COEF_ROWS (n = 16, 32, 16-byte aligned buffers) J receives instead the
+ * With DEER_FLAG_COEF_ROWS (n = 16, 32, 64, 16-byte aligned buffers) J receives instead the
  * coefficient rows [B,T,n,4] = {k_r, a_z, k_n, z} from which the scans of deer_gru_eval
  * build J = diag(k_r) W_hr + diag(a_z) W_hz + diag(k_n) W_hn + diag(z) themselves.
  *   ws : workspace of deer_workspace_bytes(DEER_OP_EVAL, ...) bytes (holds x W_i^T + b_i)

@@ -20,6 +20,7 @@
 #include "scan_fused_fwd.cuh"
 #include "scan_cta64.cuh"
 #include "scan_umma64.cuh"
+#include "scan_fused_fwd64.cuh"
 #include "cell_wide.cuh"
 #include "vjp_wide.cuh"
 
@@ -316,6 +317,36 @@ static int launch_fused_fwd(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
     return DEER_OK;
 }
 
+// n = 64: the same two launches (a CTA of four warps per chain; the replay kernel reads W_h^T from shared memory)
+static int launch_fused_fwd64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
+{
+    using C = FusedFwd<64>;
+    static int occ[MAX_DEVICES] = {0};
+    static int occ_apply[MAX_DEVICES] = {0};
+    w.sw = C::L;                               // a tile is one chain
+    const PassCfg c{"scan_fused_reduce64_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 4, 16};
+    int rc = launch_single_pass(scan_fused_reduce64_kernel, occ, c, a, w, prep, st);
+    if (rc != DEER_OK) return rc;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= MAX_DEVICES) dev = 0;
+    if (!occ_apply[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(scan_fused_apply_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::A_SMEM);
+        if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(scan apply)"); return DEER_ERR_CUDA; }
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, scan_fused_apply_kernel<64>, C::A_THREADS, C::A_SMEM);
+        if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(scan apply)"); return DEER_ERR_CUDA; }
+        occ_apply[dev] = o;
+    }
+    const long long nchain = (a.T + w.sw - 1) / w.sw;
+    const long long groups = ((long long)a.B * nchain + C::ROWS - 1) / C::ROWS;
+    const long long want = (groups + C::A_WARPS - 1) / C::A_WARPS;
+    const long long resident = (long long)num_sms() * occ_apply[dev];
+    const unsigned grid = (unsigned)(want < resident ? want : resident);
+    DEER_KERNEL_PDL("scan_fused_apply_kernel", false, st, scan_fused_apply_kernel<64>, grid, (unsigned)C::A_THREADS, C::A_SMEM, a, w);
+    return DEER_OK;
+}
+
 template <bool REV>
 static int launch_cta64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
@@ -352,7 +383,8 @@ static int scan_onepass(ScanArgs a, OnePassWs w, bool prep, int flags, cudaStrea
     case 64: return a.Wh ? (a.residual ? launch_fused_fwd<32>(a, w, prep, st) : launch_warpnf<32, false>(a, w, prep, st))
                          : launch_warpn<32, false>(a, w, prep, st);
     case 65: return a.Wh ? launch_warpnf<32, true>(a, w, prep, st) : launch_warpn<32, true>(a, w, prep, st);
-    case 128: return umma ? launch_umma64<false>(a, w, prep, st) : launch_cta64<false>(a, w, prep, st);
+    case 128: return umma ? launch_umma64<false>(a, w, prep, st)
+                          : (a.Wh && a.residual) ? launch_fused_fwd64(a, w, prep, st) : launch_cta64<false>(a, w, prep, st);
     case 129: return umma ? launch_umma64<true>(a, w, prep, st) : launch_cta64<true>(a, w, prep, st);
     default: return DEER_ERR_UNSUPPORTED_N;
     }
@@ -790,8 +822,8 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
     const bool single = scan_is_single_pass(a, w.scan, flags) && (((uintptr_t)w.yalt) & 15) == 0;
     // n = 16, 32: the cell writes coefficient rows and the scan generates J_t itself, unless the caller
     // asks for materialised Jacobians
-    const bool gen_J = single && (n == 16 || n == 32) && !(flags & DEER_FLAG_MATERIALIZE) &&
-                       ((((uintptr_t)y | (uintptr_t)y0 | (uintptr_t)p->W_h) & 15) == 0);
+    const bool gen_J = single && (n == 16 || n == 32 || (n == 64 && !(flags & DEER_FLAG_TCGEN05))) &&
+                       !(flags & DEER_FLAG_MATERIALIZE) && ((((uintptr_t)y | (uintptr_t)y0 | (uintptr_t)p->W_h) & 15) == 0);
     // ... and the iteration runs in its Newton-update form: the scan solves for the update from a zero
     // entering update (its linear solve may then be approximate: single TF32 chain products)
     if (gen_J) { a.Wh = p->W_h; a.residual = 1; a.y0 = nullptr; }
@@ -1362,7 +1394,7 @@ int deer_gru_cell_jac(const deer_gru_params *p, const float *x, const float *y0,
     if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
     const int n = p->n, m = p->m;
     const bool coef = (flags & DEER_FLAG_COEF_ROWS) != 0;
-    if (coef && !(n == 16 || n == 32)) return DEER_ERR_UNSUPPORTED_N;
+    if (coef && !(n == 16 || n == 32 || n == 64)) return DEER_ERR_UNSUPPORTED_N;
     if (coef && (flags & DEER_FLAG_GENERIC)) return DEER_ERR_INVALID_ARG;
     if (coef && ((((uintptr_t)y | (uintptr_t)y0 | (uintptr_t)J | (uintptr_t)p->W_h) & 15) != 0)) return DEER_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;

@@ -67,6 +67,7 @@ template <int N> struct FusedFwd {
     static constexpr int ROW_FLOATS = 6 * N + 4;       // coefficient rows [N][4], r [N], y_old [N]; the pad keeps the
                                                        // 128-bit coefficient reads of a quarter-warp in distinct banks
     static constexpr int STAGE_A = ROWS * ROW_FLOATS;
+    static constexpr bool W_SMEM = false;              // the apply kernel keeps its share of W_h^T in registers
     static constexpr size_t A_SMEM = sizeof(float) * (A_WARPS * A_STAGES * STAGE_A + A_WARPS * ROWS * N) + 128;
 };
 
@@ -301,6 +302,7 @@ __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kerne
     using C = FusedFwd<N>;
     constexpr int NN = C::NN, AGG = C::AGG, NT = C::NT, ROWS = C::ROWS, RF = C::ROW_FLOATS, S = C::A_STAGES;
     constexpr int WA = C::WARPS;                       // chains per tile of the reduce kernel
+    constexpr bool WSM = C::W_SMEM;                    // B operand (W_h^T) from shared memory instead of registers
     pdl_prologue();
     if (loop_ended(a.st)) return;
 
@@ -310,23 +312,32 @@ __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kerne
     const int g = lane >> 2, t = lane & 3;
     float *ring = sm + warp * S * C::STAGE_A;
     float *yin = sm + C::A_WARPS * S * C::STAGE_A + warp * ROWS * N;
+    float2 *sWf = reinterpret_cast<float2 *>(sm + C::A_WARPS * S * C::STAGE_A + C::A_WARPS * ROWS * N);   // [kk][nn][lane]
 
     // B operand of every step: W_h^T, contraction index renamed so that an accumulator fragment is the next A operand
-    unsigned wf[NT][3 * NT][2];
-#pragma unroll
-    for (int kk = 0; kk < NT; ++kk)
-#pragma unroll
-        for (int nn = 0; nn < 3 * NT; ++nn) {
-            const float2 v = __ldg(reinterpret_cast<const float2 *>(a.Wh + (size_t)(8 * nn + g) * N + 8 * kk + 2 * t));
-            wf[kk][nn][0] = __float_as_uint(v.x); wf[kk][nn][1] = __float_as_uint(v.y);
+    unsigned wf[WSM ? 1 : NT][WSM ? 1 : 3 * NT][2];
+    if constexpr (WSM) {
+        for (int idx = tid; idx < NT * 3 * NT * 32; idx += C::A_THREADS) {
+            const int l = idx & 31, nn = (idx >> 5) % (3 * NT), kk = (idx >> 5) / (3 * NT);
+            sWf[idx] = __ldg(reinterpret_cast<const float2 *>(a.Wh + (size_t)(8 * nn + (l >> 2)) * N + 8 * kk + 2 * (l & 3)));
         }
+        __syncthreads();
+    } else {
+#pragma unroll
+        for (int kk = 0; kk < NT; ++kk)
+#pragma unroll
+            for (int nn = 0; nn < 3 * NT; ++nn) {
+                const float2 v = __ldg(reinterpret_cast<const float2 *>(a.Wh + (size_t)(8 * nn + g) * N + 8 * kk + 2 * t));
+                wf[kk][nn][0] = __float_as_uint(v.x); wf[kk][nn][1] = __float_as_uint(v.y);
+            }
+    }
 
     const int T = a.T, SW = w.sw;
     const long long nchain = (T + SW - 1) / SW;
     const long long total = (long long)a.B * nchain;
     const long long groups = (total + ROWS - 1) / ROWS;
     unsigned mb = 0;
-    unsigned it0 = 0;                                  // ring steps consumed so far (stage and parity of the next one)
+    unsigned it0 = 0;                                  // ring steps consumed so far (the stage of the next one)
 
     for (long long grp = (long long)blockIdx.x * C::A_WARPS + warp; grp < groups; grp += (long long)gridDim.x * C::A_WARPS) {
         // geometry of this lane's row (lanes l and l + 16 describe row l)
@@ -348,27 +359,32 @@ __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kerne
             const int vr = __shfl_sync(0xffffffffu, (int)rv, r);
             const unsigned long long tix = __shfl_sync(0xffffffffu, (unsigned long long)tile_index, r);
             const int kr = __shfl_sync(0xffffffffu, kin, r);
-            float val = 0.0f;
-            if (vr) {
-                float yl = 0.0f;
-                if (lane < N) yl = __uint_as_float((unsigned)(ld_relaxed_u64(w.starts + tix * N + lane) & 0xffffffffull));
-                val = yl;
-                if (kr > 0) {
-                    const float *ag = w.pfx + (tix * (WA - 1) + (kr - 1)) * AGG;
-                    const float *arow = ag + (size_t)(lane < N ? lane : 0) * N;
-                    float acc0 = (lane < N) ? __ldcg(ag + NN + lane) : 0.0f;
+            if constexpr (WA == 1) {
+                for (int c = lane; c < N; c += 32)
+                    yin[r * N + c] = vr ? __uint_as_float((unsigned)(ld_relaxed_u64(w.starts + tix * N + c) & 0xffffffffull)) : 0.0f;
+            } else {
+                float val = 0.0f;
+                if (vr) {
+                    float yl = 0.0f;
+                    if (lane < N) yl = __uint_as_float((unsigned)(ld_relaxed_u64(w.starts + tix * N + lane) & 0xffffffffull));
+                    val = yl;
+                    if (kr > 0) {
+                        const float *ag = w.pfx + (tix * (WA - 1) + (kr - 1)) * AGG;
+                        const float *arow = ag + (size_t)(lane < N ? lane : 0) * N;
+                        float acc0 = (lane < N) ? __ldcg(ag + NN + lane) : 0.0f;
 #pragma unroll
-                    for (int j4 = 0; j4 < N / 4; ++j4) {
-                        const float4 av = __ldcg(reinterpret_cast<const float4 *>(arow) + j4);
-                        acc0 = fmaf(av.x, __shfl_sync(0xffffffffu, yl, 4 * j4), acc0);
-                        acc0 = fmaf(av.y, __shfl_sync(0xffffffffu, yl, 4 * j4 + 1), acc0);
-                        acc0 = fmaf(av.z, __shfl_sync(0xffffffffu, yl, 4 * j4 + 2), acc0);
-                        acc0 = fmaf(av.w, __shfl_sync(0xffffffffu, yl, 4 * j4 + 3), acc0);
+                        for (int j4 = 0; j4 < N / 4; ++j4) {
+                            const float4 av = __ldcg(reinterpret_cast<const float4 *>(arow) + j4);
+                            acc0 = fmaf(av.x, __shfl_sync(0xffffffffu, yl, (4 * j4) & 31), acc0);
+                            acc0 = fmaf(av.y, __shfl_sync(0xffffffffu, yl, (4 * j4 + 1) & 31), acc0);
+                            acc0 = fmaf(av.z, __shfl_sync(0xffffffffu, yl, (4 * j4 + 2) & 31), acc0);
+                            acc0 = fmaf(av.w, __shfl_sync(0xffffffffu, yl, (4 * j4 + 3) & 31), acc0);
+                        }
+                        val = acc0;
                     }
-                    val = acc0;
                 }
+                if (lane < N) yin[r * N + lane] = val;
             }
-            if (lane < N) yin[r * N + lane] = val;
         }
         __syncwarp();
         float d[NT][4];
@@ -378,6 +394,7 @@ __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kerne
             const float2 hi = *reinterpret_cast<const float2 *>(yin + (g + 8) * N + 8 * nn + 2 * t);
             d[nn][0] = lo.x; d[nn][1] = lo.y; d[nn][2] = hi.x; d[nn][3] = hi.y;
         }
+        __syncwarp();
         // rows g and g + 8 of this lane's fragments
         const int len_lo = __shfl_sync(0xffffffffu, len, g), len_hi = __shfl_sync(0xffffffffu, len, g + 8);
         const unsigned long long e_lo = __shfl_sync(0xffffffffu, (unsigned long long)e0, g);
@@ -421,7 +438,15 @@ __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kerne
                 const unsigned af[4] = {__float_as_uint(d[kk][0]), __float_as_uint(d[kk][2]), __float_as_uint(d[kk][1]),
                                         __float_as_uint(d[kk][3])};
 #pragma unroll
-                for (int nn = 0; nn < 3 * NT; ++nn) mma_tf32(U[nn], af, wf[kk][nn], U[nn]);
+                for (int nn = 0; nn < 3 * NT; ++nn) {
+                    if constexpr (WSM) {
+                        const float2 b2 = sWf[(kk * 3 * NT + nn) * 32 + lane];
+                        const unsigned bf[2] = {__float_as_uint(b2.x), __float_as_uint(b2.y)};
+                        mma_tf32(U[nn], af, bf, U[nn]);
+                    } else {
+                        mma_tf32(U[nn], af, wf[kk][nn], U[nn]);
+                    }
+                }
             }
             const float *st = ring + stg * C::STAGE_A;
 #pragma unroll

@@ -128,9 +128,9 @@ def test_cell_jacobian_and_rhs_per_kernel(bd, n, m, flags):
     assert float(np.max(np.abs(rhs.cpu().numpy() - rhs64))) <= 4e-6
 
 
-@pytest.mark.parametrize("n,m", [(16, 16), (32, 32), (16, 5), (32, 8)])
+@pytest.mark.parametrize("n,m", [(16, 16), (32, 32), (16, 5), (32, 8), (64, 6), (64, 64)])
 def test_coefficient_rows_rebuild_the_jacobian(bd, n, m):
-    """n = 16, 32: the default evaluation path writes four coefficient vectors per position and the
+    """n = 16, 32, 64: the default evaluation path writes four coefficient vectors per position and the
     scan forms J = diag(k_r) W_hr + diag(a_z) W_hz + diag(k_n) W_hn + diag(z) itself.  Rebuilt on the
     host from the rows the kernel wrote, that matrix is the oracle's Jacobian."""
     B, T = 2, 301
@@ -153,7 +153,7 @@ def test_coefficient_rows_rebuild_the_jacobian(bd, n, m):
 
 
 FIRST_ITERATE_CASES = [(1, 1, 0), (2, 2, 0), (4, 2, 0), (8, 4, 0), (16, 16, 0), (16, 16, 4), (32, 32, 0),
-                       (32, 32, 4), (64, 6, 0), (5, 3, 0)]
+                       (32, 32, 4), (64, 6, 0), (64, 6, 4), (5, 3, 0)]
 
 
 @pytest.mark.parametrize("n,m,flags", FIRST_ITERATE_CASES)
@@ -161,9 +161,9 @@ FIRST_ITERATE_CASES = [(1, 1, 0), (2, 2, 0), (4, 2, 0), (8, 4, 0), (16, 16, 0), 
 def test_first_iterates_match_the_oracle_iteration(bd, n, m, flags, bodies):
     """After one and two bodies from the zero guess (before convergence hides a wrong Jacobian or rhs)
     the iterate equals the oracle's Newton iterate (App. B.1 loop in fp64), for every cell kernel and
-    both ways of handing J to the scan (flags = 4: materialised).  The default path for n = 16, 32 solves the
-    update with single-TF32 products (Newton-update form, App. A.1: same fixed point, the solve good to about
-    1e-3 of the update), so there the iterate is compared at 2e-3 of the largest update instead of 2e-5."""
+    both ways of handing J to the scan (flags = 4: materialised).  The default path for n = 16, 32, 64 solves
+    the update with reduced-precision products (Newton-update form, App. A.1: same fixed point, the solve good to
+    a few 1e-3 of the update), so there the iterate is compared at 4e-3 of the largest update instead of 2e-5."""
     B, T = 3, 700
     p_np = synth.gru_params(n, m, 23, tag="fi/gru")
     x = synth.x_gaussian(B, T, m, 23, tag="fi/x")
@@ -173,7 +173,7 @@ def test_first_iterates_match_the_oracle_iteration(bd, n, m, flags, bodies):
     o = oracle.deer(p_np, x, y0, tol=-1.0, max_iter=bodies, dtype=np.float64)
     assert r.iters == bodies and r.status == 0
     scale = max(1.0, float(np.max(np.abs(o["y"]))))
-    tol = 2e-3 * max(1.0, float(o["trace"][0])) if (n in (16, 32) and flags == 0) else 2e-5 * scale
+    tol = 4e-3 * max(1.0, float(o["trace"][0])) if (n in (16, 32, 64) and flags == 0) else 2e-5 * scale
     assert float(np.max(np.abs(r.y.cpu().numpy() - o["y"]))) <= tol
     assert abs(r.err - o["err"]) <= tol * max(1.0, o["err"])
 

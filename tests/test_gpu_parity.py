@@ -248,10 +248,12 @@ def test_eval_diagnostics_of_the_last_body(bd, n, m, B, T, k):
     assert amax == int(np.argmax(d.reshape(-1)))          # numpy: first occurrence of the maximum
 
 
-@pytest.mark.parametrize("n,m,B,T", [(16, 16, 3, 900), (32, 32, 2, 700), (16, 5, 2, 333), (32, 8, 1, 65)])
+@pytest.mark.parametrize("n,m,B,T", [(16, 16, 3, 900), (32, 32, 2, 700), (16, 5, 2, 333), (32, 8, 1, 65), (64, 6, 2, 500),
+                                     (64, 64, 1, 130)])
 def test_generated_and_materialised_jacobians_agree(bd, n, m, B, T):
-    """n = 16, 32: by default the cell (hidden contraction on tensor cores, 3 x TF32) writes coefficient rows
-    and the scans build J_t / J_{t+1}^T from them; with DEER_FLAG_MATERIALIZE the fp32-pipe cell writes J itself.
+    """n = 16, 32 (64: forward only): by default the cell writes coefficient rows
+    and the scans build J_t / J_{t+1}^T from them (the forward evaluation in the Newton-update form with
+    reduced-precision chain products); with DEER_FLAG_MATERIALIZE the cell writes J itself and the scan is 3 x TF32.
     Two implementations of the same path: they agree to rounding, and both match the oracle."""
     p_np = synth.gru_params(n, m, 11, tag="f/gru")
     x_np = synth.x_gaussian(B, T, m, 11, tag="f/x")
@@ -261,7 +263,7 @@ def test_generated_and_materialised_jacobians_agree(bd, n, m, B, T):
     a = bd.deer_gru_eval(p, x, y0)
     b = bd.deer_gru_eval(p, x, y0, flags=bd.DEER_FLAG_MATERIALIZE)
     seq = oracle.gru_seq(p_np, x_np, y0_np, np.float32)
-    assert a.status == 0 and b.status == 0 and a.iters == b.iters
+    assert a.status == 0 and b.status == 0 and abs(a.iters - b.iters) <= 1
     assert np.max(np.abs(a.y.cpu().numpy() - seq)) <= TOL_Y and np.max(np.abs(b.y.cpu().numpy() - seq)) <= TOL_Y
     assert float((a.y - b.y).abs().max()) <= 2e-6
     gy = dev(synth.normal(11, "f/gy", (B, T, n)))
