@@ -227,3 +227,19 @@ def multihead_bptt(heads, strides, x, y0, y, gy, dtype=np.float64):
                                                    _p(y0), _p(y), _p(gy), B, T, _p(g["dW_i"]), _p(g["dW_h"]),
                                                    _p(g["db_i"]), _p(g["db_h"]), _p(g["dx"]), _p(g["dy0"]))
     return g
+
+
+def gru_jvp(p, dp, x, dx, y0, dy0, y, dtype=np.float64):
+    """O-7: forward-mode derivative of the trajectory along (dp, dx, dy0); dp is a parameter-shaped
+    object (W_i, W_h, b_i, b_h) or None, dx / dy0 arrays or None.  Returns dy [B,T,n]."""
+    sfx, _ = _sfx(dtype)
+    W_i, W_h, b_i, b_h = _params(p, dtype)
+    x = _c(x, dtype); y0 = _c(y0, dtype); y = _c(y, dtype)
+    B, T, m = x.shape
+    t = (None,) * 4 if dp is None else _params(dp, dtype)
+    dxc = None if dx is None else _c(dx, dtype)
+    dy0c = None if dy0 is None else _c(dy0, dtype)
+    dy = np.empty((B, T, p.n), dtype)
+    getattr(lib(), f"oracle_gru_jvp_{sfx}")(p.n, m, _p(W_i), _p(W_h), _p(b_i), _p(b_h), _p(t[0]), _p(t[1]), _p(t[2]),
+                                            _p(t[3]), _p(x), _p(dxc), _p(y0), _p(dy0c), _p(y), B, T, _p(dy))
+    return dy

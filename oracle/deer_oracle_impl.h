@@ -420,6 +420,73 @@ REAL FN(oracle_classifier_)(int n, int m, int ncls, const REAL *W_i1, const REAL
 }
 
 /* ------------------------------------------------------------------------
+ * O-7  Forward-mode derivative (Sec. 3.1.1, the forward derivative equation:
+ * dy = L_G^{-1}[ (df/dtheta) dtheta ], likewise for x): the first-order
+ * change of the trajectory under a change (dW_i, dW_h, db_i, db_h) of the
+ * parameters, dx [B,T,m] of the inputs and dy0 [B,n] of the initial state,
+ * written out as the sequential tangent recurrence
+ *     dy[t] = J[t] dy[t-1] + df[t],   dy[-1] = dy0,
+ * with df[t] the cell's first-order change at fixed y[t-1]:
+ *     da_r = dW_ir x + W_ir dx + db_ir + dW_hr h + db_hr      (same for z)
+ *     dq   = dW_hn h + db_hn,       du_n = dW_in x + W_in dx + db_in
+ *     dr = r (1-r) da_r,  dz = z (1-z) da_z,  dc = (1-c^2)(du_n + dr q + r dq)
+ *     df = (1-z) dc + (h - c) dz
+ * Any of the tangent arrays may be NULL (= zero).  y is the trajectory.
+ * Pinned by central finite differences of oracle_gru_seq along the direction.
+ * ------------------------------------------------------------------------ */
+void FN(oracle_gru_jvp_)(int n, int m, const REAL *W_i, const REAL *W_h, const REAL *b_i,
+                         const REAL *b_h, const REAL *dW_i, const REAL *dW_h, const REAL *db_i,
+                         const REAL *db_h, const REAL *x, const REAL *dx, const REAL *y0,
+                         const REAL *dy0, const REAL *y, int B, int T, REAL *dy)
+{
+    REAL *gates = (REAL *)malloc(sizeof(REAL) * 4 * (size_t)n);
+    REAL *fv = (REAL *)malloc(sizeof(REAL) * (size_t)n);
+    REAL *J = (REAL *)malloc(sizeof(REAL) * (size_t)n * n);
+    for (int s = 0; s < B; ++s)
+        for (int t = 0; t < T; ++t) {
+            size_t e = (size_t)s * T + t;
+            const REAL *h = (t == 0) ? y0 + (size_t)s * n : y + (e - 1) * n;
+            const REAL *xe = x + e * m;
+            FN(gru_cell_)(n, m, W_i, W_h, b_i, b_h, h, xe, fv, gates);
+            FN(gru_jac_)(n, W_h, h, gates, J);
+            const REAL *r = gates, *z = gates + n, *q = gates + 2 * n, *c = gates + 3 * n;
+            for (int i = 0; i < n; ++i) {
+                REAL dar = 0, daz = 0, dun = 0, dq = 0;
+                for (int k = 0; k < m; ++k) {
+                    if (dW_i) {
+                        dar += dW_i[(size_t)i * m + k] * xe[k];
+                        daz += dW_i[(size_t)(n + i) * m + k] * xe[k];
+                        dun += dW_i[(size_t)(2 * n + i) * m + k] * xe[k];
+                    }
+                    if (dx) {
+                        dar += W_i[(size_t)i * m + k] * dx[e * m + k];
+                        daz += W_i[(size_t)(n + i) * m + k] * dx[e * m + k];
+                        dun += W_i[(size_t)(2 * n + i) * m + k] * dx[e * m + k];
+                    }
+                }
+                if (db_i) { dar += db_i[i]; daz += db_i[n + i]; dun += db_i[2 * n + i]; }
+                if (dW_h)
+                    for (int k = 0; k < n; ++k) {
+                        dar += dW_h[(size_t)i * n + k] * h[k];
+                        daz += dW_h[(size_t)(n + i) * n + k] * h[k];
+                        dq += dW_h[(size_t)(2 * n + i) * n + k] * h[k];
+                    }
+                if (db_h) { dar += db_h[i]; daz += db_h[n + i]; dq += db_h[2 * n + i]; }
+                REAL dr = r[i] * ((REAL)1 - r[i]) * dar;
+                REAL dz = z[i] * ((REAL)1 - z[i]) * daz;
+                REAL dc = ((REAL)1 - c[i] * c[i]) * (dun + dr * q[i] + r[i] * dq);
+                REAL acc = ((REAL)1 - z[i]) * dc + (h[i] - c[i]) * dz;            /* df */
+                for (int k = 0; k < n; ++k) {
+                    REAL dprev = (t == 0) ? (dy0 ? dy0[(size_t)s * n + k] : (REAL)0) : dy[(e - 1) * n + k];
+                    acc += J[(size_t)i * n + k] * dprev;
+                }
+                dy[e * n + i] = acc;
+            }
+        }
+    free(gates); free(fv); free(J);
+}
+
+/* ------------------------------------------------------------------------
  * O-6  Multi-head GRU (Sec. 4.4; App. B.4): H independent GRU heads of hidden
  * size n read the same input x[b][t] (m channels); head h has its own
  * parameters and a stride s_h and advances

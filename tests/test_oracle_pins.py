@@ -469,3 +469,46 @@ def test_multihead_bptt_reduces_to_plain_bptt_per_phase():
     for k in ("dW_i", "dW_h", "db_i", "db_h"):
         assert np.allclose(g[k][0], acc[k], atol=1e-12), k
     assert np.allclose(g["dy0"][:, 0], acc["dy0"], atol=1e-13)
+
+
+# ----------------------------------------------------------------------------- forward-mode derivative (Sec. 3.1.1)
+def test_jvp_matches_central_differences_of_the_sequential_trajectory():
+    """dy = L_G^{-1}[df/dtheta dtheta] (+ the x and y0 directions): the tangent recurrence against the
+    difference quotient of the sequential evaluation along the same direction."""
+    p, x, y0 = small(3, 2, 2, 25, seed=8)
+    p64 = p.astype(np.float64); x64 = x.astype(np.float64); y064 = y0.astype(np.float64)
+    dp = synth.GruParams(3, 2, *(synth.normal(8, f"t/dp{i}", a.shape).astype(np.float64)
+                                 for i, a in enumerate((p.W_i, p.W_h, p.b_i, p.b_h))))
+    dx = synth.normal(8, "t/dx", x.shape).astype(np.float64)
+    dy0 = synth.normal(8, "t/dy0", y0.shape).astype(np.float64)
+    y = oracle.gru_seq(p64, x64, y064)
+    eps = 1e-6
+
+    def shifted(sign, use_p, use_x, use_y0):
+        q = synth.GruParams(3, 2, *((a + sign * eps * d) if use_p else a for a, d in
+                                    ((p64.W_i, dp.W_i), (p64.W_h, dp.W_h), (p64.b_i, dp.b_i), (p64.b_h, dp.b_h))))
+        return oracle.gru_seq(q, x64 + (sign * eps * dx if use_x else 0.0), y064 + (sign * eps * dy0 if use_y0 else 0.0))
+
+    for use_p, use_x, use_y0 in ((True, False, False), (False, True, False), (False, False, True), (True, True, True)):
+        fd = (shifted(+1, use_p, use_x, use_y0) - shifted(-1, use_p, use_x, use_y0)) / (2 * eps)
+        got = oracle.gru_jvp(p64, dp if use_p else None, x64, dx if use_x else None, y064,
+                             dy0 if use_y0 else None, y)
+        assert np.max(np.abs(got - fd)) <= 2e-8, (use_p, use_x, use_y0)
+
+
+def test_jvp_is_the_transpose_of_the_gradient():
+    """<gy, dy> = <dL/dtheta, dtheta> + <dL/dx, dx> + <dL/dy0, dy0>: the forward derivative paired with any
+    gy equals the backward derivative (Sec. 3.1.1, both equations) paired with the direction."""
+    p, x, y0 = small(4, 3, 2, 30, seed=9)
+    p64 = p.astype(np.float64)
+    y = oracle.gru_seq(p64, x, y0)
+    dp = synth.GruParams(4, 3, *(synth.normal(9, f"t/dq{i}", a.shape).astype(np.float64)
+                                 for i, a in enumerate((p.W_i, p.W_h, p.b_i, p.b_h))))
+    dx = synth.normal(9, "t/dx2", x.shape).astype(np.float64)
+    dy0 = synth.normal(9, "t/dy02", y0.shape).astype(np.float64)
+    gy = synth.normal(9, "t/gy2", y.shape).astype(np.float64)
+    dy = oracle.gru_jvp(p64, dp, x, dx, y0, dy0, y)
+    g = oracle.gru_bptt(p64, x, y0, y, gy)
+    rhs = sum(float(np.sum(g["d" + k] * getattr(dp, k))) for k in ("W_i", "W_h", "b_i", "b_h"))
+    rhs += float(np.sum(g["dx"] * dx)) + float(np.sum(g["dy0"] * dy0))
+    assert abs(float(np.sum(gy * dy)) - rhs) <= 1e-10 * max(1.0, abs(rhs))
