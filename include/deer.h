@@ -243,6 +243,20 @@ int deer_gru_vjp(const deer_gru_params *params, const float *x, const float *y0,
                  const float *gy, int B, int T, const deer_gru_grads *dparams, float *dx,
                  float *dy0, void *ws, size_t ws_bytes, int flags, void *stream);
 
+/* Forward-mode derivative (Sec. 3.1.1, the forward derivative equation): the first-order change dy of the
+ * trajectory y under a change of the parameters, the inputs and the initial state,
+ *     dy = L_G^{-1}[ (df/dtheta) dtheta + (df/dx) dx ]   started from dy0,
+ * by ONE forward scan with the Jacobians at y (the same operator the iteration inverts; Eq. 9-10):
+ * df at every position from the direction, then dy[t] = J[t] dy[t-1] + df[t], dy[-1] = dy0.
+ *   params  : the parameters          dparams : the direction in parameter space, same n and m; device
+ *             arrays W_i with b_i and/or W_h with b_h may be NULL pairs (= 0); dparams itself may be NULL
+ *   x [B,T,m]   dx [B,T,m] or NULL    y0 [B,n]   dy0 [B,n] or NULL    y [B,T,n] the trajectory
+ *   dy [B,T,n] out          ws : deer_workspace_bytes(DEER_OP_VJP, ...) bytes
+ * Asynchronous on `stream` (see deer_workspace_status).  Returns DEER_OK or a negative status. */
+int deer_gru_jvp(const deer_gru_params *params, const deer_gru_params *dparams, const float *x, const float *dx,
+                 const float *y0, const float *dy0, const float *y, int B, int T, float *dy, void *ws,
+                 size_t ws_bytes, int flags, void *stream);
+
 /* One training step of the long-series classifier (App. B.3 shapes: mean
  * over the sequence, then a linear decoder and cross-entropy): two stacked
  * GRU layers of equal hidden size n (layer 1 reads x [B,T,m], layer 2 reads

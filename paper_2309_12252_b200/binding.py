@@ -28,7 +28,7 @@ EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc
            "deer_gru_eval_diag", "deer_gru_eval_host", "deer_gru_vjp",
            "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count",
            "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_cell_jac",
-           "deer_multihead_workspace_bytes", "deer_gru_multihead_eval", "deer_gru_multihead_vjp"]
+           "deer_multihead_workspace_bytes", "deer_gru_multihead_eval", "deer_gru_multihead_vjp", "deer_gru_jvp"]
 
 
 class _Params(ctypes.Structure):
@@ -93,6 +93,8 @@ def lib():
         L.deer_gru_multihead_vjp.restype = ci
         L.deer_gru_multihead_vjp.argtypes = [ctypes.POINTER(_Params), ctypes.POINTER(ci), ci, vp, vp, vp, vp, ci, ci,
                                              ctypes.POINTER(_Grads), vp, vp, vp, sz, ci, vp]
+        L.deer_gru_jvp.restype = ci
+        L.deer_gru_jvp.argtypes = [ctypes.POINTER(_Params), ctypes.POINTER(_Params), vp, vp, vp, vp, vp, ci, ci, vp, vp, sz, ci, vp]
         L.deer_status_string.restype = ctypes.c_char_p
         L.deer_status_string.argtypes = [ci]
         L.deer_last_error.restype = ctypes.c_char_p
@@ -421,3 +423,21 @@ def deer_gru_multihead_vjp(heads, strides, x, y0, y, gy, ws=None, flags=0, strea
         raise DeerError(rc)
     g["dx"], g["dy0"] = dx, dy0
     return g
+
+
+def deer_gru_jvp(params, dparams, x, dx, y0, dy0, y, ws=None, flags=0, stream=None):
+    """Forward-mode derivative dy [B,T,n] of the trajectory y along (dparams, dx, dy0); any of the three may be
+    None.  dparams: a GruParamsDev holding the direction; see include/deer.h."""
+    B, T, m = x.shape
+    n = params.n
+    dy = torch.empty((B, T, n), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = alloc_workspace(DEER_OP_VJP, B, T, n, m, flags, x.device)
+    ps = params.c_struct()
+    dps = None if dparams is None else dparams.c_struct()
+    rc = lib().deer_gru_jvp(ctypes.byref(ps), None if dps is None else ctypes.byref(dps), _ptr(_f32(x)), _ptr(dx),
+                            _ptr(_f32(y0)), _ptr(dy0), _ptr(_f32(y)), B, T, _ptr(dy), _ptr(ws), ws.numel(), flags,
+                            _stream(stream))
+    if rc != DEER_OK:
+        raise DeerError(rc)
+    return dy

@@ -1230,6 +1230,61 @@ int deer_gru_classifier_step(const deer_gru_params *l1, const deer_gru_params *l
     return s1 > s2 ? s1 : s2;
 }
 
+int deer_gru_jvp(const deer_gru_params *p, const deer_gru_params *dp, const float *x, const float *dx, const float *y0,
+                 const float *dy0, const float *y, int B, int T, float *dy, void *ws, size_t ws_bytes, int flags,
+                 void *stream)
+{
+    if (!p || !x || !y0 || !y || !dy || !p->W_i || !p->W_h || !p->b_i || !p->b_h) return DEER_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || p->n <= 0 || p->m <= 0) return DEER_ERR_INVALID_ARG;
+    if (dp && (dp->n != p->n || dp->m != p->m)) return DEER_ERR_INVALID_ARG;
+    if (!supported(p->n, p->m)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
+    const int n = p->n, m = p->m, n3 = 3 * n;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the gradient's workspace layout holds what is needed: u, J, and three [B,T,3n] / [B,T,n] arrays
+    VjpWs w = carve_vjp(ws, B, T, n, m);
+    int rc = check_ws(ws, ws_bytes, w.bytes);
+    if (rc != DEER_OK) return rc;
+    const size_t N = (size_t)B * T;
+    DEER_CHECK_CUDA(cudaMemsetAsync(w.st, 0, sizeof(StatusBlock), st), "memset status");
+    if ((rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
+    // du1 = x dW_i^T + db_i ;  du2 = dx W_i^T
+    float *du1 = nullptr, *du2 = nullptr;
+    const bool have_di = dp && (dp->W_i || dp->b_i);
+    if (have_di) {
+        if (!dp->W_i || !dp->b_i) return DEER_ERR_INVALID_ARG;       // the input-side pair comes together
+        deer_gru_params q = *p;
+        q.W_i = dp->W_i; q.b_i = dp->b_i;
+        du1 = w.dGi;
+        if ((rc = run_proj(&q, x, du1, N, st)) != DEER_OK) return rc;
+    }
+    if (dx) {
+        du2 = w.dGh;
+        if ((rc = run_affine(dx, p->W_i, nullptr, du2, N, m, n3, 0, st)) != DEER_OK) return rc;
+    }
+    if (dp && ((dp->W_h == nullptr) != (dp->b_h == nullptr))) return DEER_ERR_INVALID_ARG;
+    {
+        JvpArgs j{p->W_h, p->b_h, dp ? dp->W_h : nullptr, dp ? dp->b_h : nullptr, w.u, du1, du2, y, y0, w.lam, B, T, n};
+        const size_t sm = sizeof(float) * (6 * (size_t)n * (n + 1) + 6 * n);
+        if ((rc = opt_in_smem((const void *)jvp_cell_kernel, sm)) != DEER_OK) return rc;
+        const int epb = 256 / n;
+        size_t blocks = (N + epb - 1) / epb;
+        const size_t cap = (size_t)num_sms() * 8;
+        if (blocks > cap) blocks = cap;
+        DEER_KERNEL("jvp_cell_kernel", st, jvp_cell_kernel<<<(unsigned)blocks, 256, sm, st>>>(j));
+    }
+    // the Jacobians at the trajectory (exact: a one-shot solve), then dy = L_G^{-1}[df] from dy0 (Sec. 3.1.1)
+    ScanArgs a{};
+    a.J = w.J; a.b = w.lam; a.y0 = dy0; a.y = dy; a.yold = nullptr;
+    a.B = B; a.T = T; a.n = n; a.reverse = 0;
+    a.L = w.scan.L; a.nch = w.scan.nch;
+    a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
+    a.st = w.st;
+    CellArgs c{p->W_h, p->b_h, w.u, x, p->W_i, p->b_i, m, y, y0, w.J, nullptr, B, T, n, nullptr, 0, 0};
+    if ((rc = run_cell(c, st)) != DEER_OK) return rc;
+    return run_scan(a, w.scan, flags, st);
+}
+
 size_t deer_multihead_workspace_bytes(const int *strides, int H, int B, int T, int n, int m, int flags)
 {
     (void)flags;

@@ -846,6 +846,64 @@ __global__ void broadcast_gy_kernel(const float *__restrict__ gpool, float *__re
 }
 
 
+// ------------------------------------------------------------------ forward-mode derivative of the cell (Sec. 3.1.1)
+// df at every position for a direction (dW_i, dW_h, db_i, db_h, dx) at fixed h = y_prev:
+//   da_r = du_r + dW_hr h + db_hr,  da_z likewise,  dq = dW_hn h + db_hn,  du = x dW_i^T + db_i + dx W_i^T (precomputed)
+//   dr = r (1-r) da_r,  dz = z (1-z) da_z,  dc = (1-c^2)(du_n + dr q + r dq),  df = (1-z) dc + (h-c) dz
+// One thread per (position, row); W_h and dW_h in shared memory (rows padded by one float).
+struct JvpArgs {
+    const float *W_h, *b_h, *dW_h, *db_h;    // dW_h, db_h may be nullptr (= 0)
+    const float *u;                          // [B,T,3n]  x W_i^T + b_i
+    const float *du1, *du2;                  // [B,T,3n]  x dW_i^T + db_i  and  dx W_i^T (either may be nullptr)
+    const float *y, *y0;
+    float *df;                               // [B,T,n] out
+    int B, T, n;
+};
+
+__global__ void jvp_cell_kernel(JvpArgs a)
+{
+    extern __shared__ float sW[];
+    const int n = a.n, ld = n + 1;
+    float *sD = sW + 3 * n * ld;
+    float *sb = sD + 3 * n * ld, *sdb = sb + 3 * n;
+    for (int i = threadIdx.x; i < 3 * n * n; i += blockDim.x) {
+        sW[(i / n) * ld + (i % n)] = a.W_h[i];
+        sD[(i / n) * ld + (i % n)] = a.dW_h ? a.dW_h[i] : 0.0f;
+    }
+    for (int i = threadIdx.x; i < 3 * n; i += blockDim.x) { sb[i] = a.b_h[i]; sdb[i] = a.db_h ? a.db_h[i] : 0.0f; }
+    __syncthreads();
+    const int epb = blockDim.x / n;
+    const int le = threadIdx.x / n, i = threadIdx.x % n;
+    const size_t N = (size_t)a.B * a.T;
+    for (size_t e = (size_t)blockIdx.x * epb + le; le < epb && e < N; e += (size_t)gridDim.x * epb) {
+        const int t = (int)(e % a.T);
+        const size_t seq = e / a.T;
+        const float *hp = (t == 0) ? a.y0 + seq * n : a.y + (e - 1) * n;
+        float gr = sb[i], gz = sb[n + i], gq = sb[2 * n + i];
+        float dar = sdb[i], daz = sdb[n + i], dq = sdb[2 * n + i];
+        for (int k = 0; k < n; ++k) {
+            const float h = hp[k];
+            gr = fmaf(sW[i * ld + k], h, gr);
+            gz = fmaf(sW[(n + i) * ld + k], h, gz);
+            gq = fmaf(sW[(2 * n + i) * ld + k], h, gq);
+            dar = fmaf(sD[i * ld + k], h, dar);
+            daz = fmaf(sD[(n + i) * ld + k], h, daz);
+            dq = fmaf(sD[(2 * n + i) * ld + k], h, dq);
+        }
+        const float *ue = a.u + e * 3 * n;
+        float dun = 0.0f;
+        if (a.du1) { const float *d = a.du1 + e * 3 * n; dar += d[i]; daz += d[n + i]; dun += d[2 * n + i]; }
+        if (a.du2) { const float *d = a.du2 + e * 3 * n; dar += d[i]; daz += d[n + i]; dun += d[2 * n + i]; }
+        const float r = sigmoidf_acc(ue[i] + gr);
+        const float z = sigmoidf_acc(ue[n + i] + gz);
+        const float c = tanhf(ue[2 * n + i] + r * gq);
+        const float dr = r * (1.0f - r) * dar;
+        const float dz = z * (1.0f - z) * daz;
+        const float dc = (1.0f - c * c) * (dun + dr * gq + r * dq);
+        a.df[e * n + i] = (1.0f - z) * dc + (hp[i] - c) * dz;
+    }
+}
+
 // ---------------------------------------------------------------- multi-head GRU: strided views <-> dense batches
 // A head of stride s over [B,T] is s interleaved sequences per batch entry (Sec. 4.4): sequence (b, p) holds the
 // positions t = p + s t', t' = 0 .. T'-1 with T' = ceil(T / s); shorter phases are padded at the END with zeros
