@@ -68,7 +68,8 @@ def tf32_peak_tflops(pk) -> float:
 # DRAM bytes (read + write) per position from the ncu captures summarised under profiles/ (inputs larger
 # than L2; traffic grows in proportion to the positions processed, so a launch's traffic is this times B*T).
 NCU_SCAN_TRAFFIC_PER_POSITION = {1: 12.8, 2: 32.7, 4: 95.3, 8: 606.6, 16: 2213.0, 32: 8622.0, 64: 34116.0}
-NCU_FUSED_SCAN_TRAFFIC_PER_POSITION = {32: 1375.0}      # scan_warpnf_kernel<32> inside deer_gru_eval
+# the two launches of the scan inside deer_gru_eval (n = 16, 32, 64): reduce, apply
+NCU_FUSED_TRAFFIC_PER_POSITION = {"scan_fused_reduce_kernel": {32: 686.0}, "scan_fused_apply_kernel": {32: 916.0}}
 NCU_CONFIG2_SCAN_TRAFFIC = 51.43e6                      # scan_warp8_kernel inside the config-2 step, per launch
 
 
@@ -78,9 +79,12 @@ def scan_bytes_per_position(n: int) -> int:
 
 
 def fused_scan_bytes_per_position(n: int) -> int:
-    """The scan inside deer_gru_eval for n = 16, 32 (J generated from four coefficient vectors per position):
-    read the coefficient rows (16n), the right-hand side (4n) and the previous iterate (4n), write y (4n)."""
+    """The scan inside deer_gru_eval for n = 16, 32, 64 (J generated from four coefficient vectors per position):
+    read the coefficient rows (16n), the residual (4n) and the previous iterate (4n) once, write y (4n)."""
     return 28 * n
+
+
+FUSED_KERNEL_BYTES = {"scan_fused_reduce_kernel": 20, "scan_fused_reduce64_kernel": 20, "scan_fused_apply_kernel": 32}   # x n
 
 
 def scan_flops_per_position(n: int) -> int:
@@ -88,11 +92,12 @@ def scan_flops_per_position(n: int) -> int:
     return 2 * n * n * (n + 1)
 
 
-def roofline_of_scan(n, positions, ms, pk, bytes_per_position, traffic_per_position, kernel, extra=None):
-    """The slower of the byte bound (measured HBM copy rate) and the flop bound (TF32 tensor peak) is the scan's
-    roofline; `frac` = that bound's time / measured time, `achieved` in the unit of the binding resource."""
+def roofline_of_scan(n, positions, ms, pk, bytes_per_position, traffic_per_position, kernel, extra=None, bf16=False):
+    """The slower of the byte bound (measured HBM copy rate) and the flop bound (tensor peak of the kernel's MMA
+    type: TF32, or bf16 when `bf16`) is the scan's roofline; `frac` = that bound's time / measured time,
+    `achieved` in the unit of the binding resource."""
     t_bytes = bytes_per_position * positions / (pk["hbm_gbs"] * 1e9) * 1e3
-    tf32 = tf32_peak_tflops(pk)
+    tf32 = pk["bf16_tflops"] if bf16 else tf32_peak_tflops(pk)
     t_flops = scan_flops_per_position(n) * positions / (tf32 * 1e12) * 1e3
     hbm_bound = t_bytes >= t_flops
     gbs = bytes_per_position * positions / (ms * 1e-3) / 1e9
@@ -100,7 +105,8 @@ def roofline_of_scan(n, positions, ms, pk, bytes_per_position, traffic_per_posit
     out = dict(bound="hbm" if hbm_bound else "tensor", kernel=kernel,
                achieved=gbs if hbm_bound else tfs, peak=pk["hbm_gbs"] if hbm_bound else tf32,
                unit="GB/s" if hbm_bound else "TFLOP/s", frac=(t_bytes if hbm_bound else t_flops) / ms,
-               peak_source=pk["source"] + ("" if hbm_bound else " bf16 burst x 1.1/2.25 (nominal TF32/bf16 ratio)"),
+               peak_source=pk["source"] + ("" if hbm_bound else " bf16 burst" if bf16 else " bf16 burst x 1.1/2.25 (nominal TF32/bf16 ratio)"),
+               tensor_peak_tflops=tf32, tensor_dtype="bf16" if bf16 else "tf32",
                ms_per_launch=ms, positions_per_launch=positions, bytes_per_position=bytes_per_position,
                flops_per_position=scan_flops_per_position(n),
                hbm_frac=t_bytes / ms, tensor_frac=t_flops / ms, achieved_gbs=gbs, achieved_tflops=tfs,
@@ -338,7 +344,7 @@ def eval_point(bd, synth, device, n, m, B, T, flags, steps, warmup, vjp=False, b
         if scan_ms > 0 and r.iters > 0:
             pk = peaks()
             per = scan_ms / r.iters
-            fused = any(k.startswith("scan_warpnf") for k in prof)
+            fused = any(k.startswith("scan_fused") or k.startswith("scan_warpnf") for k in prof)
             bpp = fused_scan_bytes_per_position(n) if fused else scan_bytes_per_position(n)
             rl = roofline_of_scan(n, B * T, per, pk, bpp, None, "+".join(k for k in prof if is_scan_kernel(k)))
             out["scan_ms_per_iter"] = per
@@ -585,13 +591,24 @@ def step_scan_roofline(m, pk):
         return None
     n, positions = m["n"], m["B"] * m["T"]
     per = scan_ms / launches
-    fused = any(k.startswith("scan_warpnf") for k in names)
+    fused = [k for k in names if k.startswith("scan_fused")]
     if fused:
-        return roofline_of_scan(n, positions, per, pk, fused_scan_bytes_per_position(n),
-                                NCU_FUSED_SCAN_TRAFFIC_PER_POSITION.get(n), "+".join(names),
-                                dict(note="scan inside the step, J generated from coefficient rows: bytes = coefficient rows, "
-                                          "rhs, previous iterate read once + y written; flops = 2 n^2 (n+1) per position",
-                                     traffic_note="ncu capture of this kernel at T = 20,000 scaled by positions (profiles/)"))
+        # two launches per scan: the roofline object is the dominant kernel's (its own bytes and flops); the pair
+        # is reported against the scan's algorithmic bytes (everything read once) beside it
+        per_kernel = {k: prof[k]["total_ms"] / prof[k]["launches"] for k in fused}
+        dom = max(per_kernel, key=per_kernel.get)
+        reduce_k = dom.startswith("scan_fused_reduce")
+        out = roofline_of_scan(n, positions, per_kernel[dom], pk, FUSED_KERNEL_BYTES[dom] * n,
+                               NCU_FUSED_TRAFFIC_PER_POSITION.get(dom, {}).get(n), dom, bf16=reduce_k,
+                               extra=dict(note="dominant kernel of the step: the chunk reduce of the two-launch scan (J generated from "
+                                               "coefficient rows; bf16 m16n8k16 chain products).  bytes = coefficient rows + residual "
+                                               "read once (20 n per position); flops = 2 n^2 (n+1) per position",
+                                          traffic_note="ncu capture of this kernel at T = 20,000 scaled by positions (profiles/)"))
+        pair_ms = sum(per_kernel.values())
+        out["scan_pair"] = dict(kernels=per_kernel, ms_per_scan=pair_ms, bytes_per_position=fused_scan_bytes_per_position(n),
+                                hbm_frac=fused_scan_bytes_per_position(n) * positions / (pk["hbm_gbs"] * 1e9) * 1e3 / pair_ms,
+                                note="reduce + apply of one Newton body against the scan's algorithmic bytes (28 n per position)")
+        return out
     extra = None
     traffic = NCU_SCAN_TRAFFIC_PER_POSITION.get(n)
     if m["cfg"] is WORKLOADS[2]:
@@ -679,14 +696,19 @@ def main():
         torch.cuda.empty_cache()
         # ---- config 4: full training step of the 2-layer n = 64 classifier
         c4 = time_classifier(bd, synth, torch, device, 32, 17_984, 0, 3, 2)
-        scan_ms = sum(v["ms"] for k, v in c4["kernels"].items() if is_scan_kernel(k))
-        scan_launches = sum(v["launches"] for k, v in c4["kernels"].items() if is_scan_kernel(k))
+        k4 = c4["kernels"]
+        per4 = lambda name: k4[name]["ms"] / k4[name]["launches"] if name in k4 else None
+        fwd_ms = (per4("scan_fused_reduce64_kernel") or 0.0) + (per4("scan_fused_apply_kernel") or 0.0)
         extras["config4_training_step"] = dict(
             workload="config4: 2-layer GRU n=64 m=6 B=32 T=17984, mean-pool, 5-class head; loss + all gradients",
             ms_per_step=c4["ms"], value=c4["steps_per_s"], unit=UNIT, newton_iters=c4["iters"], loss=c4["loss"],
-            kernels=c4["kernels"],
-            scan_roofline=roofline_of_scan(64, 32 * 17_984, scan_ms / max(scan_launches, 1), pk, scan_bytes_per_position(64),
-                                           NCU_SCAN_TRAFFIC_PER_POSITION[64], "scan_cta64_kernel (forward and reverse)"))
+            kernels=k4,
+            forward_scan=dict(ms_per_scan=fwd_ms, kernels="scan_fused_reduce64_kernel + scan_fused_apply_kernel",
+                              bytes_per_position=fused_scan_bytes_per_position(64),
+                              hbm_frac=fused_scan_bytes_per_position(64) * 32 * 17_984 / (pk["hbm_gbs"] * 1e9) * 1e3 / max(fwd_ms, 1e-9),
+                              tensor_frac_bf16=scan_flops_per_position(64) * 32 * 17_984 / (pk["bf16_tflops"] * 1e12) * 1e3 / max(fwd_ms, 1e-9)),
+            reverse_scan_roofline=roofline_of_scan(64, 32 * 17_984, per4("scan_cta64_kernel") or 1.0, pk, scan_bytes_per_position(64),
+                                                   NCU_SCAN_TRAFFIC_PER_POSITION[64], "scan_cta64_kernel (reverse, 3 x TF32)"))
         torch.cuda.empty_cache()
         # ---- the multi-head GRU unit of the paper's sequential-image model
         extras["multihead_unit"] = time_multihead(bd, synth, torch, device, 32, 1024, 32, 8, 256, 5, 2, cpu_seconds=2.0)
