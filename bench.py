@@ -222,7 +222,7 @@ def run_reference(args):
         return
     from paper_2309_12252_b200 import synth
     import oracle
-    w = synth.config(HEADLINE)
+    w = synth.config(args.workload)
     for _ in range(max(args.warmup, 1)):
         oracle.gru_seq(w.params, w.x, w.y0, np.float32)
     t0 = time.perf_counter()
@@ -233,7 +233,7 @@ def run_reference(args):
     cores = min(oracle.num_threads(), w.B)
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
                 ms_per_step=1e3 * dt / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
-                dtype="f32", data="synthetic", impl="reference", config=dict(WORKLOADS[HEADLINE]),
+                dtype="f32", data="synthetic", impl="reference", config=dict(WORKLOADS[args.workload]),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle",
                                   sample=f"{args.steps} full passes of the sequential fp32 GRU loop over the whole workload"),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
@@ -346,7 +346,7 @@ def eval_point(bd, synth, device, n, m, B, T, flags, steps, warmup, vjp=False, b
             per = scan_ms / r.iters
             fused = any(k.startswith("scan_fused") or k.startswith("scan_warpnf") for k in prof)
             bpp = fused_scan_bytes_per_position(n) if fused else scan_bytes_per_position(n)
-            rl = roofline_of_scan(n, B * T, per, pk, bpp, None, "+".join(k for k in prof if is_scan_kernel(k)))
+            rl = roofline_of_scan(n, B * T, per, pk, bpp, None, "+".join(k for k in prof if is_scan_kernel(k)), bf16=fused)
             out["scan_ms_per_iter"] = per
             out["scan_bound"] = rl["bound"]
             out["scan_frac"] = rl["frac"]
@@ -633,6 +633,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="deer", choices=["deer", "reference"])
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--workload", type=int, default=HEADLINE, choices=sorted(WORKLOADS),
+                    help="configuration measured as the step (default: the headline, config 3)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the other workloads and the HBM-sized stand-alone scans (headline workload only)")
     args = ap.parse_args()
@@ -681,7 +683,7 @@ def main():
 
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
-    head = measure_workload(bd, torch, synth, HEADLINE, rank, device, dist, args.steps, args.warmup, flush, sampler)
+    head = measure_workload(bd, torch, synth, args.workload, rank, device, dist, args.steps, args.warmup, flush, sampler)
     roofline = step_scan_roofline(head, pk)
 
     extras = {}
@@ -689,8 +691,9 @@ def main():
     if rank == 0 and not args.no_extras:
         torch.cuda.empty_cache()
         # ---- the other forward workload of the definition (L2-resident)
-        c2 = measure_workload(bd, torch, synth, 2, 0, device, None, max(args.steps, 20), args.warmup, flush)
-        extras["config2"] = dict(workload=c2["cfg"]["workload"], value=c2["value"], unit=UNIT, ms_per_step=c2["ms_per_step"],
+        other = 2 if args.workload != 2 else 3
+        c2 = measure_workload(bd, torch, synth, other, 0, device, None, max(args.steps, 20), args.warmup, flush)
+        extras[f"config{other}"] = dict(workload=c2["cfg"]["workload"], value=c2["value"], unit=UNIT, ms_per_step=c2["ms_per_step"],
                                  newton_iters=c2["iters"], e2e=c2["e2e"], kernels=c2["kernels"],
                                  roofline=step_scan_roofline(c2, pk))
         torch.cuda.empty_cache()
@@ -730,7 +733,7 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1:
-        v, reps, dt, cores = cpu_oracle_rate(synth.config(HEADLINE), args.cpu_seconds)
+        v, reps, dt, cores = cpu_oracle_rate(synth.config(args.workload), args.cpu_seconds)
         cpu = dict(value=v, unit=UNIT, cores=cores, kind="oracle",
                    sample=f"{reps} full passes of the oracle's sequential fp32 GRU loop over the whole workload ({dt:.1f} s)")
 
