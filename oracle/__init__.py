@@ -243,3 +243,17 @@ def gru_jvp(p, dp, x, dx, y0, dy0, y, dtype=np.float64):
     getattr(lib(), f"oracle_gru_jvp_{sfx}")(p.n, m, _p(W_i), _p(W_h), _p(b_i), _p(b_h), _p(t[0]), _p(t[1]), _p(t[2]),
                                             _p(t[3]), _p(x), _p(dxc), _p(y0), _p(dy0c), _p(y), B, T, _p(dy))
     return dy
+
+
+def ode_linear(G, z, t, y0, dtype=np.float64, want_discrete=False):
+    """O-8: y = L_G^{-1}[z] for dy/dt + G(t) y = z(t), y(t_0) = y0 (Sec. 3.3): G [B,T,n,n], z [B,T,n] at the
+    time points t [T], mid-point values per interval.  Returns y [B,T,n] (and Gbar, zbar if asked)."""
+    sfx, _ = _sfx(dtype)
+    G = _c(G, dtype); z = _c(z, dtype); t = _c(t, dtype); y0 = _c(y0, dtype)
+    B, T, n = z.shape
+    assert G.shape == (B, T, n, n) and t.shape == (T,) and y0.shape == (B, n)
+    y = np.empty((B, T, n), dtype)
+    Gb = np.empty((B, max(T - 1, 0), n, n), dtype) if want_discrete else None
+    zb = np.empty((B, max(T - 1, 0), n), dtype) if want_discrete else None
+    getattr(lib(), f"oracle_ode_linear_{sfx}")(_p(G), _p(z), _p(t), _p(y0), B, T, n, _p(y), _p(Gb), _p(zb))
+    return (y, Gb, zb) if want_discrete else y

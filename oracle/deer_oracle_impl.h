@@ -487,6 +487,96 @@ void FN(oracle_gru_jvp_)(int n, int m, const REAL *W_i, const REAL *W_h, const R
 }
 
 /* ------------------------------------------------------------------------
+ * O-8  The linear operator L_G^{-1} of an ODE (Sec. 3.3): dy/dt + G(t) y = z(t),
+ * y(t_0) = y0, with G and z given at the time points t_0 < ... < t_{T-1} and
+ * taken constant at their MID-POINT values on every interval,
+ *     G_i = (G(t_i) + G(t_{i+1})) / 2,   z_i likewise,   D_i = t_{i+1} - t_i,
+ *     y_{i+1} = Gbar_i y_i + zbar_i,  Gbar_i = exp(-G_i D_i),  zbar_i = G_i^{-1}(I - Gbar_i) z_i.
+ * Both come from ONE matrix exponential of the augmented matrix
+ *     exp( [ -G_i D_i   z_i D_i ] )  =  [ Gbar_i  zbar_i ]
+ *        ( [     0         0    ] )     [   0       1    ]
+ * (an identity of the matrix exponential: it needs no inverse, so singular G is
+ * fine), evaluated by scaling and squaring with a Taylor polynomial.
+ * y [B,T,n] with y[b][0] = y0[b].  Optionally returns Gbar [B,T-1,n,n], zbar [B,T-1,n].
+ * Pinned by: scalar closed form, a library matrix exponential, the exact
+ * solution for constant coefficients, second-order convergence for varying
+ * ones (App. A.5), G = 0.
+ * ------------------------------------------------------------------------ */
+static void FN(expm_aug_)(int n, const REAL *G, const REAL *z, REAL D, REAL *Gbar, REAL *zbar, REAL *work /* 3 (n+1)^2 */)
+{
+    const int m = n + 1;
+    REAL *A = work, *P = work + m * m, *Q = work + 2 * m * m;
+    REAL norm = 0;
+    for (int i = 0; i < m; ++i) {
+        REAL rs = 0;
+        for (int j = 0; j < m; ++j) {
+            REAL v = 0;
+            if (i < n) v = (j < n) ? -G[(size_t)i * n + j] * D : z[i] * D;
+            A[i * m + j] = v;
+            rs += R_ABS(v);
+        }
+        if (rs > norm) norm = rs;
+    }
+    int s = 0;
+    while (norm > (REAL)0.25 && s < 60) { norm *= (REAL)0.5; ++s; }
+    REAL scale = (REAL)1;
+    for (int k = 0; k < s; ++k) scale *= (REAL)0.5;
+    for (int i = 0; i < m * m; ++i) A[i] *= scale;
+    /* Horner: P = I + A (I + A/2 (I + A/3 ( ... (I + A/K)))) */
+    const int K = 18;
+    for (int i = 0; i < m * m; ++i) P[i] = (i / m == i % m) ? (REAL)1 : (REAL)0;
+    for (int k = K; k >= 1; --k) {
+        for (int i = 0; i < m; ++i)
+            for (int j = 0; j < m; ++j) {
+                REAL acc = 0;
+                for (int l = 0; l < m; ++l) acc += A[i * m + l] * P[l * m + j];
+                Q[i * m + j] = acc / (REAL)k + ((i == j) ? (REAL)1 : (REAL)0);
+            }
+        for (int i = 0; i < m * m; ++i) P[i] = Q[i];
+    }
+    for (int k = 0; k < s; ++k) {
+        for (int i = 0; i < m; ++i)
+            for (int j = 0; j < m; ++j) {
+                REAL acc = 0;
+                for (int l = 0; l < m; ++l) acc += P[i * m + l] * P[l * m + j];
+                Q[i * m + j] = acc;
+            }
+        for (int i = 0; i < m * m; ++i) P[i] = Q[i];
+    }
+    for (int i = 0; i < n; ++i) {
+        for (int j = 0; j < n; ++j) Gbar[(size_t)i * n + j] = P[i * m + j];
+        zbar[i] = P[i * m + n];
+    }
+}
+
+void FN(oracle_ode_linear_)(const REAL *G, const REAL *z, const REAL *t, const REAL *y0, int B, int T, int n,
+                            REAL *y, REAL *Gbar_out, REAL *zbar_out)
+{
+    REAL *Gm = (REAL *)malloc(sizeof(REAL) * (size_t)n * n);
+    REAL *zm = (REAL *)malloc(sizeof(REAL) * (size_t)n);
+    REAL *Gb = (REAL *)malloc(sizeof(REAL) * (size_t)n * n);
+    REAL *zb = (REAL *)malloc(sizeof(REAL) * (size_t)n);
+    REAL *work = (REAL *)malloc(sizeof(REAL) * 3 * (size_t)(n + 1) * (n + 1));
+    for (int b = 0; b < B; ++b) {
+        for (int i = 0; i < n; ++i) y[((size_t)b * T) * n + i] = y0[(size_t)b * n + i];
+        for (int k = 0; k + 1 < T; ++k) {
+            const size_t e = (size_t)b * T + k;
+            for (int i = 0; i < n * n; ++i) Gm[i] = (REAL)0.5 * (G[e * n * n + i] + G[(e + 1) * n * n + i]);
+            for (int i = 0; i < n; ++i) zm[i] = (REAL)0.5 * (z[e * n + i] + z[(e + 1) * n + i]);
+            FN(expm_aug_)(n, Gm, zm, t[k + 1] - t[k], Gb, zb, work);
+            for (int i = 0; i < n; ++i) {
+                REAL acc = zb[i];
+                for (int j = 0; j < n; ++j) acc += Gb[(size_t)i * n + j] * y[e * n + j];
+                y[(e + 1) * n + i] = acc;
+            }
+            if (Gbar_out) memcpy(Gbar_out + ((size_t)b * (T - 1) + k) * n * n, Gb, sizeof(REAL) * (size_t)n * n);
+            if (zbar_out) memcpy(zbar_out + ((size_t)b * (T - 1) + k) * n, zb, sizeof(REAL) * (size_t)n);
+        }
+    }
+    free(Gm); free(zm); free(Gb); free(zb); free(work);
+}
+
+/* ------------------------------------------------------------------------
  * O-6  Multi-head GRU (Sec. 4.4; App. B.4): H independent GRU heads of hidden
  * size n read the same input x[b][t] (m channels); head h has its own
  * parameters and a stride s_h and advances

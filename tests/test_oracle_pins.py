@@ -512,3 +512,68 @@ def test_jvp_is_the_transpose_of_the_gradient():
     rhs = sum(float(np.sum(g["d" + k] * getattr(dp, k))) for k in ("W_i", "W_h", "b_i", "b_h"))
     rhs += float(np.sum(g["dx"] * dx)) + float(np.sum(g["dy0"] * dy0))
     assert abs(float(np.sum(gy * dy)) - rhs) <= 1e-10 * max(1.0, abs(rhs))
+
+
+# ----------------------------------------------------------------------------- ODE instantiation of L_G^{-1} (Sec. 3.3)
+def test_ode_scalar_closed_form():
+    """n = 1, constant g and z: y_{i+1} = e^{-g D} y_i + (1 - e^{-g D}) z / g exactly."""
+    g, zc, T = 0.7, -0.4, 40
+    t = np.cumsum(synth.uniform(1, "o/dt", (T,), 0.01, 0.3, dtype=np.float64))
+    y = oracle.ode_linear(np.full((1, T, 1, 1), g), np.full((1, T, 1), zc), t, np.array([[1.5]]))
+    want = zc / g + (1.5 - zc / g) * np.exp(-g * (t - t[0]))
+    assert np.max(np.abs(y[0, :, 0] - want)) <= 1e-13
+
+
+def test_ode_discretisation_against_a_library_exponential():
+    scipy_linalg = pytest.importorskip("scipy.linalg")
+    B, T, n = 2, 6, 4
+    G = synth.normal(2, "o/G", (B, T, n, n)).astype(np.float64)
+    z = synth.normal(2, "o/z", (B, T, n)).astype(np.float64)
+    t = np.cumsum(synth.uniform(2, "o/dt2", (T,), 0.05, 0.5, dtype=np.float64))
+    y0 = synth.normal(2, "o/y0", (B, n)).astype(np.float64)
+    y, Gb, zb = oracle.ode_linear(G, z, t, y0, want_discrete=True)
+    for b in range(B):
+        for k in range(T - 1):
+            Gm = 0.5 * (G[b, k] + G[b, k + 1]); zm = 0.5 * (z[b, k] + z[b, k + 1]); D = t[k + 1] - t[k]
+            E = scipy_linalg.expm(-Gm * D)
+            assert np.max(np.abs(Gb[b, k] - E)) <= 1e-12 * max(1.0, np.max(np.abs(E)))
+            zbar = np.linalg.solve(Gm, (np.eye(n) - E) @ zm)           # G^{-1}(I - Gbar) z as printed in Sec. 3.3
+            assert np.max(np.abs(zb[b, k] - zbar)) <= 1e-10 * max(1.0, np.max(np.abs(zbar)))
+            assert np.allclose(y[b, k + 1], E @ y[b, k] + zbar, atol=1e-10)
+
+
+def test_ode_constant_coefficients_are_exact_and_singular_G_is_fine():
+    scipy_linalg = pytest.importorskip("scipy.linalg")
+    n, T = 3, 30
+    G0 = synth.normal(3, "o/G0", (n, n)).astype(np.float64) * 0.8 + 1.5 * np.eye(n)
+    z0 = synth.normal(3, "o/z0", (n,)).astype(np.float64)
+    t = np.linspace(0.0, 3.0, T)
+    y0 = np.array([[0.5, -1.0, 2.0]])
+    y = oracle.ode_linear(np.broadcast_to(G0, (1, T, n, n)), np.broadcast_to(z0, (1, T, n)), t, y0)
+    yinf = np.linalg.solve(G0, z0)
+    for k in range(T):
+        want = scipy_linalg.expm(-G0 * t[k]) @ (y0[0] - yinf) + yinf
+        assert np.max(np.abs(y[0, k] - want)) <= 1e-11
+    # G = 0: dy/dt = z(t), mid-point rule = trapezoid
+    zt = np.sin(t)[None, :, None] * np.ones((1, T, n))
+    y = oracle.ode_linear(np.zeros((1, T, n, n)), zt, t, y0)
+    trap = np.concatenate([[0.0], np.cumsum(0.5 * (np.sin(t[1:]) + np.sin(t[:-1])) * np.diff(t))])
+    assert np.max(np.abs(y[0] - (y0[0][None, :] + trap[:, None]))) <= 1e-13
+
+
+def test_ode_midpoint_rule_converges_with_second_order():
+    """App. A.5: local truncation error O(D^3) with mid-point values, hence global O(D^2):
+    halving the step divides the error by about four (reference: a very fine grid)."""
+    n = 2
+    Gf = lambda tt: np.array([[1.0 + 0.5 * np.sin(tt), 0.3 * tt], [-0.4, 0.8 + 0.2 * np.cos(2 * tt)]])
+    zf = lambda tt: np.array([np.cos(tt), 0.5 * tt])
+    y0 = np.array([[1.0, -0.5]])
+
+    def solve(T):
+        t = np.linspace(0.0, 2.0, T)
+        G = np.stack([Gf(v) for v in t])[None]; z = np.stack([zf(v) for v in t])[None]
+        return oracle.ode_linear(G, z, t, y0)[0, -1]
+
+    ref = solve(20001)
+    e1, e2, e3 = (np.max(np.abs(solve(T) - ref)) for T in (21, 41, 81))
+    assert 3.5 <= e1 / e2 <= 4.5 and 3.5 <= e2 / e3 <= 4.5
