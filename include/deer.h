@@ -73,7 +73,7 @@ typedef struct deer_gru_grads {
 } deer_gru_grads;
 
 /* Operations for deer_workspace_bytes(). */
-enum { DEER_OP_EVAL = 0, DEER_OP_SCAN = 1, DEER_OP_VJP = 2, DEER_OP_CLASSIFIER = 3 };
+enum { DEER_OP_EVAL = 0, DEER_OP_SCAN = 1, DEER_OP_VJP = 2, DEER_OP_CLASSIFIER = 3, DEER_OP_ODE = 4 };
 
 /* Flags (bit-or). */
 enum {
@@ -256,6 +256,21 @@ int deer_gru_vjp(const deer_gru_params *params, const float *x, const float *y0,
 int deer_gru_jvp(const deer_gru_params *params, const deer_gru_params *dparams, const float *x, const float *dx,
                  const float *y0, const float *dy0, const float *y, int B, int T, float *dy, void *ws,
                  size_t ws_bytes, int flags, void *stream);
+
+/* The linear operator L_G^{-1} of an ordinary differential equation (Sec. 3.3): solve
+ *     dy/dt + G(t) y = z(t),   y(t_0) = y0
+ * on the time points t_0 < ... < t_{T-1}, with G and z taken constant at their MID-POINT values on every interval
+ * (third-order local truncation error, App. A.5):
+ *     y_{k+1} = Gbar_k y_k + zbar_k,   Gbar_k = exp(-G_k D_k),   zbar_k = G_k^{-1} (I - Gbar_k) z_k,
+ *     G_k = (G(t_k) + G(t_{k+1})) / 2,  z_k likewise,  D_k = t_{k+1} - t_k
+ * -- a batched small matrix exponential per interval (of the augmented matrix [[-G_k D_k, z_k D_k], [0, 0]], which
+ * yields Gbar_k and zbar_k together and needs no inverse), then the same associative scan as the discrete case (Eq. 9).
+ * This is the operator a DEER iteration for an ODE applies once per body (the caller evaluates f and its Jacobian).
+ *   G [B,T,n,n]   z [B,T,n]   t [T] (device, increasing)   y0 [B,n]   y [B,T,n] out, y[b][0] = y0[b]
+ *   n <= 8 (DEER_ERR_UNSUPPORTED_N above);  ws : deer_workspace_bytes(DEER_OP_ODE, B, T, n, 0, 0) bytes
+ * Asynchronous on `stream` (see deer_workspace_status).  Returns DEER_OK or a negative status. */
+int deer_ode_linear_solve(const float *G, const float *z, const float *t, const float *y0, int B, int T, int n,
+                          float *y, void *ws, size_t ws_bytes, int flags, void *stream);
 
 /* One training step of the long-series classifier (App. B.3 shapes: mean
  * over the sequence, then a linear decoder and cross-entropy): two stacked

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libdeer_b200.so")
 DEER_OK, DEER_NOT_CONVERGED, DEER_NONFINITE = 0, 1, 2
 DEER_ERR_INVALID_ARG, DEER_ERR_UNSUPPORTED_N, DEER_ERR_WORKSPACE = -1, -2, -3
 DEER_ERR_CUDA, DEER_ERR_DEVICE_TIMEOUT = -4, -5
-DEER_OP_EVAL, DEER_OP_SCAN, DEER_OP_VJP, DEER_OP_CLASSIFIER = 0, 1, 2, 3
+DEER_OP_EVAL, DEER_OP_SCAN, DEER_OP_VJP, DEER_OP_CLASSIFIER, DEER_OP_ODE = 0, 1, 2, 3, 4
 DEER_FLAG_WARM_START, DEER_FLAG_GENERIC, DEER_FLAG_MATERIALIZE, DEER_FLAG_TCGEN05 = 1, 2, 4, 8
 DEER_FLAG_EXPIRE_WAITS, DEER_FLAG_COEF_ROWS = 16, 32
 
@@ -28,7 +28,8 @@ EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc
            "deer_gru_eval_diag", "deer_gru_eval_host", "deer_gru_vjp",
            "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count",
            "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_cell_jac",
-           "deer_multihead_workspace_bytes", "deer_gru_multihead_eval", "deer_gru_multihead_vjp", "deer_gru_jvp"]
+           "deer_multihead_workspace_bytes", "deer_gru_multihead_eval", "deer_gru_multihead_vjp", "deer_gru_jvp",
+           "deer_ode_linear_solve"]
 
 
 class _Params(ctypes.Structure):
@@ -93,6 +94,8 @@ def lib():
         L.deer_gru_multihead_vjp.restype = ci
         L.deer_gru_multihead_vjp.argtypes = [ctypes.POINTER(_Params), ctypes.POINTER(ci), ci, vp, vp, vp, vp, ci, ci,
                                              ctypes.POINTER(_Grads), vp, vp, vp, sz, ci, vp]
+        L.deer_ode_linear_solve.restype = ci
+        L.deer_ode_linear_solve.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp, vp, sz, ci, vp]
         L.deer_gru_jvp.restype = ci
         L.deer_gru_jvp.argtypes = [ctypes.POINTER(_Params), ctypes.POINTER(_Params), vp, vp, vp, vp, vp, ci, ci, vp, vp, sz, ci, vp]
         L.deer_status_string.restype = ctypes.c_char_p
@@ -441,3 +444,17 @@ def deer_gru_jvp(params, dparams, x, dx, y0, dy0, y, ws=None, flags=0, stream=No
     if rc != DEER_OK:
         raise DeerError(rc)
     return dy
+
+
+def deer_ode_linear_solve(G, z, t, y0, ws=None, flags=0, stream=None):
+    """y = L_G^{-1}[z] for dy/dt + G(t) y = z(t), y(t_0) = y0, mid-point values per interval; see include/deer.h."""
+    B, T, n = z.shape
+    assert tuple(G.shape) == (B, T, n, n) and tuple(t.shape) == (T,) and tuple(y0.shape) == (B, n)
+    y = torch.empty_like(z)
+    if ws is None:
+        ws = alloc_workspace(DEER_OP_ODE, B, T, n, 1, flags, z.device)
+    rc = lib().deer_ode_linear_solve(_ptr(_f32(G)), _ptr(_f32(z)), _ptr(_f32(t)), _ptr(_f32(y0)), B, T, n, _ptr(y), _ptr(ws),
+                                     ws.numel(), flags, _stream(stream))
+    if rc != DEER_OK:
+        raise DeerError(rc)
+    return y

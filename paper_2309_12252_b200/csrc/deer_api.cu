@@ -717,6 +717,25 @@ static ClsWs carve_cls(void *ws, int B, int T, int n, int m, int ncls)
     return w;
 }
 
+struct OdeWs {
+    StatusBlock *st;
+    float *J, *rhs;
+    ScanWs scan;
+    size_t bytes;
+};
+
+static OdeWs carve_ode(void *ws, int B, int T, int n)
+{
+    Carver cv(ws);
+    OdeWs w;
+    w.st = cv.take<StatusBlock>(1);
+    w.J = cv.take<float>((size_t)B * T * n * n);
+    w.rhs = cv.take<float>((size_t)B * T * n);
+    w.scan = carve_scan(cv, B, T, n);
+    w.bytes = cv.off;
+    return w;
+}
+
 // multi-head unit: dense batches of one stride group at a time + the inner evaluation / gradient workspace
 struct MhWs {
     float *xs, *y0s, *ys, *gys, *dxs, *dy0s;
@@ -1098,13 +1117,14 @@ extern "C" {
 size_t deer_workspace_bytes(int op, int B, int T, int n, int m, int flags)
 {
     (void)flags;
-    if (op == DEER_OP_SCAN) m = 1;
+    if (op == DEER_OP_SCAN || op == DEER_OP_ODE) m = 1;
     if (!valid_sizes(B, T, n, m) || !supported(n, m)) return 0;
     switch (op) {
     case DEER_OP_EVAL: return carve_eval(nullptr, B, T, n, m).bytes;
     case DEER_OP_SCAN: return carve_scan_only(nullptr, B, T, n).bytes;
     case DEER_OP_VJP: return carve_vjp(nullptr, B, T, n, m).bytes;
     case DEER_OP_CLASSIFIER: return carve_cls(nullptr, B, T, n, m, 64).bytes;
+    case DEER_OP_ODE: return n <= ODE_MAX_N ? carve_ode(nullptr, B, T, n).bytes : 0;
     default: return 0;
     }
 }
@@ -1282,6 +1302,34 @@ int deer_gru_jvp(const deer_gru_params *p, const deer_gru_params *dp, const floa
     a.st = w.st;
     CellArgs c{p->W_h, p->b_h, w.u, x, p->W_i, p->b_i, m, y, y0, w.J, nullptr, B, T, n, nullptr, 0, 0};
     if ((rc = run_cell(c, st)) != DEER_OK) return rc;
+    return run_scan(a, w.scan, flags, st);
+}
+
+int deer_ode_linear_solve(const float *G, const float *z, const float *t, const float *y0, int B, int T, int n, float *y,
+                          void *ws, size_t ws_bytes, int flags, void *stream)
+{
+    if (!G || !z || !t || !y0 || !y || B <= 0 || T <= 0 || n <= 0) return DEER_ERR_INVALID_ARG;
+    if (n > ODE_MAX_N) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, n, 1)) return DEER_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    OdeWs w = carve_ode(ws, B, T, n);
+    int rc = check_ws(ws, ws_bytes, w.bytes);
+    if (rc != DEER_OK) return rc;
+    DEER_CHECK_CUDA(cudaMemsetAsync(w.st, 0, sizeof(StatusBlock), st), "memset status");
+    {
+        const size_t sm = sizeof(float) * 3 * (size_t)(n + 1) * (n + 1) * ODE_THREADS;
+        if ((rc = opt_in_smem((const void *)ode_discretise_kernel, sm)) != DEER_OK) return rc;
+        size_t blocks = ((size_t)B * T + ODE_THREADS - 1) / ODE_THREADS;
+        const size_t cap = (size_t)num_sms() * 8;
+        if (blocks > cap) blocks = cap;
+        DEER_KERNEL("ode_discretise_kernel", st, ode_discretise_kernel<<<(unsigned)blocks, ODE_THREADS, sm, st>>>(G, z, t, w.J, w.rhs, B, T, n));
+    }
+    ScanArgs a{};
+    a.J = w.J; a.b = w.rhs; a.y0 = y0; a.y = y; a.yold = nullptr;
+    a.B = B; a.T = T; a.n = n; a.reverse = 0;
+    a.L = w.scan.L; a.nch = w.scan.nch;
+    a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
+    a.st = w.st;
     return run_scan(a, w.scan, flags, st);
 }
 

@@ -904,6 +904,84 @@ __global__ void jvp_cell_kernel(JvpArgs a)
     }
 }
 
+// ---------------------------------------------------------------- ODE instantiation of L_G^{-1} (Sec. 3.3)
+// dy/dt + G(t) y = z(t) with G, z constant at their mid-point values on every interval [t_k, t_{k+1}]:
+//     y_{k+1} = Gbar_k y_k + zbar_k,   Gbar_k = exp(-G_k D_k),   zbar_k = G_k^{-1} (I - Gbar_k) z_k,
+// both read off ONE exponential of the augmented (n+1) x (n+1) matrix [[-G_k D_k, z_k D_k], [0, 0]] =
+// [[Gbar_k, zbar_k], [0, 1]] (no inverse: singular G is fine).  One thread per interval: scaling and squaring with a
+// degree-9 Taylor polynomial (norm <= 1/4 after scaling: truncation 3e-13), the three work matrices in shared memory
+// laid out [element][thread] (conflict-free).  Writes the scan's inputs: J[b][k+1] = Gbar_k, rhs[b][k+1] = zbar_k,
+// and J[b][0] = I, rhs[b][0] = 0, so that the forward scan from y0 returns y[b][0] = y0.
+constexpr int ODE_THREADS = 64;
+constexpr int ODE_MAX_N = 8;
+
+__global__ void __launch_bounds__(ODE_THREADS) ode_discretise_kernel(const float *__restrict__ G, const float *__restrict__ z,
+                                                                     const float *__restrict__ t, float *__restrict__ J,
+                                                                     float *__restrict__ rhs, int B, int T, int n)
+{
+    extern __shared__ float sm_ode[];
+    const int m = n + 1, mm = m * m, tid = threadIdx.x;
+    float *A = sm_ode, *P = A + mm * ODE_THREADS, *Q = P + mm * ODE_THREADS;
+#define AT(M_, i_, j_) M_[((i_) * m + (j_)) * ODE_THREADS + tid]
+    const size_t total = (size_t)B * T;
+    for (size_t e = (size_t)blockIdx.x * ODE_THREADS + tid; e < total; e += (size_t)gridDim.x * ODE_THREADS) {
+        const int k = (int)(e % T);                    // this thread writes position k of its sequence
+        float *Jo = J + e * n * n, *ro = rhs + e * n;
+        if (k == 0) {
+            for (int i = 0; i < n; ++i) {
+                ro[i] = 0.0f;
+                for (int j = 0; j < n; ++j) Jo[i * n + j] = (i == j) ? 1.0f : 0.0f;
+            }
+            continue;
+        }
+        const float D = t[k] - t[k - 1];
+        const float *G0 = G + (e - 1) * n * n, *G1 = G + e * n * n, *z0 = z + (e - 1) * n, *z1 = z + e * n;
+        float norm = 0.0f;
+        for (int i = 0; i < m; ++i) {
+            float rs = 0.0f;
+            for (int j = 0; j < m; ++j) {
+                float v = 0.0f;
+                if (i < n) v = (j < n) ? -0.5f * (G0[i * n + j] + G1[i * n + j]) * D : 0.5f * (z0[i] + z1[i]) * D;
+                AT(A, i, j) = v;
+                rs += fabsf(v);
+            }
+            norm = fmaxf(norm, rs);
+        }
+        int s = 0;
+        float scale = 1.0f;
+        while (norm * scale > 0.25f && s < 60) { scale *= 0.5f; ++s; }
+        if (!(norm <= 3.0e38f)) s = 0;                 // non-finite input: let it propagate
+        for (int i = 0; i < m; ++i)
+            for (int j = 0; j < m; ++j) { AT(A, i, j) *= scale; AT(P, i, j) = (i == j) ? 1.0f : 0.0f; }
+        for (int kk = 9; kk >= 1; --kk) {              // Horner: P <- I + (A P) / kk
+            const float inv = 1.0f / (float)kk;
+            for (int i = 0; i < m; ++i)
+                for (int j = 0; j < m; ++j) {
+                    float acc = 0.0f;
+                    for (int l = 0; l < m; ++l) acc = fmaf(AT(A, i, l), AT(P, l, j), acc);
+                    AT(Q, i, j) = fmaf(acc, inv, (i == j) ? 1.0f : 0.0f);
+                }
+            for (int i = 0; i < m; ++i)
+                for (int j = 0; j < m; ++j) AT(P, i, j) = AT(Q, i, j);
+        }
+        for (int q = 0; q < s; ++q) {                  // undo the scaling: square s times
+            for (int i = 0; i < m; ++i)
+                for (int j = 0; j < m; ++j) {
+                    float acc = 0.0f;
+                    for (int l = 0; l < m; ++l) acc = fmaf(AT(P, i, l), AT(P, l, j), acc);
+                    AT(Q, i, j) = acc;
+                }
+            for (int i = 0; i < m; ++i)
+                for (int j = 0; j < m; ++j) AT(P, i, j) = AT(Q, i, j);
+        }
+        for (int i = 0; i < n; ++i) {
+            for (int j = 0; j < n; ++j) Jo[i * n + j] = AT(P, i, j);
+            ro[i] = AT(P, i, n);
+        }
+    }
+#undef AT
+}
+
 // ---------------------------------------------------------------- multi-head GRU: strided views <-> dense batches
 // A head of stride s over [B,T] is s interleaved sequences per batch entry (Sec. 4.4): sequence (b, p) holds the
 // positions t = p + s t', t' = 0 .. T'-1 with T' = ceil(T / s); shorter phases are padded at the END with zeros
