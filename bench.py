@@ -84,7 +84,10 @@ def fused_scan_bytes_per_position(n: int) -> int:
     return 28 * n
 
 
-FUSED_KERNEL_BYTES = {"scan_fused_reduce_kernel": 20, "scan_fused_reduce64_kernel": 20, "scan_fused_apply_kernel": 32}   # x n
+def fused_kernel_bytes(name: str, n: int) -> int:
+    """Algorithmic bytes per position of one launch of the two-launch scan: the reduce kernels read the coefficient
+    rows and the residual (20 n), the apply kernel those, y_old, and writes y (32 n)."""
+    return (20 if "reduce" in name else 32) * n
 
 
 def scan_flops_per_position(n: int) -> int:
@@ -598,7 +601,7 @@ def step_scan_roofline(m, pk):
         per_kernel = {k: prof[k]["total_ms"] / prof[k]["launches"] for k in fused}
         dom = max(per_kernel, key=per_kernel.get)
         reduce_k = dom.startswith("scan_fused_reduce")
-        out = roofline_of_scan(n, positions, per_kernel[dom], pk, FUSED_KERNEL_BYTES[dom] * n,
+        out = roofline_of_scan(n, positions, per_kernel[dom], pk, fused_kernel_bytes(dom, n),
                                NCU_FUSED_TRAFFIC_PER_POSITION.get(dom, {}).get(n), dom, bf16=reduce_k,
                                extra=dict(note="dominant kernel of the step: the chunk reduce of the two-launch scan (J generated from "
                                                "coefficient rows; bf16 m16n8k16 chain products).  bytes = coefficient rows + residual "
