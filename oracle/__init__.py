@@ -106,17 +106,23 @@ def deer(p, x, y0, tol=None, max_iter=100, y_guess=None, dtype=np.float64, form=
          cell="gru", want_history=False):
     """O-3: DEER/Newton iteration.  Returns dict(y, iters, err, trace[, history]).
 
-    ``cell='affine'`` uses f(h, x) = W_h[:n] h + x (W_h's first n rows)."""
+    ``cell='affine'`` uses f(h, x) = W_h[:n] h + x (W_h's first n rows); ``cell='lstm'`` takes
+    synth.LstmParams and states [h; c] of 2k components."""
     sfx, cty = _sfx(dtype)
     if tol is None:
         tol = 1e-7 if np.dtype(dtype) == np.float64 else 1e-4
     x = _c(x, dtype); y0 = _c(y0, dtype)
     B, T, m = x.shape
-    n = p.n
+    n = 2 * p.k if cell == "lstm" else p.n
     if cell == "affine":
         assert m == n
         W_h = _c(p.W_h[:n], dtype); W_i = b_i = b_h = W_h
         cell_id = 1
+    elif cell == "lstm":
+        n = 2 * p.k
+        W_i, W_h, b_i = _c(p.W_i, dtype), _c(p.W_h, dtype), _c(p.b, dtype)
+        b_h = b_i
+        cell_id = 2
     else:
         W_i, W_h, b_i, b_h = _params(p, dtype)
         cell_id = 0
@@ -257,3 +263,27 @@ def ode_linear(G, z, t, y0, dtype=np.float64, want_discrete=False):
     zb = np.empty((B, max(T - 1, 0), n), dtype) if want_discrete else None
     getattr(lib(), f"oracle_ode_linear_{sfx}")(_p(G), _p(z), _p(t), _p(y0), B, T, n, _p(y), _p(Gb), _p(zb))
     return (y, Gb, zb) if want_discrete else y
+
+
+def lstm_seq(p, x, s0, dtype=np.float64):
+    """Sequential LSTM trajectory [B,T,2k] of states [h; c] (p: synth.LstmParams; gate order i, f, g, o)."""
+    sfx, _ = _sfx(dtype)
+    W_i, W_h, b = _c(p.W_i, dtype), _c(p.W_h, dtype), _c(p.b, dtype)
+    x = _c(x, dtype); s0 = _c(s0, dtype)
+    B, T, m = x.shape
+    y = np.empty((B, T, 2 * p.k), dtype)
+    getattr(lib(), f"oracle_lstm_seq_{sfx}")(p.k, m, _p(W_i), _p(W_h), _p(b), _p(x), _p(s0), B, T, _p(y))
+    return y
+
+
+def lstm_cell_jac(p, sprev, x, dtype=np.float64, want_J=True):
+    """LSTM cell value f [N,2k] and state Jacobian J [N,2k,2k] at N given (s_prev, x) rows."""
+    sfx, _ = _sfx(dtype)
+    W_i, W_h, b = _c(p.W_i, dtype), _c(p.W_h, dtype), _c(p.b, dtype)
+    sprev = _c(sprev, dtype).reshape(-1, 2 * p.k); x = _c(x, dtype).reshape(-1, p.m)
+    N = sprev.shape[0]
+    f = np.empty((N, 2 * p.k), dtype)
+    J = np.empty((N, 2 * p.k, 2 * p.k), dtype) if want_J else None
+    getattr(lib(), f"oracle_lstm_cell_jac_{sfx}")(p.k, p.m, _p(W_i), _p(W_h), _p(b), _p(sprev), _p(x), ctypes.c_long(N),
+                                                  _p(f), _p(J))
+    return f, J

@@ -164,11 +164,77 @@ void FN(oracle_linrec_)(const REAL *J, const REAL *b, const REAL *y0, int B, int
 }
 
 /* ------------------------------------------------------------------------
+ * A second cell behind the same interface (Sec. 3.4: any y_i = f(y_{i-1}, x_i, theta)): LSTM with k units,
+ * state s = [h; c] of 2k components, gates in the order (i, f, g, o):
+ *   a = W_i x + b + W_h h   (4k rows),  i = sigma(a_i), f = sigma(a_f), g = tanh(a_g), o = sigma(a_o)
+ *   c' = f * c + i * g,     h' = o * tanh(c'),     f(s, x) = [h'; c']
+ * Closed-form state Jacobian (rows: h' then c'; columns: h then c):
+ *   dc'/dc = diag(f),  dc'/dh = diag(c f(1-f)) W_hf + diag(g i(1-i)) W_hi + diag(i (1-g^2)) W_hg
+ *   dh'/dc = diag(o (1 - tanh^2 c')) dc'/dc,  dh'/dh = diag(tanh(c') o(1-o)) W_ho + diag(o (1 - tanh^2 c')) dc'/dh
+ * Pinned by: a library LSTM, central differences, the DEER fixed point.
+ * ------------------------------------------------------------------------ */
+static void FN(lstm_cell_)(int k, int m, const REAL *W_i, const REAL *W_h, const REAL *b, const REAL *s,
+                           const REAL *x, REAL *out, REAL *J)
+{
+    const REAL *h = s, *c = s + k;
+    for (int u = 0; u < k; ++u) {
+        REAL a[4];
+        for (int q = 0; q < 4; ++q) {
+            REAL acc = b[q * k + u];
+            for (int j = 0; j < m; ++j) acc += W_i[(size_t)(q * k + u) * m + j] * x[j];
+            for (int j = 0; j < k; ++j) acc += W_h[(size_t)(q * k + u) * k + j] * h[j];
+            a[q] = acc;
+        }
+        REAL gi = (REAL)1 / ((REAL)1 + R_EXP(-a[0])), gf = (REAL)1 / ((REAL)1 + R_EXP(-a[1]));
+        REAL gg = R_TANH(a[2]), go = (REAL)1 / ((REAL)1 + R_EXP(-a[3]));
+        REAL cn = gf * c[u] + gi * gg;
+        REAL tc = R_TANH(cn);
+        out[u] = go * tc;
+        out[k + u] = cn;
+        if (J) {
+            const int n = 2 * k;
+            REAL dti = gg * gi * ((REAL)1 - gi), dtf = c[u] * gf * ((REAL)1 - gf), dtg = gi * ((REAL)1 - gg * gg);
+            REAL dho = tc * go * ((REAL)1 - go), dhc = go * ((REAL)1 - tc * tc);
+            for (int j = 0; j < k; ++j) {
+                REAL dcdh = dti * W_h[(size_t)(0 * k + u) * k + j] + dtf * W_h[(size_t)(1 * k + u) * k + j]
+                          + dtg * W_h[(size_t)(2 * k + u) * k + j];
+                J[(size_t)(k + u) * n + j] = dcdh;
+                J[(size_t)u * n + j] = dho * W_h[(size_t)(3 * k + u) * k + j] + dhc * dcdh;
+                J[(size_t)(k + u) * n + k + j] = (j == u) ? gf : (REAL)0;
+                J[(size_t)u * n + k + j] = (j == u) ? dhc * gf : (REAL)0;
+            }
+        }
+    }
+}
+
+void FN(oracle_lstm_seq_)(int k, int m, const REAL *W_i, const REAL *W_h, const REAL *b, const REAL *x,
+                          const REAL *s0, int B, int T, REAL *y)
+{
+#pragma omp parallel for schedule(static)
+    for (int bb = 0; bb < B; ++bb) {
+        const REAL *s = s0 + (size_t)bb * 2 * k;
+        for (int t = 0; t < T; ++t) {
+            REAL *out = y + ((size_t)bb * T + t) * 2 * k;
+            FN(lstm_cell_)(k, m, W_i, W_h, b, s, x + ((size_t)bb * T + t) * m, out, NULL);
+            s = out;
+        }
+    }
+}
+
+void FN(oracle_lstm_cell_jac_)(int k, int m, const REAL *W_i, const REAL *W_h, const REAL *b, const REAL *sprev,
+                               const REAL *x, long N, REAL *f, REAL *J)
+{
+    for (long e = 0; e < N; ++e)
+        FN(lstm_cell_)(k, m, W_i, W_h, b, sprev + e * 2 * k, x + e * m, f + e * 2 * k, J ? J + e * 4 * k * k : NULL);
+}
+
+/* ------------------------------------------------------------------------
  * O-3  DEER / Newton iteration, in the order of the paper's iteration body
  * (Eq. 3 with Eq. 5; App. B.1): shift, Jacobian, f, rhs = f - J y_prev,
  * linear solve, err = max|y_new - y|, k += 1; repeat while err > tol and
  * k < max_iter.  One global err over the whole batch.
- *   cell   : 0 = GRU, 1 = affine test cell (W_h = M, x added)
+ *   cell   : 0 = GRU, 1 = affine test cell (W_h = M, x added), 2 = LSTM (n = 2k state components,
+ *            W_i [4k,m], W_h [4k,k], b_i [4k] the bias; b_h unused)
  *   form   : 0 = paper's form above; 1 = Newton-update (residual) form of
  *            App. A.1: delta = L_J^{-1}[f - y], y += delta
  *   y      : in = initial guess, out = last iterate
@@ -200,6 +266,8 @@ int FN(oracle_deer_)(int cell, int form, int n, int m, const REAL *W_i, const RE
                 if (cell == 0) {
                     FN(gru_cell_)(n, m, W_i, W_h, b_i, b_h, hp, x + e * m, fv, gates);
                     FN(gru_jac_)(n, W_h, hp, gates, Je);
+                } else if (cell == 2) {
+                    FN(lstm_cell_)(n / 2, m, W_i, W_h, b_i, hp, x + e * m, fv, Je);
                 } else {
                     FN(affine_cell_)(n, W_h, hp, x + e * m, fv);
                     for (int i = 0; i < n * n; ++i) Je[i] = W_h[i];

@@ -222,6 +222,23 @@ def config4(seed: int = 0, B: int = 32, T: int = 17984, n: int = 64, m: int = 6,
     return ClassifierWorkload("config4", B, T, [l1, l2], W_o, b_o, x, labels)
 
 
+@dataclass
+class LstmParams:
+    """Packed LSTM parameters, gate order (i, f, g, o) along the leading 4k axis; one bias vector."""
+    k: int
+    m: int
+    W_i: np.ndarray  # [4k, m]
+    W_h: np.ndarray  # [4k, k]
+    b: np.ndarray    # [4k]
+
+
+def lstm_params(k: int, m: int, seed: int = 0, tag: str = "lstm") -> LstmParams:
+    """Every entry ~ U(-1/sqrt(k), 1/sqrt(k)); streams W_i, W_h, b."""
+    a = 1.0 / math.sqrt(k)
+    return LstmParams(k, m, uniform(seed, f"{tag}/W_i", (4 * k, m), -a, a), uniform(seed, f"{tag}/W_h", (4 * k, k), -a, a),
+                      uniform(seed, f"{tag}/b", (4 * k,), -a, a))
+
+
 def multihead_params(H: int, n: int, m: int, seed: int = 0, tag: str = "mh") -> list:
     """H independent parameter sets (one GRU head each), streams ``{tag}/head{h}/...``."""
     return [gru_params(n, m, seed, tag=f"{tag}/head{h}") for h in range(H)]

@@ -577,3 +577,49 @@ def test_ode_midpoint_rule_converges_with_second_order():
     ref = solve(20001)
     e1, e2, e3 = (np.max(np.abs(solve(T) - ref)) for T in (21, 41, 81))
     assert 3.5 <= e1 / e2 <= 4.5 and 3.5 <= e2 / e3 <= 4.5
+
+
+# ----------------------------------------------------------------------------- a second cell: LSTM (Sec. 3.4: any f)
+def test_lstm_matches_a_library_lstm():
+    """The oracle's LSTM against torch.nn.LSTM on CPU with the same weights (gate order i, f, g, o)."""
+    torch = pytest.importorskip("torch")
+    k, m, B, T = 5, 3, 2, 40
+    p = synth.lstm_params(k, m, 3, tag="t/lstm")
+    x = synth.x_gaussian(B, T, m, 3, tag="t/lx").astype(np.float64)
+    s0 = synth.normal(3, "t/ls0", (B, 2 * k)).astype(np.float64) * 0.5
+    net = torch.nn.LSTM(m, k, batch_first=True).double()
+    with torch.no_grad():
+        net.weight_ih_l0.copy_(torch.from_numpy(p.W_i.astype(np.float64)))
+        net.weight_hh_l0.copy_(torch.from_numpy(p.W_h.astype(np.float64)))
+        net.bias_ih_l0.copy_(torch.from_numpy(p.b.astype(np.float64)))
+        net.bias_hh_l0.zero_()
+        h0 = torch.from_numpy(s0[:, :k].copy())[None]; c0 = torch.from_numpy(s0[:, k:].copy())[None]
+        hs = []
+        state = (h0, c0)
+        for t in range(T):                        # step by step to read c as well
+            out, state = net(torch.from_numpy(x[:, t:t + 1]), state)
+            hs.append(np.concatenate([state[0][0].numpy(), state[1][0].numpy()], axis=1))
+    want = np.stack(hs, axis=1)
+    got = oracle.lstm_seq(p, x, s0)
+    assert np.max(np.abs(got - want)) <= 1e-12
+
+
+def test_lstm_jacobian_matches_central_differences_and_deer_returns_the_sequence():
+    k, m, B, T = 3, 2, 2, 60
+    p = synth.lstm_params(k, m, 4, tag="t/lstm2")
+    x = synth.x_gaussian(B, T, m, 4, tag="t/lx2").astype(np.float64)
+    s0 = synth.normal(4, "t/ls02", (B, 2 * k)).astype(np.float64) * 0.5
+    sp = synth.normal(4, "t/lsp", (7, 2 * k)).astype(np.float64)
+    xs = synth.normal(4, "t/lxs", (7, m)).astype(np.float64)
+    f, J = oracle.lstm_cell_jac(p, sp, xs)
+    eps = 1e-6
+    for j in range(2 * k):
+        d = np.zeros(2 * k); d[j] = eps
+        fp, _ = oracle.lstm_cell_jac(p, sp + d, xs, want_J=False)
+        fm, _ = oracle.lstm_cell_jac(p, sp - d, xs, want_J=False)
+        assert np.max(np.abs((fp - fm) / (2 * eps) - J[:, :, j])) <= 1e-8
+    seq = oracle.lstm_seq(p, x, s0)
+    o = oracle.deer(p, x, s0, tol=1e-9, dtype=np.float64, cell="lstm")
+    assert o["iters"] < 30 and np.max(np.abs(o["y"] - seq)) <= 1e-11
+    o32 = oracle.deer(p, x, s0, tol=1e-4, dtype=np.float32, cell="lstm")
+    assert np.max(np.abs(o32["y"] - seq)) <= 5e-6
