@@ -73,7 +73,8 @@ typedef struct deer_gru_grads {
 } deer_gru_grads;
 
 /* Operations for deer_workspace_bytes(). */
-enum { DEER_OP_EVAL = 0, DEER_OP_SCAN = 1, DEER_OP_VJP = 2, DEER_OP_CLASSIFIER = 3, DEER_OP_ODE = 4 };
+enum { DEER_OP_EVAL = 0, DEER_OP_SCAN = 1, DEER_OP_VJP = 2, DEER_OP_CLASSIFIER = 3, DEER_OP_ODE = 4,
+       DEER_OP_LSTM = 5 /* n = the number of LSTM units k */ };
 
 /* Flags (bit-or). */
 enum {
@@ -256,6 +257,27 @@ int deer_gru_vjp(const deer_gru_params *params, const float *x, const float *y0,
 int deer_gru_jvp(const deer_gru_params *params, const deer_gru_params *dparams, const float *x, const float *dx,
                  const float *y0, const float *dy0, const float *y, int B, int T, float *dy, void *ws,
                  size_t ws_bytes, int flags, void *stream);
+
+/* A second cell behind the same iteration (Sec. 3.4: the method applies to any y_i = f(y_{i-1}, x_i, theta); Eq. 3
+ * with Eq. 5): an LSTM with k units, state s = [h; c] of 2k components, gates in the order (i, f, g, o),
+ *     a = W_i x + b + W_h h,  c' = sigmoid(a_f) c + sigmoid(a_i) tanh(a_g),  h' = sigmoid(a_o) tanh(c'),
+ * evaluated over whole sequences exactly as deer_gru_eval evaluates the GRU: cell + closed-form 2k x 2k state
+ * Jacobian + rhs at every position (one kernel), the scan kernels of deer_linrec_scan at state size 2k, the same
+ * device-side loop control.  (Forward evaluation only; no tuned cell kernel.) */
+typedef struct deer_lstm_params {
+    int k;              /* units; the state has 2k components, 2k <= 64 */
+    int m;              /* input size */
+    const float *W_i;   /* [4k, m] */
+    const float *W_h;   /* [4k, k] */
+    const float *b;     /* [4k]    */
+} deer_lstm_params;
+
+/*   x [B,T,m]   s0 [B,2k]   s [B,T,2k] out (the guess on entry if DEER_FLAG_WARM_START)
+ *   iters, err : host out (may be NULL)     ws : deer_workspace_bytes(DEER_OP_LSTM, B, T, k, m, 0) bytes
+ * Synchronises `stream`.  Returns DEER_OK, DEER_NOT_CONVERGED, DEER_NONFINITE or a negative status. */
+int deer_lstm_eval(const deer_lstm_params *params, const float *x, const float *s0, int B, int T, float tol,
+                   int max_iter, float *s, int *iters, float *err, void *ws, size_t ws_bytes, int flags,
+                   void *stream);
 
 /* The linear operator L_G^{-1} of an ordinary differential equation (Sec. 3.3): solve
  *     dy/dt + G(t) y = z(t),   y(t_0) = y0

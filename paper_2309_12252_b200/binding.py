@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libdeer_b200.so")
 DEER_OK, DEER_NOT_CONVERGED, DEER_NONFINITE = 0, 1, 2
 DEER_ERR_INVALID_ARG, DEER_ERR_UNSUPPORTED_N, DEER_ERR_WORKSPACE = -1, -2, -3
 DEER_ERR_CUDA, DEER_ERR_DEVICE_TIMEOUT = -4, -5
-DEER_OP_EVAL, DEER_OP_SCAN, DEER_OP_VJP, DEER_OP_CLASSIFIER, DEER_OP_ODE = 0, 1, 2, 3, 4
+DEER_OP_EVAL, DEER_OP_SCAN, DEER_OP_VJP, DEER_OP_CLASSIFIER, DEER_OP_ODE, DEER_OP_LSTM = 0, 1, 2, 3, 4, 5
 DEER_FLAG_WARM_START, DEER_FLAG_GENERIC, DEER_FLAG_MATERIALIZE, DEER_FLAG_TCGEN05 = 1, 2, 4, 8
 DEER_FLAG_EXPIRE_WAITS, DEER_FLAG_COEF_ROWS = 16, 32
 
@@ -29,12 +29,17 @@ EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc
            "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count",
            "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_cell_jac",
            "deer_multihead_workspace_bytes", "deer_gru_multihead_eval", "deer_gru_multihead_vjp", "deer_gru_jvp",
-           "deer_ode_linear_solve"]
+           "deer_ode_linear_solve", "deer_lstm_eval"]
 
 
 class _Params(ctypes.Structure):
     _fields_ = [("n", ctypes.c_int), ("m", ctypes.c_int), ("W_i", ctypes.c_void_p),
                 ("W_h", ctypes.c_void_p), ("b_i", ctypes.c_void_p), ("b_h", ctypes.c_void_p)]
+
+
+class _LstmParams(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_int), ("m", ctypes.c_int), ("W_i", ctypes.c_void_p), ("W_h", ctypes.c_void_p),
+                ("b", ctypes.c_void_p)]
 
 
 class _Grads(ctypes.Structure):
@@ -94,6 +99,9 @@ def lib():
         L.deer_gru_multihead_vjp.restype = ci
         L.deer_gru_multihead_vjp.argtypes = [ctypes.POINTER(_Params), ctypes.POINTER(ci), ci, vp, vp, vp, vp, ci, ci,
                                              ctypes.POINTER(_Grads), vp, vp, vp, sz, ci, vp]
+        L.deer_lstm_eval.restype = ci
+        L.deer_lstm_eval.argtypes = [ctypes.POINTER(_LstmParams), vp, vp, ci, ci, cf, ci, vp, ctypes.POINTER(ci),
+                                     ctypes.POINTER(cf), vp, sz, ci, vp]
         L.deer_ode_linear_solve.restype = ci
         L.deer_ode_linear_solve.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp, vp, sz, ci, vp]
         L.deer_gru_jvp.restype = ci
@@ -458,3 +466,25 @@ def deer_ode_linear_solve(G, z, t, y0, ws=None, flags=0, stream=None):
     if rc != DEER_OK:
         raise DeerError(rc)
     return y
+
+
+def deer_lstm_eval(p, x, s0, tol=1e-4, max_iter=100, s=None, ws=None, flags=0, stream=None) -> EvalResult:
+    """DEER evaluation of an LSTM (p: synth.LstmParams-like with numpy arrays; moved to the device here);
+    returns EvalResult with y = states [B,T,2k] = [h; c]; see include/deer.h."""
+    B, T, m = x.shape
+    k = p.k
+    mk = lambda a: torch.from_numpy(np.ascontiguousarray(a, np.float32)).to(x.device)
+    W_i, W_h, b = mk(p.W_i), mk(p.W_h), mk(p.b)
+    if s is None:
+        assert not (flags & DEER_FLAG_WARM_START)
+        s = torch.empty((B, T, 2 * k), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = alloc_workspace(DEER_OP_LSTM, B, T, k, m, flags, x.device)
+    ps = _LstmParams(k, m, W_i.data_ptr(), W_h.data_ptr(), b.data_ptr())
+    iters = ctypes.c_int(0)
+    err = ctypes.c_float(0.0)
+    rc = lib().deer_lstm_eval(ctypes.byref(ps), _ptr(_f32(x)), _ptr(_f32(s0)), B, T, float(tol), int(max_iter), _ptr(s),
+                              ctypes.byref(iters), ctypes.byref(err), _ptr(ws), ws.numel(), flags, _stream(stream))
+    if rc < 0:
+        raise DeerError(rc)
+    return EvalResult(s, iters.value, err.value, rc, np.zeros((0,), np.float32))

@@ -736,6 +736,30 @@ static OdeWs carve_ode(void *ws, int B, int T, int n)
     return w;
 }
 
+struct LstmWs {
+    StatusBlock *st;
+    float *trace, *u, *J, *rhs, *yalt;
+    ScanWs scan;
+    size_t bytes;
+};
+
+static LstmWs carve_lstm(void *ws, int B, int T, int k)
+{
+    Carver cv(ws);
+    LstmWs w;
+    const size_t N = (size_t)B * T;
+    const int n = 2 * k;
+    w.st = cv.take<StatusBlock>(1);
+    w.trace = cv.take<float>(ERR_TRACE_CAP);
+    w.u = cv.take<float>(N * 4 * k);
+    w.J = cv.take<float>(N * n * n);
+    w.rhs = cv.take<float>(N * n);
+    w.yalt = cv.take<float>(N * n);
+    w.scan = carve_scan(cv, B, T, n);
+    w.bytes = cv.off;
+    return w;
+}
+
 // multi-head unit: dense batches of one stride group at a time + the inner evaluation / gradient workspace
 struct MhWs {
     float *xs, *y0s, *ys, *gys, *dxs, *dy0s;
@@ -1125,6 +1149,7 @@ size_t deer_workspace_bytes(int op, int B, int T, int n, int m, int flags)
     case DEER_OP_VJP: return carve_vjp(nullptr, B, T, n, m).bytes;
     case DEER_OP_CLASSIFIER: return carve_cls(nullptr, B, T, n, m, 64).bytes;
     case DEER_OP_ODE: return n <= ODE_MAX_N ? carve_ode(nullptr, B, T, n).bytes : 0;
+    case DEER_OP_LSTM: return supported(2 * n, m) ? carve_lstm(nullptr, B, T, n).bytes : 0;
     default: return 0;
     }
 }
@@ -1303,6 +1328,102 @@ int deer_gru_jvp(const deer_gru_params *p, const deer_gru_params *dp, const floa
     CellArgs c{p->W_h, p->b_h, w.u, x, p->W_i, p->b_i, m, y, y0, w.J, nullptr, B, T, n, nullptr, 0, 0};
     if ((rc = run_cell(c, st)) != DEER_OK) return rc;
     return run_scan(a, w.scan, flags, st);
+}
+
+int deer_lstm_eval(const deer_lstm_params *p, const float *x, const float *s0, int B, int T, float tol, int max_iter,
+                   float *s_out, int *iters, float *err, void *ws, size_t ws_bytes, int flags, void *stream)
+{
+    if (!p || !x || !s0 || !s_out || !p->W_i || !p->W_h || !p->b) return DEER_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || p->k <= 0 || p->m <= 0 || max_iter < 1 || tol != tol) return DEER_ERR_INVALID_ARG;
+    if (!supported(2 * p->k, p->m)) return DEER_ERR_UNSUPPORTED_N;
+    if (!valid_sizes(B, T, 2 * p->k, p->m)) return DEER_ERR_INVALID_ARG;
+    const int k = p->k, m = p->m, n = 2 * k;
+    cudaStream_t st = (cudaStream_t)stream;
+    LstmWs w = carve_lstm(ws, B, T, k);
+    int rc = check_ws(ws, ws_bytes, w.bytes);
+    if (rc != DEER_OK) return rc;
+    const size_t N = (size_t)B * T;
+
+    ScanArgs a{};
+    a.J = w.J; a.b = w.rhs; a.y0 = s0; a.y = s_out;
+    a.B = B; a.T = T; a.n = n; a.reverse = 0;
+    a.L = w.scan.L; a.nch = w.scan.nch;
+    a.carA = w.scan.carA; a.carB = w.scan.carB; a.starts = w.scan.starts;
+    a.st = w.st;
+    apply_test_flags(a, flags);
+    const bool single = scan_is_single_pass(a, w.scan, flags) && (((uintptr_t)w.yalt) & 15) == 0;
+    {
+        StatusBlock init;
+        memset(&init, 0, sizeof(init));
+        init.ctl_mode = single ? 1 : 0;
+        init.max_iter = max_iter;
+        init.tol = tol;
+        init.trace = w.trace;
+        EvalBeginArgs e{};
+        if (!(flags & DEER_FLAG_WARM_START)) { e.y = s_out; e.ny = N * n; }
+        if (single) {
+            const OnePassWs &op = w.scan.op;
+            const size_t tiles = (size_t)B * op.nch;
+            e.flags = op.flags; e.nflags = tiles;
+            e.starts = op.starts; e.nstarts = tiles * (size_t)n;
+            if (onepass_ll_aggs(n)) { e.agg_words = (unsigned long long *)op.aggs; e.nagg_words = tiles * (size_t)(n * n + n); }
+        }
+        const size_t words = e.ny / 4 + e.nflags + e.nstarts + e.nagg_words;
+        unsigned blocks = (unsigned)((words + 1023) / 1024);
+        const unsigned cap = 4u * (unsigned)num_sms();
+        if (blocks > cap) blocks = cap;
+        if (blocks < 1u) blocks = 1u;
+        DEER_KERNEL("eval_begin_kernel", st, eval_begin_kernel<<<blocks, 256, 0, st>>>(w.st, init, e));
+    }
+    // u = x W_i^T + b  (4k outputs per position; iteration-invariant)
+    if (sizeof(float) * ((size_t)m * 4 * k + (size_t)PROJ_PP * (m + 1)) <= 200 * 1024 && 4 * k <= 256) {
+        if ((rc = run_affine(x, p->W_i, p->b, w.u, N, m, 4 * k, 0, st)) != DEER_OK) return rc;
+    } else {
+        const size_t total = N * (size_t)(4 * k);
+        DEER_KERNEL("proj_kernel", st, proj_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(x, p->W_i, p->b, w.u, N, m, 4 * k));
+    }
+    const size_t sm = sizeof(float) * 4 * (size_t)k * (k + 1);
+    if ((rc = opt_in_smem((const void *)lstm_cell_kernel, sm)) != DEER_OK) return rc;
+    const int threads = 256 / k * k;
+    size_t cblocks = (N + (size_t)(256 / k) - 1) / (size_t)(256 / k);
+    if (cblocks > (size_t)num_sms() * 16) cblocks = (size_t)num_sms() * 16;
+
+    float *buf[2] = {s_out, w.yalt};
+    int enq = 0, group = 4;
+    StatusBlock hs;
+    for (;;) {
+        int todo = max_iter - enq;
+        if (todo > group) todo = group;
+        for (int j = 0; j < todo; ++j, ++enq) {
+            float *cur = buf[enq & 1], *nxt = buf[(enq + 1) & 1];
+            LstmCellArgs c{p->W_h, w.u, cur, s0, w.J, w.rhs, B, T, k, w.st};
+            DEER_KERNEL("lstm_cell_kernel", st, lstm_cell_kernel<<<(unsigned)cblocks, threads, sm, st>>>(c));
+            a.y = nxt; a.yold = cur;
+            if (single) {
+                if ((rc = scan_onepass(a, w.scan.op, false, flags, st)) != DEER_OK) return rc;
+            } else {
+                if ((rc = scan_generic(a, st)) != DEER_OK) return rc;
+                DEER_KERNEL("newton_control_kernel", st, newton_control_kernel<<<1, 1, 0, st>>>(w.st, tol, max_iter, w.trace));
+            }
+        }
+        DEER_CHECK_CUDA(cudaMemcpyAsync(&hs, w.st, 32, cudaMemcpyDeviceToHost, st), "read status");
+        DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+        if (hs.flags & FLAG_TIMEOUT) return DEER_ERR_DEVICE_TIMEOUT;
+        if (hs.done || enq >= max_iter) break;
+        group = 2;
+    }
+    const int kk = hs.iters;
+    float e;
+    memcpy(&e, &hs.err_last_bits, sizeof(float));
+    if (kk & 1)
+        DEER_CHECK_CUDA(cudaMemcpyAsync(s_out, w.yalt, N * n * sizeof(float), cudaMemcpyDeviceToDevice, st), "copy result");
+    DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
+    int status = DEER_OK;
+    if (!isfinite(e)) status = DEER_NONFINITE;
+    else if (e > tol && !(tol < 0.0f)) status = DEER_NOT_CONVERGED;
+    if (iters) *iters = kk;
+    if (err) *err = e;
+    return status;
 }
 
 int deer_ode_linear_solve(const float *G, const float *z, const float *t, const float *y0, int B, int T, int n, float *y,

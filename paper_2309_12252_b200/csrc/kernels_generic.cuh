@@ -904,6 +904,70 @@ __global__ void jvp_cell_kernel(JvpArgs a)
     }
 }
 
+// ---------------------------------------------------------------- a second cell: LSTM (Sec. 3.4: any f behind the same iteration)
+// State s = [h; c] of 2k components, gates (i, f, g, o):  c' = f c + i g,  h' = o tanh(c'),  f(s, x) = [h'; c'].
+// One thread per (position, unit): the unit's four pre-activations from W_h in shared memory and the projected input
+// u = x W_i^T + b, then its two rows of the closed-form state Jacobian (rows h'_u and c'_u; columns h then c)
+//   dc'/dh = c f(1-f) W_hf + g i(1-i) W_hi + i(1-g^2) W_hg,   dc'/dc = f,
+//   dh'/dh = tanh(c') o(1-o) W_ho + o(1 - tanh^2 c') dc'/dh,  dh'/dc = o(1 - tanh^2 c') f
+// and rhs = f - J s_prev (Eq. 3).
+struct LstmCellArgs {
+    const float *W_h;    // [4k,k]
+    const float *u;      // [B,T,4k]
+    const float *s;      // [B,T,2k] current guess
+    const float *s0;     // [B,2k]
+    float *J;            // [B,T,2k,2k]
+    float *rhs;          // [B,T,2k]
+    int B, T, k;
+    const StatusBlock *st;
+};
+
+__global__ void lstm_cell_kernel(LstmCellArgs a)
+{
+    if (loop_ended(a.st)) return;
+    extern __shared__ float sWl[];
+    const int k = a.k, ld = k + 1, n = 2 * k;
+    for (int i = threadIdx.x; i < 4 * k * k; i += blockDim.x) sWl[(i / k) * ld + (i % k)] = a.W_h[i];
+    __syncthreads();
+    const int epb = blockDim.x / k;
+    const int le = threadIdx.x / k, un = threadIdx.x % k;
+    const size_t N = (size_t)a.B * a.T;
+    for (size_t e = (size_t)blockIdx.x * epb + le; le < epb && e < N; e += (size_t)gridDim.x * epb) {
+        const int t = (int)(e % a.T);
+        const size_t seq = e / a.T;
+        const float *sp = (t == 0) ? a.s0 + seq * n : a.s + (e - 1) * n;
+        const float *ue = a.u + e * 4 * k;
+        float ai = ue[un], af = ue[k + un], ag = ue[2 * k + un], ao = ue[3 * k + un];
+        for (int j = 0; j < k; ++j) {
+            const float h = sp[j];
+            ai = fmaf(sWl[un * ld + j], h, ai);
+            af = fmaf(sWl[(k + un) * ld + j], h, af);
+            ag = fmaf(sWl[(2 * k + un) * ld + j], h, ag);
+            ao = fmaf(sWl[(3 * k + un) * ld + j], h, ao);
+        }
+        const float gi = sigmoidf_acc(ai), gf = sigmoidf_acc(af), gg = tanhf(ag), go = sigmoidf_acc(ao);
+        const float c = sp[k + un];
+        const float cn = fmaf(gf, c, gi * gg);
+        const float tc = tanhf(cn);
+        const float hn = go * tc;
+        const float dti = gg * gi * (1.0f - gi), dtf = c * gf * (1.0f - gf), dtg = gi * (1.0f - gg * gg);
+        const float dho = tc * go * (1.0f - go), dhc = go * (1.0f - tc * tc);
+        float *Jh = a.J + (e * n + un) * n, *Jc = a.J + (e * n + k + un) * n;
+        float jh_s = dhc * gf * c, jc_s = gf * c;                  // (J s_prev) of the two rows: the diagonal c-parts first
+        for (int j = 0; j < k; ++j) {
+            const float dcdh = fmaf(dti, sWl[un * ld + j], fmaf(dtf, sWl[(k + un) * ld + j], dtg * sWl[(2 * k + un) * ld + j]));
+            const float dhdh = fmaf(dho, sWl[(3 * k + un) * ld + j], dhc * dcdh);
+            Jc[j] = dcdh; Jh[j] = dhdh;
+            Jc[k + j] = (j == un) ? gf : 0.0f;
+            Jh[k + j] = (j == un) ? dhc * gf : 0.0f;
+            jc_s = fmaf(dcdh, sp[j], jc_s);
+            jh_s = fmaf(dhdh, sp[j], jh_s);
+        }
+        a.rhs[e * n + un] = hn - jh_s;
+        a.rhs[e * n + k + un] = cn - jc_s;
+    }
+}
+
 // ---------------------------------------------------------------- ODE instantiation of L_G^{-1} (Sec. 3.3)
 // dy/dt + G(t) y = z(t) with G, z constant at their mid-point values on every interval [t_k, t_{k+1}]:
 //     y_{k+1} = Gbar_k y_k + zbar_k,   Gbar_k = exp(-G_k D_k),   zbar_k = G_k^{-1} (I - Gbar_k) z_k,
