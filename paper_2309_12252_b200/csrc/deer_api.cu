@@ -509,16 +509,28 @@ template <int N> static int launch_cell_wide(CellArgs c, cudaStream_t st)
 }
 
 // coefficient rows + rhs only (the scan builds J_t): the hidden contraction on tensor cores
+// the tensor-core coefficient cell can contract the input projection itself (no u buffer, no projection pass)
+static bool coef_cell_projects(int n, int m, const float *x)
+{
+    return n == 32 && m % 8 == 0 && m >= 8 && m <= 64 && (((uintptr_t)x) & 7) == 0;
+}
+
 template <int N> static int launch_cell_coef_mma(CellArgs c, cudaStream_t st)
 {
-    constexpr size_t SM = sizeof(float) * (2 * (size_t)N * (3 * N + 4) + 3 * N);
+    const bool proj = c.u == nullptr;
+    const size_t SM = sizeof(float) * (2 * (size_t)N * (3 * N + 4) + 6 * N + (proj ? 2 * (size_t)c.m * (3 * N + 4) : 0));
     int rc;
-    if ((rc = opt_in_smem((const void *)cell_coef_mma_kernel<N>, SM)) != DEER_OK) return rc;
     const size_t total = (size_t)c.B * c.T;
     const size_t tiles = (total + 127) / 128;
     const size_t cap = (size_t)num_sms() * 4;
     const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
-    DEER_KERNEL_PDL("cell_coef_mma_kernel", false, st, cell_coef_mma_kernel<N>, blocks, 256u, SM, c);
+    if (proj) {
+        if ((rc = opt_in_smem((const void *)cell_coef_mma_kernel<N, true>, SM)) != DEER_OK) return rc;
+        DEER_KERNEL_PDL("cell_coef_mma_kernel", false, st, (cell_coef_mma_kernel<N, true>), blocks, 256u, SM, c);
+    } else {
+        if ((rc = opt_in_smem((const void *)cell_coef_mma_kernel<N, false>, SM)) != DEER_OK) return rc;
+        DEER_KERNEL_PDL("cell_coef_mma_kernel", false, st, (cell_coef_mma_kernel<N, false>), blocks, 256u, SM, c);
+    }
     return DEER_OK;
 }
 
@@ -561,7 +573,7 @@ static int run_cell(CellArgs c, cudaStream_t st, bool generic = false)
         case 8: return launch_cell_small<8>(c, st);
         default: break;
         }
-        if (c.u && (((uintptr_t)c.W_h) & 15) == 0) {
+        if ((c.u || (c.coef_only && c.residual && coef_cell_projects(c.n, c.m, c.x))) && (((uintptr_t)c.W_h) & 15) == 0) {
             switch (c.n) {
             case 16: return launch_cell_wide<16>(c, st);      // (coefficient rows too: measured equal to the tensor-core kernel)
             case 32: return c.coef_only ? launch_cell_coef_mma<32>(c, st) : launch_cell_wide<32>(c, st);
@@ -895,7 +907,8 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
         if (blocks < 1u) blocks = 1u;
         DEER_KERNEL("eval_begin_kernel", st, eval_begin_kernel<<<blocks, 256, 0, st>>>(w.st, init, e));
     }
-    if (!fused_proj && (rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
+    const bool cell_proj = gen_J && coef_cell_projects(n, m, x);     // (n = 32: the coefficient cell contracts x W_i^T itself)
+    if (!fused_proj && !cell_proj && (rc = run_proj(p, x, w.u, N, st)) != DEER_OK) return rc;
 
     // Newton loop (App. B.1): bodies are enqueued ahead of the convergence test -- the decision at
     // the end of each body is taken on the device, and the kernels of bodies past the end return
@@ -908,7 +921,7 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
         if (todo > group) todo = group;
         for (int j = 0; j < todo; ++j, ++enq) {
             float *cur = buf[enq & 1], *nxt = buf[(enq + 1) & 1];
-            CellArgs c{p->W_h, p->b_h, fused_proj ? nullptr : w.u, x, p->W_i, p->b_i, m, cur, y0, w.J, w.rhs, B, T, n, w.st,
+            CellArgs c{p->W_h, p->b_h, (fused_proj || cell_proj) ? nullptr : w.u, x, p->W_i, p->b_i, m, cur, y0, w.J, w.rhs, B, T, n, w.st,
                        gen_J ? 1 : 0, gen_J ? 1 : 0};
             if ((rc = run_cell(c, st)) != DEER_OK) return rc;
             a.y = nxt; a.yold = cur;

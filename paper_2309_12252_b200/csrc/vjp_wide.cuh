@@ -218,21 +218,27 @@ __global__ void __launch_bounds__(256) affine_mma_kernel(const float *__restrict
 
 // ------------------------------------------------------------------ a1-a4 for n in {16, 32} when the scan builds J_t itself
 // The cell as one tensor-core contraction with the gate math as its epilogue: [B*T, n] x [n, 3n]
-// (h_prev times W_h^T; the input half u = x W_i^T + b_i comes from affine_mma_kernel) as m16n8k8 TF32 MMAs
+// (h_prev times W_h^T; the input half u = x W_i^T + b_i comes from affine_mma_kernel, or, PROJ, is contracted here) as m16n8k8 TF32 MMAs
 // issued three times on hi/lo splits, warp = 16 positions x all 3n outputs, weights split once per CTA
 // into padded shared memory.  A lane's accumulator fragments hold, for its two positions and each of
 // its columns i, the three bias-free products (W_hr h)_i, (W_hz h)_i, (W_hn h)_i -- the column blocks of
 // the gates are n/8 apart -- so r, z, c, f, the coefficient row {k_r, a_z, k_n, z}_i and
 // rhs_i = f_i - (J h)_i  (J h = z h + a_z W_hz h + k_n W_hn h + k_r W_hr h) follow in registers.
 // Writes 16 n + 4 n bytes per position; no Jacobian.
-template <int N>
-__global__ void __launch_bounds__(256) cell_coef_mma_kernel(CellArgs a)
+template <int N, bool PROJ = false>
+__global__ void __launch_bounds__(256, 2) cell_coef_mma_kernel(CellArgs a)
 {
     pdl_prologue();
     if (loop_ended(a.st)) return;
     constexpr int NOUT = 3 * N, NB = NOUT / 8, NBG = N / 8, NS = NOUT + 4;      // 2 * NS = 8 (mod 32) words
     extern __shared__ __align__(16) float smw[];
     float *sBh = smw, *sBl = smw + N * NS, *sb = sBl + N * NS;
+    // PROJ: the input projection is part of the same contraction ([B*T, m] x [m, 3n] with W_i^T, also 3 x TF32), so
+    // neither a u buffer nor a projection pass exists: the r and z halves add into the hidden products' accumulators,
+    // the candidate's input part keeps accumulators of its own (c = tanh(u_n + r q) needs the two apart).  Only with
+    // the residual form (rhs = f - y), which does not need the bias-free hidden products.
+    const int m = PROJ ? a.m : 0;
+    float *sIh = sb + 2 * NOUT, *sIl = sIh + m * NS;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     for (int idx = tid; idx < N * NOUT; idx += 256) {
@@ -241,7 +247,15 @@ __global__ void __launch_bounds__(256) cell_coef_mma_kernel(CellArgs a)
         sBh[k * NS + c] = v;
         sBl[k * NS + c] = v - __uint_as_float(__float_as_uint(v) & 0xffffe000u);
     }
-    for (int idx = tid; idx < NOUT; idx += 256) sb[idx] = a.b_h[idx];
+    for (int idx = tid; idx < NOUT; idx += 256) { sb[idx] = a.b_h[idx]; sb[NOUT + idx] = PROJ ? a.b_i[idx] : 0.0f; }
+    if constexpr (PROJ) {
+        for (int idx = tid; idx < m * NOUT; idx += 256) {
+            const int k = idx / NOUT, c = idx % NOUT;
+            const float v = a.W_i[(size_t)c * m + k];
+            sIh[k * NS + c] = v;
+            sIl[k * NS + c] = v - __uint_as_float(__float_as_uint(v) & 0xffffe000u);
+        }
+    }
     __syncthreads();
     const size_t total = (size_t)a.B * a.T;
     const size_t ntiles = (total + 127) / 128;
@@ -261,6 +275,9 @@ __global__ void __launch_bounds__(256) cell_coef_mma_kernel(CellArgs a)
         float acc[NB][4];
 #pragma unroll
         for (int nn = 0; nn < NB; ++nn) { acc[nn][0] = 0.0f; acc[nn][1] = 0.0f; acc[nn][2] = 0.0f; acc[nn][3] = 0.0f; }
+        float accn[PROJ ? NBG : 1][4];                 // input part of the candidate gate (PROJ)
+#pragma unroll
+        for (int nn = 0; nn < (PROJ ? NBG : 1); ++nn) { accn[nn][0] = 0.0f; accn[nn][1] = 0.0f; accn[nn][2] = 0.0f; accn[nn][3] = 0.0f; }
 #pragma unroll
         for (int k0 = 0; k0 < N; k0 += 8) {
             // slots t and t+4 of the K step hold k0+2t and k0+2t+1
@@ -282,18 +299,49 @@ __global__ void __launch_bounds__(256) cell_coef_mma_kernel(CellArgs a)
                 mma_tf32(acc[nn], ah, bh, acc[nn]);
             }
         }
+        if constexpr (PROJ) {
+            const float *xp0 = a.x + rr[0] * m, *xp1 = a.x + rr[1] * m;
+#pragma unroll 2
+            for (int k0 = 0; k0 < m; k0 += 8) {
+                const float2 x0 = vv[0] ? __ldg(reinterpret_cast<const float2 *>(xp0 + k0 + 2 * t)) : make_float2(0.f, 0.f);
+                const float2 x1 = vv[1] ? __ldg(reinterpret_cast<const float2 *>(xp1 + k0 + 2 * t)) : make_float2(0.f, 0.f);
+                unsigned ah[4], al[4];
+                split_tf32(x0.x, ah[0], al[0]);
+                split_tf32(x1.x, ah[1], al[1]);
+                split_tf32(x0.y, ah[2], al[2]);
+                split_tf32(x1.y, ah[3], al[3]);
+                const float *bh0 = sIh + (k0 + 2 * t) * NS + g, *bl0 = sIl + (k0 + 2 * t) * NS + g;
+#pragma unroll
+                for (int nn = 0; nn < NB; ++nn) {
+                    unsigned bh[2], bl[2];
+                    bh[0] = __float_as_uint(bh0[8 * nn]); bh[1] = __float_as_uint(bh0[8 * nn + NS]);
+                    bl[0] = __float_as_uint(bl0[8 * nn]); bl[1] = __float_as_uint(bl0[8 * nn + NS]);
+                    float (&dst)[4] = nn < 2 * NBG ? acc[nn] : accn[nn - 2 * NBG];
+                    mma_tf32(dst, al, bh, dst);
+                    mma_tf32(dst, ah, bl, dst);
+                    mma_tf32(dst, ah, bh, dst);
+                }
+            }
+        }
         // ---- epilogue: gates, coefficient rows, rhs for (position rr[h], columns 8nn+2t, 8nn+2t+1)
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             if (!vv[h]) continue;
             const size_t e = rr[h];
-            const float *ue = a.u + e * NOUT;
+            const float *ue = PROJ ? nullptr : a.u + e * NOUT;
 #pragma unroll
             for (int nn = 0; nn < NBG; ++nn) {
                 const int i0 = 8 * nn + 2 * t;
-                const float2 ur2 = __ldg(reinterpret_cast<const float2 *>(ue + i0));
-                const float2 uz2 = __ldg(reinterpret_cast<const float2 *>(ue + N + i0));
-                const float2 un2 = __ldg(reinterpret_cast<const float2 *>(ue + 2 * N + i0));
+                float2 ur2 = make_float2(0.f, 0.f), uz2 = ur2, un2 = ur2;
+                if constexpr (!PROJ) {
+                    ur2 = __ldg(reinterpret_cast<const float2 *>(ue + i0));
+                    uz2 = __ldg(reinterpret_cast<const float2 *>(ue + N + i0));
+                    un2 = __ldg(reinterpret_cast<const float2 *>(ue + 2 * N + i0));
+                } else {
+                    ur2 = make_float2(sb[NOUT + i0], sb[NOUT + i0 + 1]);
+                    uz2 = make_float2(sb[NOUT + N + i0], sb[NOUT + N + i0 + 1]);
+                    un2 = make_float2(accn[nn][2 * h] + sb[NOUT + 2 * N + i0], accn[nn][2 * h + 1] + sb[NOUT + 2 * N + i0 + 1]);
+                }
                 const float2 h2 = __ldg(reinterpret_cast<const float2 *>(hp[h] + i0));
                 float out_rhs[2];
 #pragma unroll
@@ -317,9 +365,9 @@ __global__ void __launch_bounds__(256) cell_coef_mma_kernel(CellArgs a)
                     jh = fmaf(kn, sq, jh);
                     jh = fmaf(kr, sr, jh);
                     out_rhs[el] = f - jh;
-                    if (a.residual) out_rhs[el] = f;
+                    if (PROJ || a.residual) out_rhs[el] = f;
                 }
-                if (a.rhs && a.residual) {
+                if (a.rhs && (PROJ || a.residual)) {
                     const float2 yc = __ldg(reinterpret_cast<const float2 *>(a.y + e * N + i0));
                     out_rhs[0] -= yc.x; out_rhs[1] -= yc.y;
                 }
