@@ -216,19 +216,33 @@ int deer_gru_eval_diag(const deer_gru_params *params, const float *x, const floa
 
 /* deer_gru_eval with the sequence data in HOST memory (the end-to-end call):
  * copies x_host to x_dev, evaluates into y_dev as deer_gru_eval does, copies
- * the result to y_host; the copies run on `stream` (asynchronously when the
- * host buffers are page-locked) and the result copy is enqueued behind the
- * Newton bodies, so an evaluation that converges within the first group of
- * bodies synchronises the host once.
+ * the result to y_host (asynchronously when the host buffers are page-locked).
+ * A batch of more than deer_gru_eval_host_chunk(B, T) sequences is evaluated
+ * in chunks of that many sequences, each with its own Newton loop (sequences
+ * are independent: the batch is a map over sequences, Sec. 3), so that on
+ * copy streams owned by the library chunk c + 1 arrives and chunk c - 1
+ * leaves while chunk c is evaluated; each chunk's result is exactly what
+ * deer_gru_eval returns for those sequences alone, `iters` and `err` are the
+ * largest over the chunks, the status is the worst.  A batch of one chunk runs
+ * copy, bodies and copy on `stream`, the result copy enqueued behind the first
+ * group of bodies.
  *   x_host [B,T,m] host in     y_host [B,T,n] host out
  *   x_dev  [B,T,m], y_dev [B,T,n] : device staging buffers owned by the caller
  *            (y_dev holds the guess on entry if DEER_FLAG_WARM_START, and the
  *            result on return)
- *   params, y0, ws : device, as for deer_gru_eval
- * Synchronises `stream`.  Returns what deer_gru_eval returns. */
+ *   params, y0, ws : device, as for deer_gru_eval (ws sized for the whole B)
+ * Work already enqueued on `stream` is waited for before the first copy; the
+ * call synchronises `stream` and its copy streams, and calls on one device
+ * are serialised.  Returns what deer_gru_eval returns. */
 int deer_gru_eval_host(const deer_gru_params *params, const float *x_host, const float *y0, int B, int T,
                        float tol, int max_iter, float *y_host, int *iters, float *err, float *x_dev,
                        float *y_dev, void *ws, size_t ws_bytes, int flags, void *stream);
+
+/* Sequences per chunk of deer_gru_eval_host for a batch of B sequences of
+ * length T (B when the batch is not split; at most DEER_HOST_MAX_CHUNKS
+ * chunks).  Host only; 0 for invalid sizes. */
+#define DEER_HOST_MAX_CHUNKS 8
+int deer_gru_eval_host_chunk(int B, int T);
 
 /* Gradient through the evaluated sequence (Eq. 7): given gy = dL/dy at a
  * trajectory y, lambda = gy L_G^{-1} by ONE reverse scan with the Jacobians

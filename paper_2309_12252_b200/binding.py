@@ -27,7 +27,7 @@ NOALLOC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc", "deer_gru_eval",
            "deer_gru_eval_diag", "deer_gru_eval_host", "deer_gru_vjp",
            "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count",
-           "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_cell_jac",
+           "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_eval_host_chunk", "deer_gru_cell_jac",
            "deer_multihead_workspace_bytes", "deer_gru_multihead_eval", "deer_gru_multihead_vjp", "deer_gru_jvp",
            "deer_ode_linear_solve", "deer_lstm_eval"]
 
@@ -87,6 +87,8 @@ def lib():
         L.deer_workspace_status.argtypes = [vp, vp]
         L.deer_noalloc_status.restype = ci
         L.deer_noalloc_status.argtypes = [vp]
+        L.deer_gru_eval_host_chunk.restype = ci
+        L.deer_gru_eval_host_chunk.argtypes = [ci, ci]
         L.deer_scan_geometry.restype = ci
         L.deer_scan_geometry.argtypes = [ci, ci, ci, ci, ctypes.POINTER(ci)]
         L.deer_gru_cell_jac.restype = ci
@@ -212,6 +214,11 @@ def deer_workspace_status(ws, stream=None) -> int:
 
 def deer_noalloc_status(stream=None) -> int:
     return int(lib().deer_noalloc_status(_stream(stream)))
+
+
+def deer_gru_eval_host_chunk(B: int, T: int) -> int:
+    """Sequences per chunk of deer_gru_eval_host (B when the batch is not split)."""
+    return int(lib().deer_gru_eval_host_chunk(int(B), int(T)))
 
 
 def deer_scan_geometry(B: int, T: int, n: int, flags: int = 0) -> dict:

@@ -189,6 +189,10 @@ static long long single_pass_max_batch(int n, bool umma)
     return (long long)(num_sms() / 4) * resolver_cta_capacity(n, umma);
 }
 
+// n = 16, 32: warps of a resolver CTA that resolve.  A resolver CTA's staging area is shared by its resolving warps,
+// and the walk over ONE sequence's tiles is the serial part of a scan: small batches give each sequence a deeper ring.
+static int big_res_warps(int B) { return B <= 4 ? 1 : B <= 8 ? 2 : 4; }
+
 struct PassCfg {
     const char *name;
     int threads;
@@ -272,7 +276,8 @@ static int launch_warpn(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = WarpN<N>;
     static int occ[MAX_DEVICES] = {0};
-    const PassCfg c{"scan_warpn_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 8};
+    w.res_warps = big_res_warps(a.B);
+    const PassCfg c{"scan_warpn_kernel", C::THREADS, C::SMEM, w.res_warps, C::MAX_SEQ_PER_WARP, 8, 8};
     return launch_single_pass(scan_warpn_kernel<N, REV>, occ, c, a, w, prep, st);
 }
 
@@ -282,7 +287,8 @@ static int launch_warpnf(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = WarpNF<N, REV>;
     static int occ[MAX_DEVICES] = {0};
-    const PassCfg c{"scan_warpnf_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 8};
+    w.res_warps = big_res_warps(a.B);
+    const PassCfg c{"scan_warpnf_kernel", C::THREADS, C::SMEM, w.res_warps, C::MAX_SEQ_PER_WARP, 8, 8};
     return launch_single_pass(scan_warpnf_kernel<N, REV>, occ, c, a, w, prep, st);
 }
 
@@ -294,7 +300,8 @@ static int launch_fused_fwd(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
     using C = FusedFwd<N>;
     static int occ[MAX_DEVICES] = {0};
     static int occ_apply[MAX_DEVICES] = {0};
-    const PassCfg c{"scan_fused_reduce_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 8};
+    w.res_warps = big_res_warps(a.B);
+    const PassCfg c{"scan_fused_reduce_kernel", C::THREADS, C::SMEM, w.res_warps, C::MAX_SEQ_PER_WARP, 8, 8};
     int rc = launch_single_pass(scan_fused_reduce_kernel<N>, occ, c, a, w, prep, st);
     if (rc != DEER_OK) return rc;
     int dev = 0;
@@ -851,13 +858,15 @@ static int linrec_scan_impl(const float *J, const float *b, const float *y0, int
     return run_scan(a, w.scan, flags, st);
 }
 
+// copy_st / copy_ev (optional): the stream the copy to y_host is enqueued on, and an event to order it behind `st`.
 // y_host (optional, host memory): the result is also copied there.  The copy is enqueued behind every
 // group of bodies, after a device-side selection of the buffer that holds the current iterate, so that
 // an evaluation that converges within its first group costs one host synchronisation in all.
 static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *y0, int B, int T,
                          float tol, int max_iter, float *y, int *iters, float *err,
                          float *err_trace, void *ws, size_t ws_bytes, int flags, cudaStream_t st,
-                         float *y_host = nullptr, float *err_b = nullptr, unsigned long long *err_argmax = nullptr)
+                         float *y_host = nullptr, float *err_b = nullptr, unsigned long long *err_argmax = nullptr,
+                         cudaStream_t copy_st = nullptr, cudaEvent_t copy_ev = nullptr)
 {
     const int n = p->n, m = p->m;
     EvalWs w = carve_eval(ws, B, T, n, m);
@@ -939,7 +948,12 @@ static int gru_eval_impl(const deer_gru_params *p, const float *x, const float *
             if (blocks > cap) blocks = cap;
             if (blocks < 1u) blocks = 1u;
             DEER_KERNEL("result_select_kernel", st, result_select_kernel<<<blocks, 256, 0, st>>>(w.st, y, w.yalt, N * n));
-            DEER_CHECK_CUDA(cudaMemcpyAsync(y_host, y, N * n * sizeof(float), cudaMemcpyDeviceToHost, st), "copy result to host");
+            if (copy_st) {      // the result leaves on a stream of its own, behind the selection
+                DEER_CHECK_CUDA(cudaEventRecord(copy_ev, st), "record result event");
+                DEER_CHECK_CUDA(cudaStreamWaitEvent(copy_st, copy_ev, 0), "wait result event");
+            }
+            DEER_CHECK_CUDA(cudaMemcpyAsync(y_host, y, N * n * sizeof(float), cudaMemcpyDeviceToHost, copy_st ? copy_st : st),
+                            "copy result to host");
         }
         DEER_CHECK_CUDA(cudaMemcpyAsync(&hs, w.st, 32, cudaMemcpyDeviceToHost, st), "read status");
         DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
@@ -1201,6 +1215,48 @@ int deer_gru_eval_diag(const deer_gru_params *p, const float *x, const float *y0
                          (cudaStream_t)stream, nullptr, err_b, err_argmax);
 }
 
+// Copy streams and events of the pipelined host call, one set per device, made on first use.
+struct HostPipe {
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t ev_in = nullptr, ev_sel = nullptr, ev_out = nullptr, ev_chunk[DEER_HOST_MAX_CHUNKS] = {};
+    bool ready = false;
+    std::mutex mu;
+};
+static HostPipe g_host_pipe[MAX_DEVICES];
+
+static int host_pipe_for_current_device(HostPipe **out)
+{
+    int dev = 0;
+    DEER_CHECK_CUDA(cudaGetDevice(&dev), "cudaGetDevice");
+    if (dev < 0 || dev >= MAX_DEVICES) return DEER_ERR_INVALID_ARG;
+    HostPipe &hp = g_host_pipe[dev];
+    if (!hp.ready) {
+        DEER_CHECK_CUDA(cudaStreamCreateWithFlags(&hp.h2d, cudaStreamNonBlocking), "create copy stream");
+        DEER_CHECK_CUDA(cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking), "create copy stream");
+        DEER_CHECK_CUDA(cudaEventCreateWithFlags(&hp.ev_in, cudaEventDisableTiming), "create event");
+        DEER_CHECK_CUDA(cudaEventCreateWithFlags(&hp.ev_sel, cudaEventDisableTiming), "create event");
+        DEER_CHECK_CUDA(cudaEventCreateWithFlags(&hp.ev_out, cudaEventDisableTiming), "create event");
+        for (int c = 0; c < DEER_HOST_MAX_CHUNKS; ++c)
+            DEER_CHECK_CUDA(cudaEventCreateWithFlags(&hp.ev_chunk[c], cudaEventDisableTiming), "create event");
+        hp.ready = true;
+    }
+    *out = &hp;
+    return DEER_OK;
+}
+
+int deer_gru_eval_host_chunk(int B, int T)
+{
+    if (B <= 0 || T <= 0) return 0;
+    // chunks of about 3 x 2^17 positions: long enough to fill the GPU, short enough that the first copy in and the last
+    // copy out (the two that nothing hides) are a small part of the call
+    const long long N = (long long)B * T;
+    long long nc = (N + 196608) / 393216;
+    if (nc > DEER_HOST_MAX_CHUNKS) nc = DEER_HOST_MAX_CHUNKS;
+    if (nc > B) nc = B;
+    if (nc < 1) nc = 1;
+    return (int)((B + nc - 1) / nc);
+}
+
 int deer_gru_eval_host(const deer_gru_params *p, const float *x_host, const float *y0, int B, int T, float tol,
                        int max_iter, float *y_host, int *iters, float *err, float *x_dev, float *y_dev,
                        void *ws, size_t ws_bytes, int flags, void *stream)
@@ -1211,9 +1267,54 @@ int deer_gru_eval_host(const deer_gru_params *p, const float *x_host, const floa
     if (!supported(p->n, p->m)) return DEER_ERR_UNSUPPORTED_N;
     if (!valid_sizes(B, T, p->n, p->m)) return DEER_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    DEER_CHECK_CUDA(cudaMemcpyAsync(x_dev, x_host, sizeof(float) * (size_t)B * T * p->m, cudaMemcpyHostToDevice, st),
-                    "copy x to the device");
-    return gru_eval_impl(p, x_dev, y0, B, T, tol, max_iter, y_dev, iters, err, nullptr, ws, ws_bytes, flags, st, y_host);
+    const int Bc = deer_gru_eval_host_chunk(B, T);
+    if (Bc >= B) {
+        DEER_CHECK_CUDA(cudaMemcpyAsync(x_dev, x_host, sizeof(float) * (size_t)B * T * p->m, cudaMemcpyHostToDevice, st),
+                        "copy x to the device");
+        return gru_eval_impl(p, x_dev, y0, B, T, tol, max_iter, y_dev, iters, err, nullptr, ws, ws_bytes, flags, st, y_host);
+    }
+    // Sequences are independent (the batch is a map over sequences), so the batch is evaluated in chunks of Bc sequences,
+    // each with its own Newton loop: chunk c + 1 arrives and chunk c - 1 leaves while chunk c is evaluated.
+    {
+        EvalWs wfull = carve_eval(ws, B, T, p->n, p->m);       // (the caller sized ws for the whole batch: checked as documented)
+        int rc = check_ws(ws, ws_bytes, wfull.bytes);
+        if (rc != DEER_OK) return rc;
+    }
+    HostPipe *hp = nullptr;
+    int rc = host_pipe_for_current_device(&hp);
+    if (rc != DEER_OK) return rc;
+    std::lock_guard<std::mutex> lk(hp->mu);
+    const int nc = (B + Bc - 1) / Bc;
+    const size_t xs = (size_t)T * p->m, ys = (size_t)T * p->n;
+    DEER_CHECK_CUDA(cudaEventRecord(hp->ev_in, st), "record entry event");
+    DEER_CHECK_CUDA(cudaStreamWaitEvent(hp->h2d, hp->ev_in, 0), "wait entry event");
+    DEER_CHECK_CUDA(cudaStreamWaitEvent(hp->d2h, hp->ev_in, 0), "wait entry event");
+    for (int c = 0; c < nc; ++c) {
+        const int b0 = c * Bc, bn = (B - b0 < Bc) ? B - b0 : Bc;
+        DEER_CHECK_CUDA(cudaMemcpyAsync(x_dev + b0 * xs, x_host + b0 * xs, sizeof(float) * bn * xs, cudaMemcpyHostToDevice, hp->h2d),
+                        "copy x to the device");
+        DEER_CHECK_CUDA(cudaEventRecord(hp->ev_chunk[c], hp->h2d), "record chunk event");
+    }
+    int status = DEER_OK, k_max = 0;
+    float e_max = 0.0f;
+    for (int c = 0; c < nc; ++c) {
+        const int b0 = c * Bc, bn = (B - b0 < Bc) ? B - b0 : Bc;
+        DEER_CHECK_CUDA(cudaStreamWaitEvent(st, hp->ev_chunk[c], 0), "wait chunk event");
+        int k = 0;
+        float e = 0.0f;
+        rc = gru_eval_impl(p, x_dev + b0 * xs, y0 + (size_t)b0 * p->n, bn, T, tol, max_iter, y_dev + b0 * ys, &k, &e, nullptr,
+                           ws, ws_bytes, flags, st, y_host + b0 * ys, nullptr, nullptr, hp->d2h, hp->ev_sel);
+        if (rc < 0) { cudaStreamSynchronize(hp->h2d); cudaStreamSynchronize(hp->d2h); return rc; }
+        if (k > k_max) k_max = k;
+        if (!(e <= e_max)) e_max = e;                              // (keeps a NaN)
+        if (rc == DEER_NONFINITE || (rc == DEER_NOT_CONVERGED && status == DEER_OK)) status = rc;
+    }
+    DEER_CHECK_CUDA(cudaEventRecord(hp->ev_out, hp->d2h), "record exit event");
+    DEER_CHECK_CUDA(cudaStreamWaitEvent(st, hp->ev_out, 0), "wait exit event");
+    DEER_CHECK_CUDA(cudaStreamSynchronize(hp->d2h), "sync");
+    if (iters) *iters = k_max;
+    if (err) *err = e_max;
+    return status;
 }
 
 int deer_gru_vjp(const deer_gru_params *p, const float *x, const float *y0, const float *y,
@@ -1609,7 +1710,7 @@ int deer_scan_geometry(int B, int T, int n, int flags, int *out)
         switch (n) {
         case 1: case 2: case 4: res_warps = n == 4 ? OnePass<4>::WARPS : OnePass<1>::WARPS; max_seq = OnePass<1>::MAX_SEQ_PER_WARP; break;
         case 8: res_warps = Warp8::RES_WARPS; max_seq = OnePass<8>::MAX_SEQ_PER_WARP; break;
-        case 16: case 32: res_warps = WarpN<16>::RES_WARPS; max_seq = WarpN<16>::MAX_SEQ_PER_WARP; break;
+        case 16: case 32: res_warps = big_res_warps(B); max_seq = WarpN<16>::MAX_SEQ_PER_WARP; break;
         default: res_warps = umma ? Umma64::RES_WARPS : Cta64::RES_WARPS; max_seq = Cta64::MAX_SEQ_PER_WARP; res_cap = umma ? 8 : 16; break;
         }
         out[0] = 1; out[1] = L1; out[2] = sw; out[3] = (T + L1 - 1) / L1;

@@ -56,9 +56,9 @@ template <int N> struct FusedFwd {
     static constexpr bool BF16 = DEER_FUSED_BF16;                      // chain products of the reduce kernel as bf16 m16n8k16
     static constexpr int R_CTAS = 2;                                   // reduce kernel: weights in registers (n = 32: 252 registers)
     static constexpr int STAGES = F::STAGES, STAGE_FLOATS = F::STAGE_FLOATS, WS = F::WS;
-    static constexpr int RES_WARPS = F::RES_WARPS, RES_BATCH = F::RES_BATCH, MAX_SEQ_PER_WARP = F::MAX_SEQ_PER_WARP;
+    static constexpr int RES_WARPS = F::RES_WARPS, MAX_SEQ_PER_WARP = F::MAX_SEQ_PER_WARP;
     static constexpr int SM_WORK = WARPS * AGG + 16 + WARPS * STAGES * STAGE_FLOATS;
-    static constexpr int SM_RES = RES_WARPS * RES_BATCH * AGG;
+    static constexpr int SM_RES = F::SM_RES;
     static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
     // apply kernel
@@ -108,8 +108,8 @@ __global__ void __launch_bounds__(FusedFwd<N>::THREADS, FusedFwd<N>::R_CTAS) sca
     if (tid == 0) s_role = (int)atomicAdd(&a.st->role_counter, 1u);
     __syncthreads();
     if (s_role < w.resolvers) {
-        if (warp < C::RES_WARPS)
-            resolver_big<N>(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        if (warp < w.res_warps)
+            resolver_big<N>(a, w, sm, s_role * w.res_warps + warp, w.resolvers * w.res_warps, lane);
         __syncthreads();
         if (tid == 0) scan_epilogue(a.st, false);
         return;

@@ -76,6 +76,7 @@ struct OnePassWs {
     int nch, Wd, nwin;            // tiles per sequence, tiles per sequence per window, windows
     unsigned total_ids;
     int resolvers;                // CTAs that take the resolver role
+    int res_warps;                // warps of a resolver CTA that resolve (n = 16, 32: chosen per launch)
     int sw;                       // positions per warp chain where the kernel takes it at run time (n = 8)
     float *pfx;                   // [B*nch][chains per tile - 1][n*n+n] prefix aggregates inside each tile (n = 16, 32:
                                   // written by the reduce launch of the two-launch scan of deer_gru_eval)
@@ -123,6 +124,9 @@ __device__ __forceinline__ void cp_async4(void *dst, const void *src)
 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_0() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_2() { asm volatile("cp.async.wait_group 2;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_3() { asm volatile("cp.async.wait_group 3;" ::: "memory"); }
 
 __device__ __forceinline__ void fence_proxy_async()
 {

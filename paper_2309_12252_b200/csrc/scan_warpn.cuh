@@ -39,27 +39,119 @@ template <int N> struct WarpN {
     static constexpr int Q = 2;                        // pending tiles per CTA
     static constexpr int STAGES = (N == 16) ? 4 : 2;   // ring depth per warp (positions)
     static constexpr int STAGE_FLOATS = N * (N + 8) + N;   // matrix with padded rows, then the vector
-    static constexpr int RES_WARPS = 4;                // warps of a resolver CTA that resolve
-    static constexpr int RES_BATCH = (N == 16) ? 8 : 2;   // aggregates a resolver warp stages at once
+    static constexpr int RES_WARPS = 4;                // warps of a resolver CTA that resolve, at most (see big_res_warps)
+    static constexpr int RES_SLOTS = (N == 16) ? 64 : 16; // tile aggregates a resolver CTA stages, shared by its resolving warps
     static constexpr int PEND = (WARPS - 1) * AGG;     // warp aggregates kept for the B item (the last warp's
                                                        // is only needed by the tile combine: it sits in that warp's ring)
     static constexpr int SM_WORK = Q * PEND + WARPS * N + N + 16 + WARPS * STAGES * STAGE_FLOATS;
-    static constexpr int SM_RES = RES_WARPS * RES_BATCH * AGG;
+    static constexpr int SM_RES = RES_SLOTS * AGG;
     static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
     static constexpr int MAX_SEQ_PER_WARP = 8;
     static_assert(N == 16 || N == 32, "one row of the state per resolver lane");
 };
 
-// Resolver for n in {16, 32}: as resolver_loop of scan_onepass.cuh (lane i holds component i of the
-// running state, flags of the next window requested ahead), with a smaller staging batch.
+// Resolver for n in {16, 32}: a warp walks Y <- A Y + beta over the published tile aggregates of its sequences and
+// writes the state entering every tile (lane i holds component i of the running state).  The walk over a sequence's
+// tiles is the serial part of a scan, so the memory round trips are kept off it: a warp that serves ONE sequence
+// (batches up to the resolver warp count) keeps two batches of aggregates in shared memory, fetched by asynchronous
+// copies once their flags have been seen (a ring of tile slots, up to four fetch groups in flight), so that the flags
+// of the tiles after next and the bytes of the next tiles travel while the current ones are walked.  The fewer
+// sequences a launch has, the fewer warps of a resolver CTA resolve and the deeper each one's ring (big_res_warps).  A warp with several sequences visits them in turn (one batch per visit,
+// all of its bytes in flight at once).
+template <int N>
+__device__ __forceinline__ void resolver_big_fetch(float *dst, const float *src, int cnt, int lane)
+{
+    constexpr int AGG = WarpN<N>::AGG;
+    const int total4 = cnt * AGG / 4;
+    for (int i = lane; i < total4; i += 32) cp_async16(dst + 4 * i, src + 4 * i);
+    cp_async_commit();
+}
+
+// the walk over `cnt` staged aggregates; out: the tiles' entering-state words
+template <int N>
+__device__ __forceinline__ float resolver_big_walk(const float *stage, int cnt, unsigned long long *out, float y, int lane)
+{
+    constexpr int AGG = WarpN<N>::AGG, NN = WarpN<N>::NN;
+    for (int q = 0; q < cnt; ++q) {
+        if (lane < N) st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y));
+        const float *ag = stage + q * AGG;
+        float acc0 = (lane < N) ? ag[NN + lane] : 0.0f, acc1 = 0.0f;
+        const float *row = ag + (lane < N ? lane : 0) * N;
+#pragma unroll
+        for (int i = 0; i < N; i += 2) {       // skewed column order: conflict-free row reads
+            const int c0i = (i + lane) & (N - 1), c1i = (i + 1 + lane) & (N - 1);
+            const float y0 = __shfl_sync(0xffffffffu, y, c0i), y1 = __shfl_sync(0xffffffffu, y, c1i);
+            acc0 = fmaf(row[c0i], y0, acc0);
+            acc1 = fmaf(row[c1i], y1, acc1);
+        }
+        y = acc0 + acc1;
+    }
+    return y;
+}
+
 template <int N>
 __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
 {
     if (a.no_resolve) return;     // (wait-expiry test: nobody publishes entering states)
     using C = WarpN<N>;
-    constexpr int AGG = C::AGG, NN = C::NN, BATCH = C::RES_BATCH;
-    float *stage = stage_all + (threadIdx.x >> 5) * BATCH * AGG;
+    constexpr int AGG = C::AGG;
+    const int RING = C::RES_SLOTS / w.res_warps;                           // this warp's tile slots (a power of two)
+    float *stage = stage_all + (threadIdx.x >> 5) * RING * AGG;
+    unsigned spins = 0;
+    if (rw + nrw >= a.B) {
+        // ---- one sequence: a ring of RING tile slots, up to four fetch groups in flight
+        const int s = rw;
+        if (s >= a.B) return;
+        const unsigned *flags = w.flags + (size_t)s * w.nch;
+        const float *aggs = w.aggs + (size_t)s * w.nch * AGG;
+        unsigned long long *starts = w.starts + (size_t)s * w.nch * N;
+        float y = (lane < N && a.y0) ? a.y0[(size_t)s * N + lane] : 0.0f;
+        int c = 0, f = 0;                      // next tile to walk, next tile to fetch (tile i sits in slot i % RING)
+        int ng = 0, ghead = 0, gcnt[4] = {0, 0, 0, 0};
+        unsigned fl = (lane < w.nch) ? ld_acquire_u32(flags + lane) : 0u;      // flags of tiles f + lane
+        while (c < w.nch) {
+            bool progressed = false;
+            if (ng < 4 && f < w.nch && f - c < RING) {
+                const unsigned m = __ballot_sync(0xffffffffu, fl >= 1u);
+                __syncwarp();      // orders every lane's aggregate copies below after the acquiring lanes' flag loads
+                int r = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
+                r = min(r, RING - (f - c));            // (all free slots at once: measured better than smaller groups)
+                if (r > 0) {
+                    // tiles f .. f+r-1 into their slots (the range may wrap around the ring): one group
+                    const int s0 = f & (RING - 1), first = min(r, RING - s0);
+                    const int n4a = first * AGG / 4, n4b = (r - first) * AGG / 4;
+                    const float *src = aggs + (size_t)f * AGG;
+                    for (int i = lane; i < n4a; i += 32) cp_async16(stage + s0 * AGG + 4 * i, src + 4 * i);
+                    for (int i = lane; i < n4b; i += 32) cp_async16(stage + 4 * i, src + first * AGG + 4 * i);
+                    cp_async_commit();
+                    gcnt[(ghead + ng) & 3] = r;
+                    f += r;
+                    ++ng;
+                    progressed = true;
+                }
+                fl = (f + lane < w.nch) ? ld_acquire_u32(flags + f + lane) : 0u;
+            }
+            if (ng > 0) {
+                if (ng == 1) cp_async_wait_0(); else if (ng == 2) cp_async_wait_1(); else if (ng == 3) cp_async_wait_2(); else cp_async_wait_3();
+                __syncwarp();
+                const int cnt = gcnt[ghead];
+                const int s0 = c & (RING - 1), first = min(cnt, RING - s0);
+                y = resolver_big_walk<N>(stage + s0 * AGG, first, starts + (size_t)c * N, y, lane);
+                if (cnt > first) y = resolver_big_walk<N>(stage, cnt - first, starts + (size_t)(c + first) * N, y, lane);
+                __syncwarp();
+                if (lane < cnt) w.flags[(size_t)s * w.nch + c + lane] = 0u;   // consumed: cleared for the next launch
+                c += cnt;
+                ghead = (ghead + 1) & 3;
+                --ng;
+                progressed = true;
+            }
+            if (progressed) spins = 0;
+            else if (!keep_spinning(a, spins)) { cp_async_wait_0(); return; }
+        }
+        return;
+    }
+    // ---- several sequences per warp
     int nseq = 0;
     int pos[C::MAX_SEQ_PER_WARP];
     float yv[C::MAX_SEQ_PER_WARP];
@@ -75,7 +167,6 @@ __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage
         }
     }
     int remaining = nseq;
-    unsigned spins = 0;
     while (remaining > 0) {
         bool progressed = false;
 #pragma unroll
@@ -86,49 +177,19 @@ __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage
             const int s = rw + k * nrw;
             const unsigned *flags = w.flags + (size_t)s * w.nch;
             const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
-            __syncwarp();      // orders every lane's aggregate loads below after the acquiring lanes' flag loads
+            __syncwarp();      // orders every lane's aggregate copies below after the acquiring lanes' flag loads
             int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
-            if (cnt > BATCH) cnt = BATCH;
+            if (cnt > RING) cnt = RING;
             {
                 const int j = c0 + cnt + lane;
                 fnext[k] = (j < w.nch) ? ld_acquire_u32(flags + j) : 0u;
             }
             if (cnt == 0) continue;
             progressed = true;
-            const float4 *src = reinterpret_cast<const float4 *>(w.aggs + ((size_t)s * w.nch + c0) * AGG);
-            float4 *dst = reinterpret_cast<float4 *>(stage);
-            const int total4 = cnt * AGG / 4;
-            for (int i0 = 0; i0 < total4; i0 += 32 * 8) {
-                float4 v[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int i = i0 + u * 32 + lane;
-                    if (i < total4) v[u] = __ldcg(src + i);
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int i = i0 + u * 32 + lane;
-                    if (i < total4) dst[i] = v[u];
-                }
-            }
+            resolver_big_fetch<N>(stage, w.aggs + ((size_t)s * w.nch + c0) * AGG, cnt, lane);
+            cp_async_wait_0();
             __syncwarp();
-            unsigned long long *out = w.starts + ((size_t)s * w.nch + c0) * N;
-            float y = yv[k];
-            for (int q = 0; q < cnt; ++q) {
-                if (lane < N) st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y));
-                const float *ag = stage + q * AGG;
-                float acc0 = (lane < N) ? ag[NN + lane] : 0.0f, acc1 = 0.0f;
-                const float *row = ag + (lane < N ? lane : 0) * N;
-#pragma unroll
-                for (int i = 0; i < N; i += 2) {       // skewed column order: conflict-free row reads
-                    const int c0i = (i + lane) & (N - 1), c1i = (i + 1 + lane) & (N - 1);
-                    const float y0 = __shfl_sync(0xffffffffu, y, c0i), y1 = __shfl_sync(0xffffffffu, y, c1i);
-                    acc0 = fmaf(row[c0i], y0, acc0);
-                    acc1 = fmaf(row[c1i], y1, acc1);
-                }
-                y = acc0 + acc1;
-            }
-            yv[k] = y;
+            yv[k] = resolver_big_walk<N>(stage, cnt, w.starts + ((size_t)s * w.nch + c0) * N, yv[k], lane);
             __syncwarp();
             if (lane < cnt) w.flags[(size_t)s * w.nch + c0 + lane] = 0u;   // consumed: cleared for the next launch
             pos[k] = c0 + cnt;
@@ -388,8 +449,8 @@ __global__ void __launch_bounds__(WarpN<N>::THREADS, WarpN<N>::CTAS_PER_SM) scan
     }
     __syncthreads();
     if (s_role < w.resolvers) {
-        if (warp < C::RES_WARPS)
-            resolver_big<N>(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        if (warp < w.res_warps)
+            resolver_big<N>(a, w, sm, s_role * w.res_warps + warp, w.resolvers * w.res_warps, lane);
         __syncthreads();
         if (tid == 0) scan_epilogue(a.st);
         return;

@@ -33,10 +33,10 @@ template <int N, bool REV = false> struct WarpNF {
     //   reverse: row i holds, for g = 0..7, W[i][8nn+g] for nn = 0..NT-1
     // (128-bit reads at n = 32); the row stride makes the reads of a quarter- or half-warp fall in distinct banks
     static constexpr int WS = N + (N == 32 ? 4 : (REV ? 4 : 0));
-    static constexpr int RES_WARPS = B_::RES_WARPS, RES_BATCH = B_::RES_BATCH;
+    static constexpr int RES_WARPS = B_::RES_WARPS;
     static constexpr int PEND = B_::PEND;
     static constexpr int SM_WORK = Q * PEND + WARPS * N + N + 16 + 3 * N * WS + WARPS * STAGES * STAGE_FLOATS;
-    static constexpr int SM_RES = RES_WARPS * RES_BATCH * AGG;
+    static constexpr int SM_RES = B_::SM_RES;
     static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
     static constexpr int MAX_SEQ_PER_WARP = B_::MAX_SEQ_PER_WARP;
@@ -148,8 +148,8 @@ __global__ void __launch_bounds__(WarpNF<N, REV>::THREADS, WarpNF<N, REV>::CTAS_
     }
     __syncthreads();
     if (s_role < w.resolvers) {
-        if (warp < C::RES_WARPS)
-            resolver_big<N>(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        if (warp < w.res_warps)
+            resolver_big<N>(a, w, sm, s_role * w.res_warps + warp, w.resolvers * w.res_warps, lane);
         __syncthreads();
         if (tid == 0) scan_epilogue(a.st);
         return;

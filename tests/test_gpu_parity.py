@@ -227,6 +227,37 @@ def test_eval_with_host_buffers_matches_device_call(bd, max_iter, tol):
     assert torch.equal(y_host, ref.y.cpu()) and torch.equal(y_dev, ref.y)
 
 
+@pytest.mark.parametrize("n,m,B,T", [(8, 4, 5, 200_000), (32, 32, 3, 300_000)])
+def test_eval_with_host_buffers_in_chunks_of_sequences(bd, n, m, B, T):
+    """A batch that deer_gru_eval_host splits (copies of the neighbouring chunks overlap an evaluation): every chunk
+    holds exactly what deer_gru_eval returns for those sequences alone, iters / err are the largest over the chunks, and
+    the whole agrees with the unsplit device call within the tolerance the iteration is solved to."""
+    Bc = bd.deer_gru_eval_host_chunk(B, T)
+    assert 1 <= Bc < B
+    p_np = synth.gru_params(n, m, 5, tag="hc/gru")
+    x_np = synth.x_gaussian(B, T, m, 5, tag="hc/x")
+    y0_np = (synth.normal(5, "hc/y0", (B, n)) * 0.3).astype(np.float32)
+    p = bd.GruParamsDev.from_numpy(p_np)
+    x_host = torch.from_numpy(np.ascontiguousarray(x_np)).pin_memory()
+    y_host = torch.empty((B, T, n), dtype=torch.float32).pin_memory()
+    x_dev = torch.empty((B, T, m), device="cuda"); y_dev = torch.empty((B, T, n), device="cuda")
+    ws = bd.alloc_workspace(bd.DEER_OP_EVAL, B, T, n, m, 0, x_dev.device)
+    r = bd.deer_gru_eval_host(p, x_host, dev(y0_np), y_host, x_dev, y_dev, ws)
+    assert r.status == 0 and torch.equal(y_dev.cpu(), y_host)
+    its, errs = [], []
+    for b0 in range(0, B, Bc):
+        rc = bd.deer_gru_eval(p, dev(x_np[b0:b0 + Bc]), dev(y0_np[b0:b0 + Bc]))
+        assert torch.equal(rc.y.cpu(), y_host[b0:b0 + Bc])
+        its.append(rc.iters); errs.append(rc.err)
+    assert r.iters == max(its) and r.err == max(errs)
+    whole = bd.deer_gru_eval(p, dev(x_np), dev(y0_np))
+    assert torch.max(torch.abs(whole.y.cpu() - y_host)).item() <= 1e-4
+    # the second call on the same buffers (copy streams and events are reused)
+    y_host.zero_()
+    r2 = bd.deer_gru_eval_host(p, x_host, dev(y0_np), y_host, x_dev, y_dev, ws)
+    assert (r2.iters, r2.err) == (r.iters, r.err) and torch.equal(y_dev.cpu(), y_host)
+
+
 @pytest.mark.parametrize("n,m,B,T,k", [(8, 4, 5, 700, 3), (8, 4, 5, 700, 4), (4, 2, 3, 1000, 2), (32, 32, 2, 300, 3),
                                        (2, 2, 4, 50, 1)])
 def test_eval_diagnostics_of_the_last_body(bd, n, m, B, T, k):
