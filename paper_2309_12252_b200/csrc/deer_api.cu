@@ -5,6 +5,7 @@
 #include <string.h>
 #include <stdlib.h>
 
+#include <algorithm>
 #include <map>
 #include <mutex>
 #include <string>
@@ -1099,10 +1100,10 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
         wa.N = N; wa.slice = (N + P - 1) / P;
         wa.partial = w.partial;
         int outs = n3 * (wa.K + 1);
-        if (n3 % 16 == 0 && n3 <= 192 && wa.K <= 64) {
-            DEER_KERNEL("wgrad_mma_kernel", st, wgrad_mma_kernel<<<P, 32 * (n3 / 16), 0, st>>>(wa));
-        } else if (n3 <= 32 && wa.K <= 8) {
+        if (n3 <= 32 && wa.K <= 8) {
             DEER_KERNEL("wgrad_small_kernel", st, wgrad_small_kernel<<<P, 256, 0, st>>>(wa));
+        } else if (n3 <= 192) {
+            DEER_KERNEL("wgrad_mma_kernel", st, wgrad_mma_kernel<<<dim3(P, (wa.K + 63) / 64), 32 * ((n3 + 15) / 16), 0, st>>>(wa));
         } else {
             int tile = 32;
             while (tile > 1 && sizeof(float) * tile * (size_t)(n3 + wa.K + 1) > 160 * 1024) tile >>= 1;
@@ -1577,6 +1578,15 @@ size_t deer_multihead_workspace_bytes(const int *strides, int H, int B, int T, i
     return carve_mh(nullptr, H, strides, B, T, n, m).bytes;
 }
 
+// Heads in order of stride (stable): heads of equal stride read the same dense batch of x, which is then packed once.
+static std::vector<int> mh_order(const int *strides, int H)
+{
+    std::vector<int> order((size_t)H);
+    for (int h = 0; h < H; ++h) order[(size_t)h] = h;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return strides[a] < strides[b]; });
+    return order;
+}
+
 int deer_gru_multihead_eval(const deer_gru_params *heads, const int *strides, int H, const float *x, const float *y0,
                             int B, int T, float tol, int max_iter, float *y, int *iters, void *ws, size_t ws_bytes,
                             int flags, void *stream)
@@ -1589,18 +1599,21 @@ int deer_gru_multihead_eval(const deer_gru_params *heads, const int *strides, in
     MhWs w = carve_mh(ws, H, strides, B, T, n, m);
     if ((rc = check_ws(ws, ws_bytes, w.bytes)) != DEER_OK) return rc;
     int worst = DEER_OK;
-    int packed_stride = 0;                     // stride whose dense batch of x is in w.xs
-    for (int h = 0; h < H; ++h) {
+    int packed_stride = 1;                     // stride whose dense batch of x is in w.xs (stride 1: x itself)
+    const std::vector<int> order = mh_order(strides, H);
+    for (int oi = 0; oi < H; ++oi) {
+        const int h = order[(size_t)oi];
         const int s = strides[h], Tp = (T + s - 1) / s, Bs = B * s;
         if (s != packed_stride) {              // heads of equal stride read the same dense batch of x
             DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(x, w.xs, B, T, s, Tp, m, m, 0));
             packed_stride = s;
         }
+        const float *xs = s == 1 ? x : w.xs;
         DEER_KERNEL("mh_y0_pack_kernel", st, mh_y0_pack_kernel<<<mh_blocks((size_t)Bs * n), 256, 0, st>>>(y0, w.y0s, B, s, n, H, h));
         if (flags & DEER_FLAG_WARM_START)
             DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(y, w.ys, B, T, s, Tp, n, H * n, h * n));
         int it = 0;
-        rc = gru_eval_impl(&heads[h], w.xs, w.y0s, Bs, Tp, tol, max_iter, w.ys, &it, nullptr, nullptr, w.inner, w.inner_bytes,
+        rc = gru_eval_impl(&heads[h], xs, w.y0s, Bs, Tp, tol, max_iter, w.ys, &it, nullptr, nullptr, w.inner, w.inner_bytes,
                            flags, st);
         if (rc < 0) return rc;
         if (iters) iters[h] = it;
@@ -1625,21 +1638,24 @@ int deer_gru_multihead_vjp(const deer_gru_params *heads, const int *strides, int
     MhWs w = carve_mh(ws, H, strides, B, T, n, m);
     if ((rc = check_ws(ws, ws_bytes, w.bytes)) != DEER_OK) return rc;
     unsigned timeout_flags = 0;
-    int packed_stride = 0;
-    for (int h = 0; h < H; ++h) {
+    int packed_stride = 1;                     // (stride 1: x itself)
+    const std::vector<int> order = mh_order(strides, H);
+    for (int oi = 0; oi < H; ++oi) {
+        const int h = order[(size_t)oi];
         const int s = strides[h], Tp = (T + s - 1) / s, Bs = B * s;
         if (s != packed_stride) {
             DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(x, w.xs, B, T, s, Tp, m, m, 0));
             packed_stride = s;
         }
+        const float *xs = s == 1 ? x : w.xs;
         DEER_KERNEL("mh_y0_pack_kernel", st, mh_y0_pack_kernel<<<mh_blocks((size_t)Bs * n), 256, 0, st>>>(y0, w.y0s, B, s, n, H, h));
         DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(y, w.ys, B, T, s, Tp, n, H * n, h * n));
         DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(gy, w.gys, B, T, s, Tp, n, H * n, h * n));
-        rc = gru_vjp_impl(&heads[h], w.xs, w.y0s, w.ys, w.gys, Bs, Tp, &dheads[h], dx ? w.dxs : nullptr, dy0 ? w.dy0s : nullptr,
+        rc = gru_vjp_impl(&heads[h], xs, w.y0s, w.ys, w.gys, Bs, Tp, &dheads[h], dx ? w.dxs : nullptr, dy0 ? w.dy0s : nullptr,
                           w.inner, w.inner_bytes, flags, st);
         if (rc != DEER_OK) return rc;
-        if (dx)     // the heads' input gradients add up, head by head in a fixed order
-            DEER_KERNEL("mh_unpack_kernel", st, mh_unpack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(w.dxs, dx, B, T, s, Tp, m, m, 0, h > 0));
+        if (dx)     // the heads' input gradients add up, head by head in a fixed order (that of the strides)
+            DEER_KERNEL("mh_unpack_kernel", st, mh_unpack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(w.dxs, dx, B, T, s, Tp, m, m, 0, oi > 0));
         if (dy0)
             DEER_KERNEL("mh_dy0_reduce_kernel", st, mh_dy0_reduce_kernel<<<mh_blocks((size_t)B * n), 256, 0, st>>>(w.dy0s, dy0, B, s, n, H, h));
         // the inner gradient calls share one status block: keep every head's flags

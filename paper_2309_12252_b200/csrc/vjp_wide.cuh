@@ -68,17 +68,19 @@ __global__ void __launch_bounds__(256) vjp_cell_wide_kernel(VjpArgs a)
 
 // Stage 1 of the deterministic parameter-gradient reduction on tensor cores.
 //   out[g][k] = sum_e dG[e][g] V[e][k]   (k == K: bias column, V = 1)
-// CTA p covers slice p of the positions; warp w owns output rows 16w .. 16w+15 and all (K+7)/8
-// column blocks.  The contraction index is the position: per step of 8 positions the A fragment
-// is dG^T (rows = gates), the B fragments are V; both are read straight from global memory as
-// 32-byte row segments.  Products use the 3 x TF32 split (fp32-level accuracy); the bias column is
-// the running sum of the A fragment.  blockDim.x = 32 * n3 / 16, K <= 64.
+// CTA (p, c) covers slice p of the positions and columns 64c .. 64c+63; warp w owns output rows
+// 16w .. 16w+15 (rows past n3 are idle) and the chunk's column blocks.  The contraction index is the
+// position: per step of 8 positions the A fragment is dG^T (rows = gates), the B fragments are V; both
+// are read straight from global memory as 32-byte row segments.  Products use the 3 x TF32 split
+// (fp32-level accuracy); the bias column is the running sum of the A fragment (chunk 0 writes it).
+// blockDim.x = 32 * ceil(n3 / 16), gridDim.y = ceil(K / 64).
 __global__ void __launch_bounds__(384) wgrad_mma_kernel(WgradArgs a)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int n3 = a.n3, K = a.K, K1 = K + 1;
-    const int nb = (K + 7) >> 3;
+    const int kb = 64 * blockIdx.y;
+    const int nb = min(8, (K - kb + 7) >> 3);
     const size_t e0 = (size_t)blockIdx.x * a.slice;
     const size_t e1 = e0 + a.slice < a.N ? e0 + a.slice : a.N;
     float acc[8][4];
@@ -88,6 +90,7 @@ __global__ void __launch_bounds__(384) wgrad_mma_kernel(WgradArgs a)
         for (int i = 0; i < 4; ++i) acc[nn][i] = 0.0f;
     float bs0 = 0.0f, bs1 = 0.0f;
     const int row = 16 * warp + g;
+    const bool rv0 = row < n3, rv1 = row + 8 < n3;
     auto vrow = [&](size_t e) -> const float * {
         if (!a.shifted) return a.V + e * K;
         size_t seq;
@@ -98,15 +101,15 @@ __global__ void __launch_bounds__(384) wgrad_mma_kernel(WgradArgs a)
         const size_t p0 = e + t, p1 = e + t + 4;
         const bool v0 = p0 < e1, v1 = p1 < e1;
         float av[4];
-        av[0] = v0 ? __ldg(a.dG + p0 * n3 + row) : 0.0f;
-        av[1] = v0 ? __ldg(a.dG + p0 * n3 + row + 8) : 0.0f;
-        av[2] = v1 ? __ldg(a.dG + p1 * n3 + row) : 0.0f;
-        av[3] = v1 ? __ldg(a.dG + p1 * n3 + row + 8) : 0.0f;
+        av[0] = (v0 && rv0) ? __ldg(a.dG + p0 * n3 + row) : 0.0f;
+        av[1] = (v0 && rv1) ? __ldg(a.dG + p0 * n3 + row + 8) : 0.0f;
+        av[2] = (v1 && rv0) ? __ldg(a.dG + p1 * n3 + row) : 0.0f;
+        av[3] = (v1 && rv1) ? __ldg(a.dG + p1 * n3 + row + 8) : 0.0f;
         const float *r0 = v0 ? vrow(p0) : a.V, *r1 = v1 ? vrow(p1) : a.V;
         float bv[8][2];
 #pragma unroll
         for (int nn = 0; nn < 8; ++nn) {
-            const int col = 8 * nn + g;
+            const int col = kb + 8 * nn + g;
             const bool cv = nn < nb && col < K;
             bv[nn][0] = (cv && v0) ? __ldg(r0 + col) : 0.0f;
             bv[nn][1] = (cv && v1) ? __ldg(r1 + col) : 0.0f;
@@ -132,16 +135,26 @@ __global__ void __launch_bounds__(384) wgrad_mma_kernel(WgradArgs a)
 #pragma unroll
     for (int nn = 0; nn < 8; ++nn) {
         if (nn < nb) {
-            const int col = 8 * nn + 2 * t;
-            if (col < K) { out[row * K1 + col] = acc[nn][0]; out[(row + 8) * K1 + col] = acc[nn][2]; }
-            if (col + 1 < K) { out[row * K1 + col + 1] = acc[nn][1]; out[(row + 8) * K1 + col + 1] = acc[nn][3]; }
+            const int col = kb + 8 * nn + 2 * t;
+            if (col < K) {
+                if (rv0) out[row * K1 + col] = acc[nn][0];
+                if (rv1) out[(row + 8) * K1 + col] = acc[nn][2];
+            }
+            if (col + 1 < K) {
+                if (rv0) out[row * K1 + col + 1] = acc[nn][1];
+                if (rv1) out[(row + 8) * K1 + col + 1] = acc[nn][3];
+            }
         }
     }
+    if (blockIdx.y != 0) return;
     bs0 += __shfl_xor_sync(0xffffffffu, bs0, 1);
     bs0 += __shfl_xor_sync(0xffffffffu, bs0, 2);
     bs1 += __shfl_xor_sync(0xffffffffu, bs1, 1);
     bs1 += __shfl_xor_sync(0xffffffffu, bs1, 2);
-    if (t == 0) { out[row * K1 + K] = bs0; out[(row + 8) * K1 + K] = bs1; }
+    if (t == 0) {
+        if (rv0) out[row * K1 + K] = bs0;
+        if (rv1) out[(row + 8) * K1 + K] = bs1;
+    }
 }
 
 // ------------------------------------------------------------------ a0 / a8: dense affine map on tensor cores
