@@ -44,6 +44,26 @@ __device__ __forceinline__ unsigned pack_bf16(float lo, float hi)
     return *reinterpret_cast<const unsigned *>(&v);
 }
 
+// packed bf16 arithmetic on register pairs (two values per 32-bit register, one instruction)
+__device__ __forceinline__ unsigned hfma2_bf16(unsigned a, unsigned b, unsigned c)
+{
+    unsigned d;
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned hmul2_bf16(unsigned a, unsigned b)
+{
+    unsigned d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ unsigned hadd2_bf16(unsigned a, unsigned b)
+{
+    unsigned d;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
 #ifndef DEER_FUSED_BF16
 #define DEER_FUSED_BF16 1
 #endif
@@ -54,7 +74,7 @@ template <int N> struct FusedFwd {
     static constexpr int WARPS = F::WARPS, THREADS = F::THREADS;       // chains per tile of the reduce kernel
     static constexpr int CTAS_PER_SM = F::CTAS_PER_SM;                 // (sets the tile length: tiles per resident CTA)
     static constexpr bool BF16 = DEER_FUSED_BF16;                      // chain products of the reduce kernel as bf16 m16n8k16
-    static constexpr int R_CTAS = 2;                                   // reduce kernel: weights in registers (n = 32: 252 registers)
+    static constexpr int R_CTAS = 3;                                   // reduce kernel: CTAs per SM (n = 32: 168 registers, the weights as bf16 pairs)
     static constexpr int STAGES = F::STAGES, STAGE_FLOATS = F::STAGE_FLOATS, WS = F::WS;
     static constexpr int RES_WARPS = F::RES_WARPS, MAX_SEQ_PER_WARP = F::MAX_SEQ_PER_WARP;
     static constexpr int SM_WORK = WARPS * AGG + 16 + WARPS * STAGES * STAGE_FLOATS;
@@ -93,15 +113,23 @@ __global__ void __launch_bounds__(FusedFwd<N>::THREADS, FusedFwd<N>::R_CTAS) sca
     // This lane's share of W_h stays in registers for the whole launch: the pieces it multiplies into its operand
     // pieces of J_t, {W[8nn+g][8kk+2t], W[8nn+g][8kk+2t+1]} per gate (3 n^2 / 32 values).  Read from shared memory
     // instead (12 KB per warp and position at n = 32) they kept the shared-memory pipe 69 % busy and bound the kernel.
-    float2 wR[NT][NT], wZ[NT][NT], wN[NT][NT];
+    // (bf16 products: the pieces are kept as bf16 pairs, half the registers)
+    float2 wR[C::BF16 ? 1 : NT][C::BF16 ? 1 : NT], wZ[C::BF16 ? 1 : NT][C::BF16 ? 1 : NT], wN[C::BF16 ? 1 : NT][C::BF16 ? 1 : NT];
+    unsigned wRb[NT][NT], wZb[NT][NT], wNb[NT][NT];
 #pragma unroll
     for (int nn = 0; nn < NT; ++nn)
 #pragma unroll
         for (int kk = 0; kk < NT; ++kk) {
             const float *wp = a.Wh + (size_t)(8 * nn + g) * N + 8 * kk + 2 * t;
-            wR[nn][kk] = __ldg(reinterpret_cast<const float2 *>(wp));
-            wZ[nn][kk] = __ldg(reinterpret_cast<const float2 *>(wp + NN));
-            wN[nn][kk] = __ldg(reinterpret_cast<const float2 *>(wp + 2 * NN));
+            const float2 r2 = __ldg(reinterpret_cast<const float2 *>(wp));
+            const float2 z2 = __ldg(reinterpret_cast<const float2 *>(wp + NN));
+            const float2 n2 = __ldg(reinterpret_cast<const float2 *>(wp + 2 * NN));
+            if constexpr (C::BF16) {
+                wRb[nn][kk] = pack_bf16(r2.x, r2.y); wZb[nn][kk] = pack_bf16(z2.x, z2.y); wNb[nn][kk] = pack_bf16(n2.x, n2.y);
+            } else {
+                wR[nn][kk] = r2; wZ[nn][kk] = z2; wN[nn][kk] = n2;
+                wRb[nn][kk] = 0u; wZb[nn][kk] = 0u; wNb[nn][kk] = 0u;
+            }
         }
     const bool d0 = g == 2 * t, d1 = g == 2 * t + 1;      // this lane's pieces touch the diagonal where nn == kk
 
@@ -169,8 +197,9 @@ __global__ void __launch_bounds__(FusedFwd<N>::THREADS, FusedFwd<N>::R_CTAS) sca
         float acc[MT][NT][4];
         identity_fragments<N>(acc, g, t);
         float yv[NT][2];
+        float bacc[NT][2];                 // (bf16 form) beta, columns 8nn+2t, 8nn+2t+1, live in the lanes g == 0
 #pragma unroll
-        for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = 0.0f; yv[kk][1] = 0.0f; }
+        for (int kk = 0; kk < NT; ++kk) { yv[kk][0] = 0.0f; yv[kk][1] = 0.0f; bacc[kk][0] = 0.0f; bacc[kk][1] = 0.0f; }
 #pragma unroll
         for (int q = 0; q < S - 1; ++q) issue(q);
 #pragma unroll 1
@@ -183,6 +212,7 @@ __global__ void __launch_bounds__(FusedFwd<N>::THREADS, FusedFwd<N>::R_CTAS) sca
             // from the coefficient rows and the weights in registers, multiply them into the new X (MT * NT
             // independent accumulators in flight) and into beta's partial sums
             float nacc[MT][NT][4];
+            float nb[NT][4];               // (bf16 form) the beta row tile's new accumulators
             float4 cf[NT];
             float2 p2[NT];
 #pragma unroll
@@ -193,36 +223,67 @@ __global__ void __launch_bounds__(FusedFwd<N>::THREADS, FusedFwd<N>::R_CTAS) sca
                 for (int mm = 0; mm < MT; ++mm) { nacc[mm][nn][0] = 0.0f; nacc[mm][nn][1] = 0.0f; nacc[mm][nn][2] = 0.0f; nacc[mm][nn][3] = 0.0f; }
             }
             if constexpr (C::BF16) {
-                // operands rounded to nearest bf16, m16n8k16: half the MMAs and accumulator chains half as long
-                // (the chain's pace is set by the MMA latency, not by its issue rate).  The accumulator tiles
-                // 2j, 2j+1 of X are the A operand of contraction block j as they stand.
+                // bf16 m16n8k16 products (half the MMAs of the TF32 form and chains half as long).  J_t is BUILT in packed
+                // bf16 arithmetic, three instructions per pair of entries, and the result is the B fragment as it stands;
+                // beta rides along as row 32 of X (a third row tile whose only live row is held by the lanes g == 0), so
+                // its update is one more MMA per block instead of an fp32 mat-vec with its shuffles.  The accumulator
+                // tiles 2j, 2j+1 of X are the A operand of contraction block j as they stand.
+                unsigned cr[NT], cz[NT], cn[NT], zd[NT];
 #pragma unroll
-                for (int j = 0; j < NT / 2; ++j) {
-                    unsigned af[MT][4];
+                for (int nn = 0; nn < NT; ++nn) {
+                    cr[nn] = pack_bf16(cf[nn].x, cf[nn].x);
+                    cz[nn] = pack_bf16(cf[nn].y, cf[nn].y);
+                    cn[nn] = pack_bf16(cf[nn].z, cf[nn].z);
+                    zd[nn] = pack_bf16(d0 ? cf[nn].w : 0.0f, d1 ? cf[nn].w : 0.0f);
+                    nb[nn][0] = 0.0f; nb[nn][1] = 0.0f; nb[nn][2] = 0.0f; nb[nn][3] = 0.0f;
+                }
+                // all B fragments first: they do not depend on X, so their (three-deep) chains run while the previous
+                // position's MMAs drain; written level by level so that independent instructions follow one another
+                unsigned bf[NT / 2][NT][2];
 #pragma unroll
-                    for (int mm = 0; mm < MT; ++mm) {
-                        af[mm][0] = pack_bf16(acc[mm][2 * j][0], acc[mm][2 * j][1]);
-                        af[mm][1] = pack_bf16(acc[mm][2 * j][2], acc[mm][2 * j][3]);
-                        af[mm][2] = pack_bf16(acc[mm][2 * j + 1][0], acc[mm][2 * j + 1][1]);
-                        af[mm][3] = pack_bf16(acc[mm][2 * j + 1][2], acc[mm][2 * j + 1][3]);
-                    }
+                for (int j = 0; j < NT / 2; ++j)
 #pragma unroll
-                    for (int nn = 0; nn < NT; ++nn) {
-                        const float2 cx = make_float2(cf[nn].x, cf[nn].x), cy = make_float2(cf[nn].y, cf[nn].y),
-                                     cz = make_float2(cf[nn].z, cf[nn].z);
-                        float2 v[2];
+                    for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) bf[j][nn][h] = hmul2_bf16(cn[nn], wNb[nn][2 * j + h]);
+#pragma unroll
+                for (int j = 0; j < NT / 2; ++j)
+#pragma unroll
+                    for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) bf[j][nn][h] = hfma2_bf16(cz[nn], wZb[nn][2 * j + h], bf[j][nn][h]);
+#pragma unroll
+                for (int j = 0; j < NT / 2; ++j)
+#pragma unroll
+                    for (int nn = 0; nn < NT; ++nn)
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const int kk = 2 * j + h;
-                            v[h] = ffma2(cx, wR[nn][kk], ffma2(cy, wZ[nn][kk], fmul2(cz, wN[nn][kk])));
-                            if (nn == kk) { v[h].x += d0 ? cf[nn].w : 0.0f; v[h].y += d1 ? cf[nn].w : 0.0f; }
-                            p2[nn] = ffma2(v[h], make_float2(yv[kk][0], yv[kk][1]), p2[nn]);
+                            bf[j][nn][h] = hfma2_bf16(cr[nn], wRb[nn][2 * j + h], bf[j][nn][h]);
+                            if (nn == 2 * j + h) bf[j][nn][h] = hadd2_bf16(bf[j][nn][h], zd[nn]);
                         }
-                        const unsigned bf[2] = {pack_bf16(v[0].x, v[0].y), pack_bf16(v[1].x, v[1].y)};
+                unsigned af[NT / 2][MT + 1][4];
 #pragma unroll
-                        for (int mm = 0; mm < MT; ++mm) mma_bf16(nacc[mm][nn], af[mm], bf, nacc[mm][nn]);
+                for (int j = 0; j < NT / 2; ++j) {
+#pragma unroll
+                    for (int mm = 0; mm < MT; ++mm) {
+                        af[j][mm][0] = pack_bf16(acc[mm][2 * j][0], acc[mm][2 * j][1]);
+                        af[j][mm][1] = pack_bf16(acc[mm][2 * j][2], acc[mm][2 * j][3]);
+                        af[j][mm][2] = pack_bf16(acc[mm][2 * j + 1][0], acc[mm][2 * j + 1][1]);
+                        af[j][mm][3] = pack_bf16(acc[mm][2 * j + 1][2], acc[mm][2 * j + 1][3]);
                     }
+                    af[j][MT][0] = pack_bf16(bacc[2 * j][0], bacc[2 * j][1]);
+                    af[j][MT][1] = 0u;
+                    af[j][MT][2] = pack_bf16(bacc[2 * j + 1][0], bacc[2 * j + 1][1]);
+                    af[j][MT][3] = 0u;
                 }
+#pragma unroll
+                for (int j = 0; j < NT / 2; ++j)
+#pragma unroll
+                    for (int nn = 0; nn < NT; ++nn) {
+#pragma unroll
+                        for (int mm = 0; mm < MT; ++mm) mma_bf16(nacc[mm][nn], af[j][mm], bf[j][nn], nacc[mm][nn]);
+                        mma_bf16(nb[nn], af[j][MT], bf[j][nn], nb[nn]);
+                    }
             } else {
 #pragma unroll
             for (int kk = 0; kk < NT; ++kk) {
@@ -246,28 +307,47 @@ __global__ void __launch_bounds__(FusedFwd<N>::THREADS, FusedFwd<N>::R_CTAS) sca
                 }
             }
             }
-            float ynew[NT];
-#pragma unroll
-            for (int nn = 0; nn < NT; ++nn) {
-                float part = p2[nn].x + p2[nn].y;
-                part += __shfl_xor_sync(0xffffffffu, part, 1);
-                part += __shfl_xor_sync(0xffffffffu, part, 2);
-                ynew[nn] = part + Ms[4 * N + 8 * nn + g];
-            }
 #pragma unroll
             for (int mm = 0; mm < MT; ++mm)
 #pragma unroll
                 for (int nn = 0; nn < NT; ++nn)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) acc[mm][nn][i] = nacc[mm][nn][i];
+            if constexpr (C::BF16) {
+                // beta <- beta J_t^T + r_t: the live row of the tile, columns 8nn+2t, 8nn+2t+1 in the lanes g == 0
 #pragma unroll
-            for (int kk = 0; kk < NT; ++kk) {
-                yv[kk][0] = __shfl_sync(0xffffffffu, ynew[kk], 4 * (2 * t));
-                yv[kk][1] = __shfl_sync(0xffffffffu, ynew[kk], 4 * (2 * t + 1));
+                for (int nn = 0; nn < NT; ++nn) {
+                    float2 r2 = make_float2(0.0f, 0.0f);
+                    if (g == 0) r2 = *reinterpret_cast<const float2 *>(Ms + 4 * N + 8 * nn + 2 * t);
+                    bacc[nn][0] = nb[nn][0] + r2.x;
+                    bacc[nn][1] = nb[nn][1] + r2.y;
+                }
+            } else {
+                float ynew[NT];
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn) {
+                    float part = p2[nn].x + p2[nn].y;
+                    part += __shfl_xor_sync(0xffffffffu, part, 1);
+                    part += __shfl_xor_sync(0xffffffffu, part, 2);
+                    ynew[nn] = part + Ms[4 * N + 8 * nn + g];
+                }
+#pragma unroll
+                for (int kk = 0; kk < NT; ++kk) {
+                    yv[kk][0] = __shfl_sync(0xffffffffu, ynew[kk], 4 * (2 * t));
+                    yv[kk][1] = __shfl_sync(0xffffffffu, ynew[kk], 4 * (2 * t + 1));
+                }
             }
         }
         cp_async_wait_n<0>();
         __syncwarp();
+        if constexpr (C::BF16) {
+            // beta from the lanes g == 0 to every lane's (2t, 2t+1) pairs, as store_aggregate takes it
+#pragma unroll
+            for (int kk = 0; kk < NT; ++kk) {
+                yv[kk][0] = __shfl_sync(0xffffffffu, bacc[kk][0], t);
+                yv[kk][1] = __shfl_sync(0xffffffffu, bacc[kk][1], t);
+            }
+        }
         store_aggregate<N>(wagg + warp * AGG, acc, yv, g, t);
         __syncthreads();
         if (warp == 0) {
