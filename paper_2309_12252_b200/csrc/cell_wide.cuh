@@ -140,9 +140,9 @@ __global__ void __launch_bounds__(256, (N <= 32) ? 4 : 0) cell_wide_kernel(CellA
                 if (p < np) {
                     const size_t e = e0 + p;
                     const float qn = gq[q] + bN;                 // q = W_hn h + b_hn
-                    const float r = sigmoidf_acc(ur[q] + (gr[q] + bR));
-                    const float z = sigmoidf_acc(uz[q] + (gz[q] + bZ));
-                    const float c = tanhf(un[q] + r * qn);
+                    const float r = sigmoidf_gate(ur[q] + (gr[q] + bR));
+                    const float z = sigmoidf_gate(uz[q] + (gz[q] + bZ));
+                    const float c = tanhf_gate(un[q] + r * qn);
                     const float hi = hrow[q * C::HS + gi];
                     const float f = (1.0f - z) * c + z * hi;
                     const float az = (hi - c) * z * (1.0f - z);

@@ -50,9 +50,9 @@ __global__ void __launch_bounds__(256) vjp_cell_wide_kernel(VjpArgs a)
             if (p < np) {
                 const size_t e = e0 + p;
                 const float qn = gq[q] + bN;
-                const float r = sigmoidf_acc(ur[q] + (gr[q] + bR));
-                const float z = sigmoidf_acc(uz[q] + (gz[q] + bZ));
-                const float c = tanhf(un[q] + r * qn);
+                const float r = sigmoidf_gate(ur[q] + (gr[q] + bR));
+                const float z = sigmoidf_gate(uz[q] + (gz[q] + bZ));
+                const float c = tanhf_gate(un[q] + r * qn);
                 const float hi = hrow[q * C::HS + gi];
                 const float dan = lam[q] * (1.0f - z) * (1.0f - c * c);
                 const float daz = lam[q] * (hi - c) * z * (1.0f - z);
@@ -364,9 +364,9 @@ __global__ void __launch_bounds__(256, 2) cell_coef_mma_kernel(CellArgs a)
                     const float ur = el ? ur2.y : ur2.x, uz = el ? uz2.y : uz2.x, un = el ? un2.y : un2.x;
                     const float hi = el ? h2.y : h2.x;
                     const float qn = sq + sb[2 * N + i];                 // q = W_hn h + b_hn
-                    const float r = sigmoidf_acc(ur + (sr + sb[i]));
-                    const float z = sigmoidf_acc(uz + (sz + sb[N + i]));
-                    const float c = tanhf(un + r * qn);
+                    const float r = sigmoidf_gate(ur + (sr + sb[i]));
+                    const float z = sigmoidf_gate(uz + (sz + sb[N + i]));
+                    const float c = tanhf_gate(un + r * qn);
                     const float f = (1.0f - z) * c + z * hi;
                     const float az = (hi - c) * z * (1.0f - z);
                     const float an = (1.0f - z) * (1.0f - c * c);
