@@ -69,7 +69,7 @@ def tf32_peak_tflops(pk) -> float:
 # than L2; traffic grows in proportion to the positions processed, so a launch's traffic is this times B*T).
 NCU_SCAN_TRAFFIC_PER_POSITION = {1: 12.8, 2: 32.7, 4: 95.3, 8: 606.6, 16: 2213.0, 32: 8622.0, 64: 34116.0}
 # the two launches of the scan inside deer_gru_eval (n = 16, 32, 64): reduce, apply
-NCU_FUSED_TRAFFIC_PER_POSITION = {"scan_fused_reduce_kernel": {32: 686.0}, "scan_fused_apply_kernel": {32: 916.0}}
+NCU_FUSED_TRAFFIC_PER_POSITION = {"scan_fused_reduce_kernel": {32: 684.0}, "scan_fused_apply_kernel": {32: 916.0}}
 NCU_CONFIG2_SCAN_TRAFFIC = 51.43e6                      # scan_warp8_kernel inside the config-2 step, per launch
 
 
