@@ -520,7 +520,7 @@ template <int N> static int launch_cell_wide(CellArgs c, cudaStream_t st)
 // the tensor-core coefficient cell can contract the input projection itself (no u buffer, no projection pass)
 static bool coef_cell_projects(int n, int m, const float *x)
 {
-    return n == 32 && m % 8 == 0 && m >= 8 && m <= 64 && (((uintptr_t)x) & 7) == 0;
+    return (n == 32 || n == 16) && m % 8 == 0 && m >= 8 && m <= 64 && (((uintptr_t)x) & 7) == 0;
 }
 
 template <int N> static int launch_cell_coef_mma(CellArgs c, cudaStream_t st)
@@ -583,7 +583,7 @@ static int run_cell(CellArgs c, cudaStream_t st, bool generic = false)
         }
         if ((c.u || (c.coef_only && c.residual && coef_cell_projects(c.n, c.m, c.x))) && (((uintptr_t)c.W_h) & 15) == 0) {
             switch (c.n) {
-            case 16: return launch_cell_wide<16>(c, st);      // (coefficient rows too: measured equal to the tensor-core kernel)
+            case 16: return (c.coef_only && !c.u) ? launch_cell_coef_mma<16>(c, st) : launch_cell_wide<16>(c, st);
             case 32: return c.coef_only ? launch_cell_coef_mma<32>(c, st) : launch_cell_wide<32>(c, st);
             case 64: return launch_cell_wide<64>(c, st);
             default: break;
