@@ -827,6 +827,28 @@ static int check_mh_args(const deer_gru_params *heads, const int *strides, int H
     return DEER_OK;
 }
 
+static unsigned mh_blocks(size_t total);
+
+// strided view -> dense batch and back (128-bit moves when the layout allows)
+static int mh_pack(const float *src, float *dst, int B, int T, int s, int Tp, int C, int C_src, int off, cudaStream_t st)
+{
+    const size_t total = (size_t)B * s * Tp * C;
+    const bool v4 = C % 4 == 0 && C_src % 4 == 0 && off % 4 == 0 && ((((uintptr_t)src | (uintptr_t)dst) & 15) == 0);
+    if (v4) { DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<4><<<mh_blocks(total / 4), 256, 0, st>>>(src, dst, B, T, s, Tp, C, C_src, off)); }
+    else { DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<1><<<mh_blocks(total), 256, 0, st>>>(src, dst, B, T, s, Tp, C, C_src, off)); }
+    return DEER_OK;
+}
+
+static int mh_unpack(const float *src, float *dst, int B, int T, int s, int Tp, int C, int C_dst, int off, int accumulate,
+                     cudaStream_t st)
+{
+    const size_t total = (size_t)B * s * Tp * C;
+    const bool v4 = C % 4 == 0 && C_dst % 4 == 0 && off % 4 == 0 && ((((uintptr_t)src | (uintptr_t)dst) & 15) == 0);
+    if (v4) { DEER_KERNEL("mh_unpack_kernel", st, mh_unpack_kernel<4><<<mh_blocks(total / 4), 256, 0, st>>>(src, dst, B, T, s, Tp, C, C_dst, off, accumulate)); }
+    else { DEER_KERNEL("mh_unpack_kernel", st, mh_unpack_kernel<1><<<mh_blocks(total), 256, 0, st>>>(src, dst, B, T, s, Tp, C, C_dst, off, accumulate)); }
+    return DEER_OK;
+}
+
 static unsigned mh_blocks(size_t total)
 {
     size_t b = (total + 255) / 256;
@@ -1605,20 +1627,20 @@ int deer_gru_multihead_eval(const deer_gru_params *heads, const int *strides, in
         const int h = order[(size_t)oi];
         const int s = strides[h], Tp = (T + s - 1) / s, Bs = B * s;
         if (s != packed_stride) {              // heads of equal stride read the same dense batch of x
-            DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(x, w.xs, B, T, s, Tp, m, m, 0));
+            { if ((rc = mh_pack(x, w.xs, B, T, s, Tp, m, m, 0, st)) != DEER_OK) return rc; }
             packed_stride = s;
         }
         const float *xs = s == 1 ? x : w.xs;
         DEER_KERNEL("mh_y0_pack_kernel", st, mh_y0_pack_kernel<<<mh_blocks((size_t)Bs * n), 256, 0, st>>>(y0, w.y0s, B, s, n, H, h));
         if (flags & DEER_FLAG_WARM_START)
-            DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(y, w.ys, B, T, s, Tp, n, H * n, h * n));
+            { if ((rc = mh_pack(y, w.ys, B, T, s, Tp, n, H * n, h * n, st)) != DEER_OK) return rc; }
         int it = 0;
         rc = gru_eval_impl(&heads[h], xs, w.y0s, Bs, Tp, tol, max_iter, w.ys, &it, nullptr, nullptr, w.inner, w.inner_bytes,
                            flags, st);
         if (rc < 0) return rc;
         if (iters) iters[h] = it;
         if (rc > worst) worst = rc;
-        DEER_KERNEL("mh_unpack_kernel", st, mh_unpack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(w.ys, y, B, T, s, Tp, n, H * n, h * n, 0));
+        { if ((rc = mh_unpack(w.ys, y, B, T, s, Tp, n, H * n, h * n, 0, st)) != DEER_OK) return rc; }
     }
     DEER_CHECK_CUDA(cudaStreamSynchronize(st), "sync");
     return worst;
@@ -1644,18 +1666,18 @@ int deer_gru_multihead_vjp(const deer_gru_params *heads, const int *strides, int
         const int h = order[(size_t)oi];
         const int s = strides[h], Tp = (T + s - 1) / s, Bs = B * s;
         if (s != packed_stride) {
-            DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(x, w.xs, B, T, s, Tp, m, m, 0));
+            { if ((rc = mh_pack(x, w.xs, B, T, s, Tp, m, m, 0, st)) != DEER_OK) return rc; }
             packed_stride = s;
         }
         const float *xs = s == 1 ? x : w.xs;
         DEER_KERNEL("mh_y0_pack_kernel", st, mh_y0_pack_kernel<<<mh_blocks((size_t)Bs * n), 256, 0, st>>>(y0, w.y0s, B, s, n, H, h));
-        DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(y, w.ys, B, T, s, Tp, n, H * n, h * n));
-        DEER_KERNEL("mh_pack_kernel", st, mh_pack_kernel<<<mh_blocks((size_t)Bs * Tp * n), 256, 0, st>>>(gy, w.gys, B, T, s, Tp, n, H * n, h * n));
+        { if ((rc = mh_pack(y, w.ys, B, T, s, Tp, n, H * n, h * n, st)) != DEER_OK) return rc; }
+        { if ((rc = mh_pack(gy, w.gys, B, T, s, Tp, n, H * n, h * n, st)) != DEER_OK) return rc; }
         rc = gru_vjp_impl(&heads[h], xs, w.y0s, w.ys, w.gys, Bs, Tp, &dheads[h], dx ? w.dxs : nullptr, dy0 ? w.dy0s : nullptr,
                           w.inner, w.inner_bytes, flags, st);
         if (rc != DEER_OK) return rc;
         if (dx)     // the heads' input gradients add up, head by head in a fixed order (that of the strides)
-            DEER_KERNEL("mh_unpack_kernel", st, mh_unpack_kernel<<<mh_blocks((size_t)Bs * Tp * m), 256, 0, st>>>(w.dxs, dx, B, T, s, Tp, m, m, 0, oi > 0));
+            { if ((rc = mh_unpack(w.dxs, dx, B, T, s, Tp, m, m, 0, oi > 0, st)) != DEER_OK) return rc; }
         if (dy0)
             DEER_KERNEL("mh_dy0_reduce_kernel", st, mh_dy0_reduce_kernel<<<mh_blocks((size_t)B * n), 256, 0, st>>>(w.dy0s, dy0, B, s, n, H, h));
         // the inner gradient calls share one status block: keep every head's flags

@@ -1052,29 +1052,40 @@ __global__ void __launch_bounds__(ODE_THREADS) ode_discretise_kernel(const float
 // (a GRU is causal: padding behind the last position changes nothing before it).
 //   pack  : dst[(b s + p), t', c] = src[b, p + s t', off + c]     (src rows of C_src channels; 0 past T)
 //   unpack: dst[b, p + s t', off + c] (+)= src[(b s + p), t', c]  (valid positions only)
+// V = 4: channels moved as 128-bit words (C, the row strides, off and the pointers multiples of 4 floats / 16 bytes).
+template <int V>
 __global__ void mh_pack_kernel(const float *__restrict__ src, float *__restrict__ dst, int B, int T, int s, int Tp, int C,
                                int C_src, int off)
 {
-    const size_t total = (size_t)B * s * Tp * C;
+    const int Cv = C / V;
+    const size_t total = (size_t)B * s * Tp * Cv;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % C);
-        const size_t r = i / C;
+        const int c = (int)(i % Cv) * V;
+        const size_t r = i / Cv;
         const int tp = (int)(r % Tp);
         const size_t q = r / Tp;
         const int p = (int)(q % s);
         const size_t b = q / s;
         const long long t = (long long)p + (long long)s * tp;
-        dst[i] = t < T ? src[(b * T + (size_t)t) * C_src + off + c] : 0.0f;
+        if constexpr (V == 4) {
+            float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (t < T) v = *reinterpret_cast<const float4 *>(src + (b * T + (size_t)t) * C_src + off + c);
+            *reinterpret_cast<float4 *>(dst + r * C + c) = v;
+        } else {
+            dst[r * C + c] = t < T ? src[(b * T + (size_t)t) * C_src + off + c] : 0.0f;
+        }
     }
 }
 
+template <int V>
 __global__ void mh_unpack_kernel(const float *__restrict__ src, float *__restrict__ dst, int B, int T, int s, int Tp, int C,
                                  int C_dst, int off, int accumulate)
 {
-    const size_t total = (size_t)B * s * Tp * C;
+    const int Cv = C / V;
+    const size_t total = (size_t)B * s * Tp * Cv;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % C);
-        const size_t r = i / C;
+        const int c = (int)(i % Cv) * V;
+        const size_t r = i / Cv;
         const int tp = (int)(r % Tp);
         const size_t q = r / Tp;
         const int p = (int)(q % s);
@@ -1082,7 +1093,16 @@ __global__ void mh_unpack_kernel(const float *__restrict__ src, float *__restric
         const long long t = (long long)p + (long long)s * tp;
         if (t < T) {
             float *d = dst + (b * T + (size_t)t) * C_dst + off + c;
-            *d = accumulate ? *d + src[i] : src[i];
+            if constexpr (V == 4) {
+                float4 v = *reinterpret_cast<const float4 *>(src + r * C + c);
+                if (accumulate) {
+                    const float4 o = *reinterpret_cast<const float4 *>(d);
+                    v = make_float4(o.x + v.x, o.y + v.y, o.z + v.z, o.w + v.w);
+                }
+                *reinterpret_cast<float4 *>(d) = v;
+            } else {
+                *d = accumulate ? *d + src[r * C + c] : src[r * C + c];
+            }
         }
     }
 }
