@@ -58,6 +58,53 @@ def test_scan_at_full_size_launch_geometries(bd, n, B, T, chain):
         del want, got
 
 
+# (n, B, T): batches small enough that a resolver warp serves ONE sequence through its ring of staged tile aggregates,
+# with 1, 2 or 4 resolving warps per resolver CTA (B <= 4, <= 8, more) and hundreds of tiles per sequence (the ring
+# wraps many times), and a batch with several sequences per resolver warp
+SMALL_BATCH_CASES = [(32, 1, 40_000), (32, 3, 30_000), (32, 6, 16_000), (32, 12, 9_000), (16, 1, 60_000), (16, 5, 20_000),
+                     (16, 70, 1_500), (32, 40, 1_200)]
+
+
+@pytest.mark.parametrize("n,B,T", SMALL_BATCH_CASES)
+def test_scan_small_batches_of_long_sequences(bd, n, B, T):
+    """Eq. 9-10 where the resolver's walk over one sequence's tiles is the critical path: stand-alone scans, forward
+    and reverse, against the sequential solve."""
+    geo = bd.deer_scan_geometry(B, T, n)
+    assert geo["single_pass"] and geo["tiles_per_seq"] >= 8
+    J = synth.contractive_J(B, T, n, seed=n + T + B, tag="sb/J", scale=1.0)
+    b = synth.normal(n + T + B, "sb/b", (B, T, n))
+    y0 = synth.normal(n + T + B, "sb/y0", (B, n))
+    Jd, bdv, y0d = dev(J), dev(b), dev(y0)
+    ws = bd.alloc_workspace(bd.DEER_OP_SCAN, B, T, n)
+    for reverse in (False, True):
+        want = oracle.linrec(J, b, y0, reverse=reverse, dtype=np.float64)
+        got = bd.deer_linrec_scan(Jd, bdv, y0d, reverse=reverse, ws=ws)
+        assert bd.deer_workspace_status(ws) == bd.DEER_OK
+        err = float(np.max(np.abs(got.cpu().numpy() - want)))
+        assert err <= TOL_SCAN * max(1.0, float(np.max(np.abs(want)))), (reverse, err)
+        del want, got
+
+
+@pytest.mark.parametrize("n,B,T", [(32, 1, 50_000), (32, 4, 25_000), (16, 2, 40_000), (16, 7, 12_000)])
+def test_eval_small_batches_of_long_sequences(bd, n, B, T):
+    """The same batches through deer_gru_eval (two-launch scan: the reduce launch's resolvers) and its gradient (the
+    generated-J reverse scan), against the sequential trajectory and BPTT."""
+    p_np = synth.gru_params(n, n, 31, tag="sbe/gru")
+    x = synth.x_gaussian(B, T, n, 31, tag="sbe/x")
+    y0 = (synth.normal(31, "sbe/y0", (B, n)) * 0.3).astype(np.float32)
+    p = bd.GruParamsDev.from_numpy(p_np)
+    r = bd.deer_gru_eval(p, dev(x), dev(y0))
+    seq = oracle.gru_seq(p_np, x, y0, np.float32)
+    assert r.status == 0
+    assert float(np.max(np.abs(r.y.cpu().numpy() - seq))) <= TOL_Y
+    gy = (synth.normal(31, "sbe/gy", (B, T, n)) / np.sqrt(T)).astype(np.float32)
+    got = bd.deer_gru_vjp(p, dev(x), dev(y0), dev(seq.astype(np.float32)), dev(gy))
+    want = oracle.gru_bptt(p_np, x, y0, seq.astype(np.float64), gy, np.float64)
+    for k in ("dW_i", "dW_h", "db_i", "db_h", "dx", "dy0"):
+        a, b_ = got[k].cpu().numpy().astype(np.float64), np.asarray(want[k])
+        assert np.max(np.abs(a - b_)) <= 1e-3 * max(1e-30, np.max(np.abs(b_))), k
+
+
 # the points of the speed grid (n = m, B = 16, x ~ N(0,1)) whose Jacobians exceed L2
 SWEEP_POINTS = [(1, 1_000_000), (2, 1_000_000), (4, 1_000_000), (8, 1_000_000), (16, 100_000), (64, 10_000)]
 
