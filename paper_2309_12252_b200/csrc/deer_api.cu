@@ -585,7 +585,7 @@ static int run_cell(CellArgs c, cudaStream_t st, bool generic = false)
             switch (c.n) {
             case 16: return (c.coef_only && !c.u) ? launch_cell_coef_mma<16>(c, st) : launch_cell_wide<16>(c, st);
             case 32: return c.coef_only ? launch_cell_coef_mma<32>(c, st) : launch_cell_wide<32>(c, st);
-            case 64: return launch_cell_wide<64>(c, st);
+            case 64: return (c.coef_only && c.u) ? launch_cell_coef_mma<64>(c, st) : launch_cell_wide<64>(c, st);
             default: break;
             }
         }
