@@ -530,7 +530,7 @@ template <int N> static int launch_cell_coef_mma(CellArgs c, cudaStream_t st)
     int rc;
     const size_t total = (size_t)c.B * c.T;
     const size_t tiles = (total + 127) / 128;
-    const size_t cap = (size_t)num_sms() * 4;
+    const size_t cap = (size_t)num_sms() * 2;          // (the kernel's launch bounds: two CTAs per SM; one wave, the weights split once per CTA)
     const unsigned blocks = (unsigned)(tiles < cap ? tiles : cap);
     if (proj) {
         if ((rc = opt_in_smem((const void *)cell_coef_mma_kernel<N, true>, SM)) != DEER_OK) return rc;
