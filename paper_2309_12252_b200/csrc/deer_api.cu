@@ -193,6 +193,8 @@ static long long single_pass_max_batch(int n, bool umma)
 // n = 16, 32: warps of a resolver CTA that resolve.  A resolver CTA's staging area is shared by its resolving warps,
 // and the walk over ONE sequence's tiles is the serial part of a scan: small batches give each sequence a deeper ring.
 static int big_res_warps(int B) { return B <= 4 ? 1 : B <= 8 ? 2 : 4; }
+// n = 64 (two resolving warps per CTA at most): one warp with all the CTA's tile slots for small batches
+static int res_warps64(int B) { return B <= 8 ? 1 : 2; }
 
 struct PassCfg {
     const char *name;
@@ -332,7 +334,8 @@ static int launch_fused_fwd64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t s
     static int occ[MAX_DEVICES] = {0};
     static int occ_apply[MAX_DEVICES] = {0};
     w.sw = C::L;                               // a tile is one chain
-    const PassCfg c{"scan_fused_reduce64_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 4, 16};
+    w.res_warps = res_warps64(a.B);
+    const PassCfg c{"scan_fused_reduce64_kernel", C::THREADS, C::SMEM, w.res_warps, C::MAX_SEQ_PER_WARP, 4, 16};
     int rc = launch_single_pass(scan_fused_reduce64_kernel, occ, c, a, w, prep, st);
     if (rc != DEER_OK) return rc;
     int dev = 0;
@@ -360,7 +363,8 @@ static int launch_cta64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = Cta64;
     static int occ[MAX_DEVICES] = {0};
-    const PassCfg c{"scan_cta64_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 8, 16};
+    w.res_warps = res_warps64(a.B);
+    const PassCfg c{"scan_cta64_kernel", C::THREADS, C::SMEM, w.res_warps, C::MAX_SEQ_PER_WARP, 8, 16};
     return launch_single_pass(scan_cta64_kernel<REV>, occ, c, a, w, prep, st);
 }
 
@@ -369,6 +373,7 @@ static int launch_umma64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t st)
 {
     using C = Umma64;
     static int occ[MAX_DEVICES] = {0};
+    w.res_warps = C::RES_WARPS;
     const PassCfg c{"scan_umma64_kernel", C::THREADS, C::SMEM, C::RES_WARPS, C::MAX_SEQ_PER_WARP, 2, 8};
     return launch_single_pass(scan_umma64_kernel<REV>, occ, c, a, w, prep, st);
 }
@@ -1749,7 +1754,7 @@ int deer_scan_geometry(int B, int T, int n, int flags, int *out)
         case 1: case 2: case 4: res_warps = n == 4 ? OnePass<4>::WARPS : OnePass<1>::WARPS; max_seq = OnePass<1>::MAX_SEQ_PER_WARP; break;
         case 8: res_warps = Warp8::RES_WARPS; max_seq = OnePass<8>::MAX_SEQ_PER_WARP; break;
         case 16: case 32: res_warps = big_res_warps(B); max_seq = WarpN<16>::MAX_SEQ_PER_WARP; break;
-        default: res_warps = umma ? Umma64::RES_WARPS : Cta64::RES_WARPS; max_seq = Cta64::MAX_SEQ_PER_WARP; res_cap = umma ? 8 : 16; break;
+        default: res_warps = umma ? Umma64::RES_WARPS : res_warps64(B); max_seq = Cta64::MAX_SEQ_PER_WARP; res_cap = umma ? 8 : 16; break;
         }
         out[0] = 1; out[1] = L1; out[2] = sw; out[3] = (T + L1 - 1) / L1;
         out[4] = resolver_ctas(B, res_warps, max_seq, res_cap);

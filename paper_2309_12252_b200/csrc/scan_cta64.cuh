@@ -28,7 +28,8 @@ struct Cta64 {
     static constexpr int STAGE_FLOATS = N * (N + 8) + N;   // matrix with padded rows, then the vector
     static constexpr int RES_WARPS = 2;
     static constexpr int SM_WORK = STAGES * STAGE_FLOATS + 2 * N;
-    static constexpr int SM_RES = RES_WARPS * (AGG + N);
+    static constexpr int RES_SLOTS = 3;                // tile aggregates a resolver CTA stages, shared by its resolving warps
+    static constexpr int SM_RES = RES_SLOTS * AGG + RES_WARPS * N;
     static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
     static constexpr int MAX_SEQ_PER_WARP = 8;
@@ -36,15 +37,84 @@ struct Cta64 {
 
 template <int K> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(K) : "memory"); }
 
-// Resolver for n = 64: lane i holds components i and i + 32 of the running state; one aggregate
-// is staged per step (16.6 KB).
-__device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_all, int rw, int nrw, int lane)
+// Resolver for n = 64: lane i holds components i and i + 32 of the running state.  An aggregate is 16.6 KB: it is
+// fetched by asynchronous copies, all of it in flight at once, into one of the warp's tile slots; a warp that serves
+// ONE sequence requests the following tiles (as many as it has slots) while it walks the current one, so the round
+// trips stay off the serial walk.  The resolver CTA's `slots` tile slots are shared by its w.res_warps resolving warps
+// (small batches: one warp with all the slots).
+__device__ __forceinline__ float2 resolver64_walk(const float *stage, float *ysm, float y0v, float y1v, int lane)
+{
+    constexpr int N = 64, NN = N * N;
+    ysm[lane] = y0v; ysm[32 + lane] = y1v;
+    __syncwarp();
+    float a0 = stage[NN + lane], a1 = stage[NN + 32 + lane];
+    const float *r0 = stage + lane * N, *r1 = stage + (32 + lane) * N;
+#pragma unroll 8
+    for (int i = 0; i < N; ++i) {           // skewed column order: conflict-free reads
+        const int c = (i + lane) & (N - 1);
+        const float yc = ysm[c];
+        a0 = fmaf(r0[c], yc, a0);
+        a1 = fmaf(r1[c], yc, a1);
+    }
+    __syncwarp();
+    return make_float2(a0, a1);
+}
+
+__device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_all, int slots, int rw, int nrw, int lane)
 {
     if (a.no_resolve) return;     // (wait-expiry test: nobody publishes entering states)
     using C = Cta64;
-    constexpr int N = C::N, AGG = C::AGG, NN = C::NN;
-    float *stage = stage_all + (threadIdx.x >> 5) * (AGG + N);
-    float *ysm = stage + AGG;
+    constexpr int N = C::N, AGG = C::AGG;
+    const int wib = threadIdx.x >> 5;                              // resolving warp of this CTA
+    const int RING = max(1, min(4, slots / w.res_warps));          // this warp's tile slots
+    float *stage = stage_all + (size_t)wib * RING * AGG;
+    float *ysm = stage_all + (size_t)slots * AGG + wib * N;
+    auto fetch = [&](float *dst, const float *src) {
+        for (int i = lane; i < AGG / 4; i += 32) cp_async16(dst + 4 * i, src + 4 * i);
+        cp_async_commit();
+    };
+    unsigned spins = 0;
+    if (rw + nrw >= a.B) {
+        // ---- one sequence: tile i in slot i % RING, one fetch group per tile, up to RING in flight
+        const int s = rw;
+        if (s >= a.B) return;
+        const unsigned *flags = w.flags + (size_t)s * w.nch;
+        const float *aggs = w.aggs + (size_t)s * w.nch * AGG;
+        unsigned long long *starts = w.starts + (size_t)s * w.nch * N;
+        float y0v = 0.0f, y1v = 0.0f;
+        if (a.y0) { y0v = a.y0[(size_t)s * N + lane]; y1v = a.y0[(size_t)s * N + 32 + lane]; }
+        int c = 0, f = 0;                      // next tile to walk, next tile to fetch
+        unsigned fl = (lane < w.nch) ? ld_acquire_u32(flags + lane) : 0u;      // flags of tiles f + lane
+        while (c < w.nch) {
+            bool progressed = false;
+            if (f - c < RING && f < w.nch) {
+                const unsigned m = __ballot_sync(0xffffffffu, fl >= 1u);
+                __syncwarp();      // orders every lane's aggregate copies below after the acquiring lanes' flag loads
+                int r = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
+                r = min(r, RING - (f - c));
+                for (int i = 0; i < r; ++i) fetch(stage + (size_t)((f + i) % RING) * AGG, aggs + (size_t)(f + i) * AGG);
+                if (r > 0) progressed = true;
+                f += r;
+                fl = (f + lane < w.nch) ? ld_acquire_u32(flags + f + lane) : 0u;
+            }
+            if (f > c) {
+                const int ng = f - c;          // groups in flight, oldest first
+                if (ng == 1) cp_async_wait<0>(); else if (ng == 2) cp_async_wait<1>(); else if (ng == 3) cp_async_wait<2>(); else cp_async_wait<3>();
+                __syncwarp();
+                st_relaxed_u64(starts + (size_t)c * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y0v));
+                st_relaxed_u64(starts + (size_t)c * N + 32 + lane, LL_FLAG | (unsigned long long)__float_as_uint(y1v));
+                const float2 yn = resolver64_walk(stage + (size_t)(c % RING) * AGG, ysm, y0v, y1v, lane);
+                y0v = yn.x; y1v = yn.y;
+                if (lane == 0) w.flags[(size_t)s * w.nch + c] = 0u;     // consumed: cleared for the next launch
+                ++c;
+                progressed = true;
+            }
+            if (progressed) spins = 0;
+            else if (!keep_spinning(a, spins)) { cp_async_wait<0>(); return; }
+        }
+        return;
+    }
+    // ---- several sequences per warp: one tile per visit
     int nseq = 0;
     int pos[C::MAX_SEQ_PER_WARP];
     float ya[C::MAX_SEQ_PER_WARP], yb[C::MAX_SEQ_PER_WARP];
@@ -60,7 +130,6 @@ __device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_a
         }
     }
     int remaining = nseq;
-    unsigned spins = 0;
     while (remaining > 0) {
         bool progressed = false;
 #pragma unroll
@@ -71,7 +140,7 @@ __device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_a
             const int s = rw + k * nrw;
             const unsigned *flags = w.flags + (size_t)s * w.nch;
             const unsigned m = __ballot_sync(0xffffffffu, fnext[k] >= 1u);
-            __syncwarp();      // orders every lane's aggregate loads below after the acquiring lanes' flag loads
+            __syncwarp();      // orders every lane's aggregate copies below after the acquiring lanes' flag loads
             const int cnt = (m == 0xffffffffu) ? 32 : (__ffs(~m) - 1);
             if (cnt == 0) {
                 fnext[k] = (c0 + lane < w.nch) ? ld_acquire_u32(flags + c0 + lane) : 0u;
@@ -83,34 +152,11 @@ __device__ void resolver64(const ScanArgs &a, const OnePassWs &w, float *stage_a
             for (int q = 0; q < cnt; ++q) {
                 st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y0v));
                 st_relaxed_u64(out + q * N + 32 + lane, LL_FLAG | (unsigned long long)__float_as_uint(y1v));
-                const float4 *src = reinterpret_cast<const float4 *>(w.aggs + ((size_t)s * w.nch + c0 + q) * AGG);
-                float4 *dst = reinterpret_cast<float4 *>(stage);
-                for (int i0 = 0; i0 < AGG / 4; i0 += 32 * 8) {
-                    float4 v[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        if (i < AGG / 4) v[u] = __ldcg(src + i);
-                    }
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        if (i < AGG / 4) dst[i] = v[u];
-                    }
-                }
-                ysm[lane] = y0v; ysm[32 + lane] = y1v;
+                fetch(stage, w.aggs + ((size_t)s * w.nch + c0 + q) * AGG);
+                cp_async_wait<0>();
                 __syncwarp();
-                float a0 = stage[NN + lane], a1 = stage[NN + 32 + lane];
-                const float *r0 = stage + lane * N, *r1 = stage + (32 + lane) * N;
-#pragma unroll 8
-                for (int i = 0; i < N; ++i) {           // skewed column order: conflict-free reads
-                    const int c = (i + lane) & (N - 1);
-                    const float yc = ysm[c];
-                    a0 = fmaf(r0[c], yc, a0);
-                    a1 = fmaf(r1[c], yc, a1);
-                }
-                y0v = a0; y1v = a1;
-                __syncwarp();
+                const float2 yn = resolver64_walk(stage, ysm, y0v, y1v, lane);
+                y0v = yn.x; y1v = yn.y;
             }
             ya[k] = y0v; yb[k] = y1v;
             if (lane < cnt) w.flags[(size_t)s * w.nch + c0 + lane] = 0u;   // consumed: cleared for the next launch
@@ -231,7 +277,7 @@ __global__ void __launch_bounds__(Cta64::THREADS) scan_cta64_kernel(ScanArgs a, 
     }
     __syncthreads();
     if (s_role < w.resolvers) {
-        resolver64(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        if (warp < w.res_warps) resolver64(a, w, sm, C::RES_SLOTS, s_role * w.res_warps + warp, w.resolvers * w.res_warps, lane);
         __syncthreads();
         if (tid == 0) scan_epilogue(a.st);
         return;

@@ -5,11 +5,14 @@
 // four warps, and a tile is a single chain (the resolver CTAs, those of scan_cta64.cuh, walk the chain
 // aggregates directly: no prefix aggregates).  Per position:
 //   * warp w builds rows 16w .. 16w+15 of J_t from the staged coefficient rows and ITS share of W_h, which it
-//     keeps in registers for the whole launch (96 per lane), rounds them to bf16 and writes them to shared
-//     memory in the layout of the m16n8k16 B operand (8 KB per position, double-buffered); it also advances
-//     its 16 components of beta (fp32 mat-vec from the same values, beta exchanged through shared memory);
-//   * after a CTA barrier every warp multiplies ITS 16 rows of X = P^T by J_t^T: 32 bf16 MMAs with the
-//     accumulator tiles of X as the A operand as they stand (fp32 accumulate, 8 independent accumulators).
+//     keeps in registers for the whole launch as bf16 pairs (48 per lane), in packed bf16 arithmetic (the result
+//     is the m16n8k16 B operand as it stands), and writes them to shared memory (8 KB per position,
+//     double-buffered); it also advances its 16 components of beta: beta^T J_t^T for its columns is eight more
+//     MMAs on the fragments it has just built (beta exchanged through shared memory);
+//   * every warp multiplies ITS 16 rows of X = P^T by J_t^T: 32 bf16 MMAs with the accumulator tiles of X as the
+//     A operand as they stand (fp32 accumulate, 8 independent accumulators).
+// The rows of position q + 1 do not depend on X: they are built in the same loop body as the products of position q,
+// so a position costs ONE CTA barrier and the two kinds of work fill each other's gaps.
 // The replay kernel is scan_fused_apply_kernel<64>: W_h^T as the B operand from shared memory (48 KB: it does
 // not fit the registers of one warp), TF32.
 #pragma once
@@ -28,7 +31,8 @@ template <> struct FusedFwd<64> {
     static constexpr int JB_WORDS = NT * 2 * 32 * 4;   // bf16 B fragments of one position: [nn][half][lane][4 words]
     static constexpr int RES_WARPS = Cta64::RES_WARPS, MAX_SEQ_PER_WARP = Cta64::MAX_SEQ_PER_WARP;
     static constexpr int SM_WORK = STAGES * STAGE_FLOATS + 2 * JB_WORDS + 2 * N + 16;
-    static constexpr int SM_RES = RES_WARPS * (AGG + N);
+    static constexpr int RES_SLOTS = 4;                // tile aggregates a resolver CTA stages, shared by its resolving warps
+    static constexpr int SM_RES = RES_SLOTS * AGG + RES_WARPS * N;
     static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
     // apply kernel
@@ -60,7 +64,7 @@ __global__ void __launch_bounds__(FusedFwd<64>::THREADS, 2) scan_fused_reduce64_
 
     // this warp's rows of J: i = 8 (2 warp + h) + g, h = 0, 1; its weights for them, by B-operand piece (j, e):
     // columns 16 j + 8 e + 2t, + 1
-    float2 wR[2][4][2], wZ[2][4][2], wN[2][4][2];
+    unsigned wR[2][4][2], wZ[2][4][2], wN[2][4][2];
 #pragma unroll
     for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -68,17 +72,18 @@ __global__ void __launch_bounds__(FusedFwd<64>::THREADS, 2) scan_fused_reduce64_
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const float *wp = a.Wh + (size_t)(8 * (2 * warp + h) + g) * N + 16 * j + 8 * e + 2 * t;
-                wR[h][j][e] = __ldg(reinterpret_cast<const float2 *>(wp));
-                wZ[h][j][e] = __ldg(reinterpret_cast<const float2 *>(wp + NN));
-                wN[h][j][e] = __ldg(reinterpret_cast<const float2 *>(wp + 2 * NN));
+                const float2 r2 = __ldg(reinterpret_cast<const float2 *>(wp));
+                const float2 z2 = __ldg(reinterpret_cast<const float2 *>(wp + NN));
+                const float2 n2 = __ldg(reinterpret_cast<const float2 *>(wp + 2 * NN));
+                wR[h][j][e] = pack_bf16(r2.x, r2.y); wZ[h][j][e] = pack_bf16(z2.x, z2.y); wN[h][j][e] = pack_bf16(n2.x, n2.y);
             }
     const bool d0 = g == 2 * t, d1 = g == 2 * t + 1;      // the piece (j, e) = ((2 warp + h) / 2, (2 warp + h) % 2) holds the diagonal
 
     if (tid == 0) s_role = (int)atomicAdd(&a.st->role_counter, 1u);
     __syncthreads();
     if (s_role < w.resolvers) {
-        if (warp < C::RES_WARPS)
-            resolver64(a, w, sm, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+        if (warp < w.res_warps)
+            resolver64(a, w, sm, C::RES_SLOTS, s_role * w.res_warps + warp, w.resolvers * w.res_warps, lane);
         __syncthreads();
         if (tid == 0) scan_epilogue(a.st, false);
         return;
@@ -139,46 +144,68 @@ __global__ void __launch_bounds__(FusedFwd<64>::THREADS, 2) scan_fused_reduce64_
 #pragma unroll
         for (int q = 0; q < S - 1; ++q) issue(q);
 
-#pragma unroll 1
-        for (int q = 0; q < cnt; ++q) {
-            cp_async_wait_n<S - 2>();
-            __syncthreads();                   // stage q visible to all; buffers of position q - 2 and ring stage q - 1 are free
-            issue(q + S - 1);
-            const float *Ms = ring + (q % S) * C::STAGE_FLOATS;
-            const float *bin = beta + (q & 1) * N;
-            float *bout = beta + ((q + 1) & 1) * N;
-            uint4 *Jq = Jb + (q & 1) * (C::JB_WORDS / 4);
-            // ---- this warp's 16 rows of J_t: bf16 B fragments to shared memory, and its 16 components of beta
-            float2 bp[4][2];
+        // this warp's 16 rows of J_p (bf16 B fragments to shared memory) and its 16 components of beta_{p+1} = J_p beta_p + r_p
+        auto build = [&](int p) {
+            const float *Ms = ring + (p % S) * C::STAGE_FLOATS;
+            const float *bin = beta + (p & 1) * N;
+            float *bout = beta + ((p + 1) & 1) * N;
+            uint4 *Jp = Jb + (p & 1) * (C::JB_WORDS / 4);
+            // beta^T as the live row of an A operand (lanes g == 0), one k block of 16 per j
+            unsigned ab[4][2];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) bp[j][e] = *reinterpret_cast<const float2 *>(bin + 16 * j + 8 * e + 2 * t);
+            for (int j = 0; j < 4; ++j) {
+                const float2 lo = *reinterpret_cast<const float2 *>(bin + 16 * j + 2 * t);
+                const float2 hi = *reinterpret_cast<const float2 *>(bin + 16 * j + 8 + 2 * t);
+                ab[j][0] = g == 0 ? pack_bf16(lo.x, lo.y) : 0u;
+                ab[j][1] = g == 0 ? pack_bf16(hi.x, hi.y) : 0u;
+            }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int nn = 2 * warp + h, i = 8 * nn + g;
                 const float4 cf = *reinterpret_cast<const float4 *>(Ms + 4 * i);
-                const float2 cx = make_float2(cf.x, cf.x), cy = make_float2(cf.y, cf.y), cz = make_float2(cf.z, cf.z);
+                const unsigned cr = pack_bf16(cf.x, cf.x), cz = pack_bf16(cf.y, cf.y), cn = pack_bf16(cf.z, cf.z);
+                const unsigned zd = pack_bf16(d0 ? cf.w : 0.0f, d1 ? cf.w : 0.0f);
                 unsigned words[4][2];
-                float2 p2 = make_float2(0.0f, 0.0f);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) words[j][e] = hmul2_bf16(cn, wN[h][j][e]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) words[j][e] = hfma2_bf16(cz, wZ[h][j][e], words[j][e]);
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
-                        float2 v = ffma2(cx, wR[h][j][e], ffma2(cy, wZ[h][j][e], fmul2(cz, wN[h][j][e])));
-                        if (2 * j + e == nn) { v.x += d0 ? cf.w : 0.0f; v.y += d1 ? cf.w : 0.0f; }
-                        p2 = ffma2(v, bp[j][e], p2);
-                        words[j][e] = pack_bf16(v.x, v.y);
+                        words[j][e] = hfma2_bf16(cr, wR[h][j][e], words[j][e]);
+                        if (2 * j + e == nn) words[j][e] = hadd2_bf16(words[j][e], zd);
                     }
-                Jq[(nn * 2 + 0) * 32 + lane] = make_uint4(words[0][0], words[0][1], words[1][0], words[1][1]);
-                Jq[(nn * 2 + 1) * 32 + lane] = make_uint4(words[2][0], words[2][1], words[3][0], words[3][1]);
-                float part = p2.x + p2.y;
-                part += __shfl_xor_sync(0xffffffffu, part, 1);
-                part += __shfl_xor_sync(0xffffffffu, part, 2);
-                if (t == 0) bout[i] = part + Ms[4 * N + i];
+                Jp[(nn * 2 + 0) * 32 + lane] = make_uint4(words[0][0], words[0][1], words[1][0], words[1][1]);
+                Jp[(nn * 2 + 1) * 32 + lane] = make_uint4(words[2][0], words[2][1], words[3][0], words[3][1]);
+                float cb[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const unsigned af[4] = {ab[j][0], 0u, ab[j][1], 0u};
+                    mma_bf16(cb, af, words[j], cb);
+                }
+                if (g == 0) {
+                    const float2 r2 = *reinterpret_cast<const float2 *>(Ms + 4 * N + 8 * nn + 2 * t);
+                    *reinterpret_cast<float2 *>(bout + 8 * nn + 2 * t) = make_float2(cb[0] + r2.x, cb[1] + r2.y);
+                }
             }
-            __syncthreads();                   // J_t and the new beta are visible
-            // ---- X <- X J_t^T for this warp's 16 rows: accumulator tiles 2j, 2j+1 are the A operand of block j
+        };
+        cp_async_wait_n<S - 2>();
+        __syncthreads();                       // stage 0 and beta_0 visible
+        if (cnt > 0) build(0);
+
+#pragma unroll 1
+        for (int q = 0; q < cnt; ++q) {
+            cp_async_wait_n<S - 3>();
+            __syncthreads();                   // J_q, beta_{q+1} and stage q + 1 visible to all; the buffers of position q - 1 are free
+            issue(q + S - 1);
+            const uint4 *Jq = Jb + (q & 1) * (C::JB_WORDS / 4);
+            // ---- X <- X J_q^T for this warp's 16 rows: accumulator tiles 2j, 2j+1 are the A operand of block j
             unsigned af[4][4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -205,6 +232,8 @@ __global__ void __launch_bounds__(FusedFwd<64>::THREADS, 2) scan_fused_reduce64_
                     mma_bf16(acc[nn], af[2 * half + 1], bf, acc[nn]);
                 }
             }
+            // ---- the rows of the next position and beta_{q+2}, while those MMAs are in flight
+            if (q + 1 < cnt) build(q + 1);
         }
         cp_async_wait_n<0>();
         __syncthreads();

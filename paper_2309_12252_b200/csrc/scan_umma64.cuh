@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(Umma64::THREADS) scan_umma64_kernel(ScanArgs a
     __syncthreads();
     if (s_role < w.resolvers) {
         if (warp < C::RES_WARPS)
-            resolver64(a, w, reinterpret_cast<float *>(sm), s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
+            resolver64(a, w, reinterpret_cast<float *>(sm), C::RES_WARPS, s_role * C::RES_WARPS + warp, w.resolvers * C::RES_WARPS, lane);
         __syncthreads();
         if (tid == 0) scan_epilogue(a.st);
         return;
