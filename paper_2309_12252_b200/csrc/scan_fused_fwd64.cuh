@@ -44,7 +44,7 @@ template <> struct FusedFwd<64> {
     static constexpr size_t A_SMEM = sizeof(float) * (A_WARPS * A_STAGES * STAGE_A + A_WARPS * ROWS * N + 2 * NT * 3 * NT * 32) + 128;
 };
 
-__global__ void __launch_bounds__(FusedFwd<64>::THREADS, 2) scan_fused_reduce64_kernel(ScanArgs a, OnePassWs w)
+__global__ void __launch_bounds__(FusedFwd<64>::THREADS, 3) scan_fused_reduce64_kernel(ScanArgs a, OnePassWs w)
 {
     using C = FusedFwd<64>;
     constexpr int N = C::N, NN = C::NN, AGG = C::AGG, NT = C::NT, S = C::STAGES, L = C::L;
