@@ -1275,10 +1275,10 @@ static int host_pipe_for_current_device(HostPipe **out)
 int deer_gru_eval_host_chunk(int B, int T)
 {
     if (B <= 0 || T <= 0) return 0;
-    // chunks of about 3 x 2^17 positions: long enough to fill the GPU, short enough that the first copy in and the last
-    // copy out (the two that nothing hides) are a small part of the call
+    // chunks of about 2^19 positions: long enough to fill the GPU, short enough that the first copy in and the last
+    // copy out (the two that nothing hides) are a small part of the call (config 3: three chunks measured best of 1 ... 8)
     const long long N = (long long)B * T;
-    long long nc = (N + 196608) / 393216;
+    long long nc = (N + 262144) / 524288;
     if (nc > DEER_HOST_MAX_CHUNKS) nc = DEER_HOST_MAX_CHUNKS;
     if (nc > B) nc = B;
     if (nc < 1) nc = 1;

@@ -85,15 +85,15 @@ def test_scan_geometry_bounds_the_resolver_ctas(L):
 
 
 def test_host_call_chunking_rule(L):
-    """deer_gru_eval_host splits a batch into chunks of whole sequences of about 3 x 2^17 positions, at most eight, and
+    """deer_gru_eval_host splits a batch into chunks of whole sequences of about 2^19 positions, at most eight, and
     leaves small batches and single sequences whole (host logic only)."""
     f = L.deer_gru_eval_host_chunk
     assert f(0, 10) == 0 and f(3, 0) == 0
     assert f(3, 1200) == 3 and f(1, 10_000_000) == 1 and f(16, 10_000) == 16
-    assert f(16, 100_000) == 4                                   # four chunks of four sequences
+    assert f(16, 100_000) == 6                                   # three chunks: 6, 6 and 4 sequences
     for B, T in ((5, 200_000), (3, 300_000), (32, 17_984), (16, 1_000_000), (7, 123_457), (1000, 1000)):
         Bc = f(B, T)
         nc = (B + Bc - 1) // Bc
         assert 1 <= Bc <= B and nc <= 8
         if nc > 1:
-            assert Bc * T >= 196_608                             # no chunk (but the last) shorter than half the target
+            assert Bc * T >= 262_144                             # no chunk (but the last) shorter than half the target
