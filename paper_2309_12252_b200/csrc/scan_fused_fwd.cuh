@@ -83,7 +83,7 @@ template <int N> struct FusedFwd {
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
     // apply kernel
     static constexpr int ROWS = 16;                    // chains per warp
-    static constexpr int A_WARPS = 2, A_THREADS = 64, A_STAGES = 4;
+    static constexpr int A_WARPS = 3, A_THREADS = 96, A_STAGES = 2;   // two CTAs per SM at n = 32: six warps, each one step ahead of itself
     static constexpr int ROW_FLOATS = 6 * N + 4;       // coefficient rows [N][4], r [N], y_old [N]; the pad keeps the
                                                        // 128-bit coefficient reads of a quarter-warp in distinct banks
     static constexpr int STAGE_A = ROWS * ROW_FLOATS;
