@@ -482,20 +482,34 @@ __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kerne
         float *yp[2] = {a.y + e_lo * N + 2 * t, a.y + e_hi * N + 2 * t};
         const int lens[2] = {len_lo, len_hi};
 
-        // one step into ring stage (it0 + s) % S: the two lanes of a row (l, l + 16) copy alternate 16-byte
-        // pieces of the row's coefficient record, residual and previous iterate (always one commit group)
-        const int hsel = lane >> 4;
-        const float *pc = a.J + e0 * 4 * N + 4 * hsel, *pr = a.b + e0 * N + 4 * hsel, *po = a.yold + e0 * N + 4 * hsel;
+        // one step into ring stage (it0 + s) % S (always one commit group).  Eight lanes copy 128 contiguous bytes of a
+        // row, so a warp instruction covers four rows with one full line each: lane l serves the rows 4k + (l >> 3),
+        // k = 0 .. 3, whose chain starts and lengths it fetches from the lanes that own them
+        const int rsub = lane >> 3, cpos = 4 * (lane & 7);
+        unsigned long long e0q[4];
+        int lenq[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            e0q[k] = __shfl_sync(0xffffffffu, (unsigned long long)e0, 4 * k + rsub);
+            lenq[k] = __shfl_sync(0xffffffffu, len, 4 * k + rsub);
+        }
         auto issue = [&](int s) {
-            if (s < len) {
-                float *dst = ring + ((it0 + (unsigned)s) % S) * C::STAGE_A + row * RF + 4 * hsel;
-                const float *sc = pc + (size_t)s * 4 * N, *sr = pr + (size_t)s * N, *so = po + (size_t)s * N;
+            float *stg_dst = ring + ((it0 + (unsigned)s) % S) * C::STAGE_A + rsub * RF + cpos;
 #pragma unroll
-                for (int u = 0; u < N / 2; ++u) cp_async16(dst + 8 * u, sc + 8 * u);
+            for (int k = 0; k < 4; ++k) {
+                if (s < lenq[k]) {
+                    float *dst = stg_dst + 4 * k * RF;
+                    const size_t e = (size_t)e0q[k] + (size_t)s;
+                    const float *sc = a.J + e * 4 * N + cpos, *sr = a.b + e * N + cpos, *so = a.yold + e * N + cpos;
 #pragma unroll
-                for (int u = 0; u < N / 8; ++u) {
-                    cp_async16(dst + 4 * N + 8 * u, sr + 8 * u);
-                    cp_async16(dst + 5 * N + 8 * u, so + 8 * u);
+                    for (int j = 0; j < N / 8; ++j) cp_async16(dst + 32 * j, sc + 32 * j);
+#pragma unroll
+                    for (int j = 0; j < (N + 31) / 32; ++j) {
+                        if (N >= 32 || cpos < N) {
+                            cp_async16(dst + 4 * N + 32 * j, sr + 32 * j);
+                            cp_async16(dst + 5 * N + 32 * j, so + 32 * j);
+                        }
+                    }
                 }
             }
             cp_async_commit();
