@@ -1130,7 +1130,14 @@ static int gru_vjp_impl(const deer_gru_params *p, const float *x, const float *y
         if (n3 <= 32 && wa.K <= 8) {
             DEER_KERNEL("wgrad_small_kernel", st, wgrad_small_kernel<<<P, 256, 0, st>>>(wa));
         } else if (n3 <= 192) {
-            DEER_KERNEL("wgrad_mma_kernel", st, wgrad_mma_kernel<<<dim3(P, (wa.K + 63) / 64), 32 * ((n3 + 15) / 16), 0, st>>>(wa));
+            const bool aligned16 = ((((uintptr_t)wa.dG | (uintptr_t)wa.V | (uintptr_t)wa.y0) & 15) == 0) && n3 % 4 == 0 && wa.K % 4 == 0;
+            if (aligned16) {
+                const size_t sm = wgrad_staged_smem(n3);
+                if ((rc = opt_in_smem((const void *)wgrad_mma_staged_kernel, sm)) != DEER_OK) return rc;
+                DEER_KERNEL("wgrad_mma_kernel", st, wgrad_mma_staged_kernel<<<dim3(P, (wa.K + 63) / 64), 32 * ((n3 + 15) / 16), sm, st>>>(wa));
+            } else {
+                DEER_KERNEL("wgrad_mma_kernel", st, wgrad_mma_kernel<<<dim3(P, (wa.K + 63) / 64), 32 * ((n3 + 15) / 16), 0, st>>>(wa));
+            }
         } else {
             int tile = 32;
             while (tile > 1 && sizeof(float) * tile * (size_t)(n3 + wa.K + 1) > 160 * 1024) tile >>= 1;

@@ -157,6 +157,129 @@ __global__ void __launch_bounds__(384) wgrad_mma_kernel(WgradArgs a)
     }
 }
 
+// The same reduction with both operands staged through shared memory: the tiles of dG (WG_S positions x n3, one
+// contiguous block) and of V (WG_S rows of the chunk's columns) arrive by 16-byte asynchronous copies in which
+// consecutive lanes copy consecutive pieces -- full lines per instruction, where the direct 4-byte fragment loads above
+// touch four rows with one sector each -- in a ring of WG_STAGES stages; the fragments are then read from shared memory
+// (row strides = 8 mod 32 words: conflict-free).  Needs n3 % 4 == 0, K % 4 == 0 and 16-byte aligned operands.
+constexpr int WG_S = 16, WG_STAGES = 3, WG_VS = 72;
+__host__ __device__ inline int wgrad_gs(int n3) { return n3 + ((8 - n3 % 32) + 32) % 32; }
+inline size_t wgrad_staged_smem(int n3) { return sizeof(float) * WG_STAGES * WG_S * (size_t)(wgrad_gs(n3) + WG_VS); }
+
+__global__ void __launch_bounds__(384) wgrad_mma_staged_kernel(WgradArgs a)
+{
+    extern __shared__ __align__(16) float wg_sm[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
+    const int g = lane >> 2, t = lane & 3;
+    const int n3 = a.n3, K = a.K, K1 = K + 1;
+    const int GS = wgrad_gs(n3);
+    const int kb = 64 * blockIdx.y;
+    const int kc = min(64, K - kb);                    // columns of this chunk (a multiple of 4)
+    const int nb = (kc + 7) >> 3;
+    const size_t e0 = (size_t)blockIdx.x * a.slice;
+    const size_t e1 = e0 + a.slice < a.N ? e0 + a.slice : a.N;
+    const int nst = e1 > e0 ? (int)((e1 - e0 + WG_S - 1) / WG_S) : 0;
+    float acc[8][4];
+#pragma unroll
+    for (int nn = 0; nn < 8; ++nn)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nn][i] = 0.0f;
+    float bs0 = 0.0f, bs1 = 0.0f;
+    const int row = 16 * warp + g;
+    const bool rv0 = row < n3, rv1 = row + 8 < n3;
+    const int gq = n3 >> 2, vq = kc >> 2;              // 16-byte pieces per row of the two tiles
+    auto issue = [&](int s) {
+        if (s < nst) {
+            float *sG = wg_sm + (size_t)(s % WG_STAGES) * WG_S * (GS + WG_VS), *sV = sG + WG_S * GS;
+            const size_t pb = e0 + (size_t)s * WG_S;
+            for (int c = tid; c < WG_S * gq; c += nthr) {
+                const int r = c / gq, cc = c - r * gq;
+                float *dst = sG + r * GS + 4 * cc;
+                if (pb + r < e1) cp_async16(dst, a.dG + (pb + r) * n3 + 4 * cc);
+                else *reinterpret_cast<float4 *>(dst) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            }
+            for (int c = tid; c < WG_S * vq; c += nthr) {
+                const int r = c / vq, cc = c - r * vq;
+                float *dst = sV + r * WG_VS + 4 * cc;
+                const size_t e = pb + r;
+                if (e < e1) {
+                    const float *src = a.V + e * K;
+                    if (a.shifted) {
+                        size_t seq;
+                        src = seq_start(e, a.T, seq) ? a.y0 + seq * K : a.V + (e - 1) * K;
+                    }
+                    cp_async16(dst, src + kb + 4 * cc);
+                } else {
+                    *reinterpret_cast<float4 *>(dst) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                }
+            }
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int s = 0; s < WG_STAGES - 1; ++s) issue(s);
+#pragma unroll 1
+    for (int s = 0; s < nst; ++s) {
+        static_assert(WG_STAGES == 3, "the wait below leaves one group in flight");
+        cp_async_wait_1();
+        __syncthreads();                   // stage s landed for every thread; the stage of step s - 1 is free again
+        issue(s + WG_STAGES - 1);
+        const float *sG = wg_sm + (size_t)(s % WG_STAGES) * WG_S * (GS + WG_VS), *sV = sG + WG_S * GS;
+#pragma unroll
+        for (int sub = 0; sub < WG_S / 8; ++sub) {
+            const float *g0 = sG + (8 * sub + t) * GS + row, *g1 = g0 + 4 * GS;
+            float av[4];
+            av[0] = rv0 ? g0[0] : 0.0f;
+            av[1] = rv1 ? g0[8] : 0.0f;
+            av[2] = rv0 ? g1[0] : 0.0f;
+            av[3] = rv1 ? g1[8] : 0.0f;
+            bs0 += av[0] + av[2];
+            bs1 += av[1] + av[3];
+            unsigned ah[4], al[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) split_tf32(av[i], ah[i], al[i]);
+            const float *v0 = sV + (8 * sub + t) * WG_VS + g, *v1 = v0 + 4 * WG_VS;
+#pragma unroll
+            for (int nn = 0; nn < 8; ++nn) {
+                if (nn < nb) {
+                    const bool cv = 8 * nn + g < kc;
+                    unsigned bh[2], bl[2];
+                    split_tf32(cv ? v0[8 * nn] : 0.0f, bh[0], bl[0]);
+                    split_tf32(cv ? v1[8 * nn] : 0.0f, bh[1], bl[1]);
+                    mma_tf32(acc[nn], al, bh, acc[nn]);
+                    mma_tf32(acc[nn], ah, bl, acc[nn]);
+                    mma_tf32(acc[nn], ah, bh, acc[nn]);
+                }
+            }
+        }
+    }
+    cp_async_wait_0();
+    float *out = a.partial + (size_t)blockIdx.x * n3 * K1;
+#pragma unroll
+    for (int nn = 0; nn < 8; ++nn) {
+        if (nn < nb) {
+            const int col = kb + 8 * nn + 2 * t;
+            if (col < K) {
+                if (rv0) out[row * K1 + col] = acc[nn][0];
+                if (rv1) out[(row + 8) * K1 + col] = acc[nn][2];
+            }
+            if (col + 1 < K) {
+                if (rv0) out[row * K1 + col + 1] = acc[nn][1];
+                if (rv1) out[(row + 8) * K1 + col + 1] = acc[nn][3];
+            }
+        }
+    }
+    if (blockIdx.y != 0) return;
+    bs0 += __shfl_xor_sync(0xffffffffu, bs0, 1);
+    bs0 += __shfl_xor_sync(0xffffffffu, bs0, 2);
+    bs1 += __shfl_xor_sync(0xffffffffu, bs1, 1);
+    bs1 += __shfl_xor_sync(0xffffffffu, bs1, 2);
+    if (t == 0) {
+        if (rv0) out[row * K1 + K] = bs0;
+        if (rv1) out[(row + 8) * K1 + K] = bs1;
+    }
+}
+
 // ------------------------------------------------------------------ a0 / a8: dense affine map on tensor cores
 //   out[e][c] = bias[c] + sum_k W(c,k) in[e][k],   W(c,k) = W[c*K + k]  (weights [out][in], the input
 //   projection u = x W_i^T + b_i)  or  W[k*NOUT + c]  (WT_GIVEN: weights [in][out], dx = dG_i W_i).
