@@ -319,11 +319,17 @@ __global__ void __launch_bounds__(256) affine_mma_kernel(const float *__restrict
             acc[nn][0] = b0; acc[nn][1] = b1; acc[nn][2] = b0; acc[nn][3] = b1;
         }
         const float *a0p = in + (v0 ? r0 : 0) * K + 2 * t, *a1p = in + (v1 ? r1 : 0) * K + 2 * t;
+        // the A values of the next K step are requested before the products of the current one
+        float2 xn0 = v0 ? __ldg(reinterpret_cast<const float2 *>(a0p)) : make_float2(0.f, 0.f);
+        float2 xn1 = v1 ? __ldg(reinterpret_cast<const float2 *>(a1p)) : make_float2(0.f, 0.f);
 #pragma unroll 1
         for (int k0 = 0; k0 < K; k0 += 8) {
             // slots t and t+4 of the K step hold k0+2t and k0+2t+1
-            const float2 x0 = v0 ? __ldg(reinterpret_cast<const float2 *>(a0p + k0)) : make_float2(0.f, 0.f);
-            const float2 x1 = v1 ? __ldg(reinterpret_cast<const float2 *>(a1p + k0)) : make_float2(0.f, 0.f);
+            const float2 x0 = xn0, x1 = xn1;
+            if (k0 + 8 < K) {
+                if (v0) xn0 = __ldg(reinterpret_cast<const float2 *>(a0p + k0 + 8));
+                if (v1) xn1 = __ldg(reinterpret_cast<const float2 *>(a1p + k0 + 8));
+            }
             unsigned ah[4], al[4];
             split_tf32(x0.x, ah[0], al[0]);      // a0: (row g,   slot t)
             split_tf32(x1.x, ah[1], al[1]);      // a1: (row g+8, slot t)
