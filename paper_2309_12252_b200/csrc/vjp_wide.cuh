@@ -372,30 +372,35 @@ __global__ void __launch_bounds__(256, 2) cell_coef_mma_kernel(CellArgs a)
 {
     pdl_prologue();
     if (loop_ended(a.st)) return;
-    constexpr int NOUT = 3 * N, NB = NOUT / 8, NBG = N / 8, NS = NOUT + 4;      // 2 * NS = 8 (mod 32) words
+    constexpr int NOUT = 3 * N, NB = NOUT / 8, NBG = N / 8;
+    // B operands in shared memory as one 16-byte record per (pair of contraction rows, column):
+    // {hi(W[2p][c]), hi(W[2p+1][c]), lo(W[2p][c]), lo(W[2p+1][c])} -- the four words a lane needs for one column block of
+    // one K step, fetched by ONE 128-bit load; row stride NSQ = 2 (mod 8) records: the eight lanes of a quarter-warp
+    // (two columns x four row pairs) read distinct bank groups
+    constexpr int NSQ = NOUT + 2;
     extern __shared__ __align__(16) float smw[];
-    float *sBh = smw, *sBl = smw + N * NS, *sb = sBl + N * NS;
+    float4 *sQ = reinterpret_cast<float4 *>(smw);
+    float *sb = smw + 4 * (N / 2) * NSQ;
     // PROJ: the input projection is part of the same contraction ([B*T, m] x [m, 3n] with W_i^T, also 3 x TF32), so
     // neither a u buffer nor a projection pass exists: the r and z halves add into the hidden products' accumulators,
     // the candidate's input part keeps accumulators of its own (c = tanh(u_n + r q) needs the two apart).  Only with
     // the residual form (rhs = f - y), which does not need the bias-free hidden products.
     const int m = PROJ ? a.m : 0;
-    float *sIh = sb + 2 * NOUT, *sIl = sIh + m * NS;
+    float4 *sQi = reinterpret_cast<float4 *>(sb + 2 * NOUT);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
-    for (int idx = tid; idx < N * NOUT; idx += 256) {
-        const int k = idx / NOUT, c = idx % NOUT;
-        const float v = a.W_h[(size_t)c * N + k];
-        sBh[k * NS + c] = v;
-        sBl[k * NS + c] = v - __uint_as_float(__float_as_uint(v) & 0xffffe000u);
+    auto tf32_lo = [](float v) { return v - __uint_as_float(__float_as_uint(v) & 0xffffe000u); };
+    for (int idx = tid; idx < (N / 2) * NOUT; idx += 256) {
+        const int kp = idx / NOUT, c = idx % NOUT;
+        const float v0 = a.W_h[(size_t)c * N + 2 * kp], v1 = a.W_h[(size_t)c * N + 2 * kp + 1];
+        sQ[kp * NSQ + c] = make_float4(v0, v1, tf32_lo(v0), tf32_lo(v1));
     }
     for (int idx = tid; idx < NOUT; idx += 256) { sb[idx] = a.b_h[idx]; sb[NOUT + idx] = PROJ ? a.b_i[idx] : 0.0f; }
     if constexpr (PROJ) {
-        for (int idx = tid; idx < m * NOUT; idx += 256) {
-            const int k = idx / NOUT, c = idx % NOUT;
-            const float v = a.W_i[(size_t)c * m + k];
-            sIh[k * NS + c] = v;
-            sIl[k * NS + c] = v - __uint_as_float(__float_as_uint(v) & 0xffffe000u);
+        for (int idx = tid; idx < (m / 2) * NOUT; idx += 256) {
+            const int kp = idx / NOUT, c = idx % NOUT;
+            const float v0 = a.W_i[(size_t)c * m + 2 * kp], v1 = a.W_i[(size_t)c * m + 2 * kp + 1];
+            sQi[kp * NSQ + c] = make_float4(v0, v1, tf32_lo(v0), tf32_lo(v1));
         }
     }
     __syncthreads();
@@ -430,12 +435,11 @@ __global__ void __launch_bounds__(256, 2) cell_coef_mma_kernel(CellArgs a)
             split_tf32(x1.x, ah[1], al[1]);
             split_tf32(x0.y, ah[2], al[2]);
             split_tf32(x1.y, ah[3], al[3]);
-            const float *bh0 = sBh + (k0 + 2 * t) * NS + g, *bl0 = sBl + (k0 + 2 * t) * NS + g;
+            const float4 *q0 = sQ + (k0 / 2 + t) * NSQ + g;
 #pragma unroll
             for (int nn = 0; nn < NB; ++nn) {
-                unsigned bh[2], bl[2];
-                bh[0] = __float_as_uint(bh0[8 * nn]); bh[1] = __float_as_uint(bh0[8 * nn + NS]);
-                bl[0] = __float_as_uint(bl0[8 * nn]); bl[1] = __float_as_uint(bl0[8 * nn + NS]);
+                const float4 q = q0[8 * nn];
+                const unsigned bh[2] = {__float_as_uint(q.x), __float_as_uint(q.y)}, bl[2] = {__float_as_uint(q.z), __float_as_uint(q.w)};
                 mma_tf32(acc[nn], al, bh, acc[nn]);
                 mma_tf32(acc[nn], ah, bl, acc[nn]);
                 mma_tf32(acc[nn], ah, bh, acc[nn]);
@@ -452,12 +456,11 @@ __global__ void __launch_bounds__(256, 2) cell_coef_mma_kernel(CellArgs a)
                 split_tf32(x1.x, ah[1], al[1]);
                 split_tf32(x0.y, ah[2], al[2]);
                 split_tf32(x1.y, ah[3], al[3]);
-                const float *bh0 = sIh + (k0 + 2 * t) * NS + g, *bl0 = sIl + (k0 + 2 * t) * NS + g;
+                const float4 *q0 = sQi + (k0 / 2 + t) * NSQ + g;
 #pragma unroll
                 for (int nn = 0; nn < NB; ++nn) {
-                    unsigned bh[2], bl[2];
-                    bh[0] = __float_as_uint(bh0[8 * nn]); bh[1] = __float_as_uint(bh0[8 * nn + NS]);
-                    bl[0] = __float_as_uint(bl0[8 * nn]); bl[1] = __float_as_uint(bl0[8 * nn + NS]);
+                    const float4 q = q0[8 * nn];
+                    const unsigned bh[2] = {__float_as_uint(q.x), __float_as_uint(q.y)}, bl[2] = {__float_as_uint(q.z), __float_as_uint(q.w)};
                     float (&dst)[4] = nn < 2 * NBG ? acc[nn] : accn[nn - 2 * NBG];
                     mma_tf32(dst, al, bh, dst);
                     mma_tf32(dst, ah, bl, dst);
