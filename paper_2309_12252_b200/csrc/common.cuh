@@ -245,18 +245,12 @@ __device__ __forceinline__ unsigned absdiff_bits(float a, float b) {
     return __float_as_uint(fabsf(a - b));   // NaN keeps bits above +inf: an integer max propagates it
 }
 
-// 256-bit global accesses (sm_100): one request per 32 contiguous bytes of a lane; the address must be 32-byte aligned
+// 256-bit global store (sm_100): one request per 32 contiguous bytes of a lane; the address must be 32-byte aligned
 __device__ __forceinline__ void st_global_v8(float *p, const float4 &a, const float4 &b)
 {
     asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "f"(a.x), "f"(a.y), "f"(a.z), "f"(a.w),
                  "f"(b.x), "f"(b.y), "f"(b.z), "f"(b.w)
                  : "memory");
-}
-__device__ __forceinline__ void ld_global_nc_v8(const float *p, float (&v)[8])
-{
-    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
-                 : "l"(p));
 }
 
 static inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
