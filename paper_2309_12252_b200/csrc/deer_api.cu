@@ -342,19 +342,19 @@ static int launch_fused_fwd64(ScanArgs a, OnePassWs w, bool prep, cudaStream_t s
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= MAX_DEVICES) dev = 0;
     if (!occ_apply[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(scan_fused_apply_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::A_SMEM);
+        cudaError_t e = cudaFuncSetAttribute(scan_fused_apply64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::P_SMEM);
         if (e != cudaSuccess) { set_error(e, "cudaFuncSetAttribute(scan apply)"); return DEER_ERR_CUDA; }
         int o = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, scan_fused_apply_kernel<64>, C::A_THREADS, C::A_SMEM);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, scan_fused_apply64_kernel, C::P_THREADS, C::P_SMEM);
         if (e != cudaSuccess || o < 1) { set_error(e, "occupancy(scan apply)"); return DEER_ERR_CUDA; }
         occ_apply[dev] = o;
     }
     const long long nchain = (a.T + w.sw - 1) / w.sw;
     const long long groups = ((long long)a.B * nchain + C::ROWS - 1) / C::ROWS;
-    const long long want = (groups + C::A_WARPS - 1) / C::A_WARPS;
+    const long long want = (groups + C::P_PAIRS - 1) / C::P_PAIRS;
     const long long resident = (long long)num_sms() * occ_apply[dev];
     const unsigned grid = (unsigned)(want < resident ? want : resident);
-    DEER_KERNEL_PDL("scan_fused_apply_kernel", false, st, scan_fused_apply_kernel<64>, grid, (unsigned)C::A_THREADS, C::A_SMEM, a, w);
+    DEER_KERNEL_PDL("scan_fused_apply_kernel", false, st, scan_fused_apply64_kernel, grid, (unsigned)C::P_THREADS, C::P_SMEM, a, w);
     return DEER_OK;
 }
 

@@ -87,7 +87,6 @@ template <int N> struct FusedFwd {
     static constexpr int ROW_FLOATS = 6 * N + 4;       // coefficient rows [N][4], r [N], y_old [N]; the pad keeps the
                                                        // 128-bit coefficient reads of a quarter-warp in distinct banks
     static constexpr int STAGE_A = ROWS * ROW_FLOATS;
-    static constexpr bool W_SMEM = false;              // the apply kernel keeps its share of W_h^T in registers
     static constexpr size_t A_SMEM = sizeof(float) * (A_WARPS * A_STAGES * STAGE_A + A_WARPS * ROWS * N) + 128;
 };
 
@@ -379,10 +378,10 @@ __global__ void __launch_bounds__(FusedFwd<N>::THREADS, FusedFwd<N>::R_CTAS) sca
 template <int N>
 __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kernel(ScanArgs a, OnePassWs w)
 {
+    static_assert(N == 16 || N == 32, "n = 64 has a replay kernel of its own (scan_fused_fwd64.cuh)");
     using C = FusedFwd<N>;
     constexpr int NN = C::NN, AGG = C::AGG, NT = C::NT, ROWS = C::ROWS, RF = C::ROW_FLOATS, S = C::A_STAGES;
     constexpr int WA = C::WARPS;                       // chains per tile of the reduce kernel
-    constexpr bool WSM = C::W_SMEM;                    // B operand (W_h^T) from shared memory instead of registers
     pdl_prologue();
     if (loop_ended(a.st)) return;
 
@@ -392,25 +391,16 @@ __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kerne
     const int g = lane >> 2, t = lane & 3;
     float *ring = sm + warp * S * C::STAGE_A;
     float *yin = sm + C::A_WARPS * S * C::STAGE_A + warp * ROWS * N;
-    float2 *sWf = reinterpret_cast<float2 *>(sm + C::A_WARPS * S * C::STAGE_A + C::A_WARPS * ROWS * N);   // [kk][nn][lane]
 
     // B operand of every step: W_h^T, contraction index renamed so that an accumulator fragment is the next A operand
-    unsigned wf[WSM ? 1 : NT][WSM ? 1 : 3 * NT][2];
-    if constexpr (WSM) {
-        for (int idx = tid; idx < NT * 3 * NT * 32; idx += C::A_THREADS) {
-            const int l = idx & 31, nn = (idx >> 5) % (3 * NT), kk = (idx >> 5) / (3 * NT);
-            sWf[idx] = __ldg(reinterpret_cast<const float2 *>(a.Wh + (size_t)(8 * nn + (l >> 2)) * N + 8 * kk + 2 * (l & 3)));
+    unsigned wf[NT][3 * NT][2];
+#pragma unroll
+    for (int kk = 0; kk < NT; ++kk)
+#pragma unroll
+        for (int nn = 0; nn < 3 * NT; ++nn) {
+            const float2 v = __ldg(reinterpret_cast<const float2 *>(a.Wh + (size_t)(8 * nn + g) * N + 8 * kk + 2 * t));
+            wf[kk][nn][0] = __float_as_uint(v.x); wf[kk][nn][1] = __float_as_uint(v.y);
         }
-        __syncthreads();
-    } else {
-#pragma unroll
-        for (int kk = 0; kk < NT; ++kk)
-#pragma unroll
-            for (int nn = 0; nn < 3 * NT; ++nn) {
-                const float2 v = __ldg(reinterpret_cast<const float2 *>(a.Wh + (size_t)(8 * nn + g) * N + 8 * kk + 2 * t));
-                wf[kk][nn][0] = __float_as_uint(v.x); wf[kk][nn][1] = __float_as_uint(v.y);
-            }
-    }
 
     const int T = a.T, SW = w.sw;
     const long long nchain = (T + SW - 1) / SW;
@@ -439,10 +429,7 @@ __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kerne
             const int vr = __shfl_sync(0xffffffffu, (int)rv, r);
             const unsigned long long tix = __shfl_sync(0xffffffffu, (unsigned long long)tile_index, r);
             const int kr = __shfl_sync(0xffffffffu, kin, r);
-            if constexpr (WA == 1) {
-                for (int c = lane; c < N; c += 32)
-                    yin[r * N + c] = vr ? __uint_as_float((unsigned)(ld_relaxed_u64(w.starts + tix * N + c) & 0xffffffffull)) : 0.0f;
-            } else {
+            {
                 float val = 0.0f;
                 if (vr) {
                     float yl = 0.0f;
@@ -532,15 +519,7 @@ __global__ void __launch_bounds__(FusedFwd<N>::A_THREADS) scan_fused_apply_kerne
                 const unsigned af[4] = {__float_as_uint(d[kk][0]), __float_as_uint(d[kk][2]), __float_as_uint(d[kk][1]),
                                         __float_as_uint(d[kk][3])};
 #pragma unroll
-                for (int nn = 0; nn < 3 * NT; ++nn) {
-                    if constexpr (WSM) {
-                        const float2 b2 = sWf[(kk * 3 * NT + nn) * 32 + lane];
-                        const unsigned bf[2] = {__float_as_uint(b2.x), __float_as_uint(b2.y)};
-                        mma_tf32(U[nn], af, bf, U[nn]);
-                    } else {
-                        mma_tf32(U[nn], af, wf[kk][nn], U[nn]);
-                    }
-                }
+                for (int nn = 0; nn < 3 * NT; ++nn) mma_tf32(U[nn], af, wf[kk][nn], U[nn]);
             }
             const float *st = ring + stg * C::STAGE_A;
 #pragma unroll
