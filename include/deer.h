@@ -217,8 +217,8 @@ int deer_gru_eval_diag(const deer_gru_params *params, const float *x, const floa
 /* deer_gru_eval with the sequence data in HOST memory (the end-to-end call):
  * copies x_host to x_dev, evaluates into y_dev as deer_gru_eval does, copies
  * the result to y_host (asynchronously when the host buffers are page-locked).
- * A batch of more than deer_gru_eval_host_chunk(B, T) sequences is evaluated
- * in chunks of that many sequences, each with its own Newton loop (sequences
+ * A batch that deer_gru_eval_host_chunks(B, T, ...) splits is evaluated
+ * chunk by chunk, each chunk with its own Newton loop (sequences
  * are independent: the batch is a map over sequences, Sec. 3), so that on
  * copy streams owned by the library chunk c + 1 arrives and chunk c - 1
  * leaves while chunk c is evaluated; each chunk's result is exactly what
@@ -238,10 +238,17 @@ int deer_gru_eval_host(const deer_gru_params *params, const float *x_host, const
                        float tol, int max_iter, float *y_host, int *iters, float *err, float *x_dev,
                        float *y_dev, void *ws, size_t ws_bytes, int flags, void *stream);
 
-/* Sequences per chunk of deer_gru_eval_host for a batch of B sequences of
- * length T (B when the batch is not split; at most DEER_HOST_MAX_CHUNKS
- * chunks).  Host only; 0 for invalid sizes. */
+/* The chunks of deer_gru_eval_host for a batch of B sequences of length T:
+ * returns their number nc (1 when the batch is not split, at most
+ * DEER_HOST_MAX_CHUNKS; 0 for invalid sizes) and, when `first` is not NULL
+ * (host, room for DEER_HOST_MAX_CHUNKS + 1 entries), writes the first
+ * sequence of every chunk and B itself to first[0 .. nc].  Chunks hold about
+ * 2^19 positions; from three chunks on the first and the last are about half
+ * as long as the others, because their copies are the two that no evaluation
+ * hides.  deer_gru_eval_host_chunk returns the largest chunk's sequence
+ * count.  Host only. */
 #define DEER_HOST_MAX_CHUNKS 8
+int deer_gru_eval_host_chunks(int B, int T, int *first);
 int deer_gru_eval_host_chunk(int B, int T);
 
 /* Gradient through the evaluated sequence (Eq. 7): given gy = dL/dy at a

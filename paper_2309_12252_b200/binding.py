@@ -27,7 +27,7 @@ NOALLOC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ["deer_workspace_bytes", "deer_linrec_scan", "deer_linrec_scan_noalloc", "deer_gru_eval",
            "deer_gru_eval_diag", "deer_gru_eval_host", "deer_gru_vjp",
            "deer_gru_classifier_step", "deer_status_string", "deer_last_error", "deer_launch_count",
-           "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_eval_host_chunk", "deer_gru_cell_jac",
+           "deer_workspace_status", "deer_noalloc_status", "deer_scan_geometry", "deer_gru_eval_host_chunk", "deer_gru_eval_host_chunks", "deer_gru_cell_jac",
            "deer_multihead_workspace_bytes", "deer_gru_multihead_eval", "deer_gru_multihead_vjp", "deer_gru_jvp",
            "deer_ode_linear_solve", "deer_lstm_eval"]
 
@@ -89,6 +89,8 @@ def lib():
         L.deer_noalloc_status.argtypes = [vp]
         L.deer_gru_eval_host_chunk.restype = ci
         L.deer_gru_eval_host_chunk.argtypes = [ci, ci]
+        L.deer_gru_eval_host_chunks.restype = ci
+        L.deer_gru_eval_host_chunks.argtypes = [ci, ci, ctypes.POINTER(ci)]
         L.deer_scan_geometry.restype = ci
         L.deer_scan_geometry.argtypes = [ci, ci, ci, ci, ctypes.POINTER(ci)]
         L.deer_gru_cell_jac.restype = ci
@@ -217,8 +219,15 @@ def deer_noalloc_status(stream=None) -> int:
 
 
 def deer_gru_eval_host_chunk(B: int, T: int) -> int:
-    """Sequences per chunk of deer_gru_eval_host (B when the batch is not split)."""
+    """Sequences of the largest chunk of deer_gru_eval_host (B when the batch is not split)."""
     return int(lib().deer_gru_eval_host_chunk(int(B), int(T)))
+
+
+def deer_gru_eval_host_chunks(B: int, T: int) -> list:
+    """First sequence of every chunk of deer_gru_eval_host, then B: [0, ..., B] ([] for invalid sizes)."""
+    first = (ctypes.c_int * 9)()
+    nc = int(lib().deer_gru_eval_host_chunks(int(B), int(T), first))
+    return [int(first[k]) for k in range(nc + 1)] if nc > 0 else []
 
 
 def deer_scan_geometry(B: int, T: int, n: int, flags: int = 0) -> dict:

@@ -232,8 +232,8 @@ def test_eval_with_host_buffers_in_chunks_of_sequences(bd, n, m, B, T):
     """A batch that deer_gru_eval_host splits (copies of the neighbouring chunks overlap an evaluation): every chunk
     holds exactly what deer_gru_eval returns for those sequences alone, iters / err are the largest over the chunks, and
     the whole agrees with the unsplit device call within the tolerance the iteration is solved to."""
-    Bc = bd.deer_gru_eval_host_chunk(B, T)
-    assert 1 <= Bc < B
+    first = bd.deer_gru_eval_host_chunks(B, T)
+    assert len(first) >= 3 and first[0] == 0 and first[-1] == B
     p_np = synth.gru_params(n, m, 5, tag="hc/gru")
     x_np = synth.x_gaussian(B, T, m, 5, tag="hc/x")
     y0_np = (synth.normal(5, "hc/y0", (B, n)) * 0.3).astype(np.float32)
@@ -245,9 +245,9 @@ def test_eval_with_host_buffers_in_chunks_of_sequences(bd, n, m, B, T):
     r = bd.deer_gru_eval_host(p, x_host, dev(y0_np), y_host, x_dev, y_dev, ws)
     assert r.status == 0 and torch.equal(y_dev.cpu(), y_host)
     its, errs = [], []
-    for b0 in range(0, B, Bc):
-        rc = bd.deer_gru_eval(p, dev(x_np[b0:b0 + Bc]), dev(y0_np[b0:b0 + Bc]))
-        assert torch.equal(rc.y.cpu(), y_host[b0:b0 + Bc])
+    for b0, b1 in zip(first[:-1], first[1:]):
+        rc = bd.deer_gru_eval(p, dev(x_np[b0:b1]), dev(y0_np[b0:b1]))
+        assert torch.equal(rc.y.cpu(), y_host[b0:b1])
         its.append(rc.iters); errs.append(rc.err)
     assert r.iters == max(its) and r.err == max(errs)
     whole = bd.deer_gru_eval(p, dev(x_np), dev(y0_np))

@@ -85,15 +85,32 @@ def test_scan_geometry_bounds_the_resolver_ctas(L):
 
 
 def test_host_call_chunking_rule(L):
-    """deer_gru_eval_host splits a batch into chunks of whole sequences of about 2^19 positions, at most eight, and
-    leaves small batches and single sequences whole (host logic only)."""
+    """deer_gru_eval_host splits a batch into chunks of whole sequences of about 2^19 positions, at most eight, the
+    first and the last about half as long as the others from three chunks on, and leaves small batches and single
+    sequences whole (host logic only)."""
+    import ctypes
     f = L.deer_gru_eval_host_chunk
-    assert f(0, 10) == 0 and f(3, 0) == 0
+    fs = L.deer_gru_eval_host_chunks
+    fs.restype = ctypes.c_int
+    fs.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+
+    def chunks(B, T):
+        first = (ctypes.c_int * 9)()
+        nc = fs(B, T, first)
+        return [first[k] for k in range(nc + 1)] if nc else []
+
+    assert f(0, 10) == 0 and f(3, 0) == 0 and fs(0, 10, None) == 0 and fs(3, 0, None) == 0
     assert f(3, 1200) == 3 and f(1, 10_000_000) == 1 and f(16, 10_000) == 16
-    assert f(16, 100_000) == 6                                   # three chunks: 6, 6 and 4 sequences
-    for B, T in ((5, 200_000), (3, 300_000), (32, 17_984), (16, 1_000_000), (7, 123_457), (1000, 1000)):
-        Bc = f(B, T)
-        nc = (B + Bc - 1) // Bc
-        assert 1 <= Bc <= B and nc <= 8
-        if nc > 1:
-            assert Bc * T >= 262_144                             # no chunk (but the last) shorter than half the target
+    assert chunks(3, 1200) == [0, 3] and chunks(16, 10_000) == [0, 16] and fs(16, 100_000, None) == 3
+    assert chunks(16, 100_000) == [0, 4, 12, 16] and f(16, 100_000) == 8      # three chunks: 4, 8 and 4 sequences
+    assert chunks(2, 600_000) == [0, 1, 2] and chunks(3, 600_000) == [0, 1, 2, 3]
+    for B, T in ((5, 200_000), (3, 300_000), (32, 17_984), (16, 1_000_000), (7, 123_457), (1000, 1000), (9, 2_000_000)):
+        first = chunks(B, T)
+        nc = len(first) - 1
+        sizes = [b - a for a, b in zip(first[:-1], first[1:])]
+        assert 1 <= nc <= 8 and first[0] == 0 and first[-1] == B and min(sizes) >= 1
+        assert f(B, T) == max(sizes)
+        if nc >= 3:                                                  # the edges are the short ones
+            assert max(sizes[0], sizes[-1]) <= min(sizes[1:-1]) and min(sizes[0], sizes[-1]) * 2 + 1 >= max(sizes[1:-1]) - 1
+        if nc == 2:
+            assert abs(sizes[0] - sizes[1]) <= 1
