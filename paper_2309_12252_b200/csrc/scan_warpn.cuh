@@ -44,7 +44,7 @@ template <int N> struct WarpN {
     static constexpr int PEND = (WARPS - 1) * AGG;     // warp aggregates kept for the B item (the last warp's
                                                        // is only needed by the tile combine: it sits in that warp's ring)
     static constexpr int SM_WORK = Q * PEND + WARPS * N + N + 16 + WARPS * STAGES * STAGE_FLOATS;
-    static constexpr int SM_RES = RES_SLOTS * AGG;
+    static constexpr int SM_RES = RES_SLOTS * AGG + RES_WARPS * N;   // tile slots, then a state vector per resolving warp
     static constexpr int SM_FLOATS = SM_WORK > SM_RES ? SM_WORK : SM_RES;
     static constexpr size_t SMEM = SM_FLOATS * sizeof(float) + 128;
     static constexpr int MAX_SEQ_PER_WARP = 8;
@@ -68,24 +68,35 @@ __device__ __forceinline__ void resolver_big_fetch(float *dst, const float *src,
     cp_async_commit();
 }
 
-// the walk over `cnt` staged aggregates; out: the tiles' entering-state words
+// the walk over `cnt` staged aggregates; out: the tiles' entering-state words.  Lane i owns component i of the state
+// and row i of A; the state goes through a vector in shared memory (ybuf) so that a row and the state are read as
+// 16-byte pieces -- 2 x n/4 loads and n FMAs per tile where a shuffle per element took three times the instructions --
+// each lane starting at a different piece (the eight lanes of a 128-bit access phase then hit distinct banks).
 template <int N>
-__device__ __forceinline__ float resolver_big_walk(const float *stage, int cnt, unsigned long long *out, float y, int lane)
+__device__ __forceinline__ float resolver_big_walk(const float *stage, int cnt, unsigned long long *out, float y, float *ybuf, int lane)
 {
-    constexpr int AGG = WarpN<N>::AGG, NN = WarpN<N>::NN;
+    constexpr int AGG = WarpN<N>::AGG, NN = WarpN<N>::NN, CH = N / 4;
+    const int sw = (N == 32) ? (lane & 7) : ((lane >> 1) & 3);
+    const int rl = lane < N ? lane : 0;
+    const float4 *yb = reinterpret_cast<const float4 *>(ybuf);
     for (int q = 0; q < cnt; ++q) {
-        if (lane < N) st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y));
-        const float *ag = stage + q * AGG;
-        float acc0 = (lane < N) ? ag[NN + lane] : 0.0f, acc1 = 0.0f;
-        const float *row = ag + (lane < N ? lane : 0) * N;
-#pragma unroll
-        for (int i = 0; i < N; i += 2) {       // skewed column order: conflict-free row reads
-            const int c0i = (i + lane) & (N - 1), c1i = (i + 1 + lane) & (N - 1);
-            const float y0 = __shfl_sync(0xffffffffu, y, c0i), y1 = __shfl_sync(0xffffffffu, y, c1i);
-            acc0 = fmaf(row[c0i], y0, acc0);
-            acc1 = fmaf(row[c1i], y1, acc1);
+        if (lane < N) {
+            st_relaxed_u64(out + q * N + lane, LL_FLAG | (unsigned long long)__float_as_uint(y));
+            ybuf[lane] = y;
         }
-        y = acc0 + acc1;
+        __syncwarp();
+        const float *ag = stage + q * AGG;
+        const float4 *row = reinterpret_cast<const float4 *>(ag + rl * N);
+        float a0 = (lane < N) ? ag[NN + lane] : 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+#pragma unroll
+        for (int k = 0; k < CH; ++k) {
+            const int kk = k ^ sw;
+            const float4 av = row[kk], yv = yb[kk];
+            a0 = fmaf(av.x, yv.x, a0); a1 = fmaf(av.y, yv.y, a1);
+            a2 = fmaf(av.z, yv.z, a2); a3 = fmaf(av.w, yv.w, a3);
+        }
+        y = (a0 + a1) + (a2 + a3);
+        __syncwarp();              // every lane has read the state before the next tile's is written
     }
     return y;
 }
@@ -98,6 +109,7 @@ __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage
     constexpr int AGG = C::AGG;
     const int RING = C::RES_SLOTS / w.res_warps;                           // this warp's tile slots (a power of two)
     float *stage = stage_all + (threadIdx.x >> 5) * RING * AGG;
+    float *ybuf = stage_all + C::RES_SLOTS * AGG + (threadIdx.x >> 5) * N;
     unsigned spins = 0;
     if (rw + nrw >= a.B) {
         // ---- one sequence: a ring of RING tile slots, up to four fetch groups in flight
@@ -137,8 +149,8 @@ __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage
                 __syncwarp();
                 const int cnt = gcnt[ghead];
                 const int s0 = c & (RING - 1), first = min(cnt, RING - s0);
-                y = resolver_big_walk<N>(stage + s0 * AGG, first, starts + (size_t)c * N, y, lane);
-                if (cnt > first) y = resolver_big_walk<N>(stage, cnt - first, starts + (size_t)(c + first) * N, y, lane);
+                y = resolver_big_walk<N>(stage + s0 * AGG, first, starts + (size_t)c * N, y, ybuf, lane);
+                if (cnt > first) y = resolver_big_walk<N>(stage, cnt - first, starts + (size_t)(c + first) * N, y, ybuf, lane);
                 __syncwarp();
                 if (lane < cnt) w.flags[(size_t)s * w.nch + c + lane] = 0u;   // consumed: cleared for the next launch
                 c += cnt;
@@ -189,7 +201,7 @@ __device__ void resolver_big(const ScanArgs &a, const OnePassWs &w, float *stage
             resolver_big_fetch<N>(stage, w.aggs + ((size_t)s * w.nch + c0) * AGG, cnt, lane);
             cp_async_wait_0();
             __syncwarp();
-            yv[k] = resolver_big_walk<N>(stage, cnt, w.starts + ((size_t)s * w.nch + c0) * N, yv[k], lane);
+            yv[k] = resolver_big_walk<N>(stage, cnt, w.starts + ((size_t)s * w.nch + c0) * N, yv[k], ybuf, lane);
             __syncwarp();
             if (lane < cnt) w.flags[(size_t)s * w.nch + c0 + lane] = 0u;   // consumed: cleared for the next launch
             pos[k] = c0 + cnt;
