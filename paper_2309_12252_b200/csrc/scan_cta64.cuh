@@ -47,15 +47,20 @@ __device__ __forceinline__ float2 resolver64_walk(const float *stage, float *ysm
     constexpr int N = 64, NN = N * N;
     ysm[lane] = y0v; ysm[32 + lane] = y1v;
     __syncwarp();
-    float a0 = stage[NN + lane], a1 = stage[NN + 32 + lane];
-    const float *r0 = stage + lane * N, *r1 = stage + (32 + lane) * N;
-#pragma unroll 8
-    for (int i = 0; i < N; ++i) {           // skewed column order: conflict-free reads
-        const int c = (i + lane) & (N - 1);
-        const float yc = ysm[c];
-        a0 = fmaf(r0[c], yc, a0);
-        a1 = fmaf(r1[c], yc, a1);
+    // rows lane and lane + 32 and the state as 16-byte pieces, each lane starting at a different piece (the eight lanes
+    // of a 128-bit access phase then hit distinct banks): a third of the instructions of the element-wise loop
+    const float4 *r0 = reinterpret_cast<const float4 *>(stage + lane * N), *r1 = reinterpret_cast<const float4 *>(stage + (32 + lane) * N);
+    const float4 *yb = reinterpret_cast<const float4 *>(ysm);
+    float a0 = stage[NN + lane], a1 = stage[NN + 32 + lane], b0 = 0.0f, b1 = 0.0f, c0 = 0.0f, c1 = 0.0f, d0 = 0.0f, d1 = 0.0f;
+#pragma unroll
+    for (int k = 0; k < N / 4; ++k) {
+        const int kk = k ^ (lane & 7);
+        const float4 yv = yb[kk], u = r0[kk], v = r1[kk];
+        a0 = fmaf(u.x, yv.x, a0); b0 = fmaf(u.y, yv.y, b0); c0 = fmaf(u.z, yv.z, c0); d0 = fmaf(u.w, yv.w, d0);
+        a1 = fmaf(v.x, yv.x, a1); b1 = fmaf(v.y, yv.y, b1); c1 = fmaf(v.z, yv.z, c1); d1 = fmaf(v.w, yv.w, d1);
     }
+    a0 = (a0 + b0) + (c0 + d0);
+    a1 = (a1 + b1) + (c1 + d1);
     __syncwarp();
     return make_float2(a0, a1);
 }
