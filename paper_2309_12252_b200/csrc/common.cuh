@@ -241,6 +241,37 @@ __device__ __forceinline__ float2 fmul2(float2 a, float2 b)
     return d;
 }
 
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b)
+{
+    unsigned long long ra, rb, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+__device__ __forceinline__ float ex2_approx(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float rcp_approx(float x) { float y; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+
+// The gate activations on a pair of values: the arithmetic around the two special-function-unit results (the scaling of
+// the exponent, 1 +- e, the final product) runs as packed f32x2 instructions; same approximate units as the scalar forms.
+__device__ __forceinline__ float2 sigmoid2_gate(float2 a)
+{
+    const float2 t = fmul2(a, make_float2(-1.4426950408889634f, -1.4426950408889634f));
+    const float2 d = fadd2(make_float2(ex2_approx(t.x), ex2_approx(t.y)), make_float2(1.0f, 1.0f));
+    return make_float2(rcp_approx(d.x), rcp_approx(d.y));
+}
+__device__ __forceinline__ float2 tanh2_gate(float2 a)
+{
+    const float2 t = fmul2(make_float2(fabsf(a.x), fabsf(a.y)), make_float2(-2.8853900817779268f, -2.8853900817779268f));
+    const float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));                     // exp(-2 |a|) in (0, 1]
+    const float2 one = make_float2(1.0f, 1.0f);
+    const float2 num = ffma2(e, make_float2(-1.0f, -1.0f), one), den = fadd2(e, one);
+    const float2 q = fmul2(num, make_float2(rcp_approx(den.x), rcp_approx(den.y)));
+    return make_float2(copysignf(q.x, a.x), copysignf(q.y, a.y));
+}
+
 __device__ __forceinline__ unsigned absdiff_bits(float a, float b) {
     return __float_as_uint(fabsf(a - b));   // NaN keeps bits above +inf: an integer max propagates it
 }

@@ -483,35 +483,40 @@ __global__ void __launch_bounds__(256, 2) cell_coef_mma_kernel(CellArgs a)
                     uz2 = __ldg(reinterpret_cast<const float2 *>(ue + N + i0));
                     un2 = __ldg(reinterpret_cast<const float2 *>(ue + 2 * N + i0));
                 } else {
-                    ur2 = make_float2(sb[NOUT + i0], sb[NOUT + i0 + 1]);
-                    uz2 = make_float2(sb[NOUT + N + i0], sb[NOUT + N + i0 + 1]);
-                    un2 = make_float2(accn[nn][2 * h] + sb[NOUT + 2 * N + i0], accn[nn][2 * h + 1] + sb[NOUT + 2 * N + i0 + 1]);
+                    ur2 = *reinterpret_cast<const float2 *>(sb + NOUT + i0);
+                    uz2 = *reinterpret_cast<const float2 *>(sb + NOUT + N + i0);
+                    un2 = fadd2(make_float2(accn[nn][2 * h], accn[nn][2 * h + 1]), *reinterpret_cast<const float2 *>(sb + NOUT + 2 * N + i0));
                 }
                 const float2 h2 = __ldg(reinterpret_cast<const float2 *>(hp[h] + i0));
-                float out_rhs[2];
+                // the pair of columns i0, i0 + 1 as packed f32x2 arithmetic (half the instructions of two scalar passes)
+                const float2 one = make_float2(1.0f, 1.0f), mone = make_float2(-1.0f, -1.0f);
+                const float2 sr = make_float2(acc[nn][2 * h], acc[nn][2 * h + 1]);
+                const float2 sz = make_float2(acc[nn + NBG][2 * h], acc[nn + NBG][2 * h + 1]);
+                const float2 sq = make_float2(acc[nn + 2 * NBG][2 * h], acc[nn + 2 * NBG][2 * h + 1]);
+                const float2 bR = *reinterpret_cast<const float2 *>(sb + i0), bZ = *reinterpret_cast<const float2 *>(sb + N + i0);
+                const float2 qn = fadd2(sq, *reinterpret_cast<const float2 *>(sb + 2 * N + i0));   // q = W_hn h + b_hn
+                const float2 r = sigmoid2_gate(fadd2(ur2, fadd2(sr, bR)));
+                const float2 z = sigmoid2_gate(fadd2(uz2, fadd2(sz, bZ)));
+                const float2 c = tanh2_gate(ffma2(r, qn, un2));
+                const float2 omz = ffma2(z, mone, one), omr = ffma2(r, mone, one);
+                const float2 f = ffma2(omz, c, fmul2(z, h2));
+                const float2 az = fmul2(fmul2(ffma2(c, mone, h2), z), omz);
+                const float2 an = fmul2(omz, ffma2(fmul2(c, mone), c, one));
+                const float2 kr = fmul2(fmul2(fmul2(an, qn), r), omr);
+                const float2 kn = fmul2(an, r);
                 float4 cf2[2];
-#pragma unroll
-                for (int el = 0; el < 2; ++el) {
-                    const int i = i0 + el;
-                    const float sr = acc[nn][2 * h + el], sz = acc[nn + NBG][2 * h + el], sq = acc[nn + 2 * NBG][2 * h + el];
-                    const float ur = el ? ur2.y : ur2.x, uz = el ? uz2.y : uz2.x, un = el ? un2.y : un2.x;
-                    const float hi = el ? h2.y : h2.x;
-                    const float qn = sq + sb[2 * N + i];                 // q = W_hn h + b_hn
-                    const float r = sigmoidf_gate(ur + (sr + sb[i]));
-                    const float z = sigmoidf_gate(uz + (sz + sb[N + i]));
-                    const float c = tanhf_gate(un + r * qn);
-                    const float f = (1.0f - z) * c + z * hi;
-                    const float az = (hi - c) * z * (1.0f - z);
-                    const float an = (1.0f - z) * (1.0f - c * c);
-                    const float kr = an * qn * r * (1.0f - r);
-                    const float kn = an * r;
-                    cf2[el] = make_float4(kr, az, kn, z);
-                    float jh = z * hi;
-                    jh = fmaf(az, sz, jh);
-                    jh = fmaf(kn, sq, jh);
-                    jh = fmaf(kr, sr, jh);
-                    out_rhs[el] = f - jh;
-                    if (PROJ || a.residual) out_rhs[el] = f;
+                cf2[0] = make_float4(kr.x, az.x, kn.x, z.x);
+                cf2[1] = make_float4(kr.y, az.y, kn.y, z.y);
+                float out_rhs[2];
+                if (PROJ || a.residual) {
+                    out_rhs[0] = f.x; out_rhs[1] = f.y;
+                } else {
+                    float2 jh = fmul2(z, h2);
+                    jh = ffma2(az, sz, jh);
+                    jh = ffma2(kn, sq, jh);
+                    jh = ffma2(kr, sr, jh);
+                    const float2 o = ffma2(jh, mone, f);
+                    out_rhs[0] = o.x; out_rhs[1] = o.y;
                 }
                 // the rows of columns i0 and i0 + 1 are 32 contiguous bytes: one 256-bit store, so that the four lanes of a
                 // position write one full line per instruction instead of eight half sectors
